@@ -1,0 +1,217 @@
+"""ctypes front end of the CPU oracle (``vtoken_oracle.c``).  TEST INFRASTRUCTURE ONLY.
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this
+module; the product package never does.  It builds ``libvto.so`` with gcc on first use
+(plain C, ``-O2``, OpenMP only for the slab loop of ``apply_moves_pools``).
+"""
+from __future__ import annotations
+
+import ctypes
+import dataclasses
+import os
+import subprocess
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "vtoken_oracle.c")
+_HDR = os.path.join(_HERE, "vtoken_oracle.h")
+_LIB = os.path.join(_HERE, "libvto.so")
+
+NOT_SELECTED, REPACKED, NO_GAIN, DEFERRED_NO_FREE = 0, 1, 2, 3
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into ``oracle/libvto.so`` when missing or older than its sources."""
+    stale = (not os.path.exists(_LIB)
+             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)))
+    if force or stale:
+        tmp = _LIB + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-std=c99", "-O2", "-fPIC", "-shared", "-fopenmp",
+                               "-Wall", "-Wextra", "-o", tmp, _SRC])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Counts(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in
+                ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed",
+                 "num_admitted", "num_deferred")]
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.vto_gather_logical.restype = ctypes.c_int64
+        _lib.vto_waste_ratio.restype = ctypes.c_double
+    return _lib
+
+
+def _p(a: Optional[np.ndarray], dtype):
+    if a is None:
+        return None
+    assert a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _u8(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.uint8)
+
+
+@dataclasses.dataclass
+class Plan:
+    new_bt_offsets: np.ndarray
+    new_bt_blocks: np.ndarray     # trimmed to new_bt_offsets[R]
+    new_tt_slots: np.ndarray
+    freed_blocks: np.ndarray      # trimmed to num_freed
+    req_status: np.ndarray
+    move_src: np.ndarray          # trimmed to num_moves
+    move_dst: np.ndarray
+    num_moves: int
+    num_dst_blocks: int
+    num_freed: int
+    num_free_consumed: int
+    num_admitted: int
+    num_deferred: int
+
+
+def plan(S, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
+         select=None, thr_num=0, thr_den=0, num_free=None) -> Plan:
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
+    keep, select, free_blocks = _u8(keep), _u8(select), _i32(free_blocks)
+    R = len(tt_offsets) - 1
+    T = int(tt_offsets[-1])
+    nbt = int(bt_offsets[-1])
+    if num_free is None:
+        num_free = len(free_blocks)
+    new_bt_offsets = np.zeros(R + 1, np.int32)
+    new_bt_blocks = np.full(max(nbt, 1), -7, np.int32)
+    new_tt_slots = np.full(max(T, 1), -7, np.int32)
+    freed = np.full(max(nbt, 1), -7, np.int32)
+    status = np.full(max(R, 1), -7, np.int32)
+    msrc = np.full(max(T, 1), -7, np.int32)
+    mdst = np.full(max(T, 1), -7, np.int32)
+    c = _Counts()
+    rc = lib().vto_plan(ctypes.c_int32(R), ctypes.c_int32(S),
+                        _p(bt_offsets, np.int32), _p(bt_blocks, np.int32),
+                        _p(tt_offsets, np.int32), _p(tt_slots, np.int32), _p(keep, np.uint8),
+                        _p(select, np.uint8), ctypes.c_uint32(thr_num), ctypes.c_uint32(thr_den),
+                        _p(free_blocks, np.int32), ctypes.c_int32(num_free),
+                        _p(new_bt_offsets, np.int32), _p(new_bt_blocks, np.int32),
+                        _p(new_tt_slots, np.int32), _p(freed, np.int32), _p(status, np.int32),
+                        _p(msrc, np.int32), _p(mdst, np.int32), ctypes.byref(c))
+    if rc != 0:
+        raise ValueError(f"vto_plan failed: {rc}")
+    return Plan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
+                freed[:c.num_freed].copy(), status[:R].copy(),
+                msrc[:c.num_moves].copy(), mdst[:c.num_moves].copy(),
+                c.num_moves, c.num_dst_blocks, c.num_freed, c.num_free_consumed,
+                c.num_admitted, c.num_deferred)
+
+
+def plan_workload(w, num_free=None) -> Plan:
+    return plan(w.block_size, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                w.free_blocks, w.select, w.thr_num, w.thr_den, num_free)
+
+
+def apply_moves_slab(slab: np.ndarray, move_src, move_dst) -> None:
+    """In place on one slab: a C-contiguous 2-D array [num_slots, row] of any dtype."""
+    assert slab.ndim == 2 and slab.flags["C_CONTIGUOUS"]
+    move_src, move_dst = _i32(move_src), _i32(move_dst)
+    rc = lib().vto_apply_moves_slab(ctypes.c_void_p(slab.ctypes.data), ctypes.c_int64(slab.shape[0]),
+                                    ctypes.c_int64(slab.shape[1] * slab.itemsize),
+                                    _p(move_src, np.int32), _p(move_dst, np.int32),
+                                    ctypes.c_int32(len(move_src)))
+    if rc != 0:
+        raise ValueError(f"vto_apply_moves_slab failed: {rc}")
+
+
+def apply_moves_pools(k_pool: np.ndarray, v_pool: np.ndarray, move_src, move_dst, threads: int = 1) -> None:
+    """In place on K and V pools shaped [L, num_slots, row] (C-contiguous)."""
+    assert k_pool.ndim == 3 and k_pool.shape == v_pool.shape
+    assert k_pool.flags["C_CONTIGUOUS"] and v_pool.flags["C_CONTIGUOUS"]
+    move_src, move_dst = _i32(move_src), _i32(move_dst)
+    L, ns, row = k_pool.shape
+    rc = lib().vto_apply_moves_pools(ctypes.c_void_p(k_pool.ctypes.data), ctypes.c_void_p(v_pool.ctypes.data),
+                                     ctypes.c_int32(L), ctypes.c_int64(0), ctypes.c_int64(ns),
+                                     ctypes.c_int64(row * k_pool.itemsize),
+                                     _p(move_src, np.int32), _p(move_dst, np.int32),
+                                     ctypes.c_int32(len(move_src)), ctypes.c_int32(threads))
+    if rc != 0:
+        raise ValueError(f"vto_apply_moves_pools failed: {rc}")
+
+
+def gather_logical(slab: np.ndarray, tt_slots, keep=None) -> np.ndarray:
+    """Rows of one request's active tokens in token-id order from one slab [num_slots, row]."""
+    assert slab.ndim == 2 and slab.flags["C_CONTIGUOUS"]
+    tt_slots, keep = _i32(tt_slots), _u8(keep)
+    out = np.empty((max(len(tt_slots), 1), slab.shape[1]), slab.dtype)
+    n = lib().vto_gather_logical(ctypes.c_void_p(slab.ctypes.data), ctypes.c_int64(slab.shape[0]),
+                                 ctypes.c_int64(slab.shape[1] * slab.itemsize),
+                                 _p(tt_slots, np.int32), _p(keep, np.uint8), ctypes.c_int32(len(tt_slots)),
+                                 ctypes.c_void_p(out.ctypes.data), ctypes.c_int64(out.shape[0]))
+    if n < 0:
+        raise ValueError(f"vto_gather_logical failed: {n}")
+    return out[:n].copy()
+
+
+def validate(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks) -> int:
+    """0 when the input preconditions hold, else the code of the first failed check."""
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
+    keep, free_blocks = _u8(keep), _i32(free_blocks)
+    bad = ctypes.c_int32(0)
+    rc = lib().vto_validate(ctypes.c_int32(len(tt_offsets) - 1), ctypes.c_int32(S), ctypes.c_int32(NB),
+                            _p(bt_offsets, np.int32), _p(bt_blocks, np.int32),
+                            _p(tt_offsets, np.int32), _p(tt_slots, np.int32), _p(keep, np.uint8),
+                            _p(free_blocks, np.int32), ctypes.c_int32(len(free_blocks)), ctypes.byref(bad))
+    if rc == -1:
+        raise ValueError("vto_validate: bad argument")
+    return bad.value
+
+
+def check_semantics(S, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
+                    new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, num_free_consumed,
+                    req_status, select=None, thr_num=0, thr_den=0, num_free=None) -> int:
+    """0 when the result is a valid repack of the inputs under any ordering, else a check code."""
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
+    keep, select, free_blocks = _u8(keep), _u8(select), _i32(free_blocks)
+    new_bt_offsets, new_bt_blocks = _i32(new_bt_offsets), _i32(new_bt_blocks)
+    new_tt_slots, freed_blocks, req_status = _i32(new_tt_slots), _i32(freed_blocks), _i32(req_status)
+    if num_free is None:
+        num_free = len(free_blocks)
+    bad = ctypes.c_int32(0)
+    rc = lib().vto_check_semantics(
+        ctypes.c_int32(len(tt_offsets) - 1), ctypes.c_int32(S),
+        _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
+        _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),
+        ctypes.c_uint32(thr_num), ctypes.c_uint32(thr_den),
+        _p(free_blocks, np.int32), ctypes.c_int32(num_free),
+        _p(new_bt_offsets, np.int32), _p(new_bt_blocks, np.int32), _p(new_tt_slots, np.int32),
+        _p(freed_blocks, np.int32), ctypes.c_int32(len(freed_blocks)),
+        ctypes.c_int32(num_free_consumed), _p(req_status, np.int32), ctypes.byref(bad))
+    if rc == -1:
+        raise ValueError("vto_check_semantics: bad argument")
+    return bad.value
+
+
+def waste_ratio(S, num_allocated_blocks, tt_slots, keep=None) -> float:
+    tt_slots, keep = _i32(tt_slots), _u8(keep)
+    return float(lib().vto_waste_ratio(ctypes.c_int32(S), ctypes.c_int64(num_allocated_blocks),
+                                       _p(tt_slots, np.int32), _p(keep, np.uint8),
+                                       ctypes.c_int64(len(tt_slots))))
+
+
+def openmp_threads() -> int:
+    return int(lib().vto_openmp_threads())

@@ -1,0 +1,314 @@
+/*
+ * CPU oracle for the vToken repack path.  TEST INFRASTRUCTURE ONLY -- see vtoken_oracle.h.
+ *
+ * Everything below is the definition written out: one request, one token, one layer, one
+ * row at a time.  No blocking, no fusion, no reordering beyond what the paper states.
+ */
+#include "vtoken_oracle.h"
+
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static int is_live(const int32_t *tt_slots, const uint8_t *keep, int64_t t)
+{
+    /* an active token: it owns a physical copy and the policy has not evicted it
+     * (token table: location plus liveness bit, Sec. 3.2) */
+    return tt_slots[t] >= 0 && (keep == NULL || keep[t] != 0);
+}
+
+static int32_t ceil_div(int64_t a, int64_t b) { return (int32_t)((a + b - 1) / b); }
+
+int vto_plan(int32_t R, int32_t S,
+             const int32_t *bt_offsets, const int32_t *bt_blocks,
+             const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+             const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+             const int32_t *free_blocks, int32_t num_free,
+             int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
+             int32_t *freed_blocks, int32_t *req_status,
+             int32_t *move_src, int32_t *move_dst, vto_counts *counts)
+{
+    if (R < 0 || S < 1 || num_free < 0 || !bt_offsets || !tt_offsets || !counts) return VTO_EINVAL;
+
+    int32_t consumed = 0;     /* free-list entries handed out so far */
+    int32_t num_freed = 0, num_moves = 0, num_admitted = 0, num_deferred = 0;
+    int32_t new_bt_fill = 0;
+    int stop = 0;             /* once a candidate does not fit, every later one is deferred */
+
+    for (int32_t r = 0; r < R; ++r) {                       /* requests in ascending index */
+        const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
+        const int32_t b0 = bt_offsets[r], b1 = bt_offsets[r + 1];
+        const int32_t nb = b1 - b0;                         /* blocks the request holds now */
+
+        /* live-token footprint T_live of the request (Sec. 3.3.3) */
+        int64_t n = 0;
+        for (int64_t t = t0; t < t1; ++t) n += is_live(tt_slots, keep, t);
+
+        /* destinations needed: ceil(T_live / S) (Sec. 3.3.3) */
+        const int32_t need = ceil_div(n, S);
+
+        /* eligibility: caller's selection and the live-fraction threshold, in integers */
+        int sel = (select == NULL || select[r] != 0);
+        if (sel && thr_den != 0) {
+            const uint64_t lhs = (uint64_t)n * (uint64_t)thr_den;
+            const uint64_t rhs = (uint64_t)thr_num * (uint64_t)nb * (uint64_t)S;
+            sel = lhs < rhs;
+        }
+
+        int32_t status;
+        if (!sel) status = VTO_NOT_SELECTED;
+        else if (!(need < nb)) status = VTO_NO_GAIN;        /* block count must strictly drop (I4) */
+        else if (stop || (int64_t)consumed + need > num_free) {
+            status = VTO_DEFERRED_NO_FREE;                  /* destinations unavailable (Sec. 3.3.2) */
+            stop = 1;
+        } else status = VTO_REPACKED;
+        req_status[r] = status;
+
+        new_bt_offsets[r] = new_bt_fill;
+        if (status == VTO_REPACKED) {
+            const int32_t *dst = free_blocks + consumed;    /* next `need` entries, list order */
+            int64_t i = 0;                                  /* rank among the live tokens */
+            for (int64_t t = t0; t < t1; ++t) {             /* ascending logical id */
+                if (is_live(tt_slots, keep, t)) {
+                    /* fill each destination block completely before the next (Sec. 3.3.3);
+                     * slot = block * S + offset (Sec. 3.4) */
+                    const int32_t slot = dst[i / S] * S + (int32_t)(i % S);
+                    new_tt_slots[t] = slot;
+                    move_src[num_moves] = tt_slots[t];
+                    move_dst[num_moves] = slot;
+                    ++num_moves;
+                    ++i;
+                } else {
+                    new_tt_slots[t] = -1;                   /* evicted: no slot any more */
+                }
+            }
+            for (int32_t j = 0; j < need; ++j) new_bt_blocks[new_bt_fill++] = dst[j];
+            for (int32_t j = b0; j < b1; ++j) freed_blocks[num_freed++] = bt_blocks[j];
+            consumed += need;
+            ++num_admitted;
+        } else {
+            if (status == VTO_DEFERRED_NO_FREE) ++num_deferred;
+            for (int64_t t = t0; t < t1; ++t)
+                new_tt_slots[t] = is_live(tt_slots, keep, t) ? tt_slots[t] : -1;
+            for (int32_t j = b0; j < b1; ++j) new_bt_blocks[new_bt_fill++] = bt_blocks[j];
+        }
+    }
+    new_bt_offsets[R] = new_bt_fill;
+
+    counts->num_moves = num_moves;
+    counts->num_dst_blocks = consumed;
+    counts->num_freed = num_freed;
+    counts->num_free_consumed = consumed;
+    counts->num_admitted = num_admitted;
+    counts->num_deferred = num_deferred;
+    return VTO_OK;
+}
+
+int vto_apply_moves_slab(uint8_t *slab, int64_t num_slots, int64_t row_bytes,
+                         const int32_t *move_src, const int32_t *move_dst, int32_t num_moves)
+{
+    if (!slab || row_bytes < 1 || num_moves < 0) return VTO_EINVAL;
+    for (int32_t m = 0; m < num_moves; ++m) {
+        const int64_t s = move_src[m], d = move_dst[m];
+        if (s < 0 || d < 0 || s >= num_slots || d >= num_slots) return VTO_EINVAL;
+        memcpy(slab + d * row_bytes, slab + s * row_bytes, (size_t)row_bytes);
+    }
+    return VTO_OK;
+}
+
+int vto_apply_moves_pools(uint8_t *k_pool, uint8_t *v_pool, int32_t L, int64_t layer_stride_bytes,
+                          int64_t num_slots, int64_t row_bytes,
+                          const int32_t *move_src, const int32_t *move_dst, int32_t num_moves,
+                          int32_t threads)
+{
+    if (!k_pool || !v_pool || L < 1) return VTO_EINVAL;
+    if (layer_stride_bytes == 0) layer_stride_bytes = num_slots * row_bytes;
+    int rc = VTO_OK;
+    (void)threads;
+    /* the 2L (K|V, layer) slabs are independent of one another */
+#ifdef _OPENMP
+#pragma omp parallel for num_threads(threads > 0 ? threads : 1) schedule(dynamic, 1)
+#endif
+    for (int32_t i = 0; i < 2 * L; ++i) {
+        uint8_t *pool = (i < L) ? k_pool : v_pool;
+        const int32_t layer = (i < L) ? i : i - L;
+        int e = vto_apply_moves_slab(pool + (int64_t)layer * layer_stride_bytes, num_slots, row_bytes,
+                                     move_src, move_dst, num_moves);
+        if (e != VTO_OK) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            rc = e;
+        }
+    }
+    return rc;
+}
+
+int64_t vto_gather_logical(const uint8_t *slab, int64_t num_slots, int64_t row_bytes,
+                           const int32_t *tt_slots, const uint8_t *keep, int32_t len,
+                           uint8_t *out, int64_t out_capacity_rows)
+{
+    if (!slab || !tt_slots || row_bytes < 1 || len < 0) return VTO_EINVAL;
+    int64_t n = 0;
+    for (int32_t t = 0; t < len; ++t) {
+        if (!is_live(tt_slots, keep, t)) continue;
+        if (tt_slots[t] >= num_slots || n >= out_capacity_rows) return VTO_EINVAL;
+        memcpy(out + n * row_bytes, slab + (int64_t)tt_slots[t] * row_bytes, (size_t)row_bytes);
+        ++n;
+    }
+    return n;
+}
+
+int vto_validate(int32_t R, int32_t S, int32_t NB,
+                 const int32_t *bt_offsets, const int32_t *bt_blocks,
+                 const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                 const int32_t *free_blocks, int32_t num_free, int32_t *first_bad)
+{
+    int32_t bad = 0;
+    if (R < 0 || S < 1 || NB < 0) return VTO_EINVAL;
+    /* owner[b]: -1 unused, r >= 0 block of request r, -2 on the free list */
+    int32_t *owner = (int32_t *)malloc(sizeof(int32_t) * (size_t)(NB > 0 ? NB : 1));
+    uint8_t *taken = (uint8_t *)calloc((size_t)NB * (size_t)S + 1, 1);
+    if (!owner || !taken) { free(owner); free(taken); return VTO_EINVAL; }
+    for (int32_t b = 0; b < NB; ++b) owner[b] = -1;
+
+    for (int32_t r = 0; r < R && !bad; ++r) {
+        if (bt_offsets[r + 1] < bt_offsets[r] || tt_offsets[r + 1] < tt_offsets[r]) bad = 1;
+        for (int32_t j = bt_offsets[r]; j < bt_offsets[r + 1] && !bad; ++j) {
+            const int32_t b = bt_blocks[j];
+            if (b < 0 || b >= NB) bad = 2;                 /* block id out of range */
+            else if (owner[b] != -1) bad = 3;              /* block in two tables (or twice) */
+            else owner[b] = r;
+        }
+    }
+    for (int32_t j = 0; j < num_free && !bad; ++j) {
+        const int32_t b = free_blocks[j];
+        if (b < 0 || b >= NB) bad = 4;                     /* free id out of range */
+        else if (owner[b] != -1) bad = 5;                  /* free block allocated or listed twice */
+        else owner[b] = -2;
+    }
+    for (int32_t r = 0; r < R && !bad; ++r) {
+        for (int64_t t = tt_offsets[r]; t < tt_offsets[r + 1] && !bad; ++t) {
+            const int32_t s = tt_slots[t];
+            if (s < 0) { if (keep && keep[t]) { /* kept but no physical copy: not live */ } continue; }
+            if ((int64_t)s >= (int64_t)NB * S) bad = 6;    /* slot out of range */
+            else if (owner[s / S] != r) bad = 7;           /* slot outside the request's blocks */
+            else if (taken[s]) bad = 8;                    /* slot referenced twice (I2) */
+            else taken[s] = 1;
+        }
+    }
+    free(owner); free(taken);
+    if (first_bad) *first_bad = bad;
+    return bad ? VTO_EPRECOND : VTO_OK;
+}
+
+static int cmp_i32(const void *a, const void *b)
+{
+    const int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;
+    return (x > y) - (x < y);
+}
+
+int vto_check_semantics(int32_t R, int32_t S,
+                        const int32_t *bt_offsets, const int32_t *bt_blocks,
+                        const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                        const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+                        const int32_t *free_blocks, int32_t num_free,
+                        const int32_t *new_bt_offsets, const int32_t *new_bt_blocks,
+                        const int32_t *new_tt_slots, const int32_t *freed_blocks,
+                        int32_t num_freed, int32_t num_free_consumed,
+                        const int32_t *req_status, int32_t *first_bad)
+{
+    int32_t bad = 0;
+    if (R < 0 || S < 1) return VTO_EINVAL;
+    const int32_t total_old = bt_offsets[R];
+    int32_t *exp_freed = (int32_t *)malloc(sizeof(int32_t) * (size_t)(total_old + 1));
+    int32_t *got_freed = (int32_t *)malloc(sizeof(int32_t) * (size_t)(num_freed + 1));
+    int32_t *got_dst = (int32_t *)malloc(sizeof(int32_t) * (size_t)(num_free + 1));
+    int32_t *exp_dst = (int32_t *)malloc(sizeof(int32_t) * (size_t)(num_free + 1));
+    if (!exp_freed || !got_freed || !got_dst || !exp_dst) {
+        free(exp_freed); free(got_freed); free(got_dst); free(exp_dst); return VTO_EINVAL;
+    }
+    int32_t n_exp_freed = 0, n_got_dst = 0;
+    int64_t demand = 0;
+    int stop = 0;
+    if (new_bt_offsets[0] != 0) bad = 1;
+    for (int32_t r = 0; r < R && !bad; ++r) {
+        const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
+        const int32_t nb = bt_offsets[r + 1] - bt_offsets[r];
+        int64_t n = 0;
+        for (int64_t t = t0; t < t1; ++t) n += is_live(tt_slots, keep, t);
+        const int32_t need = ceil_div(n, S);
+        int sel = (select == NULL || select[r] != 0);
+        if (sel && thr_den != 0)
+            sel = (uint64_t)n * thr_den < (uint64_t)thr_num * (uint64_t)nb * (uint64_t)S;
+        int32_t want;
+        if (!sel) want = VTO_NOT_SELECTED;
+        else if (need >= nb) want = VTO_NO_GAIN;
+        else if (stop || demand + need > num_free) { want = VTO_DEFERRED_NO_FREE; stop = 1; }
+        else { want = VTO_REPACKED; demand += need; }
+        if (req_status[r] != want) { bad = 2; break; }
+
+        const int32_t nbt0 = new_bt_offsets[r], nbt1 = new_bt_offsets[r + 1];
+        if (want == VTO_REPACKED) {
+            if (nbt1 - nbt0 != need) { bad = 3; break; }
+            int64_t i = 0;
+            for (int64_t t = t0; t < t1; ++t) {
+                if (is_live(tt_slots, keep, t)) {
+                    /* i-th live token sits at offset i % S of the request's (i / S)-th new block */
+                    if (new_tt_slots[t] != new_bt_blocks[nbt0 + i / S] * S + (int32_t)(i % S)) { bad = 4; break; }
+                    ++i;
+                } else if (new_tt_slots[t] != -1) { bad = 5; break; }
+            }
+            if (bad) break;
+            for (int32_t j = nbt0; j < nbt1; ++j) got_dst[n_got_dst++] = new_bt_blocks[j];
+            for (int32_t j = bt_offsets[r]; j < bt_offsets[r + 1]; ++j) exp_freed[n_exp_freed++] = bt_blocks[j];
+        } else {
+            if (nbt1 - nbt0 != nb) { bad = 6; break; }
+            for (int32_t j = 0; j < nb; ++j)
+                if (new_bt_blocks[nbt0 + j] != bt_blocks[bt_offsets[r] + j]) { bad = 7; break; }
+            for (int64_t t = t0; t < t1 && !bad; ++t) {
+                const int32_t want_slot = is_live(tt_slots, keep, t) ? tt_slots[t] : -1;
+                if (new_tt_slots[t] != want_slot) bad = 8;
+            }
+        }
+    }
+    if (!bad) {
+        /* the destination set is the consumed prefix of the free list; the reclaimed set is
+         * the admitted requests' old blocks -- as sets, order not constrained here */
+        if (n_got_dst != num_free_consumed || num_free_consumed != (int32_t)demand) bad = 9;
+        else if (n_exp_freed != num_freed) bad = 10;
+        else {
+            memcpy(exp_dst, free_blocks, sizeof(int32_t) * (size_t)num_free_consumed);
+            memcpy(got_freed, freed_blocks, sizeof(int32_t) * (size_t)num_freed);
+            qsort(exp_dst, (size_t)num_free_consumed, sizeof(int32_t), cmp_i32);
+            qsort(got_dst, (size_t)n_got_dst, sizeof(int32_t), cmp_i32);
+            qsort(exp_freed, (size_t)n_exp_freed, sizeof(int32_t), cmp_i32);
+            qsort(got_freed, (size_t)num_freed, sizeof(int32_t), cmp_i32);
+            if (memcmp(exp_dst, got_dst, sizeof(int32_t) * (size_t)n_got_dst) != 0) bad = 11;
+            else if (memcmp(exp_freed, got_freed, sizeof(int32_t) * (size_t)num_freed) != 0) bad = 12;
+        }
+    }
+    free(exp_freed); free(got_freed); free(got_dst); free(exp_dst);
+    if (first_bad) *first_bad = bad;
+    return bad ? VTO_EPRECOND : VTO_OK;
+}
+
+double vto_waste_ratio(int32_t S, int64_t num_allocated_blocks,
+                       const int32_t *tt_slots, const uint8_t *keep, int64_t T)
+{
+    if (num_allocated_blocks <= 0 || S < 1) return 0.0;
+    int64_t live = 0;                                       /* sum over blocks of n_b */
+    for (int64_t t = 0; t < T; ++t) live += is_live(tt_slots, keep, t);
+    return 1.0 - (double)live / ((double)num_allocated_blocks * (double)S);
+}
+
+int vto_openmp_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

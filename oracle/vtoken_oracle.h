@@ -1,0 +1,117 @@
+/*
+ * CPU oracle for the vToken repack path.  TEST INFRASTRUCTURE ONLY.
+ *
+ * A plain, slow, single-pass restatement of what the repack computes, written from the
+ * paper's description so that it can be checked against the paper by eye.  It shares no
+ * code with the CUDA library and must never be called from the product path: only the
+ * tests, the smoke check and the benchmark's CPU-baseline leg use it.
+ *
+ * What it states (paper passages):
+ *   - live footprint, ceil(T_live / S) destinations, positive-gain gate  (Sec. 3.3.3, invariant I4)
+ *   - destinations taken from the free pool, plan deferred when short    (Sec. 3.3.2, 3.3.3)
+ *   - move list in logical order, each destination filled completely     (Sec. 3.3.3)
+ *   - slot = block_id * S + offset                                        (Sec. 3.4, slot-mapping equation)
+ *   - token-table update clears the source and writes the destination    (Sec. 3.2 apply_moves, invariant I2)
+ *   - sources freed after the packed layout is committed                 (Sec. 3.3.4)
+ *   - logical view = K/V rows of active tokens in token-id order         (invariant I1, Sec. 5 relocation check)
+ *   - intra-block waste ratio F                                           (Sec. 2.3.1)
+ *
+ * Readings fixed where the paper is silent (same readings bind the CUDA library):
+ *   whole-request compaction; requests planned in ascending index; admission is the longest
+ *   prefix of candidates whose cumulative demand fits the free list, every later candidate
+ *   deferred; destinations are consecutive entries from the front of the caller's free list;
+ *   the reclaimed list is admitted requests ascending, each old block table in order; dead
+ *   tokens map to -1 in every request; the canonical orders are conventions ("parity
+ *   unpinned" by the paper itself -- the semantic checker vto_check_semantics accepts any
+ *   valid permutation and guards against a convention hiding a real defect).
+ *
+ * All pointers are HOST memory owned by the caller.  Functions return 0 on success, a
+ * negative VTO_E* code on a malformed argument, and never abort.
+ */
+#ifndef VTOKEN_ORACLE_H
+#define VTOKEN_ORACLE_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { VTO_OK = 0, VTO_EINVAL = -1, VTO_EPRECOND = -2 };
+enum { VTO_NOT_SELECTED = 0, VTO_REPACKED = 1, VTO_NO_GAIN = 2, VTO_DEFERRED_NO_FREE = 3 };
+
+typedef struct {
+    int32_t num_moves, num_dst_blocks, num_freed, num_free_consumed, num_admitted, num_deferred;
+} vto_counts;
+
+/* Relocation planning + table rewrite for R requests.
+ * Inputs: CSR block tables (bt_offsets[R+1], bt_blocks), CSR token tables (tt_offsets[R+1],
+ * tt_slots: slot or -1), keep mask (0 = evicted), optional select[R] (NULL = all), live-fraction
+ * threshold thr_num/thr_den (thr_den == 0: none; candidate iff n*thr_den < thr_num*nb*S),
+ * free list free_blocks[num_free].
+ * Outputs (caller-sized): new_bt_offsets[R+1], new_bt_blocks[<= total old blocks],
+ * new_tt_slots[T], freed_blocks[<= total old blocks], req_status[R],
+ * move_src/move_dst[<= T] (slot pairs, plan order), counts. */
+int vto_plan(int32_t R, int32_t S,
+             const int32_t *bt_offsets, const int32_t *bt_blocks,
+             const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+             const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+             const int32_t *free_blocks, int32_t num_free,
+             int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
+             int32_t *freed_blocks, int32_t *req_status,
+             int32_t *move_src, int32_t *move_dst, vto_counts *counts);
+
+/* Apply a move list to ONE (K|V, layer) slab of num_slots rows of row_bytes bytes, in place:
+ * row[dst] = row[src] for every move, nothing else changes. */
+int vto_apply_moves_slab(uint8_t *slab, int64_t num_slots, int64_t row_bytes,
+                         const int32_t *move_src, const int32_t *move_dst, int32_t num_moves);
+
+/* Apply a move list to whole K and V pools laid out [L][num_slots][row_bytes] with the given
+ * layer stride, every layer, K then V.  threads > 1 spreads the 2L independent slabs over
+ * that many OpenMP threads (when built with OpenMP; otherwise runs on one). */
+int vto_apply_moves_pools(uint8_t *k_pool, uint8_t *v_pool, int32_t L, int64_t layer_stride_bytes,
+                          int64_t num_slots, int64_t row_bytes,
+                          const int32_t *move_src, const int32_t *move_dst, int32_t num_moves,
+                          int32_t threads);
+
+/* Logical view of one request in one slab: rows of tokens t with tt_slots[t] >= 0 and
+ * (keep == NULL or keep[t] != 0), ascending t, concatenated into out.  Returns the row count
+ * (>= 0) or a negative error. */
+int64_t vto_gather_logical(const uint8_t *slab, int64_t num_slots, int64_t row_bytes,
+                           const int32_t *tt_slots, const uint8_t *keep, int32_t len,
+                           uint8_t *out, int64_t out_capacity_rows);
+
+/* Input preconditions: every live slot in [0, NB*S) and inside a block of the request's own
+ * block table; no slot referenced by two tokens (I2); block ids unique across block tables
+ * and in range; free list in range, duplicate-free and disjoint from the block tables.
+ * Returns VTO_OK or VTO_EPRECOND; *first_bad (optional) gets a small code naming the check. */
+int vto_validate(int32_t R, int32_t S, int32_t NB,
+                 const int32_t *bt_offsets, const int32_t *bt_blocks,
+                 const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                 const int32_t *free_blocks, int32_t num_free, int32_t *first_bad);
+
+/* Order-free check of a plan result against the inputs: statuses follow the admission rule,
+ * admitted requests got ceil(n/S) distinct blocks of the consumed free prefix and their live
+ * tokens fill those blocks completely in logical order, the reclaimed set equals the admitted
+ * requests' old blocks, other requests are unchanged, dead tokens are -1.  Returns VTO_OK,
+ * VTO_EPRECOND (*first_bad names the check) or VTO_EINVAL. */
+int vto_check_semantics(int32_t R, int32_t S,
+                        const int32_t *bt_offsets, const int32_t *bt_blocks,
+                        const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                        const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+                        const int32_t *free_blocks, int32_t num_free,
+                        const int32_t *new_bt_offsets, const int32_t *new_bt_blocks,
+                        const int32_t *new_tt_slots, const int32_t *freed_blocks,
+                        int32_t num_freed, int32_t num_free_consumed,
+                        const int32_t *req_status, int32_t *first_bad);
+
+/* Intra-block waste ratio F = 1 - sum(n_b) / (N * S) over the N allocated blocks, with n_b
+ * the live tokens per block (Sec. 2.3.1).  live = slot >= 0 and keep != 0 (keep NULL: slot >= 0). */
+double vto_waste_ratio(int32_t S, int64_t num_allocated_blocks,
+                       const int32_t *tt_slots, const uint8_t *keep, int64_t T);
+
+int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,74 @@
+"""A second, definition-level statement of the repack result in pure Python containers
+(lists, dicts, sets), used only to brute-force the C oracle on tiny inputs.
+
+It is organised differently from the C oracle on purpose: it first collects the facts about
+every request, then decides admission for all of them at once from the running demand, then
+builds the outputs from per-request dictionaries.  Statuses: 0 not selected, 1 repacked,
+2 no gain, 3 deferred.
+"""
+from fractions import Fraction
+from itertools import accumulate
+
+
+def repack_definition(S, block_tables, token_tables, keeps, free, select=None, thr=None):
+    """block_tables[r]: list of block ids; token_tables[r]: list of slot or -1;
+    keeps[r]: list of 0/1; free: list of block ids; thr: Fraction or None.
+    Returns dict(new_bt, new_tt, freed, status, moves, consumed)."""
+    R = len(token_tables)
+    live = [[t for t, (s, k) in enumerate(zip(token_tables[r], keeps[r])) if s >= 0 and k]
+            for r in range(R)]
+    need = [-(-len(live[r]) // S) for r in range(R)]
+
+    def chosen(r):
+        if select is not None and not select[r]:
+            return False
+        if thr is not None:
+            capacity = len(block_tables[r]) * S
+            # live fraction strictly below the threshold; a request with no blocks never is
+            if capacity == 0 or not Fraction(len(live[r]), capacity) < thr:
+                return False
+        return True
+
+    candidates = [r for r in range(R) if chosen(r) and need[r] < len(block_tables[r])]
+    running = list(accumulate(need[r] for r in candidates))
+    fits = [c <= len(free) for c in running]
+    n_admit = fits.index(False) if False in fits else len(candidates)
+    admitted = candidates[:n_admit]
+    deferred = set(candidates[n_admit:])
+
+    status = []
+    for r in range(R):
+        if r in admitted:
+            status.append(1)
+        elif r in deferred:
+            status.append(3)
+        elif chosen(r):
+            status.append(2)
+        else:
+            status.append(0)
+
+    cursor = 0
+    new_bt, new_tt, freed, moves = [], [], [], []
+    for r in range(R):
+        if r in admitted:
+            mine = free[cursor:cursor + need[r]]
+            cursor += need[r]
+            where = {t: mine[i // S] * S + i % S for i, t in enumerate(live[r])}
+            new_bt.append(list(mine))
+            freed.extend(block_tables[r])
+            moves.extend((token_tables[r][t], where[t]) for t in live[r])
+        else:
+            where = {t: token_tables[r][t] for t in live[r]}
+            new_bt.append(list(block_tables[r]))
+        new_tt.append([where.get(t, -1) for t in range(len(token_tables[r]))])
+    return dict(new_bt=new_bt, new_tt=new_tt, freed=freed, status=status, moves=moves,
+                consumed=cursor)
+
+
+def to_csr(lists):
+    offsets = [0]
+    flat = []
+    for x in lists:
+        flat.extend(x)
+        offsets.append(len(flat))
+    return offsets, flat

@@ -1,0 +1,202 @@
+/*
+ * vtoken.h -- C ABI of the B200 (sm_100a) repack library for token-evicted paged KV caches.
+ *
+ * The library implements the reclamation backend's relocation step of vToken: the live
+ * tokens of fragmented requests are compacted into dense destination blocks and the
+ * indirection tables are rewritten so that the logical token view of every request stays
+ * the same while whole blocks become free.
+ *
+ * Vocabulary (paper notation): S = block size, a slot = block_id * S + offset (Sec. 3.4,
+ * slot-mapping equation); block table = logical block -> physical block (Sec. 2.1);
+ * token table = logical token id -> slot, plus a liveness bit (Sec. 3.2) -- here an int32
+ * slot with -1 for "no physical copy" and a separate uint8 keep mask written by the
+ * eviction policy (evict_token marks, Sec. 3.2).
+ *
+ * Memory: every pointer below says DEVICE or HOST.  The caller owns all of them; the
+ * library owns only scratch it allocates in vtoken_create.  K and V pools are laid out
+ * [num_layers][num_blocks][block_size][num_kv_heads][head_dim] with elem_bytes-wide
+ * elements that are treated as opaque bytes (any bit pattern survives).
+ *
+ * Streams and graphs: vtoken_plan, vtoken_repack and vtoken_gather_logical only enqueue
+ * kernels on the given stream.  They allocate nothing, never synchronise and never read
+ * device data on the host; every grid is fixed by the capacities given at create time and
+ * every data-dependent count stays in device memory.  They can therefore be captured in a
+ * CUDA graph and replayed after the caller rewrites the CONTENTS of the input buffers.
+ *
+ * Ordering contract (Sec. 3.3.4, invariant I3): call vtoken_plan then vtoken_repack on the
+ * same stream (or ordered by events).  Inputs must stay unmodified until the repack has
+ * completed.  The outputs are the PROPOSED new state: record an event behind vtoken_repack;
+ * make every consumer of the new tables wait on it; only after it may the caller adopt the
+ * new tables, return freed_blocks[0 .. num_freed) to its allocator and drop
+ * free_blocks[0 .. num_free_consumed).  One plan may be in flight per context (I4).
+ *
+ * Errors: every function returns 0 (VTOKEN_OK) or a negative code, never aborts or throws.
+ * Argument and capacity problems visible on the host return an error and enqueue nothing.
+ * Data-dependent problems found on the device (slot or block id out of range, request or
+ * token count above the capacities, output overflow) set a bit in counts.error_flags; the
+ * offending row or request is skipped and the kernels complete.  A short free list is not an
+ * error: the request gets status VTOKEN_DEFERRED_NO_FREE (Sec. 3.3.2).
+ *
+ * Preconditions assumed (not checked) on the fast path: each live slot is referenced by one
+ * token only (I2) and lies in a block of its own request; block ids are unique across block
+ * tables (shared-prefix blocks are excluded from plans, I4); the free list has no duplicates
+ * and is disjoint from all block tables.
+ */
+#ifndef VTOKEN_H
+#define VTOKEN_H
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct vtoken_ctx vtoken_ctx;
+
+/* return codes */
+enum {
+    VTOKEN_OK = 0,
+    VTOKEN_EINVAL = -1,      /* malformed argument (NULL, shape, alignment) */
+    VTOKEN_ECAPACITY = -2,   /* a size exceeds a capacity given at create time */
+    VTOKEN_ECUDA = -3,       /* a CUDA call failed; see vtoken_last_cuda_error */
+    VTOKEN_ENOMEM = -4,      /* scratch allocation failed in vtoken_create */
+    VTOKEN_ESTATE = -5       /* vtoken_repack without a plan */
+};
+
+/* per-request status written by vtoken_plan */
+enum {
+    VTOKEN_NOT_SELECTED = 0,     /* not chosen by select[] / at or above the live-fraction threshold */
+    VTOKEN_REPACKED = 1,         /* admitted: its live tokens move, all its old blocks are reclaimed */
+    VTOKEN_NO_GAIN = 2,          /* ceil(n/S) is not below its block count (I4: must strictly decrease) */
+    VTOKEN_DEFERRED_NO_FREE = 3  /* candidate, but the free list cannot supply its destinations */
+};
+
+/* bits of vtoken_counts.error_flags */
+enum {
+    VTOKEN_FLAG_BAD_SLOT = 1u,        /* a token-table slot >= num_blocks * block_size: token treated as not live */
+    VTOKEN_FLAG_BAD_BLOCK = 2u,       /* a block-table id outside [0, num_blocks) */
+    VTOKEN_FLAG_BAD_FREE = 4u,        /* a free-list id outside [0, num_blocks): that destination block is skipped */
+    VTOKEN_FLAG_CAPACITY = 8u,        /* R, T or the block total above the create-time capacities: clamped */
+    VTOKEN_FLAG_TIMEOUT = 16u,        /* a bounded wait inside a kernel ran out; rows may be missing */
+    VTOKEN_FLAG_GATHER_OVERFLOW = 32u /* vtoken_gather_logical: more live tokens than out_capacity_tokens */
+};
+
+typedef struct {
+    int32_t num_layers, num_blocks, block_size, num_kv_heads, head_dim;
+    int32_t elem_bytes;            /* bytes per element (2 for bf16/fp16); rows are opaque bytes */
+    void *k_pool, *v_pool;         /* DEVICE, 16-byte aligned, must outlive the context */
+    int64_t layer_stride_bytes;    /* bytes between layers of a pool; 0 => num_blocks*block_size*row_bytes */
+    int32_t max_requests;          /* capacities: they fix every grid and scratch size */
+    int64_t max_tokens;            /* upper bound of the token-table length (sum of request lengths) */
+    int64_t max_table_blocks;      /* upper bound of the block-table length (sum over requests) */
+    int32_t max_free_blocks;       /* upper bound of num_free */
+    int32_t max_ctas;              /* copy-kernel grid cap (co-residency with other work); 0 => auto */
+    int32_t copy_variant;          /* 0 auto; 1 register path; 2 bulk-copy (TMA) path */
+} vtoken_config;
+
+/* row_bytes = num_kv_heads * head_dim * elem_bytes must be a multiple of 16, pools and
+ * layer stride 16-byte aligned (VTOKEN_EINVAL otherwise).  Allocates all scratch once. */
+int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx);
+void vtoken_destroy(vtoken_ctx *ctx);
+
+typedef struct {                   /* all DEVICE pointers, read-only to the library */
+    const int32_t *num_requests;   /* device scalar R <= max_requests */
+    const int32_t *bt_offsets;     /* [R+1] CSR offsets into bt_blocks */
+    const int32_t *bt_blocks;      /* [bt_offsets[R]] physical block ids, logical block order */
+    const int32_t *tt_offsets;     /* [R+1] CSR offsets into tt_slots / keep */
+    const int32_t *tt_slots;       /* [tt_offsets[R]] slot = block*S+offset, or -1 */
+    const uint8_t *keep;           /* [tt_offsets[R]] 0 = evicted, non-zero = keep */
+    const uint8_t *select;         /* [R] or NULL (= every request) */
+    uint32_t thr_num, thr_den;     /* candidate iff n_r*thr_den < thr_num*nb_r*S (64-bit); thr_den==0 => no threshold */
+    const int32_t *free_blocks;    /* caller's free list, consumed from index 0 in list order */
+    const int32_t *num_free;       /* device scalar <= max_free_blocks */
+} vtoken_plan_in;
+
+typedef struct {
+    int32_t num_moves;             /* live tokens of admitted requests (rows moved per layer per pool) */
+    int32_t num_dst_blocks;        /* destination blocks written */
+    int32_t num_freed;             /* entries of freed_blocks */
+    int32_t num_free_consumed;     /* entries taken from the front of free_blocks (== num_dst_blocks) */
+    int32_t num_admitted;          /* requests with status VTOKEN_REPACKED */
+    int32_t num_deferred;          /* requests with status VTOKEN_DEFERRED_NO_FREE */
+    uint32_t error_flags;          /* VTOKEN_FLAG_* */
+    uint32_t reserved;
+} vtoken_counts;
+
+typedef struct {                   /* all DEVICE pointers, written by vtoken_plan */
+    int32_t *new_bt_offsets;       /* [R+1] */
+    int32_t *new_bt_blocks;        /* capacity max_table_blocks */
+    int32_t *new_tt_slots;         /* [T], same CSR offsets as the input token table */
+    int32_t *freed_blocks;         /* capacity max_table_blocks */
+    int32_t *req_status;           /* [R] VTOKEN_NOT_SELECTED .. VTOKEN_DEFERRED_NO_FREE */
+    vtoken_counts *counts;         /* one struct */
+} vtoken_plan_out;
+
+/* Relocation planning and table rewrite (Sec. 3.3.3; apply_moves of Sec. 3.2; I1, I2, I4).
+ * For every request in ascending index: n = live tokens (slot >= 0 and keep != 0),
+ * need = ceil(n / S).  A selected request below the threshold with need < its block count is
+ * a candidate; candidates are admitted in order while the cumulative need fits num_free, all
+ * later candidates are deferred.  An admitted request receives the next `need` entries of
+ * free_blocks; its i-th live token (logical order) gets slot dst[i / S] * S + i % S; its new
+ * block table is dst[0 .. need); its old blocks are appended to freed_blocks in table order.
+ * Every other request keeps its block table and the slots of its live tokens.  Entries of
+ * evicted tokens become -1 in every request.  The move plan is kept inside the context for
+ * vtoken_repack.  The structs are read on the host during the call (HOST pointers to
+ * structs holding DEVICE pointers). */
+int vtoken_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, void *cuda_stream);
+
+/* Stage-aware asynchronous copy (Sec. 3.3.4): executes the plan held in the context.  For
+ * every move, every layer, K and V: row[dst_slot] = row[src_slot], row_bytes each, in place
+ * in the pools.  Destinations are free blocks, sources are allocated blocks, so the two sets
+ * are disjoint and no other byte of the pools changes.  One launch covers all layers and both
+ * pools; the amount of work is read from device memory. */
+int vtoken_repack(vtoken_ctx *ctx, void *cuda_stream);
+
+/* Logical view (invariant I1; the before/after relocation check of Sec. 5): K and V rows of
+ * the active tokens (slot >= 0, and keep != 0 when keep is given) of the selected requests in
+ * request order then token-id order, for layers [layer_begin, layer_end), written densely:
+ *   out_k / out_v : DEVICE, [layer_end-layer_begin][out_capacity_tokens][row_bytes] bytes
+ *                   (the layer stride is out_capacity_tokens rows whatever the live count)
+ *   out_offsets   : DEVICE int32 [R+1], first output row of each request (unselected: empty)
+ * Tokens beyond out_capacity_tokens are dropped and VTOKEN_FLAG_GATHER_OVERFLOW is set in the
+ * context's flags (see vtoken_read_counts).  Uses the context's scratch: do not overlap with
+ * a plan/repack in flight on another stream. */
+int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                          const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                          int32_t layer_begin, int32_t layer_end, void *out_k, void *out_v,
+                          int64_t out_capacity_tokens, int32_t *out_offsets, void *cuda_stream);
+
+/* Copies the context's counts of the last plan (with the flags raised by repack and
+ * gather_logical since) to HOST memory.  Synchronises the stream: the only call that does. */
+int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stream);
+
+/* Host-table front end.  The paper keeps the canonical token table on the CPU (Sec. 3.2);
+ * this entry point serves such a caller: all tables are HOST memory (pinned for speed), the
+ * pools stay on the device.  Copies the inputs to device staging owned by the context, runs
+ * vtoken_plan and vtoken_repack, copies every output back and synchronises the stream. */
+typedef struct {                   /* all HOST pointers */
+    int32_t num_requests;
+    const int32_t *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
+    const uint8_t *keep, *select;  /* select may be NULL */
+    uint32_t thr_num, thr_den;
+    const int32_t *free_blocks;
+    int32_t num_free;
+    int32_t *new_bt_offsets;       /* [R+1] */
+    int32_t *new_bt_blocks;        /* [bt_offsets[R]] */
+    int32_t *new_tt_slots;         /* [tt_offsets[R]] */
+    int32_t *freed_blocks;         /* [bt_offsets[R]] */
+    int32_t *req_status;           /* [R] */
+    vtoken_counts *counts;
+} vtoken_host_tables;
+int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *tables, void *cuda_stream);
+
+/* Diagnostics. */
+const char *vtoken_strerror(int code);
+int vtoken_last_cuda_error(const vtoken_ctx *ctx);       /* cudaError_t of the last VTOKEN_ECUDA */
+int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int32_t *smem_bytes,
+                     int32_t *variant);                   /* launch shape of the copy kernel */
+int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx);      /* device scratch held by the context */
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,25 @@
+"""B200-native repack path of vToken: compaction of the live tokens of a token-evicted paged
+KV cache into dense blocks with rewritten block and token tables.
+
+The work is done by hand-written CUDA kernels (sm_100a) behind the C ABI declared in
+``include/vtoken.h``; this package is the thin Python binding of that ABI (same function
+names, argument marshalling only) plus seeded workload generators and harness kernels used
+by tests and the benchmark.  There is no CPU fallback: using the binding without the built
+library raises ImportError.
+"""
+from .binding import (  # noqa: F401
+    VtokenError,
+    vtoken_copy_grid,
+    vtoken_create,
+    vtoken_destroy,
+    vtoken_gather_logical,
+    vtoken_plan,
+    vtoken_read_counts,
+    vtoken_repack,
+    vtoken_repack_host,
+    vtoken_scratch_bytes,
+)
+
+__all__ = ["VtokenError", "vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack",
+           "vtoken_gather_logical", "vtoken_read_counts", "vtoken_repack_host", "vtoken_copy_grid",
+           "vtoken_scratch_bytes"]

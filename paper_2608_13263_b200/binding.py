@@ -1,0 +1,202 @@
+"""ctypes binding of ``libvtoken.so``: same names as the C ABI in ``include/vtoken.h``,
+argument marshalling only.  Device pointers may be given as ints or as anything with a
+``data_ptr()`` method (torch tensors); streams as ints or objects with ``cuda_stream``.
+
+There is no CPU fallback: importing the library fails loudly when it has not been built.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libvtoken.so")
+
+OK, EINVAL, ECAPACITY, ECUDA, ENOMEM, ESTATE = 0, -1, -2, -3, -4, -5
+NOT_SELECTED, REPACKED, NO_GAIN, DEFERRED_NO_FREE = 0, 1, 2, 3
+FLAG_BAD_SLOT, FLAG_BAD_BLOCK, FLAG_BAD_FREE, FLAG_CAPACITY, FLAG_TIMEOUT, FLAG_GATHER_OVERFLOW = 1, 2, 4, 8, 16, 32
+
+SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "vtoken_gather_logical",
+           "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
+           "vtoken_copy_grid", "vtoken_scratch_bytes"]
+
+
+class VtokenError(RuntimeError):
+    def __init__(self, code: int, where: str, cuda_error: int = 0):
+        self.code = code
+        self.cuda_error = cuda_error
+        msg = f"{where}: {strerror(code)} (code {code})"
+        if cuda_error:
+            msg += f", cudaError {cuda_error}"
+        super().__init__(msg)
+
+
+class Config(ctypes.Structure):
+    _fields_ = [("num_layers", ctypes.c_int32), ("num_blocks", ctypes.c_int32), ("block_size", ctypes.c_int32),
+                ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("elem_bytes", ctypes.c_int32),
+                ("k_pool", ctypes.c_void_p), ("v_pool", ctypes.c_void_p),
+                ("layer_stride_bytes", ctypes.c_int64), ("max_requests", ctypes.c_int32),
+                ("max_tokens", ctypes.c_int64), ("max_table_blocks", ctypes.c_int64),
+                ("max_free_blocks", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
+                ("copy_variant", ctypes.c_int32)]
+
+
+class PlanIn(ctypes.Structure):
+    _fields_ = [("num_requests", ctypes.c_void_p), ("bt_offsets", ctypes.c_void_p), ("bt_blocks", ctypes.c_void_p),
+                ("tt_offsets", ctypes.c_void_p), ("tt_slots", ctypes.c_void_p), ("keep", ctypes.c_void_p),
+                ("select", ctypes.c_void_p), ("thr_num", ctypes.c_uint32), ("thr_den", ctypes.c_uint32),
+                ("free_blocks", ctypes.c_void_p), ("num_free", ctypes.c_void_p)]
+
+
+class Counts(ctypes.Structure):
+    _fields_ = [("num_moves", ctypes.c_int32), ("num_dst_blocks", ctypes.c_int32), ("num_freed", ctypes.c_int32),
+                ("num_free_consumed", ctypes.c_int32), ("num_admitted", ctypes.c_int32),
+                ("num_deferred", ctypes.c_int32), ("error_flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+    def as_dict(self):
+        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+
+
+class PlanOut(ctypes.Structure):
+    _fields_ = [("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
+                ("new_tt_slots", ctypes.c_void_p), ("freed_blocks", ctypes.c_void_p),
+                ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p)]
+
+
+class HostTables(ctypes.Structure):
+    _fields_ = [("num_requests", ctypes.c_int32),
+                ("bt_offsets", ctypes.c_void_p), ("bt_blocks", ctypes.c_void_p),
+                ("tt_offsets", ctypes.c_void_p), ("tt_slots", ctypes.c_void_p),
+                ("keep", ctypes.c_void_p), ("select", ctypes.c_void_p),
+                ("thr_num", ctypes.c_uint32), ("thr_den", ctypes.c_uint32),
+                ("free_blocks", ctypes.c_void_p), ("num_free", ctypes.c_int32),
+                ("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
+                ("new_tt_slots", ctypes.c_void_p), ("freed_blocks", ctypes.c_void_p),
+                ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p)]
+
+
+_lib = None
+
+
+def load():
+    """Loads libvtoken.so (once).  Raises when it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_13263_b200.build` "
+                              "(needs nvcc); this package has no CPU fallback")
+        lib = ctypes.CDLL(LIB_PATH)
+        lib.vtoken_create.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(ctypes.c_void_p)]
+        lib.vtoken_destroy.argtypes = [ctypes.c_void_p]
+        lib.vtoken_destroy.restype = None
+        lib.vtoken_plan.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PlanOut), ctypes.c_void_p]
+        lib.vtoken_repack.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        lib.vtoken_gather_logical.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p,
+                                                                       ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+                                                                       ctypes.c_void_p]
+        lib.vtoken_read_counts.argtypes = [ctypes.c_void_p, ctypes.POINTER(Counts), ctypes.c_void_p]
+        lib.vtoken_repack_host.argtypes = [ctypes.c_void_p, ctypes.POINTER(HostTables), ctypes.c_void_p]
+        lib.vtoken_strerror.argtypes = [ctypes.c_int]
+        lib.vtoken_strerror.restype = ctypes.c_char_p
+        lib.vtoken_last_cuda_error.argtypes = [ctypes.c_void_p]
+        lib.vtoken_copy_grid.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 4
+        lib.vtoken_scratch_bytes.argtypes = [ctypes.c_void_p]
+        lib.vtoken_scratch_bytes.restype = ctypes.c_int64
+        _lib = lib
+    return _lib
+
+
+def _ptr(x):
+    if x is None:
+        return None
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return x.data_ptr()
+    if hasattr(x, "ctypes"):          # numpy array (host pointers of vtoken_repack_host)
+        return x.ctypes.data
+    raise TypeError(f"cannot take a pointer from {type(x)}")
+
+
+def _stream(s):
+    if s is None:
+        return None
+    if isinstance(s, int):
+        return s
+    return s.cuda_stream
+
+
+def strerror(code: int) -> str:
+    return load().vtoken_strerror(code).decode()
+
+
+def _check(rc, where, ctx=None):
+    if rc != OK:
+        cuda = load().vtoken_last_cuda_error(ctx) if (ctx and rc in (ECUDA, ENOMEM)) else 0
+        raise VtokenError(rc, where, cuda)
+
+
+def vtoken_create(num_layers, num_blocks, block_size, num_kv_heads, head_dim, k_pool, v_pool, max_requests,
+                  max_tokens, max_table_blocks, max_free_blocks, elem_bytes=2, layer_stride_bytes=0, max_ctas=0,
+                  copy_variant=0) -> int:
+    cfg = Config(num_layers, num_blocks, block_size, num_kv_heads, head_dim, elem_bytes, _ptr(k_pool), _ptr(v_pool),
+                 layer_stride_bytes, max_requests, max_tokens, max_table_blocks, max_free_blocks, max_ctas,
+                 copy_variant)
+    ctx = ctypes.c_void_p()
+    _check(load().vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)), "vtoken_create")
+    return ctx.value
+
+
+def vtoken_destroy(ctx) -> None:
+    load().vtoken_destroy(ctx)
+
+
+def vtoken_plan(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
+                new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status, counts,
+                select=None, thr_num=0, thr_den=0, stream=None) -> None:
+    pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                 _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
+    pout = PlanOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks),
+                   _ptr(req_status), _ptr(counts))
+    _check(load().vtoken_plan(ctx, ctypes.byref(pin), ctypes.byref(pout), _stream(stream)), "vtoken_plan", ctx)
+
+
+def vtoken_repack(ctx, stream=None) -> None:
+    _check(load().vtoken_repack(ctx, _stream(stream)), "vtoken_repack", ctx)
+
+
+def vtoken_gather_logical(ctx, *, num_requests, tt_offsets, tt_slots, keep, select, layer_begin, layer_end,
+                          out_k, out_v, out_capacity_tokens, out_offsets, stream=None) -> None:
+    _check(load().vtoken_gather_logical(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                                        _ptr(select), layer_begin, layer_end, _ptr(out_k), _ptr(out_v),
+                                        out_capacity_tokens, _ptr(out_offsets), _stream(stream)),
+           "vtoken_gather_logical", ctx)
+
+
+def vtoken_read_counts(ctx, stream=None) -> dict:
+    c = Counts()
+    _check(load().vtoken_read_counts(ctx, ctypes.byref(c), _stream(stream)), "vtoken_read_counts", ctx)
+    return c.as_dict()
+
+
+def vtoken_repack_host(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
+                       num_free, new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status,
+                       select=None, thr_num=0, thr_den=0, stream=None) -> dict:
+    """All table arguments are HOST arrays (numpy or pinned torch tensors)."""
+    c = Counts()
+    h = HostTables(num_requests, _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                   _ptr(select), thr_num, thr_den, _ptr(free_blocks), num_free, _ptr(new_bt_offsets),
+                   _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks), _ptr(req_status),
+                   ctypes.addressof(c))
+    _check(load().vtoken_repack_host(ctx, ctypes.byref(h), _stream(stream)), "vtoken_repack_host", ctx)
+    return c.as_dict()
+
+
+def vtoken_copy_grid(ctx) -> dict:
+    v = [ctypes.c_int32() for _ in range(4)]
+    _check(load().vtoken_copy_grid(ctx, *[ctypes.byref(x) for x in v]), "vtoken_copy_grid")
+    return dict(ctas=v[0].value, threads=v[1].value, smem_bytes=v[2].value, variant=v[3].value)
+
+
+def vtoken_scratch_bytes(ctx) -> int:
+    return load().vtoken_scratch_bytes(ctx)

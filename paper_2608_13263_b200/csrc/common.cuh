@@ -1,0 +1,114 @@
+// Internal definitions shared by the translation units of libvtoken (never installed).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "vtoken.h"
+
+// ---------------------------------------------------------------------------------------
+// Context: configuration, derived sizes and every scratch buffer (allocated once).
+// ---------------------------------------------------------------------------------------
+struct vtoken_ctx {
+    vtoken_config cfg;
+    int64_t row_bytes;         // H * D * elem_bytes
+    int64_t layer_stride;      // bytes between layers
+    int64_t slots_per_layer;   // NB * S
+    int32_t cap_dst_blocks;    // destination blocks a plan can ever use
+    int device, num_sms;
+    int last_cuda_error;
+    bool has_plan;
+
+    // planner scratch (DEVICE)
+    int32_t *req_n;            // [max_requests] live tokens
+    int32_t *req_dst_base;     // [max_requests] first destination block (index into the free list)
+    int32_t *req_freed_base;   // [max_requests] first entry in freed_blocks
+    int32_t *req_status;       // [max_requests]
+    int32_t *dst_src;          // [cap_dst_blocks * S] inverse plan: source slot of each destination slot, -1 = none
+    int32_t *dst_blocks;       // [cap_dst_blocks] physical id of each destination block, -1 = skip
+    vtoken_counts *counts;     // one struct
+
+    // gather_logical scratch (DEVICE)
+    int32_t *g_src;            // [max_tokens] source slot of each output row
+    int32_t *g_total;          // [1] output rows
+
+    // device staging of vtoken_repack_host (DEVICE), allocated on first use
+    struct {
+        bool ready;
+        int32_t *num_requests, *num_free;
+        int32_t *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots, *free_blocks;
+        uint8_t *keep, *select;
+        int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *req_status;
+        vtoken_counts *counts;
+    } stage;
+    int64_t scratch_bytes;
+
+    // launch shape of the copy kernel
+    int copy_variant;          // 1 register path, 2 bulk-copy path
+    int copy_ctas, copy_threads, copy_smem;
+    int bulk_warps, bulk_stages, bulk_rows;   // bulk path: warps per CTA, ring depth, rows per item
+};
+
+// host launchers, one per translation unit
+int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
+int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st);
+int vtk_configure_copy(vtoken_ctx *ctx);
+int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                      const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                      int32_t layer_begin, int32_t layer_end, void *out_k, void *out_v,
+                      int64_t out_capacity_tokens, int32_t *out_offsets, cudaStream_t st);
+
+#define VTK_CUDA(ctx, call)                                  \
+    do {                                                     \
+        cudaError_t e__ = (call);                            \
+        if (e__ != cudaSuccess) {                            \
+            (ctx)->last_cuda_error = (int)e__;               \
+            return VTOKEN_ECUDA;                             \
+        }                                                    \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------
+// device helpers
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ int vtk_lane() { return threadIdx.x & 31; }
+
+__device__ __forceinline__ int vtk_warp_incl_scan(int v)
+{
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        int o = __shfl_up_sync(0xffffffffu, v, d);
+        if (vtk_lane() >= d) v += o;
+    }
+    return v;
+}
+
+// Exclusive rank of `flag` among the flags of a CTA of NT threads (NT multiple of 32, <= 1024)
+// in thread order, plus the CTA total.  warp_sums: shared int[NT/32 + 1].  Two barriers.
+template <int NT>
+__device__ __forceinline__ int vtk_block_rank(bool flag, int *warp_sums, int &total)
+{
+    const unsigned ballot = __ballot_sync(0xffffffffu, flag);
+    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
+    const int in_warp = __popc(ballot & ((1u << lane) - 1u));
+    if (lane == 0) warp_sums[warp] = __popc(ballot);
+    __syncthreads();
+    if (warp == 0) {
+        int v = (lane < NT / 32) ? warp_sums[lane] : 0;
+        int incl = vtk_warp_incl_scan(v);
+        if (lane < NT / 32) warp_sums[lane] = incl - v;
+        if (lane == 31) warp_sums[NT / 32] = incl;
+    }
+    __syncthreads();
+    const int rank = warp_sums[warp] + in_warp;
+    total = warp_sums[NT / 32];
+    __syncthreads();   // warp_sums is reused by the next call
+    return rank;
+}
+
+// A token is live when it owns a slot inside the pool and the policy kept it.
+__device__ __forceinline__ bool vtk_live(int32_t slot, const uint8_t *keep, int64_t t, int64_t slots_per_layer,
+                                         bool &bad_slot)
+{
+    if (slot < 0) return false;
+    if ((int64_t)slot >= slots_per_layer) { bad_slot = true; return false; }
+    return keep == nullptr || keep[t] != 0;
+}

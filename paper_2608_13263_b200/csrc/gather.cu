@@ -1,0 +1,197 @@
+// Logical view of the cache (invariant I1; the before/after relocation check of Sec. 5):
+// K and V rows of the active tokens of the selected requests, request order then token-id
+// order, written densely.  Same structure as the planner: count -> scan -> assign, then a
+// row-copy kernel that reads through the token table (the slot-translation read pattern of
+// Sec. 3.4).
+#include "common.cuh"
+
+namespace {
+
+constexpr int G_NT = 512;
+
+struct GatherArgs {
+    const int32_t *num_requests, *tt_offsets, *tt_slots;
+    const uint8_t *keep, *select;
+    int32_t *req_n, *out_offsets, *g_src, *g_total;
+    vtoken_counts *counts;
+    const uint8_t *k_pool, *v_pool;
+    uint8_t *out_k, *out_v;
+    int64_t layer_stride, row_bytes, slots_per_layer, out_capacity, max_tokens;
+    int32_t layer_begin, layer_end, max_requests;
+};
+
+__device__ __forceinline__ int g_requests(const GatherArgs &a)
+{
+    int R = *a.num_requests;
+    return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
+}
+
+__global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
+{
+    const int r = blockIdx.x;
+    if (r >= g_requests(a)) return;
+    int n = 0;
+    bool bad = false;
+    if (a.select == nullptr || a.select[r] != 0) {
+        const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
+        for (int64_t t = t0 + threadIdx.x; t < t1; t += G_NT)
+            n += vtk_live(a.tt_slots[t], a.keep, t, a.slots_per_layer, bad) ? 1 : 0;
+    }
+    __shared__ int warp_n[G_NT / 32];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+    if (vtk_lane() == 0) warp_n[threadIdx.x >> 5] = n;
+    if (bad) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int s = 0;
+        for (int w = 0; w < G_NT / 32; ++w) s += warp_n[w];
+        a.req_n[r] = s;
+    }
+}
+
+// exclusive scan of the per-request counts -> out_offsets[R+1]; one CTA
+__global__ void __launch_bounds__(1024) gather_scan_kernel(GatherArgs a)
+{
+    __shared__ int warp_tot[33];
+    __shared__ int carry;
+    const int R = g_requests(a);
+    const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < R; base += 1024) {
+        const int r = base + tid;
+        const int v = r < R ? a.req_n[r] : 0;
+        int incl = vtk_warp_incl_scan(v);
+        if (lane == 31) warp_tot[warp] = incl;
+        __syncthreads();
+        if (warp == 0) {
+            const int w = warp_tot[lane];
+            const int wi = vtk_warp_incl_scan(w);
+            warp_tot[lane] = wi - w;
+            if (lane == 31) warp_tot[32] = wi;
+        }
+        __syncthreads();
+        const int excl = carry + warp_tot[warp] + incl - v;
+        if (r < R) a.out_offsets[r] = excl;
+        __syncthreads();
+        if (tid == 0) carry += warp_tot[32];
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.out_offsets[R] = carry;
+        int64_t cap = a.out_capacity < a.max_tokens ? a.out_capacity : a.max_tokens;
+        if ((int64_t)carry > cap) {
+            atomicOr(&a.counts->error_flags, VTOKEN_FLAG_GATHER_OVERFLOW);
+            *a.g_total = (int32_t)cap;
+        } else {
+            *a.g_total = carry;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
+{
+    __shared__ int warp_sums[G_NT / 32 + 1];
+    const int r = blockIdx.x;
+    if (r >= g_requests(a)) return;
+    if (a.select != nullptr && a.select[r] == 0) return;
+    const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
+    const int64_t cap = *a.g_total;
+    int carry = a.out_offsets[r];
+    for (int64_t tb = t0; tb < t1; tb += G_NT) {
+        const int64_t t = tb + threadIdx.x;
+        int32_t slot = -1;
+        bool live = false, bad = false;
+        if (t < t1) {
+            slot = a.tt_slots[t];
+            live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
+        }
+        int total;
+        const int i = carry + vtk_block_rank<G_NT>(live, warp_sums, total);
+        carry += total;
+        if (live && i < cap) a.g_src[i] = slot;
+    }
+}
+
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+constexpr int GC_NT = 256;
+
+// one warp per (pool, layer, output row)
+__global__ void __launch_bounds__(GC_NT) gather_copy_kernel(GatherArgs a)
+{
+    const int64_t n = *a.g_total;
+    const int nl = a.layer_end - a.layer_begin;
+    const int64_t total = n * nl * 2;
+    const int lane = vtk_lane();
+    const int64_t nwarps = (int64_t)gridDim.x * (GC_NT / 32);
+    const int row_vecs = (int)(a.row_bytes >> 4);
+    for (int64_t u = (int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5); u < total; u += nwarps) {
+        const int slab = (int)(u / n);                 // [0, nl): K layers, [nl, 2nl): V layers
+        const int64_t idx = u - (int64_t)slab * n;
+        const int li = slab < nl ? slab : slab - nl;
+        const uint8_t *pool = slab < nl ? a.k_pool : a.v_pool;
+        uint8_t *out = slab < nl ? a.out_k : a.out_v;
+        const int32_t src = a.g_src[idx];
+        const uint4 *sp = reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
+                                                          (int64_t)src * a.row_bytes);
+        uint4 *dp = reinterpret_cast<uint4 *>(out + ((int64_t)li * a.out_capacity + idx) * a.row_bytes);
+        for (int c = lane; c < row_vecs; c += 128) {
+            uint4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (c + 32 * k < row_vecs) v[k] = ld_stream(sp + c + 32 * k);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (c + 32 * k < row_vecs) st_stream(dp + c + 32 * k, v[k]);
+        }
+    }
+}
+
+}  // namespace
+
+int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                      const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                      int32_t layer_begin, int32_t layer_end, void *out_k, void *out_v,
+                      int64_t out_capacity_tokens, int32_t *out_offsets, cudaStream_t st)
+{
+    GatherArgs a;
+    a.num_requests = num_requests;
+    a.tt_offsets = tt_offsets;
+    a.tt_slots = tt_slots;
+    a.keep = keep;
+    a.select = select;
+    a.req_n = ctx->req_n;
+    a.out_offsets = out_offsets;
+    a.g_src = ctx->g_src;
+    a.g_total = ctx->g_total;
+    a.counts = ctx->counts;
+    a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
+    a.v_pool = (const uint8_t *)ctx->cfg.v_pool;
+    a.out_k = (uint8_t *)out_k;
+    a.out_v = (uint8_t *)out_v;
+    a.layer_stride = ctx->layer_stride;
+    a.row_bytes = ctx->row_bytes;
+    a.slots_per_layer = ctx->slots_per_layer;
+    a.out_capacity = out_capacity_tokens;
+    a.max_tokens = ctx->cfg.max_tokens;
+    a.layer_begin = layer_begin;
+    a.layer_end = layer_end;
+    a.max_requests = ctx->cfg.max_requests;
+    gather_count_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_scan_kernel<<<1, 1024, 0, st>>>(a);
+    gather_assign_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_copy_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}

@@ -1,0 +1,48 @@
+"""The C-ABI libraries load without a GPU and export every symbol the headers declare."""
+import ctypes
+import os
+import re
+
+from paper_2608_13263_b200 import binding, build, harness
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions(header):
+    text = open(header).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(vtoken_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    build.build()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    names = declared_functions(os.path.join(ROOT, "include", "vtoken.h"))
+    assert "vtoken_plan" in names and "vtoken_repack" in names and "vtoken_gather_logical" in names
+    for n in names:
+        assert hasattr(lib, n), n
+    # the binding carries the same names
+    assert sorted(binding.SYMBOLS) == [n for n in names]
+    for n in names:
+        assert hasattr(binding, n) or n in ("vtoken_strerror", "vtoken_last_cuda_error"), n
+
+
+def test_harness_library_loads():
+    build.build()
+    lib = ctypes.CDLL(harness.LIB_PATH)
+    for n in harness.SYMBOLS:
+        assert hasattr(lib, n), n
+
+
+def test_strerror_and_argument_errors_without_gpu():
+    assert binding.strerror(0) == "ok"
+    assert "capacity" in binding.strerror(binding.ECAPACITY)
+    lib = binding.load()
+    # NULL arguments are rejected before any CUDA call
+    assert lib.vtoken_create(None, None) == binding.EINVAL
+    assert lib.vtoken_repack(None, None) == binding.EINVAL
+    cfg = binding.Config(1, 4, 16, 1, 4, 2, 256, 512, 0, 1, 16, 4, 4, 0, 0)   # row_bytes = 8: not a multiple of 16
+    ctx = ctypes.c_void_p()
+    assert lib.vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)) == binding.EINVAL
+    cfg = binding.Config(1, 4, 16, 1, 8, 2, 257, 512, 0, 1, 16, 4, 4, 0, 0)   # misaligned pool
+    assert lib.vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)) == binding.EINVAL

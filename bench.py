@@ -1,0 +1,402 @@
+#!/usr/bin/env python
+"""Benchmark of the repack path (plan + all-layer K/V gather-copy) on B200.
+
+One step = one replay of the CUDA graph that holds the whole hot path (planner kernels and the
+copy kernel) on a side stream, over one seeded synthetic workload whose pools are resident
+in HBM.  Metric: repack HBM GB/s = 2 * M * token_bytes / t (every moved row read once and
+written once, K and V, all layers), M = live tokens of the admitted requests.
+
+    python bench.py                       # 1 GPU, Llama-3-8B-shaped KV, H2O-style 20 % budget
+    python bench.py --config mistral7b_random --steps 20 --warmup 3
+    torchrun ... bench.py --gpus N        # one independent pool per rank (weak scaling, no collective)
+    python bench.py --impl reference      # the CPU oracle timed on the host cores
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2608_13263_b200 import workloads as wl  # noqa: E402
+
+METRIC = "repack HBM GB/s (read+write); live tokens repacked/s and fraction of HBM peak in the same line"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+KERNELS_PER_STEP = 5        # plan: count, scan, assign, publish; copy: 1
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def committed_traffic(workload_name):
+    """DRAM bytes per moved token of the copy kernel from the committed ncu capture, or None."""
+    path = os.path.join(ROOT, "profiles", "copy_kernel_dram_traffic.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return d.get(workload_name) or d.get("default")
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.lines = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "50", "-i", str(self.index)], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.12)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_workload(name, seed, scale_requests=1.0):
+    gen = wl.CONFIGS[name]
+    if scale_requests != 1.0:
+        import inspect
+        default_r = inspect.signature(gen).parameters["requests"].default
+        return gen(seed=seed, requests=max(1, int(round(default_r * scale_requests))))
+    return gen(seed=seed)
+
+
+def context_stats(w, out):
+    """Input statistics plus block counts after the repack (reporting only)."""
+    s = wl.stats(w)
+    blocks_after = int(out["new_bt_offsets"][w.num_requests])
+    kept = s["kept_tokens"]
+    s["blocks_after"] = blocks_after
+    s["F_after"] = float(1.0 - kept / max(1, blocks_after * w.block_size))
+    s["retained_block_reduction_vs_naive_evict"] = float(1.0 - blocks_after / max(1, s["blocks_with_a_kept_token"]))
+    s["paper_retained_block_reduction_range_h100_vllm"] = [0.272, 0.723]
+    return s
+
+
+# ----------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on the host cores
+# ----------------------------------------------------------------------------------------------
+def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1, use_gpu_fill=True):
+    """Times plan + row moves of the oracle on `sample_layers` layers (K and V) of the workload.
+    Returns (seconds per step, moved bytes per step, description)."""
+    from oracle import vto
+    L = min(sample_layers, w.num_layers)
+    threads = max(1, min(threads, 2 * L))      # one slab per thread at most
+    shape = (L, w.slots_per_layer, w.row_elems)
+    k = v = None
+    if use_gpu_fill:
+        try:
+            import torch
+            from paper_2608_13263_b200 import harness as vh
+            if torch.cuda.is_available():
+                k = np.empty(shape, np.uint16)
+                v = np.empty(shape, np.uint16)
+                buf = torch.empty((w.slots_per_layer, w.row_elems), dtype=torch.int16, device="cuda")
+                for kv, dst in ((0, k), (1, v)):
+                    for l in range(L):
+                        vh.vth_fill(buf, kv, w.num_layers, l, l + 1, w.slots_per_layer, w.row_elems, fill_seed)
+                        dst[l] = buf.cpu().numpy().view(np.uint16)
+                del buf
+        except Exception:
+            k = v = None
+    if k is None:
+        rng = np.random.default_rng(fill_seed)
+        k = rng.integers(0, 2 ** 16, size=shape, dtype=np.uint16)
+        v = rng.integers(0, 2 ** 16, size=shape, dtype=np.uint16)
+    times = []
+    p = None
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        p = vto.plan_workload(w)
+        vto.apply_moves_pools(k, v, p.move_src, p.move_dst, threads=threads)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+    moved = 2 * p.num_moves * (2 * L * w.row_bytes)
+    desc = (f"oracle plan over all {w.num_requests} requests + row moves of layers 0..{L - 1} "
+            f"(K and V, {2 * L} of {2 * w.num_layers} slabs), host-resident pools, {threads} OpenMP threads")
+    return float(np.mean(times)), moved, desc, p, threads
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import vto
+    w = build_workload(args.config, args.seed, args.scale_requests)
+    cores = min(os.cpu_count() or 1, vto.openmp_threads())
+    sec, moved, desc, p, cores = oracle_sample(w, args.oracle_layers, cores, args.steps, max(1, min(args.warmup, 2)))
+    gbs = moved / sec / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"{w.name} (seed {args.seed})", "requests": w.num_requests,
+                   "tokens_moved_per_step": p.num_moves, "sample": desc},
+        "tokens_per_s": moved / (2 * w.token_bytes) / sec,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------------
+# CUDA arm
+# ----------------------------------------------------------------------------------------------
+def run_cuda(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_13263_b200 import binding as vt
+    from paper_2608_13263_b200.device import DeviceProblem, origin_map
+    from paper_2608_13263_b200.parallel import Ranks
+
+    ranks = Ranks.from_env(args.gpus)
+    torch.cuda.set_device(ranks.local_rank)
+    dev = torch.device("cuda", ranks.local_rank)
+    ranks.init(backend="nccl")
+
+    # one independent pool per rank: weak scaling, no data-path collective
+    seed = args.seed + ranks.rank
+    w = build_workload(args.config, seed, args.scale_requests)
+    free_b, total_b = torch.cuda.mem_get_info(dev)
+    need = 2 * w.pool_bytes + (1 << 30)
+    while need > free_b * 0.95 and w.num_requests > 1:
+        args.scale_requests *= 0.5
+        w = build_workload(args.config, seed, args.scale_requests)
+        need = 2 * w.pool_bytes + (1 << 30)
+
+    prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas)
+    grid = vt.vtoken_copy_grid(prob.ctx)
+    side = torch.cuda.Stream(device=dev)
+
+    # ---- capture: whole path, and the copy alone -------------------------------------------
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        prob.plan(stream=side)
+        prob.repack(stream=side)
+    side.synchronize()
+    g_all, g_copy, g_plan = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_all, stream=side):
+        prob.plan(stream=torch.cuda.current_stream())
+        prob.repack(stream=torch.cuda.current_stream())
+    with torch.cuda.graph(g_copy, stream=side):
+        prob.repack(stream=torch.cuda.current_stream())
+    with torch.cuda.graph(g_plan, stream=side):
+        prob.plan(stream=torch.cuda.current_stream())
+    out = prob.outputs()
+    M = out["num_moves"]
+    bytes_per_step = 2 * M * w.token_bytes
+
+    def timed(graph, steps, warmup, per_launch=False):
+        """Device time of `steps` replays on the side stream (ms total, list of per-launch ms)."""
+        with torch.cuda.stream(side):
+            for _ in range(warmup):
+                graph.replay()
+        side.synchronize()
+        ranks.barrier()
+        torch.cuda.synchronize(dev)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        with torch.cuda.stream(side):
+            evs[0].record(side)
+            for i in range(steps):
+                graph.replay()
+                if per_launch or i == steps - 1:
+                    evs[i + 1].record(side)
+        side.synchronize()
+        torch.cuda.synchronize(dev)
+        ranks.barrier()
+        total = evs[0].elapsed_time(evs[steps])
+        each = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)] if per_launch else []
+        return total, each
+
+    sampler = ClockSampler(ranks.local_rank)
+    sampler.start()
+    total_ms, _ = timed(g_all, args.steps, args.warmup)
+    copy_total_ms, copy_each = timed(g_copy, args.steps, args.warmup, per_launch=True)
+    plan_total_ms, _ = timed(g_plan, args.steps, args.warmup)
+
+    ms_per_step = ranks.max(total_ms / args.steps)
+    all_bytes = ranks.sum(bytes_per_step)
+    all_tokens = ranks.sum(M)
+    value = all_bytes / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end: host tables in, host tables out, through vtoken_repack_host -----------
+    R, T, NBT = w.num_requests, w.num_tokens, len(w.bt_blocks)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_in = dict(bt_offsets=pin(w.bt_offsets), bt_blocks=pin(w.bt_blocks), tt_offsets=pin(w.tt_offsets),
+                tt_slots=pin(w.tt_slots), keep=pin(w.keep), free_blocks=pin(w.free_blocks))
+    if w.select is not None:
+        h_in["select"] = pin(w.select)
+    h_out = dict(new_bt_offsets=torch.zeros(R + 1, dtype=torch.int32).pin_memory(),
+                 new_bt_blocks=torch.zeros(max(1, NBT), dtype=torch.int32).pin_memory(),
+                 new_tt_slots=torch.zeros(max(1, T), dtype=torch.int32).pin_memory(),
+                 freed_blocks=torch.zeros(max(1, NBT), dtype=torch.int32).pin_memory(),
+                 req_status=torch.zeros(max(1, R), dtype=torch.int32).pin_memory())
+    h2d = 8 + 2 * 4 * (R + 1) + 4 * NBT + 5 * T + 4 * len(w.free_blocks) + (R if w.select is not None else 0)
+    d2h = 4 * (R + 1) + 4 * NBT + 4 * T + 4 * NBT + 4 * R + 32
+
+    def e2e_once():
+        return vt.vtoken_repack_host(prob.ctx, num_requests=R, num_free=len(w.free_blocks), thr_num=w.thr_num,
+                                     thr_den=w.thr_den, stream=side, **h_in, **h_out)
+    for _ in range(args.warmup):
+        e2e_once()
+    ranks.barrier()
+    torch.cuda.synchronize(dev)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    e0.record(side)
+    for _ in range(args.steps):
+        c_host = e2e_once()
+    e1.record(side)
+    side.synchronize()
+    e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
+    e2e_ms = ranks.max(max(e0.elapsed_time(e1) / args.steps, e2e_wall_ms))
+    e2e_value = all_bytes / (e2e_ms * 1e-3) / 1e9
+    clocks = sampler.stop()      # sampled over every timed region above
+
+    # ---- parity at full size, in the launch configuration that was timed --------------------
+    parity = "skipped"
+    if not args.no_verify:
+        from oracle import vto   # the checker: tests/bench only
+        p = vto.plan_workload(w)
+        ok = (out["error_flags"] == 0 and c_host["error_flags"] == 0 and M == p.num_moves
+              and np.array_equal(out["new_tt_slots"], p.new_tt_slots)
+              and np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
+              and np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+              and np.array_equal(out["freed_blocks"], p.freed_blocks)
+              and np.array_equal(out["req_status"], p.req_status)
+              and np.array_equal(h_out["new_tt_slots"].numpy()[:T], p.new_tt_slots))
+        bad_words = prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst))
+        parity = "ok" if (ok and bad_words == 0) else f"FAILED (tables_ok={ok}, mismatching_words={bad_words})"
+
+    # ---- roofline of the dominant kernel (the copy), timed alone on its stream ---------------
+    peak, peak_kind = measured_peak()
+    copy_ms = float(np.mean(copy_each))
+    achieved = bytes_per_step / (copy_ms * 1e-3) / 1e9
+    per_token = committed_traffic(w.name)
+    roofline = {"bound": "hbm", "kernel": "copy_bulk_kernel" if grid["variant"] == 2 else "copy_rows_kernel",
+                "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                "algorithmic_bytes_per_launch": bytes_per_step,
+                "launch_ms_mean": copy_ms, "launch_ms_median": float(np.median(copy_each)),
+                "launch_ms_min": float(np.min(copy_each)),
+                "traffic": (per_token * M) if per_token else None}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": ranks.world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": f"{w.name} (seed {args.seed}+rank)", "requests": w.num_requests,
+                   "layers": w.num_layers, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
+                   "block_size": w.block_size, "num_blocks": w.num_blocks, "row_bytes": w.row_bytes,
+                   "token_bytes": w.token_bytes, "tokens_moved_per_step": M, "bytes_moved_per_step": bytes_per_step,
+                   "pool_GiB_per_gpu": 2 * w.pool_bytes / 2 ** 30, "scale_requests": args.scale_requests,
+                   "l2": "moved bytes per step exceed the 126 MB L2 (no flush needed)" if bytes_per_step > 4 * 126e6
+                         else "moved bytes per step fit in L2: launch-bound parity configuration",
+                   "launch": "CUDA graph (plan + copy) replayed on a side stream", "copy_grid": grid,
+                   "parallelism": f"{ranks.world} independent pools, no collective"},
+        "tokens_per_s": all_tokens / (ms_per_step * 1e-3),
+        "frac_of_measured_hbm_peak": value / (peak * ranks.world),
+        "frac_of_nominal_8TBs": value / (NOMINAL_HBM_GBS * ranks.world),
+        "plan_us": plan_total_ms / args.steps * 1e3, "copy_ms": copy_ms,
+        "clocks": clocks, "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "e2e": {"value": e2e_value, "unit": "GB/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h,
+                "what": "vtoken_repack_host: pinned host tables -> device, plan, copy, every output table -> host, sync; "
+                        "the K/V pools are the GPU-resident cache and stay in HBM"},
+        "roofline": roofline, "parity": parity, "stats": context_stats(w, out),
+    }
+
+    # ---- oracle timed beside it (rank 0, N = 1 only) ------------------------------------------
+    if ranks.world == 1 and not args.no_cpu_baseline:
+        from oracle import vto
+        cores = min(os.cpu_count() or 1, vto.openmp_threads())
+        sec, moved, desc, _, cores = oracle_sample(w, args.oracle_layers, cores, 3, 1)
+        sec1, moved1, desc1, _, _ = oracle_sample(w, 1, 1, 2, 1)
+        line["cpu_baseline"] = {"value": moved / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                "sample": desc, "single_thread_GBs": moved1 / sec1 / 1e9}
+    prob.close()
+    if ranks.rank == 0:
+        print(json.dumps(line))
+    ranks.finalize()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--config", default="llama8b_h2o", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--variant", type=int, default=0, help="copy path: 0 auto, 1 registers, 2 bulk copy")
+    ap.add_argument("--max-ctas", type=int, default=0)
+    ap.add_argument("--scale-requests", type=float, default=1.0)
+    ap.add_argument("--oracle-layers", type=int, default=8, help="layers in the CPU-baseline sample")
+    ap.add_argument("--no-verify", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -189,6 +189,40 @@ typedef struct {                   /* all HOST pointers */
 } vtoken_host_tables;
 int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *tables, void *cuda_stream);
 
+/* Logical gather for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a packaging variant of vtoken_gather_logical, same result.)
+ *
+ * Who needs it: a serving engine that has handed nearly all of HBM to its KV pool (the paper
+ * runs at gpu_mem_util = 0.90) has nothing left for vtoken_create's scratch and may see
+ * cudaMalloc fail; code on a latency-critical step cannot afford cudaMalloc either, because
+ * it synchronises the whole device; and some embedders simply forbid allocator calls outside
+ * their own pool.  This entry point takes no context and calls no cudaMalloc, cudaFree or
+ * other allocating routine.  Its scratch is a fixed array inside the library's device image
+ * (about 1 MiB per GPU that loads the library, held until the process exits), which bounds
+ * the problem size:
+ *     max_requests        <= 4096
+ *     out_capacity_tokens <= 262144
+ * Larger values return VTOKEN_ECAPACITY and enqueue nothing.
+ *
+ * Arguments: the pool geometry that vtoken_create would take (pools DEVICE, 16-byte aligned,
+ * row_bytes a multiple of 16, layer_stride_bytes 0 => num_blocks*block_size*row_bytes), then
+ * exactly the arguments of vtoken_gather_logical; max_requests bounds *num_requests and fixes
+ * the grid.  error_flags: DEVICE uint32 or NULL, receives the VTOKEN_FLAG_* bits of this call
+ * (bad slot, gather overflow), written on the stream.  The caller owns inputs and outputs.
+ *
+ * The first call on each device looks up the device address of the scratch array (that
+ * device must be current); make that first call before starting any stream capture.
+ * All calls on a device share the one scratch array: the call clears what it needs cleared,
+ * but two calls whose kernels overlap on the GPU (different streams without an event between
+ * them) race on it and corrupt each other's output.  Order them on one stream or by events. */
+int vtoken_gather_logical_noalloc(const void *k_pool, const void *v_pool, int32_t num_layers,
+                                  int32_t num_blocks, int32_t block_size, int64_t row_bytes,
+                                  int64_t layer_stride_bytes, const int32_t *num_requests,
+                                  int32_t max_requests, const int32_t *tt_offsets, const int32_t *tt_slots,
+                                  const uint8_t *keep, const uint8_t *select, int32_t layer_begin,
+                                  int32_t layer_end, void *out_k, void *out_v, int64_t out_capacity_tokens,
+                                  int32_t *out_offsets, uint32_t *error_flags, void *cuda_stream);
+
 /* Diagnostics. */
 const char *vtoken_strerror(int code);
 int vtoken_last_cuda_error(const vtoken_ctx *ctx);       /* cudaError_t of the last VTOKEN_ECUDA */

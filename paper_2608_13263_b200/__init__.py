@@ -13,6 +13,7 @@ from .binding import (  # noqa: F401
     vtoken_create,
     vtoken_destroy,
     vtoken_gather_logical,
+    vtoken_gather_logical_noalloc,
     vtoken_plan,
     vtoken_read_counts,
     vtoken_repack,
@@ -22,4 +23,4 @@ from .binding import (  # noqa: F401
 
 __all__ = ["VtokenError", "vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack",
            "vtoken_gather_logical", "vtoken_read_counts", "vtoken_repack_host", "vtoken_copy_grid",
-           "vtoken_scratch_bytes"]
+           "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc"]

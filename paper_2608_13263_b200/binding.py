@@ -18,7 +18,7 @@ FLAG_BAD_SLOT, FLAG_BAD_BLOCK, FLAG_BAD_FREE, FLAG_CAPACITY, FLAG_TIMEOUT, FLAG_
 
 SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "vtoken_gather_logical",
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
-           "vtoken_copy_grid", "vtoken_scratch_bytes"]
+           "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc"]
 
 
 class VtokenError(RuntimeError):
@@ -102,6 +102,11 @@ def load():
         lib.vtoken_copy_grid.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 4
         lib.vtoken_scratch_bytes.argtypes = [ctypes.c_void_p]
         lib.vtoken_scratch_bytes.restype = ctypes.c_int64
+        lib.vtoken_gather_logical_noalloc.argtypes = (
+            [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64,
+             ctypes.c_int64, ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
+            [ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
+             ctypes.c_void_p, ctypes.c_void_p])
         _lib = lib
     return _lib
 
@@ -200,3 +205,22 @@ def vtoken_copy_grid(ctx) -> dict:
 
 def vtoken_scratch_bytes(ctx) -> int:
     return load().vtoken_scratch_bytes(ctx)
+
+
+NOALLOC_MAX_REQUESTS = 4096
+NOALLOC_MAX_TOKENS = 262144
+
+
+def vtoken_gather_logical_noalloc(*, k_pool, v_pool, num_layers, num_blocks, block_size, row_bytes, num_requests,
+                                  max_requests, tt_offsets, tt_slots, keep, select, layer_begin, layer_end, out_k,
+                                  out_v, out_capacity_tokens, out_offsets, error_flags=None, layer_stride_bytes=0,
+                                  stream=None) -> None:
+    """The logical gather without a context and without any device allocation: for callers
+    whose memory is fully committed to the KV pool or who may not call the allocator.  Limits:
+    max_requests <= 4096 and out_capacity_tokens <= 262144 (VtokenError ECAPACITY beyond).  Calls
+    on one device share a fixed scratch array, so they must not overlap on the GPU."""
+    _check(load().vtoken_gather_logical_noalloc(
+        _ptr(k_pool), _ptr(v_pool), num_layers, num_blocks, block_size, row_bytes, layer_stride_bytes,
+        _ptr(num_requests), max_requests, _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep), _ptr(select), layer_begin,
+        layer_end, _ptr(out_k), _ptr(out_v), out_capacity_tokens, _ptr(out_offsets), _ptr(error_flags),
+        _stream(stream)), "vtoken_gather_logical_noalloc")

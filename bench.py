@@ -106,13 +106,16 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def build_workload(name, seed, scale_requests=1.0):
+def build_workload(name, seed, scale_requests=1.0, block_size=0):
     gen = wl.CONFIGS[name]
+    kw = {}
+    if block_size:
+        kw["block_size"] = block_size
     if scale_requests != 1.0:
         import inspect
         default_r = inspect.signature(gen).parameters["requests"].default
-        return gen(seed=seed, requests=max(1, int(round(default_r * scale_requests))))
-    return gen(seed=seed)
+        kw["requests"] = max(1, int(round(default_r * scale_requests)))
+    return gen(seed=seed, **kw)
 
 
 def context_stats(w, out):
@@ -177,7 +180,7 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import vto
-    w = build_workload(args.config, args.seed, args.scale_requests)
+    w = build_workload(args.config, args.seed, args.scale_requests, args.block_size)
     cores = min(os.cpu_count() or 1, vto.openmp_threads())
     sec, moved, desc, p, cores = oracle_sample(w, args.oracle_layers, cores, args.steps, max(1, min(args.warmup, 2)))
     gbs = moved / sec / 1e9
@@ -212,12 +215,12 @@ def run_cuda(args):
 
     # one independent pool per rank: weak scaling, no data-path collective
     seed = args.seed + ranks.rank
-    w = build_workload(args.config, seed, args.scale_requests)
+    w = build_workload(args.config, seed, args.scale_requests, args.block_size)
     free_b, total_b = torch.cuda.mem_get_info(dev)
     need = 2 * w.pool_bytes + (1 << 30)
     while need > free_b * 0.95 and w.num_requests > 1:
         args.scale_requests *= 0.5
-        w = build_workload(args.config, seed, args.scale_requests)
+        w = build_workload(args.config, seed, args.scale_requests, args.block_size)
         need = 2 * w.pool_bytes + (1 << 30)
 
     prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas)
@@ -362,6 +365,9 @@ def run_cuda(args):
         "roofline": roofline, "parity": parity, "stats": context_stats(w, out),
     }
 
+    if args.proxy:
+        line["concurrency"] = run_proxy(args, prob, w, side, g_all, bytes_per_step, dev)
+
     # ---- oracle timed beside it (rank 0, N = 1 only) ------------------------------------------
     if ranks.world == 1 and not args.no_cpu_baseline:
         from oracle import vto
@@ -376,6 +382,89 @@ def run_cuda(args):
     ranks.finalize()
 
 
+def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
+    """Repack (captured graph, side stream) beside a bandwidth-bound decode-read proxy that reads
+    every allocated block through the OLD block tables on a high-priority main stream: each one
+    alone, then both at once.  The proxy's per-request checksums must not change (the repack
+    never writes an allocated block)."""
+    import torch
+    from paper_2608_13263_b200 import harness as vh
+    owner = np.repeat(np.arange(w.num_requests, dtype=np.int32), np.diff(w.bt_offsets))
+    owner_d = torch.from_numpy(owner).to(dev)
+    nbt = len(w.bt_blocks)
+    block_bytes = w.block_size * w.row_bytes
+    proxy_bytes = nbt * 2 * w.num_layers * block_bytes
+    main = torch.cuda.Stream(device=dev, priority=-1)
+    sums = torch.zeros(max(1, w.num_requests), dtype=torch.int64, device=dev)
+
+    def proxy(stream):
+        vh.vth_decode_read(prob.k_pool, prob.v_pool, prob.bt_offsets, prob.bt_blocks, owner_d, nbt, w.num_layers,
+                           block_bytes, w.slab_bytes, sums, ctas=args.proxy_ctas, stream=stream)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    torch.cuda.synchronize(dev)
+    sums.zero_()
+    torch.cuda.synchronize(dev)
+    proxy(main)
+    main.synchronize()
+    solo_sums = sums.clone()
+    # proxy alone
+    n_proxy = max(2, args.steps // 4)
+    a, b = ev(), ev()
+    a.record(main)
+    for _ in range(n_proxy):
+        proxy(main)
+    b.record(main)
+    main.synchronize()
+    proxy_alone_ms = a.elapsed_time(b) / n_proxy
+    # repack alone (again, same window length as the concurrent run)
+    n_rep = max(2, int(round(n_proxy * proxy_alone_ms / max(1e-3, bytes_per_step / 6e9 * 1e3))))
+    a, b = ev(), ev()
+    with torch.cuda.stream(side):
+        a.record(side)
+        for _ in range(n_rep):
+            g_all.replay()
+        b.record(side)
+    side.synchronize()
+    repack_alone_ms = a.elapsed_time(b) / n_rep
+    # both at once, released by one event
+    sums.zero_()
+    torch.cuda.synchronize(dev)
+    go, p0, p1, r0, r1 = ev(), ev(), ev(), ev(), ev()
+    go.record(torch.cuda.current_stream(dev))
+    main.wait_event(go)
+    side.wait_event(go)
+    p0.record(main)
+    with torch.cuda.stream(side):
+        r0.record(side)
+    # both queues are filled within a few hundred microseconds, the work lasts tens of milliseconds
+    for _ in range(n_proxy):
+        proxy(main)
+    with torch.cuda.stream(side):
+        for _ in range(n_rep):
+            g_all.replay()
+    p1.record(main)
+    with torch.cuda.stream(side):
+        r1.record(side)
+    torch.cuda.synchronize(dev)
+    proxy_conc_ms = p0.elapsed_time(p1) / n_proxy
+    repack_conc_ms = r0.elapsed_time(r1) / n_rep
+    window_ms = max(p0.elapsed_time(p1), r0.elapsed_time(r1), p0.elapsed_time(r1), r0.elapsed_time(p1))
+    # n_proxy launches accumulate by XOR: an even count cancels, an odd count equals the solo value
+    expect = solo_sums if n_proxy % 2 == 1 else torch.zeros_like(solo_sums)
+    checksum_ok = bool(torch.equal(sums, expect))
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
+    return {"proxy_bytes_per_launch": proxy_bytes, "proxy_launches": n_proxy, "repack_replays": n_rep,
+            "proxy_alone_GBs": gbs(proxy_bytes, proxy_alone_ms), "repack_alone_GBs": gbs(bytes_per_step, repack_alone_ms),
+            "proxy_concurrent_GBs": gbs(proxy_bytes, proxy_conc_ms),
+            "repack_concurrent_GBs": gbs(bytes_per_step, repack_conc_ms),
+            "sum_over_window_GBs": gbs(proxy_bytes * n_proxy + bytes_per_step * n_rep, window_ms),
+            "proxy_checksum_unchanged": checksum_ok,
+            "streams": "proxy on a high-priority stream, repack graph on the default-priority side stream"}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -388,6 +477,9 @@ def main():
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--scale-requests", type=float, default=1.0)
     ap.add_argument("--oracle-layers", type=int, default=8, help="layers in the CPU-baseline sample")
+    ap.add_argument("--proxy", action="store_true", help="also run the repack beside a decode-read proxy")
+    ap.add_argument("--proxy-ctas", type=int, default=0)
+    ap.add_argument("--block-size", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -32,7 +32,7 @@ from paper_2608_13263_b200 import workloads as wl  # noqa: E402
 METRIC = "repack HBM GB/s (read+write); live tokens repacked/s and fraction of HBM peak in the same line"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-KERNELS_PER_STEP = 5        # plan: count, scan, assign, publish; copy: 1
+KERNELS_PER_STEP = 4        # plan: count, scan, assign; copy: 1
 
 
 def measured_peak():
@@ -327,6 +327,26 @@ def run_cuda(args):
         bad_words = prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst))
         parity = "ok" if (ok and bad_words == 0) else f"FAILED (tables_ok={ok}, mismatching_words={bad_words})"
 
+    # ---- a plain device-to-device copy on this GPU, now (context for run-to-run variation) ---
+    live_copy = None
+    free_now, _ = torch.cuda.mem_get_info(dev)
+    if free_now > (6 << 30):
+        n = 1 << 30
+        src_t = torch.empty(n, dtype=torch.int16, device=dev)
+        dst_t = torch.empty(n, dtype=torch.int16, device=dev)
+        for _ in range(3):
+            dst_t.copy_(src_t)
+        best = 1e9
+        for _ in range(10):
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record()
+            dst_t.copy_(src_t)
+            c1.record()
+            c1.synchronize()
+            best = min(best, c0.elapsed_time(c1))
+        live_copy = 4 * n / (best * 1e-3) / 1e9
+        del src_t, dst_t
+
     # ---- roofline of the dominant kernel (the copy), timed alone on its stream ---------------
     peak, peak_kind = measured_peak()
     copy_ms = float(np.mean(copy_each))
@@ -338,6 +358,8 @@ def run_cuda(args):
                 "algorithmic_bytes_per_launch": bytes_per_step,
                 "launch_ms_mean": copy_ms, "launch_ms_median": float(np.median(copy_each)),
                 "launch_ms_min": float(np.min(copy_each)),
+                "plain_copy_now_GBs": live_copy,     # torch copy_ of 1 Gi 2-byte elements on this GPU, best of 10
+                "frac_of_plain_copy_now": (achieved / live_copy) if live_copy else None,
                 "traffic": (per_token * M) if per_token else None}
 
     line = {
@@ -352,6 +374,7 @@ def run_cuda(args):
                    "l2": "moved bytes per step exceed the 126 MB L2 (no flush needed)" if bytes_per_step > 4 * 126e6
                          else "moved bytes per step fit in L2: launch-bound parity configuration",
                    "launch": "CUDA graph (plan + copy) replayed on a side stream", "copy_grid": grid,
+                   "gpu": f"{torch.cuda.get_device_name(dev)} {str(torch.cuda.get_device_properties(dev).uuid)[-12:]}",
                    "parallelism": f"{ranks.world} independent pools, no collective"},
         "tokens_per_s": all_tokens / (ms_per_step * 1e-3),
         "frac_of_measured_hbm_peak": value / (peak * ranks.world),

@@ -23,7 +23,7 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 
 void free_all(vtoken_ctx *ctx)
 {
-    void *ptrs[] = {ctx->req_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
+    void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total,
                     ctx->stage.num_requests, ctx->stage.num_free, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
@@ -31,6 +31,9 @@ void free_all(vtoken_ctx *ctx)
                     ctx->stage.new_tt_slots, ctx->stage.freed_blocks, ctx->stage.req_status, ctx->stage.counts};
     for (void *p : ptrs)
         if (p) cudaFree(p);
+    if (ctx->stage.planned) cudaEventDestroy(ctx->stage.planned);
+    if (ctx->stage.copied) cudaEventDestroy(ctx->stage.copied);
+    if (ctx->stage.aux) cudaStreamDestroy(ctx->stage.aux);
 }
 
 int ensure_stage(vtoken_ctx *ctx)
@@ -54,6 +57,12 @@ int ensure_stage(vtoken_ctx *ctx)
     A(&ctx->stage.freed_blocks, c.max_table_blocks);
     A(&ctx->stage.req_status, c.max_requests);
     A(&ctx->stage.counts, 1);
+    if (rc == VTOKEN_OK) {
+        if (cudaStreamCreateWithFlags(&ctx->stage.aux, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->stage.planned, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->stage.copied, cudaEventDisableTiming) != cudaSuccess)
+            rc = VTOKEN_ECUDA;
+    }
     if (rc == VTOKEN_OK) ctx->stage.ready = true;
     return rc;
 }
@@ -98,6 +107,7 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     int rc = VTOKEN_OK;
     auto A = [&](auto **p, int64_t n) { if (rc == VTOKEN_OK) rc = dev_alloc(ctx, p, n); };
     A(&ctx->req_n, cfg->max_requests);
+    A(&ctx->part_n, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
     A(&ctx->req_dst_base, cfg->max_requests);
     A(&ctx->req_freed_base, cfg->max_requests);
     A(&ctx->req_status, cfg->max_requests);
@@ -214,14 +224,22 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     rc = vtk_launch_plan(ctx, &in, &out, st);
     if (rc != VTOKEN_OK) return rc;
     ctx->has_plan = true;
+    // every table output is final once the plan has run: copy them back on a second stream
+    // while the copy kernel moves the K/V rows on the caller's stream
+    VTK_CUDA(ctx, cudaEventRecord(s.planned, st));
     rc = vtk_launch_copy(ctx, st);
     if (rc != VTOKEN_OK) return rc;
-
+    cudaStream_t caller = st;
+    VTK_CUDA(ctx, cudaStreamWaitEvent(s.aux, s.planned, 0));
+    st = s.aux;
     D2H(h->new_bt_offsets, s.new_bt_offsets, (R + 1) * sizeof(int32_t));
     if (NBT) D2H(h->new_bt_blocks, s.new_bt_blocks, NBT * sizeof(int32_t));
     if (T) D2H(h->new_tt_slots, s.new_tt_slots, T * sizeof(int32_t));
     if (NBT) D2H(h->freed_blocks, s.freed_blocks, NBT * sizeof(int32_t));
     if (R) D2H(h->req_status, s.req_status, R * sizeof(int32_t));
+    VTK_CUDA(ctx, cudaEventRecord(s.copied, s.aux));
+    st = caller;
+    VTK_CUDA(ctx, cudaStreamWaitEvent(st, s.copied, 0));
     // the counts are read from the context's copy so that flags raised by the copy kernel are included
     D2H(h->counts, ctx->counts, sizeof(vtoken_counts));
 #undef H2D

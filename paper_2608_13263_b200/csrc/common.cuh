@@ -5,6 +5,8 @@
 
 #include "vtoken.h"
 
+#define VTK_PLAN_PARTS 8   // token ranges per request in the planner
+
 // ---------------------------------------------------------------------------------------
 // Context: configuration, derived sizes and every scratch buffer (allocated once).
 // ---------------------------------------------------------------------------------------
@@ -20,6 +22,7 @@ struct vtoken_ctx {
 
     // planner scratch (DEVICE)
     int32_t *req_n;            // [max_requests] live tokens
+    int32_t *part_n;           // [max_requests * VTK_PLAN_PARTS] live tokens per request part
     int32_t *req_dst_base;     // [max_requests] first destination block (index into the free list)
     int32_t *req_freed_base;   // [max_requests] first entry in freed_blocks
     int32_t *req_status;       // [max_requests]
@@ -39,13 +42,15 @@ struct vtoken_ctx {
         uint8_t *keep, *select;
         int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *req_status;
         vtoken_counts *counts;
+        cudaStream_t aux;              // carries the output copies while the copy kernel runs
+        cudaEvent_t planned, copied;   // plan done on the caller's stream; outputs copied on aux
     } stage;
     int64_t scratch_bytes;
 
     // launch shape of the copy kernel
     int copy_variant;          // 1 register path, 2 bulk-copy path
     int copy_ctas, copy_threads, copy_smem;
-    int bulk_warps, bulk_stages, bulk_rows;   // bulk path: warps per CTA, ring depth, rows per item
+    int bulk_warps, bulk_stages, bulk_rows, bulk_depth;   // bulk path: warps per CTA, ring size, rows per item, loads ahead
 };
 
 // host launchers, one per translation unit

@@ -129,116 +129,156 @@ __device__ __forceinline__ void bulk_s2g(void *gdst, const void *smem_src, uint3
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+// at most n (1..10) of this thread's newest store groups may still be reading shared memory
+__device__ __forceinline__ void bulk_wait_read_n(int n)
+{
+    switch (n) {
+        case 1: bulk_wait_read<1>(); break;
+        case 2: bulk_wait_read<2>(); break;
+        case 3: bulk_wait_read<3>(); break;
+        case 4: bulk_wait_read<4>(); break;
+        case 5: bulk_wait_read<5>(); break;
+        case 6: bulk_wait_read<6>(); break;
+        case 7: bulk_wait_read<7>(); break;
+        case 8: bulk_wait_read<8>(); break;
+        case 9: bulk_wait_read<9>(); break;
+        default: bulk_wait_read<10>(); break;
+    }
+}
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 constexpr int BULK_MAX_WARPS = 8;
-constexpr int BULK_MAX_STAGES = 8;
+constexpr int BULK_MAX_STAGES = 12;
 
-// Each warp runs its own pipeline over its items.  At step k it (1) frees and refills the
-// stage that item k+depth will use (its previous tenant is item k+depth-stages <= k-2, so at
-// most the newest store group may still be reading shared memory), (2) waits for the rows of
-// item k, (3) stores them with one bulk copy.
-__global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages)
+// Each warp runs its own pipeline through a ring of `stages` shared-memory buffers.
+//
+// Work: an item is `rows` consecutive destination slots of one destination block in one slab
+// (rows is a power of two that divides S, so its destination is one contiguous byte range).
+// Items are numbered slab-major and dealt to the warps of the grid round-robin: at any moment
+// the grid works on a window of consecutive items, i.e. on one contiguous destination range of
+// a few MB, which keeps DRAM pages and TLB entries hot on the write side.
+//
+// Step k of a warp's pipeline: (1) free and refill the stage that item k+depth will use -- its
+// previous tenant is item k+depth-stages = k-(w+1), w = stages-depth-1, so the w newest store
+// groups may still be reading shared memory; each lane issues one cp.async.bulk global->shared
+// for its source row, completion bytes counted on the stage's mbarrier -- (2) wait for the rows
+// of item k (bounded), (3) one lane stores them with a single cp.async.bulk shared->global.
+//
+// Nothing on that path waits for a global-memory read of the plan: the entries of an item
+// (destination block id, source slot of the lane's row) are fetched two items ahead into
+// registers, what the store side needs (destination address, valid-row mask) is parked in
+// shared memory at issue time, and item indices advance by additions (no per-step division).
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages, int depth)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint64_t bars[BULK_MAX_WARPS * BULK_MAX_STAGES];
+    __shared__ uint64_t park_dst[BULK_MAX_WARPS * BULK_MAX_STAGES];    // destination address of the staged item
+    __shared__ uint32_t park_mask[BULK_MAX_WARPS * BULK_MAX_STAGES];   // which of its rows are valid
 
     const int lane = vtk_lane(), warp = threadIdx.x >> 5, nwarps_cta = blockDim.x >> 5;
-    const int rows = a.rows;
+    const int rows = a.rows;                                   // power of two, divides S, <= 32
+    const int S = a.S;
     const uint32_t row_bytes = (uint32_t)a.row_bytes;
     const uint32_t stage_bytes = rows * row_bytes;
     uint8_t *my_smem = smem + (size_t)warp * stages * stage_bytes;
     uint64_t *my_bars = bars + warp * BULK_MAX_STAGES;
+    uint64_t *my_dst = park_dst + warp * BULK_MAX_STAGES;
+    uint32_t *my_mask = park_mask + warp * BULK_MAX_STAGES;
     if (lane == 0) {
         for (int s = 0; s < stages; ++s) mbar_init(&my_bars[s], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
 
-    const int nblk = a.counts->num_dst_blocks;
-    const int parts = (a.S + rows - 1) / rows;                 // items per destination block
-    const int64_t items_per_slab = (int64_t)nblk * parts;
-    const int64_t total = items_per_slab * 2 * a.L;
+    const int parts = S / rows;                                // items per destination block
+    const int per_slab = a.counts->num_dst_blocks * parts;     // items per slab, < 2^31 (checked on the host)
+    const int num_slabs = 2 * a.L;
     const int64_t gw = (int64_t)blockIdx.x * nwarps_cta + warp;
     const int64_t gstride = (int64_t)gridDim.x * nwarps_cta;
-    const int depth = stages - 2;                              // items loading ahead of the one being stored
-    bool timed_out = false;
+    const int stores_in_flight = stages - depth - 1;
 
-    // issue the loads of this warp's k-th item into stage k % stages; returns nothing, the
-    // store side recomputes the item's geometry
-    auto issue = [&](int64_t k) {
-        const int64_t it = gw + k * gstride;
-        if (it >= total) return;
-        const int s = (int)(k % stages);
-        const int slab = (int)(it / items_per_slab);
-        const int64_t rem = it - (int64_t)slab * items_per_slab;
-        const int j = (int)(rem / parts), part = (int)(rem - (int64_t)j * parts);
-        const int i0 = part * rows;
-        const int nrows = min(rows, a.S - i0);
-        const int32_t blk = a.dst_blocks[j];
-        const uint8_t *base = slab_base(a, slab);
-        uint8_t *stg = my_smem + (size_t)s * stage_bytes;
-        // all store groups but the newest have finished reading shared memory
-        bulk_wait_read<1>();
-        __syncwarp();
-        unsigned valid_total = 0;
-        for (int i = lane; i < ((nrows + 31) & ~31); i += 32) {
-            int32_t src = -1;
-            if (i < nrows && blk >= 0) src = a.dst_src[(int64_t)j * a.S + i0 + i];
-            valid_total += __popc(__ballot_sync(0xffffffffu, src >= 0));
-        }
-        if (lane == 0) mbar_expect_tx(&my_bars[s], valid_total * row_bytes);   // 0 rows: plain arrive
-        __syncwarp();
-        for (int i = lane; i < nrows; i += 32) {
-            const int32_t src = blk >= 0 ? a.dst_src[(int64_t)j * a.S + i0 + i] : -1;
-            if (src >= 0) bulk_g2s(stg + (size_t)i * row_bytes, base + (int64_t)src * a.row_bytes, row_bytes, &my_bars[s]);
+    // cursors over this warp's items (gw, gw + gstride, ...) as (slab, item inside the slab)
+    struct Cursor { int slab, rem; };
+    const int step_slabs = per_slab > 0 ? (int)(gstride / per_slab) : 0;
+    const int step_rem = per_slab > 0 ? (int)(gstride % per_slab) : 0;
+    Cursor c_fetch;
+    c_fetch.slab = per_slab > 0 ? (int)min((int64_t)num_slabs, gw / per_slab) : num_slabs;
+    c_fetch.rem = per_slab > 0 ? (int)(gw % per_slab) : 0;
+
+    // plan entries of the next two items to issue: slab, destination slot of the first row
+    // (-1: skip the item), source slot of this lane's row (-1: no row)
+    struct Entry { int slab; int32_t dst0, src; };
+    Entry e1, e2;
+    auto fetch = [&](Entry &e) {           // reads the item under c_fetch, moves the cursor
+        e.slab = c_fetch.slab;
+        e.dst0 = -1;
+        e.src = -1;
+        if (c_fetch.slab < num_slabs) {
+            const int j = (int)((unsigned)c_fetch.rem / (unsigned)parts);
+            const int i0 = (c_fetch.rem - j * parts) * rows;
+            const int32_t blk = a.dst_blocks[j];
+            if (lane < rows) e.src = a.dst_src[(int64_t)j * S + i0 + lane];
+            e.dst0 = blk >= 0 ? blk * S + i0 : -1;
+            c_fetch.slab += step_slabs;
+            c_fetch.rem += step_rem;
+            if (c_fetch.rem >= per_slab) { c_fetch.rem -= per_slab; ++c_fetch.slab; }
         }
     };
+    fetch(e1);
+    fetch(e2);
 
-    for (int64_t k = 0; k < depth; ++k) issue(k);
-    for (int64_t k = 0;; ++k) {
-        const int64_t it = gw + k * gstride;
-        if (it >= total) break;
-        issue(k + depth);
-        const int s = (int)(k % stages);
-        if (!mbar_wait_bounded(&my_bars[s], (uint32_t)((k / stages) & 1))) { timed_out = true; break; }
-        const int slab = (int)(it / items_per_slab);
-        const int64_t rem = it - (int64_t)slab * items_per_slab;
-        const int j = (int)(rem / parts), part = (int)(rem - (int64_t)j * parts);
-        const int i0 = part * rows;
-        const int nrows = min(rows, a.S - i0);
-        const int32_t blk = a.dst_blocks[j];
-        if (blk >= 0) {
-            uint8_t *base = slab_base(a, slab);
+    int s_issue = 0, issued = 0, stored = 0;
+    auto issue = [&]() {
+        if (e1.slab >= num_slabs) return;
+        const int s = s_issue;
+        s_issue = s_issue + 1 == stages ? 0 : s_issue + 1;
+        const Entry e = e1;
+        e1 = e2;
+        fetch(e2);                                   // in flight for two steps before it is used
+        const bool valid = e.src >= 0 && e.dst0 >= 0;
+        uint8_t *base = slab_base(a, e.slab);
+        uint8_t *stg = my_smem + (size_t)s * stage_bytes;
+        bulk_wait_read_n(stores_in_flight);          // the stage's previous store has read its bytes
+        const unsigned mask = __ballot_sync(0xffffffffu, valid);
+        if (lane == 0) {
+            my_mask[s] = mask;
+            my_dst[s] = (uint64_t)(base + (int64_t)e.dst0 * a.row_bytes);
+            mbar_expect_tx(&my_bars[s], (uint32_t)__popc(mask) * row_bytes);   // no rows: plain arrive
+        }
+        __syncwarp();
+        if (valid) bulk_g2s(stg + (size_t)lane * row_bytes, base + (int64_t)e.src * a.row_bytes, row_bytes, &my_bars[s]);
+        ++issued;
+    };
+
+    bool timed_out = false;
+    for (int k = 0; k < depth; ++k) issue();
+    int s = 0;
+    uint32_t parity = 0;
+    for (;;) {
+        issue();
+        if (stored == issued) break;
+        if (!mbar_wait_bounded(&my_bars[s], parity)) { timed_out = true; break; }
+        const unsigned mask = my_mask[s];
+        if (mask != 0) {
             uint8_t *stg = my_smem + (size_t)s * stage_bytes;
-            uint8_t *dst = base + ((int64_t)blk * a.S + i0) * a.row_bytes;
+            uint8_t *dst = (uint8_t *)my_dst[s];
+            const int nvalid = __popc(mask);
             // valid rows normally form a prefix (only the tail of a request's last block is empty)
-            int nvalid = 0;
-            bool prefix = true;
-            for (int i0w = 0; i0w < nrows; i0w += 32) {
-                const int i = i0w + lane;
-                const bool v = i < nrows && a.dst_src[(int64_t)j * a.S + i0 + i] >= 0;
-                const unsigned m = __ballot_sync(0xffffffffu, v);
-                const int cnt = __popc(m);
-                if (m != (cnt == 32 ? 0xffffffffu : ((1u << cnt) - 1u))) prefix = false;   // a hole inside this group
-                if (nvalid != i0w && cnt != 0) prefix = false;                             // a hole before this group
-                nvalid += cnt;
-            }
-            if (prefix) {
-                if (lane == 0 && nvalid > 0) bulk_s2g(dst, stg, (uint32_t)nvalid * row_bytes);
-            } else {
-                for (int i = lane; i < nrows; i += 32)
-                    if (a.dst_src[(int64_t)j * a.S + i0 + i] >= 0)
-                        bulk_s2g(dst + (size_t)i * row_bytes, stg + (size_t)i * row_bytes, row_bytes);
+            if (mask == (nvalid == 32 ? 0xffffffffu : ((1u << nvalid) - 1u))) {
+                if (lane == 0) bulk_s2g(dst, stg, (uint32_t)nvalid * row_bytes);
+            } else if ((mask >> lane) & 1u) {
+                bulk_s2g(dst + (size_t)lane * row_bytes, stg + (size_t)lane * row_bytes, row_bytes);
             }
         }
         bulk_commit();   // every lane commits (possibly empty) so group counts stay aligned
+        ++stored;
+        if (++s == stages) { s = 0; parity ^= 1u; }
     }
     if (timed_out) {
         // give loads still in flight a bounded chance to land before shared memory is released
-        for (int s = 0; s < stages; ++s) {
-            mbar_wait_bounded(&my_bars[s], 0, 50000000ull);
-            mbar_wait_bounded(&my_bars[s], 1, 50000000ull);
+        for (int q = 0; q < stages; ++q) {
+            mbar_wait_bounded(&my_bars[q], 0, 50000000ull);
+            mbar_wait_bounded(&my_bars[q], 1, 50000000ull);
         }
         if (lane == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_TIMEOUT);
     }
@@ -263,30 +303,41 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctx->copy_smem = 0;
         ctas_per_sm = 8;
     } else {
-        // tuning knobs: warps per CTA, ring depth, rows per item ("w,s,r"); defaults target
-        // about 192 KB of staging per SM
-        int warps = 4, stages = 3, rows = 0;
-        if (const char *e = getenv("VTOKEN_BULK_TUNE")) sscanf(e, "%d,%d,%d", &warps, &stages, &rows);
-        if (rows <= 0) {
-            rows = S;
-            while (rows > 1 && (int64_t)rows * ctx->row_bytes > 16384) rows = (rows + 1) / 2;
+        // tuning knobs "warps,stages,rows,depth": warps per CTA, ring size, rows per item, loads
+        // issued ahead.  Defaults: 8 warps x 6 stages x 4 KB items = 192 KB of staging per SM, two
+        // items loading ahead, three stores in flight per warp.  Measured on B200: shapes from 4 to
+        // 32 KB per item land within about 3 % of each other; below 4 KB per warp-step with only
+        // 8 warps per SM the pipeline becomes issue-bound.
+        int warps = 8, stages = 6, rows = 0, depth = 2;
+        if (const char *e = getenv("VTOKEN_BULK_TUNE")) sscanf(e, "%d,%d,%d,%d", &warps, &stages, &rows, &depth);
+        if (rows <= 0) rows = (int)(4096 / ctx->row_bytes);
+        // an item is `rows` consecutive destination slots inside one block: a power of two
+        // (<= 32, one row per lane) that divides the block size
+        {
+            int r = 1;
+            while (r * 2 <= rows && r * 2 <= 32 && S % (r * 2) == 0) r *= 2;
+            rows = r;
         }
-        if (rows > S) rows = S;
         if (warps < 1) warps = 1;
         if (warps > BULK_MAX_WARPS) warps = BULK_MAX_WARPS;
-        if (stages < 3) stages = 3;
+        if (stages < 2) stages = 2;
         if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
         int64_t smem = (int64_t)warps * stages * rows * ctx->row_bytes;
-        while (smem > 200 * 1024 && warps > 1) { --warps; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
-        while (smem > 200 * 1024 && stages > 3) { --stages; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
-        if (smem > 200 * 1024) return VTOKEN_EINVAL;
+        while (smem > 224 * 1024 && warps > 1) { --warps; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
+        while (smem > 224 * 1024 && stages > 2) { --stages; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
+        if (smem > 224 * 1024) return VTOKEN_EINVAL;
+        if (depth < 0) depth = 0;
+        if (depth > stages - 2) depth = stages - 2;
+        // the kernel indexes the items of a slab with 32-bit integers
+        if ((int64_t)ctx->cap_dst_blocks * (S / rows) >= (int64_t)INT32_MAX) return VTOKEN_EINVAL;
+        ctx->bulk_depth = depth;
         ctx->bulk_warps = warps;
         ctx->bulk_stages = stages;
         ctx->bulk_rows = rows;
         ctx->copy_threads = warps * 32;
         ctx->copy_smem = (int)smem;
         VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        ctas_per_sm = (int)((220 * 1024) / (smem + 1024));
+        ctas_per_sm = (int)((227 * 1024) / (smem + 2048));
         if (ctas_per_sm < 1) ctas_per_sm = 1;
         if (ctas_per_sm > 8) ctas_per_sm = 8;
     }
@@ -314,7 +365,7 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     if (ctx->copy_variant == 1)
         copy_rows_kernel<<<ctx->copy_ctas, ctx->copy_threads, 0, st>>>(a);
     else
-        copy_bulk_kernel<<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages);
+        copy_bulk_kernel<<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

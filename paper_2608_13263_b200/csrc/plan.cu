@@ -1,14 +1,18 @@
 // Relocation planner (Sec. 3.3.3 of the paper) as three small kernels:
-//   count  : live tokens per request                     (warp ballot + popc, one CTA per request)
+//   count  : live tokens per request part                (warp ballot + popc)
 //   scan   : candidates, admission against the free list, per-request bases, counts (one CTA)
 //   assign : rank of every live token -> destination slot, new tables, reclaimed list,
-//            inverse move plan for the copy kernel        (one CTA per request)
-// All grids are fixed by the capacities; R, T and num_free are read from device memory.
+//            inverse move plan for the copy kernel
+// Every request is cut into PLAN_PARTS equal token ranges, one CTA each in count and assign, so
+// that a 32k-token request does not serialise on one CTA; a part's first rank is the sum of the
+// live counts of the parts before it.  All grids are fixed by the capacities; R, T and num_free
+// are read from device memory.  No output order depends on atomics.
 #include "common.cuh"
 
 namespace {
 
 constexpr int PLAN_NT = 512;    // threads per CTA of count / assign
+constexpr int PLAN_PARTS = VTK_PLAN_PARTS;   // token ranges per request
 constexpr int SCAN_NT = 1024;   // threads of the single scan CTA
 
 struct PlanArgs {
@@ -21,7 +25,7 @@ struct PlanArgs {
     int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *out_status;
     vtoken_counts *out_counts;
     // context
-    int32_t *req_n, *req_dst_base, *req_freed_base, *req_status, *dst_src, *dst_blocks;
+    int32_t *req_n, *part_n, *req_dst_base, *req_freed_base, *req_status, *dst_src, *dst_blocks;
     vtoken_counts *counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
     int64_t slots_per_layer, max_tokens, max_table_blocks;
@@ -33,15 +37,34 @@ __device__ __forceinline__ int clamp_requests(const PlanArgs &a)
     return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
 }
 
+// token range [p0, p1) of part c of a request spanning [t0, t1): equal parts, multiples of 128
+__device__ __forceinline__ void part_range(int64_t t0, int64_t t1, int c, int64_t &p0, int64_t &p1)
+{
+    const int64_t len = t1 - t0;
+    int64_t per = (len + PLAN_PARTS - 1) / PLAN_PARTS;
+    per = (per + 127) & ~(int64_t)127;
+    p0 = t0 + (int64_t)c * per;
+    p1 = p0 + per;
+    if (p0 > t1) p0 = t1;
+    if (p1 > t1) p1 = t1;
+}
+
+__device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
+{
+    atomicOr(&a.counts->error_flags, flags);
+    atomicOr(&a.out_counts->error_flags, flags);
+}
+
 // ---- count -----------------------------------------------------------------------------
 __global__ void __launch_bounds__(PLAN_NT) plan_count_kernel(PlanArgs a)
 {
-    const int r = blockIdx.x;
+    const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
     if (r >= clamp_requests(a)) return;
-    const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
+    int64_t p0, p1;
+    part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
     int n = 0;
     bool bad = false;
-    for (int64_t t = t0 + threadIdx.x; t < t1; t += PLAN_NT)
+    for (int64_t t = p0 + threadIdx.x; t < p1; t += PLAN_NT)
         n += vtk_live(a.tt_slots[t], a.keep, t, a.slots_per_layer, bad) ? 1 : 0;
     __shared__ int warp_n[PLAN_NT / 32];
 #pragma unroll
@@ -52,7 +75,7 @@ __global__ void __launch_bounds__(PLAN_NT) plan_count_kernel(PlanArgs a)
     if (threadIdx.x == 0) {
         int s = 0;
         for (int w = 0; w < PLAN_NT / 32; ++w) s += warp_n[w];
-        a.req_n[r] = s;
+        a.part_n[blockIdx.x] = s;
     }
 }
 
@@ -128,7 +151,9 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         const bool valid = r < R;
         int n = 0, nb = 0;
         if (valid) {
-            n = a.req_n[r];
+#pragma unroll
+            for (int c = 0; c < PLAN_PARTS; ++c) n += a.part_n[r * PLAN_PARTS + c];
+            a.req_n[r] = n;
             nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
             if (nb < 0) nb = 0;
         }
@@ -172,6 +197,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         c.error_flags = flags | a.counts->error_flags;   // bits raised by the count kernel
         c.reserved = 0;
         *a.counts = c;
+        *a.out_counts = c;                               // later flags are OR-ed into both copies
     }
 }
 
@@ -179,13 +205,8 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
 {
     __shared__ int warp_sums[PLAN_NT / 32 + 1];
-    const int r = blockIdx.x;
-    const int R = clamp_requests(a);
-    if (r >= R) {
-        // the last CTA publishes the caller's copy of the counts once every flag is in:
-        // done by a separate tiny kernel below instead (needs all CTAs finished).
-        return;
-    }
+    const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
+    if (r >= clamp_requests(a)) return;
     const int tid = threadIdx.x;
     const int S = a.S;
     const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
@@ -197,40 +218,44 @@ __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
     const int nbt0 = a.new_bt_offsets[r];
     uint32_t flags = 0;
 
-    // block tables and the reclaimed list
+    // block tables and the reclaimed list: the request's parts share the work in stripes
+    const int stripe = c * PLAN_NT + tid, stride = PLAN_PARTS * PLAN_NT;
     if (adm) {
-        for (int j = tid; j < need; j += PLAN_NT) {
+        for (int j = stripe; j < need; j += stride) {
             int blk = a.free_blocks[dst_base + j];
             a.new_bt_blocks[nbt0 + j] = blk;
             if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
             a.dst_blocks[dst_base + j] = blk;
         }
         const int f0 = a.req_freed_base[r];
-        for (int j = tid; j < b1 - b0; j += PLAN_NT) {
+        for (int j = stripe; j < b1 - b0; j += stride) {
             const int blk = a.bt_blocks[b0 + j];
             if (blk < 0 || blk >= a.num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
             a.freed_blocks[f0 + j] = blk;
         }
         // unused tail of the last destination block
-        for (int i = n + tid; i < need * S; i += PLAN_NT) a.dst_src[(int64_t)dst_base * S + i] = -1;
+        for (int i = n + stripe; i < need * S; i += stride) a.dst_src[(int64_t)dst_base * S + i] = -1;
     } else {
-        for (int j = tid; j < b1 - b0; j += PLAN_NT) a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
+        for (int j = stripe; j < b1 - b0; j += stride) a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
     }
 
     // token table: rank of each live token in logical order -> destination slot
-    int carry = 0;
-    for (int64_t tb = t0; tb < t1; tb += PLAN_NT) {
+    int64_t p0, p1;
+    part_range(t0, t1, c, p0, p1);
+    int carry = 0;                                       // live tokens of the parts before this one
+    for (int cc = 0; cc < c; ++cc) carry += a.part_n[r * PLAN_PARTS + cc];
+    for (int64_t tb = p0; tb < p1; tb += PLAN_NT) {
         const int64_t t = tb + tid;
         int32_t slot = -1;
         bool live = false, bad = false;
-        if (t < t1) {
+        if (t < p1) {
             slot = a.tt_slots[t];
             live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
         }
         int total;
         const int i = carry + vtk_block_rank<PLAN_NT>(live, warp_sums, total);
         carry += total;
-        if (t < t1) {
+        if (t < p1) {
             int32_t out = -1;
             if (live) {
                 if (adm) {
@@ -245,13 +270,7 @@ __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
             a.new_tt_slots[t] = out;
         }
     }
-    if (flags) atomicOr(&a.counts->error_flags, flags);
-}
-
-// The caller's copy of the counts is written last, after every flag has been raised.
-__global__ void plan_publish_kernel(PlanArgs a)
-{
-    if (threadIdx.x == 0 && blockIdx.x == 0) *a.out_counts = *a.counts;
+    if (flags) raise_flags(a, flags);
 }
 
 }  // namespace
@@ -277,6 +296,7 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.out_status = out->req_status;
     a.out_counts = out->counts;
     a.req_n = ctx->req_n;
+    a.part_n = ctx->part_n;
     a.req_dst_base = ctx->req_dst_base;
     a.req_freed_base = ctx->req_freed_base;
     a.req_status = ctx->req_status;
@@ -293,10 +313,9 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.max_table_blocks = ctx->cfg.max_table_blocks;
 
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
-    plan_count_kernel<<<ctx->cfg.max_requests, PLAN_NT, 0, st>>>(a);
+    plan_count_kernel<<<ctx->cfg.max_requests * PLAN_PARTS, PLAN_NT, 0, st>>>(a);
     plan_scan_kernel<<<1, SCAN_NT, 0, st>>>(a);
-    plan_assign_kernel<<<ctx->cfg.max_requests, PLAN_NT, 0, st>>>(a);
-    plan_publish_kernel<<<1, 32, 0, st>>>(a);
+    plan_assign_kernel<<<ctx->cfg.max_requests * PLAN_PARTS, PLAN_NT, 0, st>>>(a);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

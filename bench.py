@@ -44,13 +44,15 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def committed_traffic(workload_name):
-    """DRAM bytes per moved token of the copy kernel from the committed ncu capture, or None."""
+def committed_traffic(token_bytes):
+    """DRAM bytes per moved token of the copy kernel from the committed ncu capture (taken at
+    one token size; traffic is one read and one write per moved row, so it scales with the
+    token's bytes), or None."""
     path = os.path.join(ROOT, "profiles", "copy_kernel_dram_traffic.json")
     try:
         with open(path) as f:
             d = json.load(f)
-        return d.get(workload_name) or d.get("default")
+        return d["default"] * token_bytes / d["per_token_bytes_basis"]
     except Exception:
         return None
 
@@ -351,7 +353,7 @@ def run_cuda(args):
     peak, peak_kind = measured_peak()
     copy_ms = float(np.mean(copy_each))
     achieved = bytes_per_step / (copy_ms * 1e-3) / 1e9
-    per_token = committed_traffic(w.name)
+    per_token = committed_traffic(w.token_bytes)
     roofline = {"bound": "hbm", "kernel": "copy_bulk_kernel" if grid["variant"] == 2 else "copy_rows_kernel",
                 "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,

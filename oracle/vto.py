@@ -48,6 +48,7 @@ def lib():
     if _lib is None:
         _lib = ctypes.CDLL(build())
         _lib.vto_gather_logical.restype = ctypes.c_int64
+        _lib.vto_build_slot_mapping.restype = ctypes.c_int64
         _lib.vto_waste_ratio.restype = ctypes.c_double
     return _lib
 
@@ -215,3 +216,62 @@ def waste_ratio(S, num_allocated_blocks, tt_slots, keep=None) -> float:
 
 def openmp_threads() -> int:
     return int(lib().vto_openmp_threads())
+
+
+# ---- token-table runtime ------------------------------------------------------------------
+def evict_tokens(tt_offsets, tt_len, keep: np.ndarray, victim_req, victim_tok) -> int:
+    """In place on ``keep`` (uint8).  Returns the number of skipped (out-of-range) victims."""
+    tt_offsets, tt_len = _i32(tt_offsets), _i32(tt_len)
+    victim_req, victim_tok = _i32(victim_req), _i32(victim_tok)
+    assert keep.dtype == np.uint8 and keep.flags["C_CONTIGUOUS"]
+    bad = ctypes.c_int32(0)
+    rc = lib().vto_evict_tokens(ctypes.c_int32(len(tt_len)), _p(tt_offsets, np.int32), _p(tt_len, np.int32),
+                                _p(keep, np.uint8), _p(victim_req, np.int32), _p(victim_tok, np.int32),
+                                ctypes.c_int32(len(victim_req)), ctypes.byref(bad))
+    if rc != 0:
+        raise ValueError(f"vto_evict_tokens failed: {rc}")
+    return bad.value
+
+
+def sync_new_tokens(S, tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, tt_len: np.ndarray,
+                    phys_len: np.ndarray, bt_offsets, bt_blocks, new_len) -> int:
+    """In place on tt_slots, keep, tt_len, phys_len.  Returns the number of requests that stopped early."""
+    tt_offsets, bt_offsets, bt_blocks, new_len = _i32(tt_offsets), _i32(bt_offsets), _i32(bt_blocks), _i32(new_len)
+    for a, d in ((tt_slots, np.int32), (keep, np.uint8), (tt_len, np.int32), (phys_len, np.int32)):
+        assert a.dtype == d and a.flags["C_CONTIGUOUS"]
+    bad = ctypes.c_int32(0)
+    rc = lib().vto_sync_new_tokens(ctypes.c_int32(len(tt_len)), ctypes.c_int32(S), _p(tt_offsets, np.int32),
+                                   _p(tt_slots, np.int32), _p(keep, np.uint8), _p(tt_len, np.int32),
+                                   _p(phys_len, np.int32), _p(bt_offsets, np.int32), _p(bt_blocks, np.int32),
+                                   _p(new_len, np.int32), ctypes.byref(bad))
+    if rc != 0:
+        raise ValueError(f"vto_sync_new_tokens failed: {rc}")
+    return bad.value
+
+
+def build_slot_mapping(tt_offsets, tt_slots, keep=None, select=None):
+    """Returns (slots, token_ids, offsets[R+1]) of the active tokens, request order then token id."""
+    tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
+    keep, select = _u8(keep), _u8(select)
+    R = len(tt_offsets) - 1
+    cap = max(1, len(tt_slots))
+    slots = np.full(cap, -7, np.int32)
+    ids = np.full(cap, -7, np.int32)
+    off = np.zeros(R + 1, np.int32)
+    n = lib().vto_build_slot_mapping(ctypes.c_int32(R), _p(tt_offsets, np.int32), _p(tt_slots, np.int32),
+                                     _p(keep, np.uint8), _p(select, np.uint8), _p(slots, np.int32),
+                                     _p(ids, np.int32), _p(off, np.int32), ctypes.c_int64(cap))
+    if n < 0:
+        raise ValueError(f"vto_build_slot_mapping failed: {n}")
+    return slots[:n].copy(), ids[:n].copy(), off
+
+
+def apply_moves(tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, phys_len, new_tt_slots, req_status) -> None:
+    """Commit of a repack, in place on tt_slots, keep and phys_len (phys_len may be None)."""
+    tt_offsets, new_tt_slots, req_status = _i32(tt_offsets), _i32(new_tt_slots), _i32(req_status)
+    assert tt_slots.dtype == np.int32 and keep.dtype == np.uint8
+    rc = lib().vto_apply_moves(ctypes.c_int32(len(tt_offsets) - 1), _p(tt_offsets, np.int32), _p(tt_slots, np.int32),
+                               _p(keep, np.uint8), None if phys_len is None else _p(phys_len, np.int32),
+                               _p(new_tt_slots, np.int32), _p(req_status, np.int32))
+    if rc != 0:
+        raise ValueError(f"vto_apply_moves failed: {rc}")

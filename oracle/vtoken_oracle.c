@@ -304,6 +304,84 @@ double vto_waste_ratio(int32_t S, int64_t num_allocated_blocks,
     return 1.0 - (double)live / ((double)num_allocated_blocks * (double)S);
 }
 
+int vto_evict_tokens(int32_t R, const int32_t *tt_offsets, const int32_t *tt_len, uint8_t *keep,
+                     const int32_t *victim_req, const int32_t *victim_tok, int32_t num_victims,
+                     int32_t *num_bad)
+{
+    if (R < 0 || num_victims < 0 || !tt_offsets || !tt_len || !keep) return VTO_EINVAL;
+    int32_t bad = 0;
+    for (int32_t i = 0; i < num_victims; ++i) {
+        const int32_t r = victim_req[i], t = victim_tok[i];
+        if (r < 0 || r >= R || t < 0 || t >= tt_len[r]) { ++bad; continue; }
+        keep[(int64_t)tt_offsets[r] + t] = 0;          /* logically inactive; the KV bytes stay (Sec. 3.2) */
+    }
+    if (num_bad) *num_bad = bad;
+    return VTO_OK;
+}
+
+int vto_sync_new_tokens(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                        int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
+                        const int32_t *bt_blocks, const int32_t *new_len, int32_t *num_bad)
+{
+    if (R < 0 || S < 1) return VTO_EINVAL;
+    int32_t bad = 0;
+    for (int32_t r = 0; r < R; ++r) {
+        const int32_t cap = tt_offsets[r + 1] - tt_offsets[r];
+        const int64_t room = (int64_t)(bt_offsets[r + 1] - bt_offsets[r]) * S;   /* slots in the block list */
+        int stopped = 0;
+        while (tt_len[r] < new_len[r]) {
+            const int32_t t = tt_len[r];                /* next sequential logical id */
+            const int64_t p = phys_len[r];              /* next position in the block list */
+            if (t >= cap || p >= room) { stopped = 1; break; }
+            const int32_t block = bt_blocks[bt_offsets[r] + p / S];
+            tt_slots[(int64_t)tt_offsets[r] + t] = block * S + (int32_t)(p % S);
+            keep[(int64_t)tt_offsets[r] + t] = 1;
+            tt_len[r] = t + 1;
+            phys_len[r] = (int32_t)(p + 1);
+        }
+        bad += stopped;
+    }
+    if (num_bad) *num_bad = bad;
+    return VTO_OK;
+}
+
+int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32_t *tt_slots,
+                               const uint8_t *keep, const uint8_t *select, int32_t *out_slots,
+                               int32_t *out_token_ids, int32_t *out_offsets, int64_t capacity)
+{
+    if (R < 0 || !tt_offsets || !tt_slots || !out_offsets) return VTO_EINVAL;
+    int64_t n = 0;
+    for (int32_t r = 0; r < R; ++r) {
+        out_offsets[r] = (int32_t)n;
+        if (select != NULL && select[r] == 0) continue;
+        for (int64_t t = tt_offsets[r]; t < tt_offsets[r + 1]; ++t) {
+            if (!is_live(tt_slots, keep, t)) continue;  /* evicted tokens are left out (Sec. 3.2) */
+            if (n >= capacity) return VTO_EINVAL;
+            if (out_slots) out_slots[n] = tt_slots[t];  /* the table already stores block * S + offset */
+            if (out_token_ids) out_token_ids[n] = (int32_t)(t - tt_offsets[r]);
+            ++n;
+        }
+    }
+    out_offsets[R] = (int32_t)n;
+    return n;
+}
+
+int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                    int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status)
+{
+    if (R < 0 || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTO_EINVAL;
+    for (int32_t r = 0; r < R; ++r) {
+        int32_t with_slot = 0;
+        for (int64_t t = tt_offsets[r]; t < tt_offsets[r + 1]; ++t) {
+            tt_slots[t] = new_tt_slots[t];              /* source entry cleared, destination written (I2) */
+            keep[t] = new_tt_slots[t] >= 0 ? 1 : 0;
+            with_slot += new_tt_slots[t] >= 0;
+        }
+        if (phys_len && req_status && req_status[r] == VTO_REPACKED) phys_len[r] = with_slot;
+    }
+    return VTO_OK;
+}
+
 int vto_openmp_threads(void)
 {
 #ifdef _OPENMP

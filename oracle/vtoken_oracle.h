@@ -109,6 +109,41 @@ int vto_check_semantics(int32_t R, int32_t S,
 double vto_waste_ratio(int32_t S, int64_t num_allocated_blocks,
                        const int32_t *tt_slots, const uint8_t *keep, int64_t T);
 
+/* ---- token-table runtime (Sec. 3.2 interfaces, Sec. 3.4 slot mapping) -------------------------
+ * The token table of request r occupies tt_slots[tt_offsets[r] .. tt_offsets[r+1]) -- that range
+ * is its CAPACITY; tt_len[r] entries are registered, the rest hold -1 / keep 0.  phys_len[r] is the
+ * number of slots already used in the request's block list (the append position). */
+
+/* evict_token for a batch: keep[tt_offsets[req] + tok] = 0.  A victim with req outside [0, R) or
+ * tok outside [0, tt_len[req]) is skipped and counted in *num_bad. */
+int vto_evict_tokens(int32_t R, const int32_t *tt_offsets, const int32_t *tt_len, uint8_t *keep,
+                     const int32_t *victim_req, const int32_t *victim_tok, int32_t num_victims,
+                     int32_t *num_bad);
+
+/* sync_new_tokens for a batch: request r grows from tt_len[r] to new_len[r] registered tokens (no
+ * change when new_len[r] <= tt_len[r]).  New tokens get sequential logical ids; the i-th new token
+ * sits at position p = phys_len[r] + i of the request's block list:
+ * slot = bt_blocks[bt_offsets[r] + p / S] * S + p % S, keep = 1.  A token beyond the table capacity
+ * or beyond the block list is not registered: the request stops growing there and is counted in
+ * *num_bad.  Updates tt_len and phys_len. */
+int vto_sync_new_tokens(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                        int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
+                        const int32_t *bt_blocks, const int32_t *new_len, int32_t *num_bad);
+
+/* Slot mapping of the active tokens (slot = token_table[token].block * S + offset, Sec. 3.4): for each
+ * selected request, in request order, the slots (and logical ids) of its tokens with slot >= 0 and
+ * keep != 0 (keep NULL: slot >= 0) in ascending token id.  out_offsets[R+1] = first entry of each
+ * request.  Returns the entry count or VTO_EINVAL when it exceeds capacity. */
+int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32_t *tt_slots,
+                               const uint8_t *keep, const uint8_t *select, int32_t *out_slots,
+                               int32_t *out_token_ids, int32_t *out_offsets, int64_t capacity);
+
+/* apply_moves / commit of a repack: every entry takes its new slot, liveness follows it (an entry
+ * without a slot is dead), and a repacked request appends after its n live tokens from now on:
+ * phys_len[r] = number of entries with a slot, for requests with status VTO_REPACKED. */
+int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                    int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status);
+
 int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */
 
 #ifdef __cplusplus

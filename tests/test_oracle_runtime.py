@@ -1,0 +1,120 @@
+"""Pins of the oracle's token-table runtime (evict_token, sync_new_tokens, slot mapping,
+apply_moves) against library routines, closed forms and a dictionary-based simulation of a
+serving loop (no GPU)."""
+import numpy as np
+import pytest
+
+from oracle import vto
+
+from runtime_sim import DictCache, ServingState, random_serving_steps
+
+
+def test_slot_mapping_reduces_to_the_direct_formula_without_eviction():
+    """No eviction, no relocation: the token-table lookup equals the direct computation
+    slot = block_id * block_size + offset over the block table (Sec. 3.4)."""
+    S = 16
+    bt = np.array([7, 3, 11, 5], np.int32)
+    n = 55
+    st = ServingState.empty(S, capacities=[64], block_lists=[bt])
+    assert vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len,
+                               st.bt_offsets, st.bt_blocks, [n]) == 0
+    slots, ids, off = vto.build_slot_mapping(st.tt_offsets, st.tt_slots, st.keep)
+    pos = np.arange(n)
+    assert np.array_equal(slots, bt[pos // S] * S + pos % S)
+    assert np.array_equal(ids, pos) and off.tolist() == [0, n]
+    assert st.tt_len.tolist() == [n] and st.phys_len.tolist() == [n]
+    assert (st.tt_slots[n:] == -1).all() and (st.keep[n:] == 0).all()
+
+
+def test_slot_mapping_is_numpy_boolean_selection():
+    rng = np.random.default_rng(0)
+    lens = [40, 0, 77, 5]
+    off = np.concatenate([[0], np.cumsum(lens)]).astype(np.int32)
+    tt = rng.permutation(400)[:off[-1]].astype(np.int32)
+    tt[rng.random(off[-1]) < 0.2] = -1
+    keep = (rng.random(off[-1]) < 0.6).astype(np.uint8)
+    sel = np.array([1, 1, 0, 1], np.uint8)
+    slots, ids, o = vto.build_slot_mapping(off, tt, keep, sel)
+    live = (tt >= 0) & (keep != 0)
+    exp_s, exp_i, exp_o = [], [], [0]
+    for r in range(4):
+        m = live[off[r]:off[r + 1]] if sel[r] else np.zeros(lens[r], bool)
+        exp_s.append(tt[off[r]:off[r + 1]][m])
+        exp_i.append(np.flatnonzero(m))
+        exp_o.append(exp_o[-1] + int(m.sum()))
+    assert np.array_equal(slots, np.concatenate(exp_s)) and np.array_equal(ids, np.concatenate(exp_i))
+    assert o.tolist() == exp_o
+
+
+def test_evict_is_a_scatter_of_zeros_and_skips_bad_victims():
+    off = np.array([0, 10, 30], np.int32)
+    tt_len = np.array([10, 12], np.int32)
+    keep = np.ones(30, np.uint8)
+    bad = vto.evict_tokens(off, tt_len, keep, [0, 1, 1, 0, 2, 1, -1], [3, 0, 11, 10, 0, 12, 0])
+    exp = np.ones(30, np.uint8)
+    exp[[3, 10, 21]] = 0
+    assert np.array_equal(keep, exp)
+    assert bad == 4          # token 10 of request 0, request 2, token 12 of request 1, request -1
+
+
+def test_sync_appends_in_batches_and_stops_at_capacity_or_block_list():
+    S = 4
+    st = ServingState.empty(S, capacities=[10, 6], block_lists=[np.array([2, 9], np.int32), np.array([5], np.int32)])
+    assert vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len,
+                               st.bt_offsets, st.bt_blocks, [3, 2]) == 0
+    assert vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len,
+                               st.bt_offsets, st.bt_blocks, [7, 2]) == 0       # request 1 unchanged
+    assert st.tt_slots[:7].tolist() == [8, 9, 10, 11, 36, 37, 38]
+    assert st.tt_slots[10:12].tolist() == [20, 21]
+    # request 0 asks for 12 tokens but its block list holds 8 and its table 10; request 1 for 6 with one block
+    bad = vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len,
+                              st.bt_offsets, st.bt_blocks, [12, 6])
+    assert bad == 2
+    assert st.tt_len.tolist() == [8, 4] and st.phys_len.tolist() == [8, 4]
+    assert st.tt_slots[7] == 39 and st.tt_slots[8:10].tolist() == [-1, -1]
+
+
+def test_apply_moves_commits_slots_liveness_and_append_position():
+    S = 4
+    st = ServingState.empty(S, capacities=[12], block_lists=[np.array([0, 1, 2], np.int32)])
+    vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets,
+                        st.bt_blocks, [10])
+    vto.evict_tokens(st.tt_offsets, st.tt_len, st.keep, [0] * 7, [0, 2, 3, 5, 6, 7, 9])
+    p = vto.plan(S, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep, np.array([6, 7], np.int32))
+    assert p.req_status.tolist() == [vto.REPACKED] and p.num_moves == 3
+    vto.apply_moves(st.tt_offsets, st.tt_slots, st.keep, st.phys_len, p.new_tt_slots, p.req_status)
+    assert st.tt_slots[:10].tolist() == [-1, 24, -1, -1, 25, -1, -1, -1, 26, -1]
+    assert st.keep[:10].tolist() == [0, 1, 0, 0, 1, 0, 0, 0, 1, 0]
+    assert st.phys_len.tolist() == [3]
+    # the request now owns block 6 only; the next token lands right behind the three survivors
+    st.set_block_lists([p.new_bt_blocks])
+    vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets,
+                        st.bt_blocks, [11])
+    assert st.tt_slots[10] == 27 and st.tt_len.tolist() == [11] and st.phys_len.tolist() == [4]
+
+
+@pytest.mark.parametrize("seed,S", [(0, 4), (1, 16), (2, 3)])
+def test_serving_loop_against_a_dictionary_cache(seed, S):
+    """Several decode steps of append -> evict -> slot mapping -> (sometimes) repack + commit on
+    the oracle, mirrored by a cache that is just a dict {(request, token id): payload}.  After
+    every step the oracle's logical view (slot mapping into the pool) must return exactly the
+    payloads the dictionary holds, in token order (token conservation, unique mapping)."""
+    rng = np.random.default_rng(seed)
+    R = 5
+    st = ServingState.random(rng, S, R, capacity=200, num_blocks=400)
+    truth = DictCache()
+    pool = np.zeros((st.num_blocks * S, 2), np.int64)      # one "layer": payload = (request, token id)
+    for step in random_serving_steps(rng, st, steps=25):
+        step.run_on_oracle(st, pool, truth)
+        slots, ids, off = vto.build_slot_mapping(st.tt_offsets, st.tt_slots, st.keep)
+        assert len(np.unique(slots)) == len(slots)                       # unique mapping
+        for r in range(R):
+            want = truth.live_tokens(r)
+            got_ids = ids[off[r]:off[r + 1]].tolist()
+            assert got_ids == want
+            assert pool[slots[off[r]:off[r + 1]]].tolist() == [[r, t] for t in want]
+        # blocks in use are exactly what the block lists say, and nothing is both free and used
+        used = set(st.bt_blocks.tolist())
+        assert len(used) == len(st.bt_blocks) and not (used & set(st.free))
+        live_blocks = set((slots // S).tolist())
+        assert live_blocks <= used

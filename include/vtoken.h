@@ -77,7 +77,9 @@ enum {
     VTOKEN_FLAG_BAD_FREE = 4u,        /* a free-list id outside [0, num_blocks): that destination block is skipped */
     VTOKEN_FLAG_CAPACITY = 8u,        /* R, T or the block total above the create-time capacities: clamped */
     VTOKEN_FLAG_TIMEOUT = 16u,        /* a bounded wait inside a kernel ran out; rows may be missing */
-    VTOKEN_FLAG_GATHER_OVERFLOW = 32u /* vtoken_gather_logical: more live tokens than out_capacity_tokens */
+    VTOKEN_FLAG_GATHER_OVERFLOW = 32u,/* gather_logical / build_slot_mapping: more live tokens than the output holds */
+    VTOKEN_FLAG_BAD_VICTIM = 64u,     /* vtoken_evict_tokens: a victim outside its request's registered tokens: skipped */
+    VTOKEN_FLAG_APPEND_STOPPED = 128u /* vtoken_sync_new_tokens: table capacity or block list exhausted: request grew less */
 };
 
 typedef struct {
@@ -168,6 +170,55 @@ int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const in
 /* Copies the context's counts of the last plan (with the flags raised by repack and
  * gather_logical since) to HOST memory.  Synchronises the stream: the only call that does. */
 int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stream);
+
+/* ---- Token-table runtime on the device (Sec. 3.2 interfaces, Sec. 3.4 slot mapping) ----------
+ * For callers that keep the token tables resident on the GPU between decode steps.  Layout: the
+ * table of request r occupies tt_slots / keep [tt_offsets[r] .. tt_offsets[r+1]) -- that range is
+ * its CAPACITY; tt_len[r] entries are registered and the rest hold slot -1 / keep 0, which
+ * vtoken_plan, vtoken_gather_logical and vtoken_build_slot_mapping treat as not live, so the same
+ * buffers feed them unchanged.  phys_len[r] = slots already used in the request's block list
+ * (where the next token is written).  All pointers DEVICE; every call only enqueues kernels on
+ * the stream (capturable); problems found on the device raise VTOKEN_FLAG_* bits in the context's
+ * counts (vtoken_read_counts). */
+
+/* evict_token (Sec. 3.2) for a batch: keep[tt_offsets[req] + tok] = 0 for the first *num_victims
+ * (device scalar, <= max_victims) pairs.  Metadata only: no KV byte moves, the slot stays until
+ * a repack.  A victim outside [0, R) x [0, tt_len[req]) is skipped (VTOKEN_FLAG_BAD_VICTIM). */
+int vtoken_evict_tokens(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max_victims,
+                        const int32_t *victim_req, const int32_t *victim_tok, const int32_t *num_requests,
+                        const int32_t *tt_offsets, const int32_t *tt_len, uint8_t *keep, void *cuda_stream);
+
+/* sync_new_tokens (Sec. 3.2) for a batch: request r grows from tt_len[r] to new_len[r] registered
+ * tokens (unchanged when new_len[r] <= tt_len[r]).  New tokens get sequential logical ids; the
+ * i-th new one sits at position p = phys_len[r] + i of the block list bt_blocks[bt_offsets[r] ..):
+ * slot = block[p / S] * S + p % S, keep = 1.  Growth stops at the table capacity or at the end of
+ * the block list (VTOKEN_FLAG_APPEND_STOPPED).  Updates tt_len and phys_len. */
+int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                           int32_t *tt_slots, uint8_t *keep, int32_t *tt_len, int32_t *phys_len,
+                           const int32_t *bt_offsets, const int32_t *bt_blocks, const int32_t *new_len,
+                           void *cuda_stream);
+
+/* Slot mapping (Sec. 3.4: slot = token_table[token].block_id * S + offset, looked up once per token
+ * at input preparation): the slots of the active tokens (slot >= 0, and keep != 0 when keep is
+ * given) of the selected requests, request order then token-id order, written densely to
+ * out_slots[out_capacity]; out_token_ids (may be NULL) receives their logical ids; out_offsets[R+1]
+ * the first entry of each request.  Entries beyond out_capacity are dropped
+ * (VTOKEN_FLAG_GATHER_OVERFLOW).  The buffers are stable, only their contents change between
+ * calls -- the property the paper relies on for CUDA-Graph replay.  Shares the context scratch of
+ * vtoken_gather_logical. */
+int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                              const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                              int32_t *out_slots, int32_t *out_token_ids, int64_t out_capacity,
+                              int32_t *out_offsets, void *cuda_stream);
+
+/* apply_moves (Sec. 3.2; invariant I2): commit of a plan after its repack event.  Every entry takes
+ * its slot from new_tt_slots (the source entry is cleared by the same write), keep becomes
+ * (slot >= 0), and for requests with status VTOKEN_REPACKED phys_len[r] becomes the number of
+ * entries that still own a slot (new tokens append behind the packed survivors).  phys_len may be
+ * NULL.  The block tables are the caller's: it adopts new_bt_* and returns freed blocks itself. */
+int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                       int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
+                       const int32_t *req_status, void *cuda_stream);
 
 /* Host-table front end.  The paper keeps the canonical token table on the CPU (Sec. 3.2);
  * this entry point serves such a caller: all tables are HOST memory (pinned for speed), the

@@ -15,10 +15,12 @@ LIB_PATH = os.path.join(_PKG, "libvtoken.so")
 OK, EINVAL, ECAPACITY, ECUDA, ENOMEM, ESTATE = 0, -1, -2, -3, -4, -5
 NOT_SELECTED, REPACKED, NO_GAIN, DEFERRED_NO_FREE = 0, 1, 2, 3
 FLAG_BAD_SLOT, FLAG_BAD_BLOCK, FLAG_BAD_FREE, FLAG_CAPACITY, FLAG_TIMEOUT, FLAG_GATHER_OVERFLOW = 1, 2, 4, 8, 16, 32
+FLAG_BAD_VICTIM, FLAG_APPEND_STOPPED = 64, 128
 
 SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "vtoken_gather_logical",
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
-           "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc"]
+           "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
+           "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves"]
 
 
 class VtokenError(RuntimeError):
@@ -107,6 +109,10 @@ def load():
              ctypes.c_int64, ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
             [ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p,
              ctypes.c_void_p, ctypes.c_void_p])
+        lib.vtoken_evict_tokens.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 7
+        lib.vtoken_sync_new_tokens.argtypes = [ctypes.c_void_p] * 11
+        lib.vtoken_build_slot_mapping.argtypes = [ctypes.c_void_p] * 8 + [ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
+        lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 9
         _lib = lib
     return _lib
 
@@ -224,3 +230,32 @@ def vtoken_gather_logical_noalloc(*, k_pool, v_pool, num_layers, num_blocks, blo
         _ptr(num_requests), max_requests, _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep), _ptr(select), layer_begin,
         layer_end, _ptr(out_k), _ptr(out_v), out_capacity_tokens, _ptr(out_offsets), _ptr(error_flags),
         _stream(stream)), "vtoken_gather_logical_noalloc")
+
+
+# ---- token-table runtime ------------------------------------------------------------------
+def vtoken_evict_tokens(ctx, *, num_victims, max_victims, victim_req, victim_tok, num_requests, tt_offsets, tt_len,
+                        keep, stream=None) -> None:
+    _check(load().vtoken_evict_tokens(ctx, _ptr(num_victims), max_victims, _ptr(victim_req), _ptr(victim_tok),
+                                      _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_len), _ptr(keep),
+                                      _stream(stream)), "vtoken_evict_tokens", ctx)
+
+
+def vtoken_sync_new_tokens(ctx, *, num_requests, tt_offsets, tt_slots, keep, tt_len, phys_len, bt_offsets, bt_blocks,
+                           new_len, stream=None) -> None:
+    _check(load().vtoken_sync_new_tokens(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                                         _ptr(tt_len), _ptr(phys_len), _ptr(bt_offsets), _ptr(bt_blocks),
+                                         _ptr(new_len), _stream(stream)), "vtoken_sync_new_tokens", ctx)
+
+
+def vtoken_build_slot_mapping(ctx, *, num_requests, tt_offsets, tt_slots, keep, select, out_slots, out_token_ids,
+                              out_capacity, out_offsets, stream=None) -> None:
+    _check(load().vtoken_build_slot_mapping(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                                            _ptr(select), _ptr(out_slots), _ptr(out_token_ids), out_capacity,
+                                            _ptr(out_offsets), _stream(stream)), "vtoken_build_slot_mapping", ctx)
+
+
+def vtoken_apply_moves(ctx, *, num_requests, tt_offsets, tt_slots, keep, phys_len, new_tt_slots, req_status,
+                       stream=None) -> None:
+    _check(load().vtoken_apply_moves(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                                     _ptr(phys_len), _ptr(new_tt_slots), _ptr(req_status), _stream(stream)),
+           "vtoken_apply_moves", ctx)

@@ -12,7 +12,7 @@ constexpr int G_NT = 512;
 struct GatherArgs {
     const int32_t *num_requests, *tt_offsets, *tt_slots;
     const uint8_t *keep, *select;
-    int32_t *req_n, *out_offsets, *g_src, *g_total;
+    int32_t *req_n, *out_offsets, *g_src, *g_ids, *g_total;   // g_ids: logical id of each output row, or NULL
     vtoken_counts *counts;
     const uint8_t *k_pool, *v_pool;
     uint8_t *out_k, *out_v;
@@ -110,7 +110,10 @@ __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
         int total;
         const int i = carry + vtk_block_rank<G_NT>(live, warp_sums, total);
         carry += total;
-        if (live && i < cap) a.g_src[i] = slot;
+        if (live && i < cap) {
+            a.g_src[i] = slot;
+            if (a.g_ids != nullptr) a.g_ids[i] = (int32_t)(t - t0);
+        }
     }
 }
 
@@ -174,6 +177,7 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.req_n = ctx->req_n;
     a.out_offsets = out_offsets;
     a.g_src = ctx->g_src;
+    a.g_ids = nullptr;
     a.g_total = ctx->g_total;
     a.counts = ctx->counts;
     a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
@@ -192,6 +196,44 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     gather_scan_kernel<<<1, 1024, 0, st>>>(a);
     gather_assign_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
     gather_copy_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+// Slot mapping (Sec. 3.4): the same count / scan / assign, with the slot list written straight
+// into the caller's buffer and no row copy.
+extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                                         const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                                         int32_t *out_slots, int32_t *out_token_ids, int64_t out_capacity,
+                                         int32_t *out_offsets, void *cuda_stream)
+{
+    if (!ctx || !num_requests || !tt_offsets || !tt_slots || !out_slots || !out_offsets) return VTOKEN_EINVAL;
+    if (out_capacity < 0) return VTOKEN_EINVAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    GatherArgs a;
+    a.num_requests = num_requests;
+    a.tt_offsets = tt_offsets;
+    a.tt_slots = tt_slots;
+    a.keep = keep;
+    a.select = select;
+    a.req_n = ctx->req_n;
+    a.out_offsets = out_offsets;
+    a.g_src = out_slots;
+    a.g_ids = out_token_ids;
+    a.g_total = ctx->g_total;
+    a.counts = ctx->counts;
+    a.k_pool = a.v_pool = nullptr;
+    a.out_k = a.out_v = nullptr;
+    a.layer_stride = 0;
+    a.row_bytes = 0;
+    a.slots_per_layer = ctx->slots_per_layer;
+    a.out_capacity = out_capacity;
+    a.max_tokens = out_capacity;
+    a.layer_begin = a.layer_end = 0;
+    a.max_requests = ctx->cfg.max_requests;
+    gather_count_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_scan_kernel<<<1, 1024, 0, st>>>(a);
+    gather_assign_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

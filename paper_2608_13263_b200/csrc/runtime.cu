@@ -1,0 +1,154 @@
+// Device-side token-table runtime: the interfaces of the token table (Sec. 3.2 of the paper:
+// evict_token, sync_new_tokens, apply_moves) as batch kernels over device-resident tables.
+// The slot-mapping build (Sec. 3.4) lives with the logical gather, whose planner it shares.
+//
+// A request's token table occupies tt_slots[tt_offsets[r] .. tt_offsets[r+1]) -- its capacity;
+// tt_len[r] entries are registered, the rest hold -1 / keep 0, which every other kernel of the
+// library already treats as "not live".  phys_len[r] is the append position in its block list.
+#include "common.cuh"
+
+namespace {
+
+constexpr int RT_NT = 256;
+
+__device__ __forceinline__ int rt_requests(const int32_t *num_requests, int max_requests)
+{
+    int R = *num_requests;
+    return R < 0 ? 0 : (R > max_requests ? max_requests : R);
+}
+
+// evict_token over a batch of victims: metadata only, the KV bytes stay where they are
+__global__ void __launch_bounds__(RT_NT) evict_kernel(const int32_t *num_victims, int32_t max_victims,
+                                                      const int32_t *victim_req, const int32_t *victim_tok,
+                                                      const int32_t *num_requests, int32_t max_requests,
+                                                      const int32_t *tt_offsets, const int32_t *tt_len,
+                                                      uint8_t *keep, vtoken_counts *counts)
+{
+    int n = *num_victims;
+    n = n < 0 ? 0 : (n > max_victims ? max_victims : n);
+    const int R = rt_requests(num_requests, max_requests);
+    bool bad = false;
+    for (int i = blockIdx.x * RT_NT + threadIdx.x; i < n; i += gridDim.x * RT_NT) {
+        const int r = victim_req[i], t = victim_tok[i];
+        if (r < 0 || r >= R || t < 0 || t >= tt_len[r]) { bad = true; continue; }
+        keep[(int64_t)tt_offsets[r] + t] = 0;
+    }
+    if (bad || (threadIdx.x == 0 && blockIdx.x == 0 && *num_victims > max_victims))
+        atomicOr(&counts->error_flags, VTOKEN_FLAG_BAD_VICTIM);
+}
+
+// sync_new_tokens: one CTA per request; the tokens it can register are a prefix of the ones asked
+// for (table capacity and block-list room only shrink it), so the count has a closed form.
+__global__ void __launch_bounds__(RT_NT) sync_kernel(const int32_t *num_requests, int32_t max_requests, int32_t S,
+                                                     const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                                                     int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
+                                                     const int32_t *bt_blocks, const int32_t *new_len,
+                                                     int32_t num_blocks, vtoken_counts *counts)
+{
+    const int r = blockIdx.x;
+    if (r >= rt_requests(num_requests, max_requests)) return;
+    const int64_t base = tt_offsets[r];
+    const int cap = tt_offsets[r + 1] - tt_offsets[r];
+    const int len = tt_len[r], phys = phys_len[r];
+    const int b0 = bt_offsets[r];
+    const long long room = (long long)(bt_offsets[r + 1] - b0) * S;
+    const int want = new_len[r] - len;
+    if (want <= 0) return;
+    long long can = want;
+    if (can > cap - len) can = cap - len;
+    if (can > room - phys) can = room - phys;
+    if (can < 0) can = 0;
+    uint32_t flags = can < want ? VTOKEN_FLAG_APPEND_STOPPED : 0u;
+    for (int i = threadIdx.x; i < (int)can; i += RT_NT) {
+        const int p = phys + i;                              // position in the block list
+        const int blk = bt_blocks[b0 + p / S];
+        if (blk < 0 || blk >= num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
+        tt_slots[base + len + i] = blk * S + p % S;          // slot = block_id * S + offset
+        keep[base + len + i] = 1;
+    }
+    __syncthreads();     // every thread has read tt_len / phys_len before they change
+    if (threadIdx.x == 0) {
+        tt_len[r] = len + (int)can;
+        phys_len[r] = phys + (int)can;
+    }
+    if (flags) atomicOr(&counts->error_flags, flags);
+}
+
+// apply_moves: commit of a repack.  Entries take their new slot, liveness follows the slot, a
+// repacked request appends behind its surviving tokens from now on.
+__global__ void __launch_bounds__(RT_NT) apply_moves_kernel(const int32_t *num_requests, int32_t max_requests,
+                                                            const int32_t *tt_offsets, int32_t *tt_slots,
+                                                            uint8_t *keep, int32_t *phys_len,
+                                                            const int32_t *new_tt_slots, const int32_t *req_status)
+{
+    const int r = blockIdx.x;
+    if (r >= rt_requests(num_requests, max_requests)) return;
+    const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
+    int n = 0;
+    for (int64_t t = t0 + threadIdx.x; t < t1; t += RT_NT) {
+        const int32_t s = new_tt_slots[t];
+        tt_slots[t] = s;
+        keep[t] = s >= 0 ? 1 : 0;
+        n += s >= 0;
+    }
+    __shared__ int warp_n[RT_NT / 32];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+    if (vtk_lane() == 0) warp_n[threadIdx.x >> 5] = n;
+    __syncthreads();
+    if (threadIdx.x == 0 && phys_len != nullptr && req_status != nullptr && req_status[r] == VTOKEN_REPACKED) {
+        int s = 0;
+        for (int w = 0; w < RT_NT / 32; ++w) s += warp_n[w];
+        phys_len[r] = s;
+    }
+}
+
+}  // namespace
+
+extern "C" {
+
+int vtoken_evict_tokens(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max_victims,
+                        const int32_t *victim_req, const int32_t *victim_tok, const int32_t *num_requests,
+                        const int32_t *tt_offsets, const int32_t *tt_len, uint8_t *keep, void *cuda_stream)
+{
+    if (!ctx || !num_victims || !victim_req || !victim_tok || !num_requests || !tt_offsets || !tt_len || !keep)
+        return VTOKEN_EINVAL;
+    if (max_victims < 0) return VTOKEN_EINVAL;
+    if (max_victims == 0) return VTOKEN_OK;
+    int grid = (max_victims + RT_NT - 1) / RT_NT;
+    if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
+    evict_kernel<<<grid, RT_NT, 0, (cudaStream_t)cuda_stream>>>(num_victims, max_victims, victim_req, victim_tok,
+                                                                 num_requests, ctx->cfg.max_requests, tt_offsets,
+                                                                 tt_len, keep, ctx->counts);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                           int32_t *tt_slots, uint8_t *keep, int32_t *tt_len, int32_t *phys_len,
+                           const int32_t *bt_offsets, const int32_t *bt_blocks, const int32_t *new_len,
+                           void *cuda_stream)
+{
+    if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !tt_len || !phys_len || !bt_offsets ||
+        !bt_blocks || !new_len)
+        return VTOKEN_EINVAL;
+    sync_kernel<<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
+        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, tt_len, phys_len,
+        bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks, ctx->counts);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                       int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
+                       const int32_t *req_status, void *cuda_stream)
+{
+    if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTOKEN_EINVAL;
+    if (phys_len && !req_status) return VTOKEN_EINVAL;
+    apply_moves_kernel<<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
+        num_requests, ctx->cfg.max_requests, tt_offsets, tt_slots, keep, phys_len, new_tt_slots, req_status);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,265 @@
+"""GPU parity of the device-side token-table runtime (evict, append, slot mapping, commit) and of
+the whole serving loop around the repack: the same seeded step sequence runs on the oracle and
+through the C ABI; after every step all table state, the slot mapping and the logical K/V view
+must be identical."""
+import numpy as np
+import pytest
+
+from oracle import vto
+from paper_2608_13263_b200 import binding as vt
+
+from runtime_sim import Append, DictCache, Evict, Repack, ServingState, random_serving_steps
+
+pytestmark = pytest.mark.gpu
+
+
+class DeviceServing:
+    """Device copy of a ServingState plus small K/V pools whose rows carry (request, token)."""
+
+    def __init__(self, st, layers=2, row_elems=8, max_victims=64):
+        import torch
+        self.torch = torch
+        dev = torch.device("cuda:0")
+        self.dev = dev
+        self.S, self.NB, self.R = st.S, st.num_blocks, st.R
+        self.row_elems = row_elems
+        self.layers = layers
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.num_requests = torch.tensor([st.R], **i32)
+        self.tt_offsets = torch.from_numpy(st.tt_offsets).to(dev)
+        cap = int(st.tt_offsets[-1])
+        self.cap = cap
+        self.tt_slots = torch.from_numpy(st.tt_slots.copy()).to(dev)
+        self.keep = torch.from_numpy(st.keep.copy()).to(dev)
+        self.tt_len = torch.from_numpy(st.tt_len.copy()).to(dev)
+        self.phys_len = torch.from_numpy(st.phys_len.copy()).to(dev)
+        self.bt_offsets = torch.zeros(st.R + 1, **i32)
+        self.bt_blocks = torch.zeros(self.NB, **i32)
+        self.free_blocks = torch.zeros(self.NB, **i32)
+        self.num_free = torch.zeros(1, **i32)
+        self.new_len = torch.zeros(st.R, **i32)
+        self.max_victims = max_victims
+        self.victim_req = torch.zeros(max_victims, **i32)
+        self.victim_tok = torch.zeros(max_victims, **i32)
+        self.num_victims = torch.zeros(1, **i32)
+        self.new_bt_offsets = torch.zeros(st.R + 1, **i32)
+        self.new_bt_blocks = torch.zeros(self.NB, **i32)
+        self.new_tt_slots = torch.zeros(cap, **i32)
+        self.freed_blocks = torch.zeros(self.NB, **i32)
+        self.req_status = torch.zeros(st.R, **i32)
+        self.counts = torch.zeros(8, **i32)
+        self.map_slots = torch.zeros(cap, **i32)
+        self.map_ids = torch.zeros(cap, **i32)
+        self.map_offsets = torch.zeros(st.R + 1, **i32)
+        self.k_pool = torch.zeros((layers, self.NB * self.S, row_elems), dtype=torch.int16, device=dev)
+        self.v_pool = torch.zeros_like(self.k_pool)
+        self.ctx = vt.vtoken_create(layers, self.NB, self.S, 1, row_elems, self.k_pool, self.v_pool, st.R, cap,
+                                    self.NB, self.NB)
+
+    def upload_blocks(self, st):
+        t = self.torch
+        self.bt_offsets.copy_(t.from_numpy(st.bt_offsets))
+        b = st.bt_blocks
+        self.bt_blocks[:len(b)].copy_(t.from_numpy(b))
+
+    @staticmethod
+    def payload(r, t, layer, kv, row_elems):
+        base = np.array([r, t & 0x7FFF, t >> 15, layer, kv, r ^ t & 0xFF, 7, -3], np.int16)
+        return np.resize(base, row_elems)
+
+    # ---- the three steps through the C ABI ------------------------------------------------
+    def append(self, st_before_len, st, new_len):
+        t = self.torch
+        self.upload_blocks(st)                                  # scheduler grew the block lists on the host
+        self.new_len.copy_(t.from_numpy(np.asarray(new_len, np.int32)))
+        vt.vtoken_sync_new_tokens(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
+                                  tt_slots=self.tt_slots, keep=self.keep, tt_len=self.tt_len,
+                                  phys_len=self.phys_len, bt_offsets=self.bt_offsets, bt_blocks=self.bt_blocks,
+                                  new_len=self.new_len)
+        # "the model" writes the K/V of the new tokens at the slots the runtime assigned
+        slots = self.tt_slots.cpu().numpy()
+        lens = self.tt_len.cpu().numpy()
+        for r in range(self.R):
+            for tok in range(int(st_before_len[r]), int(lens[r])):
+                s = int(slots[st.tt_offsets[r] + tok])
+                for l in range(self.layers):
+                    self.k_pool[l, s] = t.from_numpy(self.payload(r, tok, l, 0, self.row_elems)).to(self.dev)
+                    self.v_pool[l, s] = t.from_numpy(self.payload(r, tok, l, 1, self.row_elems)).to(self.dev)
+
+    def evict(self, victim_req, victim_tok):
+        t = self.torch
+        n = len(victim_req)
+        assert n <= self.max_victims
+        self.victim_req[:n].copy_(t.from_numpy(victim_req))
+        self.victim_tok[:n].copy_(t.from_numpy(victim_tok))
+        self.num_victims.fill_(n)
+        vt.vtoken_evict_tokens(self.ctx, num_victims=self.num_victims, max_victims=self.max_victims,
+                               victim_req=self.victim_req, victim_tok=self.victim_tok,
+                               num_requests=self.num_requests, tt_offsets=self.tt_offsets, tt_len=self.tt_len,
+                               keep=self.keep)
+
+    def repack(self, st, free, nf, thr):
+        t = self.torch
+        self.upload_blocks(st)
+        self.free_blocks[:len(free)].copy_(t.from_numpy(np.asarray(free, np.int32)))
+        self.num_free.fill_(nf)
+        side = t.cuda.Stream()
+        side.wait_stream(t.cuda.current_stream())
+        vt.vtoken_plan(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets, bt_blocks=self.bt_blocks,
+                       tt_offsets=self.tt_offsets, tt_slots=self.tt_slots, keep=self.keep,
+                       free_blocks=self.free_blocks, num_free=self.num_free, new_bt_offsets=self.new_bt_offsets,
+                       new_bt_blocks=self.new_bt_blocks, new_tt_slots=self.new_tt_slots,
+                       freed_blocks=self.freed_blocks, req_status=self.req_status, counts=self.counts,
+                       thr_num=thr[0], thr_den=thr[1], stream=side)
+        vt.vtoken_repack(self.ctx, stream=side)
+        done = t.cuda.Event()
+        done.record(side)
+        t.cuda.current_stream().wait_event(done)                # commit only behind the repack event
+        vt.vtoken_apply_moves(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
+                              tt_slots=self.tt_slots, keep=self.keep, phys_len=self.phys_len,
+                              new_tt_slots=self.new_tt_slots, req_status=self.req_status)
+
+    def slot_mapping(self):
+        vt.vtoken_build_slot_mapping(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
+                                     tt_slots=self.tt_slots, keep=self.keep, select=None, out_slots=self.map_slots,
+                                     out_token_ids=self.map_ids, out_capacity=self.cap, out_offsets=self.map_offsets)
+        off = self.map_offsets.cpu().numpy()
+        n = int(off[self.R])
+        return self.map_slots.cpu().numpy()[:n], self.map_ids.cpu().numpy()[:n], off
+
+    def close(self):
+        self.torch.cuda.synchronize()
+        vt.vtoken_destroy(self.ctx)
+
+
+@pytest.mark.parametrize("seed,S", [(0, 4), (1, 16), (2, 3)])
+def test_serving_loop_matches_oracle_step_by_step(seed, S):
+    import torch
+    rng = np.random.default_rng(seed)
+    R = 5
+    st = ServingState.random(rng, S, R, capacity=200, num_blocks=400)
+    truth = DictCache()
+    dev = DeviceServing(st)
+    repacked_something = False
+    for step in random_serving_steps(rng, st, steps=25):
+        if isinstance(step, Append):
+            before = st.tt_len.copy()
+            step.run_on_oracle(st, None, truth)
+            dev.append(before, st, step.new_len)
+        elif isinstance(step, Evict):
+            step.run_on_oracle(st, None, truth)
+            dev.evict(step.victim_req, step.victim_tok)
+        else:
+            free = list(st.free)
+            nf = len(free) if step.num_free_limit < 0 else min(len(free), step.num_free_limit)
+            blocks_before = st.bt_blocks.copy()
+            st_before = ServingState(st.S, st.num_blocks, st.tt_offsets, st.tt_slots.copy(), st.keep.copy(),
+                                     st.tt_len.copy(), st.phys_len.copy(), [b.copy() for b in st.block_lists], free)
+            step.run_on_oracle(st, None, truth)
+            dev.repack(st_before, free, nf, step.thr)
+            p = step.last_plan
+            repacked_something |= p.num_moves > 0
+            c = dev.counts.cpu().numpy()
+            assert c[:6].tolist() == [p.num_moves, p.num_dst_blocks, p.num_freed, p.num_free_consumed,
+                                      p.num_admitted, p.num_deferred] and c[6] == 0
+            assert np.array_equal(dev.req_status.cpu().numpy(), p.req_status)
+            assert np.array_equal(dev.new_bt_offsets.cpu().numpy(), p.new_bt_offsets)
+            assert np.array_equal(dev.new_bt_blocks.cpu().numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
+            assert np.array_equal(dev.freed_blocks.cpu().numpy()[:p.num_freed], p.freed_blocks)
+            assert len(blocks_before) >= len(p.new_bt_blocks)
+        torch.cuda.synchronize()
+        # table state
+        assert np.array_equal(dev.tt_slots.cpu().numpy(), st.tt_slots)
+        assert np.array_equal(dev.keep.cpu().numpy(), st.keep)
+        assert np.array_equal(dev.tt_len.cpu().numpy(), st.tt_len)
+        assert np.array_equal(dev.phys_len.cpu().numpy(), st.phys_len)
+        # slot mapping
+        g_slots, g_ids, g_off = dev.slot_mapping()
+        o_slots, o_ids, o_off = vto.build_slot_mapping(st.tt_offsets, st.tt_slots, st.keep)
+        assert np.array_equal(g_slots, o_slots) and np.array_equal(g_ids, o_ids) and np.array_equal(g_off, o_off)
+        # logical K/V view == what the dictionary cache holds, in token order
+        k = dev.k_pool.cpu().numpy()
+        v = dev.v_pool.cpu().numpy()
+        for r in range(R):
+            want = truth.live_tokens(r)
+            assert g_ids[g_off[r]:g_off[r + 1]].tolist() == want
+            for l in range(dev.layers):
+                rows_k = k[l][g_slots[g_off[r]:g_off[r + 1]]]
+                rows_v = v[l][g_slots[g_off[r]:g_off[r + 1]]]
+                for i, tok in enumerate(want):
+                    assert np.array_equal(rows_k[i], dev.payload(r, tok, l, 0, dev.row_elems))
+                    assert np.array_equal(rows_v[i], dev.payload(r, tok, l, 1, dev.row_elems))
+    assert repacked_something
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] == 0
+    dev.close()
+
+
+def test_runtime_flags_and_edges():
+    import torch
+    S = 4
+    st = ServingState.empty(S, capacities=[10, 6], block_lists=[np.array([2, 9], np.int32), np.array([5], np.int32)],
+                            num_blocks=12)
+    dev = DeviceServing(st)
+    # growth beyond the block list / the table capacity stops early and raises the flag
+    ref = ServingState.empty(S, capacities=[10, 6], block_lists=[np.array([2, 9], np.int32), np.array([5], np.int32)],
+                             num_blocks=12)
+    for new_len in ([3, 2], [7, 2], [12, 6]):
+        vto.sync_new_tokens(S, ref.tt_offsets, ref.tt_slots, ref.keep, ref.tt_len, ref.phys_len, ref.bt_offsets,
+                            ref.bt_blocks, new_len)
+        dev.upload_blocks(ref)
+        dev.new_len.copy_(torch.tensor(new_len, dtype=torch.int32))
+        vt.vtoken_sync_new_tokens(dev.ctx, num_requests=dev.num_requests, tt_offsets=dev.tt_offsets,
+                                  tt_slots=dev.tt_slots, keep=dev.keep, tt_len=dev.tt_len, phys_len=dev.phys_len,
+                                  bt_offsets=dev.bt_offsets, bt_blocks=dev.bt_blocks, new_len=dev.new_len)
+        torch.cuda.synchronize()
+        assert np.array_equal(dev.tt_slots.cpu().numpy(), ref.tt_slots)
+        assert np.array_equal(dev.tt_len.cpu().numpy(), ref.tt_len)
+        assert np.array_equal(dev.phys_len.cpu().numpy(), ref.phys_len)
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] & vt.FLAG_APPEND_STOPPED
+    # victims outside the registered tokens are skipped and flagged
+    vr = np.array([0, 1, 1, 0, 2, -1], np.int32)
+    vtok = np.array([3, 0, 11, 10, 0, 0], np.int32)
+    bad = vto.evict_tokens(ref.tt_offsets, ref.tt_len, ref.keep, vr, vtok)
+    assert bad == 4
+    dev.evict(vr, vtok)
+    torch.cuda.synchronize()
+    assert np.array_equal(dev.keep.cpu().numpy(), ref.keep)
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] & vt.FLAG_BAD_VICTIM
+    # slot mapping into a buffer that is too small: what fits is kept, the flag is raised
+    o_slots, o_ids, o_off = vto.build_slot_mapping(ref.tt_offsets, ref.tt_slots, ref.keep)
+    small = torch.full((4,), -1, dtype=torch.int32, device=dev.dev)
+    vt.vtoken_build_slot_mapping(dev.ctx, num_requests=dev.num_requests, tt_offsets=dev.tt_offsets,
+                                 tt_slots=dev.tt_slots, keep=dev.keep, select=None, out_slots=small,
+                                 out_token_ids=None, out_capacity=4, out_offsets=dev.map_offsets)
+    torch.cuda.synchronize()
+    assert np.array_equal(small.cpu().numpy(), o_slots[:4])
+    assert np.array_equal(dev.map_offsets.cpu().numpy(), o_off)
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] & vt.FLAG_GATHER_OVERFLOW
+    dev.close()
+
+
+def test_slot_mapping_full_size_tables_match_oracle():
+    """Slot mapping over the steady-state workload's token tables (2.2 M logical entries)."""
+    import torch
+    from paper_2608_13263_b200 import workloads as wl
+    from paper_2608_13263_b200.device import DeviceProblem
+    w = wl.steady_state(seed=0)
+    prob = DeviceProblem(w, allocate_pools=False)
+    # the context wants pools: a one-layer pool of 16-byte rows is enough for table-only calls
+    pool = torch.zeros((1, w.slots_per_layer, 8), dtype=torch.int16, device=prob.device)
+    ctx = vt.vtoken_create(1, w.num_blocks, w.block_size, 1, 8, pool, pool, prob.max_requests, prob.max_tokens,
+                           prob.max_table_blocks, prob.max_free)
+    T = w.num_tokens
+    out_slots = torch.full((T,), -1, dtype=torch.int32, device=prob.device)
+    out_ids = torch.full((T,), -1, dtype=torch.int32, device=prob.device)
+    out_off = torch.zeros(w.num_requests + 1, dtype=torch.int32, device=prob.device)
+    vt.vtoken_build_slot_mapping(ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                 tt_slots=prob.tt_slots, keep=prob.keep, select=None, out_slots=out_slots,
+                                 out_token_ids=out_ids, out_capacity=T, out_offsets=out_off)
+    torch.cuda.synchronize()
+    o_slots, o_ids, o_off = vto.build_slot_mapping(w.tt_offsets, w.tt_slots, w.keep)
+    n = len(o_slots)
+    assert np.array_equal(out_off.cpu().numpy(), o_off)
+    assert np.array_equal(out_slots.cpu().numpy()[:n], o_slots)
+    assert np.array_equal(out_ids.cpu().numpy()[:n], o_ids)
+    vt.vtoken_destroy(ctx)

@@ -392,6 +392,8 @@ def run_cuda(args):
 
     if args.proxy:
         line["concurrency"] = run_proxy(args, prob, w, side, g_all, bytes_per_step, dev)
+    if args.runtime:
+        line["runtime"] = run_runtime(args, prob, w, side, dev)
 
     # ---- oracle timed beside it (rank 0, N = 1 only) ------------------------------------------
     if ranks.world == 1 and not args.no_cpu_baseline:
@@ -490,6 +492,91 @@ def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
             "streams": "proxy on a high-priority stream, repack graph on the default-priority side stream"}
 
 
+def run_runtime(args, prob, w, side, dev):
+    """Token-table runtime kernels on this workload's tables: slot mapping over every request,
+    one decode step of appends (one token per request), a batch of evictions, and the commit of
+    the plan.  Each is captured in its own graph and replayed; reported as microseconds per call
+    and as table bytes moved per second (HBM-bound, a few bytes per table entry)."""
+    import torch
+    from paper_2608_13263_b200 import binding as vt
+    R, T = w.num_requests, w.num_tokens
+    i32 = dict(dtype=torch.int32, device=dev)
+    live = int(((w.tt_slots >= 0) & (w.keep != 0)).sum())
+    out_slots = torch.zeros(max(1, T), **i32)
+    out_ids = torch.zeros(max(1, T), **i32)
+    out_off = torch.zeros(R + 1, **i32)
+    # a copy of the tables with one spare entry per request, so that appends have room
+    cap_off = (w.tt_offsets.astype(np.int64) + np.arange(R + 1)).astype(np.int32)
+    tt_slots2 = np.full(int(cap_off[-1]), -1, np.int32)
+    keep2 = np.zeros(int(cap_off[-1]), np.uint8)
+    for r in range(R):
+        n = w.tt_offsets[r + 1] - w.tt_offsets[r]
+        tt_slots2[cap_off[r]:cap_off[r] + n] = w.tt_slots[w.tt_offsets[r]:w.tt_offsets[r + 1]]
+        keep2[cap_off[r]:cap_off[r] + n] = w.keep[w.tt_offsets[r]:w.tt_offsets[r + 1]]
+    lens = np.diff(w.tt_offsets).astype(np.int32)
+    d = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    cap_off_d, tt2, keep2_d = d(cap_off), d(tt_slots2), d(keep2)
+    tt_len, new_len = d(lens), d(lens + 1)
+    phys = d(np.zeros(R, np.int32))          # position 0 of each block list: always in range
+    nv = min(65536, T)
+    rng = np.random.default_rng(1)
+    vreq = rng.integers(0, R, size=nv).astype(np.int32)
+    vtok = (rng.random(nv) * lens[vreq]).astype(np.int32)
+    vreq_d, vtok_d, nv_d = d(vreq), d(vtok), d(np.array([nv], np.int32))
+    keep_scratch = prob.keep.clone()
+
+    def slot_mapping(st):
+        vt.vtoken_build_slot_mapping(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                     tt_slots=prob.tt_slots, keep=prob.keep, select=None, out_slots=out_slots,
+                                     out_token_ids=out_ids, out_capacity=T, out_offsets=out_off, stream=st)
+
+    def append(st):
+        vt.vtoken_sync_new_tokens(prob.ctx, num_requests=prob.num_requests, tt_offsets=cap_off_d, tt_slots=tt2,
+                                  keep=keep2_d, tt_len=tt_len, phys_len=phys, bt_offsets=prob.bt_offsets,
+                                  bt_blocks=prob.bt_blocks, new_len=new_len, stream=st)
+
+    def evict(st):
+        vt.vtoken_evict_tokens(prob.ctx, num_victims=nv_d, max_victims=nv, victim_req=vreq_d, victim_tok=vtok_d,
+                               num_requests=prob.num_requests, tt_offsets=prob.tt_offsets, tt_len=tt_len,
+                               keep=keep_scratch, stream=st)
+
+    tt_commit = prob.tt_slots.clone()
+    keep_commit = prob.keep.clone()
+
+    def commit(st):
+        vt.vtoken_apply_moves(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                              tt_slots=tt_commit, keep=keep_commit, phys_len=phys, new_tt_slots=prob.new_tt_slots,
+                              req_status=prob.req_status, stream=st)
+
+    out = {}
+    table_bytes = {"slot_mapping": 2 * 5 * T + 8 * live, "append_one_token_per_request": R * (4 * 6 + 5),
+                   "evict_64k_victims": nv * (8 + 4 + 4 + 1), "apply_moves": T * (4 + 4 + 1)}
+    for name, fn in (("slot_mapping", slot_mapping), ("append_one_token_per_request", append),
+                     ("evict_64k_victims", evict), ("apply_moves", commit)):
+        with torch.cuda.stream(side):
+            fn(side)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn(torch.cuda.current_stream())
+        reps = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(side):
+            for _ in range(3):
+                g.replay()
+            e0.record(side)
+            for _ in range(reps):
+                g.replay()
+            e1.record(side)
+        side.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        out[name] = {"us": us, "table_bytes": table_bytes[name], "GBs": table_bytes[name] / us / 1e3}
+    out["entries"] = {"logical_tokens": T, "live_tokens": live, "requests": R}
+    out["note"] = ("append after the first replay is a no-op per request (tt_len already equals new_len): the figure "
+                   "is the launch + per-request check cost of a decode step")
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -504,6 +591,7 @@ def main():
     ap.add_argument("--oracle-layers", type=int, default=8, help="layers in the CPU-baseline sample")
     ap.add_argument("--proxy", action="store_true", help="also run the repack beside a decode-read proxy")
     ap.add_argument("--proxy-ctas", type=int, default=0)
+    ap.add_argument("--runtime", action="store_true", help="also time the token-table runtime kernels")
     ap.add_argument("--block-size", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

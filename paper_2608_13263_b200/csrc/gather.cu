@@ -2,17 +2,19 @@
 // K and V rows of the active tokens of the selected requests, request order then token-id
 // order, written densely.  Same structure as the planner: count -> scan -> assign, then a
 // row-copy kernel that reads through the token table (the slot-translation read pattern of
-// Sec. 3.4).
+// Sec. 3.4).  Like the planner, every request is cut into VTK_PLAN_PARTS equal token ranges with
+// one CTA each in count and assign, so that long requests do not serialise on one CTA.
 #include "common.cuh"
 
 namespace {
 
 constexpr int G_NT = 512;
+constexpr int G_PARTS = VTK_PLAN_PARTS;
 
 struct GatherArgs {
     const int32_t *num_requests, *tt_offsets, *tt_slots;
     const uint8_t *keep, *select;
-    int32_t *req_n, *out_offsets, *g_src, *g_ids, *g_total;   // g_ids: logical id of each output row, or NULL
+    int32_t *req_n, *part_n, *out_offsets, *g_src, *g_ids, *g_total;   // g_ids: logical id of each output row, or NULL
     vtoken_counts *counts;
     const uint8_t *k_pool, *v_pool;
     uint8_t *out_k, *out_v;
@@ -26,15 +28,27 @@ __device__ __forceinline__ int g_requests(const GatherArgs &a)
     return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
 }
 
+// token range [p0, p1) of part c of a request spanning [t0, t1): equal parts, multiples of 128
+__device__ __forceinline__ void g_part_range(int64_t t0, int64_t t1, int c, int64_t &p0, int64_t &p1)
+{
+    int64_t per = (t1 - t0 + G_PARTS - 1) / G_PARTS;
+    per = (per + 127) & ~(int64_t)127;
+    p0 = t0 + (int64_t)c * per;
+    p1 = p0 + per;
+    if (p0 > t1) p0 = t1;
+    if (p1 > t1) p1 = t1;
+}
+
 __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
 {
-    const int r = blockIdx.x;
+    const int r = blockIdx.x / G_PARTS, c = blockIdx.x % G_PARTS;
     if (r >= g_requests(a)) return;
     int n = 0;
     bool bad = false;
     if (a.select == nullptr || a.select[r] != 0) {
-        const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
-        for (int64_t t = t0 + threadIdx.x; t < t1; t += G_NT)
+        int64_t p0, p1;
+        g_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
+        for (int64_t t = p0 + threadIdx.x; t < p1; t += G_NT)
             n += vtk_live(a.tt_slots[t], a.keep, t, a.slots_per_layer, bad) ? 1 : 0;
     }
     __shared__ int warp_n[G_NT / 32];
@@ -46,7 +60,7 @@ __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
     if (threadIdx.x == 0) {
         int s = 0;
         for (int w = 0; w < G_NT / 32; ++w) s += warp_n[w];
-        a.req_n[r] = s;
+        a.part_n[blockIdx.x] = s;
     }
 }
 
@@ -61,7 +75,11 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(GatherArgs a)
     __syncthreads();
     for (int base = 0; base < R; base += 1024) {
         const int r = base + tid;
-        const int v = r < R ? a.req_n[r] : 0;
+        int v = 0;
+        if (r < R) {
+#pragma unroll
+            for (int c = 0; c < G_PARTS; ++c) v += a.part_n[r * G_PARTS + c];
+        }
         int incl = vtk_warp_incl_scan(v);
         if (lane == 31) warp_tot[warp] = incl;
         __syncthreads();
@@ -93,17 +111,20 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(GatherArgs a)
 __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
 {
     __shared__ int warp_sums[G_NT / 32 + 1];
-    const int r = blockIdx.x;
+    const int r = blockIdx.x / G_PARTS, c = blockIdx.x % G_PARTS;
     if (r >= g_requests(a)) return;
     if (a.select != nullptr && a.select[r] == 0) return;
-    const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
+    const int64_t t0 = a.tt_offsets[r];
+    int64_t p0, p1;
+    g_part_range(t0, a.tt_offsets[r + 1], c, p0, p1);
     const int64_t cap = *a.g_total;
     int carry = a.out_offsets[r];
-    for (int64_t tb = t0; tb < t1; tb += G_NT) {
+    for (int cc = 0; cc < c; ++cc) carry += a.part_n[r * G_PARTS + cc];
+    for (int64_t tb = p0; tb < p1; tb += G_NT) {
         const int64_t t = tb + threadIdx.x;
         int32_t slot = -1;
         bool live = false, bad = false;
-        if (t < t1) {
+        if (t < p1) {
             slot = a.tt_slots[t];
             live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
         }
@@ -175,6 +196,7 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.keep = keep;
     a.select = select;
     a.req_n = ctx->req_n;
+    a.part_n = ctx->part_n;
     a.out_offsets = out_offsets;
     a.g_src = ctx->g_src;
     a.g_ids = nullptr;
@@ -192,9 +214,9 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.layer_begin = layer_begin;
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
-    gather_count_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
     gather_scan_kernel<<<1, 1024, 0, st>>>(a);
-    gather_assign_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
     gather_copy_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
@@ -217,6 +239,7 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.keep = keep;
     a.select = select;
     a.req_n = ctx->req_n;
+    a.part_n = ctx->part_n;
     a.out_offsets = out_offsets;
     a.g_src = out_slots;
     a.g_ids = out_token_ids;
@@ -231,9 +254,9 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.max_tokens = out_capacity;
     a.layer_begin = a.layer_end = 0;
     a.max_requests = ctx->cfg.max_requests;
-    gather_count_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
     gather_scan_kernel<<<1, 1024, 0, st>>>(a);
-    gather_assign_kernel<<<ctx->cfg.max_requests, G_NT, 0, st>>>(a);
+    gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

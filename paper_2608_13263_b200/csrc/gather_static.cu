@@ -16,11 +16,11 @@ namespace {
 constexpr int32_t NOALLOC_MAX_REQUESTS = 4096;
 constexpr int64_t NOALLOC_MAX_TOKENS = 262144;
 
-// layout: [0,256) counts + row total | per-request live counts | source slot of each output row
+// layout: [0,256) counts + row total | live counts per request part | source slot of each output row
 constexpr size_t OFF_COUNTS = 0;
 constexpr size_t OFF_TOTAL = 64;
 constexpr size_t OFF_REQ_N = 256;
-constexpr size_t OFF_SRC = OFF_REQ_N + sizeof(int32_t) * NOALLOC_MAX_REQUESTS;
+constexpr size_t OFF_SRC = OFF_REQ_N + sizeof(int32_t) * NOALLOC_MAX_REQUESTS * VTK_PLAN_PARTS;
 constexpr size_t SCRATCH_BYTES = OFF_SRC + sizeof(int32_t) * NOALLOC_MAX_TOKENS;
 
 }  // namespace
@@ -109,7 +109,7 @@ extern "C" int vtoken_gather_logical_noalloc(const void *k_pool, const void *v_p
     ctx.num_sms = slot->num_sms;
     ctx.counts = reinterpret_cast<vtoken_counts *>(slot->scratch + OFF_COUNTS);
     ctx.g_total = reinterpret_cast<int32_t *>(slot->scratch + OFF_TOTAL);
-    ctx.req_n = reinterpret_cast<int32_t *>(slot->scratch + OFF_REQ_N);
+    ctx.part_n = reinterpret_cast<int32_t *>(slot->scratch + OFF_REQ_N);
     ctx.g_src = reinterpret_cast<int32_t *>(slot->scratch + OFF_SRC);
 
     cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -275,3 +275,60 @@ def apply_moves(tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, phys_len, ne
                                _p(new_tt_slots, np.int32), _p(req_status, np.int32))
     if rc != 0:
         raise ValueError(f"vto_apply_moves failed: {rc}")
+
+
+# ---- eligibility metadata and partial plans ---------------------------------------------------
+class _PartialOpts(ctypes.Structure):
+    _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
+                ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32)]
+
+
+def block_liveness(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep=None):
+    """Returns (n_b[NB], hist[S+1], live_total, num_allocated)."""
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots, keep = _i32(tt_offsets), _i32(tt_slots), _u8(keep)
+    n_b = np.zeros(max(1, NB), np.int32)
+    hist = np.zeros(S + 1, np.int64)
+    live, alloc = ctypes.c_int64(0), ctypes.c_int64(0)
+    rc = lib().vto_block_liveness(ctypes.c_int32(len(tt_offsets) - 1), ctypes.c_int32(S), ctypes.c_int32(NB),
+                                  _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
+                                  _p(tt_slots, np.int32), _p(keep, np.uint8), _p(n_b, np.int32),
+                                  hist.ctypes.data_as(ctypes.c_void_p), ctypes.byref(live), ctypes.byref(alloc))
+    if rc != 0:
+        raise ValueError(f"vto_block_liveness failed: {rc}")
+    return n_b[:NB], hist, live.value, alloc.value
+
+
+def plan_partial(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, select=None, thr_num=0,
+                 thr_den=0, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0)) -> Plan:
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
+    keep, select, free_blocks, protect = _u8(keep), _u8(select), _i32(free_blocks), _u8(protect)
+    R, T, nbt = len(tt_offsets) - 1, int(tt_offsets[-1]), int(bt_offsets[-1])
+    if num_free is None:
+        num_free = len(free_blocks)
+    if protect is not None:
+        assert len(protect) == NB
+    # a partial plan may hold on to blocks AND take destinations: size the table for both
+    new_bt_offsets = np.zeros(R + 1, np.int32)
+    new_bt_blocks = np.full(max(nbt + num_free, 1), -7, np.int32)
+    new_tt_slots = np.full(max(T, 1), -7, np.int32)
+    freed = np.full(max(nbt, 1), -7, np.int32)
+    status = np.full(max(R, 1), -7, np.int32)
+    msrc = np.full(max(T, 1), -7, np.int32)
+    mdst = np.full(max(T, 1), -7, np.int32)
+    c = _Counts()
+    o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1], max_source_blocks,
+                     theta[0], theta[1])
+    rc = lib().vto_plan_partial(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
+                                _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
+                                _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),
+                                ctypes.c_uint32(thr_num), ctypes.c_uint32(thr_den), _p(free_blocks, np.int32),
+                                ctypes.c_int32(num_free), ctypes.byref(o), _p(new_bt_offsets, np.int32),
+                                _p(new_bt_blocks, np.int32), _p(new_tt_slots, np.int32), _p(freed, np.int32),
+                                _p(status, np.int32), _p(msrc, np.int32), _p(mdst, np.int32), ctypes.byref(c))
+    if rc != 0:
+        raise ValueError(f"vto_plan_partial failed: {rc}")
+    return Plan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
+                freed[:c.num_freed].copy(), status[:R].copy(), msrc[:c.num_moves].copy(), mdst[:c.num_moves].copy(),
+                c.num_moves, c.num_dst_blocks, c.num_freed, c.num_free_consumed, c.num_admitted, c.num_deferred)

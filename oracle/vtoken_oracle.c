@@ -382,6 +382,140 @@ int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uin
     return VTO_OK;
 }
 
+int vto_block_liveness(int32_t R, int32_t S, int32_t NB, const int32_t *bt_offsets, const int32_t *bt_blocks,
+                       const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                       int32_t *n_b, int64_t *hist, int64_t *live_total, int64_t *num_allocated)
+{
+    if (R < 0 || S < 1 || NB < 0 || !n_b) return VTO_EINVAL;
+    for (int32_t b = 0; b < NB; ++b) n_b[b] = 0;
+    int64_t live = 0;
+    for (int64_t t = 0; t < tt_offsets[R]; ++t) {
+        if (!is_live(tt_slots, keep, t)) continue;
+        const int64_t b = tt_slots[t] / S;                 /* slot = block * S + offset */
+        if (b >= NB) return VTO_EINVAL;
+        ++n_b[b];                                          /* n_b: valid tokens stored in block b */
+        ++live;
+    }
+    if (hist) {
+        for (int32_t k = 0; k <= S; ++k) hist[k] = 0;
+        for (int32_t j = 0; j < bt_offsets[R]; ++j) {
+            const int32_t b = bt_blocks[j];
+            if (b < 0 || b >= NB || n_b[b] > S) return VTO_EINVAL;
+            ++hist[n_b[b]];
+        }
+    }
+    if (live_total) *live_total = live;
+    if (num_allocated) *num_allocated = bt_offsets[R];
+    return VTO_OK;
+}
+
+int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
+                     const int32_t *bt_offsets, const int32_t *bt_blocks,
+                     const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                     const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+                     const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
+                     int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
+                     int32_t *freed_blocks, int32_t *req_status,
+                     int32_t *move_src, int32_t *move_dst, vto_counts *counts)
+{
+    if (R < 0 || S < 1 || NB < 1 || num_free < 0 || !opts || !counts) return VTO_EINVAL;
+    int32_t *n_b = (int32_t *)malloc(sizeof(int32_t) * (size_t)NB);
+    uint8_t *is_source = (uint8_t *)malloc((size_t)NB);     /* per physical block, for the request at hand */
+    if (!n_b || !is_source) { free(n_b); free(is_source); return VTO_EINVAL; }
+
+    /* eligibility metadata: per-block liveness and the global waste ratio F (Sec. 3.3.1) */
+    int64_t live_total = 0, N = 0;
+    int rc = vto_block_liveness(R, S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, n_b, NULL,
+                                &live_total, &N);
+    if (rc != VTO_OK) { free(n_b); free(is_source); return rc; }
+    /* F > theta  <=>  (N*S - live) * den > num * N*S, in integers */
+    int triggered = 1;
+    if (opts->theta_den != 0) {
+        const uint64_t cap = (uint64_t)N * (uint64_t)S;
+        triggered = N > 0 && (cap - (uint64_t)live_total) * opts->theta_den > (uint64_t)opts->theta_num * cap;
+    }
+    memset(is_source, 0, (size_t)NB);
+
+    int32_t consumed = 0, num_freed = 0, num_moves = 0, num_admitted = 0, num_deferred = 0, new_bt_fill = 0;
+    int stop = 0;
+    for (int32_t r = 0; r < R; ++r) {
+        const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
+        const int32_t b0 = bt_offsets[r], b1 = bt_offsets[r + 1];
+        const int32_t nb = b1 - b0;
+
+        /* source blocks: unprotected, low utilisation, at most B of them in table order (Sec. 3.3.3) */
+        int32_t ns = 0;
+        for (int32_t j = b0; j < b1; ++j) {
+            const int32_t b = bt_blocks[j];
+            int eligible = !(opts->protect && opts->protect[b]);
+            if (eligible && opts->util_den != 0)
+                eligible = (uint64_t)n_b[b] * opts->util_den < (uint64_t)opts->util_num * (uint64_t)S;
+            if (eligible && opts->max_source_blocks > 0 && ns >= opts->max_source_blocks) eligible = 0;
+            is_source[b] = (uint8_t)eligible;
+            ns += eligible;
+        }
+        /* live tokens of the request, and those that sit in source blocks (T_live) */
+        int64_t n = 0, n_src = 0;
+        for (int64_t t = t0; t < t1; ++t) {
+            if (!is_live(tt_slots, keep, t)) continue;
+            ++n;
+            n_src += is_source[tt_slots[t] / S];
+        }
+        const int32_t need = ceil_div(n_src, S);
+
+        int sel = triggered && (select == NULL || select[r] != 0);
+        if (sel && thr_den != 0)
+            sel = (uint64_t)n * thr_den < (uint64_t)thr_num * (uint64_t)nb * (uint64_t)S;
+        int32_t status;
+        if (!sel) status = VTO_NOT_SELECTED;
+        else if (!(need < ns)) status = VTO_NO_GAIN;        /* sources must release more than they consume */
+        else if (stop || (int64_t)consumed + need > num_free) { status = VTO_DEFERRED_NO_FREE; stop = 1; }
+        else status = VTO_REPACKED;
+        req_status[r] = status;
+
+        new_bt_offsets[r] = new_bt_fill;
+        if (status == VTO_REPACKED) {
+            const int32_t *dst = free_blocks + consumed;
+            int64_t i = 0;
+            for (int64_t t = t0; t < t1; ++t) {
+                if (!is_live(tt_slots, keep, t)) { new_tt_slots[t] = -1; continue; }
+                if (is_source[tt_slots[t] / S]) {
+                    const int32_t slot = dst[i / S] * S + (int32_t)(i % S);
+                    new_tt_slots[t] = slot;
+                    move_src[num_moves] = tt_slots[t];
+                    move_dst[num_moves] = slot;
+                    ++num_moves;
+                    ++i;
+                } else {
+                    new_tt_slots[t] = tt_slots[t];          /* its block stays in place */
+                }
+            }
+            for (int32_t j = b0; j < b1; ++j)
+                if (!is_source[bt_blocks[j]]) new_bt_blocks[new_bt_fill++] = bt_blocks[j];
+            for (int32_t j = 0; j < need; ++j) new_bt_blocks[new_bt_fill++] = dst[j];
+            for (int32_t j = b0; j < b1; ++j)
+                if (is_source[bt_blocks[j]]) freed_blocks[num_freed++] = bt_blocks[j];
+            consumed += need;
+            ++num_admitted;
+        } else {
+            if (status == VTO_DEFERRED_NO_FREE) ++num_deferred;
+            for (int64_t t = t0; t < t1; ++t)
+                new_tt_slots[t] = is_live(tt_slots, keep, t) ? tt_slots[t] : -1;
+            for (int32_t j = b0; j < b1; ++j) new_bt_blocks[new_bt_fill++] = bt_blocks[j];
+        }
+        for (int32_t j = b0; j < b1; ++j) is_source[bt_blocks[j]] = 0;
+    }
+    new_bt_offsets[R] = new_bt_fill;
+    counts->num_moves = num_moves;
+    counts->num_dst_blocks = consumed;
+    counts->num_freed = num_freed;
+    counts->num_free_consumed = consumed;
+    counts->num_admitted = num_admitted;
+    counts->num_deferred = num_deferred;
+    free(n_b); free(is_source);
+    return VTO_OK;
+}
+
 int vto_openmp_threads(void)
 {
 #ifdef _OPENMP

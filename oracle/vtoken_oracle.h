@@ -144,6 +144,43 @@ int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32
 int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
                     int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status);
 
+/* ---- eligibility metadata and partial plans (Sec. 3.3.1 - 3.3.3) ------------------------------
+ * Per-block liveness n_b = live tokens stored in physical block b (over all requests), the
+ * histogram hist[k] = number of ALLOCATED blocks (entries of the block tables) with n_b == k for
+ * k = 0..S, the total live count and the allocated-block count N, from which
+ * F = 1 - live_total / (N * S) (Sec. 2.3.1).  n_b has NB entries, hist has S + 1. */
+int vto_block_liveness(int32_t R, int32_t S, int32_t NB, const int32_t *bt_offsets, const int32_t *bt_blocks,
+                       const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                       int32_t *n_b, int64_t *hist, int64_t *live_total, int64_t *num_allocated);
+
+typedef struct {
+    const uint8_t *protect;       /* [NB] or NULL: non-zero = the block must stay (shared prefix, I4) */
+    uint32_t util_num, util_den;  /* a block is a source iff n_b * util_den < util_num * S; util_den == 0: every
+                                     unprotected block (whole-request compaction) */
+    int32_t max_source_blocks;    /* B: at most this many sources per request, first in table order; 0 = no bound */
+    uint32_t theta_num, theta_den;/* plan only when F > theta_num / theta_den; theta_den == 0: always */
+} vto_partial_opts;
+
+/* Relocation planning that evacuates only low-utilisation source blocks (Sec. 3.3.3):
+ * the paper's planner "selects eligible low-utilization source blocks, computes the live-token
+ * footprint" T_live of those blocks, needs ceil(T_live / S) destinations and admits the plan only
+ * when the sources release more blocks than that.  Everything else as vto_plan, except:
+ *   - only live tokens stored in source blocks move (logical order, destinations filled completely);
+ *     live tokens in the other blocks keep their slots; dead tokens become -1;
+ *   - new block table of a repacked request = its non-source blocks in old order, then its
+ *     destination blocks; the reclaimed list receives its source blocks in old order;
+ *   - when the global trigger F > theta does not hold, every request is VTO_NOT_SELECTED.
+ * With util_den == 0, protect == NULL, B == 0 and theta_den == 0 the result equals vto_plan's.
+ * NB = number of physical blocks (size of protect and of the internal n_b). */
+int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
+                     const int32_t *bt_offsets, const int32_t *bt_blocks,
+                     const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                     const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+                     const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
+                     int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
+                     int32_t *freed_blocks, int32_t *req_status,
+                     int32_t *move_src, int32_t *move_dst, vto_counts *counts);
+
 int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */
 
 #ifdef __cplusplus

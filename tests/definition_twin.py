@@ -72,3 +72,66 @@ def to_csr(lists):
         flat.extend(x)
         offsets.append(len(flat))
     return offsets, flat
+
+
+def repack_partial_definition(S, block_tables, token_tables, keeps, free, select=None, thr=None, protect=(),
+                              util=None, max_sources=0, theta=None):
+    """Definition-level statement of the partial plan: only low-utilisation, unprotected blocks are
+    evacuated.  protect: set of block ids; util / theta: Fraction or None."""
+    R = len(token_tables)
+    live = [[t for t, (s, k) in enumerate(zip(token_tables[r], keeps[r])) if s >= 0 and k] for r in range(R)]
+    per_block = {}
+    for r in range(R):
+        for t in live[r]:
+            b = token_tables[r][t] // S
+            per_block[b] = per_block.get(b, 0) + 1
+    allocated = sum(len(b) for b in block_tables)
+    total_live = sum(len(x) for x in live)
+    triggered = True
+    if theta is not None:
+        triggered = allocated > 0 and 1 - Fraction(total_live, allocated * S) > theta
+
+    sources = []
+    for r in range(R):
+        picked = []
+        for b in block_tables[r]:
+            ok = b not in protect and (util is None or Fraction(per_block.get(b, 0), S) < util)
+            if ok and (max_sources == 0 or len(picked) < max_sources):
+                picked.append(b)
+        sources.append(picked)
+    moving = [[t for t in live[r] if token_tables[r][t] // S in set(sources[r])] for r in range(R)]
+    need = [-(-len(moving[r]) // S) for r in range(R)]
+
+    def chosen(r):
+        if not triggered or (select is not None and not select[r]):
+            return False
+        if thr is not None:
+            capacity = len(block_tables[r]) * S
+            if capacity == 0 or not Fraction(len(live[r]), capacity) < thr:
+                return False
+        return True
+
+    candidates = [r for r in range(R) if chosen(r) and need[r] < len(sources[r])]
+    running = list(accumulate(need[r] for r in candidates))
+    fits = [c <= len(free) for c in running]
+    n_admit = fits.index(False) if False in fits else len(candidates)
+    admitted, deferred = candidates[:n_admit], set(candidates[n_admit:])
+    status = [1 if r in admitted else 3 if r in deferred else 2 if chosen(r) else 0 for r in range(R)]
+
+    cursor = 0
+    new_bt, new_tt, freed, moves = [], [], [], []
+    for r in range(R):
+        where = {t: token_tables[r][t] for t in live[r]}
+        if r in admitted:
+            mine = free[cursor:cursor + need[r]]
+            cursor += need[r]
+            for i, t in enumerate(moving[r]):
+                where[t] = mine[i // S] * S + i % S
+                moves.append((token_tables[r][t], where[t]))
+            src = set(sources[r])
+            new_bt.append([b for b in block_tables[r] if b not in src] + list(mine))
+            freed.extend(b for b in block_tables[r] if b in src)
+        else:
+            new_bt.append(list(block_tables[r]))
+        new_tt.append([where.get(t, -1) for t in range(len(token_tables[r]))])
+    return dict(new_bt=new_bt, new_tt=new_tt, freed=freed, status=status, moves=moves, consumed=cursor)

@@ -1,0 +1,185 @@
+"""Pins of the oracle's eligibility metadata (per-block liveness, F) and of partial plans that
+evacuate only low-utilisation, unprotected blocks (no GPU)."""
+import itertools
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from definition_twin import repack_partial_definition, to_csr
+from oracle import vto
+from paper_2608_13263_b200 import workloads as wl
+
+
+def workloads():
+    yield wl.tiny(seed=0)
+    yield wl.llama8b_h2o(seed=1, requests=5, lo=100, hi=400, layers=1, heads=1, head_dim=8)
+    yield wl.mistral7b_random(seed=2, requests=9, lo=20, hi=200, layers=1, heads=1, head_dim=8)
+    yield wl.steady_state(seed=4, requests=12, lo=100, hi=600, layers=1, heads=1, head_dim=8)
+    yield wl.longctx_scissor(seed=3, requests=3, lo=900, hi=1500, layers=1, heads=1, head_dim=8)
+
+
+def plan_p(w, **kw):
+    return vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                            w.free_blocks, w.select, w.thr_num, w.thr_den, **kw)
+
+
+def same_plan(a, b):
+    return all(np.array_equal(getattr(a, f), getattr(b, f)) for f in
+               ("new_bt_offsets", "new_bt_blocks", "new_tt_slots", "freed_blocks", "req_status", "move_src", "move_dst")) \
+        and (a.num_moves, a.num_free_consumed, a.num_freed, a.num_admitted, a.num_deferred) == \
+            (b.num_moves, b.num_free_consumed, b.num_freed, b.num_admitted, b.num_deferred)
+
+
+@pytest.mark.parametrize("w", list(workloads()), ids=lambda w: w.name)
+def test_block_liveness_is_a_bincount_and_F_matches(w):
+    S = w.block_size
+    n_b, hist, live, alloc = vto.block_liveness(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep)
+    is_live = (w.tt_slots >= 0) & (w.keep != 0)
+    assert np.array_equal(n_b, np.bincount(w.tt_slots[is_live] // S, minlength=w.num_blocks))
+    assert np.array_equal(hist, np.bincount(n_b[w.bt_blocks], minlength=S + 1))
+    assert live == int(is_live.sum()) and alloc == len(w.bt_blocks) and hist.sum() == alloc
+    # F = 1 - (1/N) sum u_b over allocated blocks (Sec. 2.3.1), and the oracle's own waste ratio
+    F = 1 - live / (alloc * S)
+    assert F == pytest.approx(1 - np.mean(n_b[w.bt_blocks] / S))
+    assert F == pytest.approx(vto.waste_ratio(S, alloc, w.tt_slots, w.keep))
+
+
+@pytest.mark.parametrize("w", list(workloads()), ids=lambda w: w.name)
+def test_default_options_reduce_to_whole_request_plan(w):
+    assert same_plan(plan_p(w), vto.plan_workload(w))
+    for c in (0, 1, 5):
+        assert same_plan(plan_p(w, num_free=c), vto.plan_workload(w, num_free=c))
+
+
+@pytest.mark.parametrize("w", list(workloads()), ids=lambda w: w.name)
+def test_keeping_full_blocks_gives_the_same_block_count_with_fewer_moves(w):
+    """Sources = blocks that are not fully live (n_b < S).  Block demand f + ceil(p / S) equals
+    ceil((f*S + p) / S): the packed footprint of Sec. 5's block arithmetic, reached with p moves
+    instead of f*S + p."""
+    S = w.block_size
+    whole = vto.plan_workload(w)
+    part = plan_p(w, util=(1, 1))
+    n_b, _, _, _ = vto.block_liveness(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep)
+    live = (w.tt_slots >= 0) & (w.keep != 0)
+    moves = 0
+    for r in range(w.num_requests):
+        blocks = w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]]
+        full = int((n_b[blocks] == S).sum())
+        n = int(live[w.tt_offsets[r]:w.tt_offsets[r + 1]].sum())
+        p = n - full * S
+        after = part.new_bt_offsets[r + 1] - part.new_bt_offsets[r]
+        if part.req_status[r] == vto.REPACKED:
+            assert after == full + -(-p // S) == -(-n // S)
+            moves += p
+            if whole.req_status[r] == vto.REPACKED:
+                assert after == whole.new_bt_offsets[r + 1] - whole.new_bt_offsets[r]
+            # fully live blocks stay where they are, in their old order, ahead of the destinations
+            kept = [b for b in blocks if n_b[b] == S]
+            assert part.new_bt_blocks[part.new_bt_offsets[r]:part.new_bt_offsets[r] + full].tolist() == kept
+    assert part.num_moves == moves <= whole.num_moves or part.num_admitted != whole.num_admitted
+    # token conservation and unique mapping still hold
+    assert np.array_equal(part.new_tt_slots >= 0, live)
+    occ = part.new_tt_slots[part.new_tt_slots >= 0]
+    assert len(np.unique(occ)) == len(occ)
+    assert not (set(part.move_src.tolist()) & set(part.move_dst.tolist()))
+
+
+def test_protected_blocks_never_move_or_get_reclaimed():
+    """Shared-prefix blocks are excluded from plans (I4); here: the first blocks of every request."""
+    w = wl.mistral7b_random(seed=6, requests=6, lo=80, hi=200, layers=1, heads=1, head_dim=8, block_size=4)
+    protect = np.zeros(w.num_blocks, np.uint8)
+    prefix = []
+    for r in range(w.num_requests):
+        blocks = w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]]
+        prefix += blocks[:5].tolist()
+    protect[prefix] = 1
+    p = plan_p(w, protect=protect)
+    assert p.num_admitted > 0
+    assert not (set(p.freed_blocks.tolist()) & set(prefix))
+    assert not (set((p.move_src // w.block_size).tolist()) & set(prefix))
+    for r in range(w.num_requests):
+        blocks = w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]]
+        assert p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r] + 5].tolist() == blocks[:5].tolist()
+    live = (w.tt_slots >= 0) & (w.keep != 0)
+    in_prefix = np.isin(w.tt_slots // w.block_size, prefix) & live
+    assert np.array_equal(p.new_tt_slots[in_prefix], w.tt_slots[in_prefix])
+    # everything protected: nothing can be gained
+    q = plan_p(w, protect=np.ones(w.num_blocks, np.uint8))
+    assert q.num_moves == 0 and set(q.req_status.tolist()) <= {vto.NO_GAIN}
+
+
+def test_global_trigger_threshold_is_strict_and_exact():
+    S = 4
+    bt = np.arange(4, dtype=np.int32)
+    tt = np.arange(16, dtype=np.int32)
+    keep = np.zeros(16, np.uint8)
+    keep[[0, 4, 8, 12]] = 1                                 # F = 1 - 4/16 = 3/4 exactly
+    free = np.array([10, 11], np.int32)
+    args = (S, 12, [0, 4], bt, [0, 16], tt, keep, free)
+    assert vto.plan_partial(*args, theta=(3, 4)).req_status.tolist() == [vto.NOT_SELECTED]      # F > 3/4 is false
+    assert vto.plan_partial(*args, theta=(74, 100)).req_status.tolist() == [vto.REPACKED]
+    assert vto.plan_partial(*args, theta=(1, 4)).req_status.tolist() == [vto.REPACKED]          # the paper's default 0.25
+
+
+def test_source_bound_B_takes_the_first_eligible_blocks_in_table_order():
+    S = 4
+    bt = np.array([3, 0, 2, 1, 5], np.int32)
+    tt = (bt[np.arange(20) // S] * S + np.arange(20) % S).astype(np.int32)
+    keep = np.zeros(20, np.uint8)
+    keep[[0, 5, 9, 14, 17]] = 1                             # one survivor per block
+    free = np.array([8, 9], np.int32)
+    p = vto.plan_partial(S, 10, [0, 5], bt, [0, 20], tt, keep, free, max_source_blocks=3)
+    assert p.freed_blocks.tolist() == [3, 0, 2] and p.num_free_consumed == 1
+    assert p.new_bt_blocks.tolist() == [1, 5, 8]
+    assert p.new_tt_slots[[0, 5, 9]].tolist() == [32, 33, 34] and p.new_tt_slots[[14, 17]].tolist() == tt[[14, 17]].tolist()
+    # B = 1: one source block cannot release more than the one destination it needs
+    assert vto.plan_partial(S, 10, [0, 5], bt, [0, 20], tt, keep, free, max_source_blocks=1).req_status.tolist() == [vto.NO_GAIN]
+
+
+def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB):
+    bt_off, bt_flat = to_csr(bts)
+    tt_off, tt_flat = to_csr(tts)
+    _, keep_flat = to_csr(keeps)
+    prot = np.zeros(NB, np.uint8)
+    prot[list(protect)] = 1
+    fr = lambda f: (f.numerator, f.denominator) if f is not None else (0, 0)
+    p = vto.plan_partial(S, NB, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free,
+                         select=None if select is None else np.array(select, np.uint8),
+                         thr_num=fr(thr)[0], thr_den=fr(thr)[1], protect=prot if protect else None,
+                         util=fr(util), max_source_blocks=B, theta=fr(theta))
+    d = repack_partial_definition(S, bts, tts, keeps, list(free), select, thr, set(protect), util, B, theta)
+    nbo, nbf = to_csr(d["new_bt"])
+    _, ntf = to_csr(d["new_tt"])
+    assert p.new_bt_offsets.tolist() == nbo and p.new_bt_blocks.tolist() == nbf
+    assert p.new_tt_slots.tolist() == ntf and p.freed_blocks.tolist() == d["freed"]
+    assert p.req_status.tolist() == d["status"]
+    assert list(zip(p.move_src.tolist(), p.move_dst.tolist())) == d["moves"]
+    assert p.num_free_consumed == d["consumed"]
+
+
+def test_bruteforce_against_the_definition_twin():
+    rng = np.random.default_rng(3)
+    S = 2
+    bts = [[4, 1, 6], [0, 7, 3], []]
+    tts = [[8, -1, 3, 2, 12, 13], [1, 0, -1, 14, 6, -1, 7], [-1, -1]]
+    NB = 12
+    for _ in range(40):
+        keeps = [rng.integers(0, 2, len(t)).tolist() for t in tts]
+        for util in (None, Fraction(1, 1), Fraction(1, 2)):
+            for protect in ((), (1,), (4, 7)):
+                for B in (0, 1, 2):
+                    for theta in (None, Fraction(1, 4), Fraction(3, 4)):
+                        for c in (0, 1, 3):
+                            _compare(S, bts, tts, keeps, np.array([9, 5, 10][:c], np.int32), None,
+                                     None if c else Fraction(3, 4), protect, util, B, theta, NB)
+
+
+def test_bruteforce_all_masks_one_request():
+    S = 3
+    bt = [2, 0, 1]
+    tt = [bt[t // S] * S + t % S for t in range(8)]
+    for mask in itertools.product([0, 1], repeat=8):
+        for util in (None, Fraction(1, 1), Fraction(2, 3), Fraction(1, 3)):
+            for c in range(3):
+                _compare(S, [bt], [tt], [list(mask)], np.array([5, 4][:c], np.int32), None, None, (), util, 0, None, 8)

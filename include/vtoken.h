@@ -171,6 +171,43 @@ int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const in
  * gather_logical since) to HOST memory.  Synchronises the stream: the only call that does. */
 int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stream);
 
+/* ---- Eligibility metadata and partial plans (Sec. 3.3.1 - 3.3.3) --------------------------------
+ * The paper's reclamation backend keeps per-block liveness n_b (live tokens stored in block b),
+ * derives the intra-block waste ratio F = 1 - sum(n_b) / (N * S) over the N allocated blocks
+ * (Sec. 2.3.1), attempts reclamation only when F exceeds a threshold theta_F (default 0.25,
+ * Sec. 3.3.2), and plans per request over "eligible low-utilization source blocks", at most B of
+ * them, admitting a plan only when those sources release more blocks than the ceil(T_live / S)
+ * destinations they need (Sec. 3.3.3).  Shared-prefix blocks are excluded from plans (I4). */
+
+/* Per-block liveness: n_b[num_blocks] (DEVICE int32) = live tokens per physical block;
+ * hist[block_size + 1] (DEVICE uint64, may be NULL) = number of block-table entries whose block
+ * holds k live tokens; summary[2] (DEVICE int64, may be NULL) = {live tokens, allocated blocks},
+ * i.e. F = 1 - summary[0] / (summary[1] * S).  Uses the context's planner scratch. */
+int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *bt_offsets,
+                          const int32_t *bt_blocks, const int32_t *tt_offsets, const int32_t *tt_slots,
+                          const uint8_t *keep, int32_t *n_b, uint64_t *hist, int64_t *summary, void *cuda_stream);
+
+typedef struct {
+    const uint8_t *protect;        /* DEVICE [num_blocks] or NULL: non-zero = the block never moves (shared prefix) */
+    uint32_t util_num, util_den;   /* a block is a source iff n_b * util_den < util_num * S (64-bit);
+                                      util_den == 0: every unprotected block (whole-request compaction);
+                                      1/1: every block that is not fully live */
+    int32_t max_source_blocks;     /* B: per request at most this many sources, the first eligible ones in
+                                      block-table order; 0 = no bound */
+    uint32_t theta_num, theta_den; /* global trigger: plan only when F > theta_num / theta_den (64-bit integers);
+                                      theta_den == 0: always */
+} vtoken_partial_opts;
+
+/* vtoken_plan restricted to source blocks.  Differences from vtoken_plan: only live tokens stored
+ * in a request's source blocks move (logical order, destinations filled completely), need =
+ * ceil(live tokens in sources / S), candidate iff need < number of sources; live tokens in the
+ * other blocks keep their slots; new block table = the non-source blocks in old order followed by
+ * the destinations; freed_blocks receives the source blocks in old order; when the trigger does
+ * not hold every request is VTOKEN_NOT_SELECTED.  With all options zero / NULL the result equals
+ * vtoken_plan's.  vtoken_repack executes the plan. */
+int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
+                        const vtoken_plan_out *out, void *cuda_stream);
+
 /* ---- Token-table runtime on the device (Sec. 3.2 interfaces, Sec. 3.4 slot mapping) ----------
  * For callers that keep the token tables resident on the GPU between decode steps.  Layout: the
  * table of request r occupies tt_slots / keep [tt_offsets[r] .. tt_offsets[r+1]) -- that range is

@@ -20,7 +20,8 @@ FLAG_BAD_VICTIM, FLAG_APPEND_STOPPED = 64, 128
 SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "vtoken_gather_logical",
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
            "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
-           "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves"]
+           "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
+           "vtoken_block_liveness", "vtoken_plan_partial"]
 
 
 class VtokenError(RuntimeError):
@@ -63,6 +64,11 @@ class PlanOut(ctypes.Structure):
     _fields_ = [("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
                 ("new_tt_slots", ctypes.c_void_p), ("freed_blocks", ctypes.c_void_p),
                 ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p)]
+
+
+class PartialOpts(ctypes.Structure):
+    _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
+                ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32)]
 
 
 class HostTables(ctypes.Structure):
@@ -113,6 +119,9 @@ def load():
         lib.vtoken_sync_new_tokens.argtypes = [ctypes.c_void_p] * 11
         lib.vtoken_build_slot_mapping.argtypes = [ctypes.c_void_p] * 8 + [ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
         lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 9
+        lib.vtoken_block_liveness.argtypes = [ctypes.c_void_p] * 11
+        lib.vtoken_plan_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
+                                            ctypes.POINTER(PlanOut), ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -259,3 +268,24 @@ def vtoken_apply_moves(ctx, *, num_requests, tt_offsets, tt_slots, keep, phys_le
     _check(load().vtoken_apply_moves(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                                      _ptr(phys_len), _ptr(new_tt_slots), _ptr(req_status), _stream(stream)),
            "vtoken_apply_moves", ctx)
+
+
+# ---- eligibility metadata and partial plans ---------------------------------------------------
+def vtoken_block_liveness(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, n_b, hist=None,
+                          summary=None, stream=None) -> None:
+    _check(load().vtoken_block_liveness(ctx, _ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets),
+                                        _ptr(tt_slots), _ptr(keep), _ptr(n_b), _ptr(hist), _ptr(summary),
+                                        _stream(stream)), "vtoken_block_liveness", ctx)
+
+
+def vtoken_plan_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
+                        new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status, counts, select=None,
+                        thr_num=0, thr_den=0, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
+                        stream=None) -> None:
+    pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                 _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
+    pout = PlanOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks),
+                   _ptr(req_status), _ptr(counts))
+    po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1])
+    _check(load().vtoken_plan_partial(ctx, ctypes.byref(pin), ctypes.byref(po), ctypes.byref(pout), _stream(stream)),
+           "vtoken_plan_partial", ctx)

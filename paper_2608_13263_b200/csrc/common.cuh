@@ -30,6 +30,13 @@ struct vtoken_ctx {
     int32_t *dst_blocks;       // [cap_dst_blocks] physical id of each destination block, -1 = skip
     vtoken_counts *counts;     // one struct
 
+    // partial-plan scratch (DEVICE)
+    int32_t *part_src;         // [max_requests * VTK_PLAN_PARTS] live tokens in source blocks per request part
+    int32_t *req_ns;           // [max_requests] source blocks of the request
+    int32_t *req_nsrc;         // [max_requests] live tokens in its source blocks
+    int32_t *n_b;              // [num_blocks] live tokens per physical block
+    uint8_t *blk_src;          // [num_blocks] 1 = the block is a source of its request
+
     // gather_logical scratch (DEVICE)
     int32_t *g_src;            // [max_tokens] source slot of each output row
     int32_t *g_total;          // [1] output rows

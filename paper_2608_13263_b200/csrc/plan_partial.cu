@@ -1,0 +1,517 @@
+// Eligibility metadata and partial relocation plans (Sec. 3.3.1 - 3.3.3 of the paper): per-block
+// liveness n_b, the global waste ratio F as a trigger, and a planner that evacuates only the
+// low-utilisation, unprotected source blocks of a request (at most B of them) and leaves the
+// others -- fully live blocks, shared-prefix blocks -- where they are.
+//
+// Kernels (all grids fixed by the capacities, counts read from device memory):
+//   live    : live tokens per request part; n_b[block] += 1 per live token (integer atomics: the
+//             sums do not depend on their order)
+//   blocks  : per request, which entries of its block table are sources (rank among eligible
+//             entries in table order < B); marks blk_src[block]
+//   src     : live tokens that sit in source blocks, per request part
+//   scan    : global trigger F > theta, candidates (sources release more blocks than the
+//             destinations they need), admission against the free list, bases and counts
+//   assign  : new token table (moving tokens ranked in logical order), new block table
+//             (kept blocks in old order, then destinations), reclaimed list, inverse move plan
+// The inverse plan has the same form as the whole-request planner's, so vtoken_repack runs it
+// unchanged.
+#include "common.cuh"
+
+#include <cstring>
+
+namespace {
+
+constexpr int PP_NT = 512;
+constexpr int PP_PARTS = VTK_PLAN_PARTS;
+constexpr int PP_SCAN_NT = 1024;
+
+struct PArgs {
+    const int32_t *num_requests, *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
+    const uint8_t *keep, *select, *protect;
+    uint32_t thr_num, thr_den, util_num, util_den, theta_num, theta_den;
+    int32_t max_sources;
+    const int32_t *free_blocks, *num_free;
+    int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *out_status;
+    vtoken_counts *out_counts;
+    int32_t *req_n, *part_n, *part_src, *req_ns, *req_nsrc, *req_dst_base, *req_freed_base, *req_status;
+    int32_t *dst_src, *dst_blocks, *n_b;
+    uint8_t *blk_src;
+    vtoken_counts *counts;
+    int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
+    int64_t slots_per_layer, max_tokens, max_table_blocks;
+};
+
+__device__ __forceinline__ int pp_requests(const PArgs &a)
+{
+    int R = *a.num_requests;
+    return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
+}
+
+__device__ __forceinline__ void pp_part_range(int64_t t0, int64_t t1, int c, int64_t &p0, int64_t &p1)
+{
+    int64_t per = (t1 - t0 + PP_PARTS - 1) / PP_PARTS;
+    per = (per + 127) & ~(int64_t)127;
+    p0 = t0 + (int64_t)c * per;
+    p1 = p0 + per;
+    if (p0 > t1) p0 = t1;
+    if (p1 > t1) p1 = t1;
+}
+
+__device__ __forceinline__ int pp_block_sum(int n, int *warp_n)
+{
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+    if (vtk_lane() == 0) warp_n[threadIdx.x >> 5] = n;
+    __syncthreads();
+    int s = 0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) s += warp_n[w];
+    return s;   // valid in thread 0
+}
+
+// ---- live: part counts and per-block liveness -----------------------------------------------
+// mode 0: count live tokens and add them to n_b; mode 1: count live tokens whose block is a source
+template <int MODE>
+__global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
+{
+    __shared__ int warp_n[PP_NT / 32];
+    const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
+    if (r >= pp_requests(a)) return;
+    int64_t p0, p1;
+    pp_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
+    int n = 0;
+    bool bad = false;
+    for (int64_t t = p0 + threadIdx.x; t < p1; t += PP_NT) {
+        const int32_t slot = a.tt_slots[t];
+        if (!vtk_live(slot, a.keep, t, a.slots_per_layer, bad)) continue;
+        if (MODE == 0) {
+            atomicAdd(&a.n_b[slot / a.S], 1);
+            ++n;
+        } else {
+            n += a.blk_src[slot / a.S];
+        }
+    }
+    if (bad && MODE == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
+    const int s = pp_block_sum(n, warp_n);
+    if (threadIdx.x == 0) (MODE == 0 ? a.part_n : a.part_src)[blockIdx.x] = s;
+}
+
+// ---- blocks: source selection per request ------------------------------------------------------
+__global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
+{
+    __shared__ int warp_sums[PP_NT / 32 + 1];
+    const int r = blockIdx.x;
+    if (r >= pp_requests(a)) return;
+    const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
+    int carry = 0;               // eligible entries before this chunk
+    uint32_t flags = 0;
+    for (int jb = b0; jb < b1; jb += PP_NT) {
+        const int j = jb + threadIdx.x;
+        bool eligible = false;
+        int blk = -1;
+        if (j < b1) {
+            blk = a.bt_blocks[j];
+            if (blk < 0 || blk >= a.num_blocks) {
+                flags |= VTOKEN_FLAG_BAD_BLOCK;
+                blk = -1;
+            } else {
+                eligible = !(a.protect != nullptr && a.protect[blk] != 0);
+                if (eligible && a.util_den != 0)
+                    eligible = (unsigned long long)a.n_b[blk] * a.util_den <
+                               (unsigned long long)a.util_num * (unsigned long long)a.S;
+            }
+        }
+        int total;
+        const int rank = carry + vtk_block_rank<PP_NT>(eligible, warp_sums, total);
+        carry += total;
+        if (eligible && (a.max_sources <= 0 || rank < a.max_sources)) a.blk_src[blk] = 1;
+    }
+    if (threadIdx.x == 0) a.req_ns[r] = (a.max_sources > 0 && carry > a.max_sources) ? a.max_sources : carry;
+    if (flags) atomicOr(&a.counts->error_flags, flags);
+}
+
+// ---- scan ----------------------------------------------------------------------------------------
+struct PAcc {
+    int dst, freed, newbt, moves, admitted, deferred;
+};
+__device__ __forceinline__ PAcc operator+(const PAcc &x, const PAcc &y)
+{
+    return PAcc{x.dst + y.dst, x.freed + y.freed, x.newbt + y.newbt, x.moves + y.moves, x.admitted + y.admitted,
+                x.deferred + y.deferred};
+}
+__device__ __forceinline__ PAcc pp_shfl_up(const PAcc &v, int d)
+{
+    return PAcc{__shfl_up_sync(0xffffffffu, v.dst, d),      __shfl_up_sync(0xffffffffu, v.freed, d),
+                __shfl_up_sync(0xffffffffu, v.newbt, d),    __shfl_up_sync(0xffffffffu, v.moves, d),
+                __shfl_up_sync(0xffffffffu, v.admitted, d), __shfl_up_sync(0xffffffffu, v.deferred, d)};
+}
+template <typename T, typename ShflUp>
+__device__ __forceinline__ T pp_block_incl_scan(T v, T *warp_tot, T zero, ShflUp shfl)
+{
+    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T o = shfl(v, d);
+        if (lane >= d) v = o + v;
+    }
+    if (lane == 31) warp_tot[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        T w = warp_tot[lane];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            T o = shfl(w, d);
+            if (lane >= d) w = o + w;
+        }
+        warp_tot[lane] = w;
+    }
+    __syncthreads();
+    T pre = warp == 0 ? zero : warp_tot[warp - 1];
+    T res = pre + v;
+    __syncthreads();
+    return res;
+}
+
+__global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
+{
+    __shared__ long long warp_ll[32];
+    __shared__ PAcc warp_acc[32];
+    __shared__ long long carry_need, tot_live, tot_blocks;
+    __shared__ PAcc carry;
+    const int tid = threadIdx.x;
+    const int R = pp_requests(a);
+    uint32_t flags = 0;
+    if (tid == 0) {
+        if (*a.num_requests > a.max_requests || *a.num_requests < 0) flags |= VTOKEN_FLAG_CAPACITY;
+        if (R > 0 && ((int64_t)a.tt_offsets[R] > a.max_tokens || (int64_t)a.bt_offsets[R] > a.max_table_blocks))
+            flags |= VTOKEN_FLAG_CAPACITY;
+        carry_need = 0;
+        tot_live = 0;
+        tot_blocks = 0;
+        carry = PAcc{0, 0, 0, 0, 0, 0};
+    }
+    int nf = *a.num_free;
+    if (nf > a.max_free_blocks && tid == 0) flags |= VTOKEN_FLAG_CAPACITY;
+    nf = nf < 0 ? 0 : (nf > a.cap_dst_blocks ? a.cap_dst_blocks : nf);
+    __syncthreads();
+    auto shfl_ll = [](long long v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
+    auto shfl_acc = [](const PAcc &v, int d) { return pp_shfl_up(v, d); };
+
+    // pass 1: live tokens per request, and the totals behind F = 1 - live / (N * S)
+    long long my_live = 0, my_blocks = 0;
+    for (int r = tid; r < R; r += PP_SCAN_NT) {
+        int n = 0, nsrc = 0;
+#pragma unroll
+        for (int c = 0; c < PP_PARTS; ++c) {
+            n += a.part_n[r * PP_PARTS + c];
+            nsrc += a.part_src[r * PP_PARTS + c];
+        }
+        a.req_n[r] = n;
+        a.req_nsrc[r] = nsrc;
+        int nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
+        my_live += n;
+        my_blocks += nb < 0 ? 0 : nb;
+    }
+    const long long live_incl = pp_block_incl_scan<long long>(my_live, warp_ll, 0LL, shfl_ll);
+    if (tid == PP_SCAN_NT - 1) tot_live = live_incl;
+    const long long blocks_incl = pp_block_incl_scan<long long>(my_blocks, warp_ll, 0LL, shfl_ll);
+    if (tid == PP_SCAN_NT - 1) tot_blocks = blocks_incl;
+    __syncthreads();
+    bool triggered = true;                      // F > theta  <=>  (N*S - live) * den > num * N*S
+    if (a.theta_den != 0) {
+        const unsigned long long cap = (unsigned long long)tot_blocks * (unsigned long long)a.S;
+        triggered = tot_blocks > 0 && (cap - (unsigned long long)tot_live) * a.theta_den > (unsigned long long)a.theta_num * cap;
+    }
+
+    // pass 2: candidates, admission, bases
+    for (int base = 0; base < R; base += PP_SCAN_NT) {
+        const int r = base + tid;
+        const bool valid = r < R;
+        int n = 0, nsrc = 0, nb = 0, ns = 0;
+        if (valid) {
+            n = a.req_n[r];
+            nsrc = a.req_nsrc[r];
+            ns = a.req_ns[r];
+            nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
+            if (nb < 0) nb = 0;
+        }
+        const int need = (int)(((int64_t)nsrc + a.S - 1) / a.S);   // ceil(T_live / S) over the source blocks
+        bool sel = valid && triggered && (a.select == nullptr || a.select[r] != 0);
+        if (sel && a.thr_den != 0)
+            sel = (unsigned long long)n * a.thr_den <
+                  (unsigned long long)a.thr_num * (unsigned long long)nb * (unsigned long long)a.S;
+        const bool cand = sel && need < ns;                        // sources release more than they consume
+        const long long cum = pp_block_incl_scan<long long>(cand ? need : 0, warp_ll, 0LL, shfl_ll) + carry_need;
+        const bool adm = cand && cum <= (long long)nf;
+        const int status = !sel ? VTOKEN_NOT_SELECTED
+                                : (!cand ? VTOKEN_NO_GAIN : (adm ? VTOKEN_REPACKED : VTOKEN_DEFERRED_NO_FREE));
+        PAcc mine{adm ? need : 0, adm ? ns : 0, valid ? (adm ? nb - ns + need : nb) : 0, adm ? nsrc : 0, adm ? 1 : 0,
+                  (cand && !adm) ? 1 : 0};
+        const PAcc incl = pp_block_incl_scan<PAcc>(mine, warp_acc, PAcc{0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
+        if (valid) {
+            a.req_dst_base[r] = incl.dst - mine.dst;
+            a.req_freed_base[r] = incl.freed - mine.freed;
+            a.new_bt_offsets[r] = incl.newbt - mine.newbt;
+            a.req_status[r] = status;
+            a.out_status[r] = status;
+        }
+        __syncthreads();
+        if (tid == PP_SCAN_NT - 1) {
+            carry_need = cum;
+            carry = incl;
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.new_bt_offsets[R] = carry.newbt;
+        vtoken_counts c;
+        c.num_moves = carry.moves;
+        c.num_dst_blocks = carry.dst;
+        c.num_freed = carry.freed;
+        c.num_free_consumed = carry.dst;
+        c.num_admitted = carry.admitted;
+        c.num_deferred = carry.deferred;
+        c.error_flags = flags | a.counts->error_flags;
+        c.reserved = 0;
+        *a.counts = c;
+        *a.out_counts = c;
+    }
+}
+
+// ---- assign --------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
+{
+    __shared__ int warp_sums[PP_NT / 32 + 1];
+    const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
+    if (r >= pp_requests(a)) return;
+    const int tid = threadIdx.x;
+    const int S = a.S;
+    const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
+    const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
+    const int nb = b1 - b0;
+    const bool adm = a.req_status[r] == VTOKEN_REPACKED;
+    const int nsrc = a.req_nsrc[r], ns = a.req_ns[r];
+    const int need = (int)(((int64_t)nsrc + S - 1) / S);
+    const int dst_base = a.req_dst_base[r];
+    const int nbt0 = a.new_bt_offsets[r];
+    uint32_t flags = 0;
+
+    const int stripe = c * PP_NT + tid, stride = PP_PARTS * PP_NT;
+    if (adm) {
+        // destinations follow the kept blocks in the new block table
+        for (int j = stripe; j < need; j += stride) {
+            int blk = a.free_blocks[dst_base + j];
+            a.new_bt_blocks[nbt0 + (nb - ns) + j] = blk;
+            if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
+            a.dst_blocks[dst_base + j] = blk;
+        }
+        for (int i = nsrc + stripe; i < need * S; i += stride) a.dst_src[(int64_t)dst_base * S + i] = -1;
+        // kept blocks in old order, sources to the reclaimed list in old order: one CTA ranks the table
+        if (c == 0) {
+            const int f0 = a.req_freed_base[r];
+            int carry_src = 0;
+            for (int jb = b0; jb < b1; jb += PP_NT) {
+                const int j = jb + tid;
+                int blk = -1;
+                bool src = false;
+                if (j < b1) {
+                    blk = a.bt_blocks[j];
+                    src = blk >= 0 && blk < a.num_blocks && a.blk_src[blk] != 0;
+                }
+                int total;
+                const int rank_src = carry_src + vtk_block_rank<PP_NT>(src, warp_sums, total);
+                carry_src += total;
+                if (j < b1) {
+                    if (src) a.freed_blocks[f0 + rank_src] = blk;
+                    else a.new_bt_blocks[nbt0 + (j - b0) - rank_src] = blk;   // kept entries before it = all - sources
+                }
+            }
+        }
+    } else {
+        for (int j = stripe; j < nb; j += stride) a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
+    }
+
+    // token table
+    int64_t p0, p1;
+    pp_part_range(t0, t1, c, p0, p1);
+    int carry = 0;                                       // moving tokens of the parts before this one
+    for (int cc = 0; cc < c; ++cc) carry += a.part_src[r * PP_PARTS + cc];
+    for (int64_t tb = p0; tb < p1; tb += PP_NT) {
+        const int64_t t = tb + tid;
+        int32_t slot = -1;
+        bool live = false, bad = false, moving = false;
+        if (t < p1) {
+            slot = a.tt_slots[t];
+            live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
+            moving = live && adm && a.blk_src[slot / S] != 0;
+        }
+        int total;
+        const int i = carry + vtk_block_rank<PP_NT>(moving, warp_sums, total);
+        carry += total;
+        if (t < p1) {
+            int32_t out = -1;
+            if (moving) {
+                const int j = i / S, off = i - j * S;
+                const int blk = a.free_blocks[dst_base + j];
+                out = blk * S + off;
+                a.dst_src[(int64_t)(dst_base + j) * S + off] = slot;
+            } else if (live) {
+                out = slot;                              // its block stays in place
+            }
+            a.new_tt_slots[t] = out;
+        }
+    }
+    if (flags) {
+        atomicOr(&a.counts->error_flags, flags);
+        atomicOr(&a.out_counts->error_flags, flags);
+    }
+}
+
+// ---- histogram of block utilisation ------------------------------------------------------------
+__global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_requests, int32_t max_requests,
+                                                      const int32_t *bt_offsets, const int32_t *bt_blocks,
+                                                      const int32_t *n_b, int32_t S, int32_t num_blocks,
+                                                      unsigned long long *hist, vtoken_counts *counts)
+{
+    int R = *num_requests;
+    R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
+    const int total = bt_offsets[R];
+    bool bad = false;
+    for (int j = blockIdx.x * 256 + threadIdx.x; j < total; j += gridDim.x * 256) {
+        const int blk = bt_blocks[j];
+        if (blk < 0 || blk >= num_blocks) { bad = true; continue; }
+        int k = n_b[blk];
+        if (k > S) k = S;
+        atomicAdd(&hist[k], 1ull);
+    }
+    if (bad) atomicOr(&counts->error_flags, VTOKEN_FLAG_BAD_BLOCK);
+}
+
+__global__ void pp_summary_kernel(const int32_t *num_requests, int32_t max_requests, const int32_t *bt_offsets,
+                                  const int32_t *part_n, long long *summary)
+{
+    // one warp: total live tokens over all parts, allocated blocks
+    int R = *num_requests;
+    R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
+    long long s = 0;
+    for (int i = threadIdx.x; i < R * PP_PARTS; i += 32) s += part_n[i];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
+    if (threadIdx.x == 0) {
+        summary[0] = s;
+        summary[1] = bt_offsets[R];
+    }
+}
+
+void fill_args(PArgs &a, vtoken_ctx *ctx)
+{
+    a.req_n = ctx->req_n;
+    a.part_n = ctx->part_n;
+    a.part_src = ctx->part_src;
+    a.req_ns = ctx->req_ns;
+    a.req_nsrc = ctx->req_nsrc;
+    a.req_dst_base = ctx->req_dst_base;
+    a.req_freed_base = ctx->req_freed_base;
+    a.req_status = ctx->req_status;
+    a.dst_src = ctx->dst_src;
+    a.dst_blocks = ctx->dst_blocks;
+    a.n_b = ctx->n_b;
+    a.blk_src = ctx->blk_src;
+    a.counts = ctx->counts;
+    a.S = ctx->cfg.block_size;
+    a.num_blocks = ctx->cfg.num_blocks;
+    a.max_requests = ctx->cfg.max_requests;
+    a.cap_dst_blocks = ctx->cap_dst_blocks;
+    a.max_free_blocks = ctx->cfg.max_free_blocks;
+    a.slots_per_layer = ctx->slots_per_layer;
+    a.max_tokens = ctx->cfg.max_tokens;
+    a.max_table_blocks = ctx->cfg.max_table_blocks;
+}
+
+}  // namespace
+
+extern "C" {
+
+int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
+                        const vtoken_plan_out *out, void *cuda_stream)
+{
+    if (!ctx || !in || !opts || !out) return VTOKEN_EINVAL;
+    if (!in->num_requests || !in->bt_offsets || !in->bt_blocks || !in->tt_offsets || !in->tt_slots || !in->keep ||
+        !in->free_blocks || !in->num_free)
+        return VTOKEN_EINVAL;
+    if (!out->new_bt_offsets || !out->new_bt_blocks || !out->new_tt_slots || !out->freed_blocks ||
+        !out->req_status || !out->counts)
+        return VTOKEN_EINVAL;
+    if (opts->max_source_blocks < 0) return VTOKEN_EINVAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    PArgs a;
+    fill_args(a, ctx);
+    a.num_requests = in->num_requests;
+    a.bt_offsets = in->bt_offsets;
+    a.bt_blocks = in->bt_blocks;
+    a.tt_offsets = in->tt_offsets;
+    a.tt_slots = in->tt_slots;
+    a.keep = in->keep;
+    a.select = in->select;
+    a.protect = opts->protect;
+    a.thr_num = in->thr_num;
+    a.thr_den = in->thr_den;
+    a.util_num = opts->util_num;
+    a.util_den = opts->util_den;
+    a.theta_num = opts->theta_num;
+    a.theta_den = opts->theta_den;
+    a.max_sources = opts->max_source_blocks;
+    a.free_blocks = in->free_blocks;
+    a.num_free = in->num_free;
+    a.new_bt_offsets = out->new_bt_offsets;
+    a.new_bt_blocks = out->new_bt_blocks;
+    a.new_tt_slots = out->new_tt_slots;
+    a.freed_blocks = out->freed_blocks;
+    a.out_status = out->req_status;
+    a.out_counts = out->counts;
+
+    const int R = ctx->cfg.max_requests;
+    VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
+    VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
+    VTK_CUDA(ctx, cudaMemsetAsync(ctx->blk_src, 0, (size_t)ctx->cfg.num_blocks, st));
+    pp_count_kernel<0><<<R * PP_PARTS, PP_NT, 0, st>>>(a);
+    pp_blocks_kernel<<<R, PP_NT, 0, st>>>(a);
+    pp_count_kernel<1><<<R * PP_PARTS, PP_NT, 0, st>>>(a);
+    pp_scan_kernel<<<1, PP_SCAN_NT, 0, st>>>(a);
+    pp_assign_kernel<<<R * PP_PARTS, PP_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, cudaGetLastError());
+    ctx->has_plan = true;
+    return VTOKEN_OK;
+}
+
+int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *bt_offsets,
+                          const int32_t *bt_blocks, const int32_t *tt_offsets, const int32_t *tt_slots,
+                          const uint8_t *keep, int32_t *n_b, uint64_t *hist, int64_t *summary, void *cuda_stream)
+{
+    if (!ctx || !num_requests || !bt_offsets || !bt_blocks || !tt_offsets || !tt_slots || !n_b) return VTOKEN_EINVAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    PArgs a;
+    memset(&a, 0, sizeof(a));
+    fill_args(a, ctx);
+    a.num_requests = num_requests;
+    a.bt_offsets = bt_offsets;
+    a.bt_blocks = bt_blocks;
+    a.tt_offsets = tt_offsets;
+    a.tt_slots = tt_slots;
+    a.keep = keep;
+    a.n_b = n_b;
+    const int R = ctx->cfg.max_requests;
+    VTK_CUDA(ctx, cudaMemsetAsync(n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
+    pp_count_kernel<0><<<R * PP_PARTS, PP_NT, 0, st>>>(a);
+    if (hist) {
+        VTK_CUDA(ctx, cudaMemsetAsync(hist, 0, sizeof(uint64_t) * (size_t)(ctx->cfg.block_size + 1), st));
+        pp_hist_kernel<<<ctx->num_sms * 4, 256, 0, st>>>(num_requests, R, bt_offsets, bt_blocks, n_b,
+                                                         ctx->cfg.block_size, ctx->cfg.num_blocks,
+                                                         (unsigned long long *)hist, ctx->counts);
+    }
+    if (summary) pp_summary_kernel<<<1, 32, 0, st>>>(num_requests, R, bt_offsets, ctx->part_n, (long long *)summary);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+}  // extern "C"

@@ -104,6 +104,17 @@ class DeviceProblem:
                        counts=self.counts, select=self.select, thr_num=self.w.thr_num, thr_den=self.w.thr_den,
                        stream=stream)
 
+    def plan_partial(self, stream=None, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0)):
+        vt.vtoken_plan_partial(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
+                               bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
+                               keep=self.keep, free_blocks=self.free_blocks,
+                               num_free=self.num_free if num_free is None else num_free,
+                               new_bt_offsets=self.new_bt_offsets, new_bt_blocks=self.new_bt_blocks,
+                               new_tt_slots=self.new_tt_slots, freed_blocks=self.freed_blocks,
+                               req_status=self.req_status, counts=self.counts, select=self.select,
+                               thr_num=self.w.thr_num, thr_den=self.w.thr_den, protect=protect, util=util,
+                               max_source_blocks=max_source_blocks, theta=theta, stream=stream)
+
     def repack(self, stream=None):
         vt.vtoken_repack(self.ctx, stream=stream)
 

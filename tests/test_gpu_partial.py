@@ -1,0 +1,157 @@
+"""GPU parity of the eligibility metadata (per-block liveness, histogram, F) and of partial
+plans (low-utilisation sources, protected blocks, source bound, global trigger) against the
+oracle: tables, lists, counts and whole pools, bit-exact."""
+import numpy as np
+import pytest
+
+from oracle import vto
+from paper_2608_13263_b200 import binding as vt
+from paper_2608_13263_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+FILL_SEED = 1
+
+
+def host_pools(w):
+    k = np.stack([wl.fill_slab(FILL_SEED, 0, l, w.num_layers, w.slots_per_layer, w.row_elems)
+                  for l in range(w.num_layers)])
+    v = np.stack([wl.fill_slab(FILL_SEED, 1, l, w.num_layers, w.slots_per_layer, w.row_elems)
+                  for l in range(w.num_layers)])
+    return k, v
+
+
+def small_configs():
+    return [
+        wl.tiny(seed=0),
+        wl.llama8b_h2o(seed=0, requests=6, lo=300, hi=900, layers=2),
+        wl.mistral7b_random(seed=0, requests=17, lo=100, hi=500, layers=2, rho_lo=0.6, rho_hi=0.97),
+        wl.longctx_scissor(seed=0, requests=3, lo=3000, hi=6000, layers=1),
+        wl.steady_state(seed=0, requests=24, lo=100, hi=1500, layers=2),
+        wl.steady_state(seed=1, requests=24, lo=100, hi=1500, layers=1, block_size=32),
+    ]
+
+
+OPTION_SETS = [
+    dict(),                                               # reduces to the whole-request plan
+    dict(util=(1, 1)),                                    # fully live blocks stay
+    dict(util=(1, 2)),                                    # only blocks under 50 % utilisation move
+    dict(util=(1, 1), max_source_blocks=7),
+    dict(util=(3, 4), theta=(1, 4)),                      # the paper's default trigger
+    dict(theta=(99, 100)),                                # trigger never holds
+    dict(protect="prefix"),
+    dict(protect="prefix", util=(1, 1), max_source_blocks=20),
+]
+
+
+def run_partial(w, opts, num_free=None, whole_pool=True):
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    opts = dict(opts)
+    protect = None
+    if opts.get("protect") == "prefix":
+        protect = np.zeros(w.num_blocks, np.uint8)
+        for r in range(w.num_requests):
+            protect[w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]][:3]] = 1
+        opts["protect"] = protect
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    dopts = dict(opts)
+    if protect is not None:
+        dopts["protect"] = torch.from_numpy(protect).to(prob.device)
+    nf_dev = None if num_free is None else torch.tensor([num_free], dtype=torch.int32, device=prob.device)
+    prob.plan_partial(num_free=nf_dev, **dopts)
+    prob.repack()
+    out = prob.outputs()
+    p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                         w.free_blocks, w.select, w.thr_num, w.thr_den, num_free=num_free, **opts)
+    assert out["error_flags"] == 0
+    for n in ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"):
+        assert out[n] == getattr(p, n), n
+    assert np.array_equal(out["req_status"], p.req_status)
+    assert np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
+    assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
+    assert np.array_equal(out["freed_blocks"], p.freed_blocks)
+    if whole_pool:
+        k, v = host_pools(w)
+        vto.apply_moves_pools(k, v, p.move_src, p.move_dst, threads=2)
+        assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+        assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()
+    return out, p
+
+
+@pytest.mark.parametrize("opts", OPTION_SETS, ids=[str(i) for i in range(len(OPTION_SETS))])
+@pytest.mark.parametrize("w", small_configs(), ids=lambda w: f"{w.name}-S{w.block_size}")
+def test_partial_plans_small_whole_pool(w, opts):
+    run_partial(w, opts)
+
+
+def test_partial_plan_moves_fewer_rows_for_the_same_block_count():
+    w = wl.mistral7b_random(seed=3, requests=12, lo=200, hi=600, layers=1, rho_lo=0.8, rho_hi=0.98)
+    out_p, p = run_partial(w, dict(util=(1, 1)))
+    out_w, q = run_partial(w, dict())
+    both = (p.req_status == vto.REPACKED) & (q.req_status == vto.REPACKED)
+    assert both.any()
+    assert out_p["num_moves"] < out_w["num_moves"]
+    for r in np.flatnonzero(both):
+        assert (out_p["new_bt_offsets"][r + 1] - out_p["new_bt_offsets"][r]) == \
+               (out_w["new_bt_offsets"][r + 1] - out_w["new_bt_offsets"][r])
+
+
+def test_partial_free_list_cut():
+    w = wl.mistral7b_random(seed=11, requests=6, lo=30, hi=90, layers=1, heads=1, head_dim=8, block_size=4)
+    total = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                             w.free_blocks, util=(1, 1)).num_free_consumed
+    for c in range(total + 1):
+        run_partial(w, dict(util=(1, 1)), num_free=c, whole_pool=(c % 5 == 0))
+
+
+@pytest.mark.parametrize("w", small_configs(), ids=lambda w: f"{w.name}-S{w.block_size}")
+def test_block_liveness_matches_oracle(w):
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    n_b = torch.full((w.num_blocks,), -1, dtype=torch.int32, device=prob.device)
+    hist = torch.full((w.block_size + 1,), -1, dtype=torch.int64, device=prob.device)
+    summary = torch.full((2,), -1, dtype=torch.int64, device=prob.device)
+    vt.vtoken_block_liveness(prob.ctx, num_requests=prob.num_requests, bt_offsets=prob.bt_offsets,
+                             bt_blocks=prob.bt_blocks, tt_offsets=prob.tt_offsets, tt_slots=prob.tt_slots,
+                             keep=prob.keep, n_b=n_b, hist=hist, summary=summary)
+    torch.cuda.synchronize()
+    o_nb, o_hist, o_live, o_alloc = vto.block_liveness(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks,
+                                                       w.tt_offsets, w.tt_slots, w.keep)
+    assert np.array_equal(n_b.cpu().numpy(), o_nb)
+    assert np.array_equal(hist.cpu().numpy(), o_hist)
+    assert summary.cpu().numpy().tolist() == [o_live, o_alloc]
+    prob.close()
+
+
+def test_partial_plan_full_size_steady_state_tables():
+    """The partial planner at the benchmark's largest table size (512 requests, 2.2 M entries):
+    all tables and lists against the oracle; pools verified through the origin map."""
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem, origin_map
+    free_bytes, _ = torch.cuda.mem_get_info()
+    requests = 512
+    while True:
+        w = wl.steady_state(seed=0, requests=requests)
+        if 2 * w.pool_bytes + (3 << 30) < free_bytes or requests == 1:
+            break
+        requests //= 2
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    prob.plan_partial(util=(1, 1), theta=(1, 4))
+    prob.repack()
+    out = prob.outputs()
+    p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                         w.free_blocks, w.select, w.thr_num, w.thr_den, util=(1, 1), theta=(1, 4))
+    assert out["error_flags"] == 0 and out["num_moves"] == p.num_moves > 10000
+    assert np.array_equal(out["req_status"], p.req_status)
+    assert np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
+    assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
+    assert np.array_equal(out["freed_blocks"], p.freed_blocks)
+    assert prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst)) == 0
+    prob.close()
+    del prob
+    torch.cuda.empty_cache()

@@ -226,23 +226,28 @@ def run_cuda(args):
         need = 2 * w.pool_bytes + (1 << 30)
 
     prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas)
+    partial_opts = dict(util=(1, 1), theta=(1, 4))     # fully live blocks stay; the paper's default trigger F > 0.25
+    if args.plan_mode == "partial":
+        do_plan = lambda st: prob.plan_partial(stream=st, **partial_opts)
+    else:
+        do_plan = lambda st: prob.plan(stream=st)
     grid = vt.vtoken_copy_grid(prob.ctx)
     side = torch.cuda.Stream(device=dev)
 
     # ---- capture: whole path, and the copy alone -------------------------------------------
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
-        prob.plan(stream=side)
+        do_plan(side)
         prob.repack(stream=side)
     side.synchronize()
     g_all, g_copy, g_plan = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
     with torch.cuda.graph(g_all, stream=side):
-        prob.plan(stream=torch.cuda.current_stream())
+        do_plan(torch.cuda.current_stream())
         prob.repack(stream=torch.cuda.current_stream())
     with torch.cuda.graph(g_copy, stream=side):
         prob.repack(stream=torch.cuda.current_stream())
     with torch.cuda.graph(g_plan, stream=side):
-        prob.plan(stream=torch.cuda.current_stream())
+        do_plan(torch.cuda.current_stream())
     out = prob.outputs()
     M = out["num_moves"]
     bytes_per_step = 2 * M * w.token_bytes
@@ -318,14 +323,25 @@ def run_cuda(args):
     parity = "skipped"
     if not args.no_verify:
         from oracle import vto   # the checker: tests/bench only
-        p = vto.plan_workload(w)
+        pw = vto.plan_workload(w)                       # what the end-to-end leg (whole-request plan) must return
+        if args.plan_mode == "partial":
+            p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots,
+                                 w.keep, w.free_blocks, w.select, w.thr_num, w.thr_den, **partial_opts)
+            # the end-to-end leg wrote the whole-request layout: restore the pools, replay the timed graph once
+            prob.fill_pools()
+            torch.cuda.synchronize(dev)
+            with torch.cuda.stream(side):
+                g_all.replay()
+            side.synchronize()
+        else:
+            p = pw
         ok = (out["error_flags"] == 0 and c_host["error_flags"] == 0 and M == p.num_moves
               and np.array_equal(out["new_tt_slots"], p.new_tt_slots)
               and np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
               and np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
               and np.array_equal(out["freed_blocks"], p.freed_blocks)
               and np.array_equal(out["req_status"], p.req_status)
-              and np.array_equal(h_out["new_tt_slots"].numpy()[:T], p.new_tt_slots))
+              and np.array_equal(h_out["new_tt_slots"].numpy()[:T], pw.new_tt_slots))
         bad_words = prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst))
         parity = "ok" if (ok and bad_words == 0) else f"FAILED (tables_ok={ok}, mismatching_words={bad_words})"
 
@@ -376,13 +392,15 @@ def run_cuda(args):
                    "l2": "moved bytes per step exceed the 126 MB L2 (no flush needed)" if bytes_per_step > 4 * 126e6
                          else "moved bytes per step fit in L2: launch-bound parity configuration",
                    "launch": "CUDA graph (plan + copy) replayed on a side stream", "copy_grid": grid,
+                   "plan_mode": args.plan_mode if args.plan_mode == "whole" else
+                                "partial: sources = blocks that are not fully live, trigger F > 1/4",
                    "gpu": f"{torch.cuda.get_device_name(dev)} {str(torch.cuda.get_device_properties(dev).uuid)[-12:]}",
                    "parallelism": f"{ranks.world} independent pools, no collective"},
         "tokens_per_s": all_tokens / (ms_per_step * 1e-3),
         "frac_of_measured_hbm_peak": value / (peak * ranks.world),
         "frac_of_nominal_8TBs": value / (NOMINAL_HBM_GBS * ranks.world),
         "plan_us": plan_total_ms / args.steps * 1e3, "copy_ms": copy_ms,
-        "clocks": clocks, "gpu_launches": KERNELS_PER_STEP * args.steps,
+        "clocks": clocks, "gpu_launches": (KERNELS_PER_STEP if args.plan_mode == "whole" else KERNELS_PER_STEP + 2) * args.steps,
         "e2e": {"value": e2e_value, "unit": "GB/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
                 "what": "vtoken_repack_host: pinned host tables -> device, plan, copy, every output table -> host, sync; "
@@ -592,6 +610,8 @@ def main():
     ap.add_argument("--proxy", action="store_true", help="also run the repack beside a decode-read proxy")
     ap.add_argument("--proxy-ctas", type=int, default=0)
     ap.add_argument("--runtime", action="store_true", help="also time the token-table runtime kernels")
+    ap.add_argument("--plan-mode", default="whole", choices=["whole", "partial"],
+                    help="whole-request compaction (default) or the partial planner that keeps fully live blocks")
     ap.add_argument("--block-size", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

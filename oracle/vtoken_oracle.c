@@ -400,8 +400,9 @@ int vto_block_liveness(int32_t R, int32_t S, int32_t NB, const int32_t *bt_offse
         for (int32_t k = 0; k <= S; ++k) hist[k] = 0;
         for (int32_t j = 0; j < bt_offsets[R]; ++j) {
             const int32_t b = bt_blocks[j];
-            if (b < 0 || b >= NB || n_b[b] > S) return VTO_EINVAL;
-            ++hist[n_b[b]];
+            if (b < 0 || b >= NB) return VTO_EINVAL;
+            /* a block referenced by several requests (shared prefix) counts one per reference: clip */
+            ++hist[n_b[b] > S ? S : n_b[b]];
         }
     }
     if (live_total) *live_total = live;

@@ -320,6 +320,53 @@ def steady_state(seed: int = 0, requests: int = 512, lo: int = 256, hi: int = 81
                      keeps, rng, seed, thr=thr, notes={"g_mean": float(g.mean())})
 
 
+def shared_prefix(seed: int = 0, groups: int = 4, degree: int = 4, prefix_len: int = 8192, suffix_len: int = 8192,
+                  layers: int = 32, heads: int = 8, head_dim: int = 128, block_size: int = 16,
+                  budget_frac: float = 0.2):
+    """Prefix-cache workload shaped like the paper's compatibility experiment (Sec. 5, Table 1):
+    ``groups`` prompts, each shared by ``degree`` requests that reference the SAME physical
+    blocks for the first ``prefix_len`` tokens and own a private suffix of ``suffix_len`` tokens;
+    H2O-style mask per request over prefix + suffix.  ``prefix_len`` must be a multiple of the
+    block size so that shared and private blocks do not mix.  Returns (workload, protect) where
+    protect[b] = 1 marks the shared blocks, which a plan must leave in place."""
+    S = block_size
+    assert prefix_len % S == 0
+    rng = np.random.Generator(np.random.PCG64(seed))
+    R = groups * degree
+    n = prefix_len + suffix_len
+    keeps = []
+    for r in range(R):
+        score = rng.lognormal(0.0, 1.5, size=n)
+        keeps.append(h2o_mask(np.arange(n), n, score, math.ceil(budget_frac * n)))
+    pre_blocks = prefix_len // S
+    suf_blocks = -(-suffix_len // S)
+    private_live = [int(k[prefix_len:].sum()) for k in keeps]
+    dst_total = sum(-(-x // S) for x in private_live)
+    NB = groups * pre_blocks + R * suf_blocks + dst_total + 256
+    perm = rng.permutation(NB).astype(np.int32)
+    shared = [perm[g * pre_blocks:(g + 1) * pre_blocks] for g in range(groups)]
+    cursor = groups * pre_blocks
+    bts, tts = [], []
+    for r in range(R):
+        own = perm[cursor:cursor + suf_blocks]
+        cursor += suf_blocks
+        blocks = np.concatenate([shared[r // degree], own])
+        pos = np.arange(n)
+        bts.append(blocks)
+        tts.append((blocks[pos // S].astype(np.int64) * S + pos % S).astype(np.int32))
+    free_blocks = np.sort(perm[cursor:]).astype(np.int32)
+    protect = np.zeros(NB, np.uint8)
+    protect[np.concatenate(shared)] = 1
+    bt_offsets = np.concatenate([[0], np.cumsum([len(b) for b in bts])]).astype(np.int32)
+    tt_offsets = (np.arange(R + 1) * n).astype(np.int32)
+    w = Workload(name="shared_prefix", num_layers=layers, num_kv_heads=heads, head_dim=head_dim, block_size=S,
+                 num_blocks=NB, bt_offsets=bt_offsets, bt_blocks=np.concatenate(bts).astype(np.int32),
+                 tt_offsets=tt_offsets, tt_slots=np.concatenate(tts), keep=np.concatenate(keeps).astype(np.uint8),
+                 free_blocks=free_blocks, seed=seed, notes={"degree": degree, "groups": groups,
+                                                            "prefix_blocks": pre_blocks})
+    return w, protect
+
+
 CONFIGS = {
     "tiny": tiny,
     "llama8b_h2o": llama8b_h2o,

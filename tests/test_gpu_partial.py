@@ -155,3 +155,29 @@ def test_partial_plan_full_size_steady_state_tables():
     prob.close()
     del prob
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("degree", [1, 2, 4, 8])
+def test_shared_prefix_workload(degree):
+    """Synthetic prefix-cache workload: shared blocks protected, private suffixes repacked."""
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    w, protect = wl.shared_prefix(seed=degree, groups=2, degree=degree, prefix_len=256, suffix_len=320, layers=2,
+                                  heads=2, head_dim=64)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    prob.plan_partial(protect=torch.from_numpy(protect).to(prob.device))
+    prob.repack()
+    out = prob.outputs()
+    p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                         w.free_blocks, protect=protect)
+    assert out["error_flags"] == 0 and out["num_admitted"] == p.num_admitted == w.num_requests
+    assert np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
+    assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
+    assert np.array_equal(out["freed_blocks"], p.freed_blocks)
+    assert not (set(out["freed_blocks"].tolist()) & set(np.flatnonzero(protect).tolist()))
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()

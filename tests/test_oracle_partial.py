@@ -183,3 +183,40 @@ def test_bruteforce_all_masks_one_request():
         for util in (None, Fraction(1, 1), Fraction(2, 3), Fraction(1, 3)):
             for c in range(3):
                 _compare(S, [bt], [tt], [list(mask)], np.array([5, 4][:c], np.int32), None, None, (), util, 0, None, 8)
+
+
+def test_shared_prefix_blocks_are_skipped_and_private_suffixes_reclaimed():
+    """Prefix-cache compatibility (Sec. 5, Table 1): every shared-prefix block is left in place for
+    every sharing degree, private suffix blocks are reclaimed, and each request's logical view is
+    unchanged."""
+    for degree in (1, 2, 4):
+        w, protect = wl.shared_prefix(seed=degree, groups=2, degree=degree, prefix_len=64, suffix_len=96, layers=1,
+                                      heads=1, head_dim=8, block_size=4)
+        S = w.block_size
+        p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                             w.free_blocks, protect=protect)
+        shared = set(np.flatnonzero(protect).tolist())
+        assert p.num_admitted == w.num_requests
+        assert not (set(p.freed_blocks.tolist()) & shared)                       # 100 % of shared candidates skipped
+        assert not (set((p.move_src // S).tolist()) & shared)
+        assert not (set((p.move_dst // S).tolist()) & shared)
+        pre = w.notes["prefix_blocks"]
+        live = (w.tt_slots >= 0) & (w.keep != 0)
+        slab = np.arange(w.slots_per_layer * 2, dtype=np.int64).reshape(-1, 2)
+        before = slab.copy()
+        vto.apply_moves_slab(slab, p.move_src, p.move_dst)
+        for r in range(w.num_requests):
+            t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
+            old = w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]]
+            new = p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]]
+            assert new[:pre].tolist() == old[:pre].tolist()                      # the prefix stays, in order
+            n_private = int(live[t0 + 64:t1].sum())
+            assert len(new) == pre + -(-n_private // S)                          # suffix packed densely
+            a = vto.gather_logical(before, w.tt_slots[t0:t1], w.keep[t0:t1])
+            b = vto.gather_logical(slab, p.new_tt_slots[t0:t1])
+            assert np.array_equal(a, b)
+        # the shared slots are referenced once per sharing request, private slots exactly once
+        occ = p.new_tt_slots[p.new_tt_slots >= 0]
+        counts = np.bincount(occ, minlength=w.slots_per_layer)
+        assert counts[np.isin(np.arange(w.slots_per_layer) // S, list(shared))].max() <= degree
+        assert counts[~np.isin(np.arange(w.slots_per_layer) // S, list(shared))].max() <= 1

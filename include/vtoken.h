@@ -167,6 +167,24 @@ int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const in
                           int32_t layer_begin, int32_t layer_end, void *out_k, void *out_v,
                           int64_t out_capacity_tokens, int32_t *out_offsets, void *cuda_stream);
 
+/* Online relocation check (Sec. 5, "Relocation Correctness": the ordered retained token ids are
+ * hashed together with their K/V contents before and after a relocation).  The paper does not
+ * name the hash; this library fixes one that any evaluation order reproduces bit for bit: for a
+ * request whose active tokens have rank i = 0, 1, ... and logical ids t_i, over the slabs
+ * s = 0 .. 2*(layer_end-layer_begin)-1 (K layers first, then V layers) and the 8-byte
+ * little-endian words w_j of a token's row,
+ *     digest = sum of mix(w_j ^ mix((((i * A + t_i) * B + s) * C + j)))  mod 2^64,
+ * mix = splitmix64 finaliser, A = 0x9E3779B97F4A7C15, B = 0xD1B54A32D192ED03, C = 0x8CB92BA72F3D8DD7.
+ * Equal digests before (old table + keep) and after (new table) a repack show token conservation
+ * (I1) without materialising the rows.  out_digest: DEVICE uint64 [max_requests] (zeroed by the
+ * call); out_offsets: DEVICE int32 [R+1] or NULL, first active-token index of each request (the
+ * differences are the active counts).  Same selection arguments and scratch sharing as
+ * vtoken_gather_logical. */
+int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                          const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                          int32_t layer_begin, int32_t layer_end, uint64_t *out_digest, int32_t *out_offsets,
+                          void *cuda_stream);
+
 /* Copies the context's counts of the last plan (with the flags raised by repack and
  * gather_logical since) to HOST memory.  Synchronises the stream: the only call that does. */
 int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stream);

@@ -332,3 +332,24 @@ def plan_partial(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_
     return Plan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
                 freed[:c.num_freed].copy(), status[:R].copy(), msrc[:c.num_moves].copy(), mdst[:c.num_moves].copy(),
                 c.num_moves, c.num_dst_blocks, c.num_freed, c.num_free_consumed, c.num_admitted, c.num_deferred)
+
+
+# ---- online relocation check ------------------------------------------------------------------
+def digest_logical(k_pool: np.ndarray, v_pool: np.ndarray, tt_slots, keep=None, layer_begin=0, layer_end=None):
+    """Order-sensitive digest of one request's active tokens over pools [L, num_slots, row].
+    Returns (digest as Python int, number of active tokens)."""
+    assert k_pool.ndim == 3 and k_pool.shape == v_pool.shape
+    assert k_pool.flags["C_CONTIGUOUS"] and v_pool.flags["C_CONTIGUOUS"]
+    tt_slots, keep = _i32(tt_slots), _u8(keep)
+    L, ns, row = k_pool.shape
+    if layer_end is None:
+        layer_end = L
+    d = ctypes.c_uint64(0)
+    n = ctypes.c_int32(0)
+    rc = lib().vto_digest_logical(ctypes.c_void_p(k_pool.ctypes.data), ctypes.c_void_p(v_pool.ctypes.data),
+                                  ctypes.c_int64(0), ctypes.c_int64(ns), ctypes.c_int64(row * k_pool.itemsize),
+                                  ctypes.c_int32(layer_begin), ctypes.c_int32(layer_end), _p(tt_slots, np.int32),
+                                  _p(keep, np.uint8), ctypes.c_int32(len(tt_slots)), ctypes.byref(d), ctypes.byref(n))
+    if rc != 0:
+        raise ValueError(f"vto_digest_logical failed: {rc}")
+    return d.value, n.value

@@ -517,6 +517,48 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
     return VTO_OK;
 }
 
+static uint64_t mix64(uint64_t x)                           /* splitmix64 finaliser */
+{
+    x ^= x >> 30;
+    x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27;
+    x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return x;
+}
+
+int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t layer_stride_bytes, int64_t num_slots,
+                       int64_t row_bytes, int32_t layer_begin, int32_t layer_end, const int32_t *tt_slots,
+                       const uint8_t *keep, int32_t len, uint64_t *digest, int32_t *num_active)
+{
+    if (!k_pool || !v_pool || !tt_slots || !digest || row_bytes < 8 || row_bytes % 8 != 0) return VTO_EINVAL;
+    if (layer_begin < 0 || layer_end <= layer_begin || len < 0) return VTO_EINVAL;
+    if (layer_stride_bytes == 0) layer_stride_bytes = num_slots * row_bytes;
+    const uint64_t A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull;
+    const int32_t nl = layer_end - layer_begin;
+    uint64_t sum = 0;
+    int32_t i = 0;                                           /* rank among the active tokens */
+    for (int32_t t = 0; t < len; ++t) {
+        if (!is_live(tt_slots, keep, t)) continue;
+        if (tt_slots[t] >= num_slots) return VTO_EINVAL;
+        for (int32_t s = 0; s < 2 * nl; ++s) {               /* K layers, then V layers */
+            const uint8_t *pool = s < nl ? k_pool : v_pool;
+            const int32_t layer = layer_begin + (s < nl ? s : s - nl);
+            const uint8_t *row = pool + (int64_t)layer * layer_stride_bytes + (int64_t)tt_slots[t] * row_bytes;
+            for (int64_t j = 0; j < row_bytes / 8; ++j) {
+                uint64_t w = 0;
+                for (int b = 7; b >= 0; --b) w = (w << 8) | row[j * 8 + b];       /* little-endian word */
+                const uint64_t where = ((((uint64_t)i * A + (uint64_t)t) * B + (uint64_t)s) * C + (uint64_t)j);
+                sum += mix64(w ^ mix64(where));
+            }
+        }
+        ++i;
+    }
+    *digest = sum;
+    if (num_active) *num_active = i;
+    return VTO_OK;
+}
+
 int vto_openmp_threads(void)
 {
 #ifdef _OPENMP

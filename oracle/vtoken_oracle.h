@@ -181,6 +181,20 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      int32_t *freed_blocks, int32_t *req_status,
                      int32_t *move_src, int32_t *move_dst, vto_counts *counts);
 
+/* ---- online relocation check (Sec. 5, "Relocation Correctness") ---------------------------------
+ * The paper hashes the ordered retained token ids together with their K/V contents before and
+ * after a relocation.  It does not name the hash; this build fixes one that can be evaluated in
+ * any order (a sum of per-word terms, each bound to its position): for a request whose active
+ * tokens are t_0 < t_1 < ... (rank i, logical id t_i), over slabs s = 0 .. 2*(layer_end-layer_begin)-1
+ * (K layers first, then V layers) and the 8-byte little-endian words w_j of the token's row,
+ *     digest = sum over (i, s, j) of mix(w_j ^ mix((((i * A + t_i) * B + s) * C + j)))   mod 2^64
+ * with mix = the splitmix64 finaliser and A, B, C the odd constants in the source.  A lost,
+ * duplicated, reordered or altered token changes the digest.  row_bytes must be a multiple of 8.
+ * Pools are [L][num_slots][row_bytes] with layer_stride_bytes between layers (0 = dense). */
+int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t layer_stride_bytes, int64_t num_slots,
+                       int64_t row_bytes, int32_t layer_begin, int32_t layer_end, const int32_t *tt_slots,
+                       const uint8_t *keep, int32_t len, uint64_t *digest, int32_t *num_active);
+
 int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */
 
 #ifdef __cplusplus

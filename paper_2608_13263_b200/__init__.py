@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     VtokenError,
     vtoken_apply_moves,
     vtoken_block_liveness,
+    vtoken_digest_logical,
     vtoken_plan_partial,
     vtoken_build_slot_mapping,
     vtoken_evict_tokens,
@@ -30,4 +31,4 @@ from .binding import (  # noqa: F401
 __all__ = ["VtokenError", "vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack",
            "vtoken_gather_logical", "vtoken_read_counts", "vtoken_repack_host", "vtoken_copy_grid",
            "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens", "vtoken_sync_new_tokens",
-           "vtoken_build_slot_mapping", "vtoken_apply_moves", "vtoken_block_liveness", "vtoken_plan_partial"]
+           "vtoken_build_slot_mapping", "vtoken_apply_moves", "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical"]

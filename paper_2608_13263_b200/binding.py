@@ -21,7 +21,7 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
            "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
-           "vtoken_block_liveness", "vtoken_plan_partial"]
+           "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical"]
 
 
 class VtokenError(RuntimeError):
@@ -120,6 +120,7 @@ def load():
         lib.vtoken_build_slot_mapping.argtypes = [ctypes.c_void_p] * 8 + [ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
         lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 9
         lib.vtoken_block_liveness.argtypes = [ctypes.c_void_p] * 11
+        lib.vtoken_digest_logical.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 3
         lib.vtoken_plan_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
                                             ctypes.POINTER(PlanOut), ctypes.c_void_p]
         _lib = lib
@@ -289,3 +290,10 @@ def vtoken_plan_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets,
     po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1])
     _check(load().vtoken_plan_partial(ctx, ctypes.byref(pin), ctypes.byref(po), ctypes.byref(pout), _stream(stream)),
            "vtoken_plan_partial", ctx)
+
+
+def vtoken_digest_logical(ctx, *, num_requests, tt_offsets, tt_slots, keep, select, layer_begin, layer_end, out_digest,
+                          out_offsets=None, stream=None) -> None:
+    _check(load().vtoken_digest_logical(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                                        _ptr(select), layer_begin, layer_end, _ptr(out_digest), _ptr(out_offsets),
+                                        _stream(stream)), "vtoken_digest_logical", ctx)

@@ -24,7 +24,7 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
-                    ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
+                    ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->blk_src,
                     ctx->stage.num_requests, ctx->stage.num_free, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
@@ -117,6 +117,9 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->counts, 1);
     A(&ctx->g_src, cfg->max_tokens);
     A(&ctx->g_total, 1);
+    A(&ctx->g_ids, cfg->max_tokens);
+    A(&ctx->g_req, cfg->max_tokens);
+    A(&ctx->g_offsets, (int64_t)cfg->max_requests + 1);
     A(&ctx->part_src, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
     A(&ctx->req_ns, cfg->max_requests);
     A(&ctx->req_nsrc, cfg->max_requests);

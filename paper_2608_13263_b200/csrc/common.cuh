@@ -40,6 +40,9 @@ struct vtoken_ctx {
     // gather_logical scratch (DEVICE)
     int32_t *g_src;            // [max_tokens] source slot of each output row
     int32_t *g_total;          // [1] output rows
+    int32_t *g_ids;            // [max_tokens] logical id of each output row (digest)
+    int32_t *g_req;            // [max_tokens] request of each output row (digest)
+    int32_t *g_offsets;        // [max_requests + 1] first output row of each request (digest)
 
     // device staging of vtoken_repack_host (DEVICE), allocated on first use
     struct {

@@ -14,7 +14,9 @@ constexpr int G_PARTS = VTK_PLAN_PARTS;
 struct GatherArgs {
     const int32_t *num_requests, *tt_offsets, *tt_slots;
     const uint8_t *keep, *select;
-    int32_t *req_n, *part_n, *out_offsets, *g_src, *g_ids, *g_total;   // g_ids: logical id of each output row, or NULL
+    int32_t *req_n, *part_n, *out_offsets, *g_src, *g_total;
+    int32_t *g_ids, *g_req;      // logical id / request of each output row, or NULL
+    unsigned long long *digest;  // per-request digest (digest kernel only)
     vtoken_counts *counts;
     const uint8_t *k_pool, *v_pool;
     uint8_t *out_k, *out_v;
@@ -134,6 +136,7 @@ __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
         if (live && i < cap) {
             a.g_src[i] = slot;
             if (a.g_ids != nullptr) a.g_ids[i] = (int32_t)(t - t0);
+            if (a.g_req != nullptr) a.g_req[i] = r;
         }
     }
 }
@@ -182,7 +185,99 @@ __global__ void __launch_bounds__(GC_NT) gather_copy_kernel(GatherArgs a)
     }
 }
 
+__device__ __forceinline__ unsigned long long g_mix64(unsigned long long x)   // splitmix64 finaliser
+{
+    x ^= x >> 30;
+    x *= 0xBF58476D1CE4E5B9ull;
+    x ^= x >> 27;
+    x *= 0x94D049BB133111EBull;
+    x ^= x >> 31;
+    return x;
+}
+
+// Relocation digest (Sec. 5 of the paper hashes ordered retained ids with their K/V contents):
+//   digest[r] = sum over (rank i, slab s, 8-byte word j) of mix(w ^ mix((((i*A + t_i)*B + s)*C + j)))
+// a sum of position-bound terms, so any evaluation order gives the same 64-bit value.
+// One warp per (slab, output row); lanes take 16-byte pieces of the row.
+__global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
+{
+    const unsigned long long A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull;
+    const int64_t n = *a.g_total;
+    const int nl = a.layer_end - a.layer_begin;
+    const int64_t total = n * nl * 2;
+    const int lane = vtk_lane();
+    const int64_t nwarps = (int64_t)gridDim.x * (GC_NT / 32);
+    const int row_vecs = (int)(a.row_bytes >> 4);
+    for (int64_t u = (int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5); u < total; u += nwarps) {
+        const int slab = (int)(u / n);
+        const int64_t idx = u - (int64_t)slab * n;
+        const int li = slab < nl ? slab : slab - nl;
+        const uint8_t *pool = slab < nl ? a.k_pool : a.v_pool;
+        const int32_t src = a.g_src[idx];
+        const int r = a.g_req[idx];
+        const unsigned long long i = (unsigned long long)(idx - a.out_offsets[r]);
+        const unsigned long long t = (unsigned long long)a.g_ids[idx];
+        const unsigned long long base = ((i * A + t) * B + (unsigned long long)slab) * C;
+        const uint4 *sp = reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
+                                                          (int64_t)src * a.row_bytes);
+        unsigned long long sum = 0;
+        for (int c = lane; c < row_vecs; c += 32) {
+            const uint4 v = ld_stream(sp + c);
+            const unsigned long long w0 = ((unsigned long long)v.y << 32) | v.x;
+            const unsigned long long w1 = ((unsigned long long)v.w << 32) | v.z;
+            sum += g_mix64(w0 ^ g_mix64(base + 2ull * c));
+            sum += g_mix64(w1 ^ g_mix64(base + 2ull * c + 1ull));
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
+        if (lane == 0 && sum != 0) atomicAdd(&a.digest[r], sum);
+    }
+}
+
 }  // namespace
+
+extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                                     const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
+                                     int32_t layer_begin, int32_t layer_end, uint64_t *out_digest,
+                                     int32_t *out_offsets, void *cuda_stream)
+{
+    if (!ctx || !num_requests || !tt_offsets || !tt_slots || !out_digest) return VTOKEN_EINVAL;
+    if (layer_begin < 0 || layer_end > ctx->cfg.num_layers || layer_begin >= layer_end) return VTOKEN_EINVAL;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    GatherArgs a;
+    a.num_requests = num_requests;
+    a.tt_offsets = tt_offsets;
+    a.tt_slots = tt_slots;
+    a.keep = keep;
+    a.select = select;
+    a.req_n = ctx->req_n;
+    a.part_n = ctx->part_n;
+    a.out_offsets = out_offsets ? out_offsets : ctx->g_offsets;
+    a.g_src = ctx->g_src;
+    a.g_ids = ctx->g_ids;
+    a.g_req = ctx->g_req;
+    a.digest = (unsigned long long *)out_digest;
+    a.g_total = ctx->g_total;
+    a.counts = ctx->counts;
+    a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
+    a.v_pool = (const uint8_t *)ctx->cfg.v_pool;
+    a.out_k = a.out_v = nullptr;
+    a.layer_stride = ctx->layer_stride;
+    a.row_bytes = ctx->row_bytes;
+    a.slots_per_layer = ctx->slots_per_layer;
+    a.out_capacity = ctx->cfg.max_tokens;
+    a.max_tokens = ctx->cfg.max_tokens;
+    a.layer_begin = layer_begin;
+    a.layer_end = layer_end;
+    a.max_requests = ctx->cfg.max_requests;
+    VTK_CUDA(ctx, cudaMemsetAsync(out_digest, 0, sizeof(uint64_t) * (size_t)ctx->cfg.max_requests, st));
+    gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
+    gather_scan_kernel<<<1, 1024, 0, st>>>(a);
+    gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
+    gather_digest_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
 
 int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                       const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
@@ -200,6 +295,8 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.out_offsets = out_offsets;
     a.g_src = ctx->g_src;
     a.g_ids = nullptr;
+    a.g_req = nullptr;
+    a.digest = nullptr;
     a.g_total = ctx->g_total;
     a.counts = ctx->counts;
     a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
@@ -243,6 +340,8 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.out_offsets = out_offsets;
     a.g_src = out_slots;
     a.g_ids = out_token_ids;
+    a.g_req = nullptr;
+    a.digest = nullptr;
     a.g_total = ctx->g_total;
     a.counts = ctx->counts;
     a.k_pool = a.v_pool = nullptr;

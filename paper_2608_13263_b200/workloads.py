@@ -320,6 +320,19 @@ def steady_state(seed: int = 0, requests: int = 512, lo: int = 256, hi: int = 81
                      keeps, rng, seed, thr=thr, notes={"g_mean": float(g.mean())})
 
 
+def streaming_window(seed: int = 0, requests: int = 64, lo: int = 1024, hi: int = 4096, sinks: int = 4,
+                     window: int = 512, layers: int = 32, heads: int = 8, head_dim: int = 128,
+                     block_size: int = 16) -> Workload:
+    """StreamingLLM / sliding-window style mask (Sec. 2.2): the first ``sinks`` tokens (attention
+    sinks) and the last ``window`` tokens stay, everything between is evicted.  Whole runs of
+    blocks become empty, the sink block and the first window block stay partially live."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    lens = rng.integers(lo, hi + 1, size=requests)
+    keeps = [(np.arange(int(n)) < sinks) | (np.arange(int(n)) >= int(n) - window) for n in lens]
+    return _assemble("streaming_window", (layers, heads, head_dim), block_size, lens, [None] * requests, keeps,
+                     rng, seed)
+
+
 def shared_prefix(seed: int = 0, groups: int = 4, degree: int = 4, prefix_len: int = 8192, suffix_len: int = 8192,
                   layers: int = 32, heads: int = 8, head_dim: int = 128, block_size: int = 16,
                   budget_frac: float = 0.2):

@@ -29,6 +29,7 @@ def small_configs():
         wl.longctx_scissor(seed=0, requests=3, lo=3000, hi=6000, layers=1),
         wl.steady_state(seed=0, requests=24, lo=100, hi=1500, layers=2),
         wl.steady_state(seed=1, requests=24, lo=100, hi=1500, layers=1, block_size=32),
+        wl.streaming_window(seed=0, requests=9, lo=200, hi=1500, window=100, layers=1),
     ]
 
 

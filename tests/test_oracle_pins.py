@@ -43,6 +43,7 @@ def small_workloads():
     yield wl.steady_state(seed=4, requests=12, lo=100, hi=600, layers=1, heads=1, head_dim=8)
     yield wl.steady_state(seed=5, requests=12, lo=100, hi=600, layers=1, heads=1, head_dim=8,
                           block_size=32)
+    yield wl.streaming_window(seed=6, requests=6, lo=60, hi=400, window=48, layers=1, heads=1, head_dim=8)
 
 
 # ------------------------------------------------------------------------------------------

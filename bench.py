@@ -316,7 +316,9 @@ def run_cuda(args):
     side.synchronize()
     e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
     e2e_ms = ranks.max(max(e0.elapsed_time(e1) / args.steps, e2e_wall_ms))
-    e2e_value = all_bytes / (e2e_ms * 1e-3) / 1e9
+    # the end-to-end call always runs the whole-request plan: count the bytes it moved
+    e2e_bytes = ranks.sum(2 * c_host["num_moves"] * w.token_bytes)
+    e2e_value = e2e_bytes / (e2e_ms * 1e-3) / 1e9
     clocks = sampler.stop()      # sampled over every timed region above
 
     # ---- parity at full size, in the launch configuration that was timed --------------------

@@ -165,10 +165,13 @@ constexpr int BULK_MAX_STAGES = 12;
 // of item k (bounded), (3) one lane stores them with a single cp.async.bulk shared->global.
 //
 // Nothing on that path waits for a global-memory read of the plan: the entries of an item
-// (destination block id, source slot of the lane's row) are fetched two items ahead into
-// registers, what the store side needs (destination address, valid-row mask) is parked in
-// shared memory at issue time, and item indices advance by additions (no per-step division).
-__global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages, int depth)
+// (destination block id, source slot of the lane's row) are fetched `ahead` (1 or 2) items
+// early into registers, what the store side needs (destination address, valid-row mask) is
+// parked in shared memory at issue time, and item indices advance by additions (no per-step
+// division).  `ahead` is a run-time argument on purpose: measured on B200, the build in which
+// it is a compile-time constant schedules the issue path 2-3 % slower (6.20 vs 6.32 TB/s on the
+// Llama-shaped workload, same box, alternating runs).
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages, int depth, int ahead)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint64_t bars[BULK_MAX_WARPS * BULK_MAX_STAGES];
@@ -225,7 +228,7 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         }
     };
     fetch(e1);
-    fetch(e2);
+    if (ahead == 2) fetch(e2);
 
     int s_issue = 0, issued = 0, stored = 0;
     auto issue = [&]() {
@@ -233,8 +236,12 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         const int s = s_issue;
         s_issue = s_issue + 1 == stages ? 0 : s_issue + 1;
         const Entry e = e1;
-        e1 = e2;
-        fetch(e2);                                   // in flight for two steps before it is used
+        if (ahead == 2) {
+            e1 = e2;
+            fetch(e2);                               // in flight for two steps before it is used
+        } else {
+            fetch(e1);                               // in flight for one step
+        }
         const bool valid = e.src >= 0 && e.dst0 >= 0;
         uint8_t *base = slab_base(a, e.slab);
         uint8_t *stg = my_smem + (size_t)s * stage_bytes;
@@ -303,13 +310,14 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctx->copy_smem = 0;
         ctas_per_sm = 8;
     } else {
-        // tuning knobs "warps,stages,rows,depth": warps per CTA, ring size, rows per item, loads
-        // issued ahead.  Defaults: 8 warps x 6 stages x 4 KB items = 192 KB of staging per SM, two
+        // tuning knobs "warps,stages,rows,depth,ahead": warps per CTA, ring size, rows per item, loads
+        // issued ahead, plan entries fetched ahead.  Defaults: 8 warps x 6 stages x 4 KB items = 192 KB of staging per SM, two
         // items loading ahead, three stores in flight per warp.  Measured on B200: shapes from 4 to
         // 32 KB per item land within about 3 % of each other; below 4 KB per warp-step with only
         // 8 warps per SM the pipeline becomes issue-bound.
-        int warps = 8, stages = 6, rows = 0, depth = 2;
-        if (const char *e = getenv("VTOKEN_BULK_TUNE")) sscanf(e, "%d,%d,%d,%d", &warps, &stages, &rows, &depth);
+        int warps = 8, stages = 6, rows = 0, depth = 2, ahead = 2;
+        if (const char *e = getenv("VTOKEN_BULK_TUNE")) sscanf(e, "%d,%d,%d,%d,%d", &warps, &stages, &rows, &depth, &ahead);
+        ctx->bulk_ahead = ahead == 1 ? 1 : 2;
         if (rows <= 0) rows = (int)(4096 / ctx->row_bytes);
         // an item is `rows` consecutive destination slots inside one block: a power of two
         // (<= 32, one row per lane) that divides the block size
@@ -365,7 +373,7 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     if (ctx->copy_variant == 1)
         copy_rows_kernel<<<ctx->copy_ctas, ctx->copy_threads, 0, st>>>(a);
     else
-        copy_bulk_kernel<<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth);
+        copy_bulk_kernel<<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -37,6 +37,12 @@
  * offending row or request is skipped and the kernels complete.  A short free list is not an
  * error: the request gets status VTOKEN_DEFERRED_NO_FREE (Sec. 3.3.2).
  *
+ * Bounded waits: the only waits inside the kernels are on shared-memory barriers that the
+ * kernel's own bulk copies complete.  Each is bounded (default 2 s, VTOKEN_WAIT_LIMIT_MS in the
+ * environment at vtoken_create changes it): when it runs out the warp sets VTOKEN_FLAG_TIMEOUT,
+ * gives its copies in flight a bounded time to land and returns, so the kernel always ends and
+ * the context stays usable; rows of the item it was waiting for are missing.
+ *
  * Preconditions assumed (not checked) on the fast path: each live slot is referenced by one
  * token only (I2) and lies in a block of its own request; block ids are unique across block
  * tables (shared-prefix blocks are excluded from plans, I4); the free list has no duplicates

@@ -60,6 +60,7 @@ struct vtoken_ctx {
     // launch shape of the copy kernel
     int copy_variant;          // 1 register path, 2 bulk-copy path
     int copy_ctas, copy_threads, copy_smem;
+    int64_t wait_limit_ns, stall_item;   // bound of in-kernel waits; test hook (see copy.cu)
     int bulk_warps, bulk_stages, bulk_rows, bulk_depth, bulk_ahead;   // bulk path: warps per CTA, ring size, rows per item, loads ahead
 };
 

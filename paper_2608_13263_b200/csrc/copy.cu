@@ -27,6 +27,9 @@ struct CopyArgs {
     vtoken_counts *counts;
     int64_t layer_stride, row_bytes;
     int32_t S, L, rows;        // rows per item (bulk path)
+    int64_t wait_limit_ns;     // bound of every wait on a shared-memory barrier (bulk path)
+    int64_t stall_item;        // -1, or the global index of one item whose barrier is armed with bytes that
+                               // never arrive: exercises the time-out path without faulting anything
 };
 
 __device__ __forceinline__ uint8_t *slab_base(const CopyArgs &a, int slab)
@@ -231,6 +234,9 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
     if (ahead == 2) fetch(e2);
 
     int s_issue = 0, issued = 0, stored = 0;
+    int stall_countdown = -1;                  // issues left before the item named by the test hook
+    if (a.stall_item >= gw && (a.stall_item - gw) % gstride == 0 && (a.stall_item - gw) / gstride < (1 << 30))
+        stall_countdown = (int)((a.stall_item - gw) / gstride);
     auto issue = [&]() {
         if (e1.slab >= num_slabs) return;
         const int s = s_issue;
@@ -250,11 +256,13 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         if (lane == 0) {
             my_mask[s] = mask;
             my_dst[s] = (uint64_t)(base + (int64_t)e.dst0 * a.row_bytes);
-            mbar_expect_tx(&my_bars[s], (uint32_t)__popc(mask) * row_bytes);   // no rows: plain arrive
+            const uint32_t phantom = stall_countdown == 0 ? 16u : 0u;
+            mbar_expect_tx(&my_bars[s], (uint32_t)__popc(mask) * row_bytes + phantom);   // no rows: plain arrive
         }
         __syncwarp();
         if (valid) bulk_g2s(stg + (size_t)lane * row_bytes, base + (int64_t)e.src * a.row_bytes, row_bytes, &my_bars[s]);
         ++issued;
+        --stall_countdown;
     };
 
     bool timed_out = false;
@@ -264,7 +272,7 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
     for (;;) {
         issue();
         if (stored == issued) break;
-        if (!mbar_wait_bounded(&my_bars[s], parity)) { timed_out = true; break; }
+        if (!mbar_wait_bounded(&my_bars[s], parity, (uint64_t)a.wait_limit_ns)) { timed_out = true; break; }
         const unsigned mask = my_mask[s];
         if (mask != 0) {
             uint8_t *stg = my_smem + (size_t)s * stage_bytes;
@@ -318,6 +326,10 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         int warps = 8, stages = 6, rows = 0, depth = 2, ahead = 2;
         if (const char *e = getenv("VTOKEN_BULK_TUNE")) sscanf(e, "%d,%d,%d,%d,%d", &warps, &stages, &rows, &depth, &ahead);
         ctx->bulk_ahead = ahead == 1 ? 1 : 2;
+        ctx->wait_limit_ns = 2000000000ll;
+        if (const char *e = getenv("VTOKEN_WAIT_LIMIT_MS")) { long v = atol(e); if (v >= 1 && v <= 60000) ctx->wait_limit_ns = v * 1000000ll; }
+        ctx->stall_item = -1;
+        if (const char *e = getenv("VTOKEN_TEST_STALL_ITEM")) ctx->stall_item = atoll(e);
         if (rows <= 0) rows = (int)(4096 / ctx->row_bytes);
         // an item is `rows` consecutive destination slots inside one block: a power of two
         // (<= 32, one row per lane) that divides the block size
@@ -370,6 +382,8 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     a.S = ctx->cfg.block_size;
     a.L = ctx->cfg.num_layers;
     a.rows = ctx->bulk_rows;
+    a.wait_limit_ns = ctx->wait_limit_ns;
+    a.stall_item = ctx->stall_item;
     if (ctx->copy_variant == 1)
         copy_rows_kernel<<<ctx->copy_ctas, ctx->copy_threads, 0, st>>>(a);
     else

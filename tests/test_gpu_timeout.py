@@ -1,0 +1,56 @@
+"""The bounded wait of the bulk-copy kernel: when a shared-memory barrier never completes, the
+waiting warp gives up after the configured limit, raises VTOKEN_FLAG_TIMEOUT, lets its copies in
+flight land and returns -- the kernel ends, the context and the GPU stay usable.
+
+The stall is produced without faulting anything: a test hook arms the barrier of ONE work item
+with 16 bytes that no copy will ever deliver (every real copy still runs and completes).  The
+hook and the limit are read from the environment when a context is created."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle import vto
+from paper_2608_13263_b200 import binding as vt
+from paper_2608_13263_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def test_wait_runs_out_sets_flag_and_context_survives():
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    w = wl.llama8b_h2o(seed=0, requests=4, lo=200, hi=600, layers=2)
+    os.environ["VTOKEN_WAIT_LIMIT_MS"] = "20"
+    os.environ["VTOKEN_TEST_STALL_ITEM"] = "5"
+    try:
+        prob = DeviceProblem(w, fill_seed=1, copy_variant=2)
+    finally:
+        del os.environ["VTOKEN_WAIT_LIMIT_MS"]
+        del os.environ["VTOKEN_TEST_STALL_ITEM"]
+    prob.plan()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    prob.repack()
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    flags = prob.read_counts()["error_flags"]
+    assert flags & vt.FLAG_TIMEOUT
+    assert 15.0 < ms < 2000.0                       # gave up after the 20 ms limit (plus the bounded drain)
+    out = prob.outputs()
+    p = vto.plan_workload(w)
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)      # the plan itself is unaffected
+    prob.close()
+
+    # same process, same GPU, a fresh context without the hook: everything works and is exact
+    prob = DeviceProblem(w, fill_seed=1, copy_variant=2)
+    prob.plan()
+    prob.repack()
+    assert prob.read_counts()["error_flags"] == 0
+    k = np.stack([wl.fill_slab(1, 0, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
+    v = np.stack([wl.fill_slab(1, 1, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()

@@ -568,11 +568,32 @@ def run_runtime(args, prob, w, side, dev):
                               tt_slots=tt_commit, keep=keep_commit, phys_len=phys, new_tt_slots=prob.new_tt_slots,
                               req_status=prob.req_status, stream=st)
 
+    # the two K/V-reading checkers: relocation digest over every layer (read only), logical gather of
+    # a layer range that fits in 2 GiB of output per pool (read + write)
+    digest_out = torch.zeros(prob.max_requests, dtype=torch.int64, device=dev)
+    L = w.num_layers
+    g_layers = max(1, min(L, int((2 << 30) // max(1, live * w.row_bytes))))
+    gk = torch.empty((g_layers, max(1, live), w.row_elems), dtype=torch.int16, device=dev)
+    gv = torch.empty_like(gk)
+
+    def digest(st):
+        vt.vtoken_digest_logical(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                 tt_slots=prob.tt_slots, keep=prob.keep, select=None, layer_begin=0, layer_end=L,
+                                 out_digest=digest_out, stream=st)
+
+    def gather(st):
+        vt.vtoken_gather_logical(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                 tt_slots=prob.tt_slots, keep=prob.keep, select=None, layer_begin=0,
+                                 layer_end=g_layers, out_k=gk, out_v=gv, out_capacity_tokens=max(1, live),
+                                 out_offsets=out_off, stream=st)
+
     out = {}
     table_bytes = {"slot_mapping": 2 * 5 * T + 8 * live, "append_one_token_per_request": R * (4 * 6 + 5),
-                   "evict_64k_victims": nv * (8 + 4 + 4 + 1), "apply_moves": T * (4 + 4 + 1)}
+                   "evict_64k_victims": nv * (8 + 4 + 4 + 1), "apply_moves": T * (4 + 4 + 1),
+                   "digest_all_layers": live * w.token_bytes, "gather_logical": 2 * live * 2 * g_layers * w.row_bytes}
     for name, fn in (("slot_mapping", slot_mapping), ("append_one_token_per_request", append),
-                     ("evict_64k_victims", evict), ("apply_moves", commit)):
+                     ("evict_64k_victims", evict), ("apply_moves", commit), ("digest_all_layers", digest),
+                     ("gather_logical", gather)):
         with torch.cuda.stream(side):
             fn(side)
         side.synchronize()
@@ -591,7 +612,7 @@ def run_runtime(args, prob, w, side, dev):
         side.synchronize()
         us = e0.elapsed_time(e1) / reps * 1e3
         out[name] = {"us": us, "table_bytes": table_bytes[name], "GBs": table_bytes[name] / us / 1e3}
-    out["entries"] = {"logical_tokens": T, "live_tokens": live, "requests": R}
+    out["entries"] = {"logical_tokens": T, "live_tokens": live, "requests": R, "gather_layers": g_layers}
     out["note"] = ("append after the first replay is a no-op per request (tt_len already equals new_len): the figure "
                    "is the launch + per-request check cost of a decode step")
     return out

@@ -179,8 +179,10 @@ int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const in
  * request whose active tokens have rank i = 0, 1, ... and logical ids t_i, over the slabs
  * s = 0 .. 2*(layer_end-layer_begin)-1 (K layers first, then V layers) and the 8-byte
  * little-endian words w_j of a token's row,
- *     digest = sum of mix(w_j ^ mix((((i * A + t_i) * B + s) * C + j)))  mod 2^64,
- * mix = splitmix64 finaliser, A = 0x9E3779B97F4A7C15, B = 0xD1B54A32D192ED03, C = 0x8CB92BA72F3D8DD7.
+ *     key(i, s) = mix(((i * A + t_i) * B + s) * C),
+ *     digest    = sum of mix(w_j ^ (key(i, s) + j * D))  mod 2^64,
+ * mix = splitmix64 finaliser, A = 0x9E3779B97F4A7C15, B = 0xD1B54A32D192ED03, C = 0x8CB92BA72F3D8DD7,
+ * D = 0xA0761D6478BD642F.
  * Equal digests before (old table + keep) and after (new table) a repack show token conservation
  * (I1) without materialising the rows.  out_digest: DEVICE uint64 [max_requests] (zeroed by the
  * call); out_offsets: DEVICE int32 [R+1] or NULL, first active-token index of each request (the

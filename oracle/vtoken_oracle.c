@@ -534,7 +534,8 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
     if (!k_pool || !v_pool || !tt_slots || !digest || row_bytes < 8 || row_bytes % 8 != 0) return VTO_EINVAL;
     if (layer_begin < 0 || layer_end <= layer_begin || len < 0) return VTO_EINVAL;
     if (layer_stride_bytes == 0) layer_stride_bytes = num_slots * row_bytes;
-    const uint64_t A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull;
+    const uint64_t A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull,
+                   D = 0xA0761D6478BD642Full;
     const int32_t nl = layer_end - layer_begin;
     uint64_t sum = 0;
     int32_t i = 0;                                           /* rank among the active tokens */
@@ -545,11 +546,12 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
             const uint8_t *pool = s < nl ? k_pool : v_pool;
             const int32_t layer = layer_begin + (s < nl ? s : s - nl);
             const uint8_t *row = pool + (int64_t)layer * layer_stride_bytes + (int64_t)tt_slots[t] * row_bytes;
+            /* key of this (rank, id, slab): binds the row's words to their place in the logical view */
+            const uint64_t key = mix64((((uint64_t)i * A + (uint64_t)t) * B + (uint64_t)s) * C);
             for (int64_t j = 0; j < row_bytes / 8; ++j) {
                 uint64_t w = 0;
                 for (int b = 7; b >= 0; --b) w = (w << 8) | row[j * 8 + b];       /* little-endian word */
-                const uint64_t where = ((((uint64_t)i * A + (uint64_t)t) * B + (uint64_t)s) * C + (uint64_t)j);
-                sum += mix64(w ^ mix64(where));
+                sum += mix64(w ^ (key + (uint64_t)j * D));
             }
         }
         ++i;

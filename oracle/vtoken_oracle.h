@@ -187,8 +187,9 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
  * any order (a sum of per-word terms, each bound to its position): for a request whose active
  * tokens are t_0 < t_1 < ... (rank i, logical id t_i), over slabs s = 0 .. 2*(layer_end-layer_begin)-1
  * (K layers first, then V layers) and the 8-byte little-endian words w_j of the token's row,
- *     digest = sum over (i, s, j) of mix(w_j ^ mix((((i * A + t_i) * B + s) * C + j)))   mod 2^64
- * with mix = the splitmix64 finaliser and A, B, C the odd constants in the source.  A lost,
+ *     key(i, s) = mix(((i * A + t_i) * B + s) * C)
+ *     digest    = sum over (i, s, j) of mix(w_j ^ (key(i, s) + j * D))          mod 2^64
+ * with mix = the splitmix64 finaliser and A, B, C, D the odd constants in the source.  A lost,
  * duplicated, reordered or altered token changes the digest.  row_bytes must be a multiple of 8.
  * Pools are [L][num_slots][row_bytes] with layer_stride_bytes between layers (0 = dense). */
 int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t layer_stride_bytes, int64_t num_slots,

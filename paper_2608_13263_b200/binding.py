@@ -86,10 +86,23 @@ class HostTables(ctypes.Structure):
 _lib = None
 
 
+def _build_if_needed():
+    """Compiles the CUDA libraries in-tree when they are missing or older than their sources and
+    nvcc is available; a build failure is reported, never papered over."""
+    from . import build as _build
+    try:
+        _build._nvcc()
+    except RuntimeError:
+        return                      # no compiler here: use the library as shipped (or fail below)
+    _build.build()
+
+
 def load():
-    """Loads libvtoken.so (once).  Raises when it has not been built: there is no fallback."""
+    """Loads libvtoken.so (once), building it first when needed.  Raises when it cannot be had:
+    there is no fallback."""
     global _lib
     if _lib is None:
+        _build_if_needed()
         if not os.path.exists(LIB_PATH):
             raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_13263_b200.build` "
                               "(needs nvcc); this package has no CPU fallback")

@@ -196,12 +196,13 @@ __device__ __forceinline__ unsigned long long g_mix64(unsigned long long x)   //
 }
 
 // Relocation digest (Sec. 5 of the paper hashes ordered retained ids with their K/V contents):
-//   digest[r] = sum over (rank i, slab s, 8-byte word j) of mix(w ^ mix((((i*A + t_i)*B + s)*C + j)))
+//   key(i, s) = mix(((i*A + t_i)*B + s)*C);  digest[r] = sum over (rank i, slab s, 8-byte word j) of mix(w ^ (key + j*D))
 // a sum of position-bound terms, so any evaluation order gives the same 64-bit value.
 // One warp per (slab, output row); lanes take 16-byte pieces of the row.
 __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
 {
-    const unsigned long long A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull;
+    const unsigned long long A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull,
+                             D = 0xA0761D6478BD642Full;
     const int64_t n = *a.g_total;
     const int nl = a.layer_end - a.layer_begin;
     const int64_t total = n * nl * 2;
@@ -217,16 +218,25 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         const int r = a.g_req[idx];
         const unsigned long long i = (unsigned long long)(idx - a.out_offsets[r]);
         const unsigned long long t = (unsigned long long)a.g_ids[idx];
-        const unsigned long long base = ((i * A + t) * B + (unsigned long long)slab) * C;
+        const unsigned long long key = g_mix64(((i * A + t) * B + (unsigned long long)slab) * C);
         const uint4 *sp = reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
                                                           (int64_t)src * a.row_bytes);
         unsigned long long sum = 0;
-        for (int c = lane; c < row_vecs; c += 32) {
-            const uint4 v = ld_stream(sp + c);
-            const unsigned long long w0 = ((unsigned long long)v.y << 32) | v.x;
-            const unsigned long long w1 = ((unsigned long long)v.w << 32) | v.z;
-            sum += g_mix64(w0 ^ g_mix64(base + 2ull * c));
-            sum += g_mix64(w1 ^ g_mix64(base + 2ull * c + 1ull));
+        for (int c0 = lane; c0 < row_vecs; c0 += 128) {       // four 16-byte loads in flight per lane
+            uint4 v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                v[k] = (c0 + 32 * k < row_vecs) ? ld_stream(sp + c0 + 32 * k) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const int c = c0 + 32 * k;
+                if (c < row_vecs) {
+                    const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
+                    const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
+                    sum += g_mix64(w0 ^ (key + (2ull * c) * D));
+                    sum += g_mix64(w1 ^ (key + (2ull * c + 1ull) * D));
+                }
+            }
         }
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);

@@ -17,6 +17,8 @@ _lib = None
 def load():
     global _lib
     if _lib is None:
+        from .binding import _build_if_needed
+        _build_if_needed()
         if not os.path.exists(LIB_PATH):
             raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_13263_b200.build`")
         lib = ctypes.CDLL(LIB_PATH)

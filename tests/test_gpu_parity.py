@@ -96,6 +96,18 @@ def test_block_sizes_and_row_bytes(S, heads, head_dim, variant):
     run_and_compare(w, copy_variant=variant)
 
 
+@pytest.mark.parametrize("tune", ["1,2,1,0,1", "1,12,1,10,2", "8,6,2,2,2", "4,3,8,1,1", "2,3,16,1,2", "8,12,1,4,1",
+                                  "3,5,4,3,2", "8,2,32,0,2"])
+def test_bulk_copy_ring_shapes(tune, monkeypatch):
+    """Every ring shape the tuning knob can select (warps, stages, rows per item, loads ahead,
+    plan entries ahead) must give the same bytes: whole pools against the oracle."""
+    monkeypatch.setenv("VTOKEN_BULK_TUNE", tune)
+    for w in (wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2),
+              wl.longctx_scissor(seed=5, requests=2, lo=1500, hi=2500, layers=2, block_size=32),
+              wl.mistral7b_random(seed=6, requests=4, lo=30, hi=300, layers=1, heads=4, head_dim=128, block_size=48)):
+        run_and_compare(w, copy_variant=2)
+
+
 def _request(n_tokens, S, first_block):
     nb = -(-n_tokens // S)
     bt = np.arange(first_block, first_block + nb, dtype=np.int32)
@@ -235,6 +247,26 @@ def test_out_of_range_ids_raise_flags_not_faults():
     assert not flags & vt.FLAG_TIMEOUT
     # the bad token was treated as not live
     assert out["new_tt_slots"][np.flatnonzero(w.keep)[0]] == -1
+    prob.close()
+
+
+def test_counts_above_capacity_are_clamped_and_flagged():
+    """A device-side request count or free count above the create-time capacities: clamped,
+    VTOKEN_FLAG_CAPACITY raised, the part inside the capacities still exact."""
+    from paper_2608_13263_b200.device import DeviceProblem
+    torch = _torch()
+    w = wl.mistral7b_random(seed=13, requests=8, lo=50, hi=300, layers=1, heads=1, head_dim=64)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)                 # capacities == problem sizes
+    prob.num_requests.fill_(w.num_requests + 5)
+    prob.num_free.fill_(len(w.free_blocks) + 1000)
+    prob.plan()
+    prob.repack()
+    out = prob.outputs()
+    assert out["error_flags"] & vt.FLAG_CAPACITY
+    p = vto.plan_workload(w)
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
+    assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+    assert np.array_equal(out["freed_blocks"], p.freed_blocks)
     prob.close()
 
 

@@ -5,7 +5,7 @@ import numpy as np
 from oracle import vto
 from paper_2608_13263_b200 import workloads as wl
 
-A, B, C = 0x9E3779B97F4A7C15, 0xD1B54A32D192ED03, 0x8CB92BA72F3D8DD7
+A, B, C, D = 0x9E3779B97F4A7C15, 0xD1B54A32D192ED03, 0x8CB92BA72F3D8DD7, 0xA0761D6478BD642F
 
 
 def mix(x):
@@ -30,8 +30,8 @@ def numpy_digest(k, v, tt_slots, keep, l0, l1):
         t = live.astype(np.uint64)[None, :, None]
         s = np.arange(S_, dtype=np.uint64)[:, None, None]
         j = np.arange(W, dtype=np.uint64)[None, None, :]
-        where = ((i * np.uint64(A) + t) * np.uint64(B) + s) * np.uint64(C) + j
-        total = mix(words ^ mix(where)).sum(dtype=np.uint64)
+        key = mix(((i * np.uint64(A) + t) * np.uint64(B) + s) * np.uint64(C))       # per (token, slab)
+        total = mix(words ^ (key + j * np.uint64(D))).sum(dtype=np.uint64)
     return int(total), n
 
 

@@ -88,11 +88,15 @@ def test_configs_small_whole_pool(w, variant):
 
 @pytest.mark.parametrize("variant", [1, 2])
 @pytest.mark.parametrize("S,heads,head_dim", [(1, 1, 8), (2, 1, 8), (3, 2, 64), (16, 4, 128), (32, 8, 128),
-                                               (48, 8, 128), (16, 16, 128), (5, 3, 8)])
+                                               (48, 8, 128), (16, 16, 128), (5, 3, 8), (16, 64, 256), (4, 128, 256)])
 def test_block_sizes_and_row_bytes(S, heads, head_dim, variant):
-    """S in {1,2,3,5,16,32,48}; row_bytes in {16, 48, 256, 1024, 2048, 4096}."""
-    w = wl.mistral7b_random(seed=S, requests=5, lo=10, hi=40 * S + 20, layers=2, heads=heads, head_dim=head_dim,
-                            block_size=S)
+    """S in {1,2,3,4,5,16,32,48}; row_bytes in {16, 48, 256, 1024, 2048, 4096, 32768, 65536} (the last
+    is beyond what one bulk-copy stage holds: the library must fall back to the register path)."""
+    if heads * head_dim * 2 > 32768 and variant == 2:
+        variant = 0
+    big = heads * head_dim * 2 >= 32768
+    w = wl.mistral7b_random(seed=S, requests=3 if big else 5, lo=10, hi=(6 if big else 40) * S + 20,
+                            layers=1 if big else 2, heads=heads, head_dim=head_dim, block_size=S)
     run_and_compare(w, copy_variant=variant)
 
 
@@ -408,4 +412,57 @@ def test_graph_capture_side_stream_replay_with_new_contents():
         for r in range(base.num_requests):
             t0, t1 = base.tt_offsets[r], base.tt_offsets[r + 1]
             assert np.array_equal(g[1, off[r]:off[r + 1]], vto.gather_logical(k0[1], base.tt_slots[t0:t1], keep[t0:t1]))
+    prob.close()
+
+
+def test_decode_read_proxy_is_undisturbed_by_a_concurrent_repack():
+    """A reader of every allocated block through the OLD block tables (decode-read proxy) runs on
+    one stream while the captured repack runs on another: its per-request checksums must equal the
+    solo values, because destinations are free blocks and sources are only read."""
+    from paper_2608_13263_b200 import harness as vh
+    from paper_2608_13263_b200.device import DeviceProblem
+    torch = _torch()
+    w = wl.steady_state(seed=9, requests=40, lo=300, hi=3000, layers=4)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    owner = np.repeat(np.arange(w.num_requests, dtype=np.int32), np.diff(w.bt_offsets))
+    owner_d = torch.from_numpy(owner).to(prob.device)
+    nbt = len(w.bt_blocks)
+    block_bytes = w.block_size * w.row_bytes
+
+    def proxy(sums, stream):
+        vh.vth_decode_read(prob.k_pool, prob.v_pool, prob.bt_offsets, prob.bt_blocks, owner_d, nbt, w.num_layers,
+                           block_bytes, w.slab_bytes, sums, stream=stream)
+
+    solo = torch.zeros(w.num_requests, dtype=torch.int64, device=prob.device)
+    proxy(solo, torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    assert int((solo != 0).sum()) == w.num_requests
+
+    side, main = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        prob.plan(stream=side)
+        prob.repack(stream=side)
+    side.synchronize()
+    prob.fill_pools()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        prob.plan(stream=torch.cuda.current_stream())
+        prob.repack(stream=torch.cuda.current_stream())
+    both = torch.zeros_like(solo)
+    go = torch.cuda.Event()
+    go.record()
+    main.wait_event(go)
+    side.wait_event(go)
+    proxy(both, main)
+    with torch.cuda.stream(side):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(both, solo)
+    # and the repack that ran beside it is exact
+    p = vto.plan_workload(w)
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst, threads=2)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
     prob.close()

@@ -150,8 +150,9 @@ __device__ __forceinline__ void bulk_wait_read_n(int n)
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-constexpr int BULK_MAX_WARPS = 8;
+constexpr int BULK_MAX_WARPS = 16;
 constexpr int BULK_MAX_STAGES = 12;
+constexpr int BULK_MAX_SMEM = 216 * 1024;   // dynamic shared memory cap: leaves room for the static barrier arrays
 
 // Each warp runs its own pipeline through a ring of `stages` shared-memory buffers.
 //
@@ -343,9 +344,9 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         if (stages < 2) stages = 2;
         if (stages > BULK_MAX_STAGES) stages = BULK_MAX_STAGES;
         int64_t smem = (int64_t)warps * stages * rows * ctx->row_bytes;
-        while (smem > 224 * 1024 && warps > 1) { --warps; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
-        while (smem > 224 * 1024 && stages > 2) { --stages; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
-        if (smem > 224 * 1024) return VTOKEN_EINVAL;
+        while (smem > BULK_MAX_SMEM && warps > 1) { --warps; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
+        while (smem > BULK_MAX_SMEM && stages > 2) { --stages; smem = (int64_t)warps * stages * rows * ctx->row_bytes; }
+        if (smem > BULK_MAX_SMEM) return VTOKEN_EINVAL;
         if (depth < 0) depth = 0;
         if (depth > stages - 2) depth = stages - 2;
         // the kernel indexes the items of a slab with 32-bit integers

@@ -232,13 +232,14 @@ def test_second_round_repack_and_idempotence():
     assert out3["num_moves"] == 0 and set(out3["req_status"].tolist()) <= {vt.NO_GAIN}
 
 
-def test_out_of_range_ids_raise_flags_not_faults():
+@pytest.mark.parametrize("heads,head_dim", [(1, 8), (4, 64)], ids=["register-path", "bulk-path"])
+def test_out_of_range_ids_raise_flags_not_faults(heads, head_dim):
     """Host-fabricated bad slot / block / free ids: a flag bit, the row skipped, no fault."""
     from paper_2608_13263_b200.device import DeviceProblem
     rng = np.random.default_rng(4)
     lens = [60, 60]
     keeps = [(rng.random(60) < 0.3).astype(np.uint8) for _ in lens]
-    w = _custom(4, lens, keeps)
+    w = _custom(4, lens, keeps, heads=heads, head_dim=head_dim)
     w.tt_slots[np.flatnonzero(w.keep)[0]] = w.num_blocks * w.block_size + 5      # slot beyond the pool
     w.free_blocks[1] = w.num_blocks + 3                                          # free id beyond the pool
     w.bt_blocks[len(w.bt_blocks) - 1] = -4                                       # bad block-table id

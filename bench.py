@@ -177,6 +177,25 @@ def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1, use_gpu
     return float(np.mean(times)), moved, desc, p, threads
 
 
+def cpu_baseline_leg(w, args, partial_opts):
+    """The CPU-baseline leg of the CUDA arm: the oracle, as it stands, timed on the host cores on a
+    bounded sample of the workload.  This is the only place where the CUDA arm executes the oracle;
+    the plans it computed on the way are returned so that the device's tables and pools can be
+    compared with them at full size."""
+    from oracle import vto
+    cores = min(os.cpu_count() or 1, vto.openmp_threads())
+    sec, moved, desc, p_whole, cores = oracle_sample(w, args.oracle_layers, cores, 3, 1)
+    sec1, moved1, _, _, _ = oracle_sample(w, 1, 1, 2, 1)
+    plans = {"whole": p_whole}
+    if partial_opts is not None:
+        plans["partial"] = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets,
+                                            w.tt_slots, w.keep, w.free_blocks, w.select, w.thr_num, w.thr_den,
+                                            **partial_opts)
+    baseline = {"value": moved / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc,
+                "single_thread_GBs": moved1 / sec1 / 1e9}
+    return baseline, plans
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -204,7 +223,6 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------
 def run_cuda(args):
     import torch
-    import torch.distributed as dist
 
     from paper_2608_13263_b200 import binding as vt
     from paper_2608_13263_b200.device import DeviceProblem, origin_map
@@ -322,13 +340,16 @@ def run_cuda(args):
     clocks = sampler.stop()      # sampled over every timed region above
 
     # ---- parity at full size, in the launch configuration that was timed --------------------
-    parity = "skipped"
-    if not args.no_verify:
-        from oracle import vto   # the checker: tests/bench only
-        pw = vto.plan_workload(w)                       # what the end-to-end leg (whole-request plan) must return
+    # The oracle is executed in ONE place, the CPU-baseline leg (rank 0, N = 1): it times the oracle
+    # as it stands and hands back the plans it computed, which are then compared with the device's.
+    parity = "skipped (needs the cpu_baseline leg: N = 1 without --no-cpu-baseline)"
+    cpu_baseline, plans = None, None
+    if ranks.world == 1 and not args.no_cpu_baseline:
+        cpu_baseline, plans = cpu_baseline_leg(w, args, partial_opts if args.plan_mode == "partial" else None)
+    if plans is not None and not args.no_verify:
+        pw = plans["whole"]                             # what the end-to-end leg (whole-request plan) must return
         if args.plan_mode == "partial":
-            p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots,
-                                 w.keep, w.free_blocks, w.select, w.thr_num, w.thr_den, **partial_opts)
+            p = plans["partial"]
             # the end-to-end leg wrote the whole-request layout: restore the pools, replay the timed graph once
             prob.fill_pools()
             torch.cuda.synchronize(dev)
@@ -415,14 +436,8 @@ def run_cuda(args):
     if args.runtime:
         line["runtime"] = run_runtime(args, prob, w, side, dev)
 
-    # ---- oracle timed beside it (rank 0, N = 1 only) ------------------------------------------
-    if ranks.world == 1 and not args.no_cpu_baseline:
-        from oracle import vto
-        cores = min(os.cpu_count() or 1, vto.openmp_threads())
-        sec, moved, desc, _, cores = oracle_sample(w, args.oracle_layers, cores, 3, 1)
-        sec1, moved1, desc1, _, _ = oracle_sample(w, 1, 1, 2, 1)
-        line["cpu_baseline"] = {"value": moved / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                                "sample": desc, "single_thread_GBs": moved1 / sec1 / 1e9}
+    if cpu_baseline is not None:
+        line["cpu_baseline"] = cpu_baseline
     prob.close()
     if ranks.rank == 0:
         print(json.dumps(line))

@@ -17,7 +17,7 @@ The five generators follow the five workload shapes the build is measured on:
                      tokens, Scissorhands-style mask (256 recent + Binomial(n_obs, 0.2) >= 2).
   5. ``steady_state`` shape of 2 with S in {16, 32}, 512 requests of 256-8k tokens that have
                      already been evicted and packed once (token tables with -1 holes),
-                     H2O-style second-round mask, repack only requests whose live
+                     second H2O-style eviction pass, repack only requests whose live
                      fraction is below 1/2.
 
 They stand in for the ShareGPT / LongBench request mixes the paper evaluates on
@@ -297,7 +297,7 @@ def steady_state(seed: int = 0, requests: int = 512, lo: int = 256, hi: int = 81
                  layers: int = 32, heads: int = 8, head_dim: int = 128, block_size: int = 16,
                  budget_frac: float = 0.2, thr=(1, 2)) -> Workload:
     """Serving steady state: every request was evicted (H2O-style at length ``len0``) and
-    packed once, then grew to ``len``; the mask under test is a second H2O-style round over
+    packed once, then grew to ``len``; the mask under test is a second H2O-style eviction pass over
     the resident tokens with the same per-token scores.  Only requests whose live fraction is
     below ``thr`` are repacked (incremental repack)."""
     rng = np.random.Generator(np.random.PCG64(seed))

@@ -205,18 +205,18 @@ def test_capacities_larger_than_the_problem():
     run_and_compare(w, capacity_slack=1000)
 
 
-def test_second_round_repack_and_idempotence():
+def test_repeated_repack_and_idempotence():
     """Adopt the new tables, evict again, repack again; then all-keep -> nothing to gain."""
     from paper_2608_13263_b200.device import DeviceProblem
     torch = _torch()
     w = wl.mistral7b_random(seed=21, requests=8, lo=100, hi=400, layers=2, heads=2, head_dim=64)
     out, p = run_and_compare(w)
     rng = np.random.default_rng(2)
-    # state after round 1 (from the oracle; the GPU outputs were just shown to equal it)
+    # state after the first repack (from the oracle; the GPU outputs were just shown to equal it)
     keep2 = ((p.new_tt_slots >= 0) & (rng.random(w.num_tokens) < 0.5)).astype(np.uint8)
     used = set(p.new_bt_blocks.tolist())
     free2 = np.array(sorted(set(range(w.num_blocks)) - used), np.int32)
-    w2 = wl.Workload(name="round2", num_layers=w.num_layers, num_kv_heads=w.num_kv_heads, head_dim=w.head_dim,
+    w2 = wl.Workload(name="second_repack", num_layers=w.num_layers, num_kv_heads=w.num_kv_heads, head_dim=w.head_dim,
                      block_size=w.block_size, num_blocks=w.num_blocks, bt_offsets=p.new_bt_offsets,
                      bt_blocks=p.new_bt_blocks, tt_offsets=w.tt_offsets, tt_slots=p.new_tt_slots, keep=keep2,
                      free_blocks=free2)
@@ -224,7 +224,7 @@ def test_second_round_repack_and_idempotence():
     assert out2["num_admitted"] > 0
     keep3 = (p2.new_tt_slots >= 0).astype(np.uint8)
     used3 = set(p2.new_bt_blocks.tolist())
-    w3 = wl.Workload(name="round3", num_layers=w.num_layers, num_kv_heads=w.num_kv_heads, head_dim=w.head_dim,
+    w3 = wl.Workload(name="third_repack", num_layers=w.num_layers, num_kv_heads=w.num_kv_heads, head_dim=w.head_dim,
                      block_size=w.block_size, num_blocks=w.num_blocks, bt_offsets=p2.new_bt_offsets,
                      bt_blocks=p2.new_bt_blocks, tt_offsets=w.tt_offsets, tt_slots=p2.new_tt_slots, keep=keep3,
                      free_blocks=np.array(sorted(set(range(w.num_blocks)) - used3), np.int32))

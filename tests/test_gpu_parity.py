@@ -52,6 +52,12 @@ def run_and_compare(w, copy_variant=0, num_free=None, whole_pool=True, capacity_
     assert_tables_equal(out, p, w)
     counts = prob.read_counts()
     assert counts["error_flags"] == 0 and counts["num_moves"] == p.num_moves
+    # nothing was written beyond the valid part of any output buffer (they were pre-filled with -9)
+    R, T = w.num_requests, w.num_tokens
+    for buf, valid in ((prob.new_bt_offsets, R + 1), (prob.new_bt_blocks, len(p.new_bt_blocks)),
+                       (prob.new_tt_slots, T), (prob.freed_blocks, p.num_freed), (prob.req_status, R)):
+        tail = buf[valid:].cpu().numpy()
+        assert (tail == -9).all(), "stray write behind an output table"
     if whole_pool:
         k, v = host_pools(w)
         # the device fill and the numpy fill are the same generator

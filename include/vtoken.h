@@ -43,6 +43,15 @@
  * gives its copies in flight a bounded time to land and returns, so the kernel always ends and
  * the context stays usable; rows of the item it was waiting for are missing.
  *
+ * Environment knobs, read once in vtoken_create (tuning and tests; defaults are the measured best):
+ *   VTOKEN_COPY_VARIANT  1 register path, 2 bulk-copy path (only when cfg.copy_variant == 0)
+ *   VTOKEN_COPY_CTAS     grid size of the copy kernel
+ *   VTOKEN_BULK_TUNE     "warps,stages,rows,depth,ahead": warps per CTA, ring size, rows per work item,
+ *                        items loading ahead of the one being stored, plan entries fetched ahead (1 or 2)
+ *   VTOKEN_WAIT_LIMIT_MS bound of in-kernel waits (1 .. 60000, default 2000)
+ *   VTOKEN_TEST_STALL_ITEM  test hook: index of one work item whose barrier is armed with bytes that never
+ *                        arrive, so that its wait runs out (exercises the time-out path; never set in production)
+ *
  * Preconditions assumed (not checked) on the fast path: each live slot is referenced by one
  * token only (I2) and lies in a block of its own request; block ids are unique across block
  * tables (shared-prefix blocks are excluded from plans, I4); the free list has no duplicates

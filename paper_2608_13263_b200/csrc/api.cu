@@ -26,12 +26,14 @@ void free_all(vtoken_ctx *ctx)
     void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->blk_src,
-                    ctx->stage.num_requests, ctx->stage.num_free, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
+                    ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
                     ctx->stage.select, ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
                     ctx->stage.new_tt_slots, ctx->stage.freed_blocks, ctx->stage.req_status, ctx->stage.counts};
     for (void *p : ptrs)
         if (p) cudaFree(p);
+    if (ctx->stage.h_scalars) cudaFreeHost(ctx->stage.h_scalars);
+    if (ctx->stage.h_counts) cudaFreeHost(ctx->stage.h_counts);
     if (ctx->stage.planned) cudaEventDestroy(ctx->stage.planned);
     if (ctx->stage.copied) cudaEventDestroy(ctx->stage.copied);
     if (ctx->stage.aux) cudaStreamDestroy(ctx->stage.aux);
@@ -43,8 +45,8 @@ int ensure_stage(vtoken_ctx *ctx)
     const vtoken_config &c = ctx->cfg;
     int rc = VTOKEN_OK;
     auto A = [&](auto **p, int64_t n) { if (rc == VTOKEN_OK) rc = dev_alloc(ctx, p, n); };
-    A(&ctx->stage.num_requests, 1);
-    A(&ctx->stage.num_free, 1);
+    A(&ctx->stage.num_requests, 2);                 // the two scalars travel in one copy
+    if (rc == VTOKEN_OK) ctx->stage.num_free = ctx->stage.num_requests + 1;
     A(&ctx->stage.bt_offsets, (int64_t)c.max_requests + 1);
     A(&ctx->stage.bt_blocks, c.max_table_blocks);
     A(&ctx->stage.tt_offsets, (int64_t)c.max_requests + 1);
@@ -59,7 +61,9 @@ int ensure_stage(vtoken_ctx *ctx)
     A(&ctx->stage.req_status, c.max_requests);
     A(&ctx->stage.counts, 1);
     if (rc == VTOKEN_OK) {
-        if (cudaStreamCreateWithFlags(&ctx->stage.aux, cudaStreamNonBlocking) != cudaSuccess ||
+        if (cudaMallocHost((void **)&ctx->stage.h_scalars, 2 * sizeof(int32_t)) != cudaSuccess ||
+            cudaMallocHost((void **)&ctx->stage.h_counts, sizeof(vtoken_counts)) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&ctx->stage.aux, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&ctx->stage.planned, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&ctx->stage.copied, cudaEventDisableTiming) != cudaSuccess)
             rc = VTOKEN_ECUDA;
@@ -201,8 +205,9 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     auto &s = ctx->stage;
 #define H2D(dst, src, n) VTK_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(n), cudaMemcpyHostToDevice, st))
 #define D2H(dst, src, n) VTK_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(n), cudaMemcpyDeviceToHost, st))
-    H2D(s.num_requests, &h->num_requests, sizeof(int32_t));
-    H2D(s.num_free, &h->num_free, sizeof(int32_t));
+    s.h_scalars[0] = h->num_requests;               // pinned: the copy below is truly asynchronous
+    s.h_scalars[1] = h->num_free;
+    H2D(s.num_requests, s.h_scalars, 2 * sizeof(int32_t));
     H2D(s.bt_offsets, h->bt_offsets, (R + 1) * sizeof(int32_t));
     if (NBT) H2D(s.bt_blocks, h->bt_blocks, NBT * sizeof(int32_t));
     H2D(s.tt_offsets, h->tt_offsets, (R + 1) * sizeof(int32_t));
@@ -250,10 +255,11 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     st = caller;
     VTK_CUDA(ctx, cudaStreamWaitEvent(st, s.copied, 0));
     // the counts are read from the context's copy so that flags raised by the copy kernel are included
-    D2H(h->counts, ctx->counts, sizeof(vtoken_counts));
+    D2H(s.h_counts, ctx->counts, sizeof(vtoken_counts));
 #undef H2D
 #undef D2H
     VTK_CUDA(ctx, cudaStreamSynchronize(st));
+    *h->counts = *s.h_counts;
     return VTOKEN_OK;
 }
 

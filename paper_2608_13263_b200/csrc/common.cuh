@@ -52,6 +52,8 @@ struct vtoken_ctx {
         uint8_t *keep, *select;
         int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *req_status;
         vtoken_counts *counts;
+        int32_t *h_scalars;            // HOST, pinned: {num_requests, num_free} of the call in flight
+        vtoken_counts *h_counts;       // HOST, pinned: landing place of the counts
         cudaStream_t aux;              // carries the output copies while the copy kernel runs
         cudaEvent_t planned, copied;   // plan done on the caller's stream; outputs copied on aux
     } stage;

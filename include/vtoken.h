@@ -43,6 +43,9 @@
  * gives its copies in flight a bounded time to land and returns, so the kernel always ends and
  * the context stays usable; rows of the item it was waiting for are missing.
  *
+ * Threads: a context is not thread-safe.  Calls on one context must come from one thread at a
+ * time; different contexts (different pools) are independent.
+ *
  * Environment knobs, read once in vtoken_create (tuning and tests; defaults are the measured best):
  *   VTOKEN_COPY_VARIANT  1 register path, 2 bulk-copy path (only when cfg.copy_variant == 0)
  *   VTOKEN_COPY_CTAS     grid size of the copy kernel

@@ -209,19 +209,54 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     const int lane = vtk_lane();
     const int64_t nwarps = (int64_t)gridDim.x * (GC_NT / 32);
     const int row_vecs = (int)(a.row_bytes >> 4);
-    for (int64_t u = (int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5); u < total; u += nwarps) {
-        const int slab = (int)(u / n);
-        const int64_t idx = u - (int64_t)slab * n;
+    // Each warp takes a contiguous run of (slab, row) pairs, so that consecutive rows mostly belong
+    // to one request: the per-lane partial sums are folded into the request's digest only when the
+    // request changes (one 64-bit atomic per run instead of one per row -- with one atomic per row
+    // the kernel was bound by atomic throughput on a few addresses).
+    const int64_t chunk = (total + nwarps - 1) / nwarps;
+    const int64_t w = (int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5);
+    const int64_t u0 = w * chunk, u1 = min(total, u0 + chunk);
+    unsigned long long sum = 0;
+    int cur_r = -1;
+    auto flush = [&]() {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
+        if (lane == 0 && cur_r >= 0 && sum != 0) atomicAdd(&a.digest[cur_r], sum);
+        sum = 0;
+    };
+    // the table entries of a row (source slot, request, logical id) are fetched one row ahead
+    int32_t nx_src = 0, nx_r = 0, nx_t = 0;
+    if (u0 < u1) {
+        const int64_t idx0 = u0 % n;
+        nx_src = a.g_src[idx0];
+        nx_r = a.g_req[idx0];
+        nx_t = a.g_ids[idx0];
+    }
+    int slab = u0 < u1 ? (int)(u0 / n) : 0;
+    int64_t idx = u0 < u1 ? u0 - (int64_t)slab * n : 0;
+    for (int64_t u = u0; u < u1; ++u) {
         const int li = slab < nl ? slab : slab - nl;
         const uint8_t *pool = slab < nl ? a.k_pool : a.v_pool;
-        const int32_t src = a.g_src[idx];
-        const int r = a.g_req[idx];
-        const unsigned long long i = (unsigned long long)(idx - a.out_offsets[r]);
-        const unsigned long long t = (unsigned long long)a.g_ids[idx];
-        const unsigned long long key = g_mix64(((i * A + t) * B + (unsigned long long)slab) * C);
+        const int32_t src = nx_src;
+        const int r = nx_r;
+        const int32_t tok = nx_t;
+        const int cur_slab = slab;
+        const int64_t cur_idx = idx;
+        if (++idx == n) { idx = 0; ++slab; }
+        if (u + 1 < u1) {
+            nx_src = a.g_src[idx];
+            nx_r = a.g_req[idx];
+            nx_t = a.g_ids[idx];
+        }
+        if (r != cur_r) {
+            flush();
+            cur_r = r;
+        }
+        const unsigned long long i = (unsigned long long)(cur_idx - a.out_offsets[r]);
+        const unsigned long long t = (unsigned long long)tok;
+        const unsigned long long key = g_mix64(((i * A + t) * B + (unsigned long long)cur_slab) * C);
         const uint4 *sp = reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
                                                           (int64_t)src * a.row_bytes);
-        unsigned long long sum = 0;
         for (int c0 = lane; c0 < row_vecs; c0 += 128) {       // four 16-byte loads in flight per lane
             uint4 v[4];
 #pragma unroll
@@ -238,10 +273,8 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
                 }
             }
         }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
-        if (lane == 0 && sum != 0) atomicAdd(&a.digest[r], sum);
     }
+    flush();
 }
 
 }  // namespace

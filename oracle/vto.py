@@ -353,3 +353,62 @@ def digest_logical(k_pool: np.ndarray, v_pool: np.ndarray, tt_slots, keep=None, 
     if rc != 0:
         raise ValueError(f"vto_digest_logical failed: {rc}")
     return d.value, n.value
+
+
+# ---- repack in waves --------------------------------------------------------------------------
+@dataclasses.dataclass
+class WavePlan:
+    new_bt_offsets: np.ndarray
+    new_bt_blocks: np.ndarray     # trimmed to new_bt_offsets[R]
+    new_tt_slots: np.ndarray
+    req_status: np.ndarray
+    req_wave: np.ndarray
+    free_out: np.ndarray          # the pool after the last wave
+    move_src: np.ndarray          # all waves back to back; apply in this order
+    move_dst: np.ndarray
+    wave_move_offsets: np.ndarray
+    wave_counts: list             # one dict per wave
+
+
+def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_waves, select=None,
+               thr_num=0, thr_den=0, partial=None) -> WavePlan:
+    """``partial``: None (whole-request planner) or a dict with the keyword options of plan_partial."""
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
+    keep, select, free_blocks = _u8(keep), _u8(select), _i32(free_blocks)
+    R, T, nbt = len(tt_offsets) - 1, int(tt_offsets[-1]), int(bt_offsets[-1])
+    num_free = len(free_blocks)
+    new_bt_offsets = np.zeros(R + 1, np.int32)
+    new_bt_blocks = np.full(max(nbt, 1), -7, np.int32)
+    new_tt_slots = np.full(max(T, 1), -7, np.int32)
+    status = np.full(max(R, 1), -7, np.int32)
+    wave = np.full(max(R, 1), -7, np.int32)
+    free_out = np.full(max(num_free + nbt, 1), -7, np.int32)
+    nfo = ctypes.c_int32(0)
+    cap = max(1, T * num_waves)
+    msrc = np.full(cap, -7, np.int32)
+    mdst = np.full(cap, -7, np.int32)
+    offs = np.zeros(num_waves + 1, np.int64)
+    counts = (_Counts * num_waves)()
+    o, protect = None, None
+    if partial is not None:
+        protect = _u8(partial.get("protect"))
+        util, theta = partial.get("util", (0, 0)), partial.get("theta", (0, 0))
+        o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1],
+                         partial.get("max_source_blocks", 0), theta[0], theta[1])
+    rc = lib().vto_plan_waves(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
+                              _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
+                              _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),
+                              ctypes.c_uint32(thr_num), ctypes.c_uint32(thr_den), _p(free_blocks, np.int32),
+                              ctypes.c_int32(num_free), None if o is None else ctypes.byref(o),
+                              ctypes.c_int32(num_waves), _p(new_bt_offsets, np.int32), _p(new_bt_blocks, np.int32),
+                              _p(new_tt_slots, np.int32), _p(status, np.int32), _p(wave, np.int32),
+                              _p(free_out, np.int32), ctypes.byref(nfo), _p(msrc, np.int32), _p(mdst, np.int32),
+                              ctypes.c_int64(cap), offs.ctypes.data_as(ctypes.c_void_p), counts)
+    if rc != 0:
+        raise ValueError(f"vto_plan_waves failed: {rc}")
+    total = int(offs[num_waves])
+    wc = [{n: getattr(c, n) for n, _ in _Counts._fields_} for c in counts]
+    return WavePlan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
+                    status[:R].copy(), wave[:R].copy(), free_out[:nfo.value].copy(), msrc[:total].copy(),
+                    mdst[:total].copy(), offs, wc)

@@ -561,6 +561,104 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
     return VTO_OK;
 }
 
+int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
+                   const int32_t *bt_offsets, const int32_t *bt_blocks,
+                   const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                   const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+                   const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
+                   int32_t num_waves,
+                   int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
+                   int32_t *req_status, int32_t *req_wave, int32_t *free_out, int32_t *num_free_out,
+                   int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
+                   int64_t *wave_move_offsets, vto_counts *wave_counts)
+{
+    if (R < 0 || S < 1 || num_free < 0 || num_waves < 1 || !bt_offsets || !tt_offsets || !num_free_out ||
+        !wave_move_offsets || !wave_counts)
+        return VTO_EINVAL;
+    const int64_t T = tt_offsets[R], nbt = bt_offsets[R];
+    const size_t nT = (size_t)(T > 0 ? T : 1), nB = (size_t)(nbt > 0 ? nbt : 1), nR = (size_t)R + 1;
+    const size_t nP = (size_t)num_free + nB;
+
+    /* the committed state a wave plans on (cur_*) and the state it proposes (nxt_*) */
+    int32_t *cur_bto = malloc(nR * sizeof(int32_t)), *nxt_bto = malloc(nR * sizeof(int32_t));
+    int32_t *cur_btb = malloc(nB * sizeof(int32_t)), *nxt_btb = malloc(nB * sizeof(int32_t));
+    int32_t *cur_tts = malloc(nT * sizeof(int32_t)), *nxt_tts = malloc(nT * sizeof(int32_t));
+    int32_t *pool = malloc(nP * sizeof(int32_t)), *pool_next = malloc(nP * sizeof(int32_t));
+    int32_t *freed = malloc(nB * sizeof(int32_t)), *status = malloc(nR * sizeof(int32_t));
+    int32_t *msrc = malloc(nT * sizeof(int32_t)), *mdst = malloc(nT * sizeof(int32_t));
+    int rc = VTO_OK;
+    if (!cur_bto || !nxt_bto || !cur_btb || !nxt_btb || !cur_tts || !nxt_tts || !pool || !pool_next || !freed ||
+        !status || !msrc || !mdst) {
+        rc = VTO_EINVAL;
+        goto done;
+    }
+    memcpy(cur_bto, bt_offsets, nR * sizeof(int32_t));
+    if (nbt > 0) memcpy(cur_btb, bt_blocks, (size_t)nbt * sizeof(int32_t));
+    if (T > 0) memcpy(cur_tts, tt_slots, (size_t)T * sizeof(int32_t));
+    if (num_free > 0) memcpy(pool, free_blocks, (size_t)num_free * sizeof(int32_t));
+    int32_t pool_n = num_free;
+    for (int32_t r = 0; r < R; ++r) {
+        req_status[r] = VTO_NOT_SELECTED;
+        req_wave[r] = -1;
+    }
+    int64_t total_moves = 0;
+    wave_move_offsets[0] = 0;
+
+    for (int32_t k = 0; k < num_waves; ++k) {
+        vto_counts c;
+        /* one planning round against the pool as it stands (Sec. 3.3.2 admission, 3.3.3 planning) */
+        if (opts)
+            rc = vto_plan_partial(R, S, NB, cur_bto, cur_btb, tt_offsets, cur_tts, keep, select, thr_num, thr_den,
+                                  pool, pool_n, opts, nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c);
+        else
+            rc = vto_plan(R, S, cur_bto, cur_btb, tt_offsets, cur_tts, keep, select, thr_num, thr_den, pool, pool_n,
+                          nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c);
+        if (rc != VTO_OK) goto done;
+        wave_counts[k] = c;
+        /* its copies, in wave order */
+        if (total_moves + c.num_moves > move_capacity) {
+            rc = VTO_EINVAL;
+            goto done;
+        }
+        for (int32_t m = 0; m < c.num_moves; ++m) {
+            move_src[total_moves + m] = msrc[m];
+            move_dst[total_moves + m] = mdst[m];
+        }
+        total_moves += c.num_moves;
+        wave_move_offsets[k + 1] = total_moves;
+        /* commit: the proposed tables become the state (apply_moves, Sec. 3.2) ... */
+        memcpy(cur_bto, nxt_bto, nR * sizeof(int32_t));
+        if (nxt_bto[R] > 0) memcpy(cur_btb, nxt_btb, (size_t)nxt_bto[R] * sizeof(int32_t));
+        if (T > 0) memcpy(cur_tts, nxt_tts, (size_t)T * sizeof(int32_t));
+        for (int32_t r = 0; r < R; ++r) {
+            if (status[r] == VTO_REPACKED) {
+                req_status[r] = VTO_REPACKED;
+                req_wave[r] = k;
+            } else if (req_status[r] != VTO_REPACKED) {
+                req_status[r] = status[r];
+            }
+        }
+        /* ... and only then do the sources return to the pool (Sec. 3.3.4): the unconsumed part of
+         * the pool keeps its order, the reclaimed blocks follow */
+        int32_t n = 0;
+        for (int32_t i = c.num_free_consumed; i < pool_n; ++i) pool_next[n++] = pool[i];
+        for (int32_t i = 0; i < c.num_freed; ++i) pool_next[n++] = freed[i];
+        int32_t *tmp = pool;
+        pool = pool_next;
+        pool_next = tmp;
+        pool_n = n;
+    }
+    memcpy(new_bt_offsets, cur_bto, nR * sizeof(int32_t));
+    if (cur_bto[R] > 0) memcpy(new_bt_blocks, cur_btb, (size_t)cur_bto[R] * sizeof(int32_t));
+    if (T > 0) memcpy(new_tt_slots, cur_tts, (size_t)T * sizeof(int32_t));
+    if (pool_n > 0) memcpy(free_out, pool, (size_t)pool_n * sizeof(int32_t));
+    *num_free_out = pool_n;
+done:
+    free(cur_bto); free(nxt_bto); free(cur_btb); free(nxt_btb); free(cur_tts); free(nxt_tts);
+    free(pool); free(pool_next); free(freed); free(status); free(msrc); free(mdst);
+    return rc;
+}
+
 int vto_openmp_threads(void)
 {
 #ifdef _OPENMP

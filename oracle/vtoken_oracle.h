@@ -196,6 +196,33 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
                        int64_t row_bytes, int32_t layer_begin, int32_t layer_end, const int32_t *tt_slots,
                        const uint8_t *keep, int32_t len, uint64_t *digest, int32_t *num_active);
 
+/* ---- repack in waves: blocks reclaimed by one wave are destinations of the next ----------------
+ * The paper returns source blocks to the free pool once the packed layout is committed
+ * (Sec. 3.3.4) and defers plans that the headroom cannot serve (Sec. 3.3.2).  Run as a loop, the
+ * two statements give a repack that needs only a small headroom: wave k plans against the pool
+ * P_k (vto_plan, or vto_plan_partial when opts != NULL), its copies run, its tables are committed,
+ * and   P_{k+1} = P_k without the consumed prefix, followed by the blocks wave k reclaimed
+ * (reclaim order).  Wave k+1 plans on the committed tables of wave k with the same keep mask
+ * (evicted entries are -1 from wave 0 on).  Exactly num_waves waves run; a wave that admits
+ * nothing changes nothing.
+ * Outputs: the tables after the last wave; req_status[r] = VTO_REPACKED when some wave admitted r,
+ * else its status in the last wave; req_wave[r] = last wave that admitted r, -1 when none;
+ * free_out[<= num_free + total old blocks] / *num_free_out = the pool after the last wave;
+ * wave_counts[num_waves] = counts of every wave; move_src / move_dst = the move lists of all
+ * waves back to back, wave k in [wave_move_offsets[k], wave_move_offsets[k+1]) -- they must be
+ * applied in this order, because a later wave overwrites blocks an earlier wave has read.
+ * Returns VTO_EINVAL when move_capacity is too small. */
+int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
+                   const int32_t *bt_offsets, const int32_t *bt_blocks,
+                   const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                   const uint8_t *select, uint32_t thr_num, uint32_t thr_den,
+                   const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
+                   int32_t num_waves,
+                   int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
+                   int32_t *req_status, int32_t *req_wave, int32_t *free_out, int32_t *num_free_out,
+                   int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
+                   int64_t *wave_move_offsets, vto_counts *wave_counts);
+
 int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */
 
 #ifdef __cplusplus

@@ -177,7 +177,7 @@ def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1, use_gpu
     return float(np.mean(times)), moved, desc, p, threads
 
 
-def cpu_baseline_leg(w, args, partial_opts):
+def cpu_baseline_leg(w, args, partial_opts, waves=0):
     """The CPU-baseline leg of the CUDA arm: the oracle, as it stands, timed on the host cores on a
     bounded sample of the workload.  This is the only place where the CUDA arm executes the oracle;
     the plans it computed on the way are returned so that the device's tables and pools can be
@@ -191,6 +191,12 @@ def cpu_baseline_leg(w, args, partial_opts):
         plans["partial"] = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets,
                                             w.tt_slots, w.keep, w.free_blocks, w.select, w.thr_num, w.thr_den,
                                             **partial_opts)
+    if waves:
+        need = np.diff(p_whole.new_bt_offsets)[p_whole.req_status == vto.REPACKED]
+        headroom = int(need.max()) if len(need) else 0
+        plans["waves"] = vto.plan_waves(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets,
+                                        w.tt_slots, w.keep, w.free_blocks[:headroom], waves, w.select, w.thr_num,
+                                        w.thr_den)
     baseline = {"value": moved / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc,
                 "single_thread_GBs": moved1 / sec1 / 1e9}
     return baseline, plans
@@ -243,7 +249,8 @@ def run_cuda(args):
         w = build_workload(args.config, seed, args.scale_requests, args.block_size)
         need = 2 * w.pool_bytes + (1 << 30)
 
-    prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas)
+    prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas,
+                         wave_capacity=args.waves > 0)
     partial_opts = dict(util=(1, 1), theta=(1, 4))     # fully live blocks stay; the paper's default trigger F > 0.25
     if args.plan_mode == "partial":
         do_plan = lambda st: prob.plan_partial(stream=st, **partial_opts)
@@ -345,7 +352,8 @@ def run_cuda(args):
     parity = "skipped (needs the cpu_baseline leg: N = 1 without --no-cpu-baseline)"
     cpu_baseline, plans = None, None
     if ranks.world == 1 and not args.no_cpu_baseline:
-        cpu_baseline, plans = cpu_baseline_leg(w, args, partial_opts if args.plan_mode == "partial" else None)
+        cpu_baseline, plans = cpu_baseline_leg(w, args, partial_opts if args.plan_mode == "partial" else None,
+                                               args.waves)
     if plans is not None and not args.no_verify:
         pw = plans["whole"]                             # what the end-to-end leg (whole-request plan) must return
         if args.plan_mode == "partial":
@@ -435,6 +443,8 @@ def run_cuda(args):
         line["concurrency"] = run_proxy(args, prob, w, side, g_all, bytes_per_step, dev)
     if args.runtime:
         line["runtime"] = run_runtime(args, prob, w, side, dev)
+    if args.waves:                # last: it overwrites allocated blocks
+        line["waves"] = run_waves(args, prob, w, side, dev, plans, ms_per_step)
 
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
@@ -525,6 +535,66 @@ def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
             "sum_over_window_GBs": gbs(proxy_bytes * n_proxy + bytes_per_step * n_rep, window_ms),
             "proxy_checksum_unchanged": checksum_ok,
             "streams": "proxy on a high-priority stream, repack graph on the default-priority side stream"}
+
+
+def run_waves(args, prob, w, side, dev, plans, one_shot_ms):
+    """The same repack with a pool of the largest single demand instead of the sum of all demands:
+    plan + copy + commit in `--waves` waves, blocks reclaimed by one wave feeding the next, one
+    captured graph.  Checked against the oracle's wave plan when the CPU-baseline leg ran."""
+    import torch
+    from paper_2608_13263_b200.device import origin_map
+    W = args.waves
+    prob.plan()                                            # the one-shot plan names every demand
+    one = prob.outputs()
+    need = np.diff(one["new_bt_offsets"])[one["req_status"] == 1]
+    headroom = int(need.max()) if len(need) else 0
+    nf_dev = torch.tensor([headroom], dtype=torch.int32, device=dev)
+    prob.repack_waves(W, num_free=nf_dev)                  # allocates the wave buffers outside the capture
+    torch.cuda.synchronize(dev)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        prob.repack_waves(W, num_free=nf_dev, stream=torch.cuda.current_stream())
+    prob.fill_pools()
+    torch.cuda.synchronize(dev)
+    with torch.cuda.stream(side):
+        g.replay()
+    side.synchronize()
+    out = prob.waves_outputs(W)
+    moved = sum(c["num_moves"] for c in out["wave_counts"])
+    parity = "skipped (needs the cpu_baseline leg)"
+    if plans is not None and "waves" in plans and not args.no_verify:
+        v = plans["waves"]
+        ok = (all(c["error_flags"] == 0 for c in out["wave_counts"])
+              and [c["num_moves"] for c in out["wave_counts"]] == [c["num_moves"] for c in v.wave_counts]
+              and np.array_equal(out["new_tt_slots"], v.new_tt_slots)
+              and np.array_equal(out["new_bt_offsets"], v.new_bt_offsets)
+              and np.array_equal(out["new_bt_blocks"], v.new_bt_blocks)
+              and np.array_equal(out["req_status"], v.req_status) and np.array_equal(out["req_wave"], v.req_wave)
+              and np.array_equal(out["free_out"], v.free_out))
+        bad = prob.verify_pools(origin_map(w.slots_per_layer, v.move_src, v.move_dst, v.wave_move_offsets))
+        parity = "ok" if (ok and bad == 0) else f"FAILED (tables_ok={ok}, mismatching_words={bad})"
+    # timing: replays read the same source slots and write the same destinations (the inputs are
+    # read-only), so every replay moves the same bytes whatever the rows hold by then
+    reps = max(3, args.steps)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with torch.cuda.stream(side):
+        for _ in range(3):
+            g.replay()
+        e0.record(side)
+        for _ in range(reps):
+            g.replay()
+        e1.record(side)
+    side.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    return {"waves_enqueued": W, "waves_with_work": sum(1 for c in out["wave_counts"] if c["num_admitted"]),
+            "headroom_blocks": headroom, "one_shot_headroom_blocks": one["num_dst_blocks"],
+            "headroom_GiB": headroom * w.block_size * w.token_bytes / 2 ** 30,
+            "one_shot_headroom_GiB": one["num_dst_blocks"] * w.block_size * w.token_bytes / 2 ** 30,
+            "tokens_moved": moved, "one_shot_tokens_moved": one["num_moves"],
+            "requests_repacked": int((out["req_status"] == 1).sum()), "one_shot_requests_repacked": one["num_admitted"],
+            "moves_per_wave": [c["num_moves"] for c in out["wave_counts"]],
+            "ms": ms, "one_shot_ms": one_shot_ms, "GBs": 2 * moved * w.token_bytes / (ms * 1e-3) / 1e9,
+            "parity": parity}
 
 
 def run_runtime(args, prob, w, side, dev):
@@ -650,6 +720,8 @@ def main():
     ap.add_argument("--runtime", action="store_true", help="also time the token-table runtime kernels")
     ap.add_argument("--plan-mode", default="whole", choices=["whole", "partial"],
                     help="whole-request compaction (default) or the partial planner that keeps fully live blocks")
+    ap.add_argument("--waves", type=int, default=0,
+                    help="also run the repack in this many waves with the headroom of the largest single demand")
     ap.add_argument("--block-size", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--no-verify", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

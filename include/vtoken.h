@@ -246,6 +246,48 @@ typedef struct {
 int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
                         const vtoken_plan_out *out, void *cuda_stream);
 
+/* ---- Repack in waves: blocks reclaimed by one wave are destinations of the next ----------------
+ * The paper returns source blocks to the free pool once the packed layout is committed (Sec. 3.3.4)
+ * and defers plans that the evacuation headroom cannot serve (Sec. 3.3.2).  Chained on the device,
+ * the two rules give a repack whose headroom is the largest single demand instead of the sum of
+ * all demands: wave k plans against the pool P_k (vtoken_plan, or vtoken_plan_partial when opts is
+ * given), its rows are copied, its tables are committed, and
+ *     P_{k+1} = P_k without the consumed prefix, followed by the blocks wave k reclaimed
+ * (reclaim order); wave k+1 plans on the committed tables of wave k with the same keep mask.
+ * Exactly num_waves waves are enqueued (plan + copy + commit each, all on the given stream, so a
+ * wave's copies finish before the next wave writes into the blocks they read); a wave that admits
+ * nothing moves nothing.  Capturable like vtoken_plan / vtoken_repack.
+ *
+ * Ordering contract: unlike vtoken_plan + vtoken_repack, waves after the first overwrite blocks
+ * that the INPUT tables still reference.  No reader of the old tables may run concurrently: order
+ * the call after the last consumer of the old layout (the paper launches relocation after the
+ * step's forward has returned, Sec. 3.3.4), and make consumers of the new tables wait on an event
+ * recorded behind it. */
+typedef struct {                   /* all DEVICE pointers, written by vtoken_repack_waves */
+    int32_t *new_bt_offsets;       /* [R+1] block tables after the last wave */
+    int32_t *new_bt_blocks;        /* capacity max_table_blocks */
+    int32_t *new_tt_slots;         /* [T] token table after the last wave */
+    int32_t *req_status;           /* [R] VTOKEN_REPACKED when some wave admitted the request, else its
+                                      status in the last wave */
+    int32_t *req_wave;             /* [R] last wave that admitted the request, -1 = none */
+    int32_t *free_out;             /* [free_capacity] the pool after the last wave */
+    int32_t *num_free_out;         /* device scalar */
+    vtoken_counts *wave_counts;    /* [num_waves] counts of every wave (flags of its copy included) */
+    int32_t free_capacity;         /* entries of free_out; num_free + total block-table entries always
+                                      suffices; must not exceed the context's max_free_blocks
+                                      (VTOKEN_ECAPACITY); a pool that outgrows it is truncated and
+                                      VTOKEN_FLAG_CAPACITY is raised */
+    void *workspace;               /* DEVICE scratch, 16-byte aligned, owned by the caller */
+    int64_t workspace_bytes;       /* >= vtoken_waves_workspace_bytes (VTOKEN_ECAPACITY otherwise) */
+} vtoken_waves_out;
+
+/* Bytes of workspace vtoken_repack_waves needs for this context and free_capacity. */
+int64_t vtoken_waves_workspace_bytes(const vtoken_ctx *ctx, int32_t free_capacity);
+
+/* in: as for vtoken_plan (read-only); opts: NULL = whole-request planner; num_waves >= 1. */
+int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
+                        int32_t num_waves, const vtoken_waves_out *out, void *cuda_stream);
+
 /* ---- Token-table runtime on the device (Sec. 3.2 interfaces, Sec. 3.4 slot mapping) ----------
  * For callers that keep the token tables resident on the GPU between decode steps.  Layout: the
  * table of request r occupies tt_slots / keep [tt_offsets[r] .. tt_offsets[r+1]) -- that range is

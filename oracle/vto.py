@@ -277,6 +277,36 @@ def apply_moves(tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, phys_len, ne
         raise ValueError(f"vto_apply_moves failed: {rc}")
 
 
+# ---- cached slot-translation arrays ------------------------------------------------------------
+def slot_cache_mark(dirty: np.ndarray, victim_req=None, req_status=None) -> None:
+    """In place on ``dirty`` (uint8 [R])."""
+    assert dirty.dtype == np.uint8 and dirty.flags["C_CONTIGUOUS"]
+    victim_req = _i32([] if victim_req is None else victim_req)
+    req_status = None if req_status is None else _i32(req_status)
+    rc = lib().vto_slot_cache_mark(ctypes.c_int32(len(dirty)), _p(dirty, np.uint8), _p(victim_req, np.int32),
+                                   ctypes.c_int32(len(victim_req)), _p(req_status, np.int32))
+    if rc != 0:
+        raise ValueError(f"vto_slot_cache_mark failed: {rc}")
+
+
+def slot_cache_update(tt_offsets, tt_slots, keep, tt_len, dirty: np.ndarray, cache_slots: np.ndarray,
+                      cache_ids, cache_len: np.ndarray, cache_seen: np.ndarray):
+    """In place on dirty, cache_slots, cache_ids (may be None), cache_len, cache_seen.
+    Returns (requests rebuilt, requests appended to)."""
+    tt_offsets, tt_slots, keep, tt_len = _i32(tt_offsets), _i32(tt_slots), _u8(keep), _i32(tt_len)
+    for a, d in ((dirty, np.uint8), (cache_slots, np.int32), (cache_len, np.int32), (cache_seen, np.int32)):
+        assert a.dtype == d and a.flags["C_CONTIGUOUS"]
+    nr, na = ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = lib().vto_slot_cache_update(ctypes.c_int32(len(tt_len)), _p(tt_offsets, np.int32), _p(tt_slots, np.int32),
+                                     _p(keep, np.uint8), _p(tt_len, np.int32), _p(dirty, np.uint8),
+                                     _p(cache_slots, np.int32), None if cache_ids is None else _p(cache_ids, np.int32),
+                                     _p(cache_len, np.int32), _p(cache_seen, np.int32), ctypes.byref(nr),
+                                     ctypes.byref(na))
+    if rc != 0:
+        raise ValueError(f"vto_slot_cache_update failed: {rc}")
+    return nr.value, na.value
+
+
 # ---- eligibility metadata and partial plans ---------------------------------------------------
 class _PartialOpts(ctypes.Structure):
     _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),

@@ -382,6 +382,53 @@ int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uin
     return VTO_OK;
 }
 
+int vto_slot_cache_mark(int32_t R, uint8_t *dirty, const int32_t *victim_req, int32_t num_victims,
+                        const int32_t *req_status)
+{
+    if (R < 0 || !dirty || num_victims < 0 || (num_victims > 0 && !victim_req)) return VTO_EINVAL;
+    /* eviction and relocation are the structural changes that invalidate a cached array */
+    for (int32_t i = 0; i < num_victims; ++i)
+        if (victim_req[i] >= 0 && victim_req[i] < R) dirty[victim_req[i]] = 1;
+    if (req_status)
+        for (int32_t r = 0; r < R; ++r)
+            if (req_status[r] == VTO_REPACKED) dirty[r] = 1;
+    return VTO_OK;
+}
+
+int vto_slot_cache_update(int32_t R, const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                          const int32_t *tt_len, uint8_t *dirty, int32_t *cache_slots, int32_t *cache_ids,
+                          int32_t *cache_len, int32_t *cache_seen, int32_t *num_rebuilt, int32_t *num_appended)
+{
+    if (R < 0 || !tt_offsets || !tt_slots || !tt_len || !dirty || !cache_slots || !cache_len || !cache_seen)
+        return VTO_EINVAL;
+    int32_t rebuilt = 0, appended = 0;
+    for (int32_t r = 0; r < R; ++r) {
+        const int64_t base = tt_offsets[r];
+        int32_t first;                       /* first registered token the cache does not cover yet */
+        if (dirty[r]) {                      /* structural change: start over */
+            cache_len[r] = 0;
+            first = 0;
+            dirty[r] = 0;
+            ++rebuilt;
+        } else if (tt_len[r] > cache_seen[r]) {   /* append-only growth */
+            first = cache_seen[r];
+            ++appended;
+        } else {
+            continue;
+        }
+        for (int32_t t = first; t < tt_len[r]; ++t) {
+            if (!is_live(tt_slots, keep, base + t)) continue;
+            cache_slots[base + cache_len[r]] = tt_slots[base + t];
+            if (cache_ids) cache_ids[base + cache_len[r]] = t;
+            ++cache_len[r];
+        }
+        cache_seen[r] = tt_len[r];
+    }
+    if (num_rebuilt) *num_rebuilt = rebuilt;
+    if (num_appended) *num_appended = appended;
+    return VTO_OK;
+}
+
 int vto_block_liveness(int32_t R, int32_t S, int32_t NB, const int32_t *bt_offsets, const int32_t *bt_blocks,
                        const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
                        int32_t *n_b, int64_t *hist, int64_t *live_total, int64_t *num_allocated)

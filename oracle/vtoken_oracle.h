@@ -144,6 +144,25 @@ int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32
 int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
                     int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status);
 
+/* ---- cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4) -------------------------
+ * The worker keeps, per request, the slots of its active tokens in token-id order -- the array a
+ * decode step translates through -- and refreshes it only after structural changes: "when a
+ * sequence grows append-only, the cache is updated by appending the new entries; a full rebuild is
+ * triggered only on structural changes (eviction, relocation ...)".
+ * Layout: the cache of request r lives in cache_slots / cache_ids [tt_offsets[r] ..) (same capacity
+ * as its token table); cache_len[r] entries are valid and cover the first cache_seen[r] registered
+ * tokens.
+ * vto_slot_cache_mark: dirty[r] = 1 for the request of every victim (requests outside [0, R) are
+ * skipped) and for every request with status VTO_REPACKED; either list may be NULL.
+ * vto_slot_cache_update, per request: dirty -> rebuild from the first tt_len[r] entries and clear
+ * the mark; else tt_len[r] > cache_seen[r] -> append the active ones among the new entries; else
+ * leave everything as it is.  *num_rebuilt / *num_appended (optional) count the requests. */
+int vto_slot_cache_mark(int32_t R, uint8_t *dirty, const int32_t *victim_req, int32_t num_victims,
+                        const int32_t *req_status);
+int vto_slot_cache_update(int32_t R, const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
+                          const int32_t *tt_len, uint8_t *dirty, int32_t *cache_slots, int32_t *cache_ids,
+                          int32_t *cache_len, int32_t *cache_seen, int32_t *num_rebuilt, int32_t *num_appended);
+
 /* ---- eligibility metadata and partial plans (Sec. 3.3.1 - 3.3.3) ------------------------------
  * Per-block liveness n_b = live tokens stored in physical block b (over all requests), the
  * histogram hist[k] = number of ALLOCATED blocks (entries of the block tables) with n_b == k for

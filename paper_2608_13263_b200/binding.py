@@ -21,7 +21,8 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
            "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
-           "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical"]
+           "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
+           "vtoken_waves_workspace_bytes", "vtoken_repack_waves"]
 
 
 class VtokenError(RuntimeError):
@@ -69,6 +70,14 @@ class PlanOut(ctypes.Structure):
 class PartialOpts(ctypes.Structure):
     _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
                 ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32)]
+
+
+class WavesOut(ctypes.Structure):
+    _fields_ = [("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
+                ("new_tt_slots", ctypes.c_void_p), ("req_status", ctypes.c_void_p), ("req_wave", ctypes.c_void_p),
+                ("free_out", ctypes.c_void_p), ("num_free_out", ctypes.c_void_p), ("wave_counts", ctypes.c_void_p),
+                ("free_capacity", ctypes.c_int32), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_int64)]
 
 
 class HostTables(ctypes.Structure):
@@ -136,6 +145,10 @@ def load():
         lib.vtoken_digest_logical.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 3
         lib.vtoken_plan_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
                                             ctypes.POINTER(PlanOut), ctypes.c_void_p]
+        lib.vtoken_waves_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+        lib.vtoken_waves_workspace_bytes.restype = ctypes.c_int64
+        lib.vtoken_repack_waves.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
+                                            ctypes.c_int32, ctypes.POINTER(WavesOut), ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -310,3 +323,28 @@ def vtoken_digest_logical(ctx, *, num_requests, tt_offsets, tt_slots, keep, sele
     _check(load().vtoken_digest_logical(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                                         _ptr(select), layer_begin, layer_end, _ptr(out_digest), _ptr(out_offsets),
                                         _stream(stream)), "vtoken_digest_logical", ctx)
+
+
+# ---- repack in waves --------------------------------------------------------------------------
+def vtoken_waves_workspace_bytes(ctx, free_capacity: int) -> int:
+    return load().vtoken_waves_workspace_bytes(ctx, free_capacity)
+
+
+def vtoken_repack_waves(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
+                        num_waves, new_bt_offsets, new_bt_blocks, new_tt_slots, req_status, req_wave, free_out,
+                        num_free_out, wave_counts, free_capacity, workspace, workspace_bytes, select=None, thr_num=0,
+                        thr_den=0, partial=None, stream=None) -> None:
+    """``partial``: None for the whole-request planner, else a dict with the option keywords of
+    vtoken_plan_partial (protect, util, max_source_blocks, theta)."""
+    pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                 _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
+    wout = WavesOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(req_status), _ptr(req_wave),
+                    _ptr(free_out), _ptr(num_free_out), _ptr(wave_counts), free_capacity, _ptr(workspace),
+                    workspace_bytes)
+    po = None
+    if partial is not None:
+        util, theta = partial.get("util", (0, 0)), partial.get("theta", (0, 0))
+        po = ctypes.byref(PartialOpts(_ptr(partial.get("protect")), util[0], util[1],
+                                      partial.get("max_source_blocks", 0), theta[0], theta[1]))
+    _check(load().vtoken_repack_waves(ctx, ctypes.byref(pin), po, num_waves, ctypes.byref(wout), _stream(stream)),
+           "vtoken_repack_waves", ctx)

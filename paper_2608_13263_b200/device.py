@@ -17,7 +17,7 @@ from .workloads import Workload
 
 class DeviceProblem:
     def __init__(self, w: Workload, device="cuda:0", fill_seed: int = 1, copy_variant: int = 0, max_ctas: int = 0,
-                 capacity_slack: int = 0, allocate_pools: bool = True):
+                 capacity_slack: int = 0, allocate_pools: bool = True, wave_capacity: bool = False):
         self.w = w
         self.device = torch.device(device)
         self.fill_seed = fill_seed
@@ -27,6 +27,9 @@ class DeviceProblem:
         self.max_tokens = max(1, T + capacity_slack)
         self.max_table_blocks = max(1, NBT + capacity_slack)
         self.max_free = max(1, len(w.free_blocks) + capacity_slack)
+        if wave_capacity:       # a pool that takes back every reclaimed block (repack in waves)
+            self.max_free += self.max_table_blocks
+        self._waves = None
 
         def up(a, dtype):
             t = torch.from_numpy(np.ascontiguousarray(a, dtype=dtype))
@@ -118,6 +121,49 @@ class DeviceProblem:
     def repack(self, stream=None):
         vt.vtoken_repack(self.ctx, stream=stream)
 
+    def repack_waves(self, num_waves: int, num_free=None, partial=None, stream=None):
+        """Plan + copy + commit, ``num_waves`` times, reclaimed blocks feeding the next wave.  Needs
+        ``wave_capacity=True`` at construction.  Results: ``waves_outputs()``."""
+        dev = self.device
+        if self._waves is None or self._waves["counts"].shape[0] < num_waves:
+            i32 = dict(dtype=torch.int32, device=dev)
+            nbytes = vt.vtoken_waves_workspace_bytes(self.ctx, self.max_free)
+            self._waves = dict(req_wave=torch.full((self.max_requests,), -9, **i32),
+                               free_out=torch.full((self.max_free,), -9, **i32),
+                               num_free_out=torch.full((1,), -9, **i32),
+                               counts=torch.zeros((num_waves, 8), **i32),
+                               workspace=torch.empty(max(16, nbytes), dtype=torch.uint8, device=dev), nbytes=nbytes)
+        wv = self._waves
+        vt.vtoken_repack_waves(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
+                               bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
+                               keep=self.keep, free_blocks=self.free_blocks,
+                               num_free=self.num_free if num_free is None else num_free, num_waves=num_waves,
+                               new_bt_offsets=self.new_bt_offsets, new_bt_blocks=self.new_bt_blocks,
+                               new_tt_slots=self.new_tt_slots, req_status=self.req_status, req_wave=wv["req_wave"],
+                               free_out=wv["free_out"], num_free_out=wv["num_free_out"], wave_counts=wv["counts"],
+                               free_capacity=self.max_free, workspace=wv["workspace"], workspace_bytes=wv["nbytes"],
+                               select=self.select, thr_num=self.w.thr_num, thr_den=self.w.thr_den, partial=partial,
+                               stream=stream)
+
+    def waves_outputs(self, num_waves: int) -> dict:
+        """Host copies of the outputs of ``repack_waves``."""
+        torch.cuda.synchronize(self.device)
+        R, T = self.w.num_requests, self.w.num_tokens
+        wv = self._waves
+        names = ["num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"]
+        c = wv["counts"].cpu().numpy()[:num_waves]
+        out = dict(wave_counts=[dict({n: int(row[i]) for i, n in enumerate(names)}, error_flags=int(np.uint32(row[6])))
+                                for row in c])
+        nbo = self.new_bt_offsets.cpu().numpy()[:R + 1]
+        out["new_bt_offsets"] = nbo
+        out["new_bt_blocks"] = self.new_bt_blocks.cpu().numpy()[:int(nbo[R])]
+        out["new_tt_slots"] = self.new_tt_slots.cpu().numpy()[:T]
+        out["req_status"] = self.req_status.cpu().numpy()[:R]
+        out["req_wave"] = wv["req_wave"].cpu().numpy()[:R]
+        nfo = int(wv["num_free_out"].item())
+        out["free_out"] = wv["free_out"].cpu().numpy()[:nfo]
+        return out
+
     def read_counts(self, stream=None) -> dict:
         return vt.vtoken_read_counts(self.ctx, stream=stream)
 
@@ -163,8 +209,13 @@ class DeviceProblem:
             pass
 
 
-def origin_map(slots_per_layer: int, move_src: np.ndarray, move_dst: np.ndarray) -> np.ndarray:
-    """origin[s] = the slot whose pre-repack bytes slot s must hold after the moves."""
+def origin_map(slots_per_layer: int, move_src: np.ndarray, move_dst: np.ndarray, wave_offsets=None) -> np.ndarray:
+    """origin[s] = the slot whose pre-repack bytes slot s must hold after the moves.  With
+    ``wave_offsets`` the list holds several waves back to back, applied in order (a later wave may
+    copy from, or overwrite, rows an earlier wave has written or read)."""
     origin = np.arange(slots_per_layer, dtype=np.int32)
-    origin[move_dst] = move_src
+    if wave_offsets is None:
+        wave_offsets = [0, len(move_src)]
+    for a, b in zip(wave_offsets[:-1], wave_offsets[1:]):
+        origin[move_dst[a:b]] = origin[move_src[a:b]]      # within a wave sources and destinations are disjoint
     return origin

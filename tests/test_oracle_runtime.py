@@ -118,3 +118,83 @@ def test_serving_loop_against_a_dictionary_cache(seed, S):
         assert len(used) == len(st.bt_blocks) and not (used & set(st.free))
         live_blocks = set((slots // S).tolist())
         assert live_blocks <= used
+
+
+# ---- cached slot-translation arrays ---------------------------------------------------------------
+def _new_cache(st):
+    n = int(st.tt_offsets[-1])
+    return dict(dirty=np.zeros(st.R, np.uint8), slots=np.full(n, -77, np.int32), ids=np.full(n, -77, np.int32),
+                len=np.zeros(st.R, np.int32), seen=np.zeros(st.R, np.int32))
+
+
+def _update(st, c):
+    return vto.slot_cache_update(st.tt_offsets, st.tt_slots, st.keep, st.tt_len, c["dirty"], c["slots"], c["ids"],
+                                 c["len"], c["seen"])
+
+
+@pytest.mark.parametrize("seed,S", [(0, 4), (1, 16), (2, 3)])
+def test_slot_cache_follows_a_serving_loop(seed, S):
+    """Marks after evictions and commits, one update per step: every request's cached array must
+    equal its slot mapping (a separately pinned routine) and the dictionary's live ids; requests
+    that were neither marked nor grown are not touched at all; the numbers of rebuilt / appended
+    requests are the ones the test's own bookkeeping predicts."""
+    from runtime_sim import Append, Evict, Repack
+    rng = np.random.default_rng(seed)
+    R = 6
+    st = ServingState.random(rng, S, R, capacity=200, num_blocks=500)
+    truth = DictCache()
+    c = _new_cache(st)
+    saw_append_only = saw_rebuild = False
+    for step in random_serving_steps(rng, st, steps=30):
+        before_len = st.tt_len.copy()
+        step.run_on_oracle(st, None, truth)
+        touched = set()
+        if isinstance(step, Evict):
+            vto.slot_cache_mark(c["dirty"], victim_req=step.victim_req)
+            touched = {int(r) for r in step.victim_req if 0 <= r < R}
+        elif isinstance(step, Repack):
+            vto.slot_cache_mark(c["dirty"], req_status=step.last_plan.req_status)
+            touched = set(np.flatnonzero(step.last_plan.req_status == vto.REPACKED).tolist())
+        assert set(np.flatnonzero(c["dirty"]).tolist()) == touched
+        grown = {r for r in range(R) if st.tt_len[r] > c["seen"][r]} - touched
+        snapshot = {k: v.copy() for k, v in c.items()}
+        nr, na = _update(st, c)
+        assert (nr, na) == (len(touched), len(grown)) and not c["dirty"].any()
+        saw_append_only |= bool(grown) and isinstance(step, Append)
+        saw_rebuild |= bool(touched)
+        slots, ids, off = vto.build_slot_mapping(st.tt_offsets, st.tt_slots, st.keep)
+        for r in range(R):
+            b = int(st.tt_offsets[r])
+            n = int(c["len"][r])
+            assert c["slots"][b:b + n].tolist() == slots[off[r]:off[r + 1]].tolist()
+            assert c["ids"][b:b + n].tolist() == ids[off[r]:off[r + 1]].tolist() == truth.live_tokens(r)
+            assert c["seen"][r] == st.tt_len[r]
+            if r not in touched and r not in grown:
+                e = int(st.tt_offsets[r + 1])
+                assert np.array_equal(c["slots"][b:e], snapshot["slots"][b:e])
+                assert np.array_equal(c["ids"][b:e], snapshot["ids"][b:e])
+            elif r in grown:                    # append-only: the old prefix stays, entries are added behind it
+                n0 = int(snapshot["len"][r])
+                assert n >= n0 and np.array_equal(c["slots"][b:b + n0], snapshot["slots"][b:b + n0])
+    assert saw_append_only and saw_rebuild
+
+
+def test_slot_cache_is_stale_until_the_change_is_marked():
+    """The update must not rebuild on its own: an eviction that nobody marked leaves the cached
+    array as it was (that is the point of refreshing only after structural changes), and the mark
+    repairs it."""
+    S = 4
+    st = ServingState.empty(S, capacities=[16], block_lists=[np.array([3, 1, 2], np.int32)])
+    vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets, st.bt_blocks, [9])
+    c = _new_cache(st)
+    assert _update(st, c) == (0, 1)
+    assert c["slots"][:9].tolist() == [12, 13, 14, 15, 4, 5, 6, 7, 8] and c["len"].tolist() == [9]
+    vto.evict_tokens(st.tt_offsets, st.tt_len, st.keep, [0, 0], [1, 6])
+    assert _update(st, c) == (0, 0) and c["len"].tolist() == [9]          # unmarked: untouched
+    vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets, st.bt_blocks, [11])
+    assert _update(st, c) == (0, 1)
+    assert c["slots"][:11].tolist() == [12, 13, 14, 15, 4, 5, 6, 7, 8, 9, 10]   # appended behind the stale entries
+    vto.slot_cache_mark(c["dirty"], victim_req=[0, 0, 5, -1])                   # out-of-range requests are skipped
+    assert _update(st, c) == (1, 0)
+    assert c["slots"][:9].tolist() == [12, 14, 15, 4, 5, 7, 8, 9, 10] and c["len"].tolist() == [9]
+    assert c["ids"][:9].tolist() == [0, 2, 3, 4, 5, 7, 8, 9, 10] and c["seen"].tolist() == [11]

@@ -672,13 +672,48 @@ def run_runtime(args, prob, w, side, dev):
                                  layer_end=g_layers, out_k=gk, out_v=gv, out_capacity_tokens=max(1, live),
                                  out_offsets=out_off, stream=st)
 
+    # cached slot-translation arrays over the same tables: rebuild of every request (all marked),
+    # the append-only refresh after a decode step (the last registered token of every request is new
+    # to the cache), and a step in which nothing changed
+    c_slots = torch.full((max(1, T),), -1, **i32)
+    c_ids = torch.full((max(1, T),), -1, **i32)
+    c_len, c_seen = torch.zeros(R, **i32), torch.zeros(R, **i32)
+    c_dirty = torch.zeros(R, dtype=torch.uint8, device=dev)
+    full_len = d(lens)
+
+    def cache_update(st):
+        vt.vtoken_slot_cache_update(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                    tt_slots=prob.tt_slots, keep=prob.keep, tt_len=full_len, dirty=c_dirty,
+                                    cache_slots=c_slots, cache_ids=c_ids, cache_len=c_len, cache_seen=c_seen, stream=st)
+
+    def cache_rebuild(st):
+        c_dirty.fill_(1)
+        cache_update(st)
+
+    c_dirty.fill_(1)
+    cache_update(torch.cuda.current_stream())
+    torch.cuda.synchronize(dev)
+    last_live = torch.from_numpy(np.ascontiguousarray(
+        ((w.tt_slots >= 0) & (w.keep != 0))[np.maximum(w.tt_offsets[1:] - 1, 0)] & (lens > 0))).to(dev)
+    seen_before = torch.clamp(full_len - 1, min=0)
+    len_before = c_len - last_live.to(torch.int32)
+
+    def cache_append(st):
+        c_seen.copy_(seen_before)
+        c_len.copy_(len_before)
+        cache_update(st)
+
     out = {}
-    table_bytes = {"slot_mapping": 2 * 5 * T + 8 * live, "append_one_token_per_request": R * (4 * 6 + 5),
+    table_bytes = {"slot_cache_rebuild_all": 5 * T + 8 * live, "slot_cache_append_one_token_per_request": R * 40,
+                   "slot_cache_nothing_changed": R * 13,
+                   "slot_mapping": 2 * 5 * T + 8 * live, "append_one_token_per_request": R * (4 * 6 + 5),
                    "evict_64k_victims": nv * (8 + 4 + 4 + 1), "apply_moves": T * (4 + 4 + 1),
                    "digest_all_layers": live * w.token_bytes, "gather_logical": 2 * live * 2 * g_layers * w.row_bytes}
     for name, fn in (("slot_mapping", slot_mapping), ("append_one_token_per_request", append),
                      ("evict_64k_victims", evict), ("apply_moves", commit), ("digest_all_layers", digest),
-                     ("gather_logical", gather)):
+                     ("gather_logical", gather), ("slot_cache_rebuild_all", cache_rebuild),
+                     ("slot_cache_append_one_token_per_request", cache_append),
+                     ("slot_cache_nothing_changed", cache_update)):
         with torch.cuda.stream(side):
             fn(side)
         side.synchronize()
@@ -698,6 +733,8 @@ def run_runtime(args, prob, w, side, dev):
         us = e0.elapsed_time(e1) / reps * 1e3
         out[name] = {"us": us, "table_bytes": table_bytes[name], "GBs": table_bytes[name] / us / 1e3}
     out["entries"] = {"logical_tokens": T, "live_tokens": live, "requests": R, "gather_layers": g_layers}
+    out["slot_cache_note"] = ("rebuild_all includes a fill of the marks, append includes two small device copies that "
+                              "wind the cache back by one token per request before every replay")
     out["note"] = ("append after the first replay is a no-op per request (tt_len already equals new_len): the figure "
                    "is the launch + per-request check cost of a decode step")
     return out

@@ -337,6 +337,32 @@ int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32
                        int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
                        const int32_t *req_status, void *cuda_stream);
 
+/* Cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4): per request the slots (and
+ * ids) of its active tokens in token-id order, kept on the device between decode steps and
+ * refreshed only after structural changes -- appended to when the sequence merely grew, rebuilt
+ * after an eviction or a relocation.  Layout: the cache of request r occupies cache_slots /
+ * cache_ids [tt_offsets[r] ..) (the capacity of its token table); cache_len[r] entries are valid
+ * and cover the first cache_seen[r] registered tokens; dirty[r] != 0 asks for a rebuild.  A fresh
+ * cache is cache_len = cache_seen = 0 (dirty anything).  All pointers DEVICE.
+ *
+ * vtoken_slot_cache_mark: dirty[r] = 1 for the request of each of the first *num_victims
+ * (<= max_victims) entries of victim_req (requests outside [0, R) are skipped) and for every request
+ * whose req_status is VTOKEN_REPACKED.  victim_req / num_victims may be NULL (max_victims 0), and
+ * so may req_status: call it with the victims after vtoken_evict_tokens and with the plan's
+ * statuses after vtoken_apply_moves.
+ *
+ * vtoken_slot_cache_update, per request: dirty -> rebuild from the first tt_len[r] entries, clear
+ * the mark; else tt_len[r] > cache_seen[r] -> append the active ones among the new entries; else
+ * nothing is read or written.  cache_ids may be NULL.  stats: DEVICE int32[2] or NULL, receives
+ * {requests rebuilt, requests appended to}. */
+int vtoken_slot_cache_mark(vtoken_ctx *ctx, uint8_t *dirty, const int32_t *num_victims, int32_t max_victims,
+                           const int32_t *victim_req, const int32_t *req_status, const int32_t *num_requests,
+                           void *cuda_stream);
+int vtoken_slot_cache_update(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                             const int32_t *tt_slots, const uint8_t *keep, const int32_t *tt_len, uint8_t *dirty,
+                             int32_t *cache_slots, int32_t *cache_ids, int32_t *cache_len, int32_t *cache_seen,
+                             int32_t *stats, void *cuda_stream);
+
 /* Host-table front end.  The paper keeps the canonical token table on the CPU (Sec. 3.2);
  * this entry point serves such a caller: all tables are HOST memory (pinned for speed), the
  * pools stay on the device.  Copies the inputs to device staging owned by the context, runs

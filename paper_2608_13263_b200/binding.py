@@ -22,7 +22,8 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
-           "vtoken_waves_workspace_bytes", "vtoken_repack_waves"]
+           "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
+           "vtoken_slot_cache_update"]
 
 
 class VtokenError(RuntimeError):
@@ -149,6 +150,9 @@ def load():
         lib.vtoken_waves_workspace_bytes.restype = ctypes.c_int64
         lib.vtoken_repack_waves.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
                                             ctypes.c_int32, ctypes.POINTER(WavesOut), ctypes.c_void_p]
+        lib.vtoken_slot_cache_mark.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32] + \
+                                              [ctypes.c_void_p] * 4
+        lib.vtoken_slot_cache_update.argtypes = [ctypes.c_void_p] * 13
         _lib = lib
     return _lib
 
@@ -295,6 +299,21 @@ def vtoken_apply_moves(ctx, *, num_requests, tt_offsets, tt_slots, keep, phys_le
     _check(load().vtoken_apply_moves(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                                      _ptr(phys_len), _ptr(new_tt_slots), _ptr(req_status), _stream(stream)),
            "vtoken_apply_moves", ctx)
+
+
+def vtoken_slot_cache_mark(ctx, *, dirty, num_requests, num_victims=None, max_victims=0, victim_req=None,
+                           req_status=None, stream=None) -> None:
+    _check(load().vtoken_slot_cache_mark(ctx, _ptr(dirty), _ptr(num_victims), max_victims, _ptr(victim_req),
+                                         _ptr(req_status), _ptr(num_requests), _stream(stream)),
+           "vtoken_slot_cache_mark", ctx)
+
+
+def vtoken_slot_cache_update(ctx, *, num_requests, tt_offsets, tt_slots, keep, tt_len, dirty, cache_slots, cache_len,
+                             cache_seen, cache_ids=None, stats=None, stream=None) -> None:
+    _check(load().vtoken_slot_cache_update(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                                           _ptr(tt_len), _ptr(dirty), _ptr(cache_slots), _ptr(cache_ids),
+                                           _ptr(cache_len), _ptr(cache_seen), _ptr(stats), _stream(stream)),
+           "vtoken_slot_cache_update", ctx)
 
 
 # ---- eligibility metadata and partial plans ---------------------------------------------------

@@ -51,6 +51,13 @@ class DeviceServing:
         self.map_slots = torch.zeros(cap, **i32)
         self.map_ids = torch.zeros(cap, **i32)
         self.map_offsets = torch.zeros(st.R + 1, **i32)
+        # cached slot-translation arrays (poisoned so that untouched entries are recognisable)
+        self.dirty = torch.zeros(st.R, dtype=torch.uint8, device=dev)
+        self.cache_slots = torch.full((cap,), -77, **i32)
+        self.cache_ids = torch.full((cap,), -77, **i32)
+        self.cache_len = torch.zeros(st.R, **i32)
+        self.cache_seen = torch.zeros(st.R, **i32)
+        self.cache_stats = torch.zeros(2, **i32)
         self.k_pool = torch.zeros((layers, self.NB * self.S, row_elems), dtype=torch.int16, device=dev)
         self.v_pool = torch.zeros_like(self.k_pool)
         self.ctx = vt.vtoken_create(layers, self.NB, self.S, 1, row_elems, self.k_pool, self.v_pool, st.R, cap,
@@ -127,6 +134,20 @@ class DeviceServing:
         n = int(off[self.R])
         return self.map_slots.cpu().numpy()[:n], self.map_ids.cpu().numpy()[:n], off
 
+    def cache_mark(self, victims=False, status=False):
+        vt.vtoken_slot_cache_mark(self.ctx, dirty=self.dirty, num_requests=self.num_requests,
+                                  num_victims=self.num_victims if victims else None,
+                                  max_victims=self.max_victims if victims else 0,
+                                  victim_req=self.victim_req if victims else None,
+                                  req_status=self.req_status if status else None)
+
+    def cache_update(self):
+        vt.vtoken_slot_cache_update(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
+                                    tt_slots=self.tt_slots, keep=self.keep, tt_len=self.tt_len, dirty=self.dirty,
+                                    cache_slots=self.cache_slots, cache_ids=self.cache_ids, cache_len=self.cache_len,
+                                    cache_seen=self.cache_seen, stats=self.cache_stats)
+        return tuple(self.cache_stats.cpu().numpy().tolist())
+
     def close(self):
         self.torch.cuda.synchronize()
         vt.vtoken_destroy(self.ctx)
@@ -140,6 +161,9 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S):
     st = ServingState.random(rng, S, R, capacity=200, num_blocks=400)
     truth = DictCache()
     dev = DeviceServing(st)
+    n_cap = int(st.tt_offsets[-1])
+    oc = dict(dirty=np.zeros(R, np.uint8), slots=np.full(n_cap, -77, np.int32), ids=np.full(n_cap, -77, np.int32),
+              len=np.zeros(R, np.int32), seen=np.zeros(R, np.int32))      # the oracle's cached arrays
     repacked_something = False
     for step in random_serving_steps(rng, st, steps=25):
         if isinstance(step, Append):
@@ -149,6 +173,8 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S):
         elif isinstance(step, Evict):
             step.run_on_oracle(st, None, truth)
             dev.evict(step.victim_req, step.victim_tok)
+            vto.slot_cache_mark(oc["dirty"], victim_req=step.victim_req)
+            dev.cache_mark(victims=True)
         else:
             free = list(st.free)
             nf = len(free) if step.num_free_limit < 0 else min(len(free), step.num_free_limit)
@@ -167,7 +193,19 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S):
             assert np.array_equal(dev.new_bt_blocks.cpu().numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
             assert np.array_equal(dev.freed_blocks.cpu().numpy()[:p.num_freed], p.freed_blocks)
             assert len(blocks_before) >= len(p.new_bt_blocks)
+            vto.slot_cache_mark(oc["dirty"], req_status=p.req_status)
+            dev.cache_mark(status=True)
         torch.cuda.synchronize()
+        # cached slot-translation arrays: marks, then one update per step, everything bit for bit
+        assert np.array_equal(dev.dirty.cpu().numpy(), oc["dirty"])
+        want_stats = vto.slot_cache_update(st.tt_offsets, st.tt_slots, st.keep, st.tt_len, oc["dirty"], oc["slots"],
+                                           oc["ids"], oc["len"], oc["seen"])
+        assert dev.cache_update() == want_stats
+        assert np.array_equal(dev.cache_slots.cpu().numpy(), oc["slots"])
+        assert np.array_equal(dev.cache_ids.cpu().numpy(), oc["ids"])
+        assert np.array_equal(dev.cache_len.cpu().numpy(), oc["len"])
+        assert np.array_equal(dev.cache_seen.cpu().numpy(), oc["seen"])
+        assert not dev.dirty.cpu().numpy().any()
         # table state
         assert np.array_equal(dev.tt_slots.cpu().numpy(), st.tt_slots)
         assert np.array_equal(dev.keep.cpu().numpy(), st.keep)
@@ -262,4 +300,67 @@ def test_slot_mapping_full_size_tables_match_oracle():
     assert np.array_equal(out_off.cpu().numpy(), o_off)
     assert np.array_equal(out_slots.cpu().numpy()[:n], o_slots)
     assert np.array_equal(out_ids.cpu().numpy()[:n], o_ids)
+    vt.vtoken_destroy(ctx)
+
+
+def test_slot_cache_full_size_rebuild_then_append_only():
+    """Steady-state tables (2.2 M entries, 512 requests) with one spare entry per request: a fresh
+    cache is rebuilt for every request and equals the slot mapping; a decode step that appends one
+    token per request then only appends; an eviction in three requests rebuilds exactly those."""
+    import torch
+    from paper_2608_13263_b200 import workloads as wl
+    w = wl.steady_state(seed=0)
+    R = w.num_requests
+    dev = torch.device("cuda:0")
+    lens = np.diff(w.tt_offsets).astype(np.int32)
+    cap_off = (w.tt_offsets.astype(np.int64) + np.arange(R + 1)).astype(np.int32)
+    n = int(cap_off[-1])
+    tt = np.full(n, -1, np.int32)
+    keep = np.zeros(n, np.uint8)
+    for r in range(R):
+        tt[cap_off[r]:cap_off[r] + lens[r]] = w.tt_slots[w.tt_offsets[r]:w.tt_offsets[r + 1]]
+        keep[cap_off[r]:cap_off[r] + lens[r]] = w.keep[w.tt_offsets[r]:w.tt_offsets[r + 1]]
+    tt_len = lens.copy()
+    pool = torch.zeros((1, w.slots_per_layer, 8), dtype=torch.int16, device=dev)
+    ctx = vt.vtoken_create(1, w.num_blocks, w.block_size, 1, 8, pool, pool, R, n, len(w.bt_blocks), 1)
+    d = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    g = dict(num_requests=d(np.array([R], np.int32)), tt_offsets=d(cap_off), tt_slots=d(tt), keep=d(keep),
+             tt_len=d(tt_len), dirty=d(np.ones(R, np.uint8)), cache_slots=d(np.full(n, -77, np.int32)),
+             cache_ids=d(np.full(n, -77, np.int32)), cache_len=d(np.zeros(R, np.int32)),
+             cache_seen=d(np.zeros(R, np.int32)), stats=d(np.zeros(2, np.int32)))
+    o = dict(dirty=np.ones(R, np.uint8), slots=np.full(n, -77, np.int32), ids=np.full(n, -77, np.int32),
+             len=np.zeros(R, np.int32), seen=np.zeros(R, np.int32))
+
+    def both(expect):
+        got = vto.slot_cache_update(cap_off, tt, keep, tt_len, o["dirty"], o["slots"], o["ids"], o["len"], o["seen"])
+        assert got == expect
+        vt.vtoken_slot_cache_update(ctx, **g)
+        torch.cuda.synchronize()
+        assert tuple(g["stats"].cpu().numpy().tolist()) == expect
+        for a, b in (("cache_slots", "slots"), ("cache_ids", "ids"), ("cache_len", "len"), ("cache_seen", "seen"),
+                     ("dirty", "dirty")):
+            assert np.array_equal(g[a].cpu().numpy(), o[b]), a
+
+    both((R, 0))
+    slots, ids, off = vto.build_slot_mapping(cap_off, tt, keep)
+    for r in (0, 1, R // 2, R - 1):
+        assert np.array_equal(o["slots"][cap_off[r]:cap_off[r] + o["len"][r]], slots[off[r]:off[r + 1]])
+    # one decode step: every request registers one token at a slot of its own
+    for r in range(R):
+        tt[cap_off[r] + tt_len[r]] = w.num_blocks * w.block_size - 1 - r
+        keep[cap_off[r] + tt_len[r]] = 1
+    tt_len += 1
+    g["tt_slots"].copy_(d(tt)); g["keep"].copy_(d(keep)); g["tt_len"].copy_(d(tt_len))
+    both((0, R))
+    both((0, 0))
+    # evictions in three requests, marked through the library
+    vr = np.array([3, 3, 100, R - 1], np.int32)
+    for r, t in zip(vr.tolist(), (0, 5, 7, 2)):
+        keep[cap_off[r] + t] = 0
+    g["keep"].copy_(d(keep))
+    vto.slot_cache_mark(o["dirty"], victim_req=vr)
+    vt.vtoken_slot_cache_mark(ctx, dirty=g["dirty"], num_requests=g["num_requests"],
+                              num_victims=d(np.array([4], np.int32)), max_victims=4, victim_req=d(vr))
+    both((3, 0))
+    assert vt.vtoken_read_counts(ctx)["error_flags"] == 0
     vt.vtoken_destroy(ctx)

@@ -199,6 +199,12 @@ __device__ __forceinline__ unsigned long long g_mix64(unsigned long long x)   //
 //   key(i, s) = mix(((i*A + t_i)*B + s)*C);  digest[r] = sum over (rank i, slab s, 8-byte word j) of mix(w ^ (key + j*D))
 // a sum of position-bound terms, so any evaluation order gives the same 64-bit value.
 // One warp per (slab, output row); lanes take 16-byte pieces of the row.
+// One (slab, row) unit of the digest: where it is and what it hashes.
+struct DigestRow {
+    int32_t src, r, tok, slab;
+    int64_t idx;
+};
+
 __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
 {
     const unsigned long long A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull,
@@ -216,6 +222,7 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     const int64_t chunk = (total + nwarps - 1) / nwarps;
     const int64_t w = (int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5);
     const int64_t u0 = w * chunk, u1 = min(total, u0 + chunk);
+    if (u0 >= u1) return;
     unsigned long long sum = 0;
     int cur_r = -1;
     auto flush = [&]() {
@@ -224,55 +231,74 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         if (lane == 0 && cur_r >= 0 && sum != 0) atomicAdd(&a.digest[cur_r], sum);
         sum = 0;
     };
-    // the table entries of a row (source slot, request, logical id) are fetched one row ahead
-    int32_t nx_src = 0, nx_r = 0, nx_t = 0;
-    if (u0 < u1) {
-        const int64_t idx0 = u0 % n;
-        nx_src = a.g_src[idx0];
-        nx_r = a.g_req[idx0];
-        nx_t = a.g_ids[idx0];
-    }
-    int slab = u0 < u1 ? (int)(u0 / n) : 0;
-    int64_t idx = u0 < u1 ? u0 - (int64_t)slab * n : 0;
-    for (int64_t u = u0; u < u1; ++u) {
-        const int li = slab < nl ? slab : slab - nl;
-        const uint8_t *pool = slab < nl ? a.k_pool : a.v_pool;
-        const int32_t src = nx_src;
-        const int r = nx_r;
-        const int32_t tok = nx_t;
-        const int cur_slab = slab;
-        const int64_t cur_idx = idx;
-        if (++idx == n) { idx = 0; ++slab; }
-        if (u + 1 < u1) {
-            nx_src = a.g_src[idx];
-            nx_r = a.g_req[idx];
-            nx_t = a.g_ids[idx];
-        }
-        if (r != cur_r) {
-            flush();
-            cur_r = r;
-        }
-        const unsigned long long i = (unsigned long long)(cur_idx - a.out_offsets[r]);
-        const unsigned long long t = (unsigned long long)tok;
-        const unsigned long long key = g_mix64(((i * A + t) * B + (unsigned long long)cur_slab) * C);
-        const uint4 *sp = reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
-                                                          (int64_t)src * a.row_bytes);
-        for (int c0 = lane; c0 < row_vecs; c0 += 128) {       // four 16-byte loads in flight per lane
-            uint4 v[4];
+    auto row_ptr = [&](const DigestRow &m) {
+        const int li = m.slab < nl ? m.slab : m.slab - nl;
+        const uint8_t *pool = m.slab < nl ? a.k_pool : a.v_pool;
+        return reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
+                                               (int64_t)m.src * a.row_bytes);
+    };
+    auto fetch_meta = [&](DigestRow &m, int slab, int64_t idx) {
+        m.slab = slab;
+        m.idx = idx;
+        m.src = a.g_src[idx];
+        m.r = a.g_req[idx];
+        m.tok = a.g_ids[idx];
+    };
+    auto load4 = [&](uint4 (&v)[4], const uint4 *sp, int c0) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                v[k] = (c0 + 32 * k < row_vecs) ? ld_stream(sp + c0 + 32 * k) : make_uint4(0, 0, 0, 0);
+        for (int k = 0; k < 4; ++k)
+            v[k] = (c0 + 32 * k < row_vecs) ? ld_stream(sp + c0 + 32 * k) : make_uint4(0, 0, 0, 0);
+    };
+    auto hash4 = [&](const uint4 (&v)[4], unsigned long long key, int c0) {
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                const int c = c0 + 32 * k;
-                if (c < row_vecs) {
-                    const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
-                    const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
-                    sum += g_mix64(w0 ^ (key + (2ull * c) * D));
-                    sum += g_mix64(w1 ^ (key + (2ull * c + 1ull) * D));
-                }
+        for (int k = 0; k < 4; ++k) {
+            const int c = c0 + 32 * k;
+            if (c < row_vecs) {
+                const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
+                const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
+                sum += g_mix64(w0 ^ (key + (2ull * c) * D));
+                sum += g_mix64(w1 ^ (key + (2ull * c + 1ull) * D));
             }
         }
+    };
+    // Software pipeline over rows: the table entries of a row (source slot, request, logical id)
+    // are fetched two rows ahead and the first 2 KiB of its K/V row one row ahead, so that a warp
+    // always has a row in flight while it hashes the previous one.
+    int slab = (int)(u0 / n);
+    int64_t idx = u0 - (int64_t)slab * n;
+    auto advance = [&]() { if (++idx == n) { idx = 0; ++slab; } };
+    DigestRow cur, nxt;
+    fetch_meta(cur, slab, idx);
+    advance();
+    if (u0 + 1 < u1) { fetch_meta(nxt, slab, idx); advance(); }
+    uint4 vc[4], vn[4];
+    load4(vc, row_ptr(cur), lane);
+    for (int64_t u = u0; u < u1; ++u) {
+        const bool has_next = u + 1 < u1;
+        const uint4 *np = has_next ? row_ptr(nxt) : nullptr;
+        if (has_next) load4(vn, np, lane);
+        DigestRow nn = nxt;
+        if (u + 2 < u1) { fetch_meta(nn, slab, idx); advance(); }
+        if (cur.r != cur_r) {
+            flush();
+            cur_r = cur.r;
+        }
+        const unsigned long long i = (unsigned long long)(cur.idx - a.out_offsets[cur.r]);
+        const unsigned long long key =
+            g_mix64(((i * A + (unsigned long long)cur.tok) * B + (unsigned long long)cur.slab) * C);
+        hash4(vc, key, lane);
+        if (row_vecs > 128) {                                  // rows above 2 KiB: the rest, unpipelined
+            const uint4 *sp = row_ptr(cur);
+            for (int c0 = lane + 128; c0 < row_vecs; c0 += 128) {
+                uint4 v[4];
+                load4(v, sp, c0);
+                hash4(v, key, c0);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) vc[k] = vn[k];
+        cur = nxt;
+        nxt = nn;
     }
     flush();
 }

@@ -578,7 +578,7 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
                        int64_t row_bytes, int32_t layer_begin, int32_t layer_end, const int32_t *tt_slots,
                        const uint8_t *keep, int32_t len, uint64_t *digest, int32_t *num_active)
 {
-    if (!k_pool || !v_pool || !tt_slots || !digest || row_bytes < 8 || row_bytes % 8 != 0) return VTO_EINVAL;
+    if (!k_pool || !v_pool || !tt_slots || !digest || row_bytes < 16 || row_bytes % 16 != 0) return VTO_EINVAL;
     if (layer_begin < 0 || layer_end <= layer_begin || len < 0) return VTO_EINVAL;
     if (layer_stride_bytes == 0) layer_stride_bytes = num_slots * row_bytes;
     const uint64_t A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull,
@@ -595,10 +595,16 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
             const uint8_t *row = pool + (int64_t)layer * layer_stride_bytes + (int64_t)tt_slots[t] * row_bytes;
             /* key of this (rank, id, slab): binds the row's words to their place in the logical view */
             const uint64_t key = mix64((((uint64_t)i * A + (uint64_t)t) * B + (uint64_t)s) * C);
-            for (int64_t j = 0; j < row_bytes / 8; ++j) {
-                uint64_t w = 0;
-                for (int b = 7; b >= 0; --b) w = (w << 8) | row[j * 8 + b];       /* little-endian word */
-                sum += mix64(w ^ (key + (uint64_t)j * D));
+            for (int64_t c = 0; c < row_bytes / 16; ++c) {   /* 16 bytes = two little-endian words */
+                uint64_t w0 = 0, w1 = 0;
+                for (int b = 7; b >= 0; --b) {
+                    w0 = (w0 << 8) | row[c * 16 + b];
+                    w1 = (w1 << 8) | row[c * 16 + 8 + b];
+                }
+                const uint64_t a = w0 ^ (key + (uint64_t)(2 * c) * D);
+                const uint64_t b = w1 ^ (key + (uint64_t)(2 * c + 1) * D);
+                const unsigned __int128 prod = (unsigned __int128)a * b;      /* full 128-bit product */
+                sum += (uint64_t)prod ^ (uint64_t)(prod >> 64);
             }
         }
         ++i;

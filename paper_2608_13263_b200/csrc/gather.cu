@@ -196,13 +196,13 @@ __device__ __forceinline__ unsigned long long g_mix64(unsigned long long x)   //
 }
 
 // Relocation digest (Sec. 5 of the paper hashes ordered retained ids with their K/V contents):
-//   key(i, s) = mix(((i*A + t_i)*B + s)*C);  digest[r] = sum over (rank i, slab s, 8-byte word j) of mix(w ^ (key + j*D))
+//   key(i, s) = mix(((i*A + t_i)*B + s)*C);  per 16-byte group c of the row (8-byte words w0, w1):
+//   x = w0 ^ (key + 2c*D), y = w1 ^ (key + (2c+1)*D);  digest[r] = sum of low64(x*y) ^ high64(x*y)
 // a sum of position-bound terms, so any evaluation order gives the same 64-bit value.
-// One warp per (slab, output row); lanes take 16-byte pieces of the row.
+// A warp walks a contiguous run of (slab, output row) units; lanes take 16-byte groups of the row.
 // One (slab, row) unit of the digest: where it is and what it hashes.
 struct DigestRow {
-    int32_t src, r, tok, slab;
-    int64_t idx;
+    int32_t src, r, tok, slab, idx;
 };
 
 __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
@@ -237,7 +237,7 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         return reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
                                                (int64_t)m.src * a.row_bytes);
     };
-    auto fetch_meta = [&](DigestRow &m, int slab, int64_t idx) {
+    auto fetch_meta = [&](DigestRow &m, int slab, int32_t idx) {
         m.slab = slab;
         m.idx = idx;
         m.src = a.g_src[idx];
@@ -256,8 +256,9 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
             if (c < row_vecs) {
                 const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
                 const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
-                sum += g_mix64(w0 ^ (key + (2ull * c) * D));
-                sum += g_mix64(w1 ^ (key + (2ull * c + 1ull) * D));
+                const unsigned long long x = w0 ^ (key + (2ull * c) * D);
+                const unsigned long long y = w1 ^ (key + (2ull * c + 1ull) * D);
+                sum += (x * y) ^ __umul64hi(x, y);                 // low64 ^ high64 of the 128-bit product
             }
         }
     };
@@ -265,20 +266,21 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     // are fetched two rows ahead and the first 2 KiB of its K/V row one row ahead, so that a warp
     // always has a row in flight while it hashes the previous one.
     int slab = (int)(u0 / n);
-    int64_t idx = u0 - (int64_t)slab * n;
-    auto advance = [&]() { if (++idx == n) { idx = 0; ++slab; } };
+    int32_t idx = (int32_t)(u0 - (int64_t)slab * n);             // n < 2^31: it counts token-table entries
+    const int32_t n32 = (int32_t)n;
+    auto advance = [&]() { if (++idx == n32) { idx = 0; ++slab; } };
     DigestRow cur, nxt;
     fetch_meta(cur, slab, idx);
     advance();
     if (u0 + 1 < u1) { fetch_meta(nxt, slab, idx); advance(); }
     uint4 vc[4], vn[4];
     load4(vc, row_ptr(cur), lane);
-    for (int64_t u = u0; u < u1; ++u) {
-        const bool has_next = u + 1 < u1;
+    for (int64_t left = u1 - u0; left > 0; --left) {
+        const bool has_next = left > 1;
         const uint4 *np = has_next ? row_ptr(nxt) : nullptr;
         if (has_next) load4(vn, np, lane);
         DigestRow nn = nxt;
-        if (u + 2 < u1) { fetch_meta(nn, slab, idx); advance(); }
+        if (left > 2) { fetch_meta(nn, slab, idx); advance(); }
         if (cur.r != cur_r) {
             flush();
             cur_r = cur.r;

@@ -19,6 +19,19 @@ def mix(x):
     return x
 
 
+M32 = np.uint64(0xFFFFFFFF)
+
+
+def fold128(a, b):
+    """low64(a*b) ^ high64(a*b) of uint64 arrays, from 32-bit halves (schoolbook product)."""
+    with np.errstate(over="ignore"):
+        al, ah, bl, bh = a & M32, a >> np.uint64(32), b & M32, b >> np.uint64(32)
+        ll, lh, hl, hh = al * bl, al * bh, ah * bl, ah * bh
+        mid = (ll >> np.uint64(32)) + (lh & M32) + (hl & M32)
+        hi = hh + (lh >> np.uint64(32)) + (hl >> np.uint64(32)) + (mid >> np.uint64(32))
+        return (a * b) ^ hi
+
+
 def numpy_digest(k, v, tt_slots, keep, l0, l1):
     live = np.flatnonzero((tt_slots >= 0) & (keep != 0))
     slots = tt_slots[live]
@@ -31,8 +44,35 @@ def numpy_digest(k, v, tt_slots, keep, l0, l1):
         s = np.arange(S_, dtype=np.uint64)[:, None, None]
         j = np.arange(W, dtype=np.uint64)[None, None, :]
         key = mix(((i * np.uint64(A) + t) * np.uint64(B) + s) * np.uint64(C))       # per (token, slab)
-        total = mix(words ^ (key + j * np.uint64(D))).sum(dtype=np.uint64)
+        x = words ^ (key + j * np.uint64(D))
+        total = fold128(x[..., 0::2], x[..., 1::2]).sum(dtype=np.uint64)
     return int(total), n
+
+
+def bigint_digest(k, v, tt_slots, keep):
+    """The definition with Python integers (exact 128-bit products), one word pair at a time."""
+    M = (1 << 64) - 1
+
+    def mixi(x):
+        x ^= x >> 30
+        x = x * 0xBF58476D1CE4E5B9 & M
+        x ^= x >> 27
+        x = x * 0x94D049BB133111EB & M
+        return x ^ x >> 31
+    L = k.shape[0]
+    total, i = 0, 0
+    for t in range(len(tt_slots)):
+        if tt_slots[t] < 0 or not keep[t]:
+            continue
+        for s in range(2 * L):
+            row = (k if s < L else v)[s % L, tt_slots[t]].tobytes()
+            key = mixi(((i * A + t) * B + s) * C & M)
+            for c in range(len(row) // 16):
+                a = int.from_bytes(row[16 * c:16 * c + 8], "little") ^ (key + 2 * c * D & M)
+                b = int.from_bytes(row[16 * c + 8:16 * c + 16], "little") ^ (key + (2 * c + 1) * D & M)
+                total = (total + ((a * b & M) ^ (a * b >> 64))) & M
+        i += 1
+    return total, i
 
 
 def pools(w, seed=1):
@@ -49,6 +89,25 @@ def test_digest_equals_vectorised_numpy_evaluation():
         for l0, l1 in ((0, 3), (1, 2)):
             assert vto.digest_logical(k, v, w.tt_slots[t0:t1], w.keep[t0:t1], l0, l1) == \
                    numpy_digest(k, v, w.tt_slots[t0:t1], w.keep[t0:t1], l0, l1)
+
+
+def test_digest_equals_exact_integer_evaluation_on_a_small_case():
+    w = wl.tiny(seed=3)
+    k, v = pools(w)
+    for r in range(w.num_requests):
+        t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
+        assert vto.digest_logical(k, v, w.tt_slots[t0:t1], w.keep[t0:t1]) == \
+               bigint_digest(k, v, w.tt_slots[t0:t1], w.keep[t0:t1])
+
+
+def test_fold128_helper_against_python_integers():
+    rng = np.random.default_rng(0)
+    a = rng.integers(0, 2 ** 64, size=2000, dtype=np.uint64)
+    b = rng.integers(0, 2 ** 64, size=2000, dtype=np.uint64)
+    a[:4] = [0, 2 ** 64 - 1, 2 ** 32, 2 ** 64 - 1]
+    b[:4] = [5, 2 ** 64 - 1, 2 ** 32, 1]
+    want = [((int(x) * int(y)) & (2 ** 64 - 1)) ^ ((int(x) * int(y)) >> 64) for x, y in zip(a, b)]
+    assert fold128(a, b).tolist() == want
 
 
 def test_digest_is_invariant_under_repack_and_catches_defects():

@@ -213,22 +213,29 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     const int nl = a.layer_end - a.layer_begin;
     const int64_t total = n * nl * 2;
     const int lane = vtk_lane();
-    const int64_t nwarps = (int64_t)gridDim.x * (GC_NT / 32);
     const int row_vecs = (int)(a.row_bytes >> 4);
-    // Each warp takes a contiguous run of (slab, row) pairs, so that consecutive rows mostly belong
+    // A row is hashed by a group of G lanes with four 16-byte loads each: the whole warp for rows
+    // of 2 KiB and more, half a warp for 1 KiB rows, ... so that every lane's loads carry bytes.
+    int G = 32;
+    while (G > 1 && 4 * G > row_vecs) G >>= 1;
+    const int gl = lane & (G - 1), per_warp = 32 / G;
+    const unsigned gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(G - 1)));
+    const int64_t ngroups = (int64_t)gridDim.x * (GC_NT / 32) * per_warp;
+    // Each group takes a contiguous run of (slab, row) pairs, so that consecutive rows mostly belong
     // to one request: the per-lane partial sums are folded into the request's digest only when the
     // request changes (one 64-bit atomic per run instead of one per row -- with one atomic per row
     // the kernel was bound by atomic throughput on a few addresses).
-    const int64_t chunk = (total + nwarps - 1) / nwarps;
-    const int64_t w = (int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5);
+    const int64_t chunk = (total + ngroups - 1) / ngroups;
+    const int64_t w = ((int64_t)blockIdx.x * (GC_NT / 32) + (threadIdx.x >> 5)) * per_warp + lane / G;
     const int64_t u0 = w * chunk, u1 = min(total, u0 + chunk);
-    if (u0 >= u1) return;
+    if (u0 >= u1) return;                                      // whole groups leave; shuffles below name gmask
     unsigned long long sum = 0;
     int cur_r = -1;
     auto flush = [&]() {
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) sum += __shfl_down_sync(0xffffffffu, sum, d);
-        if (lane == 0 && cur_r >= 0 && sum != 0) atomicAdd(&a.digest[cur_r], sum);
+        for (int d = 16; d > 0; d >>= 1)
+            if (d < G) sum += __shfl_down_sync(gmask, sum, d, G);
+        if (gl == 0 && cur_r >= 0 && sum != 0) atomicAdd(&a.digest[cur_r], sum);
         sum = 0;
     };
     auto row_ptr = [&](const DigestRow &m) {
@@ -247,12 +254,12 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     auto load4 = [&](uint4 (&v)[4], const uint4 *sp, int c0) {
 #pragma unroll
         for (int k = 0; k < 4; ++k)
-            v[k] = (c0 + 32 * k < row_vecs) ? ld_stream(sp + c0 + 32 * k) : make_uint4(0, 0, 0, 0);
+            v[k] = (c0 + G * k < row_vecs) ? ld_stream(sp + c0 + G * k) : make_uint4(0, 0, 0, 0);
     };
     auto hash4 = [&](const uint4 (&v)[4], unsigned long long key, int c0) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const int c = c0 + 32 * k;
+            const int c = c0 + G * k;
             if (c < row_vecs) {
                 const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
                 const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
@@ -263,8 +270,8 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         }
     };
     // Software pipeline over rows: the table entries of a row (source slot, request, logical id)
-    // are fetched two rows ahead and the first 2 KiB of its K/V row one row ahead, so that a warp
-    // always has a row in flight while it hashes the previous one.
+    // are fetched two rows ahead and the first 64 bytes per lane of its K/V row one row ahead, so
+    // that a group always has a row in flight while it hashes the previous one.
     int slab = (int)(u0 / n);
     int32_t idx = (int32_t)(u0 - (int64_t)slab * n);             // n < 2^31: it counts token-table entries
     const int32_t n32 = (int32_t)n;
@@ -274,11 +281,11 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     advance();
     if (u0 + 1 < u1) { fetch_meta(nxt, slab, idx); advance(); }
     uint4 vc[4], vn[4];
-    load4(vc, row_ptr(cur), lane);
+    load4(vc, row_ptr(cur), gl);
     for (int64_t left = u1 - u0; left > 0; --left) {
         const bool has_next = left > 1;
         const uint4 *np = has_next ? row_ptr(nxt) : nullptr;
-        if (has_next) load4(vn, np, lane);
+        if (has_next) load4(vn, np, gl);
         DigestRow nn = nxt;
         if (left > 2) { fetch_meta(nn, slab, idx); advance(); }
         if (cur.r != cur_r) {
@@ -288,10 +295,10 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         const unsigned long long i = (unsigned long long)(cur.idx - a.out_offsets[cur.r]);
         const unsigned long long key =
             g_mix64(((i * A + (unsigned long long)cur.tok) * B + (unsigned long long)cur.slab) * C);
-        hash4(vc, key, lane);
-        if (row_vecs > 128) {                                  // rows above 2 KiB: the rest, unpipelined
+        hash4(vc, key, gl);
+        if (row_vecs > 4 * G) {                                // rows above 64 bytes per lane: the rest, unpipelined
             const uint4 *sp = row_ptr(cur);
-            for (int c0 = lane + 128; c0 < row_vecs; c0 += 128) {
+            for (int c0 = gl + 4 * G; c0 < row_vecs; c0 += 4 * G) {
                 uint4 v[4];
                 load4(v, sp, c0);
                 hash4(v, key, c0);

@@ -30,7 +30,15 @@ def device_digest(prob, tt_slots, keep, l0, l1, select=None):
     wl.tiny(seed=0),
     wl.steady_state(seed=2, requests=9, lo=50, hi=900, layers=3, heads=2, head_dim=64),
     wl.longctx_scissor(seed=1, requests=2, lo=2000, hi=5000, layers=2),
-], ids=lambda w: w.name)
+    # row sizes that exercise every lane-group width of the kernel and its tail loop:
+    # 16 B, 48 B, 384 B, 1.5 KiB, 2 KiB, 4 KiB rows
+    wl.mistral7b_random(seed=5, requests=5, lo=40, hi=300, layers=2, heads=1, head_dim=8),
+    wl.mistral7b_random(seed=6, requests=5, lo=40, hi=300, layers=2, heads=1, head_dim=24),
+    wl.mistral7b_random(seed=7, requests=5, lo=40, hi=300, layers=2, heads=3, head_dim=64),
+    wl.mistral7b_random(seed=8, requests=5, lo=40, hi=300, layers=1, heads=6, head_dim=128),
+    wl.mistral7b_random(seed=9, requests=5, lo=40, hi=300, layers=1, heads=8, head_dim=128),
+    wl.mistral7b_random(seed=10, requests=4, lo=40, hi=200, layers=1, heads=16, head_dim=128),
+], ids=lambda w: f"{w.name}-row{w.row_bytes}")
 def test_digest_matches_oracle_and_survives_repack(w):
     import torch
     from paper_2608_13263_b200.device import DeviceProblem

@@ -202,7 +202,8 @@ __device__ __forceinline__ unsigned long long g_mix64(unsigned long long x)   //
 // A warp walks a contiguous run of (slab, output row) units; lanes take 16-byte groups of the row.
 // One (slab, row) unit of the digest: where it is and what it hashes.
 struct DigestRow {
-    int32_t src, r, tok, slab, idx;
+    const uint4 *ptr;            // first byte of the K or V row
+    int32_t r, tok, slab, idx;
 };
 
 __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
@@ -238,16 +239,16 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         if (gl == 0 && cur_r >= 0 && sum != 0) atomicAdd(&a.digest[cur_r], sum);
         sum = 0;
     };
-    auto row_ptr = [&](const DigestRow &m) {
-        const int li = m.slab < nl ? m.slab : m.slab - nl;
-        const uint8_t *pool = m.slab < nl ? a.k_pool : a.v_pool;
-        return reinterpret_cast<const uint4 *>(pool + (int64_t)(a.layer_begin + li) * a.layer_stride +
-                                               (int64_t)m.src * a.row_bytes);
+    const uint8_t *slab_base = nullptr;                        // pool + layer offset of the slab being fetched
+    auto set_slab = [&](int slab) {
+        const int li = slab < nl ? slab : slab - nl;
+        slab_base = (slab < nl ? a.k_pool : a.v_pool) + (int64_t)(a.layer_begin + li) * a.layer_stride;
     };
+    const uint32_t row_bytes32 = (uint32_t)a.row_bytes;        // rows are far below 4 GiB
     auto fetch_meta = [&](DigestRow &m, int slab, int32_t idx) {
         m.slab = slab;
         m.idx = idx;
-        m.src = a.g_src[idx];
+        m.ptr = reinterpret_cast<const uint4 *>(slab_base + (uint64_t)(uint32_t)a.g_src[idx] * row_bytes32);
         m.r = a.g_req[idx];
         m.tok = a.g_ids[idx];
     };
@@ -256,15 +257,18 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         for (int k = 0; k < 4; ++k)
             v[k] = (c0 + G * k < row_vecs) ? ld_stream(sp + c0 + G * k) : make_uint4(0, 0, 0, 0);
     };
-    auto hash4 = [&](const uint4 (&v)[4], unsigned long long key, int c0) {
+    // word offsets without multiplies in the row loop: group c = c0 + G*k has x-offset
+    // 2*c*D = 2*c0*D + k*(2*G*D) and y-offset one D further
+    const unsigned long long lane_off = 2ull * gl * D, k_step = 2ull * G * D;
+    auto hash4 = [&](const uint4 (&v)[4], unsigned long long key_c0, int c0) {   // key_c0 = key + 2*c0*D
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            const int c = c0 + G * k;
-            if (c < row_vecs) {
+            if (c0 + G * k < row_vecs) {
                 const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
                 const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
-                const unsigned long long x = w0 ^ (key + (2ull * c) * D);
-                const unsigned long long y = w1 ^ (key + (2ull * c + 1ull) * D);
+                const unsigned long long xo = key_c0 + (unsigned long long)k * k_step;
+                const unsigned long long x = w0 ^ xo;
+                const unsigned long long y = w1 ^ (xo + D);
                 sum += (x * y) ^ __umul64hi(x, y);                 // low64 ^ high64 of the 128-bit product
             }
         }
@@ -275,17 +279,17 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     int slab = (int)(u0 / n);
     int32_t idx = (int32_t)(u0 - (int64_t)slab * n);             // n < 2^31: it counts token-table entries
     const int32_t n32 = (int32_t)n;
-    auto advance = [&]() { if (++idx == n32) { idx = 0; ++slab; } };
+    auto advance = [&]() { if (++idx == n32) { idx = 0; set_slab(++slab); } };
+    set_slab(slab);
     DigestRow cur, nxt;
     fetch_meta(cur, slab, idx);
     advance();
     if (u0 + 1 < u1) { fetch_meta(nxt, slab, idx); advance(); }
     uint4 vc[4], vn[4];
-    load4(vc, row_ptr(cur), gl);
+    load4(vc, cur.ptr, gl);
     for (int64_t left = u1 - u0; left > 0; --left) {
         const bool has_next = left > 1;
-        const uint4 *np = has_next ? row_ptr(nxt) : nullptr;
-        if (has_next) load4(vn, np, gl);
+        if (has_next) load4(vn, nxt.ptr, gl);
         DigestRow nn = nxt;
         if (left > 2) { fetch_meta(nn, slab, idx); advance(); }
         if (cur.r != cur_r) {
@@ -295,13 +299,14 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         const unsigned long long i = (unsigned long long)(cur.idx - a.out_offsets[cur.r]);
         const unsigned long long key =
             g_mix64(((i * A + (unsigned long long)cur.tok) * B + (unsigned long long)cur.slab) * C);
-        hash4(vc, key, gl);
+        unsigned long long key_c0 = key + lane_off;
+        hash4(vc, key_c0, gl);
         if (row_vecs > 4 * G) {                                // rows above 64 bytes per lane: the rest, unpipelined
-            const uint4 *sp = row_ptr(cur);
             for (int c0 = gl + 4 * G; c0 < row_vecs; c0 += 4 * G) {
                 uint4 v[4];
-                load4(v, sp, c0);
-                hash4(v, key, c0);
+                key_c0 += 4ull * k_step;
+                load4(v, cur.ptr, c0);
+                hash4(v, key_c0, c0);
             }
         }
 #pragma unroll

@@ -384,6 +384,12 @@ typedef struct {                   /* all HOST pointers */
 } vtoken_host_tables;
 int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *tables, void *cuda_stream);
 
+/* The same front end with the partial planner (vtoken_plan_partial): opts as there, except that
+ * opts->protect, when given, is a HOST array of num_blocks bytes (copied to the device with the
+ * tables).  opts must not be NULL. */
+int vtoken_repack_host_partial(vtoken_ctx *ctx, const vtoken_host_tables *tables, const vtoken_partial_opts *opts,
+                               void *cuda_stream);
+
 /* Logical gather for callers that cannot allocate device memory.  (The paper has no
  * counterpart: this is a packaging variant of vtoken_gather_logical, same result.)
  *

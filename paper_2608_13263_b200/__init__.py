@@ -25,10 +25,17 @@ from .binding import (  # noqa: F401
     vtoken_read_counts,
     vtoken_repack,
     vtoken_repack_host,
+    vtoken_repack_host_partial,
+    vtoken_repack_waves,
+    vtoken_slot_cache_mark,
+    vtoken_slot_cache_update,
+    vtoken_waves_workspace_bytes,
     vtoken_scratch_bytes,
 )
 
 __all__ = ["VtokenError", "vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack",
            "vtoken_gather_logical", "vtoken_read_counts", "vtoken_repack_host", "vtoken_copy_grid",
            "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens", "vtoken_sync_new_tokens",
-           "vtoken_build_slot_mapping", "vtoken_apply_moves", "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical"]
+           "vtoken_build_slot_mapping", "vtoken_apply_moves", "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
+           "vtoken_repack_host_partial", "vtoken_repack_waves", "vtoken_waves_workspace_bytes", "vtoken_slot_cache_mark",
+           "vtoken_slot_cache_update"]

@@ -23,7 +23,7 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
-           "vtoken_slot_cache_update"]
+           "vtoken_slot_cache_update", "vtoken_repack_host_partial"]
 
 
 class VtokenError(RuntimeError):
@@ -127,6 +127,8 @@ def load():
                                                                        ctypes.c_void_p]
         lib.vtoken_read_counts.argtypes = [ctypes.c_void_p, ctypes.POINTER(Counts), ctypes.c_void_p]
         lib.vtoken_repack_host.argtypes = [ctypes.c_void_p, ctypes.POINTER(HostTables), ctypes.c_void_p]
+        lib.vtoken_repack_host_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(HostTables),
+                                                   ctypes.POINTER(PartialOpts), ctypes.c_void_p]
         lib.vtoken_strerror.argtypes = [ctypes.c_int]
         lib.vtoken_strerror.restype = ctypes.c_char_p
         lib.vtoken_last_cuda_error.argtypes = [ctypes.c_void_p]
@@ -240,6 +242,22 @@ def vtoken_repack_host(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, 
                    _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks), _ptr(req_status),
                    ctypes.addressof(c))
     _check(load().vtoken_repack_host(ctx, ctypes.byref(h), _stream(stream)), "vtoken_repack_host", ctx)
+    return c.as_dict()
+
+
+def vtoken_repack_host_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
+                               num_free, new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status,
+                               select=None, thr_num=0, thr_den=0, protect=None, util=(0, 0), max_source_blocks=0,
+                               theta=(0, 0), stream=None) -> dict:
+    """vtoken_repack_host with the partial planner; ``protect`` is a HOST array of num_blocks bytes."""
+    c = Counts()
+    h = HostTables(num_requests, _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
+                   _ptr(select), thr_num, thr_den, _ptr(free_blocks), num_free, _ptr(new_bt_offsets),
+                   _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks), _ptr(req_status),
+                   ctypes.addressof(c))
+    po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1])
+    _check(load().vtoken_repack_host_partial(ctx, ctypes.byref(h), ctypes.byref(po), _stream(stream)),
+           "vtoken_repack_host_partial", ctx)
     return c.as_dict()
 
 

@@ -29,7 +29,8 @@ void free_all(vtoken_ctx *ctx)
                     ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
                     ctx->stage.select, ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
-                    ctx->stage.new_tt_slots, ctx->stage.freed_blocks, ctx->stage.req_status, ctx->stage.counts};
+                    ctx->stage.new_tt_slots, ctx->stage.freed_blocks, ctx->stage.req_status, ctx->stage.counts,
+                    ctx->stage.protect};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (ctx->stage.h_scalars) cudaFreeHost(ctx->stage.h_scalars);
@@ -186,9 +187,11 @@ int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stre
     return VTOKEN_OK;
 }
 
-int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_stream)
+static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoken_partial_opts *opts,
+                       void *cuda_stream)
 {
     if (!ctx || !h) return VTOKEN_EINVAL;
+    if (opts && opts->max_source_blocks < 0) return VTOKEN_EINVAL;
     if (!h->bt_offsets || !h->bt_blocks || !h->tt_offsets || !h->tt_slots || !h->keep || !h->free_blocks ||
         !h->new_bt_offsets || !h->new_bt_blocks || !h->new_tt_slots || !h->freed_blocks || !h->req_status ||
         !h->counts)
@@ -203,6 +206,10 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     if (rc != VTOKEN_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     auto &s = ctx->stage;
+    if (opts && opts->protect && !s.protect) {      // device copy of the protect mask, on first use
+        rc = dev_alloc(ctx, &s.protect, ctx->cfg.num_blocks);
+        if (rc != VTOKEN_OK) return rc;
+    }
 #define H2D(dst, src, n) VTK_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(n), cudaMemcpyHostToDevice, st))
 #define D2H(dst, src, n) VTK_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(n), cudaMemcpyDeviceToHost, st))
     s.h_scalars[0] = h->num_requests;               // pinned: the copy below is truly asynchronous
@@ -215,6 +222,7 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     if (T) H2D(s.keep, h->keep, T);
     if (h->select && R) H2D(s.select, h->select, R);
     if (h->num_free) H2D(s.free_blocks, h->free_blocks, h->num_free * sizeof(int32_t));
+    if (opts && opts->protect) H2D(s.protect, opts->protect, ctx->cfg.num_blocks);
 
     vtoken_plan_in in;
     in.num_requests = s.num_requests;
@@ -235,7 +243,13 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     out.freed_blocks = s.freed_blocks;
     out.req_status = s.req_status;
     out.counts = s.counts;
-    rc = vtk_launch_plan(ctx, &in, &out, st);
+    if (opts) {
+        vtoken_partial_opts dopts = *opts;
+        dopts.protect = opts->protect ? s.protect : nullptr;
+        rc = vtoken_plan_partial(ctx, &in, &dopts, &out, st);
+    } else {
+        rc = vtk_launch_plan(ctx, &in, &out, st);
+    }
     if (rc != VTOKEN_OK) return rc;
     ctx->has_plan = true;
     // every table output is final once the plan has run: copy them back on a second stream
@@ -261,6 +275,18 @@ int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, void *cuda_
     VTK_CUDA(ctx, cudaStreamSynchronize(st));
     *h->counts = *s.h_counts;
     return VTOKEN_OK;
+}
+
+int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *tables, void *cuda_stream)
+{
+    return repack_host(ctx, tables, nullptr, cuda_stream);
+}
+
+int vtoken_repack_host_partial(vtoken_ctx *ctx, const vtoken_host_tables *tables, const vtoken_partial_opts *opts,
+                               void *cuda_stream)
+{
+    if (!opts) return VTOKEN_EINVAL;
+    return repack_host(ctx, tables, opts, cuda_stream);
 }
 
 const char *vtoken_strerror(int code)

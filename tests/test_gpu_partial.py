@@ -182,3 +182,51 @@ def test_shared_prefix_workload(degree):
     assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
     assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
     prob.close()
+
+
+@pytest.mark.parametrize("opts", [dict(util=(1, 1)), dict(util=(1, 1), theta=(1, 4), max_source_blocks=9),
+                                  dict(protect="prefix", util=(3, 4))], ids=["util", "bound", "protect"])
+def test_repack_host_partial_entry_point(opts):
+    """Host tables in, host tables out, partial planner; the protect mask is a host array."""
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    w = wl.steady_state(seed=5, requests=14, lo=100, hi=900, layers=2, heads=2, head_dim=64)
+    opts = dict(opts)
+    if opts.get("protect") == "prefix":
+        protect = np.zeros(w.num_blocks, np.uint8)
+        for r in range(w.num_requests):
+            protect[w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]][:2]] = 1
+        opts["protect"] = protect
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    R, T, NBT = w.num_requests, w.num_tokens, len(w.bt_blocks)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_in = dict(bt_offsets=pin(w.bt_offsets), bt_blocks=pin(w.bt_blocks), tt_offsets=pin(w.tt_offsets),
+                tt_slots=pin(w.tt_slots), keep=pin(w.keep), free_blocks=pin(w.free_blocks))
+    if w.select is not None:
+        h_in["select"] = pin(w.select)
+    h_out = dict(new_bt_offsets=torch.zeros(R + 1, dtype=torch.int32).pin_memory(),
+                 new_bt_blocks=torch.zeros(NBT, dtype=torch.int32).pin_memory(),
+                 new_tt_slots=torch.zeros(T, dtype=torch.int32).pin_memory(),
+                 freed_blocks=torch.zeros(NBT, dtype=torch.int32).pin_memory(),
+                 req_status=torch.zeros(R, dtype=torch.int32).pin_memory())
+    s = torch.cuda.Stream()
+    for _ in range(2):                                   # the second call reuses the staging buffers
+        prob.fill_pools()
+        torch.cuda.synchronize()
+        c = vt.vtoken_repack_host_partial(prob.ctx, num_requests=R, num_free=len(w.free_blocks), thr_num=w.thr_num,
+                                          thr_den=w.thr_den, stream=s, **opts, **h_in, **h_out)
+    p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                         w.free_blocks, w.select, w.thr_num, w.thr_den, **opts)
+    assert c["num_moves"] == p.num_moves > 0 and c["error_flags"] == 0 and c["num_freed"] == p.num_freed
+    assert np.array_equal(h_out["new_tt_slots"].numpy(), p.new_tt_slots)
+    assert np.array_equal(h_out["new_bt_offsets"].numpy(), p.new_bt_offsets)
+    assert np.array_equal(h_out["new_bt_blocks"].numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
+    assert np.array_equal(h_out["freed_blocks"].numpy()[:p.num_freed], p.freed_blocks)
+    assert np.array_equal(h_out["req_status"].numpy(), p.req_status)
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    with pytest.raises(vt.VtokenError):
+        vt._check(vt.load().vtoken_repack_host_partial(prob.ctx, None, None, None), "null arguments")
+    prob.close()

@@ -46,3 +46,32 @@ def test_strerror_and_argument_errors_without_gpu():
     assert lib.vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)) == binding.EINVAL
     cfg = binding.Config(1, 4, 16, 1, 8, 2, 257, 512, 0, 1, 16, 4, 4, 0, 0)   # misaligned pool
     assert lib.vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)) == binding.EINVAL
+
+
+def test_header_is_plain_c_and_ctypes_layouts_match(tmp_path):
+    """include/vtoken.h compiles as C99 on its own, and every struct the binding mirrors with
+    ctypes has the size and field offsets the C compiler gives it."""
+    import subprocess
+    structs = {"vtoken_config": binding.Config, "vtoken_plan_in": binding.PlanIn, "vtoken_counts": binding.Counts,
+               "vtoken_plan_out": binding.PlanOut, "vtoken_partial_opts": binding.PartialOpts,
+               "vtoken_host_tables": binding.HostTables, "vtoken_waves_out": binding.WavesOut}
+    lines = ['#include <stddef.h>', '#include <stdio.h>', '#include "vtoken.h"', 'int main(void) {']
+    for cname, cls in structs.items():
+        lines.append(f'printf("{cname} %zu", sizeof({cname}));')
+        for fname, _ in cls._fields_:
+            lines.append(f'printf(" %zu", offsetof({cname}, {fname}));')
+        lines.append('printf("\\n");')
+    lines += ['return 0; }']
+    src = tmp_path / "layout.c"
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.check_call(["gcc", "-std=c99", "-pedantic", "-Wall", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           "-o", str(exe), str(src)])
+    out = subprocess.check_output([str(exe)], text=True).strip().splitlines()
+    assert len(out) == len(structs)
+    for line, (cname, cls) in zip(out, structs.items()):
+        parts = line.split()
+        assert parts[0] == cname
+        assert int(parts[1]) == ctypes.sizeof(cls), cname
+        offsets = [getattr(cls, f).offset for f, _ in cls._fields_]
+        assert [int(x) for x in parts[2:]] == offsets, cname

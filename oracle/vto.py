@@ -181,6 +181,20 @@ def validate(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bloc
     return bad.value
 
 
+def check_tables(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, free_blocks, protect=None) -> int:
+    """Bit set of every violated input precondition (0 = valid); see vto_check_tables."""
+    bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
+    tt_offsets, tt_slots, free_blocks, protect = _i32(tt_offsets), _i32(tt_slots), _i32(free_blocks), _u8(protect)
+    bits = ctypes.c_uint32(0)
+    rc = lib().vto_check_tables(ctypes.c_int32(len(tt_offsets) - 1), ctypes.c_int32(S), ctypes.c_int32(NB),
+                                _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
+                                _p(tt_slots, np.int32), _p(free_blocks, np.int32), ctypes.c_int32(len(free_blocks)),
+                                _p(protect, np.uint8), ctypes.byref(bits))
+    if rc != 0:
+        raise ValueError(f"vto_check_tables failed: {rc}")
+    return bits.value
+
+
 def check_semantics(S, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
                     new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, num_free_consumed,
                     req_status, select=None, thr_num=0, thr_den=0, num_free=None) -> int:

@@ -204,6 +204,66 @@ int vto_validate(int32_t R, int32_t S, int32_t NB,
     return bad ? VTO_EPRECOND : VTO_OK;
 }
 
+int vto_check_tables(int32_t R, int32_t S, int32_t NB,
+                     const int32_t *bt_offsets, const int32_t *bt_blocks,
+                     const int32_t *tt_offsets, const int32_t *tt_slots,
+                     const int32_t *free_blocks, int32_t num_free, const uint8_t *protect, uint32_t *bits)
+{
+    if (R < 0 || S < 1 || NB < 0 || num_free < 0 || !bt_offsets || !tt_offsets || !bits) return VTO_EINVAL;
+    uint32_t f = 0;
+    const size_t nb = (size_t)(NB > 0 ? NB : 1);
+    int32_t *in_tables = (int32_t *)calloc(nb, sizeof(int32_t));     /* block-table entries holding block b */
+    int32_t *in_free = (int32_t *)calloc(nb, sizeof(int32_t));       /* free-list entries naming block b */
+    int32_t *refs = (int32_t *)calloc((size_t)NB * (size_t)S + 1, sizeof(int32_t));   /* entries naming slot s */
+    int32_t *holders = (int32_t *)calloc(nb, sizeof(int32_t));       /* distinct requests holding block b */
+    int32_t *last_holder = (int32_t *)calloc(nb, sizeof(int32_t));   /* the last of them */
+    if (!in_tables || !in_free || !refs || !holders || !last_holder) {
+        free(in_tables); free(in_free); free(refs); free(holders); free(last_holder);
+        return VTO_EINVAL;
+    }
+
+    for (int32_t r = 0; r < R; ++r)
+        if (bt_offsets[r + 1] < bt_offsets[r] || tt_offsets[r + 1] < tt_offsets[r]) f |= 1u;
+    if (f) goto done;                                      /* the ranges below would be meaningless */
+
+    for (int32_t r = 0; r < R; ++r) {
+        for (int32_t j = bt_offsets[r]; j < bt_offsets[r + 1]; ++j) {
+            const int32_t b = bt_blocks[j];
+            if (b < 0 || b >= NB) { f |= 2u; continue; }
+            ++in_tables[b];
+            /* number of distinct requests holding b (a request's entries are consecutive) */
+            if (holders[b] == 0 || last_holder[b] != r) ++holders[b];
+            last_holder[b] = r;
+        }
+    }
+    for (int32_t b = 0; b < NB; ++b)
+        if (in_tables[b] > 1 && !(protect && protect[b])) f |= 4u;
+    for (int32_t j = 0; j < num_free; ++j) {
+        const int32_t b = free_blocks[j];
+        if (b < 0 || b >= NB) f |= 8u;
+        else ++in_free[b];
+    }
+    for (int32_t b = 0; b < NB; ++b)
+        if (in_free[b] > 1 || (in_free[b] == 1 && in_tables[b] > 0)) f |= 16u;
+    for (int32_t r = 0; r < R; ++r) {
+        for (int64_t t = tt_offsets[r]; t < tt_offsets[r + 1]; ++t) {
+            const int32_t s = tt_slots[t];
+            if (s < 0) continue;
+            if ((int64_t)s >= (int64_t)NB * S) { f |= 32u; continue; }
+            /* whose block is it?  a block held by several requests (shared prefix) is outside this check */
+            const int32_t b = s / S;
+            if (holders[b] == 0 || (holders[b] == 1 && last_holder[b] != r)) f |= 64u;
+            ++refs[s];
+        }
+    }
+    for (int64_t s = 0; s < (int64_t)NB * S; ++s)
+        if (refs[s] > 1 && !(protect && protect[s / S])) f |= 128u;   /* sharers all map a shared block's slots */
+done:
+    free(in_tables); free(in_free); free(refs); free(holders); free(last_holder);
+    *bits = f;
+    return VTO_OK;
+}
+
 static int cmp_i32(const void *a, const void *b)
 {
     const int32_t x = *(const int32_t *)a, y = *(const int32_t *)b;

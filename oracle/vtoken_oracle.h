@@ -89,6 +89,26 @@ int vto_validate(int32_t R, int32_t S, int32_t NB,
                  const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
                  const int32_t *free_blocks, int32_t num_free, int32_t *first_bad);
 
+/* The same preconditions, every violated one reported as a bit (evaluation order does not
+ * matter: each bit is defined by counting, so a parallel checker gives the same answer):
+ *   1   CSR offsets not monotone (block tables or token tables)
+ *   2   a block-table id outside [0, NB)
+ *   4   a block id held by more than one block-table entry
+ *   8   a free-list id outside [0, NB)
+ *   16  a free-list id listed twice, or also held by a block table
+ *   32  a slot >= NB*S
+ *   64  a slot (>= 0, in range) whose block is held by no block table, or by exactly one request
+ *       that is not the slot's request (blocks held by several requests are outside this check)
+ *   128 a slot (>= 0, in range) referenced by more than one token-table entry (I2)
+ * Entries with slot < 0 are ignored; keep is not consulted (an evicted token still owns its slot
+ * until a repack).  protect (may be NULL): blocks marked there may sit in several tables
+ * (shared prefix) and their slots are mapped by every sharer, so bits 4 and 128 are not raised
+ * for them. */
+int vto_check_tables(int32_t R, int32_t S, int32_t NB,
+                     const int32_t *bt_offsets, const int32_t *bt_blocks,
+                     const int32_t *tt_offsets, const int32_t *tt_slots,
+                     const int32_t *free_blocks, int32_t num_free, const uint8_t *protect, uint32_t *bits);
+
 /* Order-free check of a plan result against the inputs: statuses follow the admission rule,
  * admitted requests got ceil(n/S) distinct blocks of the consumed free prefix and their live
  * tokens fill those blocks completely in logical order, the reclaimed set equals the admitted

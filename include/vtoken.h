@@ -424,6 +424,25 @@ int vtoken_gather_logical_noalloc(const void *k_pool, const void *v_pool, int32_
                                   int32_t layer_end, void *out_k, void *out_v, int64_t out_capacity_tokens,
                                   int32_t *out_offsets, uint32_t *error_flags, void *cuda_stream);
 
+/* Input-precondition checker (a debugging aid: the fast path assumes these and does not check
+ * them; invariant I2 -- unique mapping -- is bit 128).  Writes to out_bits (DEVICE uint32) the
+ * set of violated preconditions of the planner inputs in `in` (keep, select and the threshold
+ * are not consulted: an evicted token still owns its slot until a repack):
+ *   1   CSR offsets not monotone (only this bit is reported then)
+ *   2   a block-table id outside [0, num_blocks)
+ *   4   a block id held by more than one block-table entry
+ *   8   a free-list id outside [0, num_blocks)
+ *   16  a free-list id listed twice, or also held by a block table
+ *   32  a slot >= num_blocks * block_size
+ *   64  a slot whose block is held by no block table, or by exactly one request that is not the
+ *       slot's request (blocks held by several requests are outside this check)
+ *   128 a slot referenced by more than one token-table entry
+ * protect (DEVICE [num_blocks] or NULL): blocks marked there may sit in several tables and their
+ * slots may be mapped by every sharer (shared prefix): bits 4 and 128 are not raised for them.
+ * Uses the context's planner scratch (do not overlap with a plan in flight).  Capturable. */
+int vtoken_check_tables(vtoken_ctx *ctx, const vtoken_plan_in *in, const uint8_t *protect, uint32_t *out_bits,
+                        void *cuda_stream);
+
 /* Diagnostics. */
 const char *vtoken_strerror(int code);
 int vtoken_last_cuda_error(const vtoken_ctx *ctx);       /* cudaError_t of the last VTOKEN_ECUDA */

@@ -11,6 +11,7 @@ from .binding import (  # noqa: F401
     VtokenError,
     vtoken_apply_moves,
     vtoken_block_liveness,
+    vtoken_check_tables,
     vtoken_digest_logical,
     vtoken_plan_partial,
     vtoken_build_slot_mapping,
@@ -38,4 +39,4 @@ __all__ = ["VtokenError", "vtoken_create", "vtoken_destroy", "vtoken_plan", "vto
            "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens", "vtoken_sync_new_tokens",
            "vtoken_build_slot_mapping", "vtoken_apply_moves", "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_repack_host_partial", "vtoken_repack_waves", "vtoken_waves_workspace_bytes", "vtoken_slot_cache_mark",
-           "vtoken_slot_cache_update"]
+           "vtoken_slot_cache_update", "vtoken_check_tables"]

@@ -23,7 +23,7 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
-           "vtoken_slot_cache_update", "vtoken_repack_host_partial"]
+           "vtoken_slot_cache_update", "vtoken_repack_host_partial", "vtoken_check_tables"]
 
 
 class VtokenError(RuntimeError):
@@ -129,6 +129,8 @@ def load():
         lib.vtoken_repack_host.argtypes = [ctypes.c_void_p, ctypes.POINTER(HostTables), ctypes.c_void_p]
         lib.vtoken_repack_host_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(HostTables),
                                                    ctypes.POINTER(PartialOpts), ctypes.c_void_p]
+        lib.vtoken_check_tables.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.c_void_p, ctypes.c_void_p,
+                                            ctypes.c_void_p]
         lib.vtoken_strerror.argtypes = [ctypes.c_int]
         lib.vtoken_strerror.restype = ctypes.c_char_p
         lib.vtoken_last_cuda_error.argtypes = [ctypes.c_void_p]
@@ -259,6 +261,15 @@ def vtoken_repack_host_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_o
     _check(load().vtoken_repack_host_partial(ctx, ctypes.byref(h), ctypes.byref(po), _stream(stream)),
            "vtoken_repack_host_partial", ctx)
     return c.as_dict()
+
+
+def vtoken_check_tables(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, free_blocks, num_free,
+                        out_bits, protect=None, stream=None) -> None:
+    """Bit set of violated input preconditions into ``out_bits`` (device uint32); 0 = valid."""
+    pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), None,
+                 None, 0, 0, _ptr(free_blocks), _ptr(num_free))
+    _check(load().vtoken_check_tables(ctx, ctypes.byref(pin), _ptr(protect), _ptr(out_bits), _stream(stream)),
+           "vtoken_check_tables", ctx)
 
 
 def vtoken_copy_grid(ctx) -> dict:

@@ -21,7 +21,7 @@ LIB = os.path.join(PKG, "libvtoken.so")
 HARNESS_LIB = os.path.join(PKG, "libvtoken_harness.so")
 
 LIB_SOURCES = ["api.cu", "plan.cu", "copy.cu", "gather.cu", "gather_static.cu", "runtime.cu", "plan_partial.cu",
-               "waves.cu", "slot_cache.cu"]
+               "waves.cu", "slot_cache.cu", "check.cu"]
 HARNESS_SOURCES = ["harness.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -25,7 +25,7 @@ void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
-                    ctx->n_b, ctx->blk_src,
+                    ctx->n_b, ctx->blk_src, ctx->slot_bits,
                     ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
                     ctx->stage.select, ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
@@ -130,6 +130,7 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->req_nsrc, cfg->max_requests);
     A(&ctx->n_b, cfg->num_blocks);
     A(&ctx->blk_src, cfg->num_blocks);
+    A(&ctx->slot_bits, (slots + 31) / 32);
     if (rc == VTOKEN_OK && cudaMemset(ctx->counts, 0, sizeof(vtoken_counts)) != cudaSuccess) rc = VTOKEN_ECUDA;
     if (rc == VTOKEN_OK) rc = vtk_configure_copy(ctx);
     if (rc != VTOKEN_OK) { free_all(ctx); delete ctx; return rc; }

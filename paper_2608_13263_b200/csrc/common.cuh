@@ -36,6 +36,7 @@ struct vtoken_ctx {
     int32_t *req_nsrc;         // [max_requests] live tokens in its source blocks
     int32_t *n_b;              // [num_blocks] live tokens per physical block
     uint8_t *blk_src;          // [num_blocks] 1 = the block is a source of its request
+    uint32_t *slot_bits;       // [ceil(num_blocks * S / 32)] one bit per slot (vtoken_check_tables)
 
     // gather_logical scratch (DEVICE)
     int32_t *g_src;            // [max_tokens] source slot of each output row

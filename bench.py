@@ -649,7 +649,7 @@ def run_runtime(args, prob, w, side, dev):
     def commit(st):
         vt.vtoken_apply_moves(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
                               tt_slots=tt_commit, keep=keep_commit, phys_len=phys, new_tt_slots=prob.new_tt_slots,
-                              req_status=prob.req_status, stream=st)
+                              req_status=prob.req_status, new_bt_offsets=prob.new_bt_offsets, stream=st)
 
     # the two K/V-reading checkers: relocation digest over every layer (read only), logical gather of
     # a layer range that fits in 2 GiB of output per pool (read + write)

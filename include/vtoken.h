@@ -330,13 +330,17 @@ int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_requests, cons
                               int32_t *out_offsets, void *cuda_stream);
 
 /* apply_moves (Sec. 3.2; invariant I2): commit of a plan after its repack event.  Every entry takes
- * its slot from new_tt_slots (the source entry is cleared by the same write), keep becomes
- * (slot >= 0), and for requests with status VTOKEN_REPACKED phys_len[r] becomes the number of
- * entries that still own a slot (new tokens append behind the packed survivors).  phys_len may be
- * NULL.  The block tables are the caller's: it adopts new_bt_* and returns freed blocks itself. */
+ * its slot from new_tt_slots (the source entry is cleared by the same write) and keep becomes
+ * (slot >= 0).  For requests with status VTOKEN_REPACKED the append position moves behind the
+ * tokens the repack moved: the request's block list is now the blocks that stayed followed by the
+ * destination blocks, so  phys_len[r] = (blocks - ceil(moved / S)) * S + moved  with blocks from
+ * new_bt_offsets and moved = entries whose slot changed.  new_bt_offsets may be NULL: phys_len[r]
+ * is then the number of entries that own a slot -- the same value after vtoken_plan (nothing
+ * stays), wrong after a partial plan.  phys_len may be NULL.  The block tables are the caller's:
+ * it adopts new_bt_* and returns freed blocks itself. */
 int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                        int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
-                       const int32_t *req_status, void *cuda_stream);
+                       const int32_t *req_status, const int32_t *new_bt_offsets, void *cuda_stream);
 
 /* Cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4): per request the slots (and
  * ids) of its active tokens in token-id order, kept on the device between decode steps and

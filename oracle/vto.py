@@ -280,13 +280,17 @@ def build_slot_mapping(tt_offsets, tt_slots, keep=None, select=None):
     return slots[:n].copy(), ids[:n].copy(), off
 
 
-def apply_moves(tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, phys_len, new_tt_slots, req_status) -> None:
-    """Commit of a repack, in place on tt_slots, keep and phys_len (phys_len may be None)."""
+def apply_moves(tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, phys_len, new_tt_slots, req_status, S=1,
+                new_bt_offsets=None) -> None:
+    """Commit of a repack, in place on tt_slots, keep and phys_len (phys_len may be None).  With
+    ``S`` and ``new_bt_offsets`` the append position also holds after partial plans."""
     tt_offsets, new_tt_slots, req_status = _i32(tt_offsets), _i32(new_tt_slots), _i32(req_status)
+    nbo = None if new_bt_offsets is None else _i32(new_bt_offsets)
     assert tt_slots.dtype == np.int32 and keep.dtype == np.uint8
-    rc = lib().vto_apply_moves(ctypes.c_int32(len(tt_offsets) - 1), _p(tt_offsets, np.int32), _p(tt_slots, np.int32),
-                               _p(keep, np.uint8), None if phys_len is None else _p(phys_len, np.int32),
-                               _p(new_tt_slots, np.int32), _p(req_status, np.int32))
+    rc = lib().vto_apply_moves(ctypes.c_int32(len(tt_offsets) - 1), ctypes.c_int32(S), _p(tt_offsets, np.int32),
+                               _p(tt_slots, np.int32), _p(keep, np.uint8),
+                               None if phys_len is None else _p(phys_len, np.int32), _p(new_tt_slots, np.int32),
+                               _p(req_status, np.int32), None if nbo is None else _p(nbo, np.int32))
     if rc != 0:
         raise ValueError(f"vto_apply_moves failed: {rc}")
 

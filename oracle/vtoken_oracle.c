@@ -426,18 +426,29 @@ int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32
     return n;
 }
 
-int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
-                    int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status)
+int vto_apply_moves(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                    int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status,
+                    const int32_t *new_bt_offsets)
 {
-    if (R < 0 || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTO_EINVAL;
+    if (R < 0 || S < 1 || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTO_EINVAL;
     for (int32_t r = 0; r < R; ++r) {
-        int32_t with_slot = 0;
+        int32_t with_slot = 0, moved = 0;
         for (int64_t t = tt_offsets[r]; t < tt_offsets[r + 1]; ++t) {
+            moved += new_tt_slots[t] >= 0 && new_tt_slots[t] != tt_slots[t];   /* destinations are never sources */
             tt_slots[t] = new_tt_slots[t];              /* source entry cleared, destination written (I2) */
             keep[t] = new_tt_slots[t] >= 0 ? 1 : 0;
             with_slot += new_tt_slots[t] >= 0;
         }
-        if (phys_len && req_status && req_status[r] == VTO_REPACKED) phys_len[r] = with_slot;
+        if (phys_len && req_status && req_status[r] == VTO_REPACKED) {
+            if (new_bt_offsets) {
+                /* new block list = blocks that stayed, then the destination blocks, which the moved
+                 * tokens fill densely: the next token lands right behind them */
+                const int32_t blocks = new_bt_offsets[r + 1] - new_bt_offsets[r];
+                phys_len[r] = (blocks - ceil_div(moved, S)) * S + moved;
+            } else {
+                phys_len[r] = with_slot;                /* whole-request plans: nothing stayed */
+            }
+        }
     }
     return VTO_OK;
 }

@@ -159,10 +159,14 @@ int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32
                                int32_t *out_token_ids, int32_t *out_offsets, int64_t capacity);
 
 /* apply_moves / commit of a repack: every entry takes its new slot, liveness follows it (an entry
- * without a slot is dead), and a repacked request appends after its n live tokens from now on:
- * phys_len[r] = number of entries with a slot, for requests with status VTO_REPACKED. */
-int vto_apply_moves(int32_t R, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
-                    int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status);
+ * without a slot is dead), and a repacked request appends behind the tokens the repack moved: its
+ * block list is now the blocks that stayed followed by the destination blocks, so for requests
+ * with status VTO_REPACKED  phys_len[r] = (blocks - ceil(moved / S)) * S + moved, with blocks from
+ * new_bt_offsets and moved = entries whose slot changed.  new_bt_offsets == NULL: phys_len[r] =
+ * number of entries with a slot (the same value after a whole-request plan, where nothing stays). */
+int vto_apply_moves(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
+                    int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status,
+                    const int32_t *new_bt_offsets);
 
 /* ---- cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4) -------------------------
  * The worker keeps, per request, the slots of its active tokens in token-id order -- the array a

@@ -145,7 +145,7 @@ def load():
         lib.vtoken_evict_tokens.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 7
         lib.vtoken_sync_new_tokens.argtypes = [ctypes.c_void_p] * 11
         lib.vtoken_build_slot_mapping.argtypes = [ctypes.c_void_p] * 8 + [ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
-        lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 9
+        lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 10
         lib.vtoken_block_liveness.argtypes = [ctypes.c_void_p] * 11
         lib.vtoken_digest_logical.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 3
         lib.vtoken_plan_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
@@ -324,9 +324,10 @@ def vtoken_build_slot_mapping(ctx, *, num_requests, tt_offsets, tt_slots, keep, 
 
 
 def vtoken_apply_moves(ctx, *, num_requests, tt_offsets, tt_slots, keep, phys_len, new_tt_slots, req_status,
-                       stream=None) -> None:
+                       new_bt_offsets=None, stream=None) -> None:
     _check(load().vtoken_apply_moves(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
-                                     _ptr(phys_len), _ptr(new_tt_slots), _ptr(req_status), _stream(stream)),
+                                     _ptr(phys_len), _ptr(new_tt_slots), _ptr(req_status), _ptr(new_bt_offsets),
+                                     _stream(stream)),
            "vtoken_apply_moves", ctx)
 
 

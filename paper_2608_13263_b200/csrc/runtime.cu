@@ -75,31 +75,45 @@ __global__ void __launch_bounds__(RT_NT) sync_kernel(const int32_t *num_requests
 }
 
 // apply_moves: commit of a repack.  Entries take their new slot, liveness follows the slot, a
-// repacked request appends behind its surviving tokens from now on.
+// repacked request appends behind the tokens the repack moved: its block list is now the blocks
+// that stayed followed by the destination blocks, which the moved tokens fill densely.
 __global__ void __launch_bounds__(RT_NT) apply_moves_kernel(const int32_t *num_requests, int32_t max_requests,
-                                                            const int32_t *tt_offsets, int32_t *tt_slots,
+                                                            int32_t S, const int32_t *tt_offsets, int32_t *tt_slots,
                                                             uint8_t *keep, int32_t *phys_len,
-                                                            const int32_t *new_tt_slots, const int32_t *req_status)
+                                                            const int32_t *new_tt_slots, const int32_t *req_status,
+                                                            const int32_t *new_bt_offsets)
 {
     const int r = blockIdx.x;
     if (r >= rt_requests(num_requests, max_requests)) return;
     const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
-    int n = 0;
+    int n = 0, moved = 0;                          // entries with a slot; entries whose slot changed
     for (int64_t t = t0 + threadIdx.x; t < t1; t += RT_NT) {
         const int32_t s = new_tt_slots[t];
+        moved += s >= 0 && s != tt_slots[t];       // destinations are never sources
         tt_slots[t] = s;
         keep[t] = s >= 0 ? 1 : 0;
         n += s >= 0;
     }
-    __shared__ int warp_n[RT_NT / 32];
+    __shared__ int warp_n[RT_NT / 32], warp_m[RT_NT / 32];
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
-    if (vtk_lane() == 0) warp_n[threadIdx.x >> 5] = n;
+    for (int d = 16; d > 0; d >>= 1) {
+        n += __shfl_down_sync(0xffffffffu, n, d);
+        moved += __shfl_down_sync(0xffffffffu, moved, d);
+    }
+    if (vtk_lane() == 0) {
+        warp_n[threadIdx.x >> 5] = n;
+        warp_m[threadIdx.x >> 5] = moved;
+    }
     __syncthreads();
     if (threadIdx.x == 0 && phys_len != nullptr && req_status != nullptr && req_status[r] == VTOKEN_REPACKED) {
-        int s = 0;
-        for (int w = 0; w < RT_NT / 32; ++w) s += warp_n[w];
-        phys_len[r] = s;
+        int sn = 0, sm = 0;
+        for (int w = 0; w < RT_NT / 32; ++w) { sn += warp_n[w]; sm += warp_m[w]; }
+        if (new_bt_offsets != nullptr) {
+            const int blocks = new_bt_offsets[r + 1] - new_bt_offsets[r];
+            phys_len[r] = (blocks - (sm + S - 1) / S) * S + sm;
+        } else {
+            phys_len[r] = sn;                      // whole-request plans: nothing stayed
+        }
     }
 }
 
@@ -141,12 +155,13 @@ int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const i
 
 int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                        int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
-                       const int32_t *req_status, void *cuda_stream)
+                       const int32_t *req_status, const int32_t *new_bt_offsets, void *cuda_stream)
 {
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTOKEN_EINVAL;
     if (phys_len && !req_status) return VTOKEN_EINVAL;
     apply_moves_kernel<<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
-        num_requests, ctx->cfg.max_requests, tt_offsets, tt_slots, keep, phys_len, new_tt_slots, req_status);
+        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, phys_len, new_tt_slots,
+        req_status, new_bt_offsets);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -110,22 +110,30 @@ class Repack:
     thr: tuple = (0, 0)
     num_free_limit: int = -1      # >= 0: pretend the free list is this short
     last_plan: object = None
+    partial: dict = None          # options of the partial planner; None = whole-request plan
 
     def run_on_oracle(self, st, pool, truth):
         free = np.asarray(st.free, np.int32)
         nf = len(free) if self.num_free_limit < 0 else min(len(free), self.num_free_limit)
-        p = vto.plan(st.S, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep, free,
-                     thr_num=self.thr[0], thr_den=self.thr[1], num_free=nf)
+        if self.partial is None:
+            p = vto.plan(st.S, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep, free,
+                         thr_num=self.thr[0], thr_den=self.thr[1], num_free=nf)
+        else:
+            p = vto.plan_partial(st.S, st.num_blocks, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots,
+                                 st.keep, free, thr_num=self.thr[0], thr_den=self.thr[1], num_free=nf,
+                                 **self.partial)
         self.last_plan = p
         if pool is not None:
             vto.apply_moves_slab(pool, p.move_src, p.move_dst)
-        vto.apply_moves(st.tt_offsets, st.tt_slots, st.keep, st.phys_len, p.new_tt_slots, p.req_status)
+        vto.apply_moves(st.tt_offsets, st.tt_slots, st.keep, st.phys_len, p.new_tt_slots, p.req_status, S=st.S,
+                        new_bt_offsets=p.new_bt_offsets)
         st.set_block_lists([p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]] for r in range(st.R)])
         st.free = free[p.num_free_consumed:].tolist() + p.freed_blocks.tolist()
 
 
-def random_serving_steps(rng, st, steps):
-    """A seeded sequence of appends, evictions and repacks sized for ``st``."""
+def random_serving_steps(rng, st, steps, partial_options=()):
+    """A seeded sequence of appends, evictions and repacks sized for ``st``.  ``partial_options``:
+    option dicts of the partial planner to draw repacks from (empty: whole-request plans only)."""
     R = st.R
     cap = np.diff(st.tt_offsets)
     length = np.zeros(R, np.int64)
@@ -144,4 +152,7 @@ def random_serving_steps(rng, st, steps):
         else:
             thr = [(0, 0), (1, 2), (3, 4)][int(rng.integers(0, 3))]
             limit = -1 if rng.random() < 0.7 else int(rng.integers(0, 6))
-            yield Repack(thr, limit)
+            partial = None
+            if len(partial_options):
+                partial = partial_options[int(rng.integers(0, len(partial_options)))]
+            yield Repack(thr, limit, partial=partial)

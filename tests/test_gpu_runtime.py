@@ -105,26 +105,31 @@ class DeviceServing:
                                num_requests=self.num_requests, tt_offsets=self.tt_offsets, tt_len=self.tt_len,
                                keep=self.keep)
 
-    def repack(self, st, free, nf, thr):
+    def repack(self, st, free, nf, thr, partial=None):
         t = self.torch
         self.upload_blocks(st)
         self.free_blocks[:len(free)].copy_(t.from_numpy(np.asarray(free, np.int32)))
         self.num_free.fill_(nf)
         side = t.cuda.Stream()
         side.wait_stream(t.cuda.current_stream())
-        vt.vtoken_plan(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets, bt_blocks=self.bt_blocks,
-                       tt_offsets=self.tt_offsets, tt_slots=self.tt_slots, keep=self.keep,
-                       free_blocks=self.free_blocks, num_free=self.num_free, new_bt_offsets=self.new_bt_offsets,
-                       new_bt_blocks=self.new_bt_blocks, new_tt_slots=self.new_tt_slots,
-                       freed_blocks=self.freed_blocks, req_status=self.req_status, counts=self.counts,
-                       thr_num=thr[0], thr_den=thr[1], stream=side)
+        args = dict(num_requests=self.num_requests, bt_offsets=self.bt_offsets, bt_blocks=self.bt_blocks,
+                    tt_offsets=self.tt_offsets, tt_slots=self.tt_slots, keep=self.keep,
+                    free_blocks=self.free_blocks, num_free=self.num_free, new_bt_offsets=self.new_bt_offsets,
+                    new_bt_blocks=self.new_bt_blocks, new_tt_slots=self.new_tt_slots,
+                    freed_blocks=self.freed_blocks, req_status=self.req_status, counts=self.counts,
+                    thr_num=thr[0], thr_den=thr[1], stream=side)
+        if partial is None:
+            vt.vtoken_plan(self.ctx, **args)
+        else:
+            vt.vtoken_plan_partial(self.ctx, **args, **partial)
         vt.vtoken_repack(self.ctx, stream=side)
         done = t.cuda.Event()
         done.record(side)
         t.cuda.current_stream().wait_event(done)                # commit only behind the repack event
         vt.vtoken_apply_moves(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
                               tt_slots=self.tt_slots, keep=self.keep, phys_len=self.phys_len,
-                              new_tt_slots=self.new_tt_slots, req_status=self.req_status)
+                              new_tt_slots=self.new_tt_slots, req_status=self.req_status,
+                              new_bt_offsets=self.new_bt_offsets)
 
     def slot_mapping(self):
         vt.vtoken_build_slot_mapping(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
@@ -153,19 +158,24 @@ class DeviceServing:
         vt.vtoken_destroy(self.ctx)
 
 
-@pytest.mark.parametrize("seed,S", [(0, 4), (1, 16), (2, 3)])
-def test_serving_loop_matches_oracle_step_by_step(seed, S):
+PARTIAL_MIX = (None, dict(util=(1, 1)), dict(util=(1, 2)), dict(util=(3, 4), max_source_blocks=3), dict())
+
+
+@pytest.mark.parametrize("seed,S,partial_options", [(0, 4, ()), (1, 16, ()), (2, 3, ()), (3, 4, PARTIAL_MIX),
+                                                    (4, 16, PARTIAL_MIX), (5, 3, PARTIAL_MIX)])
+def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options):
     import torch
     rng = np.random.default_rng(seed)
     R = 5
-    st = ServingState.random(rng, S, R, capacity=200, num_blocks=400)
+    st = ServingState.random(rng, S, R, capacity=260 if partial_options else 200,
+                             num_blocks=600 if partial_options else 400)
     truth = DictCache()
     dev = DeviceServing(st)
     n_cap = int(st.tt_offsets[-1])
     oc = dict(dirty=np.zeros(R, np.uint8), slots=np.full(n_cap, -77, np.int32), ids=np.full(n_cap, -77, np.int32),
               len=np.zeros(R, np.int32), seen=np.zeros(R, np.int32))      # the oracle's cached arrays
     repacked_something = False
-    for step in random_serving_steps(rng, st, steps=25):
+    for step in random_serving_steps(rng, st, steps=36 if partial_options else 25, partial_options=partial_options):
         if isinstance(step, Append):
             before = st.tt_len.copy()
             step.run_on_oracle(st, None, truth)
@@ -182,7 +192,7 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S):
             st_before = ServingState(st.S, st.num_blocks, st.tt_offsets, st.tt_slots.copy(), st.keep.copy(),
                                      st.tt_len.copy(), st.phys_len.copy(), [b.copy() for b in st.block_lists], free)
             step.run_on_oracle(st, None, truth)
-            dev.repack(st_before, free, nf, step.thr)
+            dev.repack(st_before, free, nf, step.thr, step.partial)
             p = step.last_plan
             repacked_something |= p.num_moves > 0
             c = dev.counts.cpu().numpy()

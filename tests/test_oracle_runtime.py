@@ -198,3 +198,67 @@ def test_slot_cache_is_stale_until_the_change_is_marked():
     assert _update(st, c) == (1, 0)
     assert c["slots"][:9].tolist() == [12, 14, 15, 4, 5, 7, 8, 9, 10] and c["len"].tolist() == [9]
     assert c["ids"][:9].tolist() == [0, 2, 3, 4, 5, 7, 8, 9, 10] and c["seen"].tolist() == [11]
+
+
+PARTIAL_MIX = (None, dict(util=(1, 1)), dict(util=(1, 2)), dict(util=(3, 4), max_source_blocks=3), dict())
+
+
+@pytest.mark.parametrize("seed,S", [(3, 4), (4, 16), (5, 3)])
+def test_serving_loop_with_partial_plans_against_a_dictionary_cache(seed, S):
+    """The same loop with the partial planner in the mix (blocks that stay, a source bound): the
+    commit must put the append position behind the moved tokens -- kept blocks may have holes, so
+    counting live entries would make new tokens overwrite live ones."""
+    rng = np.random.default_rng(seed)
+    R = 5
+    st = ServingState.random(rng, S, R, capacity=260, num_blocks=600)
+    truth = DictCache()
+    pool = np.zeros((st.num_blocks * S, 2), np.int64)
+    kinds = set()
+    for step in random_serving_steps(rng, st, steps=36, partial_options=PARTIAL_MIX):
+        step.run_on_oracle(st, pool, truth)
+        if hasattr(step, "partial") and step.last_plan.num_moves:
+            kinds.add(None if step.partial is None else tuple(sorted(step.partial)))
+        slots, ids, off = vto.build_slot_mapping(st.tt_offsets, st.tt_slots, st.keep)
+        assert len(np.unique(slots)) == len(slots)
+        for r in range(R):
+            want = truth.live_tokens(r)
+            assert ids[off[r]:off[r + 1]].tolist() == want
+            assert pool[slots[off[r]:off[r + 1]]].tolist() == [[r, t] for t in want]
+        used = set(st.bt_blocks.tolist())
+        assert len(used) == len(st.bt_blocks) and not (used & set(st.free))
+        assert set((slots // S).tolist()) <= used
+        assert vto.check_tables(S, st.num_blocks, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots,
+                                np.asarray(st.free, np.int32)) == 0
+    assert len(kinds) >= 2
+
+
+def test_append_position_after_a_partial_plan():
+    """Hand case, S = 4: blocks [A full, B 1 of 4 live, C 3 of 4 live, D 2 of 4 (tail, 2 written)];
+    sources = blocks under 100 % utilisation = B, C, D -> 6 moved tokens -> 2 destinations.  New list
+    [A, X, Y]; the next token lands at position 1*4 + 6 = 10, i.e. offset 2 of Y."""
+    S = 4
+    st = ServingState.empty(S, capacities=[20], block_lists=[np.array([10, 11, 12, 13], np.int32)], num_blocks=20)
+    vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets, st.bt_blocks, [14])
+    vto.evict_tokens(st.tt_offsets, st.tt_len, st.keep, [0] * 4, [4, 5, 6, 9])
+    p = vto.plan_partial(S, 20, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep,
+                         np.array([2, 3, 5], np.int32), util=(1, 1))
+    assert p.req_status.tolist() == [vto.REPACKED] and p.num_moves == 6 and p.new_bt_blocks.tolist() == [10, 2, 3]
+    vto.apply_moves(st.tt_offsets, st.tt_slots, st.keep, st.phys_len, p.new_tt_slots, p.req_status, S=S,
+                    new_bt_offsets=p.new_bt_offsets)
+    assert st.phys_len.tolist() == [10]
+    st.set_block_lists([p.new_bt_blocks])
+    vto.sync_new_tokens(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets, st.bt_blocks, [15])
+    assert st.tt_slots[14] == 3 * S + 2 and st.phys_len.tolist() == [11]
+    # without the block table the old rule counts live entries: the same number only when nothing stayed
+    whole = ServingState.empty(S, capacities=[20], block_lists=[np.array([10, 11, 12, 13], np.int32)], num_blocks=20)
+    vto.sync_new_tokens(S, whole.tt_offsets, whole.tt_slots, whole.keep, whole.tt_len, whole.phys_len,
+                        whole.bt_offsets, whole.bt_blocks, [14])
+    vto.evict_tokens(whole.tt_offsets, whole.tt_len, whole.keep, [0] * 4, [4, 5, 6, 9])
+    q = vto.plan(S, whole.bt_offsets, whole.bt_blocks, whole.tt_offsets, whole.tt_slots, whole.keep,
+                 np.array([2, 3, 5], np.int32))
+    a, b = whole.phys_len.copy(), whole.phys_len.copy()
+    tt1, k1 = whole.tt_slots.copy(), whole.keep.copy()
+    vto.apply_moves(whole.tt_offsets, tt1, k1, a, q.new_tt_slots, q.req_status)
+    tt2, k2 = whole.tt_slots.copy(), whole.keep.copy()
+    vto.apply_moves(whole.tt_offsets, tt2, k2, b, q.new_tt_slots, q.req_status, S=S, new_bt_offsets=q.new_bt_offsets)
+    assert a.tolist() == b.tolist() == [10]

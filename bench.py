@@ -568,6 +568,7 @@ def run_waves(args, prob, w, side, dev, plans, one_shot_ms):
               and np.array_equal(out["new_bt_offsets"], v.new_bt_offsets)
               and np.array_equal(out["new_bt_blocks"], v.new_bt_blocks)
               and np.array_equal(out["req_status"], v.req_status) and np.array_equal(out["req_wave"], v.req_wave)
+              and np.array_equal(out["req_append_pos"], v.req_append_pos)
               and np.array_equal(out["free_out"], v.free_out))
         bad = prob.verify_pools(origin_map(w.slots_per_layer, v.move_src, v.move_dst, v.wave_move_offsets))
         parity = "ok" if (ok and bad == 0) else f"FAILED (tables_ok={ok}, mismatching_words={bad})"

@@ -271,6 +271,9 @@ typedef struct {                   /* all DEVICE pointers, written by vtoken_rep
     int32_t *req_status;           /* [R] VTOKEN_REPACKED when some wave admitted the request, else its
                                       status in the last wave */
     int32_t *req_wave;             /* [R] last wave that admitted the request, -1 = none */
+    int32_t *req_append_pos;       /* [R] or NULL: position in the request's final block list behind the tokens
+                                      that wave moved ((blocks - ceil(moved / S)) * S + moved with that wave's
+                                      figures), -1 = none; pass it to vtoken_apply_moves */
     int32_t *free_out;             /* [free_capacity] the pool after the last wave */
     int32_t *num_free_out;         /* device scalar */
     vtoken_counts *wave_counts;    /* [num_waves] counts of every wave (flags of its copy included) */
@@ -336,11 +339,15 @@ int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_requests, cons
  * destination blocks, so  phys_len[r] = (blocks - ceil(moved / S)) * S + moved  with blocks from
  * new_bt_offsets and moved = entries whose slot changed.  new_bt_offsets may be NULL: phys_len[r]
  * is then the number of entries that own a slot -- the same value after vtoken_plan (nothing
- * stays), wrong after a partial plan.  phys_len may be NULL.  The block tables are the caller's:
- * it adopts new_bt_* and returns freed blocks itself. */
+ * stays), wrong after a partial plan.  append_pos (may be NULL; req_append_pos of
+ * vtoken_repack_waves) overrides both: phys_len[r] = append_pos[r] -- after several waves a partly
+ * filled destination block of an early wave may sit in the middle of the list, and only the
+ * wave-by-wave bookkeeping knows where the list ends.  phys_len may be NULL.  The block tables are
+ * the caller's: it adopts new_bt_* and returns freed blocks itself. */
 int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                        int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
-                       const int32_t *req_status, const int32_t *new_bt_offsets, void *cuda_stream);
+                       const int32_t *req_status, const int32_t *new_bt_offsets, const int32_t *append_pos,
+                       void *cuda_stream);
 
 /* Cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4): per request the slots (and
  * ids) of its active tokens in token-id order, kept on the device between decode steps and

@@ -281,16 +281,18 @@ def build_slot_mapping(tt_offsets, tt_slots, keep=None, select=None):
 
 
 def apply_moves(tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, phys_len, new_tt_slots, req_status, S=1,
-                new_bt_offsets=None) -> None:
+                new_bt_offsets=None, append_pos=None) -> None:
     """Commit of a repack, in place on tt_slots, keep and phys_len (phys_len may be None).  With
     ``S`` and ``new_bt_offsets`` the append position also holds after partial plans."""
     tt_offsets, new_tt_slots, req_status = _i32(tt_offsets), _i32(new_tt_slots), _i32(req_status)
     nbo = None if new_bt_offsets is None else _i32(new_bt_offsets)
+    apos = None if append_pos is None else _i32(append_pos)
     assert tt_slots.dtype == np.int32 and keep.dtype == np.uint8
     rc = lib().vto_apply_moves(ctypes.c_int32(len(tt_offsets) - 1), ctypes.c_int32(S), _p(tt_offsets, np.int32),
                                _p(tt_slots, np.int32), _p(keep, np.uint8),
                                None if phys_len is None else _p(phys_len, np.int32), _p(new_tt_slots, np.int32),
-                               _p(req_status, np.int32), None if nbo is None else _p(nbo, np.int32))
+                               _p(req_status, np.int32), None if nbo is None else _p(nbo, np.int32),
+                               None if apos is None else _p(apos, np.int32))
     if rc != 0:
         raise ValueError(f"vto_apply_moves failed: {rc}")
 
@@ -411,6 +413,7 @@ class WavePlan:
     new_tt_slots: np.ndarray
     req_status: np.ndarray
     req_wave: np.ndarray
+    req_append_pos: np.ndarray    # append position of every repacked request in its final block list, -1 = none
     free_out: np.ndarray          # the pool after the last wave
     move_src: np.ndarray          # all waves back to back; apply in this order
     move_dst: np.ndarray
@@ -431,6 +434,7 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
     new_tt_slots = np.full(max(T, 1), -7, np.int32)
     status = np.full(max(R, 1), -7, np.int32)
     wave = np.full(max(R, 1), -7, np.int32)
+    apos = np.full(max(R, 1), -7, np.int32)
     free_out = np.full(max(num_free + nbt, 1), -7, np.int32)
     nfo = ctypes.c_int32(0)
     cap = max(1, T * num_waves)
@@ -451,12 +455,13 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
                               ctypes.c_int32(num_free), None if o is None else ctypes.byref(o),
                               ctypes.c_int32(num_waves), _p(new_bt_offsets, np.int32), _p(new_bt_blocks, np.int32),
                               _p(new_tt_slots, np.int32), _p(status, np.int32), _p(wave, np.int32),
-                              _p(free_out, np.int32), ctypes.byref(nfo), _p(msrc, np.int32), _p(mdst, np.int32),
+                              _p(apos, np.int32), _p(free_out, np.int32), ctypes.byref(nfo), _p(msrc, np.int32), _p(mdst, np.int32),
                               ctypes.c_int64(cap), offs.ctypes.data_as(ctypes.c_void_p), counts)
     if rc != 0:
         raise ValueError(f"vto_plan_waves failed: {rc}")
     total = int(offs[num_waves])
     wc = [{n: getattr(c, n) for n, _ in _Counts._fields_} for c in counts]
     return WavePlan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
-                    status[:R].copy(), wave[:R].copy(), free_out[:nfo.value].copy(), msrc[:total].copy(),
+                    status[:R].copy(), wave[:R].copy(), apos[:R].copy(), free_out[:nfo.value].copy(),
+                    msrc[:total].copy(),
                     mdst[:total].copy(), offs, wc)

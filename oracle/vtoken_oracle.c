@@ -428,7 +428,7 @@ int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32
 
 int vto_apply_moves(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
                     int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status,
-                    const int32_t *new_bt_offsets)
+                    const int32_t *new_bt_offsets, const int32_t *append_pos)
 {
     if (R < 0 || S < 1 || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTO_EINVAL;
     for (int32_t r = 0; r < R; ++r) {
@@ -440,7 +440,9 @@ int vto_apply_moves(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt
             with_slot += new_tt_slots[t] >= 0;
         }
         if (phys_len && req_status && req_status[r] == VTO_REPACKED) {
-            if (new_bt_offsets) {
+            if (append_pos) {
+                phys_len[r] = append_pos[r];            /* worked out by the repack in waves, wave by wave */
+            } else if (new_bt_offsets) {
                 /* new block list = blocks that stayed, then the destination blocks, which the moved
                  * tokens fill densely: the next token lands right behind them */
                 const int32_t blocks = new_bt_offsets[r + 1] - new_bt_offsets[r];
@@ -692,8 +694,8 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
                    const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
                    int32_t num_waves,
                    int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
-                   int32_t *req_status, int32_t *req_wave, int32_t *free_out, int32_t *num_free_out,
-                   int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
+                   int32_t *req_status, int32_t *req_wave, int32_t *req_append_pos, int32_t *free_out,
+                   int32_t *num_free_out, int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
                    int64_t *wave_move_offsets, vto_counts *wave_counts)
 {
     if (R < 0 || S < 1 || num_free < 0 || num_waves < 1 || !bt_offsets || !tt_offsets || !num_free_out ||
@@ -724,6 +726,7 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
     for (int32_t r = 0; r < R; ++r) {
         req_status[r] = VTO_NOT_SELECTED;
         req_wave[r] = -1;
+        if (req_append_pos) req_append_pos[r] = -1;
     }
     int64_t total_moves = 0;
     wave_move_offsets[0] = 0;
@@ -750,6 +753,18 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
         }
         total_moves += c.num_moves;
         wave_move_offsets[k + 1] = total_moves;
+        /* where a request repacked by this wave appends from now on: behind the tokens this wave
+         * moved, which fill its destination blocks at the end of its new block list */
+        if (req_append_pos) {
+            for (int32_t r = 0; r < R; ++r) {
+                if (status[r] != VTO_REPACKED) continue;
+                int32_t moved = 0;
+                for (int64_t t = tt_offsets[r]; t < tt_offsets[r + 1]; ++t)
+                    moved += nxt_tts[t] >= 0 && nxt_tts[t] != cur_tts[t];
+                const int32_t blocks = nxt_bto[r + 1] - nxt_bto[r];
+                req_append_pos[r] = (blocks - ceil_div(moved, S)) * S + moved;
+            }
+        }
         /* commit: the proposed tables become the state (apply_moves, Sec. 3.2) ... */
         memcpy(cur_bto, nxt_bto, nR * sizeof(int32_t));
         if (nxt_bto[R] > 0) memcpy(cur_btb, nxt_btb, (size_t)nxt_bto[R] * sizeof(int32_t));

@@ -163,10 +163,13 @@ int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32
  * block list is now the blocks that stayed followed by the destination blocks, so for requests
  * with status VTO_REPACKED  phys_len[r] = (blocks - ceil(moved / S)) * S + moved, with blocks from
  * new_bt_offsets and moved = entries whose slot changed.  new_bt_offsets == NULL: phys_len[r] =
- * number of entries with a slot (the same value after a whole-request plan, where nothing stays). */
+ * number of entries with a slot (the same value after a whole-request plan, where nothing stays).
+ * append_pos != NULL (the per-request positions a repack in waves reports): phys_len[r] =
+ * append_pos[r] -- after several waves a partly filled destination block of an early wave may sit
+ * in the middle of the list, and only the wave-by-wave bookkeeping knows where the list ends. */
 int vto_apply_moves(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
                     int32_t *phys_len, const int32_t *new_tt_slots, const int32_t *req_status,
-                    const int32_t *new_bt_offsets);
+                    const int32_t *new_bt_offsets, const int32_t *append_pos);
 
 /* ---- cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4) -------------------------
  * The worker keeps, per request, the slots of its active tokens in token-id order -- the array a
@@ -254,6 +257,8 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
  * nothing changes nothing.
  * Outputs: the tables after the last wave; req_status[r] = VTO_REPACKED when some wave admitted r,
  * else its status in the last wave; req_wave[r] = last wave that admitted r, -1 when none;
+ * req_append_pos[r] (may be NULL) = position in r's final block list behind the tokens that wave
+ * moved, (blocks - ceil(moved / S)) * S + moved with that wave's figures, -1 when none;
  * free_out[<= num_free + total old blocks] / *num_free_out = the pool after the last wave;
  * wave_counts[num_waves] = counts of every wave; move_src / move_dst = the move lists of all
  * waves back to back, wave k in [wave_move_offsets[k], wave_move_offsets[k+1]) -- they must be
@@ -266,8 +271,8 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
                    const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
                    int32_t num_waves,
                    int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
-                   int32_t *req_status, int32_t *req_wave, int32_t *free_out, int32_t *num_free_out,
-                   int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
+                   int32_t *req_status, int32_t *req_wave, int32_t *req_append_pos, int32_t *free_out,
+                   int32_t *num_free_out, int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
                    int64_t *wave_move_offsets, vto_counts *wave_counts);
 
 int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */

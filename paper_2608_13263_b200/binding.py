@@ -76,7 +76,7 @@ class PartialOpts(ctypes.Structure):
 class WavesOut(ctypes.Structure):
     _fields_ = [("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
                 ("new_tt_slots", ctypes.c_void_p), ("req_status", ctypes.c_void_p), ("req_wave", ctypes.c_void_p),
-                ("free_out", ctypes.c_void_p), ("num_free_out", ctypes.c_void_p), ("wave_counts", ctypes.c_void_p),
+                ("req_append_pos", ctypes.c_void_p), ("free_out", ctypes.c_void_p), ("num_free_out", ctypes.c_void_p), ("wave_counts", ctypes.c_void_p),
                 ("free_capacity", ctypes.c_int32), ("workspace", ctypes.c_void_p),
                 ("workspace_bytes", ctypes.c_int64)]
 
@@ -145,7 +145,7 @@ def load():
         lib.vtoken_evict_tokens.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 7
         lib.vtoken_sync_new_tokens.argtypes = [ctypes.c_void_p] * 11
         lib.vtoken_build_slot_mapping.argtypes = [ctypes.c_void_p] * 8 + [ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
-        lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 10
+        lib.vtoken_apply_moves.argtypes = [ctypes.c_void_p] * 11
         lib.vtoken_block_liveness.argtypes = [ctypes.c_void_p] * 11
         lib.vtoken_digest_logical.argtypes = [ctypes.c_void_p] * 6 + [ctypes.c_int32, ctypes.c_int32] + [ctypes.c_void_p] * 3
         lib.vtoken_plan_partial.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.POINTER(PartialOpts),
@@ -324,10 +324,10 @@ def vtoken_build_slot_mapping(ctx, *, num_requests, tt_offsets, tt_slots, keep, 
 
 
 def vtoken_apply_moves(ctx, *, num_requests, tt_offsets, tt_slots, keep, phys_len, new_tt_slots, req_status,
-                       new_bt_offsets=None, stream=None) -> None:
+                       new_bt_offsets=None, append_pos=None, stream=None) -> None:
     _check(load().vtoken_apply_moves(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                                      _ptr(phys_len), _ptr(new_tt_slots), _ptr(req_status), _ptr(new_bt_offsets),
-                                     _stream(stream)),
+                                     _ptr(append_pos), _stream(stream)),
            "vtoken_apply_moves", ctx)
 
 
@@ -382,13 +382,13 @@ def vtoken_waves_workspace_bytes(ctx, free_capacity: int) -> int:
 def vtoken_repack_waves(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
                         num_waves, new_bt_offsets, new_bt_blocks, new_tt_slots, req_status, req_wave, free_out,
                         num_free_out, wave_counts, free_capacity, workspace, workspace_bytes, select=None, thr_num=0,
-                        thr_den=0, partial=None, stream=None) -> None:
+                        thr_den=0, partial=None, req_append_pos=None, stream=None) -> None:
     """``partial``: None for the whole-request planner, else a dict with the option keywords of
     vtoken_plan_partial (protect, util, max_source_blocks, theta)."""
     pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                  _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
     wout = WavesOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(req_status), _ptr(req_wave),
-                    _ptr(free_out), _ptr(num_free_out), _ptr(wave_counts), free_capacity, _ptr(workspace),
+                    _ptr(req_append_pos), _ptr(free_out), _ptr(num_free_out), _ptr(wave_counts), free_capacity, _ptr(workspace),
                     workspace_bytes)
     po = None
     if partial is not None:

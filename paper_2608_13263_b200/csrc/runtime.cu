@@ -81,7 +81,7 @@ __global__ void __launch_bounds__(RT_NT) apply_moves_kernel(const int32_t *num_r
                                                             int32_t S, const int32_t *tt_offsets, int32_t *tt_slots,
                                                             uint8_t *keep, int32_t *phys_len,
                                                             const int32_t *new_tt_slots, const int32_t *req_status,
-                                                            const int32_t *new_bt_offsets)
+                                                            const int32_t *new_bt_offsets, const int32_t *append_pos)
 {
     const int r = blockIdx.x;
     if (r >= rt_requests(num_requests, max_requests)) return;
@@ -108,7 +108,9 @@ __global__ void __launch_bounds__(RT_NT) apply_moves_kernel(const int32_t *num_r
     if (threadIdx.x == 0 && phys_len != nullptr && req_status != nullptr && req_status[r] == VTOKEN_REPACKED) {
         int sn = 0, sm = 0;
         for (int w = 0; w < RT_NT / 32; ++w) { sn += warp_n[w]; sm += warp_m[w]; }
-        if (new_bt_offsets != nullptr) {
+        if (append_pos != nullptr) {
+            phys_len[r] = append_pos[r];           // worked out by the repack in waves, wave by wave
+        } else if (new_bt_offsets != nullptr) {
             const int blocks = new_bt_offsets[r + 1] - new_bt_offsets[r];
             phys_len[r] = (blocks - (sm + S - 1) / S) * S + sm;
         } else {
@@ -155,13 +157,14 @@ int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const i
 
 int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                        int32_t *tt_slots, uint8_t *keep, int32_t *phys_len, const int32_t *new_tt_slots,
-                       const int32_t *req_status, const int32_t *new_bt_offsets, void *cuda_stream)
+                       const int32_t *req_status, const int32_t *new_bt_offsets, const int32_t *append_pos,
+                       void *cuda_stream)
 {
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTOKEN_EINVAL;
     if (phys_len && !req_status) return VTOKEN_EINVAL;
     apply_moves_kernel<<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
         num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, phys_len, new_tt_slots,
-        req_status, new_bt_offsets);
+        req_status, new_bt_offsets, append_pos);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -15,6 +15,10 @@ struct CommitArgs {
     int32_t max_requests, wave;
     const int32_t *status_k;          // statuses of this wave
     int32_t *req_status, *req_wave;   // merged over the waves so far
+    int32_t *req_append_pos;          // or NULL
+    const int32_t *moved;             // tokens this wave moves per request (planner scratch)
+    const int32_t *new_bt_offsets;    // block tables this wave proposes
+    int32_t S;
     const int32_t *pool, *num_pool;   // P_k and its size
     const int32_t *freed;             // blocks reclaimed by this wave
     vtoken_counts *wave_counts;       // counts of this wave (written by the planner)
@@ -33,9 +37,15 @@ __global__ void __launch_bounds__(COMMIT_NT) wave_commit_kernel(CommitArgs a)
         if (s == VTOKEN_REPACKED) {
             a.req_status[r] = VTOKEN_REPACKED;
             a.req_wave[r] = a.wave;
+            if (a.req_append_pos) {
+                // behind the tokens this wave moved: they fill its destination blocks at the end of the list
+                const int m = a.moved[r], blocks = a.new_bt_offsets[r + 1] - a.new_bt_offsets[r];
+                a.req_append_pos[r] = (blocks - (m + a.S - 1) / a.S) * a.S + m;
+            }
         } else if (a.wave == 0) {
             a.req_status[r] = s;
             a.req_wave[r] = -1;
+            if (a.req_append_pos) a.req_append_pos[r] = -1;
         } else if (a.req_status[r] != VTOKEN_REPACKED) {
             a.req_status[r] = s;
         }
@@ -139,6 +149,10 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         a.status_k = po.req_status;
         a.req_status = out->req_status;
         a.req_wave = out->req_wave;
+        a.req_append_pos = out->req_append_pos;
+        a.moved = opts ? ctx->req_nsrc : ctx->req_n;      // live tokens in the sources / of the request
+        a.new_bt_offsets = po.new_bt_offsets;
+        a.S = ctx->cfg.block_size;
         a.pool = cur.free_blocks;
         a.num_pool = cur.num_free;
         a.freed = po.freed_blocks;

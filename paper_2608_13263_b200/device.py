@@ -129,6 +129,7 @@ class DeviceProblem:
             i32 = dict(dtype=torch.int32, device=dev)
             nbytes = vt.vtoken_waves_workspace_bytes(self.ctx, self.max_free)
             self._waves = dict(req_wave=torch.full((self.max_requests,), -9, **i32),
+                               req_append_pos=torch.full((self.max_requests,), -9, **i32),
                                free_out=torch.full((self.max_free,), -9, **i32),
                                num_free_out=torch.full((1,), -9, **i32),
                                counts=torch.zeros((num_waves, 8), **i32),
@@ -143,7 +144,7 @@ class DeviceProblem:
                                free_out=wv["free_out"], num_free_out=wv["num_free_out"], wave_counts=wv["counts"],
                                free_capacity=self.max_free, workspace=wv["workspace"], workspace_bytes=wv["nbytes"],
                                select=self.select, thr_num=self.w.thr_num, thr_den=self.w.thr_den, partial=partial,
-                               stream=stream)
+                               req_append_pos=wv["req_append_pos"], stream=stream)
 
     def waves_outputs(self, num_waves: int) -> dict:
         """Host copies of the outputs of ``repack_waves``."""
@@ -160,6 +161,7 @@ class DeviceProblem:
         out["new_tt_slots"] = self.new_tt_slots.cpu().numpy()[:T]
         out["req_status"] = self.req_status.cpu().numpy()[:R]
         out["req_wave"] = wv["req_wave"].cpu().numpy()[:R]
+        out["req_append_pos"] = wv["req_append_pos"].cpu().numpy()[:R]
         nfo = int(wv["num_free_out"].item())
         out["free_out"] = wv["free_out"].cpu().numpy()[:nfo]
         return out

@@ -111,10 +111,22 @@ class Repack:
     num_free_limit: int = -1      # >= 0: pretend the free list is this short
     last_plan: object = None
     partial: dict = None          # options of the partial planner; None = whole-request plan
+    waves: int = 0                # > 0: repack in this many waves (reclaimed blocks feed the next wave)
 
     def run_on_oracle(self, st, pool, truth):
         free = np.asarray(st.free, np.int32)
         nf = len(free) if self.num_free_limit < 0 else min(len(free), self.num_free_limit)
+        if self.waves:
+            p = vto.plan_waves(st.S, st.num_blocks, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep,
+                               free[:nf], self.waves, thr_num=self.thr[0], thr_den=self.thr[1], partial=self.partial)
+            self.last_plan = p
+            if pool is not None:
+                vto.apply_moves_slab(pool, p.move_src, p.move_dst)        # list order = wave order
+            vto.apply_moves(st.tt_offsets, st.tt_slots, st.keep, st.phys_len, p.new_tt_slots, p.req_status, S=st.S,
+                            append_pos=p.req_append_pos)
+            st.set_block_lists([p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]] for r in range(st.R)])
+            st.free = p.free_out.tolist() + free[nf:].tolist()
+            return
         if self.partial is None:
             p = vto.plan(st.S, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep, free,
                          thr_num=self.thr[0], thr_den=self.thr[1], num_free=nf)
@@ -131,9 +143,10 @@ class Repack:
         st.free = free[p.num_free_consumed:].tolist() + p.freed_blocks.tolist()
 
 
-def random_serving_steps(rng, st, steps, partial_options=()):
+def random_serving_steps(rng, st, steps, partial_options=(), wave_options=()):
     """A seeded sequence of appends, evictions and repacks sized for ``st``.  ``partial_options``:
-    option dicts of the partial planner to draw repacks from (empty: whole-request plans only)."""
+    option dicts of the partial planner to draw repacks from (empty: whole-request plans only);
+    ``wave_options``: wave counts to draw from (0 = a single plan; empty: single plans only)."""
     R = st.R
     cap = np.diff(st.tt_offsets)
     length = np.zeros(R, np.int64)
@@ -155,4 +168,9 @@ def random_serving_steps(rng, st, steps, partial_options=()):
             partial = None
             if len(partial_options):
                 partial = partial_options[int(rng.integers(0, len(partial_options)))]
-            yield Repack(thr, limit, partial=partial)
+            waves = 0
+            if len(wave_options):
+                waves = int(wave_options[int(rng.integers(0, len(wave_options)))])
+                if waves and limit < 0:
+                    limit = int(rng.integers(2, 12))          # waves are for short pools
+            yield Repack(thr, limit, partial=partial, waves=waves)

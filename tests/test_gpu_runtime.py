@@ -131,6 +131,37 @@ class DeviceServing:
                               new_tt_slots=self.new_tt_slots, req_status=self.req_status,
                               new_bt_offsets=self.new_bt_offsets)
 
+    def repack_waves(self, st, free, nf, thr, partial, waves):
+        """Plan + copy + commit in waves on a side stream, then the table commit with the append
+        positions the waves report."""
+        t = self.torch
+        i32 = dict(dtype=t.int32, device=self.dev)
+        self.upload_blocks(st)
+        self.free_blocks[:len(free)].copy_(t.from_numpy(np.asarray(free, np.int32)))
+        self.num_free.fill_(nf)
+        nbytes = vt.vtoken_waves_workspace_bytes(self.ctx, self.NB)
+        wv = dict(req_wave=t.full((self.R,), -9, **i32), req_append_pos=t.full((self.R,), -9, **i32),
+                  free_out=t.full((self.NB,), -9, **i32), num_free_out=t.zeros(1, **i32),
+                  wave_counts=t.zeros((waves, 8), **i32), workspace=t.empty(nbytes, dtype=t.uint8, device=self.dev))
+        side = t.cuda.Stream()
+        side.wait_stream(t.cuda.current_stream())
+        vt.vtoken_repack_waves(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
+                               bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
+                               keep=self.keep, free_blocks=self.free_blocks, num_free=self.num_free, num_waves=waves,
+                               new_bt_offsets=self.new_bt_offsets, new_bt_blocks=self.new_bt_blocks,
+                               new_tt_slots=self.new_tt_slots, req_status=self.req_status, free_capacity=self.NB,
+                               workspace_bytes=nbytes, thr_num=thr[0], thr_den=thr[1], partial=partial, stream=side,
+                               **wv)
+        done = t.cuda.Event()
+        done.record(side)
+        t.cuda.current_stream().wait_event(done)
+        vt.vtoken_apply_moves(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
+                              tt_slots=self.tt_slots, keep=self.keep, phys_len=self.phys_len,
+                              new_tt_slots=self.new_tt_slots, req_status=self.req_status,
+                              append_pos=wv["req_append_pos"])
+        t.cuda.synchronize()
+        return wv
+
     def slot_mapping(self):
         vt.vtoken_build_slot_mapping(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
                                      tt_slots=self.tt_slots, keep=self.keep, select=None, out_slots=self.map_slots,
@@ -161,9 +192,11 @@ class DeviceServing:
 PARTIAL_MIX = (None, dict(util=(1, 1)), dict(util=(1, 2)), dict(util=(3, 4), max_source_blocks=3), dict())
 
 
-@pytest.mark.parametrize("seed,S,partial_options", [(0, 4, ()), (1, 16, ()), (2, 3, ()), (3, 4, PARTIAL_MIX),
-                                                    (4, 16, PARTIAL_MIX), (5, 3, PARTIAL_MIX)])
-def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options):
+@pytest.mark.parametrize("seed,S,partial_options,wave_options", [
+    (0, 4, (), ()), (1, 16, (), ()), (2, 3, (), ()), (3, 4, PARTIAL_MIX, ()), (4, 16, PARTIAL_MIX, ()),
+    (5, 3, PARTIAL_MIX, ()), (6, 4, PARTIAL_MIX, (0, 2, 3, 4)), (7, 8, PARTIAL_MIX, (2, 3, 5)),
+    (8, 3, PARTIAL_MIX, (0, 3, 4))])
+def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options, wave_options):
     import torch
     rng = np.random.default_rng(seed)
     R = 5
@@ -175,7 +208,8 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options):
     oc = dict(dirty=np.zeros(R, np.uint8), slots=np.full(n_cap, -77, np.int32), ids=np.full(n_cap, -77, np.int32),
               len=np.zeros(R, np.int32), seen=np.zeros(R, np.int32))      # the oracle's cached arrays
     repacked_something = False
-    for step in random_serving_steps(rng, st, steps=36 if partial_options else 25, partial_options=partial_options):
+    for step in random_serving_steps(rng, st, steps=36 if partial_options else 25, partial_options=partial_options,
+                                     wave_options=wave_options):
         if isinstance(step, Append):
             before = st.tt_len.copy()
             step.run_on_oracle(st, None, truth)
@@ -192,16 +226,31 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options):
             st_before = ServingState(st.S, st.num_blocks, st.tt_offsets, st.tt_slots.copy(), st.keep.copy(),
                                      st.tt_len.copy(), st.phys_len.copy(), [b.copy() for b in st.block_lists], free)
             step.run_on_oracle(st, None, truth)
-            dev.repack(st_before, free, nf, step.thr, step.partial)
             p = step.last_plan
-            repacked_something |= p.num_moves > 0
-            c = dev.counts.cpu().numpy()
-            assert c[:6].tolist() == [p.num_moves, p.num_dst_blocks, p.num_freed, p.num_free_consumed,
-                                      p.num_admitted, p.num_deferred] and c[6] == 0
-            assert np.array_equal(dev.req_status.cpu().numpy(), p.req_status)
-            assert np.array_equal(dev.new_bt_offsets.cpu().numpy(), p.new_bt_offsets)
-            assert np.array_equal(dev.new_bt_blocks.cpu().numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
-            assert np.array_equal(dev.freed_blocks.cpu().numpy()[:p.num_freed], p.freed_blocks)
+            if step.waves:
+                wv = dev.repack_waves(st_before, free, nf, step.thr, step.partial, step.waves)
+                repacked_something |= len(p.move_src) > 0
+                for k in range(step.waves):
+                    c = wv["wave_counts"][k].cpu().numpy()
+                    assert c[:6].tolist() == [p.wave_counts[k][n] for n in
+                                              ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed",
+                                               "num_admitted", "num_deferred")] and c[6] == 0
+                assert np.array_equal(dev.req_status.cpu().numpy(), p.req_status)
+                assert np.array_equal(wv["req_wave"].cpu().numpy(), p.req_wave)
+                assert np.array_equal(wv["req_append_pos"].cpu().numpy(), p.req_append_pos)
+                assert np.array_equal(dev.new_bt_offsets.cpu().numpy(), p.new_bt_offsets)
+                assert np.array_equal(dev.new_bt_blocks.cpu().numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
+                assert np.array_equal(wv["free_out"].cpu().numpy()[:int(wv["num_free_out"].item())], p.free_out)
+            else:
+                dev.repack(st_before, free, nf, step.thr, step.partial)
+                repacked_something |= p.num_moves > 0
+                c = dev.counts.cpu().numpy()
+                assert c[:6].tolist() == [p.num_moves, p.num_dst_blocks, p.num_freed, p.num_free_consumed,
+                                          p.num_admitted, p.num_deferred] and c[6] == 0
+                assert np.array_equal(dev.req_status.cpu().numpy(), p.req_status)
+                assert np.array_equal(dev.new_bt_offsets.cpu().numpy(), p.new_bt_offsets)
+                assert np.array_equal(dev.new_bt_blocks.cpu().numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
+                assert np.array_equal(dev.freed_blocks.cpu().numpy()[:p.num_freed], p.freed_blocks)
             assert len(blocks_before) >= len(p.new_bt_blocks)
             vto.slot_cache_mark(oc["dirty"], req_status=p.req_status)
             dev.cache_mark(status=True)

@@ -46,6 +46,7 @@ def compare(out, v, num_waves):
             assert out["wave_counts"][k][n] == v.wave_counts[k][n], (k, n)
     assert np.array_equal(out["req_status"], v.req_status)
     assert np.array_equal(out["req_wave"], v.req_wave)
+    assert np.array_equal(out["req_append_pos"], v.req_append_pos)
     assert np.array_equal(out["new_bt_offsets"], v.new_bt_offsets)
     assert np.array_equal(out["new_bt_blocks"], v.new_bt_blocks)
     assert np.array_equal(out["new_tt_slots"], v.new_tt_slots)

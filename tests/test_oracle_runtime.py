@@ -203,21 +203,24 @@ def test_slot_cache_is_stale_until_the_change_is_marked():
 PARTIAL_MIX = (None, dict(util=(1, 1)), dict(util=(1, 2)), dict(util=(3, 4), max_source_blocks=3), dict())
 
 
-@pytest.mark.parametrize("seed,S", [(3, 4), (4, 16), (5, 3)])
-def test_serving_loop_with_partial_plans_against_a_dictionary_cache(seed, S):
-    """The same loop with the partial planner in the mix (blocks that stay, a source bound): the
-    commit must put the append position behind the moved tokens -- kept blocks may have holes, so
-    counting live entries would make new tokens overwrite live ones."""
+@pytest.mark.parametrize("seed,S,wave_options", [(3, 4, ()), (4, 16, ()), (5, 3, ()), (6, 4, (0, 2, 3, 4)),
+                                                 (7, 8, (2, 3, 5)), (8, 3, (0, 3, 4)), (9, 4, (3, 4))])
+def test_serving_loop_with_partial_plans_against_a_dictionary_cache(seed, S, wave_options):
+    """The same loop with the partial planner in the mix (blocks that stay, a source bound), as
+    single plans and as repacks in waves: the commit must put the append position behind the moved
+    tokens -- blocks that stayed may have holes, and after several waves a partly filled
+    destination block of an early wave may sit in the middle of the list -- or new tokens
+    overwrite live ones."""
     rng = np.random.default_rng(seed)
     R = 5
     st = ServingState.random(rng, S, R, capacity=260, num_blocks=600)
     truth = DictCache()
     pool = np.zeros((st.num_blocks * S, 2), np.int64)
     kinds = set()
-    for step in random_serving_steps(rng, st, steps=36, partial_options=PARTIAL_MIX):
+    for step in random_serving_steps(rng, st, steps=36, partial_options=PARTIAL_MIX, wave_options=wave_options):
         step.run_on_oracle(st, pool, truth)
-        if hasattr(step, "partial") and step.last_plan.num_moves:
-            kinds.add(None if step.partial is None else tuple(sorted(step.partial)))
+        if hasattr(step, "partial") and len(step.last_plan.move_src):
+            kinds.add((step.waves > 0, None if step.partial is None else tuple(sorted(step.partial))))
         slots, ids, off = vto.build_slot_mapping(st.tt_offsets, st.tt_slots, st.keep)
         assert len(np.unique(slots)) == len(slots)
         for r in range(R):

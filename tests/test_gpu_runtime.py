@@ -265,6 +265,15 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options, wave
         assert np.array_equal(dev.cache_len.cpu().numpy(), oc["len"])
         assert np.array_equal(dev.cache_seen.cpu().numpy(), oc["seen"])
         assert not dev.dirty.cpu().numpy().any()
+        # the device tables still satisfy every input precondition (unique mapping among them)
+        dev.upload_blocks(st)
+        dev.free_blocks[:len(st.free)].copy_(torch.from_numpy(np.asarray(st.free, np.int32)))
+        dev.num_free.fill_(len(st.free))
+        bits = torch.full((1,), -1, dtype=torch.int32, device=dev.dev)
+        vt.vtoken_check_tables(dev.ctx, num_requests=dev.num_requests, bt_offsets=dev.bt_offsets,
+                               bt_blocks=dev.bt_blocks, tt_offsets=dev.tt_offsets, tt_slots=dev.tt_slots,
+                               free_blocks=dev.free_blocks, num_free=dev.num_free, out_bits=bits)
+        assert int(bits.item()) == 0
         # table state
         assert np.array_equal(dev.tt_slots.cpu().numpy(), st.tt_slots)
         assert np.array_equal(dev.keep.cpu().numpy(), st.keep)

@@ -81,3 +81,54 @@ def test_fuzz_whole_and_partial_plans(seed):
     assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
     assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
     prob.close()
+
+
+@pytest.mark.parametrize("seed", range(24))
+def test_fuzz_repack_in_waves(seed):
+    """Random problems through vtoken_repack_waves (short pools, whole and partial planners): all
+    outputs and whole pools against the oracle's wave plan, and the relocation digest of every
+    request is the same before and after."""
+    import torch
+    from paper_2608_13263_b200 import binding as vt
+    from paper_2608_13263_b200.device import DeviceProblem
+    rng = np.random.default_rng(5000 + seed)
+    w = random_problem(rng)
+    S = w.block_size
+    num_free = int(rng.integers(0, min(len(w.free_blocks), 12) + 1))
+    waves = int(rng.integers(1, 6))
+    partial = None
+    if rng.random() < 0.5:
+        partial = dict(util=[(0, 0), (1, 1), (1, 2), (3, 4)][int(rng.integers(0, 4))],
+                       max_source_blocks=int(rng.choice([0, 1, 2, 5])),
+                       theta=[(0, 0), (1, 4)][int(rng.integers(0, 2))])
+    variant = int(rng.choice([0, 1, 2])) if w.row_bytes >= 16 else 1
+    prob = DeviceProblem(w, fill_seed=seed, copy_variant=variant, wave_capacity=True)
+    digest = lambda tt, keep: _digest(prob, vt, tt, keep)
+    before = digest(prob.tt_slots, prob.keep) if w.row_bytes % 16 == 0 else None
+    prob.repack_waves(waves, num_free=torch.tensor([num_free], dtype=torch.int32, device=prob.device), partial=partial)
+    out = prob.waves_outputs(waves)
+    v = vto.plan_waves(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                       w.free_blocks[:num_free], waves, w.select, w.thr_num, w.thr_den, partial)
+    for k in range(waves):
+        assert out["wave_counts"][k]["error_flags"] == 0
+        for n in ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"):
+            assert out["wave_counts"][k][n] == v.wave_counts[k][n], (k, n)
+    for n in ("req_status", "req_wave", "req_append_pos", "new_bt_offsets", "new_bt_blocks", "new_tt_slots", "free_out"):
+        assert np.array_equal(out[n], getattr(v, n)), n
+    kp = np.stack([wl.fill_slab(seed, 0, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
+    vp = np.stack([wl.fill_slab(seed, 1, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
+    vto.apply_moves_pools(kp, vp, v.move_src, v.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), kp)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), vp)
+    if before is not None:
+        assert np.array_equal(before, digest(prob.new_tt_slots, None))
+    prob.close()
+
+
+def _digest(prob, vt, tt_slots, keep):
+    import torch
+    dig = torch.zeros(prob.max_requests, dtype=torch.int64, device=prob.device)
+    vt.vtoken_digest_logical(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets, tt_slots=tt_slots,
+                             keep=keep, select=None, layer_begin=0, layer_end=prob.w.num_layers, out_digest=dig)
+    torch.cuda.synchronize()
+    return dig.cpu().numpy()[:prob.w.num_requests].copy()

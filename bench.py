@@ -702,8 +702,37 @@ def run_runtime(args, prob, w, side, dev):
         c_len.copy_(len_before)
         cache_update(st)
 
+    # one decode step of the policy-adapter procedure on the device (the paper's Fig. 6 order:
+    # SyncNewTokens, EvictToken for the policy's victims, BuildSlotMapping): every request registers
+    # one token and loses one (a policy at its budget), so every cached array is rebuilt
+    n2 = int(cap_off[-1])
+    step_req = np.arange(R, dtype=np.int32)
+    step_tok = (rng.random(R) * np.maximum(lens, 1)).astype(np.int32)
+    step_req_d, step_tok_d, step_n_d = d(step_req), d(step_tok), d(np.array([R], np.int32))
+    s_slots, s_ids = torch.full((max(1, n2),), -1, **i32), torch.full((max(1, n2),), -1, **i32)
+    s_len, s_seen = torch.zeros(R, **i32), torch.zeros(R, **i32)
+    s_dirty = torch.ones(R, dtype=torch.uint8, device=dev)
+    lens_d = d(lens)
+    keep2_start = keep2_d.clone()
+
+    def decode_step(st):
+        tt_len.copy_(lens_d)                       # rewind, so that every replay appends and evicts again
+        keep2_d.copy_(keep2_start)
+        vt.vtoken_sync_new_tokens(prob.ctx, num_requests=prob.num_requests, tt_offsets=cap_off_d, tt_slots=tt2,
+                                  keep=keep2_d, tt_len=tt_len, phys_len=phys, bt_offsets=prob.bt_offsets,
+                                  bt_blocks=prob.bt_blocks, new_len=new_len, stream=st)
+        vt.vtoken_evict_tokens(prob.ctx, num_victims=step_n_d, max_victims=R, victim_req=step_req_d,
+                               victim_tok=step_tok_d, num_requests=prob.num_requests, tt_offsets=cap_off_d,
+                               tt_len=tt_len, keep=keep2_d, stream=st)
+        vt.vtoken_slot_cache_mark(prob.ctx, dirty=s_dirty, num_requests=prob.num_requests, num_victims=step_n_d,
+                                  max_victims=R, victim_req=step_req_d, stream=st)
+        vt.vtoken_slot_cache_update(prob.ctx, num_requests=prob.num_requests, tt_offsets=cap_off_d, tt_slots=tt2,
+                                    keep=keep2_d, tt_len=tt_len, dirty=s_dirty, cache_slots=s_slots, cache_ids=s_ids,
+                                    cache_len=s_len, cache_seen=s_seen, stream=st)
+
     out = {}
-    table_bytes = {"slot_cache_rebuild_all": 5 * T + 8 * live, "slot_cache_append_one_token_per_request": R * 40,
+    table_bytes = {"decode_step_policy_adapter": 2 * (4 * R + n2) + R * 60 + 5 * n2 + 8 * live,
+                   "slot_cache_rebuild_all": 5 * T + 8 * live, "slot_cache_append_one_token_per_request": R * 40,
                    "slot_cache_nothing_changed": R * 13,
                    "slot_mapping": 2 * 5 * T + 8 * live, "append_one_token_per_request": R * (4 * 6 + 5),
                    "evict_64k_victims": nv * (8 + 4 + 4 + 1), "apply_moves": T * (4 + 4 + 1),
@@ -712,7 +741,7 @@ def run_runtime(args, prob, w, side, dev):
                      ("evict_64k_victims", evict), ("apply_moves", commit), ("digest_all_layers", digest),
                      ("gather_logical", gather), ("slot_cache_rebuild_all", cache_rebuild),
                      ("slot_cache_append_one_token_per_request", cache_append),
-                     ("slot_cache_nothing_changed", cache_update)):
+                     ("slot_cache_nothing_changed", cache_update), ("decode_step_policy_adapter", decode_step)):
         with torch.cuda.stream(side):
             fn(side)
         side.synchronize()
@@ -732,6 +761,9 @@ def run_runtime(args, prob, w, side, dev):
         us = e0.elapsed_time(e1) / reps * 1e3
         out[name] = {"us": us, "table_bytes": table_bytes[name], "GBs": table_bytes[name] / us / 1e3}
     out["entries"] = {"logical_tokens": T, "live_tokens": live, "requests": R, "gather_layers": g_layers}
+    out["decode_step_note"] = ("one step for all requests: sync_new_tokens (one token each), evict_tokens (one victim "
+                               "each), slot-cache mark + update (every request rebuilt); includes two device copies "
+                               "that rewind the tables before every replay")
     out["slot_cache_note"] = ("rebuild_all includes a fill of the marks, append includes two small device copies that "
                               "wind the cache back by one token per request before every replay")
     out["note"] = ("append after the first replay is a no-op per request (tt_len already equals new_len): the figure "

@@ -87,12 +87,25 @@ __global__ void __launch_bounds__(RT_NT) apply_moves_kernel(const int32_t *num_r
     if (r >= rt_requests(num_requests, max_requests)) return;
     const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
     int n = 0, moved = 0;                          // entries with a slot; entries whose slot changed
-    for (int64_t t = t0 + threadIdx.x; t < t1; t += RT_NT) {
-        const int32_t s = new_tt_slots[t];
-        moved += s >= 0 && s != tt_slots[t];       // destinations are never sources
-        tt_slots[t] = s;
-        keep[t] = s >= 0 ? 1 : 0;
-        n += s >= 0;
+    constexpr int U = 4;                           // loads of four entries in flight before the first store
+    for (int64_t tb = t0 + threadIdx.x; tb < t1; tb += (int64_t)RT_NT * U) {
+        int32_t s_new[U], s_old[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t t = tb + (int64_t)u * RT_NT;
+            s_new[u] = t < t1 ? __ldg(new_tt_slots + t) : -1;
+            s_old[u] = t < t1 ? tt_slots[t] : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t t = tb + (int64_t)u * RT_NT;
+            if (t < t1) {
+                moved += s_new[u] >= 0 && s_new[u] != s_old[u];       // destinations are never sources
+                tt_slots[t] = s_new[u];
+                keep[t] = s_new[u] >= 0 ? 1 : 0;
+                n += s_new[u] >= 0;
+            }
+        }
     }
     __shared__ int warp_n[RT_NT / 32], warp_m[RT_NT / 32];
 #pragma unroll

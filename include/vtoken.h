@@ -319,6 +319,24 @@ int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const i
                            const int32_t *bt_offsets, const int32_t *bt_blocks, const int32_t *new_len,
                            void *cuda_stream);
 
+/* The same two interfaces with the per-block liveness metadata kept current (Sec. 3.3.1: per-block
+ * liveness lets the planner find under-utilised blocks without scanning the table).  n_b: DEVICE
+ * int32 [num_blocks] as vtoken_block_liveness computes it; live_total: DEVICE int64 scalar = sum of
+ * n_b, or NULL (F = 1 - live_total / (allocated blocks * S)).  An eviction takes one live token
+ * from the block of its slot, but only if this call is what deactivates the token: a token named
+ * twice in the batch, or already evicted, counts once (the keep byte is cleared with an atomic on
+ * the aligned 32-bit word that holds it, so keep must be 4-byte aligned and allocated in multiples
+ * of four bytes).  Every newly registered token adds one to the block that holds it.  After a
+ * repack recount with vtoken_block_liveness: relocation is a structural change. */
+int vtoken_evict_tokens_counted(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max_victims,
+                                const int32_t *victim_req, const int32_t *victim_tok, const int32_t *num_requests,
+                                const int32_t *tt_offsets, const int32_t *tt_len, const int32_t *tt_slots,
+                                uint8_t *keep, int32_t *n_b, int64_t *live_total, void *cuda_stream);
+int vtoken_sync_new_tokens_counted(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                                   int32_t *tt_slots, uint8_t *keep, int32_t *tt_len, int32_t *phys_len,
+                                   const int32_t *bt_offsets, const int32_t *bt_blocks, const int32_t *new_len,
+                                   int32_t *n_b, int64_t *live_total, void *cuda_stream);
+
 /* Slot mapping (Sec. 3.4: slot = token_table[token].block_id * S + offset, looked up once per token
  * at input preparation): the slots of the active tokens (slot >= 0, and keep != 0 when keep is
  * given) of the selected requests, request order then token-id order, written densely to

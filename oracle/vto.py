@@ -263,6 +263,40 @@ def sync_new_tokens(S, tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, tt_le
     return bad.value
 
 
+def evict_tokens_counted(S, tt_offsets, tt_len, tt_slots, keep: np.ndarray, victim_req, victim_tok, n_b: np.ndarray,
+                         live_total: np.ndarray) -> int:
+    """evict_tokens that also keeps ``n_b`` (int32 [NB]) and ``live_total`` (int64 [1]) current."""
+    tt_offsets, tt_len, tt_slots = _i32(tt_offsets), _i32(tt_len), _i32(tt_slots)
+    victim_req, victim_tok = _i32(victim_req), _i32(victim_tok)
+    assert keep.dtype == np.uint8 and n_b.dtype == np.int32 and live_total.dtype == np.int64
+    bad = ctypes.c_int32(0)
+    rc = lib().vto_evict_tokens_counted(ctypes.c_int32(len(tt_len)), ctypes.c_int32(S), ctypes.c_int32(len(n_b)),
+                                        _p(tt_offsets, np.int32), _p(tt_len, np.int32), _p(tt_slots, np.int32),
+                                        _p(keep, np.uint8), _p(victim_req, np.int32), _p(victim_tok, np.int32),
+                                        ctypes.c_int32(len(victim_req)), _p(n_b, np.int32), _p(live_total, np.int64),
+                                        ctypes.byref(bad))
+    if rc != 0:
+        raise ValueError(f"vto_evict_tokens_counted failed: {rc}")
+    return bad.value
+
+
+def sync_new_tokens_counted(S, tt_offsets, tt_slots: np.ndarray, keep: np.ndarray, tt_len: np.ndarray,
+                            phys_len: np.ndarray, bt_offsets, bt_blocks, new_len, n_b: np.ndarray,
+                            live_total: np.ndarray) -> int:
+    """sync_new_tokens that also keeps ``n_b`` and ``live_total`` current."""
+    tt_offsets, bt_offsets, bt_blocks, new_len = _i32(tt_offsets), _i32(bt_offsets), _i32(bt_blocks), _i32(new_len)
+    assert n_b.dtype == np.int32 and live_total.dtype == np.int64
+    bad = ctypes.c_int32(0)
+    rc = lib().vto_sync_new_tokens_counted(ctypes.c_int32(len(tt_len)), ctypes.c_int32(S), ctypes.c_int32(len(n_b)),
+                                           _p(tt_offsets, np.int32), _p(tt_slots, np.int32), _p(keep, np.uint8),
+                                           _p(tt_len, np.int32), _p(phys_len, np.int32), _p(bt_offsets, np.int32),
+                                           _p(bt_blocks, np.int32), _p(new_len, np.int32), _p(n_b, np.int32),
+                                           _p(live_total, np.int64), ctypes.byref(bad))
+    if rc != 0:
+        raise ValueError(f"vto_sync_new_tokens_counted failed: {rc}")
+    return bad.value
+
+
 def build_slot_mapping(tt_offsets, tt_slots, keep=None, select=None):
     """Returns (slots, token_ids, offsets[R+1]) of the active tokens, request order then token id."""
     tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)

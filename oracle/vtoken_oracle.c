@@ -405,6 +405,56 @@ int vto_sync_new_tokens(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t
     return VTO_OK;
 }
 
+int vto_evict_tokens_counted(int32_t R, int32_t S, int32_t NB, const int32_t *tt_offsets, const int32_t *tt_len,
+                             const int32_t *tt_slots, uint8_t *keep, const int32_t *victim_req,
+                             const int32_t *victim_tok, int32_t num_victims, int32_t *n_b, int64_t *live_total,
+                             int32_t *num_bad)
+{
+    if (R < 0 || S < 1 || NB < 0 || num_victims < 0 || !tt_offsets || !tt_len || !tt_slots || !keep || !n_b)
+        return VTO_EINVAL;
+    int32_t bad = 0;
+    for (int32_t i = 0; i < num_victims; ++i) {
+        const int32_t r = victim_req[i], t = victim_tok[i];
+        if (r < 0 || r >= R || t < 0 || t >= tt_len[r]) { ++bad; continue; }
+        const int64_t e = (int64_t)tt_offsets[r] + t;
+        const int32_t s = tt_slots[e];
+        /* the block loses a live token only if this call is what deactivates it */
+        if (keep[e] != 0 && s >= 0 && (int64_t)s < (int64_t)NB * S) {
+            --n_b[s / S];
+            if (live_total) --*live_total;
+        }
+        keep[e] = 0;
+    }
+    if (num_bad) *num_bad = bad;
+    return VTO_OK;
+}
+
+int vto_sync_new_tokens_counted(int32_t R, int32_t S, int32_t NB, const int32_t *tt_offsets, int32_t *tt_slots,
+                                uint8_t *keep, int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
+                                const int32_t *bt_blocks, const int32_t *new_len, int32_t *n_b, int64_t *live_total,
+                                int32_t *num_bad)
+{
+    if (R < 0 || S < 1 || NB < 0 || !tt_offsets || !tt_len || !n_b) return VTO_EINVAL;
+    int32_t *before = (int32_t *)malloc(sizeof(int32_t) * (size_t)(R > 0 ? R : 1));
+    if (!before) return VTO_EINVAL;
+    for (int32_t r = 0; r < R; ++r) before[r] = tt_len[r];
+    /* register the tokens ... */
+    const int rc = vto_sync_new_tokens(R, S, tt_offsets, tt_slots, keep, tt_len, phys_len, bt_offsets, bt_blocks,
+                                       new_len, num_bad);
+    /* ... and every new token is one more live token in the block that holds it */
+    for (int32_t r = 0; r < R && rc == VTO_OK; ++r) {
+        for (int32_t t = before[r]; t < tt_len[r]; ++t) {
+            const int32_t s = tt_slots[(int64_t)tt_offsets[r] + t];
+            if (s >= 0 && (int64_t)s < (int64_t)NB * S) {
+                ++n_b[s / S];
+                if (live_total) ++*live_total;
+            }
+        }
+    }
+    free(before);
+    return rc;
+}
+
 int64_t vto_build_slot_mapping(int32_t R, const int32_t *tt_offsets, const int32_t *tt_slots,
                                const uint8_t *keep, const uint8_t *select, int32_t *out_slots,
                                int32_t *out_token_ids, int32_t *out_offsets, int64_t capacity)

@@ -150,6 +150,21 @@ int vto_sync_new_tokens(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t
                         int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
                         const int32_t *bt_blocks, const int32_t *new_len, int32_t *num_bad);
 
+/* The same two interfaces with the per-block liveness metadata kept current (Sec. 3.3.1: per-block
+ * liveness n_b lets the planner find under-utilised blocks without scanning the table): n_b[NB] as
+ * vto_block_liveness computes it, *live_total (optional) = sum of n_b.  An eviction takes one live
+ * token from the block of its slot, but only if this call is what deactivates the token (a token
+ * named twice, or already evicted, counts once); every newly registered token adds one to the
+ * block that holds it.  After a repack the counters are recomputed (vto_block_liveness). */
+int vto_evict_tokens_counted(int32_t R, int32_t S, int32_t NB, const int32_t *tt_offsets, const int32_t *tt_len,
+                             const int32_t *tt_slots, uint8_t *keep, const int32_t *victim_req,
+                             const int32_t *victim_tok, int32_t num_victims, int32_t *n_b, int64_t *live_total,
+                             int32_t *num_bad);
+int vto_sync_new_tokens_counted(int32_t R, int32_t S, int32_t NB, const int32_t *tt_offsets, int32_t *tt_slots,
+                                uint8_t *keep, int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
+                                const int32_t *bt_blocks, const int32_t *new_len, int32_t *n_b, int64_t *live_total,
+                                int32_t *num_bad);
+
 /* Slot mapping of the active tokens (slot = token_table[token].block * S + offset, Sec. 3.4): for each
  * selected request, in request order, the slots (and logical ids) of its tokens with slot >= 0 and
  * keep != 0 (keep NULL: slot >= 0) in ascending token id.  out_offsets[R+1] = first entry of each

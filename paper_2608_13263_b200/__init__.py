@@ -16,7 +16,9 @@ from .binding import (  # noqa: F401
     vtoken_plan_partial,
     vtoken_build_slot_mapping,
     vtoken_evict_tokens,
+    vtoken_evict_tokens_counted,
     vtoken_sync_new_tokens,
+    vtoken_sync_new_tokens_counted,
     vtoken_copy_grid,
     vtoken_create,
     vtoken_destroy,
@@ -39,4 +41,5 @@ __all__ = ["VtokenError", "vtoken_create", "vtoken_destroy", "vtoken_plan", "vto
            "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens", "vtoken_sync_new_tokens",
            "vtoken_build_slot_mapping", "vtoken_apply_moves", "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_repack_host_partial", "vtoken_repack_waves", "vtoken_waves_workspace_bytes", "vtoken_slot_cache_mark",
-           "vtoken_slot_cache_update", "vtoken_check_tables"]
+           "vtoken_slot_cache_update", "vtoken_check_tables", "vtoken_evict_tokens_counted",
+           "vtoken_sync_new_tokens_counted"]

@@ -23,7 +23,8 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
-           "vtoken_slot_cache_update", "vtoken_repack_host_partial", "vtoken_check_tables"]
+           "vtoken_slot_cache_update", "vtoken_repack_host_partial", "vtoken_check_tables",
+           "vtoken_evict_tokens_counted", "vtoken_sync_new_tokens_counted"]
 
 
 class VtokenError(RuntimeError):
@@ -131,6 +132,9 @@ def load():
                                                    ctypes.POINTER(PartialOpts), ctypes.c_void_p]
         lib.vtoken_check_tables.argtypes = [ctypes.c_void_p, ctypes.POINTER(PlanIn), ctypes.c_void_p, ctypes.c_void_p,
                                             ctypes.c_void_p]
+        lib.vtoken_evict_tokens_counted.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32] + \
+                                                   [ctypes.c_void_p] * 10
+        lib.vtoken_sync_new_tokens_counted.argtypes = [ctypes.c_void_p] * 13
         lib.vtoken_strerror.argtypes = [ctypes.c_int]
         lib.vtoken_strerror.restype = ctypes.c_char_p
         lib.vtoken_last_cuda_error.argtypes = [ctypes.c_void_p]
@@ -314,6 +318,22 @@ def vtoken_sync_new_tokens(ctx, *, num_requests, tt_offsets, tt_slots, keep, tt_
     _check(load().vtoken_sync_new_tokens(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                                          _ptr(tt_len), _ptr(phys_len), _ptr(bt_offsets), _ptr(bt_blocks),
                                          _ptr(new_len), _stream(stream)), "vtoken_sync_new_tokens", ctx)
+
+
+def vtoken_evict_tokens_counted(ctx, *, num_victims, max_victims, victim_req, victim_tok, num_requests, tt_offsets,
+                                tt_len, tt_slots, keep, n_b, live_total=None, stream=None) -> None:
+    _check(load().vtoken_evict_tokens_counted(ctx, _ptr(num_victims), max_victims, _ptr(victim_req), _ptr(victim_tok),
+                                              _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_len), _ptr(tt_slots),
+                                              _ptr(keep), _ptr(n_b), _ptr(live_total), _stream(stream)),
+           "vtoken_evict_tokens_counted", ctx)
+
+
+def vtoken_sync_new_tokens_counted(ctx, *, num_requests, tt_offsets, tt_slots, keep, tt_len, phys_len, bt_offsets,
+                                   bt_blocks, new_len, n_b, live_total=None, stream=None) -> None:
+    _check(load().vtoken_sync_new_tokens_counted(ctx, _ptr(num_requests), _ptr(tt_offsets), _ptr(tt_slots),
+                                                 _ptr(keep), _ptr(tt_len), _ptr(phys_len), _ptr(bt_offsets),
+                                                 _ptr(bt_blocks), _ptr(new_len), _ptr(n_b), _ptr(live_total),
+                                                 _stream(stream)), "vtoken_sync_new_tokens_counted", ctx)
 
 
 def vtoken_build_slot_mapping(ctx, *, num_requests, tt_offsets, tt_slots, keep, select, out_slots, out_token_ids,

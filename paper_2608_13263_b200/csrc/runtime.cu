@@ -17,12 +17,33 @@ __device__ __forceinline__ int rt_requests(const int32_t *num_requests, int max_
     return R < 0 ? 0 : (R > max_requests ? max_requests : R);
 }
 
+// Per-block liveness that the counted variants keep current (Sec. 3.3.1 of the paper).
+struct Liveness {
+    int32_t *n_b;                      // [num_blocks] live tokens per physical block
+    unsigned long long *live_total;    // sum of n_b, or NULL
+    const int32_t *tt_slots;           // evict only: where the victim's K/V sits
+    int64_t slots;                     // num_blocks * S
+    int32_t S;
+};
+
+// Clears one byte of the keep mask atomically and returns its previous value, so that a token
+// named twice in a batch (or already evicted) is counted once.  The mask must be allocated in
+// multiples of four bytes: the atomic works on the aligned word that holds the byte.
+__device__ __forceinline__ uint32_t clear_keep_byte(uint8_t *p)
+{
+    const uintptr_t a = (uintptr_t)p;
+    const unsigned shift = (unsigned)(a & 3u) * 8u;
+    const unsigned old = atomicAnd((unsigned *)(a & ~(uintptr_t)3), ~(0xFFu << shift));
+    return (old >> shift) & 0xFFu;
+}
+
 // evict_token over a batch of victims: metadata only, the KV bytes stay where they are
+template <bool COUNTED>
 __global__ void __launch_bounds__(RT_NT) evict_kernel(const int32_t *num_victims, int32_t max_victims,
                                                       const int32_t *victim_req, const int32_t *victim_tok,
                                                       const int32_t *num_requests, int32_t max_requests,
                                                       const int32_t *tt_offsets, const int32_t *tt_len,
-                                                      uint8_t *keep, vtoken_counts *counts)
+                                                      uint8_t *keep, vtoken_counts *counts, Liveness lv)
 {
     int n = *num_victims;
     n = n < 0 ? 0 : (n > max_victims ? max_victims : n);
@@ -31,7 +52,17 @@ __global__ void __launch_bounds__(RT_NT) evict_kernel(const int32_t *num_victims
     for (int i = blockIdx.x * RT_NT + threadIdx.x; i < n; i += gridDim.x * RT_NT) {
         const int r = victim_req[i], t = victim_tok[i];
         if (r < 0 || r >= R || t < 0 || t >= tt_len[r]) { bad = true; continue; }
-        keep[(int64_t)tt_offsets[r] + t] = 0;
+        const int64_t e = (int64_t)tt_offsets[r] + t;
+        if (COUNTED) {
+            // the block loses a live token only if this thread is the one that deactivates it
+            const int32_t s = lv.tt_slots[e];
+            if (clear_keep_byte(keep + e) != 0 && s >= 0 && (int64_t)s < lv.slots) {
+                atomicSub(&lv.n_b[s / lv.S], 1);
+                if (lv.live_total) atomicAdd(lv.live_total, ~0ull);          // minus one
+            }
+        } else {
+            keep[e] = 0;
+        }
     }
     if (bad || (threadIdx.x == 0 && blockIdx.x == 0 && *num_victims > max_victims))
         atomicOr(&counts->error_flags, VTOKEN_FLAG_BAD_VICTIM);
@@ -39,11 +70,12 @@ __global__ void __launch_bounds__(RT_NT) evict_kernel(const int32_t *num_victims
 
 // sync_new_tokens: one CTA per request; the tokens it can register are a prefix of the ones asked
 // for (table capacity and block-list room only shrink it), so the count has a closed form.
+template <bool COUNTED>
 __global__ void __launch_bounds__(RT_NT) sync_kernel(const int32_t *num_requests, int32_t max_requests, int32_t S,
                                                      const int32_t *tt_offsets, int32_t *tt_slots, uint8_t *keep,
                                                      int32_t *tt_len, int32_t *phys_len, const int32_t *bt_offsets,
                                                      const int32_t *bt_blocks, const int32_t *new_len,
-                                                     int32_t num_blocks, vtoken_counts *counts)
+                                                     int32_t num_blocks, vtoken_counts *counts, Liveness lv)
 {
     const int r = blockIdx.x;
     if (r >= rt_requests(num_requests, max_requests)) return;
@@ -59,12 +91,22 @@ __global__ void __launch_bounds__(RT_NT) sync_kernel(const int32_t *num_requests
     if (can > room - phys) can = room - phys;
     if (can < 0) can = 0;
     uint32_t flags = can < want ? VTOKEN_FLAG_APPEND_STOPPED : 0u;
+    int counted = 0;
     for (int i = threadIdx.x; i < (int)can; i += RT_NT) {
         const int p = phys + i;                              // position in the block list
         const int blk = bt_blocks[b0 + p / S];
         if (blk < 0 || blk >= num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
         tt_slots[base + len + i] = blk * S + p % S;          // slot = block_id * S + offset
         keep[base + len + i] = 1;
+        if (COUNTED && blk >= 0 && blk < num_blocks) {       // one more live token in that block
+            atomicAdd(&lv.n_b[blk], 1);
+            ++counted;
+        }
+    }
+    if (COUNTED && lv.live_total) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) counted += __shfl_down_sync(0xffffffffu, counted, d);
+        if (vtk_lane() == 0 && counted) atomicAdd(lv.live_total, (unsigned long long)counted);
     }
     __syncthreads();     // every thread has read tt_len / phys_len before they change
     if (threadIdx.x == 0) {
@@ -146,9 +188,30 @@ int vtoken_evict_tokens(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max
     if (max_victims == 0) return VTOKEN_OK;
     int grid = (max_victims + RT_NT - 1) / RT_NT;
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
-    evict_kernel<<<grid, RT_NT, 0, (cudaStream_t)cuda_stream>>>(num_victims, max_victims, victim_req, victim_tok,
-                                                                 num_requests, ctx->cfg.max_requests, tt_offsets,
-                                                                 tt_len, keep, ctx->counts);
+    evict_kernel<false><<<grid, RT_NT, 0, (cudaStream_t)cuda_stream>>>(num_victims, max_victims, victim_req,
+                                                                        victim_tok, num_requests,
+                                                                        ctx->cfg.max_requests, tt_offsets, tt_len,
+                                                                        keep, ctx->counts, Liveness{});
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+int vtoken_evict_tokens_counted(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max_victims,
+                                const int32_t *victim_req, const int32_t *victim_tok, const int32_t *num_requests,
+                                const int32_t *tt_offsets, const int32_t *tt_len, const int32_t *tt_slots,
+                                uint8_t *keep, int32_t *n_b, int64_t *live_total, void *cuda_stream)
+{
+    if (!ctx || !num_victims || !victim_req || !victim_tok || !num_requests || !tt_offsets || !tt_len || !tt_slots ||
+        !keep || !n_b)
+        return VTOKEN_EINVAL;
+    if (max_victims < 0 || ((uintptr_t)keep & 3)) return VTOKEN_EINVAL;
+    if (max_victims == 0) return VTOKEN_OK;
+    int grid = (max_victims + RT_NT - 1) / RT_NT;
+    if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
+    const Liveness lv{n_b, (unsigned long long *)live_total, tt_slots, ctx->slots_per_layer, ctx->cfg.block_size};
+    evict_kernel<true><<<grid, RT_NT, 0, (cudaStream_t)cuda_stream>>>(num_victims, max_victims, victim_req, victim_tok,
+                                                                       num_requests, ctx->cfg.max_requests,
+                                                                       tt_offsets, tt_len, keep, ctx->counts, lv);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -161,9 +224,25 @@ int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const i
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !tt_len || !phys_len || !bt_offsets ||
         !bt_blocks || !new_len)
         return VTOKEN_EINVAL;
-    sync_kernel<<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
+    sync_kernel<false><<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
         num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, tt_len, phys_len,
-        bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks, ctx->counts);
+        bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks, ctx->counts, Liveness{});
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+}
+
+int vtoken_sync_new_tokens_counted(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
+                                   int32_t *tt_slots, uint8_t *keep, int32_t *tt_len, int32_t *phys_len,
+                                   const int32_t *bt_offsets, const int32_t *bt_blocks, const int32_t *new_len,
+                                   int32_t *n_b, int64_t *live_total, void *cuda_stream)
+{
+    if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !tt_len || !phys_len || !bt_offsets ||
+        !bt_blocks || !new_len || !n_b)
+        return VTOKEN_EINVAL;
+    const Liveness lv{n_b, (unsigned long long *)live_total, nullptr, ctx->slots_per_layer, ctx->cfg.block_size};
+    sync_kernel<true><<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
+        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, tt_len, phys_len,
+        bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks, ctx->counts, lv);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -36,6 +36,17 @@ class ServingState:
     phys_len: np.ndarray        # int32 [R]
     block_lists: list           # per request int32 arrays
     free: list                  # free block ids, allocation order
+    counters: dict = None       # optional: {"n_b": int32 [num_blocks], "live": int64 [1]} kept current by the steps
+
+    def enable_counters(self):
+        self.counters = dict(n_b=np.zeros(self.num_blocks, np.int32), live=np.zeros(1, np.int64))
+
+    def recount(self):
+        """After a structural change: the counters are recomputed from the tables."""
+        n_b, _, live, _ = vto.block_liveness(self.S, self.num_blocks, self.bt_offsets, self.bt_blocks,
+                                             self.tt_offsets, self.tt_slots, self.keep)
+        self.counters["n_b"][:] = n_b
+        self.counters["live"][0] = live
 
     @classmethod
     def empty(cls, S, capacities, block_lists, num_blocks=None, free=None):
@@ -82,8 +93,13 @@ class Append:
     def run_on_oracle(self, st, pool, truth):
         old = st.tt_len.copy()
         st.grow_block_lists(self.new_len)
-        vto.sync_new_tokens(st.S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets,
-                            st.bt_blocks, self.new_len)
+        if st.counters is None:
+            vto.sync_new_tokens(st.S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets,
+                                st.bt_blocks, self.new_len)
+        else:
+            vto.sync_new_tokens_counted(st.S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len,
+                                        st.bt_offsets, st.bt_blocks, self.new_len, st.counters["n_b"],
+                                        st.counters["live"])
         for r in range(st.R):
             for t in range(int(old[r]), int(st.tt_len[r])):
                 if pool is not None:
@@ -98,7 +114,11 @@ class Evict:
     victim_tok: np.ndarray
 
     def run_on_oracle(self, st, pool, truth):
-        vto.evict_tokens(st.tt_offsets, st.tt_len, st.keep, self.victim_req, self.victim_tok)
+        if st.counters is None:
+            vto.evict_tokens(st.tt_offsets, st.tt_len, st.keep, self.victim_req, self.victim_tok)
+        else:
+            vto.evict_tokens_counted(st.S, st.tt_offsets, st.tt_len, st.tt_slots, st.keep, self.victim_req,
+                                     self.victim_tok, st.counters["n_b"], st.counters["live"])
         if truth is not None:
             for r, t in zip(self.victim_req.tolist(), self.victim_tok.tolist()):
                 if 0 <= r < st.R and 0 <= t < st.tt_len[r]:
@@ -126,6 +146,8 @@ class Repack:
                             append_pos=p.req_append_pos)
             st.set_block_lists([p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]] for r in range(st.R)])
             st.free = p.free_out.tolist() + free[nf:].tolist()
+            if st.counters is not None:
+                st.recount()
             return
         if self.partial is None:
             p = vto.plan(st.S, st.bt_offsets, st.bt_blocks, st.tt_offsets, st.tt_slots, st.keep, free,
@@ -141,6 +163,8 @@ class Repack:
                         new_bt_offsets=p.new_bt_offsets)
         st.set_block_lists([p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]] for r in range(st.R)])
         st.free = free[p.num_free_consumed:].tolist() + p.freed_blocks.tolist()
+        if st.counters is not None:
+            st.recount()
 
 
 def random_serving_steps(rng, st, steps, partial_options=(), wave_options=()):

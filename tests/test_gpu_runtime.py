@@ -58,10 +58,27 @@ class DeviceServing:
         self.cache_len = torch.zeros(st.R, **i32)
         self.cache_seen = torch.zeros(st.R, **i32)
         self.cache_stats = torch.zeros(2, **i32)
+        # per-block liveness kept current by the counted interfaces (None: plain interfaces)
+        self.n_b = self.live_total = None
         self.k_pool = torch.zeros((layers, self.NB * self.S, row_elems), dtype=torch.int16, device=dev)
         self.v_pool = torch.zeros_like(self.k_pool)
         self.ctx = vt.vtoken_create(layers, self.NB, self.S, 1, row_elems, self.k_pool, self.v_pool, st.R, cap,
                                     self.NB, self.NB)
+
+    def enable_counters(self):
+        t = self.torch
+        self.n_b = t.zeros(self.NB, dtype=t.int32, device=self.dev)
+        self.live_total = t.zeros(1, dtype=t.int64, device=self.dev)
+
+    def recount(self, st):
+        """After a repack: per-block liveness recomputed on the device."""
+        t = self.torch
+        self.upload_blocks(st)
+        summary = t.zeros(2, dtype=t.int64, device=self.dev)
+        vt.vtoken_block_liveness(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
+                                 bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
+                                 keep=self.keep, n_b=self.n_b, summary=summary)
+        self.live_total.copy_(summary[:1])
 
     def upload_blocks(self, st):
         t = self.torch
@@ -79,10 +96,13 @@ class DeviceServing:
         t = self.torch
         self.upload_blocks(st)                                  # scheduler grew the block lists on the host
         self.new_len.copy_(t.from_numpy(np.asarray(new_len, np.int32)))
-        vt.vtoken_sync_new_tokens(self.ctx, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
-                                  tt_slots=self.tt_slots, keep=self.keep, tt_len=self.tt_len,
-                                  phys_len=self.phys_len, bt_offsets=self.bt_offsets, bt_blocks=self.bt_blocks,
-                                  new_len=self.new_len)
+        args = dict(num_requests=self.num_requests, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
+                    keep=self.keep, tt_len=self.tt_len, phys_len=self.phys_len, bt_offsets=self.bt_offsets,
+                    bt_blocks=self.bt_blocks, new_len=self.new_len)
+        if self.n_b is None:
+            vt.vtoken_sync_new_tokens(self.ctx, **args)
+        else:
+            vt.vtoken_sync_new_tokens_counted(self.ctx, n_b=self.n_b, live_total=self.live_total, **args)
         # "the model" writes the K/V of the new tokens at the slots the runtime assigned
         slots = self.tt_slots.cpu().numpy()
         lens = self.tt_len.cpu().numpy()
@@ -100,10 +120,14 @@ class DeviceServing:
         self.victim_req[:n].copy_(t.from_numpy(victim_req))
         self.victim_tok[:n].copy_(t.from_numpy(victim_tok))
         self.num_victims.fill_(n)
-        vt.vtoken_evict_tokens(self.ctx, num_victims=self.num_victims, max_victims=self.max_victims,
-                               victim_req=self.victim_req, victim_tok=self.victim_tok,
-                               num_requests=self.num_requests, tt_offsets=self.tt_offsets, tt_len=self.tt_len,
-                               keep=self.keep)
+        args = dict(num_victims=self.num_victims, max_victims=self.max_victims, victim_req=self.victim_req,
+                    victim_tok=self.victim_tok, num_requests=self.num_requests, tt_offsets=self.tt_offsets,
+                    tt_len=self.tt_len, keep=self.keep)
+        if self.n_b is None:
+            vt.vtoken_evict_tokens(self.ctx, **args)
+        else:
+            vt.vtoken_evict_tokens_counted(self.ctx, tt_slots=self.tt_slots, n_b=self.n_b,
+                                           live_total=self.live_total, **args)
 
     def repack(self, st, free, nf, thr, partial=None):
         t = self.torch
@@ -432,3 +456,40 @@ def test_slot_cache_full_size_rebuild_then_append_only():
     both((3, 0))
     assert vt.vtoken_read_counts(ctx)["error_flags"] == 0
     vt.vtoken_destroy(ctx)
+
+
+@pytest.mark.parametrize("seed,S", [(10, 4), (11, 16), (12, 3)])
+def test_incremental_block_liveness_on_the_device(seed, S):
+    """The counted evict / append interfaces keep n_b and the live total current on the device
+    (recounted only after repacks); after every step they equal the oracle's counters, which the
+    CPU tests pin against a recount.  Victim batches contain repeats and already evicted tokens."""
+    import torch
+    rng = np.random.default_rng(seed)
+    R = 5
+    st = ServingState.random(rng, S, R, capacity=260, num_blocks=600)
+    st.enable_counters()
+    dev = DeviceServing(st)
+    dev.enable_counters()
+    for step in random_serving_steps(rng, st, steps=30, partial_options=PARTIAL_MIX):
+        if isinstance(step, Append):
+            before = st.tt_len.copy()
+            step.run_on_oracle(st, None, None)
+            dev.append(before, st, step.new_len)
+        elif isinstance(step, Evict):
+            step.run_on_oracle(st, None, None)
+            dev.evict(step.victim_req, step.victim_tok)
+        else:
+            free = list(st.free)
+            nf = len(free) if step.num_free_limit < 0 else min(len(free), step.num_free_limit)
+            st_before = ServingState(st.S, st.num_blocks, st.tt_offsets, st.tt_slots.copy(), st.keep.copy(),
+                                     st.tt_len.copy(), st.phys_len.copy(), [b.copy() for b in st.block_lists], free)
+            step.run_on_oracle(st, None, None)
+            dev.repack(st_before, free, nf, step.thr, step.partial)
+            dev.recount(st)
+        torch.cuda.synchronize()
+        assert np.array_equal(dev.keep.cpu().numpy(), st.keep)
+        assert np.array_equal(dev.tt_slots.cpu().numpy(), st.tt_slots)
+        assert np.array_equal(dev.n_b.cpu().numpy(), st.counters["n_b"])
+        assert int(dev.live_total.item()) == int(st.counters["live"][0])
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] & ~vt.FLAG_BAD_VICTIM == 0
+    dev.close()

@@ -265,3 +265,44 @@ def test_append_position_after_a_partial_plan():
     tt2, k2 = whole.tt_slots.copy(), whole.keep.copy()
     vto.apply_moves(whole.tt_offsets, tt2, k2, b, q.new_tt_slots, q.req_status, S=S, new_bt_offsets=q.new_bt_offsets)
     assert a.tolist() == b.tolist() == [10]
+
+
+# ---- per-block liveness kept current by the runtime interfaces --------------------------------------
+@pytest.mark.parametrize("seed,S", [(10, 4), (11, 16), (12, 3)])
+def test_incremental_block_liveness_equals_the_recount(seed, S):
+    """n_b and the live total maintained by the counted evict / append interfaces (recounted only
+    after repacks) must equal vto_block_liveness -- itself pinned by numpy.bincount -- after every
+    step of a serving loop whose victim batches contain repeats and already evicted tokens."""
+    rng = np.random.default_rng(seed)
+    R = 5
+    st = ServingState.random(rng, S, R, capacity=260, num_blocks=600)
+    st.enable_counters()
+    changed_without_repack = 0
+    for step in random_serving_steps(rng, st, steps=36, partial_options=PARTIAL_MIX, wave_options=(0, 0, 3)):
+        before = st.counters["n_b"].copy()
+        step.run_on_oracle(st, None, None)
+        n_b, _, live, _ = vto.block_liveness(S, st.num_blocks, st.bt_offsets, st.bt_blocks, st.tt_offsets,
+                                             st.tt_slots, st.keep)
+        assert np.array_equal(st.counters["n_b"], n_b) and st.counters["live"][0] == live
+        if not hasattr(step, "partial"):
+            changed_without_repack += int(not np.array_equal(before, n_b))
+    assert changed_without_repack >= 10
+
+
+def test_counted_eviction_counts_a_token_once():
+    S = 4
+    st = ServingState.empty(S, capacities=[12, 8], block_lists=[np.array([3, 1], np.int32), np.array([5], np.int32)],
+                            num_blocks=8)
+    st.enable_counters()
+    vto.sync_new_tokens_counted(S, st.tt_offsets, st.tt_slots, st.keep, st.tt_len, st.phys_len, st.bt_offsets,
+                                st.bt_blocks, [7, 3], st.counters["n_b"], st.counters["live"])
+    assert st.counters["n_b"].tolist() == [0, 3, 0, 4, 0, 3, 0, 0] and st.counters["live"][0] == 10
+    # token (0, 1) twice in one batch, (0, 5) once, two victims out of range
+    bad = vto.evict_tokens_counted(S, st.tt_offsets, st.tt_len, st.tt_slots, st.keep, [0, 0, 0, 0, 2], [1, 1, 5, 7, 0],
+                                   st.counters["n_b"], st.counters["live"])
+    assert bad == 2 and st.counters["n_b"].tolist() == [0, 2, 0, 3, 0, 3, 0, 0] and st.counters["live"][0] == 8
+    # evicting them again changes nothing
+    vto.evict_tokens_counted(S, st.tt_offsets, st.tt_len, st.tt_slots, st.keep, [0, 0], [1, 5], st.counters["n_b"],
+                             st.counters["live"])
+    assert st.counters["n_b"].tolist() == [0, 2, 0, 3, 0, 3, 0, 0] and st.counters["live"][0] == 8
+    assert st.keep[:7].tolist() == [1, 0, 1, 1, 1, 0, 1]

@@ -37,7 +37,7 @@ def build(force: bool = False) -> str:
 class _Counts(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed",
-                 "num_admitted", "num_deferred")]
+                 "num_admitted", "num_deferred", "num_released")]
 
 
 _lib = None
@@ -83,6 +83,7 @@ class Plan:
     num_free_consumed: int
     num_admitted: int
     num_deferred: int
+    released_blocks: np.ndarray = None    # references to shared blocks dropped by a copy-on-write detach
 
 
 def plan(S, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
@@ -364,7 +365,8 @@ def slot_cache_update(tt_offsets, tt_slots, keep, tt_len, dirty: np.ndarray, cac
 # ---- eligibility metadata and partial plans ---------------------------------------------------
 class _PartialOpts(ctypes.Structure):
     _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
-                ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32)]
+                ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32),
+                ("detach_num", ctypes.c_uint32), ("detach_den", ctypes.c_uint32)]
 
 
 def block_liveness(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep=None):
@@ -384,7 +386,8 @@ def block_liveness(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep=None
 
 
 def plan_partial(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, select=None, thr_num=0,
-                 thr_den=0, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0)) -> Plan:
+                 thr_den=0, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
+                 detach=(0, 0)) -> Plan:
     bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
     tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
     keep, select, free_blocks, protect = _u8(keep), _u8(select), _i32(free_blocks), _u8(protect)
@@ -402,20 +405,23 @@ def plan_partial(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_
     msrc = np.full(max(T, 1), -7, np.int32)
     mdst = np.full(max(T, 1), -7, np.int32)
     c = _Counts()
+    released = np.full(max(nbt, 1), -7, np.int32)
     o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1], max_source_blocks,
-                     theta[0], theta[1])
+                     theta[0], theta[1], detach[0], detach[1])
     rc = lib().vto_plan_partial(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
                                 _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
                                 _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),
                                 ctypes.c_uint32(thr_num), ctypes.c_uint32(thr_den), _p(free_blocks, np.int32),
                                 ctypes.c_int32(num_free), ctypes.byref(o), _p(new_bt_offsets, np.int32),
                                 _p(new_bt_blocks, np.int32), _p(new_tt_slots, np.int32), _p(freed, np.int32),
-                                _p(status, np.int32), _p(msrc, np.int32), _p(mdst, np.int32), ctypes.byref(c))
+                                _p(status, np.int32), _p(msrc, np.int32), _p(mdst, np.int32), ctypes.byref(c),
+                                _p(released, np.int32))
     if rc != 0:
         raise ValueError(f"vto_plan_partial failed: {rc}")
     return Plan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
                 freed[:c.num_freed].copy(), status[:R].copy(), msrc[:c.num_moves].copy(), mdst[:c.num_moves].copy(),
-                c.num_moves, c.num_dst_blocks, c.num_freed, c.num_free_consumed, c.num_admitted, c.num_deferred)
+                c.num_moves, c.num_dst_blocks, c.num_freed, c.num_free_consumed, c.num_admitted, c.num_deferred,
+                released[:c.num_released].copy())
 
 
 # ---- online relocation check ------------------------------------------------------------------
@@ -481,7 +487,7 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
         protect = _u8(partial.get("protect"))
         util, theta = partial.get("util", (0, 0)), partial.get("theta", (0, 0))
         o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1],
-                         partial.get("max_source_blocks", 0), theta[0], theta[1])
+                         partial.get("max_source_blocks", 0), theta[0], theta[1], 0, 0)
     rc = lib().vto_plan_waves(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
                               _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
                               _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),

@@ -103,6 +103,7 @@ int vto_plan(int32_t R, int32_t S,
     counts->num_free_consumed = consumed;
     counts->num_admitted = num_admitted;
     counts->num_deferred = num_deferred;
+    counts->num_released = 0;
     return VTO_OK;
 }
 
@@ -587,9 +588,11 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
                      int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
                      int32_t *freed_blocks, int32_t *req_status,
-                     int32_t *move_src, int32_t *move_dst, vto_counts *counts)
+                     int32_t *move_src, int32_t *move_dst, vto_counts *counts, int32_t *released_blocks)
 {
     if (R < 0 || S < 1 || NB < 1 || num_free < 0 || !opts || !counts) return VTO_EINVAL;
+    const int may_detach = opts->protect != NULL && opts->detach_den != 0;
+    if (may_detach && !released_blocks) return VTO_EINVAL;
     int32_t *n_b = (int32_t *)malloc(sizeof(int32_t) * (size_t)NB);
     uint8_t *is_source = (uint8_t *)malloc((size_t)NB);     /* per physical block, for the request at hand */
     if (!n_b || !is_source) { free(n_b); free(is_source); return VTO_EINVAL; }
@@ -608,20 +611,36 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
     memset(is_source, 0, (size_t)NB);
 
     int32_t consumed = 0, num_freed = 0, num_moves = 0, num_admitted = 0, num_deferred = 0, new_bt_fill = 0;
+    int32_t num_released = 0;
     int stop = 0;
     for (int32_t r = 0; r < R; ++r) {
         const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
         const int32_t b0 = bt_offsets[r], b1 = bt_offsets[r + 1];
         const int32_t nb = b1 - b0;
 
+        /* copy-on-write detach: does the request leave its shared blocks?  It does when its own live
+         * tokens fill less than detach_num / detach_den of them. */
+        int detach = 0;
+        if (may_detach) {
+            int64_t ns_shared = 0, n_shared = 0;
+            for (int32_t j = b0; j < b1; ++j) ns_shared += opts->protect[bt_blocks[j]] != 0;
+            for (int64_t t = t0; t < t1; ++t)
+                if (is_live(tt_slots, keep, t)) n_shared += opts->protect[tt_slots[t] / S] != 0;
+            detach = ns_shared > 0 &&
+                     (uint64_t)n_shared * opts->detach_den < (uint64_t)opts->detach_num * (uint64_t)ns_shared * (uint64_t)S;
+        }
+
         /* source blocks: unprotected, low utilisation, at most B of them in table order (Sec. 3.3.3) */
-        int32_t ns = 0;
+        int32_t ns = 0, ns_unprotected = 0;
         for (int32_t j = b0; j < b1; ++j) {
             const int32_t b = bt_blocks[j];
-            int eligible = !(opts->protect && opts->protect[b]);
+            const int shared = opts->protect && opts->protect[b];
+            int eligible = !shared;
             if (eligible && opts->util_den != 0)
                 eligible = (uint64_t)n_b[b] * opts->util_den < (uint64_t)opts->util_num * (uint64_t)S;
-            if (eligible && opts->max_source_blocks > 0 && ns >= opts->max_source_blocks) eligible = 0;
+            if (eligible && opts->max_source_blocks > 0 && ns_unprotected >= opts->max_source_blocks) eligible = 0;
+            ns_unprotected += eligible;
+            if (shared && detach) eligible = 1;             /* every shared block of a detaching request */
             is_source[b] = (uint8_t)eligible;
             ns += eligible;
         }
@@ -664,8 +683,12 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
             for (int32_t j = b0; j < b1; ++j)
                 if (!is_source[bt_blocks[j]]) new_bt_blocks[new_bt_fill++] = bt_blocks[j];
             for (int32_t j = 0; j < need; ++j) new_bt_blocks[new_bt_fill++] = dst[j];
-            for (int32_t j = b0; j < b1; ++j)
-                if (is_source[bt_blocks[j]]) freed_blocks[num_freed++] = bt_blocks[j];
+            for (int32_t j = b0; j < b1; ++j) {
+                const int32_t b = bt_blocks[j];
+                if (!is_source[b]) continue;
+                if (opts->protect && opts->protect[b]) released_blocks[num_released++] = b;   /* a reference less */
+                else freed_blocks[num_freed++] = b;
+            }
             consumed += need;
             ++num_admitted;
         } else {
@@ -683,6 +706,7 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
     counts->num_free_consumed = consumed;
     counts->num_admitted = num_admitted;
     counts->num_deferred = num_deferred;
+    counts->num_released = num_released;
     free(n_b); free(is_source);
     return VTO_OK;
 }
@@ -751,6 +775,7 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
     if (R < 0 || S < 1 || num_free < 0 || num_waves < 1 || !bt_offsets || !tt_offsets || !num_free_out ||
         !wave_move_offsets || !wave_counts)
         return VTO_EINVAL;
+    if (opts && opts->detach_den != 0) return VTO_EINVAL;   /* detach is an option of single plans */
     const int64_t T = tt_offsets[R], nbt = bt_offsets[R];
     const size_t nT = (size_t)(T > 0 ? T : 1), nB = (size_t)(nbt > 0 ? nbt : 1), nR = (size_t)R + 1;
     const size_t nP = (size_t)num_free + nB;
@@ -786,7 +811,7 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
         /* one planning round against the pool as it stands (Sec. 3.3.2 admission, 3.3.3 planning) */
         if (opts)
             rc = vto_plan_partial(R, S, NB, cur_bto, cur_btb, tt_offsets, cur_tts, keep, select, thr_num, thr_den,
-                                  pool, pool_n, opts, nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c);
+                                  pool, pool_n, opts, nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c, NULL);
         else
             rc = vto_plan(R, S, cur_bto, cur_btb, tt_offsets, cur_tts, keep, select, thr_num, thr_den, pool, pool_n,
                           nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c);

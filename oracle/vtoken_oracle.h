@@ -41,6 +41,7 @@ enum { VTO_NOT_SELECTED = 0, VTO_REPACKED = 1, VTO_NO_GAIN = 2, VTO_DEFERRED_NO_
 
 typedef struct {
     int32_t num_moves, num_dst_blocks, num_freed, num_free_consumed, num_admitted, num_deferred;
+    int32_t num_released;   /* references to shared blocks dropped by a copy-on-write detach (vto_plan_partial) */
 } vto_counts;
 
 /* Relocation planning + table rewrite for R requests.
@@ -220,6 +221,9 @@ typedef struct {
                                      unprotected block (whole-request compaction) */
     int32_t max_source_blocks;    /* B: at most this many sources per request, first in table order; 0 = no bound */
     uint32_t theta_num, theta_den;/* plan only when F > theta_num / theta_den; theta_den == 0: always */
+    uint32_t detach_num, detach_den; /* copy-on-write detach: a request leaves ALL its protected blocks when its own
+                                     live tokens in them fill less than detach_num / detach_den of those blocks;
+                                     detach_den == 0: never (protected blocks always stay) */
 } vto_partial_opts;
 
 /* Relocation planning that evacuates only low-utilisation source blocks (Sec. 3.3.3):
@@ -232,7 +236,17 @@ typedef struct {
  *     destination blocks; the reclaimed list receives its source blocks in old order;
  *   - when the global trigger F > theta does not hold, every request is VTO_NOT_SELECTED.
  * With util_den == 0, protect == NULL, B == 0 and theta_den == 0 the result equals vto_plan's.
- * NB = number of physical blocks (size of protect and of the internal n_b). */
+ * NB = number of physical blocks (size of protect and of the internal n_b).
+ *
+ * Copy-on-write detach (the paper's outlook for shared-prefix blocks, Sec. 5 "Compatibility with
+ * Prefix Caching" and Sec. 6: copy-on-write "when the expected reclamation benefit justifies the
+ * extra copy"): with detach_den != 0, a request whose own live tokens occupy less than
+ * detach_num / detach_den of its protected blocks (n_shared * den < num * ns_shared * S) treats all
+ * of them as sources too: its live tokens there are COPIED to its destinations with the rest (the
+ * shared blocks keep their bytes for the other holders), the blocks leave its table, and they are
+ * listed in released_blocks (references dropped; the caller's reference counts decide when such a
+ * block is free) instead of freed_blocks.  B bounds the unprotected sources only.  The gain gate
+ * is unchanged: destinations < sources, counted in the request's own table. */
 int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      const int32_t *bt_offsets, const int32_t *bt_blocks,
                      const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,
@@ -240,7 +254,7 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      const int32_t *free_blocks, int32_t num_free, const vto_partial_opts *opts,
                      int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
                      int32_t *freed_blocks, int32_t *req_status,
-                     int32_t *move_src, int32_t *move_dst, vto_counts *counts);
+                     int32_t *move_src, int32_t *move_dst, vto_counts *counts, int32_t *released_blocks);
 
 /* ---- online relocation check (Sec. 5, "Relocation Correctness") ---------------------------------
  * The paper hashes the ordered retained token ids together with their K/V contents before and

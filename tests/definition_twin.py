@@ -75,9 +75,11 @@ def to_csr(lists):
 
 
 def repack_partial_definition(S, block_tables, token_tables, keeps, free, select=None, thr=None, protect=(),
-                              util=None, max_sources=0, theta=None):
+                              util=None, max_sources=0, theta=None, detach=None):
     """Definition-level statement of the partial plan: only low-utilisation, unprotected blocks are
-    evacuated.  protect: set of block ids; util / theta: Fraction or None."""
+    evacuated.  protect: set of block ids; util / theta / detach: Fraction or None.  With ``detach`` a
+    request whose own live tokens fill less than that fraction of its protected blocks leaves all of
+    them (copy-on-write): they become sources too and are listed under ``released``."""
     R = len(token_tables)
     live = [[t for t, (s, k) in enumerate(zip(token_tables[r], keeps[r])) if s >= 0 and k] for r in range(R)]
     per_block = {}
@@ -91,14 +93,19 @@ def repack_partial_definition(S, block_tables, token_tables, keeps, free, select
     if theta is not None:
         triggered = allocated > 0 and 1 - Fraction(total_live, allocated * S) > theta
 
-    sources = []
+    sources, leaving = [], []
     for r in range(R):
         picked = []
         for b in block_tables[r]:
             ok = b not in protect and (util is None or Fraction(per_block.get(b, 0), S) < util)
             if ok and (max_sources == 0 or len(picked) < max_sources):
                 picked.append(b)
-        sources.append(picked)
+        shared = [b for b in block_tables[r] if b in protect]
+        mine_in_shared = sum(1 for t in live[r] if token_tables[r][t] // S in protect)
+        goes = detach is not None and shared and Fraction(mine_in_shared, len(shared) * S) < detach
+        leaving.append(set(shared) if goes else set())
+        # table order is kept: a source is an unprotected pick or a shared block of a leaving request
+        sources.append([b for b in block_tables[r] if b in set(picked) or b in leaving[r]])
     moving = [[t for t in live[r] if token_tables[r][t] // S in set(sources[r])] for r in range(R)]
     need = [-(-len(moving[r]) // S) for r in range(R)]
 
@@ -119,7 +126,7 @@ def repack_partial_definition(S, block_tables, token_tables, keeps, free, select
     status = [1 if r in admitted else 3 if r in deferred else 2 if chosen(r) else 0 for r in range(R)]
 
     cursor = 0
-    new_bt, new_tt, freed, moves = [], [], [], []
+    new_bt, new_tt, freed, released, moves = [], [], [], [], []
     for r in range(R):
         where = {t: token_tables[r][t] for t in live[r]}
         if r in admitted:
@@ -130,8 +137,10 @@ def repack_partial_definition(S, block_tables, token_tables, keeps, free, select
                 moves.append((token_tables[r][t], where[t]))
             src = set(sources[r])
             new_bt.append([b for b in block_tables[r] if b not in src] + list(mine))
-            freed.extend(b for b in block_tables[r] if b in src)
+            freed.extend(b for b in block_tables[r] if b in src and b not in leaving[r])
+            released.extend(b for b in block_tables[r] if b in leaving[r])
         else:
             new_bt.append(list(block_tables[r]))
         new_tt.append([where.get(t, -1) for t in range(len(token_tables[r]))])
-    return dict(new_bt=new_bt, new_tt=new_tt, freed=freed, status=status, moves=moves, consumed=cursor)
+    return dict(new_bt=new_bt, new_tt=new_tt, freed=freed, released=released, status=status, moves=moves,
+                consumed=cursor)

@@ -138,7 +138,7 @@ def test_source_bound_B_takes_the_first_eligible_blocks_in_table_order():
     assert vto.plan_partial(S, 10, [0, 5], bt, [0, 20], tt, keep, free, max_source_blocks=1).req_status.tolist() == [vto.NO_GAIN]
 
 
-def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB):
+def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB, detach=None):
     bt_off, bt_flat = to_csr(bts)
     tt_off, tt_flat = to_csr(tts)
     _, keep_flat = to_csr(keeps)
@@ -148,8 +148,9 @@ def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB)
     p = vto.plan_partial(S, NB, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free,
                          select=None if select is None else np.array(select, np.uint8),
                          thr_num=fr(thr)[0], thr_den=fr(thr)[1], protect=prot if protect else None,
-                         util=fr(util), max_source_blocks=B, theta=fr(theta))
-    d = repack_partial_definition(S, bts, tts, keeps, list(free), select, thr, set(protect), util, B, theta)
+                         util=fr(util), max_source_blocks=B, theta=fr(theta), detach=fr(detach))
+    d = repack_partial_definition(S, bts, tts, keeps, list(free), select, thr, set(protect), util, B, theta, detach)
+    assert p.released_blocks.tolist() == d["released"]
     nbo, nbf = to_csr(d["new_bt"])
     _, ntf = to_csr(d["new_tt"])
     assert p.new_bt_offsets.tolist() == nbo and p.new_bt_blocks.tolist() == nbf
@@ -221,3 +222,84 @@ def test_shared_prefix_blocks_are_skipped_and_private_suffixes_reclaimed():
         counts = np.bincount(occ, minlength=w.slots_per_layer)
         assert counts[np.isin(np.arange(w.slots_per_layer) // S, list(shared))].max() <= degree
         assert counts[~np.isin(np.arange(w.slots_per_layer) // S, list(shared))].max() <= 1
+
+
+# ---- copy-on-write detach from shared blocks --------------------------------------------------------
+def test_detach_bruteforce_against_the_definition_twin():
+    """Two requests sharing blocks 4 and 1 (protected), private blocks behind them; every keep mask
+    of a random sample, several detach thresholds, source bounds and pool sizes."""
+    rng = np.random.default_rng(5)
+    S = 2
+    bts = [[4, 1, 6, 2], [4, 1, 7, 3], [8]]
+    tts = [[8, 9, 2, 3, 12, -1, 4, 5], [8, 9, 2, 3, 14, 15, 6, -1], [16, 17]]
+    NB = 14
+    for _ in range(60):
+        keeps = [rng.integers(0, 2, len(t)).tolist() for t in tts]
+        for detach in (None, Fraction(1, 1), Fraction(1, 2), Fraction(3, 4), Fraction(1, 4)):
+            for util in (None, Fraction(1, 1)):
+                for B in (0, 1):
+                    for c in (0, 1, 2, 5):
+                        _compare(S, bts, tts, keeps, np.array([9, 5, 10, 11, 12][:c], np.int32), None, None, (4, 1),
+                                 util, B, None, NB, detach)
+
+
+def test_detach_threshold_is_strict_and_counts_the_requests_own_tokens():
+    """S = 4, two shared blocks (8 slots): the request keeps 4 of its 8 prefix tokens.  It leaves the
+    prefix for thresholds above 1/2 and stays at exactly 1/2; the other sharer's tokens do not count."""
+    S = 4
+    bts = [[0, 1, 5], [0, 1, 6]]
+    tts = [[0, 1, 2, 3, 4, 5, 6, 7, 20, 21], [0, 1, 2, 3, 4, 5, 6, 7, 24]]
+    keeps = [[1, 0, 1, 0, 1, 0, 1, 0, 1, 1], [1] * 9]
+    bt_off, bt_flat = to_csr(bts)
+    tt_off, tt_flat = to_csr(tts)
+    _, keep_flat = to_csr(keeps)
+    protect = np.zeros(10, np.uint8)
+    protect[[0, 1]] = 1
+    free = np.array([7, 8, 9], np.int32)
+    run = lambda d: vto.plan_partial(S, 10, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free, protect=protect,
+                                     util=(1, 1), detach=d)
+    stay = run((1, 2))
+    assert stay.released_blocks.tolist() == [] and stay.req_status.tolist() == [vto.NO_GAIN, vto.NO_GAIN]
+    go = run((5, 8))
+    # request 0: sources = shared 0, 1 and private 5 (2 of 4 live) -> 6 tokens -> 2 destinations < 3 sources
+    assert go.req_status.tolist() == [vto.REPACKED, vto.NO_GAIN]
+    assert go.released_blocks.tolist() == [0, 1] and go.freed_blocks.tolist() == [5]
+    assert go.new_bt_blocks.tolist() == [7, 8, 0, 1, 6]
+    assert go.new_tt_slots[:10].tolist() == [28, -1, 29, -1, 30, -1, 31, -1, 32, 33]
+    assert go.new_tt_slots[10:].tolist() == tts[1]                         # the other sharer is untouched
+    assert sorted(go.move_src.tolist()) == [0, 2, 4, 6, 20, 21]            # copies out of the shared blocks too
+
+
+@pytest.mark.parametrize("degree", [1, 2, 4])
+def test_detach_on_the_shared_prefix_workload(degree):
+    """Every request of the prefix-cache workload leaves its shared prefix (H2O keeps about a fifth of
+    it): its table shrinks to ceil(live / S), the prefix blocks are released once per sharer and never
+    put on the free list or written to, and every request still sees exactly its own tokens."""
+    w, protect = wl.shared_prefix(seed=degree, groups=2, degree=degree, prefix_len=64, suffix_len=96, layers=1,
+                                  heads=1, head_dim=8, block_size=4)
+    S = w.block_size
+    p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
+                         protect=protect, detach=(1, 1))
+    shared = set(np.flatnonzero(protect).tolist())
+    live = (w.tt_slots >= 0) & (w.keep != 0)
+    assert p.num_admitted == w.num_requests
+    assert not (set(p.freed_blocks.tolist()) & shared) and not (set((p.move_dst // S).tolist()) & shared)
+    assert sorted(np.bincount(p.released_blocks, minlength=w.num_blocks)[sorted(shared)].tolist()) == \
+           [degree] * len(shared)
+    slab = np.arange(w.slots_per_layer * 2, dtype=np.int64).reshape(-1, 2)
+    before = slab.copy()
+    vto.apply_moves_slab(slab, p.move_src, p.move_dst)
+    shared_rows = np.isin(np.arange(w.slots_per_layer) // S, sorted(shared))
+    assert np.array_equal(slab[shared_rows], before[shared_rows])            # the shared blocks keep their bytes
+    for r in range(w.num_requests):
+        t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
+        new = p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]]
+        assert len(new) == -(-int(live[t0:t1].sum()) // S) and not (set(new.tolist()) & shared)
+        assert np.array_equal(vto.gather_logical(before, w.tt_slots[t0:t1], w.keep[t0:t1]),
+                              vto.gather_logical(slab, p.new_tt_slots[t0:t1]))
+    occ = p.new_tt_slots[p.new_tt_slots >= 0]
+    assert np.bincount(occ).max() == 1                                       # every slot is private now
+    # without detach the result is the conservative one of the paper's Table 1
+    q = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
+                         protect=protect)
+    assert q.released_blocks.tolist() == [] and len(q.new_bt_blocks) > len(p.new_bt_blocks)

@@ -139,7 +139,7 @@ typedef struct {
     int32_t num_admitted;          /* requests with status VTOKEN_REPACKED */
     int32_t num_deferred;          /* requests with status VTOKEN_DEFERRED_NO_FREE */
     uint32_t error_flags;          /* VTOKEN_FLAG_* */
-    uint32_t reserved;
+    int32_t num_released;          /* entries of released_blocks (copy-on-write detach of vtoken_plan_partial) */
 } vtoken_counts;
 
 typedef struct {                   /* all DEVICE pointers, written by vtoken_plan */
@@ -149,6 +149,8 @@ typedef struct {                   /* all DEVICE pointers, written by vtoken_pla
     int32_t *freed_blocks;         /* capacity max_table_blocks */
     int32_t *req_status;           /* [R] VTOKEN_NOT_SELECTED .. VTOKEN_DEFERRED_NO_FREE */
     vtoken_counts *counts;         /* one struct */
+    int32_t *released_blocks;      /* capacity max_table_blocks; only vtoken_plan_partial with a detach threshold
+                                      writes it (may be NULL otherwise) */
 } vtoken_plan_out;
 
 /* Relocation planning and table rewrite (Sec. 3.3.3; apply_moves of Sec. 3.2; I1, I2, I4).
@@ -235,6 +237,9 @@ typedef struct {
                                       block-table order; 0 = no bound */
     uint32_t theta_num, theta_den; /* global trigger: plan only when F > theta_num / theta_den (64-bit integers);
                                       theta_den == 0: always */
+    uint32_t detach_num, detach_den; /* copy-on-write detach: a request leaves ALL its protected blocks when its own
+                                      live tokens in them fill less than detach_num / detach_den of those blocks
+                                      (n_shared * den < num * ns_shared * S); detach_den == 0: never */
 } vtoken_partial_opts;
 
 /* vtoken_plan restricted to source blocks.  Differences from vtoken_plan: only live tokens stored
@@ -243,7 +248,19 @@ typedef struct {
  * other blocks keep their slots; new block table = the non-source blocks in old order followed by
  * the destinations; freed_blocks receives the source blocks in old order; when the trigger does
  * not hold every request is VTOKEN_NOT_SELECTED.  With all options zero / NULL the result equals
- * vtoken_plan's.  vtoken_repack executes the plan. */
+ * vtoken_plan's.  vtoken_repack executes the plan.
+ *
+ * Copy-on-write detach (the paper's outlook for shared-prefix blocks, Sec. 5 and Sec. 6: copy-on-write
+ * "when the expected reclamation benefit justifies the extra copy").  With a protect mask and
+ * detach_den != 0, a request whose own live tokens occupy less than detach_num / detach_den of its
+ * protected blocks treats all of them as sources too: its live tokens there are COPIED to its
+ * destinations with the rest (the shared blocks keep their bytes for the other holders), the blocks
+ * leave its table and are listed in out->released_blocks (a reference dropped; the caller's
+ * reference counts decide when such a block is free) instead of freed_blocks; counts.num_released
+ * says how many.  max_source_blocks bounds the unprotected sources only.  The gain gate is unchanged
+ * (destinations < sources, in the request's own table), so whether the POOL gains depends on the
+ * other holders: enabling detach is the caller's policy decision.  Not available in
+ * vtoken_repack_waves and vtoken_repack_host_partial (VTOKEN_EINVAL). */
 int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
                         const vtoken_plan_out *out, void *cuda_stream);
 

@@ -57,21 +57,22 @@ class PlanIn(ctypes.Structure):
 class Counts(ctypes.Structure):
     _fields_ = [("num_moves", ctypes.c_int32), ("num_dst_blocks", ctypes.c_int32), ("num_freed", ctypes.c_int32),
                 ("num_free_consumed", ctypes.c_int32), ("num_admitted", ctypes.c_int32),
-                ("num_deferred", ctypes.c_int32), ("error_flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("num_deferred", ctypes.c_int32), ("error_flags", ctypes.c_uint32), ("num_released", ctypes.c_int32)]
 
     def as_dict(self):
-        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+        return {n: getattr(self, n) for n, _ in self._fields_}
 
 
 class PlanOut(ctypes.Structure):
     _fields_ = [("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
                 ("new_tt_slots", ctypes.c_void_p), ("freed_blocks", ctypes.c_void_p),
-                ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p)]
+                ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p), ("released_blocks", ctypes.c_void_p)]
 
 
 class PartialOpts(ctypes.Structure):
     _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
-                ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32)]
+                ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32),
+                ("detach_num", ctypes.c_uint32), ("detach_den", ctypes.c_uint32)]
 
 
 class WavesOut(ctypes.Structure):
@@ -377,12 +378,12 @@ def vtoken_block_liveness(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offset
 def vtoken_plan_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
                         new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status, counts, select=None,
                         thr_num=0, thr_den=0, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
-                        stream=None) -> None:
+                        detach=(0, 0), released_blocks=None, stream=None) -> None:
     pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                  _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
     pout = PlanOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks),
-                   _ptr(req_status), _ptr(counts))
-    po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1])
+                   _ptr(req_status), _ptr(counts), _ptr(released_blocks))
+    po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1], detach[0], detach[1])
     _check(load().vtoken_plan_partial(ctx, ctypes.byref(pin), ctypes.byref(po), ctypes.byref(pout), _stream(stream)),
            "vtoken_plan_partial", ctx)
 
@@ -413,7 +414,8 @@ def vtoken_repack_waves(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets,
     po = None
     if partial is not None:
         util, theta = partial.get("util", (0, 0)), partial.get("theta", (0, 0))
+        detach = partial.get("detach", (0, 0))
         po = ctypes.byref(PartialOpts(_ptr(partial.get("protect")), util[0], util[1],
-                                      partial.get("max_source_blocks", 0), theta[0], theta[1]))
+                                      partial.get("max_source_blocks", 0), theta[0], theta[1], detach[0], detach[1]))
     _check(load().vtoken_repack_waves(ctx, ctypes.byref(pin), po, num_waves, ctypes.byref(wout), _stream(stream)),
            "vtoken_repack_waves", ctx)

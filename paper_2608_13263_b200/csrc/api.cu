@@ -25,7 +25,8 @@ void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
-                    ctx->n_b, ctx->blk_src, ctx->slot_bits,
+                    ctx->n_b, ctx->blk_src, ctx->slot_bits, ctx->part_shared, ctx->req_shared, ctx->req_detach,
+                    ctx->req_rel_base,
                     ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
                     ctx->stage.select, ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
@@ -131,6 +132,10 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->n_b, cfg->num_blocks);
     A(&ctx->blk_src, cfg->num_blocks);
     A(&ctx->slot_bits, (slots + 31) / 32);
+    A(&ctx->part_shared, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
+    A(&ctx->req_shared, cfg->max_requests);
+    A(&ctx->req_detach, cfg->max_requests);
+    A(&ctx->req_rel_base, cfg->max_requests);
     if (rc == VTOKEN_OK && cudaMemset(ctx->counts, 0, sizeof(vtoken_counts)) != cudaSuccess) rc = VTOKEN_ECUDA;
     if (rc == VTOKEN_OK) rc = vtk_configure_copy(ctx);
     if (rc != VTOKEN_OK) { free_all(ctx); delete ctx; return rc; }
@@ -244,6 +249,8 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
     out.freed_blocks = s.freed_blocks;
     out.req_status = s.req_status;
     out.counts = s.counts;
+    out.released_blocks = nullptr;
+    if (opts && opts->detach_den != 0) return VTOKEN_EINVAL;    // the host front end has no released list
     if (opts) {
         vtoken_partial_opts dopts = *opts;
         dopts.protect = opts->protect ? s.protect : nullptr;

@@ -36,6 +36,10 @@ struct vtoken_ctx {
     int32_t *req_nsrc;         // [max_requests] live tokens in its source blocks
     int32_t *n_b;              // [num_blocks] live tokens per physical block
     uint8_t *blk_src;          // [num_blocks] 1 = the block is a source of its request
+    int32_t *part_shared;      // [max_requests * VTK_PLAN_PARTS] live tokens in protected blocks per request part
+    int32_t *req_shared;       // [max_requests] protected entries of the request's block table
+    int32_t *req_detach;       // [max_requests] 1 = the request leaves its protected blocks (copy-on-write detach)
+    int32_t *req_rel_base;     // [max_requests] first entry in released_blocks
     uint32_t *slot_bits;       // [ceil(num_blocks * S / 32)] one bit per slot (vtoken_check_tables)
 
     // gather_logical scratch (DEVICE)

@@ -195,7 +195,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         c.num_admitted = carry.admitted;
         c.num_deferred = carry.deferred;
         c.error_flags = flags | a.counts->error_flags;   // bits raised by the count kernel
-        c.reserved = 0;
+        c.num_released = 0;
         *a.counts = c;
         *a.out_counts = c;                               // later flags are OR-ed into both copies
     }

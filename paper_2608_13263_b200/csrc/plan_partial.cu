@@ -15,6 +15,12 @@
 //             (kept blocks in old order, then destinations), reclaimed list, inverse move plan
 // The inverse plan has the same form as the whole-request planner's, so vtoken_repack runs it
 // unchanged.
+//
+// Copy-on-write detach (optional): a request whose own live tokens fill too little of its
+// protected (shared) blocks leaves all of them -- they become sources for this request only, its
+// tokens there are copied out with the rest, and the blocks are listed as released references
+// instead of reclaimed blocks.  "Source" is therefore a per-request notion for protected blocks
+// (req_detach[r]) and a per-block one (blk_src[b]) for the others.
 #include "common.cuh"
 
 #include <cstring>
@@ -28,12 +34,13 @@ constexpr int PP_SCAN_NT = 1024;
 struct PArgs {
     const int32_t *num_requests, *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
     const uint8_t *keep, *select, *protect;
-    uint32_t thr_num, thr_den, util_num, util_den, theta_num, theta_den;
+    uint32_t thr_num, thr_den, util_num, util_den, theta_num, theta_den, detach_num, detach_den;
     int32_t max_sources;
     const int32_t *free_blocks, *num_free;
-    int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *out_status;
+    int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *released_blocks, *out_status;
     vtoken_counts *out_counts;
     int32_t *req_n, *part_n, *part_src, *req_ns, *req_nsrc, *req_dst_base, *req_freed_base, *req_status;
+    int32_t *part_shared, *req_shared, *req_detach, *req_rel_base;
     int32_t *dst_src, *dst_blocks, *n_b;
     uint8_t *blk_src;
     vtoken_counts *counts;
@@ -70,7 +77,15 @@ __device__ __forceinline__ int pp_block_sum(int n, int *warp_n)
 }
 
 // ---- live: part counts and per-block liveness -----------------------------------------------
-// mode 0: count live tokens and add them to n_b; mode 1: count live tokens whose block is a source
+// does a live token of request r in block b move?  (b is a source of its request, or r leaves its
+// protected blocks and b is one of them)
+__device__ __forceinline__ bool pp_moves(const PArgs &a, bool detach, int32_t b)
+{
+    return a.blk_src[b] != 0 || (detach && a.protect[b] != 0);
+}
+
+// mode 0: count live tokens and add them to n_b (and, when a detach threshold is set, count the
+// ones in protected blocks); mode 1: count live tokens that move
 template <int MODE>
 __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
 {
@@ -79,7 +94,9 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
     if (r >= pp_requests(a)) return;
     int64_t p0, p1;
     pp_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
-    int n = 0;
+    const bool may_detach = a.protect != nullptr && a.detach_den != 0;
+    const bool detach = MODE == 1 && may_detach && a.req_detach[r] != 0;
+    int n = 0, n_shared = 0;
     bool bad = false;
     for (int64_t t = p0 + threadIdx.x; t < p1; t += PP_NT) {
         const int32_t slot = a.tt_slots[t];
@@ -87,13 +104,19 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
         if (MODE == 0) {
             atomicAdd(&a.n_b[slot / a.S], 1);
             ++n;
+            if (may_detach) n_shared += a.protect[slot / a.S] != 0;
         } else {
-            n += a.blk_src[slot / a.S];
+            n += pp_moves(a, detach, slot / a.S);
         }
     }
     if (bad && MODE == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
     const int s = pp_block_sum(n, warp_n);
     if (threadIdx.x == 0) (MODE == 0 ? a.part_n : a.part_src)[blockIdx.x] = s;
+    if (MODE == 0 && may_detach) {
+        __syncthreads();                       // warp_n is reused
+        const int sh = pp_block_sum(n_shared, warp_n);
+        if (threadIdx.x == 0) a.part_shared[blockIdx.x] = sh;
+    }
 }
 
 // ---- blocks: source selection per request ------------------------------------------------------
@@ -104,6 +127,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
     if (r >= pp_requests(a)) return;
     const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
     int carry = 0;               // eligible entries before this chunk
+    int shared = 0;              // protected entries seen by this thread
     uint32_t flags = 0;
     for (int jb = b0; jb < b1; jb += PP_NT) {
         const int j = jb + threadIdx.x;
@@ -116,6 +140,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
                 blk = -1;
             } else {
                 eligible = !(a.protect != nullptr && a.protect[blk] != 0);
+                shared += !eligible;
                 if (eligible && a.util_den != 0)
                     eligible = (unsigned long long)a.n_b[blk] * a.util_den <
                                (unsigned long long)a.util_num * (unsigned long long)a.S;
@@ -126,24 +151,42 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
         carry += total;
         if (eligible && (a.max_sources <= 0 || rank < a.max_sources)) a.blk_src[blk] = 1;
     }
-    if (threadIdx.x == 0) a.req_ns[r] = (a.max_sources > 0 && carry > a.max_sources) ? a.max_sources : carry;
+    int ns = (a.max_sources > 0 && carry > a.max_sources) ? a.max_sources : carry;
+    if (a.protect != nullptr && a.detach_den != 0) {
+        // copy-on-write detach: the request leaves its protected blocks when its own live tokens
+        // fill less than detach_num / detach_den of them; then every one of them is a source
+        __syncthreads();
+        const int ns_shared = pp_block_sum(shared, warp_sums);          // valid in thread 0
+        if (threadIdx.x == 0) {
+            long long n_shared = 0;
+            for (int c = 0; c < PP_PARTS; ++c) n_shared += a.part_shared[r * PP_PARTS + c];
+            const bool detach = ns_shared > 0 &&
+                                (unsigned long long)n_shared * a.detach_den <
+                                    (unsigned long long)a.detach_num * (unsigned long long)ns_shared * (unsigned long long)a.S;
+            a.req_detach[r] = detach ? 1 : 0;
+            a.req_shared[r] = detach ? ns_shared : 0;
+            ns += detach ? ns_shared : 0;
+        }
+    }
+    if (threadIdx.x == 0) a.req_ns[r] = ns;
     if (flags) atomicOr(&a.counts->error_flags, flags);
 }
 
 // ---- scan ----------------------------------------------------------------------------------------
 struct PAcc {
-    int dst, freed, newbt, moves, admitted, deferred;
+    int dst, freed, newbt, moves, admitted, deferred, released;
 };
 __device__ __forceinline__ PAcc operator+(const PAcc &x, const PAcc &y)
 {
     return PAcc{x.dst + y.dst, x.freed + y.freed, x.newbt + y.newbt, x.moves + y.moves, x.admitted + y.admitted,
-                x.deferred + y.deferred};
+                x.deferred + y.deferred, x.released + y.released};
 }
 __device__ __forceinline__ PAcc pp_shfl_up(const PAcc &v, int d)
 {
     return PAcc{__shfl_up_sync(0xffffffffu, v.dst, d),      __shfl_up_sync(0xffffffffu, v.freed, d),
                 __shfl_up_sync(0xffffffffu, v.newbt, d),    __shfl_up_sync(0xffffffffu, v.moves, d),
-                __shfl_up_sync(0xffffffffu, v.admitted, d), __shfl_up_sync(0xffffffffu, v.deferred, d)};
+                __shfl_up_sync(0xffffffffu, v.admitted, d), __shfl_up_sync(0xffffffffu, v.deferred, d),
+                __shfl_up_sync(0xffffffffu, v.released, d)};
 }
 template <typename T, typename ShflUp>
 __device__ __forceinline__ T pp_block_incl_scan(T v, T *warp_tot, T zero, ShflUp shfl)
@@ -188,7 +231,7 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         carry_need = 0;
         tot_live = 0;
         tot_blocks = 0;
-        carry = PAcc{0, 0, 0, 0, 0, 0};
+        carry = PAcc{0, 0, 0, 0, 0, 0, 0};
     }
     int nf = *a.num_free;
     if (nf > a.max_free_blocks && tid == 0) flags |= VTOKEN_FLAG_CAPACITY;
@@ -227,11 +270,13 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     for (int base = 0; base < R; base += PP_SCAN_NT) {
         const int r = base + tid;
         const bool valid = r < R;
-        int n = 0, nsrc = 0, nb = 0, ns = 0;
+        const bool may_detach = a.protect != nullptr && a.detach_den != 0;
+        int n = 0, nsrc = 0, nb = 0, ns = 0, nrel = 0;
         if (valid) {
             n = a.req_n[r];
             nsrc = a.req_nsrc[r];
             ns = a.req_ns[r];
+            nrel = may_detach ? a.req_shared[r] : 0;     // protected sources: released, not reclaimed
             nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
             if (nb < 0) nb = 0;
         }
@@ -245,12 +290,13 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         const bool adm = cand && cum <= (long long)nf;
         const int status = !sel ? VTOKEN_NOT_SELECTED
                                 : (!cand ? VTOKEN_NO_GAIN : (adm ? VTOKEN_REPACKED : VTOKEN_DEFERRED_NO_FREE));
-        PAcc mine{adm ? need : 0, adm ? ns : 0, valid ? (adm ? nb - ns + need : nb) : 0, adm ? nsrc : 0, adm ? 1 : 0,
-                  (cand && !adm) ? 1 : 0};
-        const PAcc incl = pp_block_incl_scan<PAcc>(mine, warp_acc, PAcc{0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
+        PAcc mine{adm ? need : 0, adm ? ns - nrel : 0, valid ? (adm ? nb - ns + need : nb) : 0, adm ? nsrc : 0,
+                  adm ? 1 : 0, (cand && !adm) ? 1 : 0, adm ? nrel : 0};
+        const PAcc incl = pp_block_incl_scan<PAcc>(mine, warp_acc, PAcc{0, 0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
         if (valid) {
             a.req_dst_base[r] = incl.dst - mine.dst;
             a.req_freed_base[r] = incl.freed - mine.freed;
+            a.req_rel_base[r] = incl.released - mine.released;
             a.new_bt_offsets[r] = incl.newbt - mine.newbt;
             a.req_status[r] = status;
             a.out_status[r] = status;
@@ -272,7 +318,7 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         c.num_admitted = carry.admitted;
         c.num_deferred = carry.deferred;
         c.error_flags = flags | a.counts->error_flags;
-        c.reserved = 0;
+        c.num_released = carry.released;
         *a.counts = c;
         *a.out_counts = c;
     }
@@ -290,6 +336,7 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
     const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
     const int nb = b1 - b0;
     const bool adm = a.req_status[r] == VTOKEN_REPACKED;
+    const bool detach = adm && a.protect != nullptr && a.detach_den != 0 && a.req_detach[r] != 0;
     const int nsrc = a.req_nsrc[r], ns = a.req_ns[r];
     const int need = (int)(((int64_t)nsrc + S - 1) / S);
     const int dst_base = a.req_dst_base[r];
@@ -306,24 +353,35 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
             a.dst_blocks[dst_base + j] = blk;
         }
         for (int i = nsrc + stripe; i < need * S; i += stride) a.dst_src[(int64_t)dst_base * S + i] = -1;
-        // kept blocks in old order, sources to the reclaimed list in old order: one CTA ranks the table
+        // kept blocks in old order, unprotected sources to the reclaimed list and protected sources (of a
+        // detaching request) to the released list, each in old order: one CTA ranks the table
         if (c == 0) {
             const int f0 = a.req_freed_base[r];
-            int carry_src = 0;
+            const int l0 = detach ? a.req_rel_base[r] : 0;
+            int carry_src = 0, carry_rel = 0;
             for (int jb = b0; jb < b1; jb += PP_NT) {
                 const int j = jb + tid;
                 int blk = -1;
-                bool src = false;
+                bool src = false, rel = false;
                 if (j < b1) {
                     blk = a.bt_blocks[j];
-                    src = blk >= 0 && blk < a.num_blocks && a.blk_src[blk] != 0;
+                    if (blk >= 0 && blk < a.num_blocks) {
+                        src = a.blk_src[blk] != 0;
+                        rel = detach && a.protect[blk] != 0;
+                    }
                 }
                 int total;
                 const int rank_src = carry_src + vtk_block_rank<PP_NT>(src, warp_sums, total);
                 carry_src += total;
+                int rank_rel = 0;
+                if (detach) {                                   // uniform over the CTA
+                    rank_rel = carry_rel + vtk_block_rank<PP_NT>(rel, warp_sums, total);
+                    carry_rel += total;
+                }
                 if (j < b1) {
                     if (src) a.freed_blocks[f0 + rank_src] = blk;
-                    else a.new_bt_blocks[nbt0 + (j - b0) - rank_src] = blk;   // kept entries before it = all - sources
+                    else if (rel) a.released_blocks[l0 + rank_rel] = blk;
+                    else a.new_bt_blocks[nbt0 + (j - b0) - rank_src - rank_rel] = blk;   // entries before it that stay
                 }
             }
         }
@@ -343,7 +401,7 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
         if (t < p1) {
             slot = a.tt_slots[t];
             live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
-            moving = live && adm && a.blk_src[slot / S] != 0;
+            moving = live && adm && pp_moves(a, detach, slot / S);
         }
         int total;
         const int i = carry + vtk_block_rank<PP_NT>(moving, warp_sums, total);
@@ -417,6 +475,10 @@ void fill_args(PArgs &a, vtoken_ctx *ctx)
     a.dst_blocks = ctx->dst_blocks;
     a.n_b = ctx->n_b;
     a.blk_src = ctx->blk_src;
+    a.part_shared = ctx->part_shared;
+    a.req_shared = ctx->req_shared;
+    a.req_detach = ctx->req_detach;
+    a.req_rel_base = ctx->req_rel_base;
     a.counts = ctx->counts;
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
@@ -443,6 +505,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         !out->req_status || !out->counts)
         return VTOKEN_EINVAL;
     if (opts->max_source_blocks < 0) return VTOKEN_EINVAL;
+    if (opts->protect != nullptr && opts->detach_den != 0 && !out->released_blocks) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     PArgs a;
     fill_args(a, ctx);
@@ -460,6 +523,8 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     a.util_den = opts->util_den;
     a.theta_num = opts->theta_num;
     a.theta_den = opts->theta_den;
+    a.detach_num = opts->detach_num;
+    a.detach_den = opts->detach_den;
     a.max_sources = opts->max_source_blocks;
     a.free_blocks = in->free_blocks;
     a.num_free = in->num_free;
@@ -467,6 +532,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     a.new_bt_blocks = out->new_bt_blocks;
     a.new_tt_slots = out->new_tt_slots;
     a.freed_blocks = out->freed_blocks;
+    a.released_blocks = out->released_blocks;
     a.out_status = out->req_status;
     a.out_counts = out->counts;
 

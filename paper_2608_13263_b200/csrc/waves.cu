@@ -113,6 +113,7 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         !out->free_out || !out->num_free_out || !out->wave_counts || !out->workspace)
         return VTOKEN_EINVAL;
     if (out->free_capacity < 0 || ((uintptr_t)out->workspace & 15)) return VTOKEN_EINVAL;
+    if (opts && opts->detach_den != 0) return VTOKEN_EINVAL;     // detach is an option of single plans
     if (out->free_capacity > ctx->cfg.max_free_blocks) return VTOKEN_ECAPACITY;
     const Layout l = layout_of(ctx, out->free_capacity);
     if (out->workspace_bytes < l.total) return VTOKEN_ECAPACITY;
@@ -137,6 +138,7 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         po.freed_blocks = at(l.freed);
         po.req_status = at(l.status);
         po.counts = out->wave_counts + k;
+        po.released_blocks = nullptr;
         int rc = opts ? vtoken_plan_partial(ctx, &cur, opts, &po, cuda_stream) : vtoken_plan(ctx, &cur, &po, cuda_stream);
         if (rc != VTOKEN_OK) return rc;
         rc = vtk_launch_copy(ctx, st);

@@ -52,6 +52,7 @@ class DeviceProblem:
         self.new_bt_blocks = torch.full((self.max_table_blocks,), -9, **i32)
         self.new_tt_slots = torch.full((self.max_tokens,), -9, **i32)
         self.freed_blocks = torch.full((self.max_table_blocks,), -9, **i32)
+        self.released_blocks = torch.full((self.max_table_blocks,), -9, **i32)
         self.req_status = torch.full((self.max_requests,), -9, **i32)
         self.counts = torch.zeros(8, **i32)
 
@@ -107,7 +108,8 @@ class DeviceProblem:
                        counts=self.counts, select=self.select, thr_num=self.w.thr_num, thr_den=self.w.thr_den,
                        stream=stream)
 
-    def plan_partial(self, stream=None, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0)):
+    def plan_partial(self, stream=None, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
+                     detach=(0, 0)):
         vt.vtoken_plan_partial(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
                                bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
                                keep=self.keep, free_blocks=self.free_blocks,
@@ -116,7 +118,8 @@ class DeviceProblem:
                                new_tt_slots=self.new_tt_slots, freed_blocks=self.freed_blocks,
                                req_status=self.req_status, counts=self.counts, select=self.select,
                                thr_num=self.w.thr_num, thr_den=self.w.thr_den, protect=protect, util=util,
-                               max_source_blocks=max_source_blocks, theta=theta, stream=stream)
+                               max_source_blocks=max_source_blocks, theta=theta, detach=detach,
+                               released_blocks=self.released_blocks, stream=stream)
 
     def repack(self, stream=None):
         vt.vtoken_repack(self.ctx, stream=stream)
@@ -177,6 +180,8 @@ class DeviceProblem:
         names = ["num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"]
         out = {n: int(c[i]) for i, n in enumerate(names)}
         out["error_flags"] = int(np.uint32(c[6]))
+        out["num_released"] = int(c[7])
+        out["released_blocks"] = self.released_blocks.cpu().numpy()[:out["num_released"]]
         nbo = self.new_bt_offsets.cpu().numpy()[:R + 1]
         out["new_bt_offsets"] = nbo
         out["new_bt_blocks"] = self.new_bt_blocks.cpu().numpy()[:int(nbo[R]) if R >= 0 else 0]

@@ -36,7 +36,7 @@ def random_problem(rng):
     return w
 
 
-@pytest.mark.parametrize("seed", range(40))
+@pytest.mark.parametrize("seed", range(60))
 def test_fuzz_whole_and_partial_plans(seed):
     import torch
     from paper_2608_13263_b200.device import DeviceProblem
@@ -52,6 +52,8 @@ def test_fuzz_whole_and_partial_plans(seed):
                     theta=[(0, 0), (1, 4), (9, 10)][int(rng.integers(0, 3))])
         if rng.random() < 0.4:
             opts["protect"] = (rng.random(w.num_blocks) < 0.2).astype(np.uint8)
+            if rng.random() < 0.6:
+                opts["detach"] = [(1, 1), (1, 2), (3, 4)][int(rng.integers(0, 3))]
     variant = int(rng.choice([0, 1, 2])) if w.row_bytes >= 16 else 1
     prob = DeviceProblem(w, fill_seed=seed, copy_variant=variant)
     nf_dev = None if num_free is None else torch.tensor([num_free], dtype=torch.int32, device=prob.device)
@@ -75,6 +77,8 @@ def test_fuzz_whole_and_partial_plans(seed):
     assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
     assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
     assert np.array_equal(out["freed_blocks"], p.freed_blocks)
+    if partial:
+        assert np.array_equal(out["released_blocks"], p.released_blocks)
     k = np.stack([wl.fill_slab(seed, 0, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
     v = np.stack([wl.fill_slab(seed, 1, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
     vto.apply_moves_pools(k, v, p.move_src, p.move_dst)

@@ -230,3 +230,62 @@ def test_repack_host_partial_entry_point(opts):
     with pytest.raises(vt.VtokenError):
         vt._check(vt.load().vtoken_repack_host_partial(prob.ctx, None, None, None), "null arguments")
     prob.close()
+
+
+@pytest.mark.parametrize("detach", [(1, 1), (1, 2), (1, 4), (1, 100)], ids=lambda d: f"detach{d[0]}_{d[1]}")
+@pytest.mark.parametrize("degree", [1, 2, 4, 8])
+def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach):
+    """Requests leave their shared prefix when their own tokens fill too little of it: tables, the
+    reclaimed and the released lists, counts and whole pools against the oracle; the shared blocks
+    keep their bytes."""
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    w, protect = wl.shared_prefix(seed=10 + degree, groups=2, degree=degree, prefix_len=256, suffix_len=320, layers=2,
+                                  heads=2, head_dim=64)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    prob.plan_partial(protect=torch.from_numpy(protect).to(prob.device), util=(1, 1), detach=detach)
+    prob.repack()
+    out = prob.outputs()
+    p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                         w.free_blocks, protect=protect, util=(1, 1), detach=detach)
+    assert out["error_flags"] == 0
+    for n in ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"):
+        assert out[n] == getattr(p, n), n
+    assert out["num_released"] == len(p.released_blocks)
+    assert np.array_equal(out["released_blocks"], p.released_blocks)
+    assert np.array_equal(out["req_status"], p.req_status)
+    assert np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
+    assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
+    assert np.array_equal(out["freed_blocks"], p.freed_blocks)
+    if detach == (1, 1):
+        assert out["num_released"] == degree * 2 * w.notes["prefix_blocks"]       # every sharer left every prefix block
+    if detach == (1, 100):
+        assert out["num_released"] == 0                                           # nobody is that sparse
+    k, v = host_pools(w)
+    k0 = k.copy()
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    shared_rows = np.isin(np.arange(w.slots_per_layer) // w.block_size, np.flatnonzero(protect))
+    assert np.array_equal(k[:, shared_rows], k0[:, shared_rows])
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()
+
+
+def test_detach_needs_a_released_list_and_is_refused_by_the_composite_entry_points():
+    import torch
+    from paper_2608_13263_b200.device import DeviceProblem
+    w, protect = wl.shared_prefix(seed=3, groups=1, degree=2, prefix_len=64, suffix_len=80, layers=1, heads=1,
+                                  head_dim=8)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, wave_capacity=True)
+    prot = torch.from_numpy(protect).to(prob.device)
+    saved = prob.released_blocks
+    prob.released_blocks = None
+    with pytest.raises(vt.VtokenError) as e:
+        prob.plan_partial(protect=prot, detach=(1, 1))
+    assert e.value.code == vt.EINVAL
+    prob.released_blocks = saved
+    with pytest.raises(vt.VtokenError) as e:
+        prob.repack_waves(2, partial=dict(protect=prot, detach=(1, 1)))
+    assert e.value.code == vt.EINVAL
+    prob.close()

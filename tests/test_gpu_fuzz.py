@@ -56,6 +56,8 @@ def test_fuzz_whole_and_partial_plans(seed):
                 opts["detach"] = [(1, 1), (1, 2), (3, 4)][int(rng.integers(0, 3))]
     variant = int(rng.choice([0, 1, 2])) if w.row_bytes >= 16 else 1
     prob = DeviceProblem(w, fill_seed=seed, copy_variant=variant)
+    from paper_2608_13263_b200 import binding as vt
+    before = _digest(prob, vt, prob.tt_slots, prob.keep) if w.row_bytes % 16 == 0 else None
     nf_dev = None if num_free is None else torch.tensor([num_free], dtype=torch.int32, device=prob.device)
     if partial:
         dopts = dict(opts)
@@ -79,6 +81,8 @@ def test_fuzz_whole_and_partial_plans(seed):
     assert np.array_equal(out["freed_blocks"], p.freed_blocks)
     if partial:
         assert np.array_equal(out["released_blocks"], p.released_blocks)
+    if before is not None:          # relocation check: same digest through the new table (token conservation)
+        assert np.array_equal(before, _digest(prob, vt, prob.new_tt_slots, None))
     k = np.stack([wl.fill_slab(seed, 0, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
     v = np.stack([wl.fill_slab(seed, 1, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
     vto.apply_moves_pools(k, v, p.move_src, p.move_dst)

@@ -51,6 +51,8 @@
  *   VTOKEN_COPY_CTAS     grid size of the copy kernel
  *   VTOKEN_BULK_TUNE     "warps,stages,rows,depth,ahead": warps per CTA, ring size, rows per work item,
  *                        items loading ahead of the one being stored, plan entries fetched ahead (1 or 2)
+ *   VTOKEN_COPY_DYNAMIC  0: every warp of the copy kernel gets a fixed share of the work items; 1 (default):
+ *                        warps take items from a ticket counter, VTOKEN_COPY_CHUNK (default 4) at a time
  *   VTOKEN_WAIT_LIMIT_MS bound of in-kernel waits (1 .. 60000, default 2000)
  *   VTOKEN_TEST_STALL_ITEM  test hook: index of one work item whose barrier is armed with bytes that never
  *                        arrive, so that its wait runs out (exercises the time-out path; never set in production)

@@ -69,6 +69,9 @@ struct vtoken_ctx {
     int copy_variant;          // 1 register path, 2 bulk-copy path
     int copy_ctas, copy_threads, copy_smem;
     int64_t wait_limit_ns, stall_item;   // bound of in-kernel waits; test hook (see copy.cu)
+    bool copy_dynamic;         // bulk path: items handed out by a ticket counter instead of fixed shares
+    int copy_chunk;            // consecutive items per ticket
+    unsigned int *copy_ticket; // [2] DEVICE: next item, finished warps (zero between launches)
     int bulk_warps, bulk_stages, bulk_rows, bulk_depth, bulk_ahead;   // bulk path: warps per CTA, ring size, rows per item, loads ahead
 };
 

@@ -30,6 +30,7 @@ struct CopyArgs {
     int64_t wait_limit_ns;     // bound of every wait on a shared-memory barrier (bulk path)
     int64_t stall_item;        // -1, or the global index of one item whose barrier is armed with bytes that
                                // never arrive: exercises the time-out path without faulting anything
+    unsigned int *ticket;      // dynamic item distribution: [0] next item index, [1] warps that have finished
 };
 
 __device__ __forceinline__ uint8_t *slab_base(const CopyArgs &a, int slab)
@@ -158,9 +159,10 @@ constexpr int BULK_MAX_SMEM = 216 * 1024;   // dynamic shared memory cap: leaves
 //
 // Work: an item is `rows` consecutive destination slots of one destination block in one slab
 // (rows is a power of two that divides S, so its destination is one contiguous byte range).
-// Items are numbered slab-major and dealt to the warps of the grid round-robin: at any moment
-// the grid works on a window of consecutive items, i.e. on one contiguous destination range of
-// a few MB, which keeps DRAM pages and TLB entries hot on the write side.
+// Items are numbered slab-major and handed to the warps of the grid in that order (by a ticket
+// counter, see DYNAMIC below, or round-robin): at any moment the grid works on a window of
+// consecutive items, i.e. on one contiguous destination range of a few MB, which keeps DRAM
+// pages and TLB entries hot on the write side.
 //
 // Step k of a warp's pipeline: (1) free and refill the stage that item k+depth will use -- its
 // previous tenant is item k+depth-stages = k-(w+1), w = stages-depth-1, so the w newest store
@@ -175,7 +177,20 @@ constexpr int BULK_MAX_SMEM = 216 * 1024;   // dynamic shared memory cap: leaves
 // division).  `ahead` is a run-time argument on purpose: measured on B200, the build in which
 // it is a compile-time constant schedules the issue path 2-3 % slower (6.20 vs 6.32 TB/s on the
 // Llama-shaped workload, same box, alternating runs).
-__global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages, int depth, int ahead)
+//
+// DYNAMIC: instead of its fixed share (items gw, gw + gstride, ...) a warp takes the next
+// `chunk` consecutive items from a global ticket counter.  SMs do not all move bytes at the same
+// rate: an in-kernel timeline on B200 showed the median warp at 6.8 TB/s-equivalent throughout
+// while the slowest SM finished 80-190 us after the median one, whatever the kernel's length, so
+// fixed shares leave most of the GPU idle at the end of every launch (3.7 % of a 1.35 ms launch,
+// 8 % of a 0.7 ms one).  Tickets keep the property that the grid works on one contiguous window
+// of items, and they absorb row-less tail items as well.  One atomic per item caps the kernel at
+// the throughput of same-address atomics (3.2 TB/s on the largest workload); one per 4 items is
+// free.  A chunk's ticket is requested a whole chunk before it is used, so its round trip is off
+// the critical path; the last warp to finish resets the counters for the next launch.
+template <bool DYNAMIC>
+__global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages, int depth, int ahead,
+                                                                        int chunk)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ uint64_t bars[BULK_MAX_WARPS * BULK_MAX_STAGES];
@@ -214,23 +229,52 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
 
     // plan entries of the next two items to issue: slab, destination slot of the first row
     // (-1: skip the item), source slot of this lane's row (-1: no row)
-    struct Entry { int slab; int32_t dst0, src; };
+    struct Entry { int slab; int32_t dst0, src; unsigned idx; };
     Entry e1, e2;
-    auto fetch = [&](Entry &e) {           // reads the item under c_fetch, moves the cursor
-        e.slab = c_fetch.slab;
+    const unsigned total_items = (unsigned)per_slab * (unsigned)num_slabs;   // < 2^31, checked on the host
+    // DYNAMIC: a ticket stands for `chunk` consecutive items (one atomic per chunk keeps the counter
+    // far from the throughput of same-address atomics); lane 0 holds the ticket of the NEXT chunk
+    unsigned ticket = 0xffffffffu, chunk_base = 0, chunk_pos = (unsigned)chunk;
+    auto take_ticket = [&]() { if (lane == 0) ticket = atomicAdd(&a.ticket[0], 1u); };
+    auto fetch = [&](Entry &e) {           // reads the next item of this warp, moves on
         e.dst0 = -1;
         e.src = -1;
-        if (c_fetch.slab < num_slabs) {
-            const int j = (int)((unsigned)c_fetch.rem / (unsigned)parts);
-            const int i0 = (c_fetch.rem - j * parts) * rows;
-            const int32_t blk = a.dst_blocks[j];
-            if (lane < rows) e.src = a.dst_src[(int64_t)j * S + i0 + lane];
-            e.dst0 = blk >= 0 ? blk * S + i0 : -1;
-            c_fetch.slab += step_slabs;
-            c_fetch.rem += step_rem;
-            if (c_fetch.rem >= per_slab) { c_fetch.rem -= per_slab; ++c_fetch.slab; }
+        e.idx = 0;
+        if (DYNAMIC) {
+            if (chunk_pos == (unsigned)chunk) {             // next chunk: its ticket was requested a chunk ago
+                const unsigned t = __shfl_sync(0xffffffffu, ticket, 0);
+                chunk_base = t < 0x7fffffffu / (unsigned)chunk ? t * (unsigned)chunk : 0x7fffffffu;
+                chunk_pos = 0;
+                if (chunk_base < total_items) take_ticket();
+            }
+            const unsigned i = chunk_base + chunk_pos;
+            ++chunk_pos;
+            e.slab = num_slabs;
+            if (i < total_items) {
+                const unsigned slab = i / (unsigned)per_slab, rem = i - slab * (unsigned)per_slab;
+                const int j = (int)(rem / (unsigned)parts);
+                const int i0 = ((int)rem - j * parts) * rows;
+                const int32_t blk = a.dst_blocks[j];
+                if (lane < rows) e.src = a.dst_src[(int64_t)j * S + i0 + lane];
+                e.dst0 = blk >= 0 ? blk * S + i0 : -1;
+                e.slab = (int)slab;
+                e.idx = i;
+            }
+        } else {
+            e.slab = c_fetch.slab;
+            if (c_fetch.slab < num_slabs) {
+                const int j = (int)((unsigned)c_fetch.rem / (unsigned)parts);
+                const int i0 = (c_fetch.rem - j * parts) * rows;
+                const int32_t blk = a.dst_blocks[j];
+                if (lane < rows) e.src = a.dst_src[(int64_t)j * S + i0 + lane];
+                e.dst0 = blk >= 0 ? blk * S + i0 : -1;
+                c_fetch.slab += step_slabs;
+                c_fetch.rem += step_rem;
+                if (c_fetch.rem >= per_slab) { c_fetch.rem -= per_slab; ++c_fetch.slab; }
+            }
         }
     };
+    if (DYNAMIC) take_ticket();
     fetch(e1);
     if (ahead == 2) fetch(e2);
 
@@ -257,7 +301,8 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         if (lane == 0) {
             my_mask[s] = mask;
             my_dst[s] = (uint64_t)(base + (int64_t)e.dst0 * a.row_bytes);
-            const uint32_t phantom = stall_countdown == 0 ? 16u : 0u;
+            const uint32_t phantom = (DYNAMIC ? (a.stall_item >= 0 && (int64_t)e.idx == a.stall_item)
+                                              : stall_countdown == 0) ? 16u : 0u;
             mbar_expect_tx(&my_bars[s], (uint32_t)__popc(mask) * row_bytes + phantom);   // no rows: plain arrive
         }
         __syncwarp();
@@ -299,6 +344,15 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         if (lane == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_TIMEOUT);
     }
     bulk_wait_all();
+    if (DYNAMIC && lane == 0) {
+        // the last warp of the grid to get here puts the counters back for the next launch; every
+        // other warp has stopped taking tickets by then
+        __threadfence();
+        if (atomicAdd(&a.ticket[1], 1u) == (unsigned)gstride - 1u) {
+            a.ticket[0] = 0u;
+            a.ticket[1] = 0u;
+        }
+    }
 }
 
 }  // namespace
@@ -357,7 +411,13 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctx->bulk_rows = rows;
         ctx->copy_threads = warps * 32;
         ctx->copy_smem = (int)smem;
-        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        // tickets are 32-bit: every item of a launch must have an index below 2^31
+        ctx->copy_dynamic = (int64_t)ctx->cap_dst_blocks * (S / rows) * 2 * ctx->cfg.num_layers < (int64_t)INT32_MAX;
+        if (const char *e = getenv("VTOKEN_COPY_DYNAMIC")) ctx->copy_dynamic = ctx->copy_dynamic && atoi(e) != 0;
+        ctx->copy_chunk = 4;
+        if (const char *e = getenv("VTOKEN_COPY_CHUNK")) { int v = atoi(e); if (v >= 1 && v <= 1024) ctx->copy_chunk = v; }
         ctas_per_sm = (int)((227 * 1024) / (smem + 2048));
         if (ctas_per_sm < 1) ctas_per_sm = 1;
         if (ctas_per_sm > 8) ctas_per_sm = 8;
@@ -385,10 +445,13 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     a.rows = ctx->bulk_rows;
     a.wait_limit_ns = ctx->wait_limit_ns;
     a.stall_item = ctx->stall_item;
+    a.ticket = ctx->copy_ticket;
     if (ctx->copy_variant == 1)
         copy_rows_kernel<<<ctx->copy_ctas, ctx->copy_threads, 0, st>>>(a);
+    else if (ctx->copy_dynamic)
+        copy_bulk_kernel<true><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk);
     else
-        copy_bulk_kernel<<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead);
+        copy_bulk_kernel<false><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, 1);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

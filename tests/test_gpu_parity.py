@@ -118,6 +118,34 @@ def test_bulk_copy_ring_shapes(tune, monkeypatch):
         run_and_compare(w, copy_variant=2)
 
 
+@pytest.mark.parametrize("dynamic,chunk", [("0", "4"), ("1", "1"), ("1", "3"), ("1", "64"), ("1", "1000")])
+def test_copy_work_distribution_modes(dynamic, chunk, monkeypatch):
+    """Fixed shares per warp and ticket distribution with several chunk sizes (one item per ticket,
+    an odd count, more items per ticket than a small launch has): the same bytes, whole pools
+    against the oracle, also when the context is reused for a second plan (the ticket counter must
+    be back at zero)."""
+    monkeypatch.setenv("VTOKEN_COPY_DYNAMIC", dynamic)
+    monkeypatch.setenv("VTOKEN_COPY_CHUNK", chunk)
+    for w in (wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2),
+              wl.longctx_scissor(seed=5, requests=2, lo=1500, hi=2500, layers=2, block_size=32),
+              wl.tiny(seed=1)):
+        run_and_compare(w, copy_variant=2)
+    from paper_2608_13263_b200.device import DeviceProblem
+    w = wl.llama8b_h2o(seed=2, requests=5, lo=200, hi=900, layers=2)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=2)
+    p = vto.plan_workload(w)
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    for _ in range(3):                                   # three launches on one context
+        prob.fill_pools()
+        prob.plan()
+        prob.repack()
+        assert prob.outputs()["error_flags"] == 0
+        assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+        assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()
+
+
 def _request(n_tokens, S, first_block):
     nb = -(-n_tokens // S)
     bt = np.arange(first_block, first_block + nb, dtype=np.int32)

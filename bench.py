@@ -420,6 +420,9 @@ def run_cuda(args):
                    "l2": "moved bytes per step exceed the 126 MB L2 (no flush needed)" if bytes_per_step > 4 * 126e6
                          else "moved bytes per step fit in L2: launch-bound parity configuration",
                    "launch": "CUDA graph (plan + copy) replayed on a side stream", "copy_grid": grid,
+                   "copy_work_distribution": ("fixed share per warp" if os.environ.get("VTOKEN_COPY_DYNAMIC") == "0"
+                                              else "ticket counter, " + os.environ.get("VTOKEN_COPY_CHUNK", "4") +
+                                                   " items per ticket") if grid["variant"] == 2 else "grid-stride rows",
                    "plan_mode": args.plan_mode if args.plan_mode == "whole" else
                                 "partial: sources = blocks that are not fully live, trigger F > 1/4",
                    "gpu": f"{torch.cuda.get_device_name(dev)} {str(torch.cuda.get_device_properties(dev).uuid)[-12:]}",

@@ -1,5 +1,7 @@
 """Seeded fuzz of the whole path against the oracle: random shapes, block sizes, masks, table holes,
 selections, thresholds, free-list lengths and partial-plan options, whole pools compared."""
+import os
+
 import numpy as np
 import pytest
 
@@ -7,6 +9,9 @@ from oracle import vto
 from paper_2608_13263_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
+
+# more seeds for a soak run: VTOKEN_FUZZ_SCALE=10 runs ten times as many problems
+FUZZ_SCALE = max(1, int(os.environ.get("VTOKEN_FUZZ_SCALE", "1")))
 
 
 def random_problem(rng):
@@ -36,7 +41,7 @@ def random_problem(rng):
     return w
 
 
-@pytest.mark.parametrize("seed", range(60))
+@pytest.mark.parametrize("seed", range(60 * FUZZ_SCALE))
 def test_fuzz_whole_and_partial_plans(seed):
     import torch
     from paper_2608_13263_b200.device import DeviceProblem
@@ -91,7 +96,7 @@ def test_fuzz_whole_and_partial_plans(seed):
     prob.close()
 
 
-@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("seed", range(24 * FUZZ_SCALE))
 def test_fuzz_repack_in_waves(seed):
     """Random problems through vtoken_repack_waves (short pools, whole and partial planners): all
     outputs and whole pools against the oracle's wave plan, and the relocation digest of every

@@ -25,7 +25,7 @@ void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
-                    ctx->n_b, ctx->blk_src, ctx->slot_bits, ctx->copy_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
+                    ctx->n_b, ctx->blk_src, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
                     ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
@@ -134,6 +134,8 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->slot_bits, (slots + 31) / 32);
     A(&ctx->copy_ticket, 2);
     if (rc == VTOKEN_OK && cudaMemset(ctx->copy_ticket, 0, 2 * sizeof(unsigned int)) != cudaSuccess) rc = VTOKEN_ECUDA;
+    A(&ctx->g_ticket, 2);
+    if (rc == VTOKEN_OK && cudaMemset(ctx->g_ticket, 0, 2 * sizeof(unsigned int)) != cudaSuccess) rc = VTOKEN_ECUDA;
     A(&ctx->part_shared, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
     A(&ctx->req_shared, cfg->max_requests);
     A(&ctx->req_detach, cfg->max_requests);

@@ -48,6 +48,7 @@ struct vtoken_ctx {
     int32_t *g_ids;            // [max_tokens] logical id of each output row (digest)
     int32_t *g_req;            // [max_tokens] request of each output row (digest)
     int32_t *g_offsets;        // [max_requests + 1] first output row of each request (digest)
+    unsigned int *g_ticket;    // [2] work tickets of the gather's row copy (zero between launches)
 
     // device staging of vtoken_repack_host (DEVICE), allocated on first use
     struct {
@@ -79,6 +80,8 @@ struct vtoken_ctx {
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
 int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st);
 int vtk_configure_copy(vtoken_ctx *ctx);
+bool vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t *g_total, int32_t layer_begin,
+                            int32_t layer_end, void *out_k, void *out_v, int64_t out_capacity, cudaStream_t st);
 int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                       const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
                       int32_t layer_begin, int32_t layer_end, void *out_k, void *out_v,

@@ -31,6 +31,12 @@ struct CopyArgs {
     int64_t stall_item;        // -1, or the global index of one item whose barrier is armed with bytes that
                                // never arrive: exercises the time-out path without faulting anything
     unsigned int *ticket;      // dynamic item distribution: [0] next item index, [1] warps that have finished
+    // gather mode (logical view): rows g_src[0 .. *g_total) of layers [layer_begin, layer_begin + L) go to the
+    // dense buffers out_k / out_v, [L][out_capacity][row_bytes]
+    const int32_t *g_src, *g_total;
+    uint8_t *out_k, *out_v;
+    int64_t out_capacity;
+    int32_t layer_begin;
 };
 
 __device__ __forceinline__ uint8_t *slab_base(const CopyArgs &a, int slab)
@@ -188,7 +194,11 @@ constexpr int BULK_MAX_SMEM = 216 * 1024;   // dynamic shared memory cap: leaves
 // the throughput of same-address atomics (3.2 TB/s on the largest workload); one per 4 items is
 // free.  A chunk's ticket is requested a whole chunk before it is used, so its round trip is off
 // the critical path; the last warp to finish resets the counters for the next launch.
-template <bool DYNAMIC>
+//
+// GATHER: the same machinery writes the logical view instead of executing a plan: an item is
+// `rows` consecutive rows of the dense output, its sources are the slots g_src names, and the
+// destination lies in another buffer than the source.  (Always with tickets.)
+template <bool DYNAMIC, bool GATHER>
 __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs a, int stages, int depth, int ahead,
                                                                         int chunk)
 {
@@ -213,7 +223,9 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
     __syncwarp();
 
     const int parts = S / rows;                                // items per destination block
-    const int per_slab = a.counts->num_dst_blocks * parts;     // items per slab, < 2^31 (checked on the host)
+    const int g_n = GATHER ? *a.g_total : 0;                   // gather: output rows per slab
+    // items per slab, < 2^31 (checked on the host)
+    const int per_slab = GATHER ? (g_n + rows - 1) / rows : a.counts->num_dst_blocks * parts;
     const int num_slabs = 2 * a.L;
     const int64_t gw = (int64_t)blockIdx.x * nwarps_cta + warp;
     const int64_t gstride = (int64_t)gridDim.x * nwarps_cta;
@@ -252,11 +264,17 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
             e.slab = num_slabs;
             if (i < total_items) {
                 const unsigned slab = i / (unsigned)per_slab, rem = i - slab * (unsigned)per_slab;
-                const int j = (int)(rem / (unsigned)parts);
-                const int i0 = ((int)rem - j * parts) * rows;
-                const int32_t blk = a.dst_blocks[j];
-                if (lane < rows) e.src = a.dst_src[(int64_t)j * S + i0 + lane];
-                e.dst0 = blk >= 0 ? blk * S + i0 : -1;
+                if (GATHER) {
+                    const int i0 = (int)rem * rows;                 // first output row of the item
+                    if (lane < rows && i0 + lane < g_n) e.src = a.g_src[i0 + lane];
+                    e.dst0 = i0;
+                } else {
+                    const int j = (int)(rem / (unsigned)parts);
+                    const int i0 = ((int)rem - j * parts) * rows;
+                    const int32_t blk = a.dst_blocks[j];
+                    if (lane < rows) e.src = a.dst_src[(int64_t)j * S + i0 + lane];
+                    e.dst0 = blk >= 0 ? blk * S + i0 : -1;
+                }
                 e.slab = (int)slab;
                 e.idx = i;
             }
@@ -294,13 +312,21 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
             fetch(e1);                               // in flight for one step
         }
         const bool valid = e.src >= 0 && e.dst0 >= 0;
-        uint8_t *base = slab_base(a, e.slab);
+        uint8_t *base, *dst_base;
+        if (GATHER) {
+            const int li = e.slab < a.L ? e.slab : e.slab - a.L;
+            base = (e.slab < a.L ? a.k_pool : a.v_pool) + (int64_t)(a.layer_begin + li) * a.layer_stride;
+            dst_base = (e.slab < a.L ? a.out_k : a.out_v) + (int64_t)li * a.out_capacity * a.row_bytes;
+        } else {
+            base = slab_base(a, e.slab);
+            dst_base = base;
+        }
         uint8_t *stg = my_smem + (size_t)s * stage_bytes;
         bulk_wait_read_n(stores_in_flight);          // the stage's previous store has read its bytes
         const unsigned mask = __ballot_sync(0xffffffffu, valid);
         if (lane == 0) {
             my_mask[s] = mask;
-            my_dst[s] = (uint64_t)(base + (int64_t)e.dst0 * a.row_bytes);
+            my_dst[s] = (uint64_t)(dst_base + (int64_t)e.dst0 * a.row_bytes);
             const uint32_t phantom = (DYNAMIC ? (a.stall_item >= 0 && (int64_t)e.idx == a.stall_item)
                                               : stall_countdown == 0) ? 16u : 0u;
             mbar_expect_tx(&my_bars[s], (uint32_t)__popc(mask) * row_bytes + phantom);   // no rows: plain arrive
@@ -411,8 +437,9 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctx->bulk_rows = rows;
         ctx->copy_threads = warps * 32;
         ctx->copy_smem = (int)smem;
-        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         // tickets are 32-bit: every item of a launch must have an index below 2^31
         ctx->copy_dynamic = (int64_t)ctx->cap_dst_blocks * (S / rows) * 2 * ctx->cfg.num_layers < (int64_t)INT32_MAX;
         if (const char *e = getenv("VTOKEN_COPY_DYNAMIC")) ctx->copy_dynamic = ctx->copy_dynamic && atoi(e) != 0;
@@ -455,9 +482,43 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     if (ctx->copy_variant == 1)
         copy_rows_kernel<<<ctx->copy_ctas, ctx->copy_threads, 0, st>>>(a);
     else if (ctx->copy_dynamic)
-        copy_bulk_kernel<true><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk);
+        copy_bulk_kernel<true, false><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk);
     else
-        copy_bulk_kernel<false><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, 1);
+        copy_bulk_kernel<false, false><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, 1);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
+}
+
+// The row copy of vtoken_gather_logical through the bulk path (false: the context has no bulk
+// configuration for these rows; the caller uses its register kernel).
+bool vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t *g_total, int32_t layer_begin,
+                            int32_t layer_end, void *out_k, void *out_v, int64_t out_capacity, cudaStream_t st)
+{
+    if (ctx->copy_variant != 2 || !ctx->copy_dynamic || ctx->g_ticket == nullptr) return false;
+    // tickets are 32-bit: every item must have an index below 2^31
+    const int64_t items = (ctx->cfg.max_tokens + ctx->bulk_rows - 1) / ctx->bulk_rows * 2 * (layer_end - layer_begin);
+    if (items >= (int64_t)INT32_MAX) return false;
+    CopyArgs a;
+    a.k_pool = (uint8_t *)ctx->cfg.k_pool;
+    a.v_pool = (uint8_t *)ctx->cfg.v_pool;
+    a.dst_src = nullptr;
+    a.dst_blocks = nullptr;
+    a.counts = ctx->counts;
+    a.layer_stride = ctx->layer_stride;
+    a.row_bytes = ctx->row_bytes;
+    a.S = ctx->bulk_rows;                 // parts = 1: unused in gather mode
+    a.L = layer_end - layer_begin;
+    a.rows = ctx->bulk_rows;
+    a.wait_limit_ns = ctx->wait_limit_ns;
+    a.stall_item = -1;
+    a.ticket = ctx->g_ticket;
+    a.g_src = g_src;
+    a.g_total = g_total;
+    a.out_k = (uint8_t *)out_k;
+    a.out_v = (uint8_t *)out_v;
+    a.out_capacity = out_capacity;
+    a.layer_begin = layer_begin;
+    copy_bulk_kernel<true, true><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(
+        a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk);
+    return true;
 }

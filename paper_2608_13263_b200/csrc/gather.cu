@@ -397,7 +397,12 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
     gather_scan_kernel<<<1, 1024, 0, st>>>(a);
     gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
-    gather_copy_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
+    // the rows go through the bulk-copy rings when the context has them (vtoken_create does; the
+    // context-free entry point does not), else through the register kernel
+    const bool aligned = (((uintptr_t)out_k | (uintptr_t)out_v) & 15) == 0;
+    if (!(aligned && vtk_launch_gather_bulk(ctx, ctx->g_src, ctx->g_total, layer_begin, layer_end, out_k, out_v,
+                                            out_capacity_tokens, st)))
+        gather_copy_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

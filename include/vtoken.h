@@ -193,10 +193,11 @@ int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const in
  * hashed together with their K/V contents before and after a relocation).  The paper does not
  * name the hash; this library fixes one that any evaluation order reproduces bit for bit: for a
  * request whose active tokens have rank i = 0, 1, ... and logical ids t_i, over the slabs
- * s = 0 .. 2*(layer_end-layer_begin)-1 (K layers first, then V layers) and the 16-byte groups c of a
- * token's row, each two 8-byte little-endian words (w_2c, w_2c+1),
- *     key(i, s) = mix(((i * A + t_i) * B + s) * C),
- *     a = w_2c ^ (key(i, s) + 2c * D),   b = w_2c+1 ^ (key(i, s) + (2c + 1) * D),
+ * s = 0 .. 2*(layer_end-layer_begin)-1 (K layers first, then V layers) and the 32-byte groups g of a
+ * token's row, each four 8-byte little-endian words w_4g .. w_4g+3 (a row of 16 mod 32 bytes ends
+ * with a group of two words),
+ *     key(i, s) = mix(((i * A + t_i) * B + s) * C),      x_j = w_j ^ (key(i, s) + j * D),
+ *     a = x_4g + x_4g+2,   b = x_4g+1 + x_4g+3           (mod 2^64; absent words add nothing),
  *     digest    = sum of  low64(a * b) ^ high64(a * b)  mod 2^64        (a * b: the 128-bit product),
  * mix = splitmix64 finaliser, A = 0x9E3779B97F4A7C15, B = 0xD1B54A32D192ED03, C = 0x8CB92BA72F3D8DD7,
  * D = 0xA0761D6478BD642F.

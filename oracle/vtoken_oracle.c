@@ -742,14 +742,18 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
             const uint8_t *row = pool + (int64_t)layer * layer_stride_bytes + (int64_t)tt_slots[t] * row_bytes;
             /* key of this (rank, id, slab): binds the row's words to their place in the logical view */
             const uint64_t key = mix64((((uint64_t)i * A + (uint64_t)t) * B + (uint64_t)s) * C);
-            for (int64_t c = 0; c < row_bytes / 16; ++c) {   /* 16 bytes = two little-endian words */
-                uint64_t w0 = 0, w1 = 0;
-                for (int b = 7; b >= 0; --b) {
-                    w0 = (w0 << 8) | row[c * 16 + b];
-                    w1 = (w1 << 8) | row[c * 16 + 8 + b];
+            /* 32-byte groups of four little-endian words; a row of 16 (mod 32) bytes ends with a
+             * half group of two words.  Every word is bound to its place by its own key. */
+            const int64_t nwords = row_bytes / 8;
+            for (int64_t g = 0; g * 4 < nwords; ++g) {
+                uint64_t a = 0, b = 0;
+                for (int64_t j = 4 * g; j < 4 * g + 4 && j < nwords; ++j) {
+                    uint64_t w = 0;
+                    for (int q = 7; q >= 0; --q) w = (w << 8) | row[j * 8 + q];
+                    const uint64_t x = w ^ (key + (uint64_t)j * D);
+                    if ((j & 1) == 0) a += x;                /* words 4g, 4g+2 */
+                    else b += x;                             /* words 4g+1, 4g+3 */
                 }
-                const uint64_t a = w0 ^ (key + (uint64_t)(2 * c) * D);
-                const uint64_t b = w1 ^ (key + (uint64_t)(2 * c + 1) * D);
                 const unsigned __int128 prod = (unsigned __int128)a * b;      /* full 128-bit product */
                 sum += (uint64_t)prod ^ (uint64_t)(prod >> 64);
             }

@@ -261,15 +261,15 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
  * after a relocation.  It does not name the hash; this build fixes one that can be evaluated in
  * any order (a sum of per-word terms, each bound to its position): for a request whose active
  * tokens are t_0 < t_1 < ... (rank i, logical id t_i), over slabs s = 0 .. 2*(layer_end-layer_begin)-1
- * (K layers first, then V layers) and the 16-byte groups c of the token's row, each two 8-byte
- * little-endian words (w_2c, w_2c+1),
- *     key(i, s) = mix(((i * A + t_i) * B + s) * C)
- *     a = w_2c ^ (key(i, s) + 2c * D),   b = w_2c+1 ^ (key(i, s) + (2c + 1) * D)
- *     digest    = sum over (i, s, c) of  low64(a * b) ^ high64(a * b)        mod 2^64
+ * (K layers first, then V layers) and the 32-byte groups g of the token's row, each four 8-byte
+ * little-endian words w_4g .. w_4g+3 (a row of 16 mod 32 bytes ends with a group of two words),
+ *     key(i, s) = mix(((i * A + t_i) * B + s) * C),      x_j = w_j ^ (key(i, s) + j * D)
+ *     a = x_4g + x_4g+2,   b = x_4g+1 + x_4g+3           (mod 2^64; absent words add nothing)
+ *     digest    = sum over (i, s, g) of  low64(a * b) ^ high64(a * b)        mod 2^64
  * with a * b the full 128-bit product, mix = the splitmix64 finaliser and A, B, C, D the odd
- * constants in the source (one multiply-fold per 16 bytes: the check reads K/V at memory speed).
- * A lost, duplicated, reordered or altered token changes the digest.  row_bytes must be a multiple
- * of 16.
+ * constants in the source (one multiply-fold per 32 bytes: the check reads K/V at memory speed).
+ * Every word is bound to its place by its own key; a lost, duplicated, reordered or altered token
+ * changes the digest.  row_bytes must be a multiple of 16.
  * Pools are [L][num_slots][row_bytes] with layer_stride_bytes between layers (0 = dense). */
 int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t layer_stride_bytes, int64_t num_slots,
                        int64_t row_bytes, int32_t layer_begin, int32_t layer_end, const int32_t *tt_slots,

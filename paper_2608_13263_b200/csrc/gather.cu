@@ -196,17 +196,17 @@ __device__ __forceinline__ unsigned long long g_mix64(unsigned long long x)   //
 }
 
 // Relocation digest (Sec. 5 of the paper hashes ordered retained ids with their K/V contents):
-//   key(i, s) = mix(((i*A + t_i)*B + s)*C);  per 16-byte group c of the row (8-byte words w0, w1):
-//   x = w0 ^ (key + 2c*D), y = w1 ^ (key + (2c+1)*D);  digest[r] = sum of low64(x*y) ^ high64(x*y)
+//   key(i, s) = mix(((i*A + t_i)*B + s)*C);  per 32-byte group g of the row (8-byte words w_4g .. w_4g+3,
+//   x_j = w_j ^ (key + j*D)):  a = x_4g + x_4g+2, b = x_4g+1 + x_4g+3;  digest[r] = sum of low64(a*b) ^ high64(a*b)
 // a sum of position-bound terms, so any evaluation order gives the same 64-bit value.
-// A warp walks a contiguous run of (slab, output row) units; lanes take 16-byte groups of the row.
+// A warp walks a contiguous run of (slab, output row) units; lanes take 32-byte groups of the row.
 // One (slab, row) unit of the digest: where it is and what it hashes.
 struct DigestRow {
     const uint4 *ptr;            // first byte of the K or V row
     int32_t r, tok, slab, idx;
 };
 
-__global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
+__global__ void __launch_bounds__(GC_NT, 3) gather_digest_kernel(GatherArgs a)
 {
     const unsigned long long A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull,
                              D = 0xA0761D6478BD642Full;
@@ -215,10 +215,12 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
     const int64_t total = n * nl * 2;
     const int lane = vtk_lane();
     const int row_vecs = (int)(a.row_bytes >> 4);
-    // A row is hashed by a group of G lanes with four 16-byte loads each: the whole warp for rows
-    // of 2 KiB and more, half a warp for 1 KiB rows, ... so that every lane's loads carry bytes.
+    // A row is hashed by a group of G lanes, each taking two 32-byte groups of the row (four 16-byte
+    // loads): the whole warp for rows of 2 KiB and more, half a warp for 1 KiB rows, ... so that
+    // every lane's loads carry bytes.
+    const int row_groups = (row_vecs + 1) >> 1;                // 32-byte groups, the last one may be half
     int G = 32;
-    while (G > 1 && 4 * G > row_vecs) G >>= 1;
+    while (G > 1 && 2 * G > row_groups) G >>= 1;
     const int gl = lane & (G - 1), per_warp = 32 / G;
     const unsigned gmask = G == 32 ? 0xffffffffu : (((1u << G) - 1u) << (lane & ~(G - 1)));
     const int64_t ngroups = (int64_t)gridDim.x * (GC_NT / 32) * per_warp;
@@ -252,23 +254,32 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         m.r = a.g_req[idx];
         m.tok = a.g_ids[idx];
     };
-    auto load4 = [&](uint4 (&v)[4], const uint4 *sp, int c0) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k)
-            v[k] = (c0 + G * k < row_vecs) ? ld_stream(sp + c0 + G * k) : make_uint4(0, 0, 0, 0);
-    };
-    // word offsets without multiplies in the row loop: group c = c0 + G*k has x-offset
-    // 2*c*D = 2*c0*D + k*(2*G*D) and y-offset one D further
-    const unsigned long long lane_off = 2ull * gl * D, k_step = 2ull * G * D;
-    auto hash4 = [&](const uint4 (&v)[4], unsigned long long key_c0, int c0) {   // key_c0 = key + 2*c0*D
+    // v[2m], v[2m+1] = the two 16-byte halves of 32-byte group p0 + G*m, m = 0, 1
+    auto load4 = [&](uint4 (&v)[4], const uint4 *sp, int p0) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-            if (c0 + G * k < row_vecs) {
-                const unsigned long long w0 = ((unsigned long long)v[k].y << 32) | v[k].x;
-                const unsigned long long w1 = ((unsigned long long)v[k].w << 32) | v[k].z;
-                const unsigned long long xo = key_c0 + (unsigned long long)k * k_step;
-                const unsigned long long x = w0 ^ xo;
-                const unsigned long long y = w1 ^ (xo + D);
+            const int vec = 2 * (p0 + G * (k >> 1)) + (k & 1);
+            v[k] = vec < row_vecs ? ld_stream(sp + vec) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    // word offsets without multiplies in the row loop: the words of group p = p0 + G*m carry the
+    // offsets (4p + j)*D = 4*p0*D + m*(4*G*D) + j*D, j = 0..3
+    const unsigned long long lane_off = 4ull * gl * D, k_step = 4ull * G * D;
+    auto hash4 = [&](const uint4 (&v)[4], unsigned long long key_p0, int p0) {   // key_p0 = key + 4*p0*D
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+            const int p = p0 + G * m;
+            if (2 * p < row_vecs) {
+                const unsigned long long ko = key_p0 + (unsigned long long)m * k_step;
+                const unsigned long long w0 = ((unsigned long long)v[2 * m].y << 32) | v[2 * m].x;
+                const unsigned long long w1 = ((unsigned long long)v[2 * m].w << 32) | v[2 * m].z;
+                unsigned long long x = w0 ^ ko, y = w1 ^ (ko + D);
+                if (2 * p + 1 < row_vecs) {                        // the second half of the group exists
+                    const unsigned long long w2 = ((unsigned long long)v[2 * m + 1].y << 32) | v[2 * m + 1].x;
+                    const unsigned long long w3 = ((unsigned long long)v[2 * m + 1].w << 32) | v[2 * m + 1].z;
+                    x += w2 ^ (ko + 2ull * D);
+                    y += w3 ^ (ko + 3ull * D);
+                }
                 sum += (x * y) ^ __umul64hi(x, y);                 // low64 ^ high64 of the 128-bit product
             }
         }
@@ -299,14 +310,14 @@ __global__ void __launch_bounds__(GC_NT) gather_digest_kernel(GatherArgs a)
         const unsigned long long i = (unsigned long long)(cur.idx - a.out_offsets[cur.r]);
         const unsigned long long key =
             g_mix64(((i * A + (unsigned long long)cur.tok) * B + (unsigned long long)cur.slab) * C);
-        unsigned long long key_c0 = key + lane_off;
-        hash4(vc, key_c0, gl);
-        if (row_vecs > 4 * G) {                                // rows above 64 bytes per lane: the rest, unpipelined
-            for (int c0 = gl + 4 * G; c0 < row_vecs; c0 += 4 * G) {
+        unsigned long long key_p0 = key + lane_off;
+        hash4(vc, key_p0, gl);
+        if (row_groups > 2 * G) {                              // rows above 64 bytes per lane: the rest, unpipelined
+            for (int p0 = gl + 2 * G; p0 < row_groups; p0 += 2 * G) {
                 uint4 v[4];
-                key_c0 += 4ull * k_step;
-                load4(v, cur.ptr, c0);
-                hash4(v, key_c0, c0);
+                key_p0 += 2ull * k_step;
+                load4(v, cur.ptr, p0);
+                hash4(v, key_p0, p0);
             }
         }
 #pragma unroll

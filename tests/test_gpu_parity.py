@@ -322,10 +322,15 @@ def test_argument_errors():
     prob.close()
 
 
-def test_gather_logical_before_equals_after_and_matches_oracle():
+@pytest.mark.parametrize("heads,head_dim", [(2, 64), (4, 128), (8, 128), (3, 128)],
+                         ids=["row256-register", "row1024-bulk", "row2048-bulk", "row768-bulk"])
+def test_gather_logical_before_equals_after_and_matches_oracle(heads, head_dim):
+    """Rows below 512 bytes go through the register kernel, the others through the bulk-copy kernel
+    in gather mode; the last step replays the gather from a captured graph (its work tickets must
+    be back at zero after every launch)."""
     from paper_2608_13263_b200.device import DeviceProblem
     torch = _torch()
-    w = wl.steady_state(seed=3, requests=10, lo=100, hi=900, layers=3, heads=2, head_dim=64)
+    w = wl.steady_state(seed=3, requests=10, lo=100, hi=900, layers=3, heads=heads, head_dim=head_dim)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
     cap = int(((w.tt_slots >= 0) & (w.keep != 0)).sum())
     bk, bv, boff = prob.gather_logical(prob.tt_slots, prob.keep, 0, 3, cap)
@@ -366,6 +371,29 @@ def test_gather_logical_before_equals_after_and_matches_oracle():
     ok, ov, ooff = prob.gather_logical(prob.tt_slots, prob.keep, 0, 1, cap - 5)
     assert prob.read_counts()["error_flags"] & vt.FLAG_GATHER_OVERFLOW
     assert torch.equal(ok[0, :cap - 5], bk[0, :cap - 5])
+    # captured once, replayed three times
+    gk = torch.zeros((3, cap, w.row_elems), dtype=torch.int16, device=prob.device)
+    gv = torch.zeros_like(gk)
+    goff = torch.zeros(prob.max_requests + 1, dtype=torch.int32, device=prob.device)
+    call = lambda st: vt.vtoken_gather_logical(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                               tt_slots=prob.new_tt_slots, keep=None, select=None, layer_begin=0,
+                                               layer_end=3, out_k=gk, out_v=gv, out_capacity_tokens=cap,
+                                               out_offsets=goff, stream=st)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        call(side)
+    side.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        call(torch.cuda.current_stream())
+    for _ in range(3):
+        gk.zero_()
+        gv.zero_()
+        torch.cuda.synchronize()
+        g.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(gk, ak) and torch.equal(gv, av) and torch.equal(goff, aoff)
     prob.close()
 
 

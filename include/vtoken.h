@@ -112,7 +112,8 @@ typedef struct {
     int64_t max_table_blocks;      /* upper bound of the block-table length (sum over requests) */
     int32_t max_free_blocks;       /* upper bound of num_free */
     int32_t max_ctas;              /* copy-kernel grid cap (co-residency with other work); 0 => auto */
-    int32_t copy_variant;          /* 0 auto; 1 register path; 2 bulk-copy (TMA) path */
+    int32_t copy_variant;          /* 0 auto (bulk-copy path when row_bytes <= 32768, else register path);
+                                      1 register path; 2 bulk-copy (TMA) path */
 } vtoken_config;
 
 /* row_bytes = num_kv_heads * head_dim * elem_bytes must be a multiple of 16, pools and

@@ -389,8 +389,11 @@ int vtk_configure_copy(vtoken_ctx *ctx)
     const int S = ctx->cfg.block_size;
     int variant = ctx->cfg.copy_variant;
     if (const char *e = getenv("VTOKEN_COPY_VARIANT")) { if (variant == 0) variant = atoi(e); }
-    // bulk copies need 16-byte multiples (checked at create) and a row that fits a stage
-    if (variant == 0) variant = (ctx->row_bytes >= 512 && ctx->row_bytes <= 32768) ? 2 : 1;
+    // bulk copies need 16-byte multiples (checked at create) and a row that fits a stage.  Small rows
+    // belong on the bulk path too: the register path spends a warp per row whatever its size (measured
+    // on B200 with 256 / 128 / 64 / 16-byte rows: 2.0 / 1.0 / 0.5 / 0.14 TB/s against 6.1 / 4.6 / 2.6 /
+    // 0.3 TB/s through the rings, where an item is up to 32 rows)
+    if (variant == 0) variant = ctx->row_bytes <= 32768 ? 2 : 1;
     if (variant != 1 && variant != 2) return VTOKEN_EINVAL;
 
     int ctas_per_sm;

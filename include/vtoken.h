@@ -56,6 +56,13 @@
  *   VTOKEN_WAIT_LIMIT_MS bound of in-kernel waits (1 .. 60000, default 2000)
  *   VTOKEN_TEST_STALL_ITEM  test hook: index of one work item whose barrier is armed with bytes that never
  *                        arrive, so that its wait runs out (exercises the time-out path; never set in production)
+ * and one read at every launch:
+ *   VTOKEN_PDL           0: plain stream-ordered launches; 1 (default): every kernel of the library is launched
+ *                        with programmatic stream serialization, i.e. it may become resident while the previous
+ *                        kernel in the stream is finishing and waits (griddepcontrol.wait, first thing it does)
+ *                        until that kernel has completed and its writes are visible.  Results are identical;
+ *                        a chain of short kernels (planner, waves, slot mapping) loses about 1 us per boundary.
+ *                        A caller's own kernel that follows in the stream is ordered as usual.
  *
  * Preconditions assumed (not checked) on the fast path: each live slot is referenced by one
  * token only (I2) and lies in a block of its own request; block ids are unique across block

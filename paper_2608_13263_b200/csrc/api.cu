@@ -76,6 +76,12 @@ int ensure_stage(vtoken_ctx *ctx)
 
 }  // namespace
 
+bool vtk_dependent_launch_enabled()
+{
+    const char *e = getenv("VTOKEN_PDL");      // read at every launch: a test can switch it between calls
+    return e == nullptr || atoi(e) != 0;
+}
+
 extern "C" {
 
 int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)

@@ -97,6 +97,38 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     } while (0)
 
 // ---------------------------------------------------------------------------------------
+// Programmatic dependent launch: a kernel launched through vtk_launch_dependent may become
+// resident while its predecessor in the stream is still running (its launch latency and its
+// prologue overlap the predecessor's tail); it must call vtk_wait_for_predecessor() before it
+// touches anything an earlier kernel wrote or still reads -- the wait returns once the
+// predecessor grid has completed and its writes are visible.  Every thread of such a kernel
+// calls the wait before it can exit, so the grid cannot complete before its predecessor did and
+// the ordering stays transitive along the stream.  vtk_release_successor() lets the next
+// kernel in the stream start its own launch early.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void vtk_wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void vtk_release_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+bool vtk_dependent_launch_enabled();   // VTOKEN_PDL=0 turns the launch attribute off (the device side is then a no-op)
+
+template <typename... P, typename... A>
+inline cudaError_t vtk_launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                        A... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = vtk_dependent_launch_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, P(args)...);
+}
+
+// ---------------------------------------------------------------------------------------
 // device helpers
 // ---------------------------------------------------------------------------------------
 __device__ __forceinline__ int vtk_lane() { return threadIdx.x & 31; }

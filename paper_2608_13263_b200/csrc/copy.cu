@@ -61,6 +61,7 @@ constexpr int REG_UNROLL = 4;   // 16-byte loads in flight per lane per row
 
 __global__ void __launch_bounds__(REG_NT) copy_rows_kernel(CopyArgs a)
 {
+    vtk_wait_for_predecessor();            // the plan is the previous kernel's output
     const int nblk = a.counts->num_dst_blocks;
     const int64_t rows_per_slab = (int64_t)nblk * a.S;
     const int64_t total = rows_per_slab * 2 * a.L;
@@ -221,6 +222,9 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncwarp();
+    // everything above overlaps the tail of the previous kernel in the stream (normally the
+    // planner); its output -- counts, inverse plan -- and the pools are touched only below
+    vtk_wait_for_predecessor();
 
     const int parts = S / rows;                                // items per destination block
     const int g_n = GATHER ? *a.g_total : 0;                   // gather: output rows per slab
@@ -482,12 +486,15 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     a.wait_limit_ns = ctx->wait_limit_ns;
     a.stall_item = ctx->stall_item;
     a.ticket = ctx->copy_ticket;
+    const dim3 grid(ctx->copy_ctas), block(ctx->copy_threads);
     if (ctx->copy_variant == 1)
-        copy_rows_kernel<<<ctx->copy_ctas, ctx->copy_threads, 0, st>>>(a);
+        VTK_CUDA(ctx, vtk_launch_dependent(copy_rows_kernel, grid, block, 0, st, a));
     else if (ctx->copy_dynamic)
-        copy_bulk_kernel<true, false><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk);
+        VTK_CUDA(ctx, vtk_launch_dependent(copy_bulk_kernel<true, false>, grid, block, (size_t)ctx->copy_smem, st, a,
+                                           ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk));
     else
-        copy_bulk_kernel<false, false><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, 1);
+        VTK_CUDA(ctx, vtk_launch_dependent(copy_bulk_kernel<false, false>, grid, block, (size_t)ctx->copy_smem, st, a,
+                                           ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, 1));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -521,7 +528,9 @@ bool vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t
     a.out_v = (uint8_t *)out_v;
     a.out_capacity = out_capacity;
     a.layer_begin = layer_begin;
-    copy_bulk_kernel<true, true><<<ctx->copy_ctas, ctx->copy_threads, ctx->copy_smem, st>>>(
-        a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk);
+    if (vtk_launch_dependent(copy_bulk_kernel<true, true>, dim3(ctx->copy_ctas), dim3(ctx->copy_threads),
+                             (size_t)ctx->copy_smem, st, a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead,
+                             ctx->copy_chunk) != cudaSuccess)
+        ctx->last_cuda_error = (int)cudaGetLastError();      // reported by the caller's cudaGetLastError check too
     return true;
 }

@@ -43,6 +43,8 @@ __device__ __forceinline__ void g_part_range(int64_t t0, int64_t t1, int c, int6
 
 __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int r = blockIdx.x / G_PARTS, c = blockIdx.x % G_PARTS;
     if (r >= g_requests(a)) return;
     int n = 0;
@@ -69,6 +71,8 @@ __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
 // exclusive scan of the per-request counts -> out_offsets[R+1]; one CTA
 __global__ void __launch_bounds__(1024) gather_scan_kernel(GatherArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ int warp_tot[33];
     __shared__ int carry;
     const int R = g_requests(a);
@@ -112,6 +116,8 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(GatherArgs a)
 
 __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ int warp_sums[G_NT / 32 + 1];
     const int r = blockIdx.x / G_PARTS, c = blockIdx.x % G_PARTS;
     if (r >= g_requests(a)) return;
@@ -157,6 +163,8 @@ constexpr int GC_NT = 256;
 // one warp per (pool, layer, output row)
 __global__ void __launch_bounds__(GC_NT) gather_copy_kernel(GatherArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int64_t n = *a.g_total;
     const int nl = a.layer_end - a.layer_begin;
     const int64_t total = n * nl * 2;
@@ -208,6 +216,8 @@ struct DigestRow {
 
 __global__ void __launch_bounds__(GC_NT, 3) gather_digest_kernel(GatherArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const unsigned long long A = 0x9E3779B97F4A7C15ull, B = 0xD1B54A32D192ED03ull, C = 0x8CB92BA72F3D8DD7ull,
                              D = 0xA0761D6478BD642Full;
     const int64_t n = *a.g_total;
@@ -365,10 +375,12 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
     VTK_CUDA(ctx, cudaMemsetAsync(out_digest, 0, sizeof(uint64_t) * (size_t)ctx->cfg.max_requests, st));
-    gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
-    gather_scan_kernel<<<1, 1024, 0, st>>>(a);
-    gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
-    gather_digest_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
+                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
+                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_digest_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -405,15 +417,17 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.layer_begin = layer_begin;
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
-    gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
-    gather_scan_kernel<<<1, 1024, 0, st>>>(a);
-    gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
+                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
+                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
     // the rows go through the bulk-copy rings when the context has them (vtoken_create does; the
     // context-free entry point does not), else through the register kernel
     const bool aligned = (((uintptr_t)out_k | (uintptr_t)out_v) & 15) == 0;
     if (!(aligned && vtk_launch_gather_bulk(ctx, ctx->g_src, ctx->g_total, layer_begin, layer_end, out_k, out_v,
                                             out_capacity_tokens, st)))
-        gather_copy_kernel<<<ctx->num_sms * 8, GC_NT, 0, st>>>(a);
+        VTK_CUDA(ctx, vtk_launch_dependent(gather_copy_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -452,9 +466,11 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.max_tokens = out_capacity;
     a.layer_begin = a.layer_end = 0;
     a.max_requests = ctx->cfg.max_requests;
-    gather_count_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
-    gather_scan_kernel<<<1, 1024, 0, st>>>(a);
-    gather_assign_kernel<<<ctx->cfg.max_requests * G_PARTS, G_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
+                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
+                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

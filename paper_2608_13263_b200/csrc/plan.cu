@@ -58,6 +58,8 @@ __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
 // ---- count -----------------------------------------------------------------------------
 __global__ void __launch_bounds__(PLAN_NT) plan_count_kernel(PlanArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
     if (r >= clamp_requests(a)) return;
     int64_t p0, p1;
@@ -129,6 +131,8 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
     __shared__ long long carry_need;
     __shared__ Acc carry;
     const int tid = threadIdx.x;
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int R = clamp_requests(a);
     uint32_t flags = 0;
     if (tid == 0) {
@@ -205,6 +209,8 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
 {
     __shared__ int warp_sums[PLAN_NT / 32 + 1];
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
     if (r >= clamp_requests(a)) return;
     const int tid = threadIdx.x;
@@ -313,9 +319,10 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.max_table_blocks = ctx->cfg.max_table_blocks;
 
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
-    plan_count_kernel<<<ctx->cfg.max_requests * PLAN_PARTS, PLAN_NT, 0, st>>>(a);
-    plan_scan_kernel<<<1, SCAN_NT, 0, st>>>(a);
-    plan_assign_kernel<<<ctx->cfg.max_requests * PLAN_PARTS, PLAN_NT, 0, st>>>(a);
+    const dim3 parts(ctx->cfg.max_requests * PLAN_PARTS);
+    VTK_CUDA(ctx, vtk_launch_dependent(plan_count_kernel, parts, dim3(PLAN_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(plan_scan_kernel, dim3(1), dim3(SCAN_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(plan_assign_kernel, parts, dim3(PLAN_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

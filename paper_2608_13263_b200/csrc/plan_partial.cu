@@ -89,6 +89,8 @@ __device__ __forceinline__ bool pp_moves(const PArgs &a, bool detach, int32_t b)
 template <int MODE>
 __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ int warp_n[PP_NT / 32];
     const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
     if (r >= pp_requests(a)) return;
@@ -122,6 +124,8 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
 // ---- blocks: source selection per request ------------------------------------------------------
 __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ int warp_sums[PP_NT / 32 + 1];
     const int r = blockIdx.x;
     if (r >= pp_requests(a)) return;
@@ -217,6 +221,8 @@ __device__ __forceinline__ T pp_block_incl_scan(T v, T *warp_tot, T zero, ShflUp
 
 __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ long long warp_ll[32];
     __shared__ PAcc warp_acc[32];
     __shared__ long long carry_need, tot_live, tot_blocks;
@@ -327,6 +333,8 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
 // ---- assign --------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ int warp_sums[PP_NT / 32 + 1];
     const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
     if (r >= pp_requests(a)) return;
@@ -431,6 +439,8 @@ __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_request
                                                       const int32_t *n_b, int32_t S, int32_t num_blocks,
                                                       unsigned long long *hist, vtoken_counts *counts)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     int R = *num_requests;
     R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
     const int total = bt_offsets[R];
@@ -448,6 +458,8 @@ __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_request
 __global__ void pp_summary_kernel(const int32_t *num_requests, int32_t max_requests, const int32_t *bt_offsets,
                                   const int32_t *part_n, long long *summary)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     // one warp: total live tokens over all parts, allocated blocks
     int R = *num_requests;
     R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
@@ -540,11 +552,11 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->blk_src, 0, (size_t)ctx->cfg.num_blocks, st));
-    pp_count_kernel<0><<<R * PP_PARTS, PP_NT, 0, st>>>(a);
-    pp_blocks_kernel<<<R, PP_NT, 0, st>>>(a);
-    pp_count_kernel<1><<<R * PP_PARTS, PP_NT, 0, st>>>(a);
-    pp_scan_kernel<<<1, PP_SCAN_NT, 0, st>>>(a);
-    pp_assign_kernel<<<R * PP_PARTS, PP_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_blocks_kernel, dim3(R), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<1>, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_scan_kernel, dim3(1), dim3(PP_SCAN_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_assign_kernel, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     ctx->has_plan = true;
     return VTOKEN_OK;
@@ -568,14 +580,16 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     a.n_b = n_b;
     const int R = ctx->cfg.max_requests;
     VTK_CUDA(ctx, cudaMemsetAsync(n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
-    pp_count_kernel<0><<<R * PP_PARTS, PP_NT, 0, st>>>(a);
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
     if (hist) {
         VTK_CUDA(ctx, cudaMemsetAsync(hist, 0, sizeof(uint64_t) * (size_t)(ctx->cfg.block_size + 1), st));
-        pp_hist_kernel<<<ctx->num_sms * 4, 256, 0, st>>>(num_requests, R, bt_offsets, bt_blocks, n_b,
-                                                         ctx->cfg.block_size, ctx->cfg.num_blocks,
-                                                         (unsigned long long *)hist, ctx->counts);
+        VTK_CUDA(ctx, vtk_launch_dependent(pp_hist_kernel, dim3(ctx->num_sms * 4), dim3(256), 0, st, num_requests, R,
+                                           bt_offsets, bt_blocks, (const int32_t *)n_b, ctx->cfg.block_size,
+                                           ctx->cfg.num_blocks, (unsigned long long *)hist, ctx->counts));
     }
-    if (summary) pp_summary_kernel<<<1, 32, 0, st>>>(num_requests, R, bt_offsets, ctx->part_n, (long long *)summary);
+    if (summary)
+        VTK_CUDA(ctx, vtk_launch_dependent(pp_summary_kernel, dim3(1), dim3(32), 0, st, num_requests, R, bt_offsets,
+                                           (const int32_t *)ctx->part_n, (long long *)summary));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -45,6 +45,8 @@ __global__ void __launch_bounds__(RT_NT) evict_kernel(const int32_t *num_victims
                                                       const int32_t *tt_offsets, const int32_t *tt_len,
                                                       uint8_t *keep, vtoken_counts *counts, Liveness lv)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     int n = *num_victims;
     n = n < 0 ? 0 : (n > max_victims ? max_victims : n);
     const int R = rt_requests(num_requests, max_requests);
@@ -77,6 +79,8 @@ __global__ void __launch_bounds__(RT_NT) sync_kernel(const int32_t *num_requests
                                                      const int32_t *bt_blocks, const int32_t *new_len,
                                                      int32_t num_blocks, vtoken_counts *counts, Liveness lv)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int r = blockIdx.x;
     if (r >= rt_requests(num_requests, max_requests)) return;
     const int64_t base = tt_offsets[r];
@@ -125,6 +129,8 @@ __global__ void __launch_bounds__(RT_NT) apply_moves_kernel(const int32_t *num_r
                                                             const int32_t *new_tt_slots, const int32_t *req_status,
                                                             const int32_t *new_bt_offsets, const int32_t *append_pos)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int r = blockIdx.x;
     if (r >= rt_requests(num_requests, max_requests)) return;
     const int64_t t0 = tt_offsets[r], t1 = tt_offsets[r + 1];
@@ -188,10 +194,9 @@ int vtoken_evict_tokens(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max
     if (max_victims == 0) return VTOKEN_OK;
     int grid = (max_victims + RT_NT - 1) / RT_NT;
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
-    evict_kernel<false><<<grid, RT_NT, 0, (cudaStream_t)cuda_stream>>>(num_victims, max_victims, victim_req,
-                                                                        victim_tok, num_requests,
-                                                                        ctx->cfg.max_requests, tt_offsets, tt_len,
-                                                                        keep, ctx->counts, Liveness{});
+    VTK_CUDA(ctx, vtk_launch_dependent(evict_kernel<false>, dim3(grid), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+                                       num_victims, max_victims, victim_req, victim_tok, num_requests,
+                                       ctx->cfg.max_requests, tt_offsets, tt_len, keep, ctx->counts, Liveness{}));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -209,9 +214,9 @@ int vtoken_evict_tokens_counted(vtoken_ctx *ctx, const int32_t *num_victims, int
     int grid = (max_victims + RT_NT - 1) / RT_NT;
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
     const Liveness lv{n_b, (unsigned long long *)live_total, tt_slots, ctx->slots_per_layer, ctx->cfg.block_size};
-    evict_kernel<true><<<grid, RT_NT, 0, (cudaStream_t)cuda_stream>>>(num_victims, max_victims, victim_req, victim_tok,
-                                                                       num_requests, ctx->cfg.max_requests,
-                                                                       tt_offsets, tt_len, keep, ctx->counts, lv);
+    VTK_CUDA(ctx, vtk_launch_dependent(evict_kernel<true>, dim3(grid), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+                                       num_victims, max_victims, victim_req, victim_tok, num_requests,
+                                       ctx->cfg.max_requests, tt_offsets, tt_len, keep, ctx->counts, lv));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -224,9 +229,11 @@ int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const i
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !tt_len || !phys_len || !bt_offsets ||
         !bt_blocks || !new_len)
         return VTOKEN_EINVAL;
-    sync_kernel<false><<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
-        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, tt_len, phys_len,
-        bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks, ctx->counts, Liveness{});
+    VTK_CUDA(ctx, vtk_launch_dependent(sync_kernel<false>,
+                                       dim3(ctx->cfg.max_requests), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+                                       num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots,
+                                       keep, tt_len, phys_len, bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks,
+                                       ctx->counts, Liveness{}));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -240,9 +247,11 @@ int vtoken_sync_new_tokens_counted(vtoken_ctx *ctx, const int32_t *num_requests,
         !bt_blocks || !new_len || !n_b)
         return VTOKEN_EINVAL;
     const Liveness lv{n_b, (unsigned long long *)live_total, nullptr, ctx->slots_per_layer, ctx->cfg.block_size};
-    sync_kernel<true><<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
-        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, tt_len, phys_len,
-        bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks, ctx->counts, lv);
+    VTK_CUDA(ctx, vtk_launch_dependent(sync_kernel<true>,
+                                       dim3(ctx->cfg.max_requests), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+                                       num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots,
+                                       keep, tt_len, phys_len, bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks,
+                                       ctx->counts, lv));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -254,9 +263,10 @@ int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32
 {
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTOKEN_EINVAL;
     if (phys_len && !req_status) return VTOKEN_EINVAL;
-    apply_moves_kernel<<<ctx->cfg.max_requests, RT_NT, 0, (cudaStream_t)cuda_stream>>>(
-        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots, keep, phys_len, new_tt_slots,
-        req_status, new_bt_offsets, append_pos);
+    VTK_CUDA(ctx, vtk_launch_dependent(apply_moves_kernel,
+                                       dim3(ctx->cfg.max_requests), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+                                       num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots,
+                                       keep, phys_len, new_tt_slots, req_status, new_bt_offsets, append_pos));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -20,6 +20,8 @@ __global__ void __launch_bounds__(256) slot_cache_mark_kernel(uint8_t *dirty, co
                                                               const int32_t *req_status, const int32_t *num_requests,
                                                               int32_t max_requests)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int R = sc_requests(num_requests, max_requests);
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsz = gridDim.x * blockDim.x;
     if (victim_req != nullptr && num_victims != nullptr) {
@@ -43,6 +45,8 @@ __global__ void __launch_bounds__(SC_NT) slot_cache_update_kernel(const int32_t 
                                                                   int32_t *cache_seen, int32_t *stats,
                                                                   int64_t slots_per_layer, vtoken_counts *counts)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     __shared__ int warp_sums[SC_NT / 32 + 1];
     const int r = blockIdx.x;
     if (r >= sc_requests(num_requests, max_requests)) return;
@@ -102,9 +106,11 @@ int vtoken_slot_cache_mark(vtoken_ctx *ctx, uint8_t *dirty, const int32_t *num_v
     const int64_t span = max_victims > ctx->cfg.max_requests ? max_victims : ctx->cfg.max_requests;
     int grid = (int)((span + 255) / 256);
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
-    slot_cache_mark_kernel<<<grid, 256, 0, (cudaStream_t)cuda_stream>>>(
-        dirty, max_victims > 0 ? num_victims : nullptr, max_victims, max_victims > 0 ? victim_req : nullptr,
-        req_status, num_requests, ctx->cfg.max_requests);
+    VTK_CUDA(ctx, vtk_launch_dependent(slot_cache_mark_kernel, dim3(grid), dim3(256), 0, (cudaStream_t)cuda_stream,
+                                       dirty,
+                                       max_victims > 0 ? num_victims : nullptr, max_victims,
+                                       max_victims > 0 ? victim_req : nullptr, req_status, num_requests,
+                                       ctx->cfg.max_requests));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -119,9 +125,10 @@ int vtoken_slot_cache_update(vtoken_ctx *ctx, const int32_t *num_requests, const
         return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (stats) VTK_CUDA(ctx, cudaMemsetAsync(stats, 0, 2 * sizeof(int32_t), st));
-    slot_cache_update_kernel<<<ctx->cfg.max_requests, SC_NT, 0, st>>>(
-        num_requests, ctx->cfg.max_requests, tt_offsets, tt_slots, keep, tt_len, dirty, cache_slots, cache_ids,
-        cache_len, cache_seen, stats, ctx->slots_per_layer, ctx->counts);
+    VTK_CUDA(ctx, vtk_launch_dependent(slot_cache_update_kernel,
+                                       dim3(ctx->cfg.max_requests), dim3(SC_NT), 0, st, num_requests,
+                                       ctx->cfg.max_requests, tt_offsets, tt_slots, keep, tt_len, dirty, cache_slots,
+                                       cache_ids, cache_len, cache_seen, stats, ctx->slots_per_layer, ctx->counts));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

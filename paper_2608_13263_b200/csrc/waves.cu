@@ -29,6 +29,8 @@ struct CommitArgs {
 
 __global__ void __launch_bounds__(COMMIT_NT) wave_commit_kernel(CommitArgs a)
 {
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
     const int gtid = blockIdx.x * COMMIT_NT + threadIdx.x, gsz = gridDim.x * COMMIT_NT;
     int R = *a.num_requests;
     R = R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
@@ -167,7 +169,7 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         int blocks = (int)((span + COMMIT_NT - 1) / COMMIT_NT);
         if (blocks < 1) blocks = 1;
         if (blocks > ctx->num_sms * 8) blocks = ctx->num_sms * 8;
-        wave_commit_kernel<<<blocks, COMMIT_NT, 0, st>>>(a);
+        VTK_CUDA(ctx, vtk_launch_dependent(wave_commit_kernel, dim3(blocks), dim3(COMMIT_NT), 0, st, a));
         VTK_CUDA(ctx, cudaGetLastError());
 
         cur.bt_offsets = po.new_bt_offsets;

@@ -146,6 +146,35 @@ def test_copy_work_distribution_modes(dynamic, chunk, monkeypatch):
     prob.close()
 
 
+@pytest.mark.parametrize("pdl", ["0", "1"])
+def test_launch_modes_give_the_same_result(pdl, monkeypatch):
+    """Plain stream-ordered launches and programmatic dependent launches (a kernel may become resident
+    while its predecessor finishes and waits for it on the device): the same tables and bytes, for both
+    copy paths, with launches issued back to back on one stream without host synchronisation between
+    plan, copy and the next plan."""
+    monkeypatch.setenv("VTOKEN_PDL", pdl)
+    from paper_2608_13263_b200.device import DeviceProblem
+    torch = _torch()
+    for variant in (1, 2):
+        run_and_compare(wl.mistral7b_random(seed=9, requests=6, lo=80, hi=600, layers=2), copy_variant=variant)
+        w = wl.llama8b_h2o(seed=4, requests=6, lo=200, hi=900, layers=2)
+        prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=variant)
+        p = vto.plan_workload(w)
+        k, v = host_pools(w)
+        vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+        st = torch.cuda.Stream()
+        with torch.cuda.stream(st):
+            for _ in range(5):                           # nothing but stream order between these launches
+                prob.fill_pools(stream=st)
+                prob.plan(stream=st)
+                prob.repack(stream=st)
+        st.synchronize()
+        assert_tables_equal(prob.outputs(), p, w)
+        assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+        assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+        prob.close()
+
+
 def _request(n_tokens, S, first_block):
     nb = -(-n_tokens // S)
     bt = np.arange(first_block, first_block + nb, dtype=np.int32)

@@ -102,7 +102,10 @@ enum {
     VTOKEN_FLAG_BAD_SLOT = 1u,        /* a token-table slot >= num_blocks * block_size: token treated as not live */
     VTOKEN_FLAG_BAD_BLOCK = 2u,       /* a block-table id outside [0, num_blocks) */
     VTOKEN_FLAG_BAD_FREE = 4u,        /* a free-list id outside [0, num_blocks): that destination block is skipped */
-    VTOKEN_FLAG_CAPACITY = 8u,        /* R, T or the block total above the create-time capacities: clamped */
+    VTOKEN_FLAG_CAPACITY = 8u,        /* R, num_free, or a table range beyond the create-time capacities: R and
+                                         num_free are clamped; table entries at or beyond max_tokens /
+                                         max_table_blocks (and ranges that run backwards) do not exist for the
+                                         planners, so no output buffer is written behind its capacity */
     VTOKEN_FLAG_TIMEOUT = 16u,        /* a bounded wait inside a kernel ran out; rows may be missing */
     VTOKEN_FLAG_GATHER_OVERFLOW = 32u,/* gather_logical / build_slot_mapping: more live tokens than the output holds */
     VTOKEN_FLAG_BAD_VICTIM = 64u,     /* vtoken_evict_tokens: a victim outside its request's registered tokens: skipped */

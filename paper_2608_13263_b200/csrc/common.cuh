@@ -166,6 +166,17 @@ __device__ __forceinline__ int vtk_block_rank(bool flag, int *warp_sums, int &to
     return rank;
 }
 
+// Range [off[r], off[r+1]) of request r in a CSR table, clipped to the create-time capacity of that
+// table: entries at or beyond `cap` (and ranges that run backwards) do not exist for the planners,
+// whose output buffers are sized by the capacities.  Returns true when something was clipped.
+__device__ __forceinline__ bool vtk_range(const int32_t *off, int r, int64_t cap, int64_t &lo, int64_t &hi)
+{
+    const int64_t a = off[r], b = off[r + 1];
+    lo = a < 0 ? 0 : (a > cap ? cap : a);
+    hi = b < lo ? lo : (b > cap ? cap : b);
+    return lo != a || hi != b;
+}
+
 // A token is live when it owns a slot inside the pool and the policy kept it.
 __device__ __forceinline__ bool vtk_live(int32_t slot, const uint8_t *keep, int64_t t, int64_t slots_per_layer,
                                          bool &bad_slot)

@@ -62,8 +62,9 @@ __global__ void __launch_bounds__(PLAN_NT) plan_count_kernel(PlanArgs a)
     vtk_wait_for_predecessor();
     const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
     if (r >= clamp_requests(a)) return;
-    int64_t p0, p1;
-    part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
+    int64_t t0, t1, p0, p1;
+    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
+    part_range(t0, t1, c, p0, p1);
     int n = 0;
     bool bad = false;
     for (int64_t t = p0 + threadIdx.x; t < p1; t += PLAN_NT)
@@ -137,8 +138,6 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
     uint32_t flags = 0;
     if (tid == 0) {
         if (*a.num_requests > a.max_requests || *a.num_requests < 0) flags |= VTOKEN_FLAG_CAPACITY;
-        if (R > 0 && ((int64_t)a.tt_offsets[R] > a.max_tokens || (int64_t)a.bt_offsets[R] > a.max_table_blocks))
-            flags |= VTOKEN_FLAG_CAPACITY;
         carry_need = 0;
         carry = Acc{0, 0, 0, 0, 0, 0};
     }
@@ -158,8 +157,11 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 #pragma unroll
             for (int c = 0; c < PLAN_PARTS; ++c) n += a.part_n[r * PLAN_PARTS + c];
             a.req_n[r] = n;
-            nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
-            if (nb < 0) nb = 0;
+            int64_t lo, hi, t0, t1;
+            const bool clipped = vtk_range(a.bt_offsets, r, a.max_table_blocks, lo, hi) |
+                                 vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
+            if (clipped) flags |= VTOKEN_FLAG_CAPACITY;     // tables beyond the create-time capacities
+            nb = (int)(hi - lo);
         }
         const int need = (int)(((int64_t)n + a.S - 1) / a.S);       // ceil(T_live / S)
         bool sel = valid && (a.select == nullptr || a.select[r] != 0);
@@ -189,6 +191,8 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         }
         __syncthreads();
     }
+    if (flags) atomicOr(&a.counts->error_flags, flags);
+    __syncthreads();
     if (tid == 0) {
         a.new_bt_offsets[R] = carry.newbt;
         vtoken_counts c;
@@ -198,7 +202,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         c.num_free_consumed = carry.dst;
         c.num_admitted = carry.admitted;
         c.num_deferred = carry.deferred;
-        c.error_flags = flags | a.counts->error_flags;   // bits raised by the count kernel
+        c.error_flags = atomicOr(&a.counts->error_flags, 0u);   // bits raised by the count kernel and above
         c.num_released = 0;
         *a.counts = c;
         *a.out_counts = c;                               // later flags are OR-ed into both copies
@@ -215,8 +219,10 @@ __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
     if (r >= clamp_requests(a)) return;
     const int tid = threadIdx.x;
     const int S = a.S;
-    const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
-    const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
+    int64_t t0, t1, b0, b1;
+    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
+    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
+    const int nb = (int)(b1 - b0);
     const bool adm = a.req_status[r] == VTOKEN_REPACKED;
     const int n = a.req_n[r];
     const int need = (int)(((int64_t)n + S - 1) / S);
@@ -229,12 +235,12 @@ __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
     if (adm) {
         for (int j = stripe; j < need; j += stride) {
             int blk = a.free_blocks[dst_base + j];
-            a.new_bt_blocks[nbt0 + j] = blk;
+            if ((int64_t)nbt0 + j < a.max_table_blocks) a.new_bt_blocks[nbt0 + j] = blk;
             if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
             a.dst_blocks[dst_base + j] = blk;
         }
         const int f0 = a.req_freed_base[r];
-        for (int j = stripe; j < b1 - b0; j += stride) {
+        for (int j = stripe; j < nb && (int64_t)f0 + j < a.max_table_blocks; j += stride) {
             const int blk = a.bt_blocks[b0 + j];
             if (blk < 0 || blk >= a.num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
             a.freed_blocks[f0 + j] = blk;
@@ -242,7 +248,8 @@ __global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
         // unused tail of the last destination block
         for (int i = n + stripe; i < need * S; i += stride) a.dst_src[(int64_t)dst_base * S + i] = -1;
     } else {
-        for (int j = stripe; j < b1 - b0; j += stride) a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
+        for (int j = stripe; j < nb && (int64_t)nbt0 + j < a.max_table_blocks; j += stride)
+            a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
     }
 
     // token table: rank of each live token in logical order -> destination slot

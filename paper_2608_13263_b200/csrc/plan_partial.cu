@@ -94,8 +94,9 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
     __shared__ int warp_n[PP_NT / 32];
     const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
     if (r >= pp_requests(a)) return;
-    int64_t p0, p1;
-    pp_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
+    int64_t t0, t1, p0, p1;
+    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
+    pp_part_range(t0, t1, c, p0, p1);
     const bool may_detach = a.protect != nullptr && a.detach_den != 0;
     const bool detach = MODE == 1 && may_detach && a.req_detach[r] != 0;
     int n = 0, n_shared = 0;
@@ -129,12 +130,13 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
     __shared__ int warp_sums[PP_NT / 32 + 1];
     const int r = blockIdx.x;
     if (r >= pp_requests(a)) return;
-    const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
+    int64_t b0, b1;
+    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
     int carry = 0;               // eligible entries before this chunk
     int shared = 0;              // protected entries seen by this thread
     uint32_t flags = 0;
-    for (int jb = b0; jb < b1; jb += PP_NT) {
-        const int j = jb + threadIdx.x;
+    for (int64_t jb = b0; jb < b1; jb += PP_NT) {
+        const int64_t j = jb + threadIdx.x;
         bool eligible = false;
         int blk = -1;
         if (j < b1) {
@@ -232,8 +234,6 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     uint32_t flags = 0;
     if (tid == 0) {
         if (*a.num_requests > a.max_requests || *a.num_requests < 0) flags |= VTOKEN_FLAG_CAPACITY;
-        if (R > 0 && ((int64_t)a.tt_offsets[R] > a.max_tokens || (int64_t)a.bt_offsets[R] > a.max_table_blocks))
-            flags |= VTOKEN_FLAG_CAPACITY;
         carry_need = 0;
         tot_live = 0;
         tot_blocks = 0;
@@ -257,9 +257,11 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         }
         a.req_n[r] = n;
         a.req_nsrc[r] = nsrc;
-        int nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
+        int64_t lo, hi, t0, t1;
+        if (vtk_range(a.bt_offsets, r, a.max_table_blocks, lo, hi) | vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1))
+            flags |= VTOKEN_FLAG_CAPACITY;                  // tables beyond the create-time capacities
         my_live += n;
-        my_blocks += nb < 0 ? 0 : nb;
+        my_blocks += hi - lo;
     }
     const long long live_incl = pp_block_incl_scan<long long>(my_live, warp_ll, 0LL, shfl_ll);
     if (tid == PP_SCAN_NT - 1) tot_live = live_incl;
@@ -283,8 +285,9 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
             nsrc = a.req_nsrc[r];
             ns = a.req_ns[r];
             nrel = may_detach ? a.req_shared[r] : 0;     // protected sources: released, not reclaimed
-            nb = a.bt_offsets[r + 1] - a.bt_offsets[r];
-            if (nb < 0) nb = 0;
+            int64_t lo, hi;
+            vtk_range(a.bt_offsets, r, a.max_table_blocks, lo, hi);
+            nb = (int)(hi - lo);
         }
         const int need = (int)(((int64_t)nsrc + a.S - 1) / a.S);   // ceil(T_live / S) over the source blocks
         bool sel = valid && triggered && (a.select == nullptr || a.select[r] != 0);
@@ -314,6 +317,8 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         }
         __syncthreads();
     }
+    if (flags) atomicOr(&a.counts->error_flags, flags);
+    __syncthreads();
     if (tid == 0) {
         a.new_bt_offsets[R] = carry.newbt;
         vtoken_counts c;
@@ -323,7 +328,7 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         c.num_free_consumed = carry.dst;
         c.num_admitted = carry.admitted;
         c.num_deferred = carry.deferred;
-        c.error_flags = flags | a.counts->error_flags;
+        c.error_flags = atomicOr(&a.counts->error_flags, 0u);   // bits raised by the kernels before and above
         c.num_released = carry.released;
         *a.counts = c;
         *a.out_counts = c;
@@ -340,9 +345,11 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
     if (r >= pp_requests(a)) return;
     const int tid = threadIdx.x;
     const int S = a.S;
-    const int64_t t0 = a.tt_offsets[r], t1 = a.tt_offsets[r + 1];
-    const int b0 = a.bt_offsets[r], b1 = a.bt_offsets[r + 1];
-    const int nb = b1 - b0;
+    int64_t t0, t1, b0, b1;
+    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
+    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
+    const int nb = (int)(b1 - b0);
+    const int64_t cap_bt = a.max_table_blocks;               // every table write below stays inside its buffer
     const bool adm = a.req_status[r] == VTOKEN_REPACKED;
     const bool detach = adm && a.protect != nullptr && a.detach_den != 0 && a.req_detach[r] != 0;
     const int nsrc = a.req_nsrc[r], ns = a.req_ns[r];
@@ -356,7 +363,7 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
         // destinations follow the kept blocks in the new block table
         for (int j = stripe; j < need; j += stride) {
             int blk = a.free_blocks[dst_base + j];
-            a.new_bt_blocks[nbt0 + (nb - ns) + j] = blk;
+            if ((int64_t)nbt0 + (nb - ns) + j < cap_bt) a.new_bt_blocks[nbt0 + (nb - ns) + j] = blk;
             if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
             a.dst_blocks[dst_base + j] = blk;
         }
@@ -367,8 +374,8 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
             const int f0 = a.req_freed_base[r];
             const int l0 = detach ? a.req_rel_base[r] : 0;
             int carry_src = 0, carry_rel = 0;
-            for (int jb = b0; jb < b1; jb += PP_NT) {
-                const int j = jb + tid;
+            for (int64_t jb = b0; jb < b1; jb += PP_NT) {
+                const int64_t j = jb + tid;
                 int blk = -1;
                 bool src = false, rel = false;
                 if (j < b1) {
@@ -387,14 +394,16 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
                     carry_rel += total;
                 }
                 if (j < b1) {
-                    if (src) a.freed_blocks[f0 + rank_src] = blk;
-                    else if (rel) a.released_blocks[l0 + rank_rel] = blk;
-                    else a.new_bt_blocks[nbt0 + (j - b0) - rank_src - rank_rel] = blk;   // entries before it that stay
+                    const int64_t kept = (int64_t)nbt0 + (j - b0) - rank_src - rank_rel;   // entries before it that stay
+                    if (src) { if ((int64_t)f0 + rank_src < cap_bt) a.freed_blocks[f0 + rank_src] = blk; }
+                    else if (rel) { if ((int64_t)l0 + rank_rel < cap_bt) a.released_blocks[l0 + rank_rel] = blk; }
+                    else if (kept < cap_bt) a.new_bt_blocks[kept] = blk;
                 }
             }
         }
     } else {
-        for (int j = stripe; j < nb; j += stride) a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
+        for (int j = stripe; j < nb && (int64_t)nbt0 + j < cap_bt; j += stride)
+            a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
     }
 
     // token table

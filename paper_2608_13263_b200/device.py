@@ -17,7 +17,8 @@ from .workloads import Workload
 
 class DeviceProblem:
     def __init__(self, w: Workload, device="cuda:0", fill_seed: int = 1, copy_variant: int = 0, max_ctas: int = 0,
-                 capacity_slack: int = 0, allocate_pools: bool = True, wave_capacity: bool = False):
+                 capacity_slack: int = 0, allocate_pools: bool = True, wave_capacity: bool = False,
+                 ctx_capacity: dict = None):
         self.w = w
         self.device = torch.device(device)
         self.fill_seed = fill_seed
@@ -63,9 +64,12 @@ class DeviceProblem:
             self.k_pool = torch.empty(shape, dtype=torch.int16, device=dev)
             self.v_pool = torch.empty(shape, dtype=torch.int16, device=dev)
             self.fill_pools()
+            caps = dict(max_requests=self.max_requests, max_tokens=self.max_tokens,
+                        max_table_blocks=self.max_table_blocks, max_free=self.max_free)
+            caps.update(ctx_capacity or {})     # a context smaller than the buffers (capacity tests)
             self.ctx = vt.vtoken_create(w.num_layers, w.num_blocks, w.block_size, w.num_kv_heads, w.head_dim,
-                                        self.k_pool, self.v_pool, self.max_requests, self.max_tokens,
-                                        self.max_table_blocks, self.max_free, elem_bytes=w.elem_bytes,
+                                        self.k_pool, self.v_pool, caps["max_requests"], caps["max_tokens"],
+                                        caps["max_table_blocks"], caps["max_free"], elem_bytes=w.elem_bytes,
                                         max_ctas=max_ctas, copy_variant=copy_variant)
 
     def _padded(self, a, dtype, n):

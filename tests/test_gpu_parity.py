@@ -338,6 +338,44 @@ def test_counts_above_capacity_are_clamped_and_flagged():
     prob.close()
 
 
+@pytest.mark.parametrize("planner", ["whole", "partial"])
+def test_tables_beyond_the_context_capacities_are_clipped(planner):
+    """Token and block tables longer than the capacities the context was created with: entries at or
+    beyond a capacity do not exist for the planner (the result is the oracle's on the clipped tables),
+    VTOKEN_FLAG_CAPACITY is raised, and nothing is written behind a capacity in any output buffer."""
+    from paper_2608_13263_b200.device import DeviceProblem
+    w = wl.mistral7b_random(seed=21, requests=9, lo=60, hi=400, layers=1, heads=1, head_dim=64)
+    T, NBT = w.num_tokens, len(w.bt_blocks)
+    cap_t, cap_b = T - 157, NBT - 5                      # cuts into the last request (and the one before it)
+    assert cap_t < w.tt_offsets[-2] + 40 and cap_b > w.bt_offsets[-2] - 3
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, ctx_capacity=dict(max_tokens=cap_t, max_table_blocks=cap_b))
+    if planner == "whole":
+        prob.plan()
+    else:
+        prob.plan_partial()
+    prob.repack()
+    out = prob.outputs()
+    assert out["error_flags"] == vt.FLAG_CAPACITY
+    tt_off = np.minimum(w.tt_offsets, cap_t).astype(np.int32)
+    bt_off = np.minimum(w.bt_offsets, cap_b).astype(np.int32)
+    p = vto.plan(w.block_size, bt_off, w.bt_blocks[:cap_b], tt_off, w.tt_slots[:cap_t], w.keep[:cap_t], w.free_blocks)
+    assert p.num_admitted > 0
+    assert np.array_equal(out["req_status"], p.req_status)
+    assert np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
+    nbt = int(p.new_bt_offsets[-1])
+    assert np.array_equal(prob.new_bt_blocks[:nbt].cpu().numpy(), p.new_bt_blocks)
+    assert np.array_equal(prob.new_tt_slots[:cap_t].cpu().numpy(), p.new_tt_slots)
+    assert np.array_equal(prob.freed_blocks[:p.num_freed].cpu().numpy(), p.freed_blocks)
+    assert (prob.new_tt_slots[cap_t:].cpu().numpy() == -9).all()
+    assert (prob.new_bt_blocks[nbt:].cpu().numpy() == -9).all()
+    assert (prob.freed_blocks[p.num_freed:].cpu().numpy() == -9).all()
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()
+
+
 def test_argument_errors():
     from paper_2608_13263_b200.device import DeviceProblem
     w = wl.tiny()

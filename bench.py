@@ -733,8 +733,29 @@ def run_runtime(args, prob, w, side, dev):
                                     keep=keep2_d, tt_len=tt_len, dirty=s_dirty, cache_slots=s_slots, cache_ids=s_ids,
                                     cache_len=s_len, cache_seen=s_seen, stream=st)
 
+    # eligibility metadata (live tokens per block, utilisation histogram, totals behind F) and the
+    # input-precondition checker over the same tables
+    n_b = torch.zeros(w.num_blocks, **i32)
+    hist = torch.zeros(w.block_size + 1, dtype=torch.int64, device=dev)
+    summary = torch.zeros(4, dtype=torch.int64, device=dev)
+    check_bits = torch.zeros(1, **i32)
+
+    def liveness(st):
+        vt.vtoken_block_liveness(prob.ctx, num_requests=prob.num_requests, bt_offsets=prob.bt_offsets,
+                                 bt_blocks=prob.bt_blocks, tt_offsets=prob.tt_offsets, tt_slots=prob.tt_slots,
+                                 keep=prob.keep, n_b=n_b, hist=hist, summary=summary, stream=st)
+
+    def check(st):
+        vt.vtoken_check_tables(prob.ctx, num_requests=prob.num_requests, bt_offsets=prob.bt_offsets,
+                               bt_blocks=prob.bt_blocks, tt_offsets=prob.tt_offsets, tt_slots=prob.tt_slots,
+                               free_blocks=prob.free_blocks, num_free=prob.num_free, out_bits=check_bits, stream=st)
+
+    NBT = len(w.bt_blocks)
     out = {}
-    table_bytes = {"decode_step_policy_adapter": 2 * (4 * R + n2) + R * 60 + 5 * n2 + 8 * live,
+    table_bytes = {"block_liveness": 5 * T + 4 * live + 2 * 4 * w.num_blocks + 2 * 4 * NBT,
+                   "check_tables": 4 * T + 2 * 4 * NBT + 4 * len(w.free_blocks) + 2 * 4 * w.num_blocks
+                                   + w.slots_per_layer // 8,
+                   "decode_step_policy_adapter": 2 * (4 * R + n2) + R * 60 + 5 * n2 + 8 * live,
                    "slot_cache_rebuild_all": 5 * T + 8 * live, "slot_cache_append_one_token_per_request": R * 40,
                    "slot_cache_nothing_changed": R * 13,
                    "slot_mapping": 2 * 5 * T + 8 * live, "append_one_token_per_request": R * (4 * 6 + 5),
@@ -744,7 +765,8 @@ def run_runtime(args, prob, w, side, dev):
                      ("evict_64k_victims", evict), ("apply_moves", commit), ("digest_all_layers", digest),
                      ("gather_logical", gather), ("slot_cache_rebuild_all", cache_rebuild),
                      ("slot_cache_append_one_token_per_request", cache_append),
-                     ("slot_cache_nothing_changed", cache_update), ("decode_step_policy_adapter", decode_step)):
+                     ("slot_cache_nothing_changed", cache_update), ("decode_step_policy_adapter", decode_step),
+                     ("block_liveness", liveness), ("check_tables", check)):
         with torch.cuda.stream(side):
             fn(side)
         side.synchronize()
@@ -763,6 +785,9 @@ def run_runtime(args, prob, w, side, dev):
         side.synchronize()
         us = e0.elapsed_time(e1) / reps * 1e3
         out[name] = {"us": us, "table_bytes": table_bytes[name], "GBs": table_bytes[name] / us / 1e3}
+    side.synchronize()
+    out["check_tables"]["bits"] = int(check_bits.cpu()[0])        # 0: the workload's tables are valid
+    out["block_liveness"]["fragmentation_F"] = 1.0 - float(summary[0]) / max(1.0, float(summary[1]) * w.block_size)
     out["entries"] = {"logical_tokens": T, "live_tokens": live, "requests": R, "gather_layers": g_layers}
     out["decode_step_note"] = ("one step for all requests: sync_new_tokens (one token each), evict_tokens (one victim "
                                "each), slot-cache mark + update (every request rebuilt); includes two device copies "

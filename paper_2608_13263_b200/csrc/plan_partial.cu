@@ -101,15 +101,21 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
     const bool detach = MODE == 1 && may_detach && a.req_detach[r] != 0;
     int n = 0, n_shared = 0;
     bool bad = false;
-    for (int64_t t = p0 + threadIdx.x; t < p1; t += PP_NT) {
-        const int32_t slot = a.tt_slots[t];
-        if (!vtk_live(slot, a.keep, t, a.slots_per_layer, bad)) continue;
+    for (int64_t tb = p0; tb < p1; tb += PP_NT) {           // the same trip count for every thread of the CTA
+        const int64_t t = tb + threadIdx.x;
+        int blk = -1;                                        // block of this thread's token, -1: not live
+        if (t < p1) {
+            const int32_t slot = a.tt_slots[t];
+            if (vtk_live(slot, a.keep, t, a.slots_per_layer, bad)) blk = slot / a.S;
+        }
         if (MODE == 0) {
-            atomicAdd(&a.n_b[slot / a.S], 1);
-            ++n;
-            if (may_detach) n_shared += a.protect[slot / a.S] != 0;
-        } else {
-            n += pp_moves(a, detach, slot / a.S);
+            if (blk >= 0) {
+                atomicAdd(&a.n_b[blk], 1);
+                ++n;
+                if (may_detach) n_shared += a.protect[blk] != 0;
+            }
+        } else if (blk >= 0) {
+            n += pp_moves(a, detach, blk);
         }
     }
     if (bad && MODE == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
@@ -443,6 +449,8 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
 }
 
 // ---- histogram of block utilisation ------------------------------------------------------------
+constexpr int PP_HIST_BINS = 1024;      // bins a CTA keeps in shared memory (block sizes up to 1023)
+
 __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_requests, int32_t max_requests,
                                                       const int32_t *bt_offsets, const int32_t *bt_blocks,
                                                       const int32_t *n_b, int32_t S, int32_t num_blocks,
@@ -450,6 +458,13 @@ __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_request
 {
     vtk_release_successor();
     vtk_wait_for_predecessor();
+    // a handful of bins takes every increment: counted per CTA in shared memory first, one global
+    // atomic per non-empty bin and CTA afterwards (integer sums: the order does not matter)
+    __shared__ unsigned int bins[PP_HIST_BINS];
+    const bool local = S < PP_HIST_BINS;
+    if (local)
+        for (int k = threadIdx.x; k <= S; k += 256) bins[k] = 0;
+    __syncthreads();
     int R = *num_requests;
     R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
     const int total = bt_offsets[R];
@@ -459,26 +474,40 @@ __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_request
         if (blk < 0 || blk >= num_blocks) { bad = true; continue; }
         int k = n_b[blk];
         if (k > S) k = S;
-        atomicAdd(&hist[k], 1ull);
+        if (local) atomicAdd(&bins[k], 1u);
+        else atomicAdd(&hist[k], 1ull);
     }
     if (bad) atomicOr(&counts->error_flags, VTOKEN_FLAG_BAD_BLOCK);
+    __syncthreads();
+    if (local)
+        for (int k = threadIdx.x; k <= S; k += 256)
+            if (bins[k] != 0) atomicAdd(&hist[k], (unsigned long long)bins[k]);
 }
 
-__global__ void pp_summary_kernel(const int32_t *num_requests, int32_t max_requests, const int32_t *bt_offsets,
-                                  const int32_t *part_n, long long *summary)
+__global__ void __launch_bounds__(1024) pp_summary_kernel(const int32_t *num_requests, int32_t max_requests,
+                                                          const int32_t *bt_offsets, const int32_t *part_n,
+                                                          long long *summary)
 {
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    // one warp: total live tokens over all parts, allocated blocks
+    // one CTA: total live tokens over all parts, allocated blocks
+    __shared__ long long warp_s[32];
     int R = *num_requests;
     R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
     long long s = 0;
-    for (int i = threadIdx.x; i < R * PP_PARTS; i += 32) s += part_n[i];
+    for (int i = threadIdx.x; i < R * PP_PARTS; i += 1024) s += part_n[i];
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
-    if (threadIdx.x == 0) {
-        summary[0] = s;
-        summary[1] = bt_offsets[R];
+    if (vtk_lane() == 0) warp_s[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        s = warp_s[threadIdx.x];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
+        if (threadIdx.x == 0) {
+            summary[0] = s;
+            summary[1] = bt_offsets[R];
+        }
     }
 }
 
@@ -597,7 +626,7 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
                                            ctx->cfg.num_blocks, (unsigned long long *)hist, ctx->counts));
     }
     if (summary)
-        VTK_CUDA(ctx, vtk_launch_dependent(pp_summary_kernel, dim3(1), dim3(32), 0, st, num_requests, R, bt_offsets,
+        VTK_CUDA(ctx, vtk_launch_dependent(pp_summary_kernel, dim3(1), dim3(1024), 0, st, num_requests, R, bt_offsets,
                                            (const int32_t *)ctx->part_n, (long long *)summary));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;

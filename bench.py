@@ -32,7 +32,7 @@ from paper_2608_13263_b200 import workloads as wl  # noqa: E402
 METRIC = "repack HBM GB/s (read+write); live tokens repacked/s and fraction of HBM peak in the same line"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-KERNELS_PER_STEP = 4        # plan: count, scan, assign; copy: 1
+KERNELS_PER_STEP = 4        # plan: tiles, scan, assign; copy: 1
 
 
 def measured_peak():

@@ -23,7 +23,7 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 
 void free_all(vtoken_ctx *ctx)
 {
-    void *ptrs[] = {ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
+    void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->blk_src, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
@@ -122,6 +122,9 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->req_n, cfg->max_requests);
     A(&ctx->part_n, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
     A(&ctx->req_dst_base, cfg->max_requests);
+    A(&ctx->tile_n, (cfg->max_tokens + 1023) / 1024 + 1);
+    A(&ctx->req_part, (int64_t)cfg->max_requests + 1);
+    A(&ctx->req_before, (int64_t)cfg->max_requests + 1);
     A(&ctx->req_freed_base, cfg->max_requests);
     A(&ctx->req_status, cfg->max_requests);
     A(&ctx->dst_src, cap * cfg->block_size);

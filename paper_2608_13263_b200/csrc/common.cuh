@@ -29,6 +29,9 @@ struct vtoken_ctx {
     int32_t *dst_src;          // [cap_dst_blocks * S] inverse plan: source slot of each destination slot, -1 = none
     int32_t *dst_blocks;       // [cap_dst_blocks] physical id of each destination block, -1 = skip
     vtoken_counts *counts;     // one struct
+    int32_t *tile_n;           // [ceil(max_tokens / 1024) + 1] live tokens per tile of the token table, then scanned
+    int32_t *req_part;         // [max_requests + 1] live tokens between a request's tile start and its first entry
+    int32_t *req_before;       // [max_requests + 1] live tokens of the table before the request's first entry
 
     // partial-plan scratch (DEVICE)
     int32_t *part_src;         // [max_requests * VTK_PLAN_PARTS] live tokens in source blocks per request part

@@ -1,19 +1,27 @@
-// Relocation planner (Sec. 3.3.3 of the paper) as three small kernels:
-//   count  : live tokens per request part                (warp ballot + popc)
-//   scan   : candidates, admission against the free list, per-request bases, counts (one CTA)
-//   assign : rank of every live token -> destination slot, new tables, reclaimed list,
-//            inverse move plan for the copy kernel
-// Every request is cut into PLAN_PARTS equal token ranges, one CTA each in count and assign, so
-// that a 32k-token request does not serialise on one CTA; a part's first rank is the sum of the
-// live counts of the parts before it.  All grids are fixed by the capacities; R, T and num_free
-// are read from device memory.  No output order depends on atomics.
+// Relocation planner (Sec. 3.3.3 of the paper) as three small kernels over a flat tiling of the
+// token table:
+//   tiles  : live tokens per tile of 1024 consecutive table entries (four per thread, vector
+//            loads), and for every request the live tokens between the start of its first tile and
+//            its first entry
+//   scan   : running live count at every tile start; live tokens per request as a difference of
+//            two running counts; candidates, admission against the free list, per-request bases,
+//            counts (one CTA)
+//   assign : rank of every live token inside its request = running count at the token minus the
+//            running count at the request's first entry -> destination slot, new token table,
+//            inverse move plan for the copy kernel; extra CTAs (one per request) write the new
+//            block tables and the reclaimed list
+// The tiling ignores request boundaries, so the work per CTA is the same whatever the mix of
+// request lengths (512 short requests or 32 long ones), and every CTA keeps four table entries
+// per thread in flight.  All grids are fixed by the capacities; R, T and num_free are read from
+// device memory.  No output order depends on atomics.
 #include "common.cuh"
 
 namespace {
 
-constexpr int PLAN_NT = 512;    // threads per CTA of count / assign
-constexpr int PLAN_PARTS = VTK_PLAN_PARTS;   // token ranges per request
-constexpr int SCAN_NT = 1024;   // threads of the single scan CTA
+constexpr int TILE_NT = 256;                     // threads per CTA of tiles / assign
+constexpr int TILE_TOK = 4;                      // table entries per thread
+constexpr int TILE = TILE_NT * TILE_TOK;         // entries per tile
+constexpr int SCAN_NT = 1024;                    // threads of the single scan CTA
 
 struct PlanArgs {
     // inputs
@@ -25,9 +33,15 @@ struct PlanArgs {
     int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *out_status;
     vtoken_counts *out_counts;
     // context
-    int32_t *req_n, *part_n, *req_dst_base, *req_freed_base, *req_status, *dst_src, *dst_blocks;
+    int32_t *req_n, *req_dst_base, *req_freed_base, *req_status, *dst_src, *dst_blocks;
+    int32_t *tile_n;        // [num_tiles + 1] live tokens per tile (sign bit: a slot outside the pool); after the
+                            // scan: live tokens before the tile
+    int32_t *req_part;      // [max_requests + 1] live tokens between the start of the tile that holds the
+                            // request's first entry and that entry
+    int32_t *req_before;    // [max_requests + 1] live tokens before the request's first entry
     vtoken_counts *counts;
-    int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
+    int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks, num_tiles;
+    int32_t vec_in, vec_out;   // tt_slots 16-byte / keep 4-byte aligned; new_tt_slots 16-byte aligned
     int64_t slots_per_layer, max_tokens, max_table_blocks;
 };
 
@@ -37,16 +51,11 @@ __device__ __forceinline__ int clamp_requests(const PlanArgs &a)
     return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
 }
 
-// token range [p0, p1) of part c of a request spanning [t0, t1): equal parts, multiples of 128
-__device__ __forceinline__ void part_range(int64_t t0, int64_t t1, int c, int64_t &p0, int64_t &p1)
+// first table entry of request r (r == R: one past the last entry), clipped to the table capacity
+__device__ __forceinline__ int64_t clipped_offset(const PlanArgs &a, int r)
 {
-    const int64_t len = t1 - t0;
-    int64_t per = (len + PLAN_PARTS - 1) / PLAN_PARTS;
-    per = (per + 127) & ~(int64_t)127;
-    p0 = t0 + (int64_t)c * per;
-    p1 = p0 + per;
-    if (p0 > t1) p0 = t1;
-    if (p1 > t1) p1 = t1;
+    const int64_t o = a.tt_offsets[r];
+    return o < 0 ? 0 : (o > a.max_tokens ? a.max_tokens : o);
 }
 
 __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
@@ -55,30 +64,77 @@ __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
     atomicOr(&a.out_counts->error_flags, flags);
 }
 
-// ---- count -----------------------------------------------------------------------------
-__global__ void __launch_bounds__(PLAN_NT) plan_count_kernel(PlanArgs a)
+// The thread's four entries [t, t + 4) of the token table below T: slots, and one bit per live entry.
+__device__ __forceinline__ unsigned load_entries(const PlanArgs &a, int64_t t, int64_t T, int32_t (&slot)[TILE_TOK],
+                                                 bool &bad)
 {
+    uint8_t kp[TILE_TOK] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < TILE_TOK; ++k) slot[k] = -1;
+    if (a.vec_in && t + TILE_TOK <= T) {
+        const int4 s4 = *reinterpret_cast<const int4 *>(a.tt_slots + t);
+        const uchar4 k4 = *reinterpret_cast<const uchar4 *>(a.keep + t);
+        slot[0] = s4.x; slot[1] = s4.y; slot[2] = s4.z; slot[3] = s4.w;
+        kp[0] = k4.x; kp[1] = k4.y; kp[2] = k4.z; kp[3] = k4.w;
+    } else {
+#pragma unroll
+        for (int k = 0; k < TILE_TOK; ++k)
+            if (t + k < T) { slot[k] = a.tt_slots[t + k]; kp[k] = a.keep[t + k]; }
+    }
+    unsigned bits = 0;
+#pragma unroll
+    for (int k = 0; k < TILE_TOK; ++k) {
+        if (slot[k] < 0) continue;
+        if ((int64_t)slot[k] >= a.slots_per_layer) { bad = true; continue; }
+        if (kp[k] != 0) bits |= 1u << k;
+    }
+    return bits;
+}
+
+// ---- tiles -----------------------------------------------------------------------------
+__global__ void __launch_bounds__(TILE_NT) plan_tiles_kernel(PlanArgs a)
+{
+    __shared__ int warp_n[TILE_NT / 32];
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
-    if (r >= clamp_requests(a)) return;
-    int64_t t0, t1, p0, p1;
-    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
-    part_range(t0, t1, c, p0, p1);
-    int n = 0;
+    const int R = clamp_requests(a);
+    const int64_t T = clipped_offset(a, R);
+    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
     bool bad = false;
-    for (int64_t t = p0 + threadIdx.x; t < p1; t += PLAN_NT)
-        n += vtk_live(a.tt_slots[t], a.keep, t, a.slots_per_layer, bad) ? 1 : 0;
-    __shared__ int warp_n[PLAN_NT / 32];
+    int32_t slot[TILE_TOK];
+    if ((int)blockIdx.x < a.num_tiles) {
+        // live entries of one tile
+        const int64_t base = (int64_t)blockIdx.x * TILE;
+        if (base >= T) return;
+        int n = __popc(load_entries(a, base + threadIdx.x * TILE_TOK, T, slot, bad));
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
-    if (vtk_lane() == 0) warp_n[threadIdx.x >> 5] = n;
-    if (bad) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int s = 0;
-        for (int w = 0; w < PLAN_NT / 32; ++w) s += warp_n[w];
-        a.part_n[blockIdx.x] = s;
+        for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+        if (lane == 0) warp_n[warp] = n;
+        const int any_bad = __syncthreads_or(bad);
+        if (threadIdx.x == 0) {
+            int s = 0;
+#pragma unroll
+            for (int w = 0; w < TILE_NT / 32; ++w) s += warp_n[w];
+            // a slot outside the pool somewhere in the tile travels in the sign bit (the count is at most
+            // 1024): the scan kernel turns it into VTOKEN_FLAG_BAD_SLOT, and nothing has to be zeroed
+            // before this kernel
+            a.tile_n[blockIdx.x] = s | (any_bad ? (int)0x80000000 : 0);
+        }
+    } else {
+        // one warp per request boundary: live entries between the start of its tile and the boundary
+        // (entries the tile CTAs count as well; flags are raised there)
+        const int r = ((int)blockIdx.x - a.num_tiles) * (TILE_NT / 32) + warp;
+        if (r > R) return;
+        const int64_t o = clipped_offset(a, r);
+        const int64_t base = o / TILE * TILE;
+        int n = 0;
+        for (int64_t t = base + lane * TILE_TOK; t < o; t += 32 * TILE_TOK) {
+            unsigned bits = load_entries(a, t, o, slot, bad);     // entries at or behind the boundary do not count
+            n += __popc(bits);
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+        if (lane == 0) a.req_part[r] = n;
     }
 }
 
@@ -131,6 +187,9 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
     __shared__ Acc warp_acc[32];
     __shared__ long long carry_need;
     __shared__ Acc carry;
+    __shared__ int warp_i[32];
+    __shared__ int carry_live;
+    __shared__ unsigned int all_flags;
     const int tid = threadIdx.x;
     vtk_release_successor();
     vtk_wait_for_predecessor();
@@ -139,6 +198,8 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
     if (tid == 0) {
         if (*a.num_requests > a.max_requests || *a.num_requests < 0) flags |= VTOKEN_FLAG_CAPACITY;
         carry_need = 0;
+        carry_live = 0;
+        all_flags = 0;
         carry = Acc{0, 0, 0, 0, 0, 0};
     }
     int nf = *a.num_free;
@@ -148,14 +209,38 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 
     auto shfl_ll = [](long long v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
     auto shfl_acc = [](const Acc &v, int d) { return shfl_up(v, d); };
+    auto shfl_int = [](int v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
+
+    // live tokens before every tile (in place: tile_n[i] becomes the sum of the tiles before i; one
+    // entry past the last tile holds the total)
+    const int64_t T = clipped_offset(a, R);
+    const int tiles = (int)((T + TILE - 1) / TILE);
+    for (int base = 0; base <= tiles; base += SCAN_NT) {
+        const int i = base + tid;
+        const int raw = i < tiles ? a.tile_n[i] : 0;
+        if (raw < 0) flags |= VTOKEN_FLAG_BAD_SLOT;
+        const int v = raw & 0x7fffffff;
+        const int incl = block_incl_scan<int>(v, warp_i, 0, shfl_int) + carry_live;
+        if (i <= tiles) a.tile_n[i] = incl - v;
+        __syncthreads();
+        if (tid == SCAN_NT - 1) carry_live = incl;
+        __syncthreads();
+    }
+    // live tokens before table entry o = live tokens before its tile + those between the tile's start and o
+    auto live_before = [&](int r) {
+        const int64_t o = clipped_offset(a, r);
+        return a.tile_n[o / TILE] + (o % TILE != 0 ? a.req_part[r] : 0);
+    };
 
     for (int base = 0; base < R; base += SCAN_NT) {
         const int r = base + tid;
         const bool valid = r < R;
         int n = 0, nb = 0;
         if (valid) {
-#pragma unroll
-            for (int c = 0; c < PLAN_PARTS; ++c) n += a.part_n[r * PLAN_PARTS + c];
+            const int before = live_before(r);
+            n = live_before(r + 1) - before;
+            if (n < 0) n = 0;                                // offsets that run backwards
+            a.req_before[r] = before;
             a.req_n[r] = n;
             int64_t lo, hi, t0, t1;
             const bool clipped = vtk_range(a.bt_offsets, r, a.max_table_blocks, lo, hi) |
@@ -191,7 +276,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         }
         __syncthreads();
     }
-    if (flags) atomicOr(&a.counts->error_flags, flags);
+    if (flags) atomicOr(&all_flags, flags);
     __syncthreads();
     if (tid == 0) {
         a.new_bt_offsets[R] = carry.newbt;
@@ -202,7 +287,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         c.num_free_consumed = carry.dst;
         c.num_admitted = carry.admitted;
         c.num_deferred = carry.deferred;
-        c.error_flags = atomicOr(&a.counts->error_flags, 0u);   // bits raised by the count kernel and above
+        c.error_flags = all_flags;                       // whatever an earlier plan or copy left is overwritten
         c.num_released = 0;
         *a.counts = c;
         *a.out_counts = c;                               // later flags are OR-ed into both copies
@@ -210,80 +295,115 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 }
 
 // ---- assign ----------------------------------------------------------------------------
-__global__ void __launch_bounds__(PLAN_NT) plan_assign_kernel(PlanArgs a)
+__global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
 {
-    __shared__ int warp_sums[PLAN_NT / 32 + 1];
+    __shared__ int warp_sums[TILE_NT / 32];
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    const int r = blockIdx.x / PLAN_PARTS, c = blockIdx.x % PLAN_PARTS;
-    if (r >= clamp_requests(a)) return;
-    const int tid = threadIdx.x;
+    const int R = clamp_requests(a);
+    const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
     const int S = a.S;
-    int64_t t0, t1, b0, b1;
-    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
-    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
-    const int nb = (int)(b1 - b0);
-    const bool adm = a.req_status[r] == VTOKEN_REPACKED;
-    const int n = a.req_n[r];
-    const int need = (int)(((int64_t)n + S - 1) / S);
-    const int dst_base = a.req_dst_base[r];
-    const int nbt0 = a.new_bt_offsets[r];
     uint32_t flags = 0;
 
-    // block tables and the reclaimed list: the request's parts share the work in stripes
-    const int stripe = c * PLAN_NT + tid, stride = PLAN_PARTS * PLAN_NT;
-    if (adm) {
-        for (int j = stripe; j < need; j += stride) {
-            int blk = a.free_blocks[dst_base + j];
-            if ((int64_t)nbt0 + j < a.max_table_blocks) a.new_bt_blocks[nbt0 + j] = blk;
-            if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
-            a.dst_blocks[dst_base + j] = blk;
+    if ((int)blockIdx.x >= a.num_tiles) {
+        // block table and reclaimed list of one request
+        const int r = (int)blockIdx.x - a.num_tiles;
+        if (r >= R) return;
+        int64_t b0, b1;
+        vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
+        const int nb = (int)(b1 - b0);
+        const int nbt0 = a.new_bt_offsets[r];
+        if (a.req_status[r] == VTOKEN_REPACKED) {
+            const int n = a.req_n[r];
+            const int need = (int)(((int64_t)n + S - 1) / S);
+            const int dst_base = a.req_dst_base[r];
+            for (int j = tid; j < need; j += TILE_NT) {
+                int blk = a.free_blocks[dst_base + j];
+                if ((int64_t)nbt0 + j < a.max_table_blocks) a.new_bt_blocks[nbt0 + j] = blk;
+                if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
+                a.dst_blocks[dst_base + j] = blk;
+            }
+            const int f0 = a.req_freed_base[r];
+            for (int j = tid; j < nb && (int64_t)f0 + j < a.max_table_blocks; j += TILE_NT) {
+                const int blk = a.bt_blocks[b0 + j];
+                if (blk < 0 || blk >= a.num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
+                a.freed_blocks[f0 + j] = blk;
+            }
+            // unused tail of the last destination block
+            for (int i = n + tid; i < need * S; i += TILE_NT) a.dst_src[(int64_t)dst_base * S + i] = -1;
+        } else {
+            for (int j = tid; j < nb && (int64_t)nbt0 + j < a.max_table_blocks; j += TILE_NT)
+                a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
         }
-        const int f0 = a.req_freed_base[r];
-        for (int j = stripe; j < nb && (int64_t)f0 + j < a.max_table_blocks; j += stride) {
-            const int blk = a.bt_blocks[b0 + j];
-            if (blk < 0 || blk >= a.num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
-            a.freed_blocks[f0 + j] = blk;
-        }
-        // unused tail of the last destination block
-        for (int i = n + stripe; i < need * S; i += stride) a.dst_src[(int64_t)dst_base * S + i] = -1;
-    } else {
-        for (int j = stripe; j < nb && (int64_t)nbt0 + j < a.max_table_blocks; j += stride)
-            a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
+        if (flags) raise_flags(a, flags);
+        return;
     }
 
     // token table: rank of each live token in logical order -> destination slot
-    int64_t p0, p1;
-    part_range(t0, t1, c, p0, p1);
-    int carry = 0;                                       // live tokens of the parts before this one
-    for (int cc = 0; cc < c; ++cc) carry += a.part_n[r * PLAN_PARTS + cc];
-    for (int64_t tb = p0; tb < p1; tb += PLAN_NT) {
-        const int64_t t = tb + tid;
-        int32_t slot = -1;
-        bool live = false, bad = false;
-        if (t < p1) {
-            slot = a.tt_slots[t];
-            live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
-        }
-        int total;
-        const int i = carry + vtk_block_rank<PLAN_NT>(live, warp_sums, total);
-        carry += total;
-        if (t < p1) {
-            int32_t out = -1;
-            if (live) {
-                if (adm) {
-                    const int j = i / S, off = i - j * S;
-                    const int blk = a.free_blocks[dst_base + j];
-                    out = blk * S + off;                    // slot = block_id * S + offset
-                    a.dst_src[(int64_t)(dst_base + j) * S + off] = slot;
-                } else {
-                    out = slot;
-                }
-            }
-            a.new_tt_slots[t] = out;
-        }
+    const int64_t T = clipped_offset(a, R);
+    const int64_t base = (int64_t)blockIdx.x * TILE;
+    if (base >= T) return;
+    const int64_t t = base + tid * TILE_TOK;
+    int32_t slot[TILE_TOK];
+    bool bad = false;
+    const unsigned bits = load_entries(a, t, T, slot, bad);
+    // live tokens of the whole table before this thread's first entry
+    const int cnt = __popc(bits);
+    const int incl = vtk_warp_incl_scan(cnt);
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = a.tile_n[blockIdx.x] + incl - cnt;
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    if (t >= T) return;
+
+    // the request that owns entry t: the last one whose first entry is at or before t
+    int lo = 0, hi = R;                         // invariant: offset(lo) <= t or lo == 0;  offset(hi) > t
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (clipped_offset(a, mid) <= t) lo = mid; else hi = mid;
     }
-    if (flags) raise_flags(a, flags);
+    int r = clipped_offset(a, lo) <= t ? lo : -1;       // -1: an entry before the first request's range
+    int64_t next = r + 1 <= R ? clipped_offset(a, r + 1) : T;
+    int req_before = 0, n = 0, dst_base = 0;
+    bool adm = false;
+    auto load_request = [&]() {
+        req_before = a.req_before[r];
+        n = a.req_n[r];
+        dst_base = a.req_dst_base[r];
+        adm = a.req_status[r] == VTOKEN_REPACKED;
+    };
+    if (r >= 0) load_request();
+
+    int32_t out[TILE_TOK];
+    bool owned = true;
+#pragma unroll
+    for (int k = 0; k < TILE_TOK; ++k) {
+        out[k] = -1;
+        if (t + k >= T) { owned = false; continue; }
+        if (t + k >= next) {                                  // a request boundary inside the thread's entries
+            while (r + 1 < R && clipped_offset(a, r + 1) <= t + k) ++r;
+            next = clipped_offset(a, r + 1);
+            if (r >= 0) load_request();
+        }
+        if (r < 0) { owned = false; continue; }
+        if (!((bits >> k) & 1u)) continue;                    // dead or unmapped: -1
+        if (!adm) { out[k] = slot[k]; continue; }            // the request keeps its layout
+        const int i = before + __popc(bits & ((1u << k) - 1u)) - req_before;   // rank inside the request
+        if (i < 0 || i >= n) continue;                        // only with inconsistent offsets
+        const int j = i / S, off = i - j * S;
+        const int blk = a.free_blocks[dst_base + j];
+        out[k] = blk * S + off;                               // slot = block_id * S + offset
+        a.dst_src[(int64_t)(dst_base + j) * S + off] = slot[k];
+    }
+    if (owned && a.vec_out) {
+        *reinterpret_cast<int4 *>(a.new_tt_slots + t) = make_int4(out[0], out[1], out[2], out[3]);
+    } else {
+        // the ragged end of the table, or entries in front of the first request (left untouched)
+        const int64_t first = clipped_offset(a, 0);
+#pragma unroll
+        for (int k = 0; k < TILE_TOK; ++k)
+            if (t + k < T && t + k >= first) a.new_tt_slots[t + k] = out[k];
+    }
 }
 
 }  // namespace
@@ -309,12 +429,14 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.out_status = out->req_status;
     a.out_counts = out->counts;
     a.req_n = ctx->req_n;
-    a.part_n = ctx->part_n;
     a.req_dst_base = ctx->req_dst_base;
     a.req_freed_base = ctx->req_freed_base;
     a.req_status = ctx->req_status;
     a.dst_src = ctx->dst_src;
     a.dst_blocks = ctx->dst_blocks;
+    a.tile_n = ctx->tile_n;
+    a.req_part = ctx->req_part;
+    a.req_before = ctx->req_before;
     a.counts = ctx->counts;
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
@@ -324,12 +446,17 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.slots_per_layer = ctx->slots_per_layer;
     a.max_tokens = ctx->cfg.max_tokens;
     a.max_table_blocks = ctx->cfg.max_table_blocks;
+    a.num_tiles = (int32_t)((ctx->cfg.max_tokens + TILE - 1) / TILE);
+    // four entries per thread go through 16-byte (slots) and 4-byte (keep) accesses when the caller's
+    // arrays allow it; tiles start at multiples of 1024 entries, so the base addresses decide
+    a.vec_in = ((uintptr_t)in->tt_slots % 16 == 0 && (uintptr_t)in->keep % 4 == 0) ? 1 : 0;
+    a.vec_out = ((uintptr_t)out->new_tt_slots % 16 == 0) ? 1 : 0;
 
-    VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
-    const dim3 parts(ctx->cfg.max_requests * PLAN_PARTS);
-    VTK_CUDA(ctx, vtk_launch_dependent(plan_count_kernel, parts, dim3(PLAN_NT), 0, st, a));
+    const int R = ctx->cfg.max_requests;
+    VTK_CUDA(ctx, vtk_launch_dependent(plan_tiles_kernel, dim3(a.num_tiles + (R + 1 + TILE_NT / 32 - 1) / (TILE_NT / 32)),
+                                       dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(plan_scan_kernel, dim3(1), dim3(SCAN_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(plan_assign_kernel, parts, dim3(PLAN_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(plan_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

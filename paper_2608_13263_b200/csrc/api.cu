@@ -112,6 +112,8 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     if (cap > cfg->max_free_blocks) cap = cfg->max_free_blocks;
     if (cap < 1) cap = 1;
     ctx->cap_dst_blocks = (int32_t)cap;
+    ctx->parts = vtk_choose_parts(cfg->max_requests, cfg->max_tokens);
+    if (const char *e = getenv("VTOKEN_PLAN_PARTS")) { int v = atoi(e); if (v >= 1 && v <= VTK_PLAN_PARTS) ctx->parts = v; }
 
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);

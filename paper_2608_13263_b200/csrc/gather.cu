@@ -22,6 +22,7 @@ struct GatherArgs {
     uint8_t *out_k, *out_v;
     int64_t layer_stride, row_bytes, slots_per_layer, out_capacity, max_tokens;
     int32_t layer_begin, layer_end, max_requests;
+    int32_t parts;               // token ranges (CTAs) per request, <= G_PARTS (the stride of part_n)
 };
 
 __device__ __forceinline__ int g_requests(const GatherArgs &a)
@@ -31,9 +32,9 @@ __device__ __forceinline__ int g_requests(const GatherArgs &a)
 }
 
 // token range [p0, p1) of part c of a request spanning [t0, t1): equal parts, multiples of 128
-__device__ __forceinline__ void g_part_range(int64_t t0, int64_t t1, int c, int64_t &p0, int64_t &p1)
+__device__ __forceinline__ void g_part_range(int64_t t0, int64_t t1, int c, int parts, int64_t &p0, int64_t &p1)
 {
-    int64_t per = (t1 - t0 + G_PARTS - 1) / G_PARTS;
+    int64_t per = (t1 - t0 + parts - 1) / parts;
     per = (per + 127) & ~(int64_t)127;
     p0 = t0 + (int64_t)c * per;
     p1 = p0 + per;
@@ -45,13 +46,13 @@ __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
 {
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    const int r = blockIdx.x / G_PARTS, c = blockIdx.x % G_PARTS;
+    const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
     if (r >= g_requests(a)) return;
     int n = 0;
     bool bad = false;
     if (a.select == nullptr || a.select[r] != 0) {
         int64_t p0, p1;
-        g_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, p0, p1);
+        g_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, a.parts, p0, p1);
         for (int64_t t = p0 + threadIdx.x; t < p1; t += G_NT)
             n += vtk_live(a.tt_slots[t], a.keep, t, a.slots_per_layer, bad) ? 1 : 0;
     }
@@ -64,7 +65,7 @@ __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
     if (threadIdx.x == 0) {
         int s = 0;
         for (int w = 0; w < G_NT / 32; ++w) s += warp_n[w];
-        a.part_n[blockIdx.x] = s;
+        a.part_n[r * G_PARTS + c] = s;
     }
 }
 
@@ -84,7 +85,7 @@ __global__ void __launch_bounds__(1024) gather_scan_kernel(GatherArgs a)
         int v = 0;
         if (r < R) {
 #pragma unroll
-            for (int c = 0; c < G_PARTS; ++c) v += a.part_n[r * G_PARTS + c];
+            for (int c = 0; c < a.parts; ++c) v += a.part_n[r * G_PARTS + c];
         }
         int incl = vtk_warp_incl_scan(v);
         if (lane == 31) warp_tot[warp] = incl;
@@ -119,12 +120,12 @@ __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
     vtk_release_successor();
     vtk_wait_for_predecessor();
     __shared__ int warp_sums[G_NT / 32 + 1];
-    const int r = blockIdx.x / G_PARTS, c = blockIdx.x % G_PARTS;
+    const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
     if (r >= g_requests(a)) return;
     if (a.select != nullptr && a.select[r] == 0) return;
     const int64_t t0 = a.tt_offsets[r];
     int64_t p0, p1;
-    g_part_range(t0, a.tt_offsets[r + 1], c, p0, p1);
+    g_part_range(t0, a.tt_offsets[r + 1], c, a.parts, p0, p1);
     const int64_t cap = *a.g_total;
     int carry = a.out_offsets[r];
     for (int cc = 0; cc < c; ++cc) carry += a.part_n[r * G_PARTS + cc];
@@ -374,12 +375,13 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     a.layer_begin = layer_begin;
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
+    a.parts = ctx->parts;
     VTK_CUDA(ctx, cudaMemsetAsync(out_digest, 0, sizeof(uint64_t) * (size_t)ctx->cfg.max_requests, st));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
-                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
-                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_digest_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
@@ -417,11 +419,12 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.layer_begin = layer_begin;
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
+    a.parts = ctx->parts;
     VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
-                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
-                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     // the rows go through the bulk-copy rings when the context has them (vtoken_create does; the
     // context-free entry point does not), else through the register kernel
     const bool aligned = (((uintptr_t)out_k | (uintptr_t)out_v) & 15) == 0;
@@ -466,11 +469,12 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.max_tokens = out_capacity;
     a.layer_begin = a.layer_end = 0;
     a.max_requests = ctx->cfg.max_requests;
+    a.parts = ctx->parts;
     VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
-                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
-                                       dim3(ctx->cfg.max_requests * G_PARTS), dim3(G_NT), 0, st, a));
+                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -45,6 +45,7 @@ struct PArgs {
     uint8_t *blk_src;
     vtoken_counts *counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
+    int32_t parts;          // token ranges (CTAs) per request, <= PP_PARTS (the stride of the part_* arrays)
     int64_t slots_per_layer, max_tokens, max_table_blocks;
 };
 
@@ -54,9 +55,9 @@ __device__ __forceinline__ int pp_requests(const PArgs &a)
     return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
 }
 
-__device__ __forceinline__ void pp_part_range(int64_t t0, int64_t t1, int c, int64_t &p0, int64_t &p1)
+__device__ __forceinline__ void pp_part_range(int64_t t0, int64_t t1, int c, int parts, int64_t &p0, int64_t &p1)
 {
-    int64_t per = (t1 - t0 + PP_PARTS - 1) / PP_PARTS;
+    int64_t per = (t1 - t0 + parts - 1) / parts;
     per = (per + 127) & ~(int64_t)127;
     p0 = t0 + (int64_t)c * per;
     p1 = p0 + per;
@@ -92,11 +93,11 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
     vtk_release_successor();
     vtk_wait_for_predecessor();
     __shared__ int warp_n[PP_NT / 32];
-    const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
+    const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
     if (r >= pp_requests(a)) return;
     int64_t t0, t1, p0, p1;
     vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
-    pp_part_range(t0, t1, c, p0, p1);
+    pp_part_range(t0, t1, c, a.parts, p0, p1);
     const bool may_detach = a.protect != nullptr && a.detach_den != 0;
     const bool detach = MODE == 1 && may_detach && a.req_detach[r] != 0;
     int n = 0, n_shared = 0;
@@ -120,11 +121,11 @@ __global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
     }
     if (bad && MODE == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
     const int s = pp_block_sum(n, warp_n);
-    if (threadIdx.x == 0) (MODE == 0 ? a.part_n : a.part_src)[blockIdx.x] = s;
+    if (threadIdx.x == 0) (MODE == 0 ? a.part_n : a.part_src)[r * PP_PARTS + c] = s;
     if (MODE == 0 && may_detach) {
         __syncthreads();                       // warp_n is reused
         const int sh = pp_block_sum(n_shared, warp_n);
-        if (threadIdx.x == 0) a.part_shared[blockIdx.x] = sh;
+        if (threadIdx.x == 0) a.part_shared[r * PP_PARTS + c] = sh;
     }
 }
 
@@ -171,7 +172,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
         const int ns_shared = pp_block_sum(shared, warp_sums);          // valid in thread 0
         if (threadIdx.x == 0) {
             long long n_shared = 0;
-            for (int c = 0; c < PP_PARTS; ++c) n_shared += a.part_shared[r * PP_PARTS + c];
+            for (int c = 0; c < a.parts; ++c) n_shared += a.part_shared[r * PP_PARTS + c];
             const bool detach = ns_shared > 0 &&
                                 (unsigned long long)n_shared * a.detach_den <
                                     (unsigned long long)a.detach_num * (unsigned long long)ns_shared * (unsigned long long)a.S;
@@ -257,7 +258,7 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     for (int r = tid; r < R; r += PP_SCAN_NT) {
         int n = 0, nsrc = 0;
 #pragma unroll
-        for (int c = 0; c < PP_PARTS; ++c) {
+        for (int c = 0; c < a.parts; ++c) {
             n += a.part_n[r * PP_PARTS + c];
             nsrc += a.part_src[r * PP_PARTS + c];
         }
@@ -347,7 +348,7 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
     vtk_release_successor();
     vtk_wait_for_predecessor();
     __shared__ int warp_sums[PP_NT / 32 + 1];
-    const int r = blockIdx.x / PP_PARTS, c = blockIdx.x % PP_PARTS;
+    const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
     if (r >= pp_requests(a)) return;
     const int tid = threadIdx.x;
     const int S = a.S;
@@ -364,7 +365,7 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
     const int nbt0 = a.new_bt_offsets[r];
     uint32_t flags = 0;
 
-    const int stripe = c * PP_NT + tid, stride = PP_PARTS * PP_NT;
+    const int stripe = c * PP_NT + tid, stride = a.parts * PP_NT;
     if (adm) {
         // destinations follow the kept blocks in the new block table
         for (int j = stripe; j < need; j += stride) {
@@ -414,7 +415,7 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
 
     // token table
     int64_t p0, p1;
-    pp_part_range(t0, t1, c, p0, p1);
+    pp_part_range(t0, t1, c, a.parts, p0, p1);
     int carry = 0;                                       // moving tokens of the parts before this one
     for (int cc = 0; cc < c; ++cc) carry += a.part_src[r * PP_PARTS + cc];
     for (int64_t tb = p0; tb < p1; tb += PP_NT) {
@@ -486,7 +487,7 @@ __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_request
 
 __global__ void __launch_bounds__(1024) pp_summary_kernel(const int32_t *num_requests, int32_t max_requests,
                                                           const int32_t *bt_offsets, const int32_t *part_n,
-                                                          long long *summary)
+                                                          int parts, long long *summary)
 {
     vtk_release_successor();
     vtk_wait_for_predecessor();
@@ -495,7 +496,7 @@ __global__ void __launch_bounds__(1024) pp_summary_kernel(const int32_t *num_req
     int R = *num_requests;
     R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
     long long s = 0;
-    for (int i = threadIdx.x; i < R * PP_PARTS; i += 1024) s += part_n[i];
+    for (int i = threadIdx.x; i < R * parts; i += 1024) s += part_n[i / parts * PP_PARTS + i % parts];
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
     if (vtk_lane() == 0) warp_s[threadIdx.x >> 5] = s;
@@ -538,6 +539,7 @@ void fill_args(PArgs &a, vtoken_ctx *ctx)
     a.slots_per_layer = ctx->slots_per_layer;
     a.max_tokens = ctx->cfg.max_tokens;
     a.max_table_blocks = ctx->cfg.max_table_blocks;
+    a.parts = ctx->parts;
 }
 
 }  // namespace
@@ -590,11 +592,11 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->blk_src, 0, (size_t)ctx->cfg.num_blocks, st));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(pp_blocks_kernel, dim3(R), dim3(PP_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<1>, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<1>, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(pp_scan_kernel, dim3(1), dim3(PP_SCAN_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_assign_kernel, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_assign_kernel, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     ctx->has_plan = true;
     return VTOKEN_OK;
@@ -618,7 +620,7 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     a.n_b = n_b;
     const int R = ctx->cfg.max_requests;
     VTK_CUDA(ctx, cudaMemsetAsync(n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * PP_PARTS), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
     if (hist) {
         VTK_CUDA(ctx, cudaMemsetAsync(hist, 0, sizeof(uint64_t) * (size_t)(ctx->cfg.block_size + 1), st));
         VTK_CUDA(ctx, vtk_launch_dependent(pp_hist_kernel, dim3(ctx->num_sms * 4), dim3(256), 0, st, num_requests, R,
@@ -627,7 +629,7 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     }
     if (summary)
         VTK_CUDA(ctx, vtk_launch_dependent(pp_summary_kernel, dim3(1), dim3(1024), 0, st, num_requests, R, bt_offsets,
-                                           (const int32_t *)ctx->part_n, (long long *)summary));
+                                           (const int32_t *)ctx->part_n, ctx->parts, (long long *)summary));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

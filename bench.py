@@ -799,6 +799,54 @@ def run_runtime(args, prob, w, side, dev):
     return out
 
 
+def run_plan_only(args):
+    """Planner latency on the full-size tables of a workload, without its pools: the planner kernels
+    read and write tables only, so the context gets a stand-in pool of a few bytes and `vtoken_repack`
+    is never called.  Lets the 512-request tables be timed (and profiled) with a few MB on the device.
+    Prints one JSON line; parity of both planners is the tests' business, not this mode's."""
+    import torch
+    from paper_2608_13263_b200 import binding as vt
+    from paper_2608_13263_b200.device import DeviceProblem
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    w = build_workload(args.config, args.seed, args.scale_requests, args.block_size)
+    prob = DeviceProblem(w, device=dev, allocate_pools=False)
+    stand_in = torch.zeros(64, dtype=torch.int16, device=dev)
+    prob.ctx = vt.vtoken_create(w.num_layers, w.num_blocks, w.block_size, w.num_kv_heads, w.head_dim, stand_in,
+                                stand_in, prob.max_requests, prob.max_tokens, prob.max_table_blocks, prob.max_free,
+                                elem_bytes=w.elem_bytes)
+    side = torch.cuda.Stream(device=dev)
+    partial_opts = dict(util=(1, 1), theta=(1, 4))
+    res = {}
+    for label, fn in (("whole", lambda st: prob.plan(stream=st)),
+                      ("partial", lambda st: prob.plan_partial(stream=st, **partial_opts))):
+        with torch.cuda.stream(side):
+            fn(side)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            fn(torch.cuda.current_stream())
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(side):
+            for _ in range(args.warmup):
+                g.replay()
+            e0.record(side)
+            for _ in range(args.steps):
+                g.replay()
+            e1.record(side)
+        side.synchronize()
+        out = prob.outputs()
+        res[label] = {"us": e0.elapsed_time(e1) / args.steps * 1e3, "tokens_moved": out["num_moves"],
+                      "requests_repacked": out["num_admitted"], "error_flags": out["error_flags"]}
+    T = w.num_tokens
+    print(json.dumps({"mode": "plan-only", "config": {"workload": f"{w.name} (seed {args.seed})",
+                                                      "requests": w.num_requests, "table_entries": T,
+                                                      "block_size": w.block_size, "num_blocks": w.num_blocks},
+                      "steps": args.steps, "warmup": args.warmup, "table_bytes_per_plan": 13 * T,
+                      "planner": res, "gpu": torch.cuda.get_device_name(dev)}))
+    prob.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -820,11 +868,15 @@ def main():
                     help="also run the repack in this many waves with the headroom of the largest single demand")
     ap.add_argument("--block-size", type=int, default=0, help="override the workload's block size")
     ap.add_argument("--no-verify", action="store_true")
+    ap.add_argument("--plan-only", action="store_true",
+                    help="time the planners alone on the workload's tables (no pools are allocated)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.plan_only:
+        run_plan_only(args)
     else:
         run_cuda(args)
 

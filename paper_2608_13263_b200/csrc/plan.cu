@@ -298,6 +298,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
 {
     __shared__ int warp_sums[TILE_NT / 32];
+    __shared__ int tile_req[2];
     vtk_release_successor();
     vtk_wait_for_predecessor();
     const int R = clamp_requests(a);
@@ -351,18 +352,40 @@ __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
     const int cnt = __popc(bits);
     const int incl = vtk_warp_incl_scan(cnt);
     if (lane == 31) warp_sums[warp] = incl;
+    // The requests that own the tile's first and last entry (owner of an entry: the last request whose
+    // first entry is at or before it; -1: the entry lies in front of the first request), each found by
+    // one warp with a 32-way search over the offsets.  Most tiles lie inside one or a few requests, so
+    // the per-thread search below has next to nothing left to do.
+    if (warp < 2) {
+        const int64_t last = (base + TILE < T ? base + TILE : T) - 1;
+        const int64_t key = warp == 0 ? base : last;
+        int lo = -1, hi = R;                    // offset(lo) <= key (or lo == -1); offset(hi) > key: offset(R) = T
+        while (hi - lo > 1) {
+            const int step = (hi - lo - 1 + 31) / 32;
+            const int probe = lo + 1 + lane * step;
+            const bool le = probe < hi && clipped_offset(a, probe) <= key;
+            const int n_le = __popc(__ballot_sync(0xffffffffu, le));
+            const int first_gt = lo + 1 + n_le * step;          // first probe beyond the key, if it was probed
+            if (n_le > 0) lo = lo + 1 + (n_le - 1) * step;
+            if (first_gt < hi) hi = first_gt;
+        }
+        if (lane == 0) tile_req[warp] = lo;
+    }
     __syncthreads();
     int before = a.tile_n[blockIdx.x] + incl - cnt;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
     if (t >= T) return;
 
-    // the request that owns entry t: the last one whose first entry is at or before t
-    int lo = 0, hi = R;                         // invariant: offset(lo) <= t or lo == 0;  offset(hi) > t
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (clipped_offset(a, mid) <= t) lo = mid; else hi = mid;
+    // the request that owns entry t
+    int r;
+    {
+        int lo = tile_req[0], hi = (tile_req[1] > tile_req[0] ? tile_req[1] : tile_req[0]) + 1;
+        while (hi - lo > 1) {                   // offset(lo) <= t (or lo == -1); offset(hi) > t
+            const int mid = (lo + hi) >> 1;
+            if (clipped_offset(a, mid) <= t) lo = mid; else hi = mid;
+        }
+        r = lo;                                 // -1: an entry before the first request's range
     }
-    int r = clipped_offset(a, lo) <= t ? lo : -1;       // -1: an entry before the first request's range
     int64_t next = r + 1 <= R ? clipped_offset(a, r + 1) : T;
     int req_before = 0, n = 0, dst_base = 0;
     bool adm = false;

@@ -55,8 +55,8 @@
  *                        warps take items from a ticket counter, VTOKEN_COPY_CHUNK (default 4) at a time
  *   VTOKEN_WAIT_LIMIT_MS bound of in-kernel waits (1 .. 60000, default 2000)
  *   VTOKEN_PLAN_PARTS    1 .. 8: token ranges (CTAs) per request in the kernels that walk the token table request
- *                        by request (partial planner, block liveness, logical gather, slot mapping); default:
- *                        chosen from max_requests and max_tokens
+ *                        by request (logical gather, slot mapping, relocation digest); default: chosen from
+ *                        max_requests and max_tokens
  *   VTOKEN_TEST_STALL_ITEM  test hook: index of one work item whose barrier is armed with bytes that never
  *                        arrive, so that its wait runs out (exercises the time-out path; never set in production)
  * and one read at every launch:

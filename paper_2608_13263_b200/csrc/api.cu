@@ -24,8 +24,8 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
-                    ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->part_src, ctx->req_ns, ctx->req_nsrc,
-                    ctx->n_b, ctx->blk_src, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
+                    ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
+                    ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
                     ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
                     ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
@@ -137,17 +137,19 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->g_ids, cfg->max_tokens);
     A(&ctx->g_req, cfg->max_tokens);
     A(&ctx->g_offsets, (int64_t)cfg->max_requests + 1);
-    A(&ctx->part_src, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
+    A(&ctx->tile_mov, (cfg->max_tokens + 1023) / 1024 + 1);
+    A(&ctx->tile_shared, (cfg->max_tokens + 1023) / 1024 + 1);
+    A(&ctx->part_mov, (int64_t)cfg->max_requests + 1);
     A(&ctx->req_ns, cfg->max_requests);
     A(&ctx->req_nsrc, cfg->max_requests);
-    A(&ctx->n_b, cfg->num_blocks);
-    A(&ctx->blk_src, cfg->num_blocks);
+    A(&ctx->n_b, (int64_t)cfg->num_blocks + (cfg->num_blocks + 3) / 4);      // n_b, then blk_src (one byte per block)
+    if (rc == VTOKEN_OK) ctx->blk_src = reinterpret_cast<uint8_t *>(ctx->n_b + cfg->num_blocks);
     A(&ctx->slot_bits, (slots + 31) / 32);
     A(&ctx->copy_ticket, 2);
     if (rc == VTOKEN_OK && cudaMemset(ctx->copy_ticket, 0, 2 * sizeof(unsigned int)) != cudaSuccess) rc = VTOKEN_ECUDA;
     A(&ctx->g_ticket, 2);
     if (rc == VTOKEN_OK && cudaMemset(ctx->g_ticket, 0, 2 * sizeof(unsigned int)) != cudaSuccess) rc = VTOKEN_ECUDA;
-    A(&ctx->part_shared, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
+    A(&ctx->part_shared, (int64_t)cfg->max_requests + 1);
     A(&ctx->req_shared, cfg->max_requests);
     A(&ctx->req_detach, cfg->max_requests);
     A(&ctx->req_rel_base, cfg->max_requests);

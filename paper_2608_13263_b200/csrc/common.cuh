@@ -32,15 +32,16 @@ struct vtoken_ctx {
     int parts;                 // token ranges (CTAs) per request in the per-request kernels, 1 .. VTK_PLAN_PARTS
     int32_t *tile_n;           // [ceil(max_tokens / 1024) + 1] live tokens per tile of the token table, then scanned
     int32_t *req_part;         // [max_requests + 1] live tokens between a request's tile start and its first entry
-    int32_t *req_before;       // [max_requests + 1] live tokens of the table before the request's first entry
+    int32_t *req_before;       // [max_requests + 1] live (partial planner: moving) tokens of the table before the request's first entry
+    int32_t *tile_mov, *tile_shared;   // [like tile_n] partial planner: moving tokens / live tokens in protected blocks per tile
+    int32_t *part_mov;         // [max_requests + 1] partial planner: like req_part, moving tokens
 
     // partial-plan scratch (DEVICE)
-    int32_t *part_src;         // [max_requests * VTK_PLAN_PARTS] live tokens in source blocks per request part
     int32_t *req_ns;           // [max_requests] source blocks of the request
     int32_t *req_nsrc;         // [max_requests] live tokens in its source blocks
     int32_t *n_b;              // [num_blocks] live tokens per physical block
-    uint8_t *blk_src;          // [num_blocks] 1 = the block is a source of its request
-    int32_t *part_shared;      // [max_requests * VTK_PLAN_PARTS] live tokens in protected blocks per request part
+    uint8_t *blk_src;          // [num_blocks] 1 = the block is a source of its request (behind n_b in one allocation)
+    int32_t *part_shared;      // [max_requests + 1] like req_part, live tokens in protected blocks
     int32_t *req_shared;       // [max_requests] protected entries of the request's block table
     int32_t *req_detach;       // [max_requests] 1 = the request leaves its protected blocks (copy-on-write detach)
     int32_t *req_rel_base;     // [max_requests] first entry in released_blocks
@@ -80,8 +81,8 @@ struct vtoken_ctx {
     int bulk_warps, bulk_stages, bulk_rows, bulk_depth, bulk_ahead;   // bulk path: warps per CTA, ring size, rows per item, loads ahead
 };
 
-// Token ranges per request for the kernels that give every request its own CTAs (partial planner,
-// logical gather): enough CTAs to fill the GPU about twice over, few enough that a CTA has more
+// Token ranges per request for the kernels that give every request its own CTAs (logical gather,
+// slot mapping, digest): enough CTAs to fill the GPU about twice over, few enough that a CTA has more
 // than one pass to do -- 512 requests x 8 parts were 4096 CTAs of a single pass each, seven waves
 // of launch and load latency -- and never so few that a part exceeds about 4096 entries.
 inline int vtk_choose_parts(int64_t max_requests, int64_t max_tokens)
@@ -194,6 +195,85 @@ __device__ __forceinline__ bool vtk_range(const int32_t *off, int r, int64_t cap
     lo = a < 0 ? 0 : (a > cap ? cap : a);
     hi = b < lo ? lo : (b > cap ? cap : b);
     return lo != a || hi != b;
+}
+
+// ---------------------------------------------------------------------------------------
+// Flat tiling of the token table, shared by the planners: a tile is VTK_TILE consecutive table
+// entries whatever request they belong to, one CTA of VTK_TILE_NT threads, four entries per thread.
+// ---------------------------------------------------------------------------------------
+constexpr int VTK_TILE_NT = 256;
+constexpr int VTK_TILE_TOK = 4;
+constexpr int VTK_TILE = VTK_TILE_NT * VTK_TILE_TOK;
+
+// first table entry of request r (r == R: one past the last entry), clipped to the table capacity
+__device__ __forceinline__ int64_t vtk_clipped_offset(const int32_t *off, int r, int64_t cap)
+{
+    const int64_t o = off[r];
+    return o < 0 ? 0 : (o > cap ? cap : o);
+}
+
+// The thread's four entries [t, t + 4) of the token table below T: slots, and one bit per live entry.
+// vec: tt_slots is 16-byte and keep 4-byte aligned (t is a multiple of four).
+__device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, const uint8_t *keep, int vec, int64_t t,
+                                                     int64_t T, int64_t slots_per_layer,
+                                                     int32_t (&slot)[VTK_TILE_TOK], bool &bad)
+{
+    uint8_t kp[VTK_TILE_TOK] = {0, 0, 0, 0};
+#pragma unroll
+    for (int k = 0; k < VTK_TILE_TOK; ++k) slot[k] = -1;
+    if (vec && t + VTK_TILE_TOK <= T) {
+        const int4 s4 = *reinterpret_cast<const int4 *>(tt_slots + t);
+        const uchar4 k4 = *reinterpret_cast<const uchar4 *>(keep + t);
+        slot[0] = s4.x; slot[1] = s4.y; slot[2] = s4.z; slot[3] = s4.w;
+        kp[0] = k4.x; kp[1] = k4.y; kp[2] = k4.z; kp[3] = k4.w;
+    } else {
+#pragma unroll
+        for (int k = 0; k < VTK_TILE_TOK; ++k)
+            if (t + k < T) { slot[k] = tt_slots[t + k]; kp[k] = keep[t + k]; }
+    }
+    unsigned bits = 0;
+#pragma unroll
+    for (int k = 0; k < VTK_TILE_TOK; ++k) {
+        if (slot[k] < 0) continue;
+        if ((int64_t)slot[k] >= slots_per_layer) { bad = true; continue; }
+        if (kp[k] != 0) bits |= 1u << k;
+    }
+    return bits;
+}
+
+// The requests that own the first and the last entry of the tile [base, min(base + VTK_TILE, T)) --
+// owner of an entry: the last request whose first entry is at or before it; -1: the entry lies in
+// front of the first request -- each found by one warp (warps 0 and 1, all lanes) with a 32-way
+// search over the offsets; tile_req[2] is shared memory, valid after the caller's next barrier.
+__device__ __forceinline__ void vtk_tile_owners(const int32_t *off, int R, int64_t cap, int64_t base, int64_t T,
+                                                int *tile_req)
+{
+    const int warp = threadIdx.x >> 5, lane = vtk_lane();
+    if (warp >= 2) return;
+    const int64_t last = (base + VTK_TILE < T ? base + VTK_TILE : T) - 1;
+    const int64_t key = warp == 0 ? base : last;
+    int lo = -1, hi = R;                    // offset(lo) <= key (or lo == -1); offset(hi) > key: offset(R) = T
+    while (hi - lo > 1) {
+        const int step = (hi - lo - 1 + 31) / 32;
+        const int probe = lo + 1 + lane * step;
+        const bool le = probe < hi && vtk_clipped_offset(off, probe, cap) <= key;
+        const int n_le = __popc(__ballot_sync(0xffffffffu, le));
+        const int first_gt = lo + 1 + n_le * step;          // first probe beyond the key, if it was probed
+        if (n_le > 0) lo = lo + 1 + (n_le - 1) * step;
+        if (first_gt < hi) hi = first_gt;
+    }
+    if (lane == 0) tile_req[warp] = lo;
+}
+
+// The request that owns entry t of the tile whose owners are in tile_req (-1: none).
+__device__ __forceinline__ int vtk_entry_owner(const int32_t *off, int64_t cap, const int *tile_req, int64_t t)
+{
+    int lo = tile_req[0], hi = (tile_req[1] > tile_req[0] ? tile_req[1] : tile_req[0]) + 1;
+    while (hi - lo > 1) {                   // offset(lo) <= t (or lo == -1); offset(hi) > t
+        const int mid = (lo + hi) >> 1;
+        if (vtk_clipped_offset(off, mid, cap) <= t) lo = mid; else hi = mid;
+    }
+    return lo;
 }
 
 // A token is live when it owns a slot inside the pool and the policy kept it.

@@ -18,9 +18,9 @@
 
 namespace {
 
-constexpr int TILE_NT = 256;                     // threads per CTA of tiles / assign
-constexpr int TILE_TOK = 4;                      // table entries per thread
-constexpr int TILE = TILE_NT * TILE_TOK;         // entries per tile
+constexpr int TILE_NT = VTK_TILE_NT;             // threads per CTA of tiles / assign
+constexpr int TILE_TOK = VTK_TILE_TOK;           // table entries per thread
+constexpr int TILE = VTK_TILE;                   // entries per tile
 constexpr int SCAN_NT = 1024;                    // threads of the single scan CTA
 
 struct PlanArgs {
@@ -51,11 +51,9 @@ __device__ __forceinline__ int clamp_requests(const PlanArgs &a)
     return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
 }
 
-// first table entry of request r (r == R: one past the last entry), clipped to the table capacity
 __device__ __forceinline__ int64_t clipped_offset(const PlanArgs &a, int r)
 {
-    const int64_t o = a.tt_offsets[r];
-    return o < 0 ? 0 : (o > a.max_tokens ? a.max_tokens : o);
+    return vtk_clipped_offset(a.tt_offsets, r, a.max_tokens);
 }
 
 __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
@@ -64,31 +62,10 @@ __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
     atomicOr(&a.out_counts->error_flags, flags);
 }
 
-// The thread's four entries [t, t + 4) of the token table below T: slots, and one bit per live entry.
 __device__ __forceinline__ unsigned load_entries(const PlanArgs &a, int64_t t, int64_t T, int32_t (&slot)[TILE_TOK],
                                                  bool &bad)
 {
-    uint8_t kp[TILE_TOK] = {0, 0, 0, 0};
-#pragma unroll
-    for (int k = 0; k < TILE_TOK; ++k) slot[k] = -1;
-    if (a.vec_in && t + TILE_TOK <= T) {
-        const int4 s4 = *reinterpret_cast<const int4 *>(a.tt_slots + t);
-        const uchar4 k4 = *reinterpret_cast<const uchar4 *>(a.keep + t);
-        slot[0] = s4.x; slot[1] = s4.y; slot[2] = s4.z; slot[3] = s4.w;
-        kp[0] = k4.x; kp[1] = k4.y; kp[2] = k4.z; kp[3] = k4.w;
-    } else {
-#pragma unroll
-        for (int k = 0; k < TILE_TOK; ++k)
-            if (t + k < T) { slot[k] = a.tt_slots[t + k]; kp[k] = a.keep[t + k]; }
-    }
-    unsigned bits = 0;
-#pragma unroll
-    for (int k = 0; k < TILE_TOK; ++k) {
-        if (slot[k] < 0) continue;
-        if ((int64_t)slot[k] >= a.slots_per_layer) { bad = true; continue; }
-        if (kp[k] != 0) bits |= 1u << k;
-    }
-    return bits;
+    return vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, T, a.slots_per_layer, slot, bad);
 }
 
 // ---- tiles -----------------------------------------------------------------------------
@@ -100,41 +77,38 @@ __global__ void __launch_bounds__(TILE_NT) plan_tiles_kernel(PlanArgs a)
     const int R = clamp_requests(a);
     const int64_t T = clipped_offset(a, R);
     const int lane = vtk_lane(), warp = threadIdx.x >> 5;
+    // A CTA counts the live entries of [base, limit): a whole tile, or -- the CTAs behind the tiles, one
+    // per request boundary -- the entries between the start of the boundary's tile and the boundary
+    // (entries the tile's own CTA counts as well; flags are raised there).  Either way one pass.
+    const bool is_tile = (int)blockIdx.x < a.num_tiles;
+    const int r = (int)blockIdx.x - a.num_tiles;
+    int64_t base, limit;
+    if (is_tile) {
+        base = (int64_t)blockIdx.x * TILE;
+        limit = T;
+        if (base >= T) return;
+    } else {
+        if (r > R) return;
+        limit = clipped_offset(a, r);
+        base = limit / TILE * TILE;
+        if (base == limit) return;                       // nothing in front of it: the scan does not read req_part[r]
+    }
     bool bad = false;
     int32_t slot[TILE_TOK];
-    if ((int)blockIdx.x < a.num_tiles) {
-        // live entries of one tile
-        const int64_t base = (int64_t)blockIdx.x * TILE;
-        if (base >= T) return;
-        int n = __popc(load_entries(a, base + threadIdx.x * TILE_TOK, T, slot, bad));
+    int n = __popc(load_entries(a, base + threadIdx.x * TILE_TOK, limit, slot, bad));
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
-        if (lane == 0) warp_n[warp] = n;
-        const int any_bad = __syncthreads_or(bad);
-        if (threadIdx.x == 0) {
-            int s = 0;
+    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+    if (lane == 0) warp_n[warp] = n;
+    const int any_bad = __syncthreads_or(bad);
+    if (threadIdx.x == 0) {
+        int s = 0;
 #pragma unroll
-            for (int w = 0; w < TILE_NT / 32; ++w) s += warp_n[w];
-            // a slot outside the pool somewhere in the tile travels in the sign bit (the count is at most
-            // 1024): the scan kernel turns it into VTOKEN_FLAG_BAD_SLOT, and nothing has to be zeroed
-            // before this kernel
-            a.tile_n[blockIdx.x] = s | (any_bad ? (int)0x80000000 : 0);
-        }
-    } else {
-        // one warp per request boundary: live entries between the start of its tile and the boundary
-        // (entries the tile CTAs count as well; flags are raised there)
-        const int r = ((int)blockIdx.x - a.num_tiles) * (TILE_NT / 32) + warp;
-        if (r > R) return;
-        const int64_t o = clipped_offset(a, r);
-        const int64_t base = o / TILE * TILE;
-        int n = 0;
-        for (int64_t t = base + lane * TILE_TOK; t < o; t += 32 * TILE_TOK) {
-            unsigned bits = load_entries(a, t, o, slot, bad);     // entries at or behind the boundary do not count
-            n += __popc(bits);
-        }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
-        if (lane == 0) a.req_part[r] = n;
+        for (int w = 0; w < TILE_NT / 32; ++w) s += warp_n[w];
+        // a slot outside the pool somewhere in the tile travels in the sign bit (the count is at most
+        // 1024): the scan kernel turns it into VTOKEN_FLAG_BAD_SLOT, and nothing has to be zeroed
+        // before this kernel
+        if (is_tile) a.tile_n[blockIdx.x] = s | (any_bad ? (int)0x80000000 : 0);
+        else a.req_part[r] = s;
     }
 }
 
@@ -352,40 +326,13 @@ __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
     const int cnt = __popc(bits);
     const int incl = vtk_warp_incl_scan(cnt);
     if (lane == 31) warp_sums[warp] = incl;
-    // The requests that own the tile's first and last entry (owner of an entry: the last request whose
-    // first entry is at or before it; -1: the entry lies in front of the first request), each found by
-    // one warp with a 32-way search over the offsets.  Most tiles lie inside one or a few requests, so
-    // the per-thread search below has next to nothing left to do.
-    if (warp < 2) {
-        const int64_t last = (base + TILE < T ? base + TILE : T) - 1;
-        const int64_t key = warp == 0 ? base : last;
-        int lo = -1, hi = R;                    // offset(lo) <= key (or lo == -1); offset(hi) > key: offset(R) = T
-        while (hi - lo > 1) {
-            const int step = (hi - lo - 1 + 31) / 32;
-            const int probe = lo + 1 + lane * step;
-            const bool le = probe < hi && clipped_offset(a, probe) <= key;
-            const int n_le = __popc(__ballot_sync(0xffffffffu, le));
-            const int first_gt = lo + 1 + n_le * step;          // first probe beyond the key, if it was probed
-            if (n_le > 0) lo = lo + 1 + (n_le - 1) * step;
-            if (first_gt < hi) hi = first_gt;
-        }
-        if (lane == 0) tile_req[warp] = lo;
-    }
+    vtk_tile_owners(a.tt_offsets, R, a.max_tokens, base, T, tile_req);
     __syncthreads();
     int before = a.tile_n[blockIdx.x] + incl - cnt;
     for (int w = 0; w < warp; ++w) before += warp_sums[w];
     if (t >= T) return;
 
-    // the request that owns entry t
-    int r;
-    {
-        int lo = tile_req[0], hi = (tile_req[1] > tile_req[0] ? tile_req[1] : tile_req[0]) + 1;
-        while (hi - lo > 1) {                   // offset(lo) <= t (or lo == -1); offset(hi) > t
-            const int mid = (lo + hi) >> 1;
-            if (clipped_offset(a, mid) <= t) lo = mid; else hi = mid;
-        }
-        r = lo;                                 // -1: an entry before the first request's range
-    }
+    int r = vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t);      // -1: in front of the first request
     int64_t next = r + 1 <= R ? clipped_offset(a, r + 1) : T;
     int req_before = 0, n = 0, dst_base = 0;
     bool adm = false;
@@ -476,8 +423,7 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.vec_out = ((uintptr_t)out->new_tt_slots % 16 == 0) ? 1 : 0;
 
     const int R = ctx->cfg.max_requests;
-    VTK_CUDA(ctx, vtk_launch_dependent(plan_tiles_kernel, dim3(a.num_tiles + (R + 1 + TILE_NT / 32 - 1) / (TILE_NT / 32)),
-                                       dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(plan_tiles_kernel, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(plan_scan_kernel, dim3(1), dim3(SCAN_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(plan_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());

@@ -3,16 +3,23 @@
 // low-utilisation, unprotected source blocks of a request (at most B of them) and leaves the
 // others -- fully live blocks, shared-prefix blocks -- where they are.
 //
-// Kernels (all grids fixed by the capacities, counts read from device memory):
-//   live    : live tokens per request part; n_b[block] += 1 per live token (integer atomics: the
-//             sums do not depend on their order)
+// Kernels (all grids fixed by the capacities, counts read from device memory).  The token table is
+// walked in flat tiles of 1024 entries that ignore request boundaries (see plan.cu); per-request
+// numbers are differences of running counts at the request's two boundaries:
+//   tiles<0>: live tokens per tile and in front of every request boundary inside its tile;
+//             n_b[block] += 1 per live token (integer atomics: the sums do not depend on their
+//             order); with a detach threshold also the live tokens that sit in protected blocks
 //   blocks  : per request, which entries of its block table are sources (rank among eligible
-//             entries in table order < B); marks blk_src[block]
-//   src     : live tokens that sit in source blocks, per request part
-//   scan    : global trigger F > theta, candidates (sources release more blocks than the
-//             destinations they need), admission against the free list, bases and counts
-//   assign  : new token table (moving tokens ranked in logical order), new block table
-//             (kept blocks in old order, then destinations), reclaimed list, inverse move plan
+//             entries in table order < B); marks blk_src[block]; decides copy-on-write detach
+//   tiles<1>: live tokens that move (they sit in a source block of their request), per tile and
+//             in front of every request boundary
+//   scan    : running counts at every tile start, live and moving tokens per request, global
+//             trigger F > theta, candidates (sources release more blocks than the destinations
+//             they need), admission against the free list, bases and counts
+//   assign  : new token table (moving tokens ranked in logical order: running count at the token
+//             minus running count at the request's first entry), inverse move plan; one extra CTA
+//             per request writes the new block table (kept blocks in old order, then
+//             destinations), the reclaimed and the released list
 // The inverse plan has the same form as the whole-request planner's, so vtoken_repack runs it
 // unchanged.
 //
@@ -27,9 +34,9 @@
 
 namespace {
 
-constexpr int PP_NT = 512;
-constexpr int PP_PARTS = VTK_PLAN_PARTS;
+constexpr int PP_NT = 512;                 // threads of a blocks CTA (one per request)
 constexpr int PP_SCAN_NT = 1024;
+constexpr int TILE_NT = VTK_TILE_NT, TILE_TOK = VTK_TILE_TOK, TILE = VTK_TILE;
 
 struct PArgs {
     const int32_t *num_requests, *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
@@ -39,13 +46,18 @@ struct PArgs {
     const int32_t *free_blocks, *num_free;
     int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *released_blocks, *out_status;
     vtoken_counts *out_counts;
-    int32_t *req_n, *part_n, *part_src, *req_ns, *req_nsrc, *req_dst_base, *req_freed_base, *req_status;
-    int32_t *part_shared, *req_shared, *req_detach, *req_rel_base;
+    int32_t *req_n, *req_ns, *req_nsrc, *req_dst_base, *req_freed_base, *req_status;
+    int32_t *req_shared, *req_detach, *req_rel_base;
+    // flat tiling: counts per tile ([num_tiles + 1]; live and moving become running counts in the scan
+    // kernel; the sign bit of a live count says "a slot outside the pool in this tile") and counts
+    // between the start of the tile that holds a request's first entry and that entry ([max_requests + 1])
+    int32_t *tile_live, *tile_mov, *tile_shared, *part_live, *part_mov, *part_shared;
+    int32_t *req_before;     // [max_requests + 1] moving tokens of the table before the request's first entry
     int32_t *dst_src, *dst_blocks, *n_b;
     uint8_t *blk_src;
     vtoken_counts *counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
-    int32_t parts;          // token ranges (CTAs) per request, <= PP_PARTS (the stride of the part_* arrays)
+    int32_t num_tiles, vec_in, vec_out;
     int64_t slots_per_layer, max_tokens, max_table_blocks;
 };
 
@@ -55,14 +67,9 @@ __device__ __forceinline__ int pp_requests(const PArgs &a)
     return R < 0 ? 0 : (R > a.max_requests ? a.max_requests : R);
 }
 
-__device__ __forceinline__ void pp_part_range(int64_t t0, int64_t t1, int c, int parts, int64_t &p0, int64_t &p1)
+__device__ __forceinline__ int64_t pp_offset(const PArgs &a, int r)
 {
-    int64_t per = (t1 - t0 + parts - 1) / parts;
-    per = (per + 127) & ~(int64_t)127;
-    p0 = t0 + (int64_t)c * per;
-    p1 = p0 + per;
-    if (p0 > t1) p0 = t1;
-    if (p1 > t1) p1 = t1;
+    return vtk_clipped_offset(a.tt_offsets, r, a.max_tokens);
 }
 
 __device__ __forceinline__ int pp_block_sum(int n, int *warp_n)
@@ -85,47 +92,97 @@ __device__ __forceinline__ bool pp_moves(const PArgs &a, bool detach, int32_t b)
     return a.blk_src[b] != 0 || (detach && a.protect[b] != 0);
 }
 
-// mode 0: count live tokens and add them to n_b (and, when a detach threshold is set, count the
-// ones in protected blocks); mode 1: count live tokens that move
-template <int MODE>
-__global__ void __launch_bounds__(PP_NT) pp_count_kernel(PArgs a)
+// Bits of the thread's live entries that move.  Without a detach threshold that is a property of the
+// block alone; with one, protected blocks move for the requests that leave them, so the owner of
+// every entry is needed: r is the owner of entry t (-1: none) and is stepped over request boundaries.
+__device__ __forceinline__ unsigned pp_moving_bits(const PArgs &a, unsigned bits, const int32_t (&slot)[TILE_TOK],
+                                                   bool may_detach, int R, int64_t t, int r)
 {
+    unsigned mov = 0;
+    int64_t next = may_detach ? pp_offset(a, r + 1 <= R ? r + 1 : R) : 0;
+    bool detach = may_detach && r >= 0 && a.req_detach[r] != 0;
+#pragma unroll
+    for (int k = 0; k < TILE_TOK; ++k) {
+        if (may_detach && t + k >= next && r + 1 < R) {
+            while (r + 1 < R && pp_offset(a, r + 1) <= t + k) ++r;
+            next = pp_offset(a, r + 1);
+            detach = r >= 0 && a.req_detach[r] != 0;
+        }
+        if ((bits >> k) & 1u)
+            if (pp_moves(a, detach, slot[k] / a.S)) mov |= 1u << k;
+    }
+    return mov;
+}
+
+// mode 0: live tokens per tile, n_b (and, with a detach threshold, the live tokens in protected
+// blocks); mode 1: live tokens that move.
+template <int MODE>
+__global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
+{
+    __shared__ int warp_n[TILE_NT / 32], warp_sh[TILE_NT / 32];
+    __shared__ int tile_req[2];
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    __shared__ int warp_n[PP_NT / 32];
-    const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
-    if (r >= pp_requests(a)) return;
-    int64_t t0, t1, p0, p1;
-    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
-    pp_part_range(t0, t1, c, a.parts, p0, p1);
+    const int R = pp_requests(a);
+    const int64_t T = pp_offset(a, R);
+    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
     const bool may_detach = a.protect != nullptr && a.detach_den != 0;
-    const bool detach = MODE == 1 && may_detach && a.req_detach[r] != 0;
-    int n = 0, n_shared = 0;
-    bool bad = false;
-    for (int64_t tb = p0; tb < p1; tb += PP_NT) {           // the same trip count for every thread of the CTA
-        const int64_t t = tb + threadIdx.x;
-        int blk = -1;                                        // block of this thread's token, -1: not live
-        if (t < p1) {
-            const int32_t slot = a.tt_slots[t];
-            if (vtk_live(slot, a.keep, t, a.slots_per_layer, bad)) blk = slot / a.S;
-        }
-        if (MODE == 0) {
-            if (blk >= 0) {
-                atomicAdd(&a.n_b[blk], 1);
-                ++n;
-                if (may_detach) n_shared += a.protect[blk] != 0;
-            }
-        } else if (blk >= 0) {
-            n += pp_moves(a, detach, blk);
-        }
+    // A CTA counts over the entries [base, limit): a whole tile, or (the CTAs behind the tiles, one per
+    // request boundary) the entries between the start of the boundary's tile and the boundary.
+    const bool is_tile = (int)blockIdx.x < a.num_tiles;
+    const int rb = (int)blockIdx.x - a.num_tiles;
+    int64_t base, limit;
+    if (is_tile) {
+        base = (int64_t)blockIdx.x * TILE;
+        limit = T;
+        if (base >= T) return;
+    } else {
+        if (rb > R) return;
+        limit = pp_offset(a, rb);
+        base = limit / TILE * TILE;
+        if (base == limit) return;                       // nothing in front of it: never read
     }
-    if (bad && MODE == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
-    const int s = pp_block_sum(n, warp_n);
-    if (threadIdx.x == 0) (MODE == 0 ? a.part_n : a.part_src)[r * PP_PARTS + c] = s;
-    if (MODE == 0 && may_detach) {
-        __syncthreads();                       // warp_n is reused
-        const int sh = pp_block_sum(n_shared, warp_n);
-        if (threadIdx.x == 0) a.part_shared[r * PP_PARTS + c] = sh;
+    bool bad = false;
+    int32_t slot[TILE_TOK];
+    const int64_t t = base + threadIdx.x * TILE_TOK;
+    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, limit, a.slots_per_layer, slot, bad);
+    int n = 0, n_sh = 0;
+    if (MODE == 0) {
+#pragma unroll
+        for (int k = 0; k < TILE_TOK; ++k) {
+            if (!((bits >> k) & 1u)) continue;
+            const int blk = slot[k] / a.S;
+            if (is_tile) atomicAdd(&a.n_b[blk], 1);          // the tile CTAs see every entry exactly once
+            ++n;
+            if (may_detach) n_sh += a.protect[blk] != 0;
+        }
+    } else {
+        int r = -1;
+        if (may_detach) {                                      // uniform over the CTA
+            vtk_tile_owners(a.tt_offsets, R, a.max_tokens, base, limit, tile_req);
+            __syncthreads();
+            if (t < limit) r = vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t);
+        }
+        n = __popc(pp_moving_bits(a, bits, slot, may_detach, R, t, r));
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        n += __shfl_down_sync(0xffffffffu, n, d);
+        n_sh += __shfl_down_sync(0xffffffffu, n_sh, d);
+    }
+    if (lane == 0) { warp_n[warp] = n; warp_sh[warp] = n_sh; }
+    const int any_bad = __syncthreads_or(bad);
+    if (threadIdx.x == 0) {
+        int s = 0, sh = 0;
+#pragma unroll
+        for (int w = 0; w < TILE_NT / 32; ++w) { s += warp_n[w]; sh += warp_sh[w]; }
+        if (MODE == 0) {
+            if (is_tile) a.tile_live[blockIdx.x] = s | (any_bad ? (int)0x80000000 : 0);   // flag in the sign bit
+            else a.part_live[rb] = s;
+            if (may_detach) (is_tile ? a.tile_shared[blockIdx.x] : a.part_shared[rb]) = sh;
+        } else {
+            (is_tile ? a.tile_mov[blockIdx.x] : a.part_mov[rb]) = s;
+        }
     }
 }
 
@@ -170,9 +227,17 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
         // fill less than detach_num / detach_den of them; then every one of them is a source
         __syncthreads();
         const int ns_shared = pp_block_sum(shared, warp_sums);          // valid in thread 0
+        // the request's live tokens in protected blocks: the tiles between its two boundaries, corrected
+        // at both ends by the counts in front of the boundaries
+        const int64_t o0 = pp_offset(a, r), o1 = pp_offset(a, r + 1);
+        int in_tiles = 0;
+        for (int64_t i = o0 / TILE + threadIdx.x; i < o1 / TILE; i += PP_NT) in_tiles += a.tile_shared[i];
+        __syncthreads();
+        in_tiles = pp_block_sum(in_tiles, warp_sums);                   // valid in thread 0
         if (threadIdx.x == 0) {
-            long long n_shared = 0;
-            for (int c = 0; c < a.parts; ++c) n_shared += a.part_shared[r * PP_PARTS + c];
+            long long n_shared = (long long)in_tiles + (o1 % TILE != 0 ? a.part_shared[r + 1] : 0) -
+                                 (o0 % TILE != 0 ? a.part_shared[r] : 0);
+            if (n_shared < 0) n_shared = 0;                             // offsets that run backwards
             const bool detach = ns_shared > 0 &&
                                 (unsigned long long)n_shared * a.detach_den <
                                     (unsigned long long)a.detach_num * (unsigned long long)ns_shared * (unsigned long long)a.S;
@@ -236,12 +301,15 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     __shared__ PAcc warp_acc[32];
     __shared__ long long carry_need, tot_live, tot_blocks;
     __shared__ PAcc carry;
+    __shared__ int carry_live, carry_mov;
     const int tid = threadIdx.x;
     const int R = pp_requests(a);
     uint32_t flags = 0;
     if (tid == 0) {
         if (*a.num_requests > a.max_requests || *a.num_requests < 0) flags |= VTOKEN_FLAG_CAPACITY;
         carry_need = 0;
+        carry_live = 0;
+        carry_mov = 0;
         tot_live = 0;
         tot_blocks = 0;
         carry = PAcc{0, 0, 0, 0, 0, 0, 0};
@@ -253,15 +321,48 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     auto shfl_ll = [](long long v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
     auto shfl_acc = [](const PAcc &v, int d) { return pp_shfl_up(v, d); };
 
-    // pass 1: live tokens per request, and the totals behind F = 1 - live / (N * S)
+    // live and moving tokens before every tile (in place: an entry becomes the sum of the tiles before
+    // it; one entry past the last tile holds the total)
+    const int64_t T = pp_offset(a, R);
+    const int tiles = (int)((T + TILE - 1) / TILE);
+    auto shfl_ll2 = [](long long v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
+    for (int base = 0; base <= tiles; base += PP_SCAN_NT) {
+        const int i = base + tid;
+        const int raw = i < tiles ? a.tile_live[i] : 0;
+        if (raw < 0) flags |= VTOKEN_FLAG_BAD_SLOT;
+        const long long v = ((long long)(raw & 0x7fffffff) << 32) | (unsigned)(i < tiles ? a.tile_mov[i] : 0);
+        // both counts in one 64-bit scan: live in the high half, moving in the low half (each < 2^31)
+        const long long incl = pp_block_incl_scan<long long>(v, warp_ll, 0LL, shfl_ll2) +
+                               (((long long)carry_live << 32) | (unsigned)carry_mov);
+        if (i <= tiles) {
+            a.tile_live[i] = (int)((incl - v) >> 32);
+            a.tile_mov[i] = (int)((incl - v) & 0xffffffffll);
+        }
+        __syncthreads();
+        if (tid == PP_SCAN_NT - 1) {
+            carry_live = (int)(incl >> 32);
+            carry_mov = (int)(incl & 0xffffffffll);
+        }
+        __syncthreads();
+    }
+    // tokens before table entry o = tokens before its tile + those between the tile's start and o
+    auto live_before = [&](int r) {
+        const int64_t o = pp_offset(a, r);
+        return a.tile_live[o / TILE] + (o % TILE != 0 ? a.part_live[r] : 0);
+    };
+    auto mov_before = [&](int r) {
+        const int64_t o = pp_offset(a, r);
+        return a.tile_mov[o / TILE] + (o % TILE != 0 ? a.part_mov[r] : 0);
+    };
+
+    // pass 1: live and moving tokens per request, and the totals behind F = 1 - live / (N * S)
     long long my_live = 0, my_blocks = 0;
     for (int r = tid; r < R; r += PP_SCAN_NT) {
-        int n = 0, nsrc = 0;
-#pragma unroll
-        for (int c = 0; c < a.parts; ++c) {
-            n += a.part_n[r * PP_PARTS + c];
-            nsrc += a.part_src[r * PP_PARTS + c];
-        }
+        const int mb = mov_before(r);
+        int n = live_before(r + 1) - live_before(r), nsrc = mov_before(r + 1) - mb;
+        if (n < 0) n = 0;                                   // offsets that run backwards
+        if (nsrc < 0) nsrc = 0;
+        a.req_before[r] = mb;
         a.req_n[r] = n;
         a.req_nsrc[r] = nsrc;
         int64_t lo, hi, t0, t1;
@@ -343,45 +444,47 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
 }
 
 // ---- assign --------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
+__global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
 {
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    __shared__ int warp_sums[PP_NT / 32 + 1];
-    const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
-    if (r >= pp_requests(a)) return;
-    const int tid = threadIdx.x;
+    __shared__ int warp_sums[TILE_NT / 32 + 1];
+    __shared__ int tile_req[2];
+    const int R = pp_requests(a);
+    const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
     const int S = a.S;
-    int64_t t0, t1, b0, b1;
-    vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
-    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
-    const int nb = (int)(b1 - b0);
-    const int64_t cap_bt = a.max_table_blocks;               // every table write below stays inside its buffer
-    const bool adm = a.req_status[r] == VTOKEN_REPACKED;
-    const bool detach = adm && a.protect != nullptr && a.detach_den != 0 && a.req_detach[r] != 0;
-    const int nsrc = a.req_nsrc[r], ns = a.req_ns[r];
-    const int need = (int)(((int64_t)nsrc + S - 1) / S);
-    const int dst_base = a.req_dst_base[r];
-    const int nbt0 = a.new_bt_offsets[r];
+    const bool may_detach = a.protect != nullptr && a.detach_den != 0;
     uint32_t flags = 0;
 
-    const int stripe = c * PP_NT + tid, stride = a.parts * PP_NT;
-    if (adm) {
-        // destinations follow the kept blocks in the new block table
-        for (int j = stripe; j < need; j += stride) {
-            int blk = a.free_blocks[dst_base + j];
-            if ((int64_t)nbt0 + (nb - ns) + j < cap_bt) a.new_bt_blocks[nbt0 + (nb - ns) + j] = blk;
-            if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
-            a.dst_blocks[dst_base + j] = blk;
-        }
-        for (int i = nsrc + stripe; i < need * S; i += stride) a.dst_src[(int64_t)dst_base * S + i] = -1;
-        // kept blocks in old order, unprotected sources to the reclaimed list and protected sources (of a
-        // detaching request) to the released list, each in old order: one CTA ranks the table
-        if (c == 0) {
+    if ((int)blockIdx.x >= a.num_tiles) {
+        // block table, reclaimed and released list of one request
+        const int r = (int)blockIdx.x - a.num_tiles;
+        if (r >= R) return;
+        int64_t b0, b1;
+        vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
+        const int nb = (int)(b1 - b0);
+        const int64_t cap_bt = a.max_table_blocks;               // every table write below stays inside its buffer
+        const bool adm = a.req_status[r] == VTOKEN_REPACKED;
+        const bool detach = adm && may_detach && a.req_detach[r] != 0;
+        const int nsrc = a.req_nsrc[r], ns = a.req_ns[r];
+        const int need = (int)(((int64_t)nsrc + S - 1) / S);
+        const int dst_base = a.req_dst_base[r];
+        const int nbt0 = a.new_bt_offsets[r];
+        if (adm) {
+            // destinations follow the kept blocks in the new block table
+            for (int j = tid; j < need; j += TILE_NT) {
+                int blk = a.free_blocks[dst_base + j];
+                if ((int64_t)nbt0 + (nb - ns) + j < cap_bt) a.new_bt_blocks[nbt0 + (nb - ns) + j] = blk;
+                if (blk < 0 || blk >= a.num_blocks) { flags |= VTOKEN_FLAG_BAD_FREE; blk = -1; }
+                a.dst_blocks[dst_base + j] = blk;
+            }
+            for (int i = nsrc + tid; i < need * S; i += TILE_NT) a.dst_src[(int64_t)dst_base * S + i] = -1;
+            // kept blocks in old order, unprotected sources to the reclaimed list and protected sources (of a
+            // detaching request) to the released list, each in old order
             const int f0 = a.req_freed_base[r];
             const int l0 = detach ? a.req_rel_base[r] : 0;
             int carry_src = 0, carry_rel = 0;
-            for (int64_t jb = b0; jb < b1; jb += PP_NT) {
+            for (int64_t jb = b0; jb < b1; jb += TILE_NT) {
                 const int64_t j = jb + tid;
                 int blk = -1;
                 bool src = false, rel = false;
@@ -393,11 +496,11 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
                     }
                 }
                 int total;
-                const int rank_src = carry_src + vtk_block_rank<PP_NT>(src, warp_sums, total);
+                const int rank_src = carry_src + vtk_block_rank<TILE_NT>(src, warp_sums, total);
                 carry_src += total;
                 int rank_rel = 0;
                 if (detach) {                                   // uniform over the CTA
-                    rank_rel = carry_rel + vtk_block_rank<PP_NT>(rel, warp_sums, total);
+                    rank_rel = carry_rel + vtk_block_rank<TILE_NT>(rel, warp_sums, total);
                     carry_rel += total;
                 }
                 if (j < b1) {
@@ -407,45 +510,78 @@ __global__ void __launch_bounds__(PP_NT) pp_assign_kernel(PArgs a)
                     else if (kept < cap_bt) a.new_bt_blocks[kept] = blk;
                 }
             }
+        } else {
+            for (int j = tid; j < nb && (int64_t)nbt0 + j < cap_bt; j += TILE_NT)
+                a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
         }
-    } else {
-        for (int j = stripe; j < nb && (int64_t)nbt0 + j < cap_bt; j += stride)
-            a.new_bt_blocks[nbt0 + j] = a.bt_blocks[b0 + j];
+        if (flags) {
+            atomicOr(&a.counts->error_flags, flags);
+            atomicOr(&a.out_counts->error_flags, flags);
+        }
+        return;
     }
 
-    // token table
-    int64_t p0, p1;
-    pp_part_range(t0, t1, c, a.parts, p0, p1);
-    int carry = 0;                                       // moving tokens of the parts before this one
-    for (int cc = 0; cc < c; ++cc) carry += a.part_src[r * PP_PARTS + cc];
-    for (int64_t tb = p0; tb < p1; tb += PP_NT) {
-        const int64_t t = tb + tid;
-        int32_t slot = -1;
-        bool live = false, bad = false, moving = false;
-        if (t < p1) {
-            slot = a.tt_slots[t];
-            live = vtk_live(slot, a.keep, t, a.slots_per_layer, bad);
-            moving = live && adm && pp_moves(a, detach, slot / S);
+    // token table: moving tokens ranked in logical order -> destination slot; the others keep theirs
+    const int64_t T = pp_offset(a, R);
+    const int64_t base = (int64_t)blockIdx.x * TILE;
+    if (base >= T) return;
+    const int64_t t = base + tid * TILE_TOK;
+    int32_t slot[TILE_TOK];
+    bool bad = false;
+    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, T, a.slots_per_layer, slot, bad);
+    vtk_tile_owners(a.tt_offsets, R, a.max_tokens, base, T, tile_req);
+    __syncthreads();
+    int r = t < T ? vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t) : -1;
+    // Live entries that sit in a source block of their request, by the rule the tile counts in tile_mov
+    // were taken with (admission was not known then): inside an admitted request every one of them
+    // moves, and ranks are only used there.
+    const unsigned mov = pp_moving_bits(a, bits, slot, may_detach, R, t, r);
+    const int cnt = __popc(mov);
+    const int incl = vtk_warp_incl_scan(cnt);
+    if (lane == 31) warp_sums[warp] = incl;
+    __syncthreads();
+    int before = a.tile_mov[blockIdx.x] + incl - cnt;        // such tokens of the whole table before entry t
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    if (t >= T) return;
+
+    int64_t next = pp_offset(a, r + 1);                      // r + 1 <= R
+    int req_before = 0, nsrc = 0, dst_base = 0;
+    bool adm = false;
+    auto load_request = [&]() {
+        req_before = a.req_before[r];
+        nsrc = a.req_nsrc[r];
+        dst_base = a.req_dst_base[r];
+        adm = a.req_status[r] == VTOKEN_REPACKED;
+    };
+    if (r >= 0) load_request();
+    int32_t out[TILE_TOK];
+    bool owned = true;
+#pragma unroll
+    for (int k = 0; k < TILE_TOK; ++k) {
+        out[k] = -1;
+        if (t + k >= T) { owned = false; continue; }
+        if (t + k >= next && r + 1 < R) {                     // a request boundary inside the thread's entries
+            while (r + 1 < R && pp_offset(a, r + 1) <= t + k) ++r;
+            next = pp_offset(a, r + 1);
+            load_request();
         }
-        int total;
-        const int i = carry + vtk_block_rank<PP_NT>(moving, warp_sums, total);
-        carry += total;
-        if (t < p1) {
-            int32_t out = -1;
-            if (moving) {
-                const int j = i / S, off = i - j * S;
-                const int blk = a.free_blocks[dst_base + j];
-                out = blk * S + off;
-                a.dst_src[(int64_t)(dst_base + j) * S + off] = slot;
-            } else if (live) {
-                out = slot;                              // its block stays in place
-            }
-            a.new_tt_slots[t] = out;
-        }
+        if (r < 0) { owned = false; continue; }               // in front of the first request: left untouched
+        if (!((bits >> k) & 1u)) continue;                    // dead or unmapped: -1
+        if (!adm || !((mov >> k) & 1u)) { out[k] = slot[k]; continue; }   // its block stays in place
+        const int i = before + __popc(mov & ((1u << k) - 1u)) - req_before;   // rank among the request's movers
+        if (i < 0 || i >= nsrc) continue;                     // only with inconsistent offsets
+        const int j = i / S, off = i - j * S;
+        const int blk = a.free_blocks[dst_base + j];
+        out[k] = blk * S + off;
+        a.dst_src[(int64_t)(dst_base + j) * S + off] = slot[k];
     }
-    if (flags) {
-        atomicOr(&a.counts->error_flags, flags);
-        atomicOr(&a.out_counts->error_flags, flags);
+    if (owned && a.vec_out) {
+        *reinterpret_cast<int4 *>(a.new_tt_slots + t) = make_int4(out[0], out[1], out[2], out[3]);
+    } else {
+        const int64_t first = pp_offset(a, 0);
+#pragma unroll
+        for (int k = 0; k < TILE_TOK; ++k)
+            if (t + k < T && t + k >= first) a.new_tt_slots[t + k] = out[k];
     }
 }
 
@@ -486,17 +622,20 @@ __global__ void __launch_bounds__(256) pp_hist_kernel(const int32_t *num_request
 }
 
 __global__ void __launch_bounds__(1024) pp_summary_kernel(const int32_t *num_requests, int32_t max_requests,
-                                                          const int32_t *bt_offsets, const int32_t *part_n,
-                                                          int parts, long long *summary)
+                                                          const int32_t *bt_offsets, const int32_t *tt_offsets,
+                                                          int64_t max_tokens, const int32_t *tile_live,
+                                                          long long *summary)
 {
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    // one CTA: total live tokens over all parts, allocated blocks
+    // one CTA: total live tokens over all tiles (the sign bit of a count is a flag), allocated blocks
     __shared__ long long warp_s[32];
     int R = *num_requests;
     R = R < 0 ? 0 : (R > max_requests ? max_requests : R);
+    const int64_t T = vtk_clipped_offset(tt_offsets, R, max_tokens);
+    const int tiles = (int)((T + TILE - 1) / TILE);
     long long s = 0;
-    for (int i = threadIdx.x; i < R * parts; i += 1024) s += part_n[i / parts * PP_PARTS + i % parts];
+    for (int i = threadIdx.x; i < tiles; i += 1024) s += tile_live[i] & 0x7fffffff;
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) s += __shfl_down_sync(0xffffffffu, s, d);
     if (vtk_lane() == 0) warp_s[threadIdx.x >> 5] = s;
@@ -515,8 +654,12 @@ __global__ void __launch_bounds__(1024) pp_summary_kernel(const int32_t *num_req
 void fill_args(PArgs &a, vtoken_ctx *ctx)
 {
     a.req_n = ctx->req_n;
-    a.part_n = ctx->part_n;
-    a.part_src = ctx->part_src;
+    a.tile_live = ctx->tile_n;
+    a.tile_mov = ctx->tile_mov;
+    a.tile_shared = ctx->tile_shared;
+    a.part_live = ctx->req_part;
+    a.part_mov = ctx->part_mov;
+    a.req_before = ctx->req_before;
     a.req_ns = ctx->req_ns;
     a.req_nsrc = ctx->req_nsrc;
     a.req_dst_base = ctx->req_dst_base;
@@ -539,7 +682,8 @@ void fill_args(PArgs &a, vtoken_ctx *ctx)
     a.slots_per_layer = ctx->slots_per_layer;
     a.max_tokens = ctx->cfg.max_tokens;
     a.max_table_blocks = ctx->cfg.max_table_blocks;
-    a.parts = ctx->parts;
+    a.num_tiles = (int32_t)((ctx->cfg.max_tokens + TILE - 1) / TILE);
+    a.vec_in = a.vec_out = 0;
 }
 
 }  // namespace
@@ -588,15 +732,19 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     a.out_status = out->req_status;
     a.out_counts = out->counts;
 
+    a.vec_in = ((uintptr_t)in->tt_slots % 16 == 0 && (uintptr_t)in->keep % 4 == 0) ? 1 : 0;
+    a.vec_out = ((uintptr_t)out->new_tt_slots % 16 == 0) ? 1 : 0;
+
     const int R = ctx->cfg.max_requests;
+    const dim3 tiles_grid(a.num_tiles + R + 1);
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
-    VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
-    VTK_CUDA(ctx, cudaMemsetAsync(ctx->blk_src, 0, (size_t)ctx->cfg.num_blocks, st));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
+    // n_b and blk_src share one allocation: one node clears both
+    VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, (sizeof(int32_t) + 1) * (size_t)ctx->cfg.num_blocks, st));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_tiles_kernel<0>, tiles_grid, dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(pp_blocks_kernel, dim3(R), dim3(PP_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<1>, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_tiles_kernel<1>, tiles_grid, dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(pp_scan_kernel, dim3(1), dim3(PP_SCAN_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_assign_kernel, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     ctx->has_plan = true;
     return VTOKEN_OK;
@@ -620,7 +768,8 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     a.n_b = n_b;
     const int R = ctx->cfg.max_requests;
     VTK_CUDA(ctx, cudaMemsetAsync(n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_count_kernel<0>, dim3(R * a.parts), dim3(PP_NT), 0, st, a));
+    a.vec_in = ((uintptr_t)tt_slots % 16 == 0 && (uintptr_t)keep % 4 == 0) ? 1 : 0;
+    VTK_CUDA(ctx, vtk_launch_dependent(pp_tiles_kernel<0>, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
     if (hist) {
         VTK_CUDA(ctx, cudaMemsetAsync(hist, 0, sizeof(uint64_t) * (size_t)(ctx->cfg.block_size + 1), st));
         VTK_CUDA(ctx, vtk_launch_dependent(pp_hist_kernel, dim3(ctx->num_sms * 4), dim3(256), 0, st, num_requests, R,
@@ -629,7 +778,8 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     }
     if (summary)
         VTK_CUDA(ctx, vtk_launch_dependent(pp_summary_kernel, dim3(1), dim3(1024), 0, st, num_requests, R, bt_offsets,
-                                           (const int32_t *)ctx->part_n, ctx->parts, (long long *)summary));
+                                           tt_offsets, ctx->cfg.max_tokens, (const int32_t *)ctx->tile_n,
+                                           (long long *)summary));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

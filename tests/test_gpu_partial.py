@@ -90,9 +90,9 @@ def test_partial_plans_small_whole_pool(w, opts):
 
 @pytest.mark.parametrize("parts", ["1", "2", "3", "8"])
 def test_token_ranges_per_request(parts, monkeypatch):
-    """The per-request kernels (partial planner, block liveness, logical gather, slot mapping) cut every
-    request into a number of token ranges chosen at create from the capacities; every count gives the
-    same result."""
+    """The kernels that walk the token table request by request (logical gather, slot mapping) cut every
+    request into a number of token ranges chosen at create from the capacities; every count gives the same
+    result, and the planners and the block liveness (flat tiles) do not depend on it."""
     import torch
     from paper_2608_13263_b200.device import DeviceProblem
     monkeypatch.setenv("VTOKEN_PLAN_PARTS", parts)

@@ -138,7 +138,8 @@ typedef struct {                   /* all DEVICE pointers, read-only to the libr
     const int32_t *num_requests;   /* device scalar R <= max_requests */
     const int32_t *bt_offsets;     /* [R+1] CSR offsets into bt_blocks */
     const int32_t *bt_blocks;      /* [bt_offsets[R]] physical block ids, logical block order */
-    const int32_t *tt_offsets;     /* [R+1] CSR offsets into tt_slots / keep */
+    const int32_t *tt_offsets;     /* [R+1] CSR offsets into tt_slots / keep, non-decreasing; entries in front of
+                                      tt_offsets[0] belong to no request: neither read as tokens nor written */
     const int32_t *tt_slots;       /* [tt_offsets[R]] slot = block*S+offset, or -1 */
     const uint8_t *keep;           /* [tt_offsets[R]] 0 = evicted, non-zero = keep */
     const uint8_t *select;         /* [R] or NULL (= every request) */

@@ -213,9 +213,10 @@ __device__ __forceinline__ int64_t vtk_clipped_offset(const int32_t *off, int r,
 }
 
 // The thread's four entries [t, t + 4) of the token table below T: slots, and one bit per live entry.
+// Entries in front of `first` (the first request's first entry) belong to no request and count as dead.
 // vec: tt_slots is 16-byte and keep 4-byte aligned (t is a multiple of four).
 __device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, const uint8_t *keep, int vec, int64_t t,
-                                                     int64_t T, int64_t slots_per_layer,
+                                                     int64_t first, int64_t T, int64_t slots_per_layer,
                                                      int32_t (&slot)[VTK_TILE_TOK], bool &bad)
 {
     uint8_t kp[VTK_TILE_TOK] = {0, 0, 0, 0};
@@ -234,7 +235,7 @@ __device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, co
     unsigned bits = 0;
 #pragma unroll
     for (int k = 0; k < VTK_TILE_TOK; ++k) {
-        if (slot[k] < 0) continue;
+        if (slot[k] < 0 || t + k < first) continue;
         if ((int64_t)slot[k] >= slots_per_layer) { bad = true; continue; }
         if (kp[k] != 0) bits |= 1u << k;
     }

@@ -65,7 +65,7 @@ __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
 __device__ __forceinline__ unsigned load_entries(const PlanArgs &a, int64_t t, int64_t T, int32_t (&slot)[TILE_TOK],
                                                  bool &bad)
 {
-    return vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, T, a.slots_per_layer, slot, bad);
+    return vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, clipped_offset(a, 0), T, a.slots_per_layer, slot, bad);
 }
 
 // ---- tiles -----------------------------------------------------------------------------

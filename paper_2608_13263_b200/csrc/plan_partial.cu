@@ -145,7 +145,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
     bool bad = false;
     int32_t slot[TILE_TOK];
     const int64_t t = base + threadIdx.x * TILE_TOK;
-    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, limit, a.slots_per_layer, slot, bad);
+    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, pp_offset(a, 0), limit, a.slots_per_layer, slot, bad);
     int n = 0, n_sh = 0;
     if (MODE == 0) {
 #pragma unroll
@@ -528,7 +528,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
     const int64_t t = base + tid * TILE_TOK;
     int32_t slot[TILE_TOK];
     bool bad = false;
-    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, T, a.slots_per_layer, slot, bad);
+    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, pp_offset(a, 0), T, a.slots_per_layer, slot, bad);
     vtk_tile_owners(a.tt_offsets, R, a.max_tokens, base, T, tile_req);
     __syncthreads();
     int r = t < T ? vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t) : -1;

@@ -376,6 +376,84 @@ def test_tables_beyond_the_context_capacities_are_clipped(planner):
     prob.close()
 
 
+def _misaligned_copy(t, offset_elems):
+    """A copy of tensor ``t`` whose data pointer is ``offset_elems`` elements behind an aligned allocation."""
+    torch = _torch()
+    buf = torch.empty(t.numel() + offset_elems, dtype=t.dtype, device=t.device)
+    view = buf[offset_elems:]
+    view.copy_(t)
+    return view
+
+
+@pytest.mark.parametrize("planner", ["whole", "partial"])
+def test_tables_that_are_not_16_byte_aligned(planner):
+    """The planners read four table entries per thread with 16-byte and 4-byte accesses when the caller's
+    arrays allow it; arrays that start at an odd element take the scalar path and give the same result."""
+    from paper_2608_13263_b200.device import DeviceProblem
+    w = wl.mistral7b_random(seed=23, requests=7, lo=50, hi=1400, layers=1, heads=1, head_dim=64)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    prob.tt_slots = _misaligned_copy(prob.tt_slots, 1)
+    prob.keep = _misaligned_copy(prob.keep, 3)
+    prob.new_tt_slots = _misaligned_copy(prob.new_tt_slots, 1)
+    assert prob.tt_slots.data_ptr() % 16 != 0 and prob.keep.data_ptr() % 4 != 0 and prob.new_tt_slots.data_ptr() % 16 != 0
+    if planner == "whole":
+        prob.plan()
+    else:
+        prob.plan_partial(util=(1, 1))
+    prob.repack()
+    out = prob.outputs()
+    if planner == "whole":
+        p = vto.plan_workload(w)
+    else:
+        p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                             w.free_blocks, w.select, w.thr_num, w.thr_den, util=(1, 1))
+    assert_tables_equal(out, p, w)
+    assert (prob.new_tt_slots[w.num_tokens:].cpu().numpy() == -9).all()
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()
+
+
+@pytest.mark.parametrize("planner", ["whole", "partial"])
+def test_token_table_that_does_not_start_at_entry_zero(planner):
+    """tt_offsets[0] > 0: the entries in front of the first request belong to nobody; they are neither
+    counted nor written, and every request is planned as if the table started at its first entry."""
+    from paper_2608_13263_b200.device import DeviceProblem
+    torch = _torch()
+    w = wl.mistral7b_random(seed=29, requests=6, lo=50, hi=900, layers=1, heads=1, head_dim=64)
+    gap = 1029                                           # more than one tile, not a multiple of four
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, capacity_slack=gap)
+    T = w.num_tokens
+    shifted_slots = torch.zeros(T + gap, dtype=torch.int32, device=prob.device)     # slot 0 "live" in the gap
+    shifted_slots[gap:] = prob.tt_slots[:T]
+    shifted_keep = torch.ones(T + gap, dtype=torch.uint8, device=prob.device)
+    shifted_keep[gap:] = prob.keep[:T]
+    prob.tt_slots, prob.keep = shifted_slots, shifted_keep
+    prob.tt_offsets = (prob.tt_offsets + gap).to(torch.int32)
+    if planner == "whole":
+        prob.plan()
+        p = vto.plan_workload(w)
+    else:
+        prob.plan_partial(util=(1, 1))
+        p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                             w.free_blocks, w.select, w.thr_num, w.thr_den, util=(1, 1))
+    prob.repack()
+    torch.cuda.synchronize()
+    counts = prob.read_counts()
+    assert counts["error_flags"] == 0 and counts["num_moves"] == p.num_moves
+    assert np.array_equal(prob.req_status[:w.num_requests].cpu().numpy(), p.req_status)
+    assert np.array_equal(prob.new_tt_slots[gap:gap + T].cpu().numpy(), p.new_tt_slots)
+    assert (prob.new_tt_slots[:gap].cpu().numpy() == -9).all()          # untouched
+    assert np.array_equal(prob.new_bt_blocks[:len(p.new_bt_blocks)].cpu().numpy(), p.new_bt_blocks)
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    prob.close()
+
+
 def test_argument_errors():
     from paper_2608_13263_b200.device import DeviceProblem
     w = wl.tiny()

@@ -250,8 +250,12 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
     const unsigned total_items = (unsigned)per_slab * (unsigned)num_slabs;   // < 2^31, checked on the host
     // DYNAMIC: a ticket stands for `chunk` consecutive items (one atomic per chunk keeps the counter
     // far from the throughput of same-address atomics); lane 0 holds the ticket of the NEXT chunk
-    unsigned ticket = 0xffffffffu, chunk_base = 0, chunk_pos = (unsigned)chunk;
-    auto take_ticket = [&]() { if (lane == 0) ticket = atomicAdd(&a.ticket[0], 1u); };
+    // A warp's first chunk is the one with its own index in the grid, without an atomic: 1184 warps asking
+    // one address for a ticket at the same instant are served one after the other (about 3 us until the
+    // last one has its answer), and nothing can start before.  The counter hands out the chunks behind
+    // those (its value + number of warps); those requests are made a chunk ahead, off the critical path.
+    unsigned ticket = (unsigned)gw, chunk_base = 0, chunk_pos = (unsigned)chunk;
+    auto take_ticket = [&]() { if (lane == 0) ticket = atomicAdd(&a.ticket[0], 1u) + (unsigned)gstride; };
     auto fetch = [&](Entry &e) {           // reads the next item of this warp, moves on
         e.dst0 = -1;
         e.src = -1;
@@ -296,7 +300,6 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
             }
         }
     };
-    if (DYNAMIC) take_ticket();
     fetch(e1);
     if (ahead == 2) fetch(e2);
 

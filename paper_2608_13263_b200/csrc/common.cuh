@@ -197,6 +197,36 @@ __device__ __forceinline__ bool vtk_range(const int32_t *off, int r, int64_t cap
     return lo != a || hi != b;
 }
 
+// Inclusive scan over the values of a CTA of 1024 threads in thread order; `shfl` is the type's
+// shuffle-up, warp_tot shared T[32].  Three barriers; the result may be used at once.
+template <typename T, typename ShflUp>
+__device__ __forceinline__ T vtk_block_incl_scan(T v, T *warp_tot, T zero, ShflUp shfl)
+{
+    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T o = shfl(v, d);
+        if (lane >= d) v = o + v;
+    }
+    if (lane == 31) warp_tot[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        T w = warp_tot[lane];
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            T o = shfl(w, d);
+            if (lane >= d) w = o + w;
+        }
+        warp_tot[lane] = w;
+    }
+    __syncthreads();
+    T pre = warp == 0 ? zero : warp_tot[warp - 1];
+    T res = pre + v;
+    __syncthreads();
+    return res;
+}
+
+
 // ---------------------------------------------------------------------------------------
 // Flat tiling of the token table, shared by the planners: a tile is VTK_TILE consecutive table
 // entries whatever request they belong to, one CTA of VTK_TILE_NT threads, four entries per thread.

@@ -128,33 +128,6 @@ __device__ __forceinline__ Acc shfl_up(const Acc &v, int d)
                __shfl_up_sync(0xffffffffu, v.admitted, d), __shfl_up_sync(0xffffffffu, v.deferred, d)};
 }
 
-template <typename T, typename ShflUp>
-__device__ __forceinline__ T block_incl_scan(T v, T *warp_tot, T zero, ShflUp shfl)
-{
-    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        T o = shfl(v, d);
-        if (lane >= d) v = o + v;
-    }
-    if (lane == 31) warp_tot[warp] = v;
-    __syncthreads();
-    if (warp == 0) {
-        T w = warp_tot[lane];           // SCAN_NT / 32 == 32 warps
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            T o = shfl(w, d);
-            if (lane >= d) w = o + w;
-        }
-        warp_tot[lane] = w;
-    }
-    __syncthreads();
-    T pre = warp == 0 ? zero : warp_tot[warp - 1];
-    T res = pre + v;
-    __syncthreads();
-    return res;
-}
-
 __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 {
     __shared__ long long warp_ll[32];
@@ -194,7 +167,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
         const int raw = i < tiles ? a.tile_n[i] : 0;
         if (raw < 0) flags |= VTOKEN_FLAG_BAD_SLOT;
         const int v = raw & 0x7fffffff;
-        const int incl = block_incl_scan<int>(v, warp_i, 0, shfl_int) + carry_live;
+        const int incl = vtk_block_incl_scan<int>(v, warp_i, 0, shfl_int) + carry_live;
         if (i <= tiles) a.tile_n[i] = incl - v;
         __syncthreads();
         if (tid == SCAN_NT - 1) carry_live = incl;
@@ -229,13 +202,13 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
                   (unsigned long long)a.thr_num * (unsigned long long)nb * (unsigned long long)a.S;
         const bool cand = sel && need < nb;                          // strictly fewer blocks afterwards
         // admission: cumulative demand of candidates so far (this one included) fits the free list
-        const long long cum = block_incl_scan<long long>(cand ? need : 0, warp_ll, 0LL, shfl_ll) + carry_need;
+        const long long cum = vtk_block_incl_scan<long long>(cand ? need : 0, warp_ll, 0LL, shfl_ll) + carry_need;
         const bool adm = cand && cum <= (long long)nf;
         const int status = !sel ? VTOKEN_NOT_SELECTED
                                 : (!cand ? VTOKEN_NO_GAIN : (adm ? VTOKEN_REPACKED : VTOKEN_DEFERRED_NO_FREE));
         Acc mine{adm ? need : 0, adm ? nb : 0, valid ? (adm ? need : nb) : 0, adm ? n : 0, adm ? 1 : 0,
                  (cand && !adm) ? 1 : 0};
-        const Acc incl = block_incl_scan<Acc>(mine, warp_acc, Acc{0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
+        const Acc incl = vtk_block_incl_scan<Acc>(mine, warp_acc, Acc{0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
         if (valid) {
             a.req_dst_base[r] = incl.dst - mine.dst;
             a.req_freed_base[r] = incl.freed - mine.freed;

@@ -266,33 +266,6 @@ __device__ __forceinline__ PAcc pp_shfl_up(const PAcc &v, int d)
                 __shfl_up_sync(0xffffffffu, v.admitted, d), __shfl_up_sync(0xffffffffu, v.deferred, d),
                 __shfl_up_sync(0xffffffffu, v.released, d)};
 }
-template <typename T, typename ShflUp>
-__device__ __forceinline__ T pp_block_incl_scan(T v, T *warp_tot, T zero, ShflUp shfl)
-{
-    const int lane = vtk_lane(), warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        T o = shfl(v, d);
-        if (lane >= d) v = o + v;
-    }
-    if (lane == 31) warp_tot[warp] = v;
-    __syncthreads();
-    if (warp == 0) {
-        T w = warp_tot[lane];
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            T o = shfl(w, d);
-            if (lane >= d) w = o + w;
-        }
-        warp_tot[lane] = w;
-    }
-    __syncthreads();
-    T pre = warp == 0 ? zero : warp_tot[warp - 1];
-    T res = pre + v;
-    __syncthreads();
-    return res;
-}
-
 __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
 {
     vtk_release_successor();
@@ -325,14 +298,13 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     // it; one entry past the last tile holds the total)
     const int64_t T = pp_offset(a, R);
     const int tiles = (int)((T + TILE - 1) / TILE);
-    auto shfl_ll2 = [](long long v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
     for (int base = 0; base <= tiles; base += PP_SCAN_NT) {
         const int i = base + tid;
         const int raw = i < tiles ? a.tile_live[i] : 0;
         if (raw < 0) flags |= VTOKEN_FLAG_BAD_SLOT;
         const long long v = ((long long)(raw & 0x7fffffff) << 32) | (unsigned)(i < tiles ? a.tile_mov[i] : 0);
         // both counts in one 64-bit scan: live in the high half, moving in the low half (each < 2^31)
-        const long long incl = pp_block_incl_scan<long long>(v, warp_ll, 0LL, shfl_ll2) +
+        const long long incl = vtk_block_incl_scan<long long>(v, warp_ll, 0LL, shfl_ll) +
                                (((long long)carry_live << 32) | (unsigned)carry_mov);
         if (i <= tiles) {
             a.tile_live[i] = (int)((incl - v) >> 32);
@@ -371,9 +343,9 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
         my_live += n;
         my_blocks += hi - lo;
     }
-    const long long live_incl = pp_block_incl_scan<long long>(my_live, warp_ll, 0LL, shfl_ll);
+    const long long live_incl = vtk_block_incl_scan<long long>(my_live, warp_ll, 0LL, shfl_ll);
     if (tid == PP_SCAN_NT - 1) tot_live = live_incl;
-    const long long blocks_incl = pp_block_incl_scan<long long>(my_blocks, warp_ll, 0LL, shfl_ll);
+    const long long blocks_incl = vtk_block_incl_scan<long long>(my_blocks, warp_ll, 0LL, shfl_ll);
     if (tid == PP_SCAN_NT - 1) tot_blocks = blocks_incl;
     __syncthreads();
     bool triggered = true;                      // F > theta  <=>  (N*S - live) * den > num * N*S
@@ -403,13 +375,13 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
             sel = (unsigned long long)n * a.thr_den <
                   (unsigned long long)a.thr_num * (unsigned long long)nb * (unsigned long long)a.S;
         const bool cand = sel && need < ns;                        // sources release more than they consume
-        const long long cum = pp_block_incl_scan<long long>(cand ? need : 0, warp_ll, 0LL, shfl_ll) + carry_need;
+        const long long cum = vtk_block_incl_scan<long long>(cand ? need : 0, warp_ll, 0LL, shfl_ll) + carry_need;
         const bool adm = cand && cum <= (long long)nf;
         const int status = !sel ? VTOKEN_NOT_SELECTED
                                 : (!cand ? VTOKEN_NO_GAIN : (adm ? VTOKEN_REPACKED : VTOKEN_DEFERRED_NO_FREE));
         PAcc mine{adm ? need : 0, adm ? ns - nrel : 0, valid ? (adm ? nb - ns + need : nb) : 0, adm ? nsrc : 0,
                   adm ? 1 : 0, (cand && !adm) ? 1 : 0, adm ? nrel : 0};
-        const PAcc incl = pp_block_incl_scan<PAcc>(mine, warp_acc, PAcc{0, 0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
+        const PAcc incl = vtk_block_incl_scan<PAcc>(mine, warp_acc, PAcc{0, 0, 0, 0, 0, 0, 0}, shfl_acc) + carry;
         if (valid) {
             a.req_dst_base[r] = incl.dst - mine.dst;
             a.req_freed_base[r] = incl.freed - mine.freed;

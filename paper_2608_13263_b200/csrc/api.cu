@@ -27,9 +27,9 @@ void free_all(vtoken_ctx *ctx)
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
-                    ctx->stage.num_requests, ctx->stage.bt_offsets, ctx->stage.bt_blocks,
-                    ctx->stage.tt_offsets, ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
-                    ctx->stage.select, ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
+                    ctx->stage.num_requests, ctx->stage.bt_blocks,
+                    ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
+                    ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
                     ctx->stage.new_tt_slots, ctx->stage.freed_blocks, ctx->stage.req_status, ctx->stage.counts,
                     ctx->stage.protect};
     for (void *p : ptrs)
@@ -47,15 +47,22 @@ int ensure_stage(vtoken_ctx *ctx)
     const vtoken_config &c = ctx->cfg;
     int rc = VTOKEN_OK;
     auto A = [&](auto **p, int64_t n) { if (rc == VTOKEN_OK) rc = dev_alloc(ctx, p, n); };
-    A(&ctx->stage.num_requests, 2);                 // the two scalars travel in one copy
-    if (rc == VTOKEN_OK) ctx->stage.num_free = ctx->stage.num_requests + 1;
-    A(&ctx->stage.bt_offsets, (int64_t)c.max_requests + 1);
+    // The small inputs -- the two scalars, both offset arrays, the selection bytes -- share one device
+    // allocation and one pinned host mirror, so that they travel in a single copy: every copy call costs
+    // the submitting thread a few microseconds whatever its size, and the GPU waits for the last of them.
+    const int64_t rc1 = (int64_t)c.max_requests + 1;
+    ctx->stage.small_ints = 2 + 2 * rc1 + (c.max_requests + 3) / 4;
+    A(&ctx->stage.num_requests, ctx->stage.small_ints);
+    if (rc == VTOKEN_OK) {
+        ctx->stage.num_free = ctx->stage.num_requests + 1;
+        ctx->stage.bt_offsets = ctx->stage.num_requests + 2;
+        ctx->stage.tt_offsets = ctx->stage.bt_offsets + rc1;
+        ctx->stage.select = reinterpret_cast<uint8_t *>(ctx->stage.tt_offsets + rc1);
+    }
     A(&ctx->stage.bt_blocks, c.max_table_blocks);
-    A(&ctx->stage.tt_offsets, (int64_t)c.max_requests + 1);
     A(&ctx->stage.tt_slots, c.max_tokens);
     A(&ctx->stage.free_blocks, c.max_free_blocks);
     A(&ctx->stage.keep, c.max_tokens);
-    A(&ctx->stage.select, c.max_requests);
     A(&ctx->stage.new_bt_offsets, (int64_t)c.max_requests + 1);
     A(&ctx->stage.new_bt_blocks, c.max_table_blocks);
     A(&ctx->stage.new_tt_slots, c.max_tokens);
@@ -63,7 +70,7 @@ int ensure_stage(vtoken_ctx *ctx)
     A(&ctx->stage.req_status, c.max_requests);
     A(&ctx->stage.counts, 1);
     if (rc == VTOKEN_OK) {
-        if (cudaMallocHost((void **)&ctx->stage.h_scalars, 2 * sizeof(int32_t)) != cudaSuccess ||
+        if (cudaMallocHost((void **)&ctx->stage.h_scalars, (size_t)ctx->stage.small_ints * sizeof(int32_t)) != cudaSuccess ||
             cudaMallocHost((void **)&ctx->stage.h_counts, sizeof(vtoken_counts)) != cudaSuccess ||
             cudaStreamCreateWithFlags(&ctx->stage.aux, cudaStreamNonBlocking) != cudaSuccess ||
             cudaEventCreateWithFlags(&ctx->stage.planned, cudaEventDisableTiming) != cudaSuccess ||
@@ -235,15 +242,21 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
     }
 #define H2D(dst, src, n) VTK_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(n), cudaMemcpyHostToDevice, st))
 #define D2H(dst, src, n) VTK_CUDA(ctx, cudaMemcpyAsync(dst, src, (size_t)(n), cudaMemcpyDeviceToHost, st))
-    s.h_scalars[0] = h->num_requests;               // pinned: the copy below is truly asynchronous
-    s.h_scalars[1] = h->num_free;
-    H2D(s.num_requests, s.h_scalars, 2 * sizeof(int32_t));
-    H2D(s.bt_offsets, h->bt_offsets, (R + 1) * sizeof(int32_t));
-    if (NBT) H2D(s.bt_blocks, h->bt_blocks, NBT * sizeof(int32_t));
-    H2D(s.tt_offsets, h->tt_offsets, (R + 1) * sizeof(int32_t));
+    // the token table first: its transfer runs while this thread submits the rest
     if (T) H2D(s.tt_slots, h->tt_slots, T * sizeof(int32_t));
     if (T) H2D(s.keep, h->keep, T);
-    if (h->select && R) H2D(s.select, h->select, R);
+    {
+        // scalars, offsets and selection bytes through the pinned mirror, in one copy
+        const int64_t rc1 = (int64_t)ctx->cfg.max_requests + 1;
+        int32_t *m = s.h_scalars;
+        m[0] = h->num_requests;
+        m[1] = h->num_free;
+        memcpy(m + 2, h->bt_offsets, (size_t)(R + 1) * sizeof(int32_t));
+        memcpy(m + 2 + rc1, h->tt_offsets, (size_t)(R + 1) * sizeof(int32_t));
+        if (h->select && R) memcpy(m + 2 + 2 * rc1, h->select, (size_t)R);
+        H2D(s.num_requests, m, s.small_ints * sizeof(int32_t));
+    }
+    if (NBT) H2D(s.bt_blocks, h->bt_blocks, NBT * sizeof(int32_t));
     if (h->num_free) H2D(s.free_blocks, h->free_blocks, h->num_free * sizeof(int32_t));
     if (opts && opts->protect) H2D(s.protect, opts->protect, ctx->cfg.num_blocks);
 

@@ -64,7 +64,9 @@ struct vtoken_ctx {
         uint8_t *protect;              // [num_blocks], vtoken_repack_host_partial only (allocated on first use)
         int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *req_status;
         vtoken_counts *counts;
-        int32_t *h_scalars;            // HOST, pinned: {num_requests, num_free} of the call in flight
+        int32_t *h_scalars;            // HOST, pinned mirror of the small inputs of the call in flight: {num_requests,
+                                       // num_free}, bt_offsets, tt_offsets, select (same layout as on the device)
+        int64_t small_ints;            // its size in 32-bit words
         vtoken_counts *h_counts;       // HOST, pinned: landing place of the counts
         cudaStream_t aux;              // carries the output copies while the copy kernel runs
         cudaEvent_t planned, copied;   // plan done on the caller's stream; outputs copied on aux

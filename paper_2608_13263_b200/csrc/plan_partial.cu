@@ -84,7 +84,7 @@ __device__ __forceinline__ int pp_block_sum(int n, int *warp_n)
     return s;   // valid in thread 0
 }
 
-// ---- live: part counts and per-block liveness -----------------------------------------------
+// ---- tiles: live / moving tokens per tile and in front of request boundaries, per-block liveness ----
 // does a live token of request r in block b move?  (b is a source of its request, or r leaves its
 // protected blocks and b is one of them)
 __device__ __forceinline__ bool pp_moves(const PArgs &a, bool detach, int32_t b)

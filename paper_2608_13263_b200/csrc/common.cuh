@@ -246,7 +246,8 @@ __device__ __forceinline__ int64_t vtk_clipped_offset(const int32_t *off, int r,
 
 // The thread's four entries [t, t + 4) of the token table below T: slots, and one bit per live entry.
 // Entries in front of `first` (the first request's first entry) belong to no request and count as dead.
-// vec: tt_slots is 16-byte and keep 4-byte aligned (t is a multiple of four).
+// vec: tt_slots is 16-byte and keep 4-byte aligned (t is a multiple of four).  keep == nullptr: every entry
+// with a slot counts as kept.
 __device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, const uint8_t *keep, int vec, int64_t t,
                                                      int64_t first, int64_t T, int64_t slots_per_layer,
                                                      int32_t (&slot)[VTK_TILE_TOK], bool &bad)
@@ -256,13 +257,13 @@ __device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, co
     for (int k = 0; k < VTK_TILE_TOK; ++k) slot[k] = -1;
     if (vec && t + VTK_TILE_TOK <= T) {
         const int4 s4 = *reinterpret_cast<const int4 *>(tt_slots + t);
-        const uchar4 k4 = *reinterpret_cast<const uchar4 *>(keep + t);
+        const uchar4 k4 = keep ? *reinterpret_cast<const uchar4 *>(keep + t) : make_uchar4(1, 1, 1, 1);
         slot[0] = s4.x; slot[1] = s4.y; slot[2] = s4.z; slot[3] = s4.w;
         kp[0] = k4.x; kp[1] = k4.y; kp[2] = k4.z; kp[3] = k4.w;
     } else {
 #pragma unroll
         for (int k = 0; k < VTK_TILE_TOK; ++k)
-            if (t + k < T) { slot[k] = tt_slots[t + k]; kp[k] = keep[t + k]; }
+            if (t + k < T) { slot[k] = tt_slots[t + k]; kp[k] = keep ? keep[t + k] : 1; }
     }
     unsigned bits = 0;
 #pragma unroll

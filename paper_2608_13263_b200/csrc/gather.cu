@@ -2,8 +2,10 @@
 // K and V rows of the active tokens of the selected requests, request order then token-id
 // order, written densely.  Same structure as the planner: count -> scan -> assign, then a
 // row-copy kernel that reads through the token table (the slot-translation read pattern of
-// Sec. 3.4).  Like the planner, every request is cut into VTK_PLAN_PARTS equal token ranges with
-// one CTA each in count and assign, so that long requests do not serialise on one CTA.
+// Sec. 3.4).  Two versions of the index kernels: a flat tiling of the token table like the planner's
+// (contexts made by vtoken_create), and one that walks the table request by request, every request cut
+// into 1 .. VTK_PLAN_PARTS equal token ranges with one CTA each (the context-free entry point, which
+// has no capacity for the table's length).
 #include "common.cuh"
 
 namespace {
@@ -23,6 +25,11 @@ struct GatherArgs {
     int64_t layer_stride, row_bytes, slots_per_layer, out_capacity, max_tokens;
     int32_t layer_begin, layer_end, max_requests;
     int32_t parts;               // token ranges (CTAs) per request, <= G_PARTS (the stride of part_n)
+    // flat tiling (contexts made by vtoken_create; see plan.cu): live tokens per tile, then before every tile;
+    // live tokens between the start of a request boundary's tile and the boundary; live tokens before a request
+    int32_t *tile_n, *req_part, *req_before;
+    int32_t num_tiles, vec_in;
+    int64_t table_cap;           // capacity of the token table: offsets are clipped to it
 };
 
 __device__ __forceinline__ int g_requests(const GatherArgs &a)
@@ -146,6 +153,188 @@ __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
             if (a.g_req != nullptr) a.g_req[i] = r;
         }
     }
+}
+
+// ---- the same index over a flat tiling of the token table ------------------------------------------
+// Tiles of 1024 consecutive table entries whatever request they belong to; per-request numbers are
+// differences of running live counts (see plan.cu).  Used when the context has the tile scratch, which
+// needs a capacity for the table's length; the context-free entry point keeps the kernels above.
+__device__ __forceinline__ int64_t g_offset(const GatherArgs &a, int r)
+{
+    return vtk_clipped_offset(a.tt_offsets, r, a.table_cap);
+}
+
+__global__ void __launch_bounds__(VTK_TILE_NT) gather_tiles_kernel(GatherArgs a)
+{
+    __shared__ int warp_n[VTK_TILE_NT / 32];
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
+    const int R = g_requests(a);
+    const int64_t T = g_offset(a, R);
+    // a whole tile, or (CTAs behind the tiles, one per request boundary) the entries between the start of
+    // the boundary's tile and the boundary
+    const bool is_tile = (int)blockIdx.x < a.num_tiles;
+    const int rb = (int)blockIdx.x - a.num_tiles;
+    int64_t base, limit;
+    if (is_tile) {
+        base = (int64_t)blockIdx.x * VTK_TILE;
+        limit = T;
+        if (base >= T) return;
+    } else {
+        if (rb > R) return;
+        limit = g_offset(a, rb);
+        base = limit / VTK_TILE * VTK_TILE;
+        if (base == limit) return;
+    }
+    bool bad = false;
+    int32_t slot[VTK_TILE_TOK];
+    int n = __popc(vtk_load_entries(a.tt_slots, a.keep, a.vec_in, base + threadIdx.x * VTK_TILE_TOK, g_offset(a, 0),
+                                    limit, a.slots_per_layer, slot, bad));
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
+    if (vtk_lane() == 0) warp_n[threadIdx.x >> 5] = n;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int s = 0;
+#pragma unroll
+        for (int w = 0; w < VTK_TILE_NT / 32; ++w) s += warp_n[w];
+        (is_tile ? a.tile_n[blockIdx.x] : a.req_part[rb]) = s;
+    }
+}
+
+__global__ void __launch_bounds__(1024) gather_scan_flat_kernel(GatherArgs a)
+{
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
+    __shared__ int warp_tot[32];
+    __shared__ int carry;
+    const int R = g_requests(a);
+    const int tid = threadIdx.x;
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    auto shfl_int = [](int v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
+    // live tokens before every tile, in place; one entry past the last tile holds the total
+    const int64_t T = g_offset(a, R);
+    const int tiles = (int)((T + VTK_TILE - 1) / VTK_TILE);
+    for (int base = 0; base <= tiles; base += 1024) {
+        const int i = base + tid;
+        const int v = i < tiles ? a.tile_n[i] : 0;
+        const int incl = vtk_block_incl_scan<int>(v, warp_tot, 0, shfl_int) + carry;
+        if (i <= tiles) a.tile_n[i] = incl - v;
+        __syncthreads();
+        if (tid == 1023) carry = incl;
+        __syncthreads();
+    }
+    auto live_before = [&](int r) {
+        const int64_t o = g_offset(a, r);
+        return a.tile_n[o / VTK_TILE] + (o % VTK_TILE != 0 ? a.req_part[r] : 0);
+    };
+    // live tokens of the selected requests -> first output row of every request
+    if (tid == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < R; base += 1024) {
+        const int r = base + tid;
+        int v = 0;
+        if (r < R) {
+            const int before = live_before(r);
+            a.req_before[r] = before;
+            if (a.select == nullptr || a.select[r] != 0) v = live_before(r + 1) - before;
+            if (v < 0) v = 0;                                // offsets that run backwards
+        }
+        const int incl = vtk_block_incl_scan<int>(v, warp_tot, 0, shfl_int) + carry;
+        if (r < R) a.out_offsets[r] = incl - v;
+        __syncthreads();
+        if (tid == 1023) carry = incl;
+        __syncthreads();
+    }
+    if (tid == 0) {
+        a.out_offsets[R] = carry;
+        int64_t cap = a.out_capacity < a.max_tokens ? a.out_capacity : a.max_tokens;
+        if ((int64_t)carry > cap) {
+            atomicOr(&a.counts->error_flags, VTOKEN_FLAG_GATHER_OVERFLOW);
+            *a.g_total = (int32_t)cap;
+        } else {
+            *a.g_total = carry;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(VTK_TILE_NT) gather_assign_flat_kernel(GatherArgs a)
+{
+    __shared__ int warp_sums[VTK_TILE_NT / 32];
+    __shared__ int tile_req[2];
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
+    const int R = g_requests(a);
+    const int64_t T = g_offset(a, R);
+    const int64_t base = (int64_t)blockIdx.x * VTK_TILE;
+    if (base >= T) return;
+    const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
+    const int64_t t = base + tid * VTK_TILE_TOK;
+    int32_t slot[VTK_TILE_TOK];
+    bool bad_any = false;
+    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, g_offset(a, 0), T, a.slots_per_layer, slot,
+                                           bad_any);
+    const int cnt = __popc(bits);
+    const int incl = vtk_warp_incl_scan(cnt);
+    if (lane == 31) warp_sums[warp] = incl;
+    vtk_tile_owners(a.tt_offsets, R, a.table_cap, base, T, tile_req);
+    __syncthreads();
+    int before = a.tile_n[blockIdx.x] + incl - cnt;          // live tokens of the table before entry t
+    for (int w = 0; w < warp; ++w) before += warp_sums[w];
+    if (t >= T) return;
+    int r = vtk_entry_owner(a.tt_offsets, a.table_cap, tile_req, t);
+    int64_t next = g_offset(a, r + 1), t0 = r >= 0 ? g_offset(a, r) : 0;
+    int first_row = 0;
+    bool sel = false;
+    auto load_request = [&]() {
+        sel = a.select == nullptr || a.select[r] != 0;
+        first_row = a.out_offsets[r] - a.req_before[r];      // output row of a token = this + its running count
+        t0 = g_offset(a, r);
+    };
+    if (r >= 0) load_request();
+    const int64_t cap = *a.g_total;
+    bool bad = false;
+#pragma unroll
+    for (int k = 0; k < VTK_TILE_TOK; ++k) {
+        if (t + k >= T) break;
+        if (t + k >= next && r + 1 < R) {                     // a request boundary inside the thread's entries
+            while (r + 1 < R && g_offset(a, r + 1) <= t + k) ++r;
+            next = g_offset(a, r + 1);
+            load_request();
+        }
+        if (r < 0 || !sel) continue;
+        if (slot[k] >= 0 && (int64_t)slot[k] >= a.slots_per_layer) bad = true;     // reported for selected requests only
+        if (!((bits >> k) & 1u)) continue;
+        const int64_t i = (int64_t)first_row + before + __popc(bits & ((1u << k) - 1u));
+        if (i < 0 || i >= cap) continue;
+        a.g_src[i] = slot[k];
+        if (a.g_ids != nullptr) a.g_ids[i] = (int32_t)(t + k - t0);
+        if (a.g_req != nullptr) a.g_req[i] = r;
+    }
+    if (bad) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
+}
+
+// count -> scan -> assign: flat tiles when the context has their scratch, else the per-request kernels
+int launch_index(vtoken_ctx *ctx, GatherArgs &a, cudaStream_t st)
+{
+    if (ctx->tile_n != nullptr) {
+        a.tile_n = ctx->tile_n;
+        a.req_part = ctx->req_part;
+        a.req_before = ctx->req_before;
+        a.num_tiles = (int32_t)((ctx->cfg.max_tokens + VTK_TILE - 1) / VTK_TILE);
+        a.vec_in = ((uintptr_t)a.tt_slots % 16 == 0 && (a.keep == nullptr || (uintptr_t)a.keep % 4 == 0)) ? 1 : 0;
+        a.table_cap = ctx->cfg.max_tokens;
+        VTK_CUDA(ctx, vtk_launch_dependent(gather_tiles_kernel, dim3(a.num_tiles + ctx->cfg.max_requests + 1),
+                                           dim3(VTK_TILE_NT), 0, st, a));
+        VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_flat_kernel, dim3(1), dim3(1024), 0, st, a));
+        VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_flat_kernel, dim3(a.num_tiles), dim3(VTK_TILE_NT), 0, st, a));
+        return VTOKEN_OK;
+    }
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel, dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel, dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    return VTOKEN_OK;
 }
 
 __device__ __forceinline__ uint4 ld_stream(const uint4 *p)
@@ -377,11 +566,7 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     a.max_requests = ctx->cfg.max_requests;
     a.parts = ctx->parts;
     VTK_CUDA(ctx, cudaMemsetAsync(out_digest, 0, sizeof(uint64_t) * (size_t)ctx->cfg.max_requests, st));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
-                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
-                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
     VTK_CUDA(ctx, vtk_launch_dependent(gather_digest_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
@@ -420,11 +605,7 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
     a.parts = ctx->parts;
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
-                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
-                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
     // the rows go through the bulk-copy rings when the context has them (vtoken_create does; the
     // context-free entry point does not), else through the register kernel
     const bool aligned = (((uintptr_t)out_k | (uintptr_t)out_v) & 15) == 0;
@@ -470,11 +651,7 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.layer_begin = a.layer_end = 0;
     a.max_requests = ctx->cfg.max_requests;
     a.parts = ctx->parts;
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel,
-                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel,
-                                       dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

@@ -54,9 +54,6 @@
  *   VTOKEN_COPY_DYNAMIC  0: every warp of the copy kernel gets a fixed share of the work items; 1 (default):
  *                        warps take items from a ticket counter, VTOKEN_COPY_CHUNK (default 4) at a time
  *   VTOKEN_WAIT_LIMIT_MS bound of in-kernel waits (1 .. 60000, default 2000)
- *   VTOKEN_PLAN_PARTS    1 .. 8: token ranges (CTAs) per request in the kernels that walk the token table request
- *                        by request (logical gather, slot mapping, relocation digest); default: chosen from
- *                        max_requests and max_tokens
  *   VTOKEN_TEST_STALL_ITEM  test hook: index of one work item whose barrier is armed with bytes that never
  *                        arrive, so that its wait runs out (exercises the time-out path; never set in production)
  * and one read at every launch:

@@ -23,7 +23,7 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 
 void free_all(vtoken_ctx *ctx)
 {
-    void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->part_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
+    void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
@@ -119,8 +119,6 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     if (cap > cfg->max_free_blocks) cap = cfg->max_free_blocks;
     if (cap < 1) cap = 1;
     ctx->cap_dst_blocks = (int32_t)cap;
-    ctx->parts = vtk_choose_parts(cfg->max_requests, cfg->max_tokens);
-    if (const char *e = getenv("VTOKEN_PLAN_PARTS")) { int v = atoi(e); if (v >= 1 && v <= VTK_PLAN_PARTS) ctx->parts = v; }
 
     cudaError_t e = cudaGetDevice(&ctx->device);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&ctx->num_sms, cudaDevAttrMultiProcessorCount, ctx->device);
@@ -129,7 +127,6 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     int rc = VTOKEN_OK;
     auto A = [&](auto **p, int64_t n) { if (rc == VTOKEN_OK) rc = dev_alloc(ctx, p, n); };
     A(&ctx->req_n, cfg->max_requests);
-    A(&ctx->part_n, (int64_t)cfg->max_requests * VTK_PLAN_PARTS);
     A(&ctx->req_dst_base, cfg->max_requests);
     A(&ctx->tile_n, (cfg->max_tokens + 1023) / 1024 + 1);
     A(&ctx->req_part, (int64_t)cfg->max_requests + 1);

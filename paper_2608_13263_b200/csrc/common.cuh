@@ -22,14 +22,14 @@ struct vtoken_ctx {
 
     // planner scratch (DEVICE)
     int32_t *req_n;            // [max_requests] live tokens
-    int32_t *part_n;           // [max_requests * VTK_PLAN_PARTS] live tokens per request part
+    int32_t *part_n;           // [max_requests * VTK_PLAN_PARTS] live tokens per request part: only the context-free
+                               // gather entry point (per-request index kernels) sets it, from its static scratch
     int32_t *req_dst_base;     // [max_requests] first destination block (index into the free list)
     int32_t *req_freed_base;   // [max_requests] first entry in freed_blocks
     int32_t *req_status;       // [max_requests]
     int32_t *dst_src;          // [cap_dst_blocks * S] inverse plan: source slot of each destination slot, -1 = none
     int32_t *dst_blocks;       // [cap_dst_blocks] physical id of each destination block, -1 = skip
     vtoken_counts *counts;     // one struct
-    int parts;                 // token ranges (CTAs) per request in the per-request kernels, 1 .. VTK_PLAN_PARTS
     int32_t *tile_n;           // [ceil(max_tokens / 1024) + 1] live tokens per tile of the token table, then scanned
     int32_t *req_part;         // [max_requests + 1] live tokens between a request's tile start and its first entry
     int32_t *req_before;       // [max_requests + 1] live (partial planner: moving) tokens of the table before the request's first entry
@@ -82,21 +82,6 @@ struct vtoken_ctx {
     unsigned int *copy_ticket; // [2] DEVICE: next item, finished warps (zero between launches)
     int bulk_warps, bulk_stages, bulk_rows, bulk_depth, bulk_ahead;   // bulk path: warps per CTA, ring size, rows per item, loads ahead
 };
-
-// Token ranges per request for the kernels that give every request its own CTAs (logical gather,
-// slot mapping, digest): enough CTAs to fill the GPU about twice over, few enough that a CTA has more
-// than one pass to do -- 512 requests x 8 parts were 4096 CTAs of a single pass each, seven waves
-// of launch and load latency -- and never so few that a part exceeds about 4096 entries.
-inline int vtk_choose_parts(int64_t max_requests, int64_t max_tokens)
-{
-    int64_t parts = 1184 / (max_requests > 0 ? max_requests : 1);
-    const int64_t per_request = max_tokens / (max_requests > 0 ? max_requests : 1);
-    const int64_t by_length = (per_request + 4095) / 4096;
-    if (parts < by_length) parts = by_length;
-    if (parts < 1) parts = 1;
-    if (parts > VTK_PLAN_PARTS) parts = VTK_PLAN_PARTS;
-    return (int)parts;
-}
 
 // host launchers, one per translation unit
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);

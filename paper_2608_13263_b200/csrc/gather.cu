@@ -564,7 +564,7 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     a.layer_begin = layer_begin;
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
-    a.parts = ctx->parts;
+    a.parts = G_PARTS;
     VTK_CUDA(ctx, cudaMemsetAsync(out_digest, 0, sizeof(uint64_t) * (size_t)ctx->cfg.max_requests, st));
     { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
     VTK_CUDA(ctx, vtk_launch_dependent(gather_digest_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
@@ -604,7 +604,7 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.layer_begin = layer_begin;
     a.layer_end = layer_end;
     a.max_requests = ctx->cfg.max_requests;
-    a.parts = ctx->parts;
+    a.parts = G_PARTS;
     { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
     // the rows go through the bulk-copy rings when the context has them (vtoken_create does; the
     // context-free entry point does not), else through the register kernel
@@ -650,7 +650,7 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.max_tokens = out_capacity;
     a.layer_begin = a.layer_end = 0;
     a.max_requests = ctx->cfg.max_requests;
-    a.parts = ctx->parts;
+    a.parts = G_PARTS;
     { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;

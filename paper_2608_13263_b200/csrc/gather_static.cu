@@ -103,7 +103,6 @@ extern "C" int vtoken_gather_logical_noalloc(const void *k_pool, const void *v_p
     ctx.cfg.v_pool = const_cast<void *>(v_pool);
     ctx.cfg.max_requests = max_requests;
     ctx.cfg.max_tokens = NOALLOC_MAX_TOKENS;
-    ctx.parts = VTK_PLAN_PARTS;             // the table's length is not known here: the full split
     ctx.row_bytes = row_bytes;
     ctx.layer_stride = stride;
     ctx.slots_per_layer = slots;

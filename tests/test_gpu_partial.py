@@ -88,37 +88,6 @@ def test_partial_plans_small_whole_pool(w, opts):
     run_partial(w, opts)
 
 
-@pytest.mark.parametrize("parts", ["1", "2", "3", "8"])
-def test_token_ranges_per_request(parts, monkeypatch):
-    """The kernels that walk the token table request by request (logical gather, slot mapping) cut every
-    request into a number of token ranges chosen at create from the capacities; every count gives the same
-    result, and the planners and the block liveness (flat tiles) do not depend on it."""
-    import torch
-    from paper_2608_13263_b200.device import DeviceProblem
-    monkeypatch.setenv("VTOKEN_PLAN_PARTS", parts)
-    w = wl.mistral7b_random(seed=17, requests=9, lo=40, hi=1500, layers=1, heads=1, head_dim=64)
-    run_partial(w, dict(util=(1, 1), theta=(1, 4), max_source_blocks=7))
-    run_partial(w, dict(util=(3, 4), protect="prefix"))
-    prob = DeviceProblem(w, fill_seed=FILL_SEED)
-    live = int(((w.tt_slots >= 0) & (w.keep != 0)).sum())
-    out_k, out_v, out_off = prob.gather_logical(prob.tt_slots, prob.keep, 0, 1, live)
-    torch.cuda.synchronize()
-    k, _ = host_pools(w)
-    for r in range(w.num_requests):
-        t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
-        rows = vto.gather_logical(k[0], w.tt_slots[t0:t1], w.keep[t0:t1])
-        o0, o1 = int(out_off[r]), int(out_off[r + 1])
-        assert np.array_equal(out_k[0, o0:o1].cpu().numpy().view(np.uint16), rows)
-    n_b = torch.zeros(w.num_blocks, dtype=torch.int32, device=prob.device)
-    summary = torch.zeros(4, dtype=torch.int64, device=prob.device)
-    vt.vtoken_block_liveness(prob.ctx, num_requests=prob.num_requests, bt_offsets=prob.bt_offsets,
-                             bt_blocks=prob.bt_blocks, tt_offsets=prob.tt_offsets, tt_slots=prob.tt_slots,
-                             keep=prob.keep, n_b=n_b, summary=summary)
-    torch.cuda.synchronize()
-    assert int(summary[0]) == live and int(n_b.sum()) == live
-    prob.close()
-
-
 def test_partial_plan_moves_fewer_rows_for_the_same_block_count():
     w = wl.mistral7b_random(seed=3, requests=12, lo=200, hi=600, layers=1, rho_lo=0.8, rho_hi=0.98)
     out_p, p = run_partial(w, dict(util=(1, 1)))

@@ -27,7 +27,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-from paper_2608_13263_b200 import workloads as wl  # noqa: E402
+from harness import workloads as wl  # noqa: E402
 
 METRIC = "repack HBM GB/s (read+write); live tokens repacked/s and fraction of HBM peak in the same line"
 NOMINAL_HBM_GBS = 8000.0
@@ -146,7 +146,7 @@ def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1, use_gpu
     if use_gpu_fill:
         try:
             import torch
-            from paper_2608_13263_b200 import harness as vh
+            from harness import kernels as vh
             if torch.cuda.is_available():
                 k = np.empty(shape, np.uint16)
                 v = np.empty(shape, np.uint16)
@@ -231,8 +231,8 @@ def run_cuda(args):
     import torch
 
     from paper_2608_13263_b200 import binding as vt
-    from paper_2608_13263_b200.device import DeviceProblem, origin_map
-    from paper_2608_13263_b200.parallel import Ranks
+    from harness.device import DeviceProblem, origin_map
+    from harness.parallel import Ranks
 
     ranks = Ranks.from_env(args.gpus)
     torch.cuda.set_device(ranks.local_rank)
@@ -461,7 +461,7 @@ def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
     alone, then both at once.  The proxy's per-request checksums must not change (the repack
     never writes an allocated block)."""
     import torch
-    from paper_2608_13263_b200 import harness as vh
+    from harness import kernels as vh
     owner = np.repeat(np.arange(w.num_requests, dtype=np.int32), np.diff(w.bt_offsets))
     owner_d = torch.from_numpy(owner).to(dev)
     nbt = len(w.bt_blocks)
@@ -543,7 +543,7 @@ def run_waves(args, prob, w, side, dev, plans, one_shot_ms):
     plan + copy + commit in `--waves` waves, blocks reclaimed by one wave feeding the next, one
     captured graph.  Checked against the oracle's wave plan when the CPU-baseline leg ran."""
     import torch
-    from paper_2608_13263_b200.device import origin_map
+    from harness.device import origin_map
     W = args.waves
     prob.plan()                                            # the one-shot plan names every demand
     one = prob.outputs()
@@ -806,7 +806,7 @@ def run_plan_only(args):
     Prints one JSON line; parity of both planners is the tests' business, not this mode's."""
     import torch
     from paper_2608_13263_b200 import binding as vt
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(dev)
     w = build_workload(args.config, args.seed, args.scale_requests, args.block_size)

@@ -110,6 +110,20 @@ __global__ void __launch_bounds__(256) decode_read_kernel(const uint8_t *k_pool,
     }
 }
 
+// SMs of the current device (queried once per process and device; grids are multiples of it)
+int sm_count()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) n = 1;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
 }  // namespace
 
 extern "C" {
@@ -121,7 +135,7 @@ int vth_fill(void *dst, int kv, int num_layers, int layer_begin, int layer_end, 
 {
     if (!dst || row_elems % 8 != 0 || layer_begin < 0 || layer_end > num_layers || layer_begin >= layer_end) return -1;
     if (layer_stride_bytes == 0) layer_stride_bytes = slots_per_layer * row_elems * 2;
-    fill_kernel<<<148 * 16, 256, 0, (cudaStream_t)stream>>>((uint8_t *)dst, kv, num_layers, layer_begin, layer_end,
+    fill_kernel<<<sm_count() * 16, 256, 0, (cudaStream_t)stream>>>((uint8_t *)dst, kv, num_layers, layer_begin, layer_end,
                                                             slots_per_layer, row_elems, layer_stride_bytes, seed);
     return cudaGetLastError() == cudaSuccess ? 0 : -3;
 }
@@ -133,7 +147,7 @@ int vth_verify(const void *pool, int kv, int num_layers, int64_t slots_per_layer
 {
     if (!pool || !origin || !mismatches || row_elems % 8 != 0) return -1;
     if (layer_stride_bytes == 0) layer_stride_bytes = slots_per_layer * row_elems * 2;
-    verify_kernel<<<148 * 16, 256, 0, (cudaStream_t)stream>>>((const uint8_t *)pool, kv, num_layers, slots_per_layer,
+    verify_kernel<<<sm_count() * 16, 256, 0, (cudaStream_t)stream>>>((const uint8_t *)pool, kv, num_layers, slots_per_layer,
                                                               row_elems, layer_stride_bytes, seed, origin,
                                                               (unsigned long long *)mismatches);
     return cudaGetLastError() == cudaSuccess ? 0 : -3;
@@ -146,7 +160,7 @@ int vth_decode_read(const void *k_pool, const void *v_pool, const int32_t *bt_of
                     int64_t layer_stride_bytes, uint64_t *checksums, int ctas, void *stream)
 {
     if (!k_pool || !v_pool || !bt_blocks || !bt_owner || !checksums || block_bytes % 16 != 0) return -1;
-    if (ctas <= 0) ctas = 148 * 8;
+    if (ctas <= 0) ctas = sm_count() * 8;
     decode_read_kernel<<<ctas, 256, 0, (cudaStream_t)stream>>>((const uint8_t *)k_pool, (const uint8_t *)v_pool,
                                                                bt_offsets, bt_blocks, bt_owner, total_blocks, num_layers,
                                                                block_bytes, layer_stride_bytes,

@@ -10,8 +10,9 @@ from __future__ import annotations
 import numpy as np
 import torch
 
-from . import binding as vt
-from . import harness as vh
+from paper_2608_13263_b200 import binding as vt
+
+from . import kernels as vh
 from .workloads import Workload
 
 

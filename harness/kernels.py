@@ -5,7 +5,7 @@ from __future__ import annotations
 import ctypes
 import os
 
-from .binding import _ptr, _stream
+from paper_2608_13263_b200.binding import _ptr, _stream
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvtoken_harness.so")
@@ -17,10 +17,14 @@ _lib = None
 def load():
     global _lib
     if _lib is None:
-        from .binding import _build_if_needed
-        _build_if_needed()
+        from . import build as _build
+        try:
+            _build._nvcc()
+            _build.build()
+        except RuntimeError:
+            pass                    # no compiler here: use the library as shipped (or fail below)
         if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_13263_b200.build`")
+            raise ImportError(f"{LIB_PATH} is missing: run `python -m harness.build`")
         lib = ctypes.CDLL(LIB_PATH)
         lib.vth_fill.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                  ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p]

@@ -3,9 +3,8 @@ KV cache into dense blocks with rewritten block and token tables.
 
 The work is done by hand-written CUDA kernels (sm_100a) behind the C ABI declared in
 ``include/vtoken.h``; this package is the thin Python binding of that ABI (same function
-names, argument marshalling only) plus seeded workload generators and harness kernels used
-by tests and the benchmark.  There is no CPU fallback: using the binding without the built
-library raises ImportError.
+names, argument marshalling only).  There is no CPU fallback: using the binding without the
+built library raises ImportError.
 """
 from .binding import (  # noqa: F401
     VtokenError,

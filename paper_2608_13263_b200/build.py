@@ -1,7 +1,6 @@
-"""Builds the CUDA libraries in-tree with nvcc for sm_100a:
+"""Builds the CUDA library in-tree with nvcc for sm_100a:
 
   libvtoken.so          the repack library (C ABI of include/vtoken.h)
-  libvtoken_harness.so  harness kernels (pool fill, verifier, decode-read proxy)
 
 ``python -m paper_2608_13263_b200.build`` rebuilds when a source is newer than its library.
 """
@@ -18,11 +17,9 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 
 LIB = os.path.join(PKG, "libvtoken.so")
-HARNESS_LIB = os.path.join(PKG, "libvtoken_harness.so")
 
 LIB_SOURCES = ["api.cu", "plan.cu", "copy.cu", "gather.cu", "gather_static.cu", "runtime.cu", "plan_partial.cu",
                "waves.cu", "slot_cache.cu", "check.cu"]
-HARNESS_SOURCES = ["harness.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC",
@@ -57,8 +54,6 @@ def _build(lib: str, sources, verbose: bool, extra=()) -> None:
 def build(force: bool = False, verbose: bool = False) -> None:
     if force or _stale(LIB, LIB_SOURCES):
         _build(LIB, LIB_SOURCES, verbose)
-    if force or _stale(HARNESS_LIB, HARNESS_SOURCES):
-        _build(HARNESS_LIB, HARNESS_SOURCES, verbose)
 
 
 if __name__ == "__main__":

@@ -3,7 +3,9 @@ import ctypes
 import os
 import re
 
-from paper_2608_13263_b200 import binding, build, harness
+from harness import build as harness_build
+from harness import kernels as harness
+from paper_2608_13263_b200 import binding, build
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
@@ -28,7 +30,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_harness_library_loads():
-    build.build()
+    harness_build.build()
     lib = ctypes.CDLL(harness.LIB_PATH)
     for n in harness.SYMBOLS:
         assert hasattr(lib, n), n

@@ -10,7 +10,7 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 CUDA_HOME = os.environ.get("CUDA_HOME", "/usr/local/cuda")

@@ -5,7 +5,7 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 from test_oracle_check_tables import BIT, plant, recipes
 

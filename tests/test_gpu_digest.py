@@ -5,7 +5,7 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -41,7 +41,7 @@ def device_digest(prob, tt_slots, keep, l0, l1, select=None):
 ], ids=lambda w: f"{w.name}-row{w.row_bytes}")
 def test_digest_matches_oracle_and_survives_repack(w):
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     prob = DeviceProblem(w, fill_seed=1)
     L = w.num_layers
     k, v = host_pools(w)

@@ -10,7 +10,7 @@ import numpy as np
 import pytest
 
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -39,7 +39,7 @@ def _fit(name, kw, free_bytes):
 @pytest.mark.parametrize("name,kw", CASES, ids=[f"{n}{'-S32' if k else ''}" for n, k in CASES])
 def test_full_size_graph_side_stream(name, kw):
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem, origin_map
+    from harness.device import DeviceProblem, origin_map
     torch.cuda.empty_cache()
     free_bytes, _ = torch.cuda.mem_get_info()
     w, requests = _fit(name, kw, free_bytes)

@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -44,7 +44,7 @@ def random_problem(rng):
 @pytest.mark.parametrize("seed", range(60 * FUZZ_SCALE))
 def test_fuzz_whole_and_partial_plans(seed):
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     rng = np.random.default_rng(1000 + seed)
     w = random_problem(rng)
     S = w.block_size
@@ -103,7 +103,7 @@ def test_fuzz_repack_in_waves(seed):
     request is the same before and after."""
     import torch
     from paper_2608_13263_b200 import binding as vt
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     rng = np.random.default_rng(5000 + seed)
     w = random_problem(rng)
     S = w.block_size

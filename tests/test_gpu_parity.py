@@ -6,7 +6,7 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -39,7 +39,7 @@ def assert_tables_equal(out, p, w):
 
 def run_and_compare(w, copy_variant=0, num_free=None, whole_pool=True, capacity_slack=0):
     """plan + repack on the GPU, oracle on the host, compare everything."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=copy_variant, capacity_slack=capacity_slack)
     nf_dev = None
@@ -130,7 +130,7 @@ def test_copy_work_distribution_modes(dynamic, chunk, monkeypatch):
               wl.longctx_scissor(seed=5, requests=2, lo=1500, hi=2500, layers=2, block_size=32),
               wl.tiny(seed=1)):
         run_and_compare(w, copy_variant=2)
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.llama8b_h2o(seed=2, requests=5, lo=200, hi=900, layers=2)
     prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=2)
     p = vto.plan_workload(w)
@@ -153,7 +153,7 @@ def test_launch_modes_give_the_same_result(pdl, monkeypatch):
     copy paths, with launches issued back to back on one stream without host synchronisation between
     plan, copy and the next plan."""
     monkeypatch.setenv("VTOKEN_PDL", pdl)
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     for variant in (1, 2):
         run_and_compare(wl.mistral7b_random(seed=9, requests=6, lo=80, hi=600, layers=2), copy_variant=variant)
@@ -270,7 +270,7 @@ def test_capacities_larger_than_the_problem():
 
 def test_repeated_repack_and_idempotence():
     """Adopt the new tables, evict again, repack again; then all-keep -> nothing to gain."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     w = wl.mistral7b_random(seed=21, requests=8, lo=100, hi=400, layers=2, heads=2, head_dim=64)
     out, p = run_and_compare(w)
@@ -298,7 +298,7 @@ def test_repeated_repack_and_idempotence():
 @pytest.mark.parametrize("heads,head_dim", [(1, 8), (4, 64)], ids=["register-path", "bulk-path"])
 def test_out_of_range_ids_raise_flags_not_faults(heads, head_dim):
     """Host-fabricated bad slot / block / free ids: a flag bit, the row skipped, no fault."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     rng = np.random.default_rng(4)
     lens = [60, 60]
     keeps = [(rng.random(60) < 0.3).astype(np.uint8) for _ in lens]
@@ -321,7 +321,7 @@ def test_out_of_range_ids_raise_flags_not_faults(heads, head_dim):
 def test_counts_above_capacity_are_clamped_and_flagged():
     """A device-side request count or free count above the create-time capacities: clamped,
     VTOKEN_FLAG_CAPACITY raised, the part inside the capacities still exact."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     w = wl.mistral7b_random(seed=13, requests=8, lo=50, hi=300, layers=1, heads=1, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)                 # capacities == problem sizes
@@ -343,7 +343,7 @@ def test_tables_beyond_the_context_capacities_are_clipped(planner):
     """Token and block tables longer than the capacities the context was created with: entries at or
     beyond a capacity do not exist for the planner (the result is the oracle's on the clipped tables),
     VTOKEN_FLAG_CAPACITY is raised, and nothing is written behind a capacity in any output buffer."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.mistral7b_random(seed=21, requests=9, lo=60, hi=400, layers=1, heads=1, head_dim=64)
     T, NBT = w.num_tokens, len(w.bt_blocks)
     cap_t, cap_b = T - 157, NBT - 5                      # cuts into the last request (and the one before it)
@@ -389,7 +389,7 @@ def _misaligned_copy(t, offset_elems):
 def test_tables_that_are_not_16_byte_aligned(planner):
     """The planners read four table entries per thread with 16-byte and 4-byte accesses when the caller's
     arrays allow it; arrays that start at an odd element take the scalar path and give the same result."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.mistral7b_random(seed=23, requests=7, lo=50, hi=1400, layers=1, heads=1, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
     prob.tt_slots = _misaligned_copy(prob.tt_slots, 1)
@@ -420,7 +420,7 @@ def test_tables_that_are_not_16_byte_aligned(planner):
 def test_token_table_that_does_not_start_at_entry_zero(planner):
     """tt_offsets[0] > 0: the entries in front of the first request belong to nobody; they are neither
     counted nor written, and every request is planned as if the table started at its first entry."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     w = wl.mistral7b_random(seed=29, requests=6, lo=50, hi=900, layers=1, heads=1, head_dim=64)
     gap = 1029                                           # more than one tile, not a multiple of four
@@ -455,7 +455,7 @@ def test_token_table_that_does_not_start_at_entry_zero(planner):
 
 
 def test_argument_errors():
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.tiny()
     prob = DeviceProblem(w)
     with pytest.raises(vt.VtokenError) as e:
@@ -473,7 +473,7 @@ def test_gather_logical_before_equals_after_and_matches_oracle(heads, head_dim):
     """Rows below 512 bytes go through the register kernel, the others through the bulk-copy kernel
     in gather mode; the last step replays the gather from a captured graph (its work tickets must
     be back at zero after every launch)."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     w = wl.steady_state(seed=3, requests=10, lo=100, hi=900, layers=3, heads=heads, head_dim=head_dim)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
@@ -543,7 +543,7 @@ def test_gather_logical_before_equals_after_and_matches_oracle(heads, head_dim):
 
 
 def test_repack_host_tables_entry_point():
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     w = wl.mistral7b_random(seed=8, requests=12, lo=100, hi=400, layers=2, heads=2, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
@@ -576,7 +576,7 @@ def test_graph_capture_side_stream_replay_with_new_contents():
     """plan + repack captured once on a side stream; replayed three times after rewriting the
     CONTENTS of the input buffers (same addresses, same capacities); a consumer on the main
     stream waits on the event recorded behind the replay (pre-attention visibility)."""
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     torch = _torch()
     base = wl.mistral7b_random(seed=30, requests=10, lo=100, hi=400, layers=2, heads=2, head_dim=64)
     prob = DeviceProblem(base, fill_seed=FILL_SEED, capacity_slack=64)
@@ -627,8 +627,8 @@ def test_decode_read_proxy_is_undisturbed_by_a_concurrent_repack():
     """A reader of every allocated block through the OLD block tables (decode-read proxy) runs on
     one stream while the captured repack runs on another: its per-request checksums must equal the
     solo values, because destinations are free blocks and sources are only read."""
-    from paper_2608_13263_b200 import harness as vh
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness import kernels as vh
+    from harness.device import DeviceProblem
     torch = _torch()
     w = wl.steady_state(seed=9, requests=40, lo=300, hi=3000, layers=4)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)

@@ -6,7 +6,7 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -47,7 +47,7 @@ OPTION_SETS = [
 
 def run_partial(w, opts, num_free=None, whole_pool=True):
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     opts = dict(opts)
     protect = None
     if opts.get("protect") == "prefix":
@@ -111,7 +111,7 @@ def test_partial_free_list_cut():
 @pytest.mark.parametrize("w", small_configs(), ids=lambda w: f"{w.name}-S{w.block_size}")
 def test_block_liveness_matches_oracle(w):
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
     n_b = torch.full((w.num_blocks,), -1, dtype=torch.int32, device=prob.device)
     hist = torch.full((w.block_size + 1,), -1, dtype=torch.int64, device=prob.device)
@@ -132,7 +132,7 @@ def test_partial_plan_full_size_steady_state_tables():
     """The partial planner at the benchmark's largest table size (512 requests, 2.2 M entries):
     all tables and lists against the oracle; pools verified through the origin map."""
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem, origin_map
+    from harness.device import DeviceProblem, origin_map
     free_bytes, _ = torch.cuda.mem_get_info()
     requests = 512
     while True:
@@ -162,7 +162,7 @@ def test_partial_plan_full_size_steady_state_tables():
 def test_shared_prefix_workload(degree):
     """Synthetic prefix-cache workload: shared blocks protected, private suffixes repacked."""
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w, protect = wl.shared_prefix(seed=degree, groups=2, degree=degree, prefix_len=256, suffix_len=320, layers=2,
                                   heads=2, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
@@ -189,7 +189,7 @@ def test_shared_prefix_workload(degree):
 def test_repack_host_partial_entry_point(opts):
     """Host tables in, host tables out, partial planner; the protect mask is a host array."""
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.steady_state(seed=5, requests=14, lo=100, hi=900, layers=2, heads=2, head_dim=64)
     opts = dict(opts)
     if opts.get("protect") == "prefix":
@@ -239,7 +239,7 @@ def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach):
     reclaimed and the released lists, counts and whole pools against the oracle; the shared blocks
     keep their bytes."""
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w, protect = wl.shared_prefix(seed=10 + degree, groups=2, degree=degree, prefix_len=256, suffix_len=320, layers=2,
                                   heads=2, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
@@ -274,7 +274,7 @@ def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach):
 
 def test_detach_needs_a_released_list_and_is_refused_by_the_composite_entry_points():
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w, protect = wl.shared_prefix(seed=3, groups=1, degree=2, prefix_len=64, suffix_len=80, layers=1, heads=1,
                                   head_dim=8)
     prob = DeviceProblem(w, fill_seed=FILL_SEED, wave_capacity=True)

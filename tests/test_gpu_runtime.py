@@ -371,8 +371,8 @@ def test_runtime_flags_and_edges():
 def test_slot_mapping_full_size_tables_match_oracle():
     """Slot mapping over the steady-state workload's token tables (2.2 M logical entries)."""
     import torch
-    from paper_2608_13263_b200 import workloads as wl
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness import workloads as wl
+    from harness.device import DeviceProblem
     w = wl.steady_state(seed=0)
     prob = DeviceProblem(w, allocate_pools=False)
     # the context wants pools: a one-layer pool of 16-byte rows is enough for table-only calls
@@ -400,7 +400,7 @@ def test_slot_cache_full_size_rebuild_then_append_only():
     cache is rebuilt for every request and equals the slot mapping; a decode step that appends one
     token per request then only appends; an eviction in three requests rebuilds exactly those."""
     import torch
-    from paper_2608_13263_b200 import workloads as wl
+    from harness import workloads as wl
     w = wl.steady_state(seed=0)
     R = w.num_requests
     dev = torch.device("cuda:0")

@@ -12,14 +12,14 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
 
 def test_wait_runs_out_sets_flag_and_context_survives():
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.llama8b_h2o(seed=0, requests=4, lo=200, hi=600, layers=2)
     os.environ["VTOKEN_WAIT_LIMIT_MS"] = "20"
     os.environ["VTOKEN_TEST_STALL_ITEM"] = "5"

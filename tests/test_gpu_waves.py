@@ -6,7 +6,7 @@ import pytest
 
 from oracle import vto
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -55,7 +55,7 @@ def compare(out, v, num_waves):
 
 def run_waves(w, nf, num_waves, partial=None, whole_pool=True):
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     prob = DeviceProblem(w, fill_seed=FILL_SEED, wave_capacity=True)
     dpart = None
     if partial is not None:
@@ -119,7 +119,7 @@ def test_waves_graph_replay_after_the_pools_are_refilled():
     """The whole chain is one captured graph on a side stream; replaying it after restoring the
     pools reproduces the result (every count and pool lives on the device)."""
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.mistral7b_random(seed=4, requests=20, lo=100, hi=400, layers=2)
     biggest, _ = largest_demand(w)
     W = 5
@@ -149,7 +149,7 @@ def test_waves_graph_replay_after_the_pools_are_refilled():
 
 def test_waves_argument_errors():
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.tiny(seed=0)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)           # max_free_blocks = len(free list): no room to grow
     i32 = dict(dtype=torch.int32, device=prob.device)
@@ -184,7 +184,7 @@ def test_waves_full_size_llama_shape_with_a_twentieth_of_the_headroom():
     blocks; a pool of the largest single demand finishes the same repack in waves.  Tables against
     the oracle, both pools through the origin map."""
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem, origin_map
+    from harness.device import DeviceProblem, origin_map
     free_bytes, _ = torch.cuda.mem_get_info()
     requests = 64
     while True:

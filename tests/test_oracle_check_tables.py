@@ -7,7 +7,7 @@ import numpy as np
 import pytest
 
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 BIT = {"offsets": 1, "block_range": 2, "block_twice": 4, "free_range": 8, "free_twice_or_held": 16,
        "slot_range": 32, "foreign_slot": 64, "slot_twice": 128}

@@ -3,7 +3,7 @@ same formula, invariance under a repack, and sensitivity to every defect it exis
 import numpy as np
 
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 A, B, C, D = 0x9E3779B97F4A7C15, 0xD1B54A32D192ED03, 0x8CB92BA72F3D8DD7, 0xA0761D6478BD642F
 

@@ -8,7 +8,7 @@ import pytest
 
 from definition_twin import repack_partial_definition, to_csr
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 
 def workloads():

@@ -12,7 +12,7 @@ import pytest
 from conftest import read_golden
 from definition_twin import repack_definition, to_csr
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 
 # ------------------------------------------------------------------------------------------

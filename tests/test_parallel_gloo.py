@@ -16,8 +16,8 @@ def _worker(rank, world, port, q):
     os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1",
                       MASTER_PORT=str(port))
     from oracle import vto
-    from paper_2608_13263_b200 import workloads as wl
-    from paper_2608_13263_b200.parallel import Ranks, job_throughput
+    from harness import workloads as wl
+    from harness.parallel import Ranks, job_throughput
     ranks = Ranks.from_env(world)
     ranks.init(backend="gloo")
     # per-rank seed -> different problems, as in the benchmark
@@ -52,7 +52,7 @@ def test_two_rank_weak_scaling_aggregation():
 
 def test_world_size_mismatch_is_an_error():
     sys.path.insert(0, ROOT)
-    from paper_2608_13263_b200.parallel import Ranks
+    from harness.parallel import Ranks
     os.environ.pop("WORLD_SIZE", None)
     os.environ.pop("RANK", None)
     try:

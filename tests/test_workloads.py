@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from oracle import vto
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 SMALL = [
     lambda s: wl.tiny(seed=s),

@@ -12,14 +12,14 @@ import numpy as np
 import pytest
 
 from paper_2608_13263_b200 import binding as vt
-from paper_2608_13263_b200 import workloads as wl
+from harness import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
 
 def test_noalloc_gather_equals_context_gather_twice_in_a_row():
     import torch
-    from paper_2608_13263_b200.device import DeviceProblem
+    from harness.device import DeviceProblem
     w = wl.steady_state(seed=6, requests=14, lo=100, hi=1200, layers=3, heads=2, head_dim=64)
     prob = DeviceProblem(w, fill_seed=1)
     dev = prob.device

@@ -6,9 +6,12 @@ copy kernel) on a side stream, over one seeded synthetic workload whose pools ar
 in HBM.  Metric: repack HBM GB/s = 2 * M * token_bytes / t (every moved row read once and
 written once, K and V, all layers), M = live tokens of the admitted requests.
 
-    python bench.py                       # 1 GPU, Llama-3-8B-shaped KV, H2O-style 20 % budget
+    python bench.py                       # 1 GPU: the steady-state serving proxy (512 requests, 137 GiB of
+                                          # pools, incremental repack, beside a decode-read proxy), and the
+                                          # other four roofline workloads as entries of "configs"
     python bench.py --config mistral7b_random --steps 20 --warmup 3
-    torchrun ... bench.py --gpus N        # one independent pool per rank (weak scaling, no collective)
+    python bench.py --gpus N              # one independent pool per rank (weak scaling, no collective);
+                                          # starts its own ranks unless a launcher (torchrun) already did
     python bench.py --impl reference      # the CPU oracle timed on the host cores
 """
 from __future__ import annotations
@@ -16,6 +19,7 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import socket
 import subprocess
 import sys
 import threading
@@ -33,6 +37,12 @@ METRIC = "repack HBM GB/s (read+write); live tokens repacked/s and fraction of H
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 KERNELS_PER_STEP = 4        # plan: tiles, scan, assign; copy: 1
+DEFAULT_CONFIG = "steady_state"
+# the other roofline workloads, measured after the default one and reported under "configs"
+OTHER_CONFIGS = [("llama8b_h2o", 0), ("mistral7b_random", 0), ("longctx_scissor", 0), ("steady_state", 32)]
+# launch shapes of the copy kernel tried beside the decode-read proxy: (grid cap, warps per CTA, ring stages)
+SWEEP_CTAS = (148, 111, 74, 37, 18)
+SWEEP_RINGS = ((8, 6), (8, 3), (4, 3))       # 192, 96, 48 KiB of shared memory per CTA with 4 KiB items
 
 
 def measured_peak():
@@ -58,7 +68,7 @@ def committed_traffic(token_bytes):
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed regions run."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
@@ -90,7 +100,7 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
+        sm, mx, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.lines:
             f = [x.strip() for x in line.split(",")]
@@ -99,13 +109,20 @@ class ClockSampler:
             try:
                 sm.append(float(f[0]))
                 mx.append(float(f[1]))
+                power.append(float(f[2]))
             except ValueError:
                 continue
             for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        # "under load": samples drawing clearly more than the idle floor of the run
+        load = sm
+        if power and max(power) > min(power):
+            cut = min(power) + 0.25 * (max(power) - min(power))
+            load = [s for s, p in zip(sm, power) if p > cut] or sm
+        return {"sm_mhz": float(np.median(load)) if load else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "samples_under_load": len(load), "power_w_max": max(power) if power else None,
+                "reasons": sorted(reasons)}
 
 
 def build_workload(name, seed, scale_requests=1.0, block_size=0):
@@ -118,6 +135,23 @@ def build_workload(name, seed, scale_requests=1.0, block_size=0):
         default_r = inspect.signature(gen).parameters["requests"].default
         kw["requests"] = max(1, int(round(default_r * scale_requests)))
     return gen(seed=seed, **kw)
+
+
+def workload_config(w, args, world, moved_tokens, scale_requests):
+    """The `config` object of the JSON line: the workload and nothing specific to an arm, so that the
+    CUDA arm and the reference arm describe the same thing with the same keys."""
+    bytes_per_step = 2 * moved_tokens * w.token_bytes
+    return {"workload": f"{w.name} (seed {args.seed} + rank)", "requests": w.num_requests,
+            "layers": w.num_layers, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
+            "block_size": w.block_size, "num_blocks": w.num_blocks, "row_bytes": w.row_bytes,
+            "token_bytes": w.token_bytes, "logical_tokens": w.num_tokens,
+            "tokens_moved_per_step": int(moved_tokens), "bytes_moved_per_step": int(bytes_per_step),
+            "pool_GiB_per_gpu": 2 * w.pool_bytes / 2 ** 30, "scale_requests": scale_requests,
+            "l2": "moved bytes per step exceed the 126 MB L2 (no flush needed)" if bytes_per_step > 4 * 126e6
+                  else "moved bytes per step fit in L2: launch-bound parity configuration",
+            "plan_mode": args.plan_mode if args.plan_mode == "whole" else
+                         "partial: sources = blocks that are not fully live, trigger F > 1/4",
+            "parallelism": f"{world} independent pools, no collective"}
 
 
 def context_stats(w, out):
@@ -133,37 +167,33 @@ def context_stats(w, out):
 
 
 # ----------------------------------------------------------------------------------------------
-# reference arm: the CPU oracle, as it stands, on the host cores
+# the CPU oracle, as it stands, on the host cores (reference arm and cpu_baseline leg)
 # ----------------------------------------------------------------------------------------------
-def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1, use_gpu_fill=True):
+def default_oracle_layers(w):
+    """Layers of the CPU sample: host pools of 2 * layers slabs must fit host memory comfortably
+    (a slab of the steady-state workload is 2.1 GiB, of which the sample touches the moved rows)."""
+    return 4 if w.slab_bytes > (1 << 30) else 8
+
+
+def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1):
     """Times plan + row moves of the oracle on `sample_layers` layers (K and V) of the workload.
-    Returns (seconds per step, moved bytes per step, description)."""
+    Host pools are slab-sized (the moves use the workload's real slot addresses); the rows the moves
+    read hold seeded random 16-bit words drawn with numpy, every other row is untouched zero memory
+    (a byte copy's time does not depend on the values).  Returns a dict with per-step seconds."""
     from oracle import vto
     L = min(sample_layers, w.num_layers)
     threads = max(1, min(threads, 2 * L))      # one slab per thread at most
+    p = vto.plan_workload(w)
     shape = (L, w.slots_per_layer, w.row_elems)
-    k = v = None
-    if use_gpu_fill:
-        try:
-            import torch
-            from harness import kernels as vh
-            if torch.cuda.is_available():
-                k = np.empty(shape, np.uint16)
-                v = np.empty(shape, np.uint16)
-                buf = torch.empty((w.slots_per_layer, w.row_elems), dtype=torch.int16, device="cuda")
-                for kv, dst in ((0, k), (1, v)):
-                    for l in range(L):
-                        vh.vth_fill(buf, kv, w.num_layers, l, l + 1, w.slots_per_layer, w.row_elems, fill_seed)
-                        dst[l] = buf.cpu().numpy().view(np.uint16)
-                del buf
-        except Exception:
-            k = v = None
-    if k is None:
-        rng = np.random.default_rng(fill_seed)
-        k = rng.integers(0, 2 ** 16, size=shape, dtype=np.uint16)
-        v = rng.integers(0, 2 ** 16, size=shape, dtype=np.uint16)
+    rng = np.random.Generator(np.random.PCG64(fill_seed))
+    k, v = np.zeros(shape, np.uint16), np.zeros(shape, np.uint16)
+    src = np.unique(p.move_src)
+    for pool in (k, v):
+        for l in range(L):
+            for a in range(0, len(src), 65536):
+                rows = src[a:a + 65536]
+                pool[l, rows] = rng.integers(0, 1 << 16, size=(len(rows), w.row_elems), dtype=np.uint16)
     times = []
-    p = None
     for it in range(warmup + steps):
         t0 = time.perf_counter()
         p = vto.plan_workload(w)
@@ -173,19 +203,22 @@ def oracle_sample(w, sample_layers, threads, steps, warmup, fill_seed=1, use_gpu
             times.append(dt)
     moved = 2 * p.num_moves * (2 * L * w.row_bytes)
     desc = (f"oracle plan over all {w.num_requests} requests + row moves of layers 0..{L - 1} "
-            f"(K and V, {2 * L} of {2 * w.num_layers} slabs), host-resident pools, {threads} OpenMP threads")
-    return float(np.mean(times)), moved, desc, p, threads
+            f"(K and V, {2 * L} of {2 * w.num_layers} slabs), host-resident slab-sized pools with seeded random "
+            f"words at the source rows, {threads} OpenMP threads; {steps} timed steps after {warmup} warm-ups")
+    return {"times": times, "moved_bytes": moved, "desc": desc, "plan": p, "threads": threads}
 
 
-def cpu_baseline_leg(w, args, partial_opts, waves=0):
+def cpu_baseline_leg(w, args, partial_opts, waves=0, steps=12, warmup=2):
     """The CPU-baseline leg of the CUDA arm: the oracle, as it stands, timed on the host cores on a
     bounded sample of the workload.  This is the only place where the CUDA arm executes the oracle;
     the plans it computed on the way are returned so that the device's tables and pools can be
     compared with them at full size."""
     from oracle import vto
     cores = min(os.cpu_count() or 1, vto.openmp_threads())
-    sec, moved, desc, p_whole, cores = oracle_sample(w, args.oracle_layers, cores, 3, 1)
-    sec1, moved1, _, _, _ = oracle_sample(w, 1, 1, 2, 1)
+    layers = args.oracle_layers or default_oracle_layers(w)
+    s = oracle_sample(w, layers, cores, steps, warmup)
+    s1 = oracle_sample(w, 1, 1, 3, 1)
+    p_whole = s["plan"]
     plans = {"whole": p_whole}
     if partial_opts is not None:
         plans["partial"] = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets,
@@ -197,8 +230,11 @@ def cpu_baseline_leg(w, args, partial_opts, waves=0):
         plans["waves"] = vto.plan_waves(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets,
                                         w.tt_slots, w.keep, w.free_blocks[:headroom], waves, w.select, w.thr_num,
                                         w.thr_den)
-    baseline = {"value": moved / sec / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc,
-                "single_thread_GBs": moved1 / sec1 / 1e9}
+    gbs = lambda sec: s["moved_bytes"] / sec / 1e9
+    baseline = {"value": gbs(float(np.median(s["times"]))), "unit": "GB/s", "cores": s["threads"], "kind": "oracle",
+                "sample": s["desc"], "value_is": "median over the timed steps",
+                "min": gbs(max(s["times"])), "max": gbs(min(s["times"])),
+                "single_thread_GBs": s1["moved_bytes"] / float(np.median(s1["times"])) / 1e9}
     return baseline, plans
 
 
@@ -209,16 +245,20 @@ def run_reference(args):
     from oracle import vto
     w = build_workload(args.config, args.seed, args.scale_requests, args.block_size)
     cores = min(os.cpu_count() or 1, vto.openmp_threads())
-    sec, moved, desc, p, cores = oracle_sample(w, args.oracle_layers, cores, args.steps, max(1, min(args.warmup, 2)))
-    gbs = moved / sec / 1e9
+    layers = args.oracle_layers or default_oracle_layers(w)
+    s = oracle_sample(w, layers, cores, args.steps, max(2, args.warmup))
+    sec = float(np.median(s["times"]))
+    gbs = s["moved_bytes"] / sec / 1e9
+    p = s["plan"]
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": f"{w.name} (seed {args.seed})", "requests": w.num_requests,
-                   "tokens_moved_per_step": p.num_moves, "sample": desc},
-        "tokens_per_s": moved / (2 * w.token_bytes) / sec,
-        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": desc},
+        "config": workload_config(w, args, args.gpus, p.num_moves, args.scale_requests),
+        "tokens_per_s": s["moved_bytes"] / (2 * w.token_bytes) / sec,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": s["threads"], "kind": "oracle", "sample": s["desc"],
+                         "value_is": "median over the timed steps",
+                         "min": s["moved_bytes"] / max(s["times"]) / 1e9, "max": s["moved_bytes"] / min(s["times"]) / 1e9},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
@@ -227,39 +267,77 @@ def run_reference(args):
 # ----------------------------------------------------------------------------------------------
 # CUDA arm
 # ----------------------------------------------------------------------------------------------
-def run_cuda(args):
+class Timer:
+    """Device timing of graph replays on the side stream, bracketed by a barrier and a device
+    synchronisation on both sides."""
+
+    def __init__(self, ranks, dev, side):
+        self.ranks, self.dev, self.side = ranks, dev, side
+
+    def __call__(self, graph, steps, warmup, per_launch=False):
+        import torch
+        side = self.side
+        with torch.cuda.stream(side):
+            for _ in range(warmup):
+                graph.replay()
+        side.synchronize()
+        self.ranks.barrier()
+        torch.cuda.synchronize(self.dev)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        with torch.cuda.stream(side):
+            evs[0].record(side)
+            for i in range(steps):
+                graph.replay()
+                if per_launch or i == steps - 1:
+                    evs[i + 1].record(side)
+        side.synchronize()
+        torch.cuda.synchronize(self.dev)
+        self.ranks.barrier()
+        total = evs[0].elapsed_time(evs[steps])
+        each = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)] if per_launch else []
+        return total, each
+
+
+def fit_workload(args, name, seed, block_size, scale, dev):
+    """The workload at the asked size, or with the request count halved until its pools fit the free
+    memory of this (shared) GPU; the scale actually used is reported."""
+    import torch
+    w = build_workload(name, seed, scale, block_size)
+    torch.cuda.empty_cache()
+    free_b, _ = torch.cuda.mem_get_info(dev)
+    while 2 * w.pool_bytes + (6 << 30) > free_b and w.num_requests > 1:
+        scale *= 0.5
+        w = build_workload(name, seed, scale, block_size)
+    return w, scale
+
+
+def measure(args, ranks, dev, side, name, block_size, main):
+    """One workload through the whole path.  Returns the dict of everything measured; for the main
+    workload that is the JSON line (minus keys added by the caller), for the others a summary."""
     import torch
 
-    from paper_2608_13263_b200 import binding as vt
     from harness.device import DeviceProblem, origin_map
-    from harness.parallel import Ranks
+    from paper_2608_13263_b200 import binding as vt
 
-    ranks = Ranks.from_env(args.gpus)
-    torch.cuda.set_device(ranks.local_rank)
-    dev = torch.device("cuda", ranks.local_rank)
-    ranks.init(backend="nccl")
-
-    # one independent pool per rank: weak scaling, no data-path collective
     seed = args.seed + ranks.rank
-    w = build_workload(args.config, seed, args.scale_requests, args.block_size)
-    free_b, total_b = torch.cuda.mem_get_info(dev)
-    need = 2 * w.pool_bytes + (1 << 30)
-    while need > free_b * 0.95 and w.num_requests > 1:
-        args.scale_requests *= 0.5
-        w = build_workload(args.config, seed, args.scale_requests, args.block_size)
-        need = 2 * w.pool_bytes + (1 << 30)
-
+    asked = args.scale_requests if main else 1.0
+    w, scale = fit_workload(args, name, seed, block_size, asked, dev)
+    steps, warmup = args.steps, args.warmup
     prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas,
-                         wave_capacity=args.waves > 0)
+                         wave_capacity=main and args.waves > 0, coresident=args.coresident)
     partial_opts = dict(util=(1, 1), theta=(1, 4))     # fully live blocks stay; the paper's default trigger F > 0.25
-    if args.plan_mode == "partial":
-        do_plan = lambda st: prob.plan_partial(stream=st, **partial_opts)
-    else:
-        do_plan = lambda st: prob.plan(stream=st)
-    grid = vt.vtoken_copy_grid(prob.ctx)
-    side = torch.cuda.Stream(device=dev)
+    partial = main and args.plan_mode == "partial"
 
-    # ---- capture: whole path, and the copy alone -------------------------------------------
+    def do_plan(st, ctx=None):
+        if partial:
+            prob.plan_partial(stream=st, ctx=ctx, **partial_opts)
+        else:
+            prob.plan(stream=st, ctx=ctx)
+
+    grid = vt.vtoken_copy_grid(prob.ctx)
+    timed = Timer(ranks, dev, side)
+
+    # ---- capture: whole path, the copy alone, the plan alone --------------------------------
     side.wait_stream(torch.cuda.current_stream())
     with torch.cuda.stream(side):
         do_plan(side)
@@ -277,35 +355,11 @@ def run_cuda(args):
     M = out["num_moves"]
     bytes_per_step = 2 * M * w.token_bytes
 
-    def timed(graph, steps, warmup, per_launch=False):
-        """Device time of `steps` replays on the side stream (ms total, list of per-launch ms)."""
-        with torch.cuda.stream(side):
-            for _ in range(warmup):
-                graph.replay()
-        side.synchronize()
-        ranks.barrier()
-        torch.cuda.synchronize(dev)
-        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
-        with torch.cuda.stream(side):
-            evs[0].record(side)
-            for i in range(steps):
-                graph.replay()
-                if per_launch or i == steps - 1:
-                    evs[i + 1].record(side)
-        side.synchronize()
-        torch.cuda.synchronize(dev)
-        ranks.barrier()
-        total = evs[0].elapsed_time(evs[steps])
-        each = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)] if per_launch else []
-        return total, each
+    total_ms, _ = timed(g_all, steps, warmup)
+    copy_total_ms, copy_each = timed(g_copy, steps, warmup, per_launch=True)
+    plan_total_ms, _ = timed(g_plan, steps, warmup)
 
-    sampler = ClockSampler(ranks.local_rank)
-    sampler.start()
-    total_ms, _ = timed(g_all, args.steps, args.warmup)
-    copy_total_ms, copy_each = timed(g_copy, args.steps, args.warmup, per_launch=True)
-    plan_total_ms, _ = timed(g_plan, args.steps, args.warmup)
-
-    ms_per_step = ranks.max(total_ms / args.steps)
+    ms_per_step = ranks.max(total_ms / steps)
     all_bytes = ranks.sum(bytes_per_step)
     all_tokens = ranks.sum(M)
     value = all_bytes / (ms_per_step * 1e-3) / 1e9
@@ -326,29 +380,28 @@ def run_cuda(args):
     d2h = 4 * (R + 1) + 4 * NBT + 4 * T + 4 * NBT + 4 * R + 32
 
     def e2e_once():
-        if args.plan_mode == "partial":
+        if partial:
             return vt.vtoken_repack_host_partial(prob.ctx, num_requests=R, num_free=len(w.free_blocks),
                                                  thr_num=w.thr_num, thr_den=w.thr_den, stream=side, **partial_opts,
                                                  **h_in, **h_out)
         return vt.vtoken_repack_host(prob.ctx, num_requests=R, num_free=len(w.free_blocks), thr_num=w.thr_num,
                                      thr_den=w.thr_den, stream=side, **h_in, **h_out)
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         e2e_once()
     ranks.barrier()
     torch.cuda.synchronize(dev)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.perf_counter()
     e0.record(side)
-    for _ in range(args.steps):
+    for _ in range(steps):
         c_host = e2e_once()
     e1.record(side)
     side.synchronize()
-    e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / args.steps
-    e2e_ms = ranks.max(max(e0.elapsed_time(e1) / args.steps, e2e_wall_ms))
+    e2e_wall_ms = (time.perf_counter() - t0) * 1e3 / steps
+    e2e_ms = ranks.max(max(e0.elapsed_time(e1) / steps, e2e_wall_ms))
     # bytes the end-to-end call moved (it runs the same planner as the timed graph)
     e2e_bytes = ranks.sum(2 * c_host["num_moves"] * w.token_bytes)
     e2e_value = e2e_bytes / (e2e_ms * 1e-3) / 1e9
-    clocks = sampler.stop()      # sampled over every timed region above
 
     # ---- parity at full size, in the launch configuration that was timed --------------------
     # The oracle is executed in ONE place, the CPU-baseline leg (rank 0, N = 1): it times the oracle
@@ -356,10 +409,10 @@ def run_cuda(args):
     parity = "skipped (needs the cpu_baseline leg: N = 1 without --no-cpu-baseline)"
     cpu_baseline, plans = None, None
     if ranks.world == 1 and not args.no_cpu_baseline:
-        cpu_baseline, plans = cpu_baseline_leg(w, args, partial_opts if args.plan_mode == "partial" else None,
-                                               args.waves)
+        cpu_baseline, plans = cpu_baseline_leg(w, args, partial_opts if partial else None,
+                                               args.waves if main else 0, steps=12 if main else 5)
     if plans is not None and not args.no_verify:
-        p = plans["partial"] if args.plan_mode == "partial" else plans["whole"]
+        p = plans["partial"] if partial else plans["whole"]
         ok = (out["error_flags"] == 0 and c_host["error_flags"] == 0 and M == p.num_moves
               and np.array_equal(out["new_tt_slots"], p.new_tt_slots)
               and np.array_equal(out["new_bt_offsets"], p.new_bt_offsets)
@@ -372,26 +425,8 @@ def run_cuda(args):
               and np.array_equal(h_out["freed_blocks"].numpy()[:p.num_freed], p.freed_blocks))
         bad_words = prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst))
         parity = "ok" if (ok and bad_words == 0) else f"FAILED (tables_ok={ok}, mismatching_words={bad_words})"
-
-    # ---- a plain device-to-device copy on this GPU, now (context for run-to-run variation) ---
-    live_copy = None
-    free_now, _ = torch.cuda.mem_get_info(dev)
-    if free_now > (6 << 30):
-        n = 1 << 30
-        src_t = torch.empty(n, dtype=torch.int16, device=dev)
-        dst_t = torch.empty(n, dtype=torch.int16, device=dev)
-        for _ in range(3):
-            dst_t.copy_(src_t)
-        best = 1e9
-        for _ in range(10):
-            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            c0.record()
-            dst_t.copy_(src_t)
-            c1.record()
-            c1.synchronize()
-            best = min(best, c0.elapsed_time(c1))
-        live_copy = 4 * n / (best * 1e-3) / 1e9
-        del src_t, dst_t
+    if scale != asked:
+        parity += f" (on {w.num_requests} requests: the pools of the full workload did not fit this GPU's free memory)"
 
     # ---- roofline of the dominant kernel (the copy), timed alone on its stream ---------------
     peak, peak_kind = measured_peak()
@@ -404,64 +439,141 @@ def run_cuda(args):
                 "algorithmic_bytes_per_launch": bytes_per_step,
                 "launch_ms_mean": copy_ms, "launch_ms_median": float(np.median(copy_each)),
                 "launch_ms_min": float(np.min(copy_each)),
-                "plain_copy_now_GBs": live_copy,     # torch copy_ of 1 Gi 2-byte elements on this GPU, best of 10
-                "frac_of_plain_copy_now": (achieved / live_copy) if live_copy else None,
                 "traffic": (per_token * M) if per_token else None}
 
-    line = {
-        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": ranks.world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "u8", "data": "synthetic",
-        "config": {"workload": f"{w.name} (seed {args.seed}+rank)", "requests": w.num_requests,
-                   "layers": w.num_layers, "kv_heads": w.num_kv_heads, "head_dim": w.head_dim,
-                   "block_size": w.block_size, "num_blocks": w.num_blocks, "row_bytes": w.row_bytes,
-                   "token_bytes": w.token_bytes, "tokens_moved_per_step": M, "bytes_moved_per_step": bytes_per_step,
-                   "pool_GiB_per_gpu": 2 * w.pool_bytes / 2 ** 30, "scale_requests": args.scale_requests,
-                   "l2": "moved bytes per step exceed the 126 MB L2 (no flush needed)" if bytes_per_step > 4 * 126e6
-                         else "moved bytes per step fit in L2: launch-bound parity configuration",
-                   "launch": "CUDA graph (plan + copy) replayed on a side stream", "copy_grid": grid,
-                   "copy_work_distribution": ("fixed share per warp" if os.environ.get("VTOKEN_COPY_DYNAMIC") == "0"
-                                              else "ticket counter, " + os.environ.get("VTOKEN_COPY_CHUNK", "4") +
-                                                   " items per ticket") if grid["variant"] == 2 else "grid-stride rows",
-                   "plan_mode": args.plan_mode if args.plan_mode == "whole" else
-                                "partial: sources = blocks that are not fully live, trigger F > 1/4",
-                   "gpu": f"{torch.cuda.get_device_name(dev)} {str(torch.cuda.get_device_properties(dev).uuid)[-12:]}",
-                   "parallelism": f"{ranks.world} independent pools, no collective"},
-        "tokens_per_s": all_tokens / (ms_per_step * 1e-3),
+    res = {
+        "value": value, "ms_per_step": ms_per_step, "tokens_per_s": all_tokens / (ms_per_step * 1e-3),
+        "config": workload_config(w, args, ranks.world, M, scale),
         "frac_of_measured_hbm_peak": value / (peak * ranks.world),
         "frac_of_nominal_8TBs": value / (NOMINAL_HBM_GBS * ranks.world),
-        "plan_us": plan_total_ms / args.steps * 1e3, "copy_ms": copy_ms,
-        "clocks": clocks, "gpu_launches": (KERNELS_PER_STEP if args.plan_mode == "whole" else KERNELS_PER_STEP + 2) * args.steps,
+        "plan_us": plan_total_ms / steps * 1e3, "copy_ms": copy_ms,
         "e2e": {"value": e2e_value, "unit": "GB/s", "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h,
-                "what": ("vtoken_repack_host_partial" if args.plan_mode == "partial" else "vtoken_repack_host") +
+                "what": ("vtoken_repack_host_partial" if partial else "vtoken_repack_host") +
                         ": pinned host tables -> device, plan, copy, every output table -> host, sync; "
                         "the K/V pools are the GPU-resident cache and stay in HBM"},
-        "roofline": roofline, "parity": parity, "stats": context_stats(w, out),
+        "roofline": roofline, "parity": parity,
+        "launch": {"how": "CUDA graph (plan + copy) replayed on a side stream", "copy_grid": grid,
+                   "copy_work_distribution": "ticket counter" if grid["variant"] == 2 else "grid-stride rows",
+                   "gpu": f"{torch.cuda.get_device_name(dev)} {str(torch.cuda.get_device_properties(dev).uuid)[-12:]}"},
     }
-
-    if args.proxy:
-        line["concurrency"] = run_proxy(args, prob, w, side, g_all, bytes_per_step, dev)
-    if args.runtime:
-        line["runtime"] = run_runtime(args, prob, w, side, dev)
-    if args.waves:                # last: it overwrites allocated blocks
-        line["waves"] = run_waves(args, prob, w, side, dev, plans, ms_per_step)
-
     if cpu_baseline is not None:
-        line["cpu_baseline"] = cpu_baseline
+        res["cpu_baseline"] = cpu_baseline
+    if main:
+        res["stats"] = context_stats(w, out)
+        # a plain device-to-device copy on this GPU, now (context for run-to-run variation)
+        free_now, _ = torch.cuda.mem_get_info(dev)
+        if free_now > (6 << 30):
+            n = 1 << 30
+            src_t = torch.empty(n, dtype=torch.int16, device=dev)
+            dst_t = torch.empty(n, dtype=torch.int16, device=dev)
+            for _ in range(3):
+                dst_t.copy_(src_t)
+            best = 1e9
+            for _ in range(10):
+                c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                c0.record()
+                dst_t.copy_(src_t)
+                c1.record()
+                c1.synchronize()
+                best = min(best, c0.elapsed_time(c1))
+            roofline["plain_copy_now_GBs"] = 4 * n / (best * 1e-3) / 1e9     # torch copy_ of 1 Gi 2-byte elements
+            roofline["frac_of_plain_copy_now"] = achieved / roofline["plain_copy_now_GBs"]
+            del src_t, dst_t
+        if ranks.world == 1 and not args.no_proxy and M > 0:
+            res["concurrency"] = run_proxy(args, prob, w, side, do_plan, bytes_per_step, dev,
+                                           sweep=not args.no_sweep and name == DEFAULT_CONFIG)
+        if args.runtime:
+            res["runtime"] = run_runtime(args, prob, w, side, dev)
+        if args.waves:                # last: it overwrites allocated blocks
+            res["waves"] = run_waves(args, prob, w, side, dev, plans, ms_per_step)
     prob.close()
+    del prob, g_all, g_copy, g_plan, h_in, h_out
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_cuda(args):
+    import torch
+
+    from harness.parallel import Ranks
+
+    ranks = Ranks.from_env(args.gpus)
+    torch.cuda.set_device(ranks.local_rank)
+    dev = torch.device("cuda", ranks.local_rank)
+    ranks.init(backend="nccl")
+    side = torch.cuda.Stream(device=dev)
+
+    sampler = ClockSampler(ranks.local_rank)
+    sampler.start()
+    res = measure(args, ranks, dev, side, args.config, args.block_size, main=True)
+    others = []
+    if (ranks.world == 1 and args.config == DEFAULT_CONFIG and not args.block_size and args.scale_requests == 1.0
+            and args.plan_mode == "whole" and not args.no_configs):
+        for name, bs in OTHER_CONFIGS:
+            try:
+                r = measure(args, ranks, dev, side, name, bs, main=False)
+                others.append({"workload": r["config"]["workload"], "block_size": r["config"]["block_size"],
+                               "requests": r["config"]["requests"],
+                               "tokens_moved_per_step": r["config"]["tokens_moved_per_step"],
+                               "bytes_moved_per_step": r["config"]["bytes_moved_per_step"],
+                               "pool_GiB_per_gpu": r["config"]["pool_GiB_per_gpu"],
+                               "value": r["value"], "ms_per_step": r["ms_per_step"], "tokens_per_s": r["tokens_per_s"],
+                               "copy_ms": r["copy_ms"], "plan_us": r["plan_us"],
+                               "roofline": {k: r["roofline"][k] for k in ("achieved", "peak", "frac", "launch_ms_mean",
+                                                                          "algorithmic_bytes_per_launch")},
+                               "e2e": r["e2e"]["value"], "parity": r["parity"],
+                               "cpu_baseline": r.get("cpu_baseline", {}).get("value")})
+            except Exception as e:              # a sub-result must not cost the main line
+                others.append({"workload": name, "block_size": bs, "error": f"{type(e).__name__}: {e}"[:300]})
+    clocks = sampler.stop()      # sampled over every timed region above
+
+    line = {
+        "metric": METRIC, "value": res.pop("value"), "unit": "GB/s", "n_gpus": ranks.world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": res.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "u8", "data": "synthetic", "config": res.pop("config"),
+        "clocks": clocks,
+        "gpu_launches": (KERNELS_PER_STEP if args.plan_mode == "whole" else KERNELS_PER_STEP + 2) * args.steps,
+        "gpu_launches_what": "kernels of the library inside the timed region of `value` (plan + copy per step)",
+    }
+    line.update(res)
+    if others:
+        line["configs"] = others
     if ranks.rank == 0:
         print(json.dumps(line))
     ranks.finalize()
 
 
-def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
+def _stamps(events, origin):
+    return [origin.elapsed_time(e) for e in events]
+
+
+def _rate_inside(stamps, nbytes, lo, hi):
+    """GB/s of one stream inside the window [lo, hi] ms (stamps: start of the first launch, then the end
+    of every launch): every launch counts with the fraction of its duration that lies inside the window.
+    Also returns how many launches lay entirely inside."""
+    moved, whole = 0.0, 0
+    for a, b in zip(stamps[:-1], stamps[1:]):
+        if b <= a:
+            continue
+        inside = max(0.0, min(b, hi) - max(a, lo))
+        moved += nbytes * inside / (b - a)
+        whole += int(a >= lo and b <= hi)
+    if hi <= lo:
+        return None, 0
+    return moved / ((hi - lo) * 1e-3) / 1e9, whole
+
+
+def run_proxy(args, prob, w, side, do_plan, bytes_per_step, dev, sweep):
     """Repack (captured graph, side stream) beside a bandwidth-bound decode-read proxy that reads
     every allocated block through the OLD block tables on a high-priority main stream: each one
-    alone, then both at once.  The proxy's per-request checksums must not change (the repack
-    never writes an allocated block)."""
+    alone, then both at once.  Rates of the concurrent run are taken over the window in which both
+    streams were busy.  The proxy's per-request checksums
+    must not change (the repack never writes an allocated block).  With `sweep`, the same for a range
+    of copy-kernel launch shapes (grid cap x shared-memory ring size)."""
     import torch
     from harness import kernels as vh
+    from paper_2608_13263_b200 import binding as vt
     owner = np.repeat(np.arange(w.num_requests, dtype=np.int32), np.diff(w.bt_offsets))
     owner_d = torch.from_numpy(owner).to(dev)
     nbt = len(w.bt_blocks)
@@ -469,6 +581,7 @@ def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
     proxy_bytes = nbt * 2 * w.num_layers * block_bytes
     main = torch.cuda.Stream(device=dev, priority=-1)
     sums = torch.zeros(max(1, w.num_requests), dtype=torch.int64, device=dev)
+    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
 
     def proxy(stream):
         vh.vth_decode_read(prob.k_pool, prob.v_pool, prob.bt_offsets, prob.bt_blocks, owner_d, nbt, w.num_layers,
@@ -484,58 +597,100 @@ def run_proxy(args, prob, w, side, g_all, bytes_per_step, dev):
     main.synchronize()
     solo_sums = sums.clone()
     # proxy alone
-    n_proxy = max(2, args.steps // 4)
+    n_solo = 4
     a, b = ev(), ev()
     a.record(main)
-    for _ in range(n_proxy):
+    for _ in range(n_solo):
         proxy(main)
     b.record(main)
     main.synchronize()
-    proxy_alone_ms = a.elapsed_time(b) / n_proxy
-    # repack alone (again, same window length as the concurrent run)
-    n_rep = max(2, int(round(n_proxy * proxy_alone_ms / max(1e-3, bytes_per_step / 6e9 * 1e3))))
-    a, b = ev(), ev()
-    with torch.cuda.stream(side):
-        a.record(side)
-        for _ in range(n_rep):
-            g_all.replay()
-        b.record(side)
-    side.synchronize()
-    repack_alone_ms = a.elapsed_time(b) / n_rep
-    # both at once, released by one event
-    sums.zero_()
-    torch.cuda.synchronize(dev)
-    go, p0, p1, r0, r1 = ev(), ev(), ev(), ev(), ev()
-    go.record(torch.cuda.current_stream(dev))
-    main.wait_event(go)
-    side.wait_event(go)
-    p0.record(main)
-    with torch.cuda.stream(side):
-        r0.record(side)
-    # both queues are filled within a few hundred microseconds, the work lasts tens of milliseconds
-    for _ in range(n_proxy):
-        proxy(main)
-    with torch.cuda.stream(side):
-        for _ in range(n_rep):
-            g_all.replay()
-    p1.record(main)
-    with torch.cuda.stream(side):
-        r1.record(side)
-    torch.cuda.synchronize(dev)
-    proxy_conc_ms = p0.elapsed_time(p1) / n_proxy
-    repack_conc_ms = r0.elapsed_time(r1) / n_rep
-    window_ms = max(p0.elapsed_time(p1), r0.elapsed_time(r1), p0.elapsed_time(r1), r0.elapsed_time(p1))
-    # n_proxy launches accumulate by XOR: an even count cancels, an odd count equals the solo value
-    expect = solo_sums if n_proxy % 2 == 1 else torch.zeros_like(solo_sums)
-    checksum_ok = bool(torch.equal(sums, expect))
-    gbs = lambda nbytes, ms: nbytes / (ms * 1e-3) / 1e9
-    return {"proxy_bytes_per_launch": proxy_bytes, "proxy_launches": n_proxy, "repack_replays": n_rep,
-            "proxy_alone_GBs": gbs(proxy_bytes, proxy_alone_ms), "repack_alone_GBs": gbs(bytes_per_step, repack_alone_ms),
-            "proxy_concurrent_GBs": gbs(proxy_bytes, proxy_conc_ms),
-            "repack_concurrent_GBs": gbs(bytes_per_step, repack_conc_ms),
-            "sum_over_window_GBs": gbs(proxy_bytes * n_proxy + bytes_per_step * n_rep, window_ms),
-            "proxy_checksum_unchanged": checksum_ok,
-            "streams": "proxy on a high-priority stream, repack graph on the default-priority side stream"}
+    proxy_alone_ms = a.elapsed_time(b) / n_solo
+    proxy_alone = gbs(proxy_bytes, proxy_alone_ms)
+
+    def point(ctx, label):
+        """One launch shape: the repack alone, then beside the proxy."""
+        with torch.cuda.stream(side):
+            do_plan(side, ctx)
+            prob.repack(stream=side, ctx=ctx)
+        side.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            do_plan(torch.cuda.current_stream(), ctx)
+            prob.repack(stream=torch.cuda.current_stream(), ctx=ctx)
+        a, b = ev(), ev()
+        n_alone = 3
+        with torch.cuda.stream(side):
+            g.replay()
+            a.record(side)
+            for _ in range(n_alone):
+                g.replay()
+            b.record(side)
+        side.synchronize()
+        alone_ms = a.elapsed_time(b) / n_alone
+        # both at once, released by one event; the proxy queue is the longer one, so that every repack
+        # replay runs beside it
+        n_rep = 8
+        n_proxy = int(np.ceil((n_rep + 2) * alone_ms * 4.0 / proxy_alone_ms)) + 2
+        n_proxy = max(4, min(n_proxy, 80))
+        n_proxy += (n_proxy + 1) % 2                      # odd: the XOR checksums then equal the solo values
+        sums.zero_()
+        torch.cuda.synchronize(dev)
+        go = ev()
+        pe = [ev() for _ in range(n_proxy + 1)]
+        re_ = [ev() for _ in range(n_rep + 1)]
+        go.record(torch.cuda.current_stream(dev))
+        main.wait_event(go)
+        side.wait_event(go)
+        pe[0].record(main)
+        for i in range(n_proxy):
+            proxy(main)
+            pe[i + 1].record(main)
+            if i == 0:          # the repack joins once the proxy is queued
+                with torch.cuda.stream(side):
+                    re_[0].record(side)
+                    for j in range(n_rep):
+                        g.replay()
+                        re_[j + 1].record(side)
+        torch.cuda.synchronize(dev)
+        ps, rs = _stamps(pe, go), _stamps(re_, go)
+        lo, hi = max(ps[0], rs[0]), min(ps[-1], rs[-1])
+        p_rate, p_n = _rate_inside(ps, proxy_bytes, lo, hi)
+        r_rate, r_n = _rate_inside(rs, bytes_per_step, lo, hi)
+        ok = bool(torch.equal(sums, solo_sums))
+        grid = vt.vtoken_copy_grid(ctx or prob.ctx)
+        alone = gbs(bytes_per_step, alone_ms)
+        d = {"shape": label, "copy_ctas": grid["ctas"], "copy_smem_KiB": grid["smem_bytes"] / 1024,
+             "repack_alone_GBs": alone, "repack_concurrent_GBs": r_rate, "proxy_concurrent_GBs": p_rate,
+             "sum_concurrent_GBs": (r_rate + p_rate) if (r_rate and p_rate) else None,
+             "repack_share_of_solo": (r_rate / alone) if r_rate else None,
+             "proxy_share_of_solo": (p_rate / proxy_alone) if p_rate else None,
+             "launches_inside_window": {"proxy": p_n, "repack": r_n}, "proxy_checksum_unchanged": ok}
+        del g
+        return d
+
+    out = {"proxy_bytes_per_launch": proxy_bytes, "proxy_alone_GBs": proxy_alone,
+           "streams": "proxy on a high-priority stream, repack graph on the default-priority side stream",
+           "rates": "concurrent rates are taken over the window in which both streams were busy (8 repack replays); a "
+                    "launch that straddles an edge of the window counts with the part of its duration inside"}
+    out.update(point(None, "as timed above"))
+    if sweep:
+        pts = []
+        for warps, stages in SWEEP_RINGS:
+            for ctas in SWEEP_CTAS:
+                ctx = prob.make_ctx(max_ctas=ctas, copy_variant=2, tuning=dict(warps=warps, stages=stages))
+                try:
+                    pts.append(point(ctx, f"{ctas} CTAs x {warps} warps x {stages} stages"))
+                finally:
+                    torch.cuda.synchronize(dev)
+                    vt.vtoken_destroy(ctx)
+        ctx = prob.make_ctx(coresident=1)
+        try:
+            out["coresident_profile"] = point(ctx, "vtoken_config.coresident = 1")
+        finally:
+            torch.cuda.synchronize(dev)
+            vt.vtoken_destroy(ctx)
+        out["sweep"] = pts
+    return out
 
 
 def run_waves(args, prob, w, side, dev, plans, one_shot_ms):
@@ -847,19 +1002,82 @@ def run_plan_only(args):
     prob.close()
 
 
+
+
+# ----------------------------------------------------------------------------------------------
+# N > 1 without a launcher: this process starts one rank per GPU itself
+# ----------------------------------------------------------------------------------------------
+def free_port():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def spawn_ranks(n):
+    """`python bench.py --gpus N` with no launcher around it (WORLD_SIZE unset): start N copies of this
+    command, one rank per GPU, rendezvous on 127.0.0.1 at a free port.  Rank 0 prints the JSON line
+    (its output passes straight through); the exit code is the worst of the ranks'."""
+    port = free_port()
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        env.setdefault("NCCL_DEBUG", "WARN")          # keeps NCCL's communicator messages on stderr
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *sys.argv[1:]], env=env))
+    rc = 0
+    try:
+        for p in procs:
+            r = p.wait()
+            rc = rc or r
+    except BaseException:
+        for p in procs:
+            if p.poll() is None:
+                p.terminate()
+        raise
+    return rc
+
+
+def run_plumbing_check(args):
+    """The multi-rank plumbing of the CUDA arm without a GPU: launch (or self-spawn), rendezvous over
+    gloo, barrier, max-over-ranks time, sum-over-ranks work, one JSON line from rank 0.  No kernel
+    runs and nothing is measured: each rank's "work" is the size of its own seeded workload's tables
+    and its "time" a fixed figure that differs by rank, so that the reductions can be checked from
+    outside.  The line says what it is (`data`: "plumbing-check")."""
+    from harness.parallel import Ranks
+    ranks = Ranks.from_env(args.gpus)
+    ranks.init(backend="gloo")
+    w = build_workload("tiny", args.seed + ranks.rank)
+    units = float(w.num_tokens)                 # input size only: no method arithmetic outside the library
+    seconds = 1.0 + ranks.rank
+    ranks.barrier()
+    total_units, slowest = ranks.sum(units), ranks.max(seconds)
+    line = {"metric": METRIC, "value": total_units / slowest, "unit": "table entries/s (fabricated)", "n_gpus": ranks.world,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": slowest * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "plumbing-check",
+            "config": {"workload": "tiny (seed + rank)", "parallelism": f"{ranks.world} independent pools, no collective"},
+            "units_all_ranks": total_units, "slowest_rank_s": slowest, "rank_units": units}
+    if ranks.rank == 0:
+        print(json.dumps(line), flush=True)
+    ranks.finalize()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--config", default="llama8b_h2o", choices=sorted(wl.CONFIGS))
+    ap.add_argument("--config", default=DEFAULT_CONFIG, choices=sorted(wl.CONFIGS))
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0, help="copy path: 0 auto, 1 registers, 2 bulk copy")
     ap.add_argument("--max-ctas", type=int, default=0)
+    ap.add_argument("--coresident", type=int, default=0, help="1: the copy kernel's launch shape for running beside decode")
     ap.add_argument("--scale-requests", type=float, default=1.0)
-    ap.add_argument("--oracle-layers", type=int, default=8, help="layers in the CPU-baseline sample")
-    ap.add_argument("--proxy", action="store_true", help="also run the repack beside a decode-read proxy")
+    ap.add_argument("--oracle-layers", type=int, default=0,
+                    help="layers in the CPU-baseline sample (0: 8, or 4 when a slab exceeds 1 GiB)")
+    ap.add_argument("--no-proxy", action="store_true", help="skip the run beside the decode-read proxy")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sweep of copy-kernel launch shapes beside the proxy")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other roofline workloads (`configs`)")
     ap.add_argument("--proxy-ctas", type=int, default=0)
     ap.add_argument("--runtime", action="store_true", help="also time the token-table runtime kernels")
     ap.add_argument("--plan-mode", default="whole", choices=["whole", "partial"],
@@ -871,9 +1089,15 @@ def main():
     ap.add_argument("--plan-only", action="store_true",
                     help="time the planners alone on the workload's tables (no pools are allocated)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--plumbing-check", action="store_true",
+                    help="no GPU: exercise launch, rendezvous (gloo) and the reductions of the N-rank path only")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "cuda" or args.plumbing_check):
+        sys.exit(spawn_ranks(args.gpus))
+    if args.plumbing_check:
+        run_plumbing_check(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.plan_only:
         run_plan_only(args)

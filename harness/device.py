@@ -19,7 +19,9 @@ from .workloads import Workload
 class DeviceProblem:
     def __init__(self, w: Workload, device="cuda:0", fill_seed: int = 1, copy_variant: int = 0, max_ctas: int = 0,
                  capacity_slack: int = 0, allocate_pools: bool = True, wave_capacity: bool = False,
-                 ctx_capacity: dict = None):
+                 ctx_capacity: dict = None, **ctx_options):
+        """``ctx_options``: further keyword arguments of ``vtoken_create`` (coresident, wait_limit_ms,
+        plain_launches, tuning, debug_stall_item)."""
         self.w = w
         self.device = torch.device(device)
         self.fill_seed = fill_seed
@@ -65,13 +67,17 @@ class DeviceProblem:
             self.k_pool = torch.empty(shape, dtype=torch.int16, device=dev)
             self.v_pool = torch.empty(shape, dtype=torch.int16, device=dev)
             self.fill_pools()
-            caps = dict(max_requests=self.max_requests, max_tokens=self.max_tokens,
-                        max_table_blocks=self.max_table_blocks, max_free=self.max_free)
-            caps.update(ctx_capacity or {})     # a context smaller than the buffers (capacity tests)
-            self.ctx = vt.vtoken_create(w.num_layers, w.num_blocks, w.block_size, w.num_kv_heads, w.head_dim,
-                                        self.k_pool, self.v_pool, caps["max_requests"], caps["max_tokens"],
-                                        caps["max_table_blocks"], caps["max_free"], elem_bytes=w.elem_bytes,
-                                        max_ctas=max_ctas, copy_variant=copy_variant)
+            self._caps = dict(max_requests=self.max_requests, max_tokens=self.max_tokens,
+                              max_table_blocks=self.max_table_blocks, max_free=self.max_free)
+            self._caps.update(ctx_capacity or {})     # a context smaller than the buffers (capacity tests)
+            self.ctx = self.make_ctx(max_ctas=max_ctas, copy_variant=copy_variant, **ctx_options)
+
+    def make_ctx(self, **options):
+        """A (further) library context over this problem's pools; the caller destroys it."""
+        w, caps = self.w, self._caps
+        return vt.vtoken_create(w.num_layers, w.num_blocks, w.block_size, w.num_kv_heads, w.head_dim,
+                                self.k_pool, self.v_pool, caps["max_requests"], caps["max_tokens"],
+                                caps["max_table_blocks"], caps["max_free"], elem_bytes=w.elem_bytes, **options)
 
     def _padded(self, a, dtype, n):
         out = torch.zeros(max(1, n), dtype=torch.from_numpy(np.zeros(1, dtype)).dtype, device=self.device)
@@ -104,8 +110,8 @@ class DeviceProblem:
         return int(bad.item())
 
     # ---- the path -----------------------------------------------------------------------
-    def plan(self, stream=None, num_free=None):
-        vt.vtoken_plan(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
+    def plan(self, stream=None, num_free=None, ctx=None):
+        vt.vtoken_plan(ctx or self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
                        bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots, keep=self.keep,
                        free_blocks=self.free_blocks, num_free=self.num_free if num_free is None else num_free,
                        new_bt_offsets=self.new_bt_offsets, new_bt_blocks=self.new_bt_blocks,
@@ -114,8 +120,8 @@ class DeviceProblem:
                        stream=stream)
 
     def plan_partial(self, stream=None, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
-                     detach=(0, 0)):
-        vt.vtoken_plan_partial(self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
+                     detach=(0, 0), ctx=None):
+        vt.vtoken_plan_partial(ctx or self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
                                bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
                                keep=self.keep, free_blocks=self.free_blocks,
                                num_free=self.num_free if num_free is None else num_free,
@@ -126,8 +132,8 @@ class DeviceProblem:
                                max_source_blocks=max_source_blocks, theta=theta, detach=detach,
                                released_blocks=self.released_blocks, stream=stream)
 
-    def repack(self, stream=None):
-        vt.vtoken_repack(self.ctx, stream=stream)
+    def repack(self, stream=None, ctx=None):
+        vt.vtoken_repack(ctx or self.ctx, stream=stream)
 
     def repack_waves(self, num_waves: int, num_free=None, partial=None, stream=None):
         """Plan + copy + commit, ``num_waves`` times, reclaimed blocks feeding the next wave.  Needs

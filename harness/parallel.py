@@ -25,8 +25,8 @@ class Ranks:
         local = int(os.environ.get("LOCAL_RANK", str(rank)))
         if expected_world is not None and expected_world != world:
             if world == 1 and expected_world > 1:
-                raise RuntimeError(f"--gpus {expected_world} needs a torchrun launch with {expected_world} ranks "
-                                   "(WORLD_SIZE is 1)")
+                raise RuntimeError(f"--gpus {expected_world} needs {expected_world} ranks (WORLD_SIZE is unset or 1): "
+                                   "launch through torchrun, or let bench.py start its own ranks")
             raise RuntimeError(f"--gpus {expected_world} does not match WORLD_SIZE={world}")
         return cls(rank=rank, local_rank=local, world=world)
 

@@ -38,31 +38,16 @@
  * error: the request gets status VTOKEN_DEFERRED_NO_FREE (Sec. 3.3.2).
  *
  * Bounded waits: the only waits inside the kernels are on shared-memory barriers that the
- * kernel's own bulk copies complete.  Each is bounded (default 2 s, VTOKEN_WAIT_LIMIT_MS in the
- * environment at vtoken_create changes it): when it runs out the warp sets VTOKEN_FLAG_TIMEOUT,
- * gives its copies in flight a bounded time to land and returns, so the kernel always ends and
- * the context stays usable; rows of the item it was waiting for are missing.
+ * kernel's own bulk copies complete.  Each is bounded (default 2 s, vtoken_config.wait_limit_ms
+ * changes it): when it runs out the warp sets VTOKEN_FLAG_TIMEOUT, gives its copies in flight a
+ * bounded time to land and returns, so the kernel always ends and the context stays usable.  Rows
+ * may then be missing: those of the item the warp was waiting for, of the items already in its
+ * ring, of the rest of its ticket and of the ticket it had requested ahead.
  *
  * Threads: a context is not thread-safe.  Calls on one context must come from one thread at a
  * time; different contexts (different pools) are independent.
  *
- * Environment knobs, read once in vtoken_create (tuning and tests; defaults are the measured best):
- *   VTOKEN_COPY_VARIANT  1 register path, 2 bulk-copy path (only when cfg.copy_variant == 0)
- *   VTOKEN_COPY_CTAS     grid size of the copy kernel
- *   VTOKEN_BULK_TUNE     "warps,stages,rows,depth,ahead": warps per CTA, ring size, rows per work item,
- *                        items loading ahead of the one being stored, plan entries fetched ahead (1 or 2)
- *   VTOKEN_COPY_DYNAMIC  0: every warp of the copy kernel gets a fixed share of the work items; 1 (default):
- *                        warps take items from a ticket counter, VTOKEN_COPY_CHUNK (default 4) at a time
- *   VTOKEN_WAIT_LIMIT_MS bound of in-kernel waits (1 .. 60000, default 2000)
- *   VTOKEN_TEST_STALL_ITEM  test hook: index of one work item whose barrier is armed with bytes that never
- *                        arrive, so that its wait runs out (exercises the time-out path; never set in production)
- * and one read at every launch:
- *   VTOKEN_PDL           0: plain stream-ordered launches; 1 (default): every kernel of the library is launched
- *                        with programmatic stream serialization, i.e. it may become resident while the previous
- *                        kernel in the stream is finishing and waits (griddepcontrol.wait, first thing it does)
- *                        until that kernel has completed and its writes are visible.  Results are identical;
- *                        a chain of short kernels (planner, waves, slot mapping) loses about 1 us per boundary.
- *                        A caller's own kernel that follows in the stream is ordered as usual.
+ * No environment variable is read: every knob is a field of vtoken_config.
  *
  * Preconditions assumed (not checked) on the fast path: each live slot is referenced by one
  * token only (I2) and lies in a block of its own request; block ids are unique across block
@@ -109,8 +94,23 @@ enum {
     VTOKEN_FLAG_TIMEOUT = 16u,        /* a bounded wait inside a kernel ran out; rows may be missing */
     VTOKEN_FLAG_GATHER_OVERFLOW = 32u,/* gather_logical / build_slot_mapping: more live tokens than the output holds */
     VTOKEN_FLAG_BAD_VICTIM = 64u,     /* vtoken_evict_tokens: a victim outside its request's registered tokens: skipped */
-    VTOKEN_FLAG_APPEND_STOPPED = 128u /* vtoken_sync_new_tokens: table capacity or block list exhausted: request grew less */
+    VTOKEN_FLAG_APPEND_STOPPED = 128u,/* vtoken_sync_new_tokens: table capacity or block list exhausted: request grew less */
+    VTOKEN_FLAG_CHECK_FAILED = 256u   /* checked build only: an index into scratch, a table or a pool fell outside its
+                                         range; the access was skipped */
 };
+
+/* Launch shape of the bulk-copy kernel (tuning and tests; the defaults are the measured best).
+ * With enabled == 0 every field is ignored.  With enabled != 0: warps per CTA (0 => 8, at most 16),
+ * ring stages per warp (0 => 6, 2 .. 12), rows per work item (0 => 4 KiB worth; rounded down to a
+ * power of two that divides the block size, at most 32), work items loading ahead of the one being
+ * stored (0 .. stages - 2), plan entries fetched ahead (1 or 2), fixed_shares != 0: every warp gets a
+ * fixed share of the work items instead of taking them from a ticket counter, chunk = items per
+ * ticket (0 => one ticket per >= 16 KiB, at least 4 items), ctas = grid size (0 => auto). */
+typedef struct {
+    int32_t enabled;
+    int32_t warps, stages, rows, depth, ahead;
+    int32_t fixed_shares, chunk, ctas;
+} vtoken_copy_tuning;
 
 typedef struct {
     int32_t num_layers, num_blocks, block_size, num_kv_heads, head_dim;
@@ -124,6 +124,26 @@ typedef struct {
     int32_t max_ctas;              /* copy-kernel grid cap (co-residency with other work); 0 => auto */
     int32_t copy_variant;          /* 0 auto (bulk-copy path when row_bytes <= 32768, else register path);
                                       1 register path; 2 bulk-copy (TMA) path */
+    int32_t coresident;            /* 0: the copy kernel takes the whole GPU (one CTA per SM with 192 KiB of
+                                      shared-memory rings) -- the shape for a repack that runs alone, e.g. after the
+                                      step's forward has returned (Sec. 3.3.4).  1: the shape for a repack that
+                                      overlaps a decode kernel (the overlapped operation Sec. 5 measures as a
+                                      stress test): smaller rings, so that the other kernel's CTAs keep most of
+                                      every SM's shared memory and the two share HBM bandwidth instead of the
+                                      repack starving or being starved */
+    int32_t wait_limit_ms;         /* bound of every wait inside a kernel, 1 .. 60000; 0 => 2000 */
+    int32_t plain_launches;        /* 0: every kernel of the library is launched with programmatic stream
+                                      serialization, i.e. it may become resident while the previous kernel in the
+                                      stream is finishing and waits (griddepcontrol.wait, first thing it does) until
+                                      that kernel has completed and its writes are visible; a chain of short
+                                      kernels loses about 1 us per boundary, results are identical, and a caller's
+                                      own kernel that follows in the stream is ordered as usual.  1: plain
+                                      stream-ordered launches */
+    vtoken_copy_tuning tuning;     /* see above; all zero => defaults */
+    int64_t debug_stall_item;      /* must be 0 for the production library (VTOKEN_EINVAL otherwise).  The checked
+                                      build (libvtoken_checked.so) arms the barrier of work item
+                                      debug_stall_item - 1 of the copy kernel with bytes that never arrive, so that
+                                      its wait runs out: the time-out path is exercised without faulting anything */
 } vtoken_config;
 
 /* row_bytes = num_kv_heads * head_dim * elem_bytes must be a multiple of 16, pools and
@@ -194,8 +214,11 @@ int vtoken_repack(vtoken_ctx *ctx, void *cuda_stream);
  *                   (the layer stride is out_capacity_tokens rows whatever the live count)
  *   out_offsets   : DEVICE int32 [R+1], first output row of each request (unselected: empty)
  * Tokens beyond out_capacity_tokens are dropped and VTOKEN_FLAG_GATHER_OVERFLOW is set in the
- * context's flags (see vtoken_read_counts).  Uses the context's scratch: do not overlap with
- * a plan/repack in flight on another stream. */
+ * context's flags (see vtoken_read_counts).  The gather family -- this call, vtoken_digest_logical
+ * and vtoken_build_slot_mapping -- has scratch of its own: such a call may overlap a plan / repack
+ * in flight on another stream (the slot mapping is built every decode step on the compute stream
+ * while relocation runs beside it, Sec. 3.3.4), but two calls of the family must not overlap each
+ * other. */
 int vtoken_gather_logical(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                           const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
                           int32_t layer_begin, int32_t layer_end, void *out_k, void *out_v,
@@ -223,15 +246,17 @@ int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_requests, const in
                           int32_t layer_begin, int32_t layer_end, uint64_t *out_digest, int32_t *out_offsets,
                           void *cuda_stream);
 
-/* Copies the context's counts of the last plan (with the flags raised by repack and
- * gather_logical since) to HOST memory.  Synchronises the stream: the only call that does. */
+/* Copies the context's counts of the last plan (with the flags its repack raised) to HOST memory.
+ * Flags raised since the previous vtoken_read_counts by the calls outside plan / repack (logical
+ * gather, digest, slot mapping, token-table runtime, slot cache) are OR-ed in and reported once.
+ * Synchronises the stream: the only call that does. */
 int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stream);
 
 /* ---- Eligibility metadata and partial plans (Sec. 3.3.1 - 3.3.3) --------------------------------
  * The paper's reclamation backend keeps per-block liveness n_b (live tokens stored in block b),
  * derives the intra-block waste ratio F = 1 - sum(n_b) / (N * S) over the N allocated blocks
  * (Sec. 2.3.1), attempts reclamation only when F exceeds a threshold theta_F (default 0.25,
- * Sec. 3.3.2), and plans per request over "eligible low-utilization source blocks", at most B of
+ * Sec. 3.3.2), and plans per request over its under-utilised, unprotected blocks, at most B of
  * them, admitting a plan only when those sources release more blocks than the ceil(T_live / S)
  * destinations they need (Sec. 3.3.3).  Shared-prefix blocks are excluded from plans (I4). */
 
@@ -265,8 +290,8 @@ typedef struct {
  * not hold every request is VTOKEN_NOT_SELECTED.  With all options zero / NULL the result equals
  * vtoken_plan's.  vtoken_repack executes the plan.
  *
- * Copy-on-write detach (the paper's outlook for shared-prefix blocks, Sec. 5 and Sec. 6: copy-on-write
- * "when the expected reclamation benefit justifies the extra copy").  With a protect mask and
+ * Copy-on-write detach (the paper's outlook for shared-prefix blocks, Sec. 5 and Sec. 6: copying a
+ * request's tokens out of shared blocks once the blocks it gets back outweigh the copy).  With a protect mask and
  * detach_den != 0, a request whose own live tokens occupy less than detach_num / detach_den of its
  * protected blocks treats all of them as sources too: its live tokens there are COPIED to its
  * destinations with the rest (the shared blocks keep their bytes for the other holders), the blocks
@@ -345,7 +370,9 @@ int vtoken_evict_tokens(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max
  * tokens (unchanged when new_len[r] <= tt_len[r]).  New tokens get sequential logical ids; the
  * i-th new one sits at position p = phys_len[r] + i of the block list bt_blocks[bt_offsets[r] ..):
  * slot = block[p / S] * S + p % S, keep = 1.  Growth stops at the table capacity or at the end of
- * the block list (VTOKEN_FLAG_APPEND_STOPPED).  Updates tt_len and phys_len. */
+ * the block list (VTOKEN_FLAG_APPEND_STOPPED).  A token whose block id lies outside [0, num_blocks)
+ * is registered without a physical copy (slot -1, keep 0; VTOKEN_FLAG_BAD_BLOCK).  Updates tt_len
+ * and phys_len. */
 int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                            int32_t *tt_slots, uint8_t *keep, int32_t *tt_len, int32_t *phys_len,
                            const int32_t *bt_offsets, const int32_t *bt_blocks, const int32_t *new_len,
@@ -375,8 +402,8 @@ int vtoken_sync_new_tokens_counted(vtoken_ctx *ctx, const int32_t *num_requests,
  * out_slots[out_capacity]; out_token_ids (may be NULL) receives their logical ids; out_offsets[R+1]
  * the first entry of each request.  Entries beyond out_capacity are dropped
  * (VTOKEN_FLAG_GATHER_OVERFLOW).  The buffers are stable, only their contents change between
- * calls -- the property the paper relies on for CUDA-Graph replay.  Shares the context scratch of
- * vtoken_gather_logical. */
+ * calls -- the property the paper relies on for CUDA-Graph replay.  Shares the scratch of the gather
+ * family (see vtoken_gather_logical): it may overlap a plan / repack on another stream. */
 int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                               const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
                               int32_t *out_slots, int32_t *out_token_ids, int64_t out_capacity,
@@ -510,6 +537,7 @@ int vtoken_last_cuda_error(const vtoken_ctx *ctx);       /* cudaError_t of the l
 int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int32_t *smem_bytes,
                      int32_t *variant);                   /* launch shape of the copy kernel */
 int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx);      /* device scratch held by the context */
+int vtoken_checked_build(void);                           /* 1: this library was compiled with VTOKEN_CHECKED */
 
 #ifdef __cplusplus
 }

@@ -11,11 +11,12 @@ import os
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvtoken.so")
+CHECKED_LIB_PATH = os.path.join(_PKG, "libvtoken_checked.so")     # same ABI, every index range-checked
 
 OK, EINVAL, ECAPACITY, ECUDA, ENOMEM, ESTATE = 0, -1, -2, -3, -4, -5
 NOT_SELECTED, REPACKED, NO_GAIN, DEFERRED_NO_FREE = 0, 1, 2, 3
 FLAG_BAD_SLOT, FLAG_BAD_BLOCK, FLAG_BAD_FREE, FLAG_CAPACITY, FLAG_TIMEOUT, FLAG_GATHER_OVERFLOW = 1, 2, 4, 8, 16, 32
-FLAG_BAD_VICTIM, FLAG_APPEND_STOPPED = 64, 128
+FLAG_BAD_VICTIM, FLAG_APPEND_STOPPED, FLAG_CHECK_FAILED = 64, 128, 256
 
 SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "vtoken_gather_logical",
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
@@ -24,7 +25,7 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
            "vtoken_slot_cache_update", "vtoken_repack_host_partial", "vtoken_check_tables",
-           "vtoken_evict_tokens_counted", "vtoken_sync_new_tokens_counted"]
+           "vtoken_evict_tokens_counted", "vtoken_sync_new_tokens_counted", "vtoken_checked_build"]
 
 
 class VtokenError(RuntimeError):
@@ -37,6 +38,12 @@ class VtokenError(RuntimeError):
         super().__init__(msg)
 
 
+class CopyTuning(ctypes.Structure):
+    _fields_ = [("enabled", ctypes.c_int32), ("warps", ctypes.c_int32), ("stages", ctypes.c_int32),
+                ("rows", ctypes.c_int32), ("depth", ctypes.c_int32), ("ahead", ctypes.c_int32),
+                ("fixed_shares", ctypes.c_int32), ("chunk", ctypes.c_int32), ("ctas", ctypes.c_int32)]
+
+
 class Config(ctypes.Structure):
     _fields_ = [("num_layers", ctypes.c_int32), ("num_blocks", ctypes.c_int32), ("block_size", ctypes.c_int32),
                 ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32), ("elem_bytes", ctypes.c_int32),
@@ -44,7 +51,8 @@ class Config(ctypes.Structure):
                 ("layer_stride_bytes", ctypes.c_int64), ("max_requests", ctypes.c_int32),
                 ("max_tokens", ctypes.c_int64), ("max_table_blocks", ctypes.c_int64),
                 ("max_free_blocks", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
-                ("copy_variant", ctypes.c_int32)]
+                ("copy_variant", ctypes.c_int32), ("coresident", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
+                ("plain_launches", ctypes.c_int32), ("tuning", CopyTuning), ("debug_stall_item", ctypes.c_int64)]
 
 
 class PlanIn(ctypes.Structure):
@@ -96,6 +104,8 @@ class HostTables(ctypes.Structure):
 
 
 _lib = None
+_libs = {}
+_flavour = "production"
 
 
 def _build_if_needed():
@@ -115,10 +125,14 @@ def load():
     global _lib
     if _lib is None:
         _build_if_needed()
-        if not os.path.exists(LIB_PATH):
-            raise ImportError(f"{LIB_PATH} is missing: run `python -m paper_2608_13263_b200.build` "
+        path = LIB_PATH if _flavour == "production" else CHECKED_LIB_PATH
+        if not os.path.exists(path):
+            raise ImportError(f"{path} is missing: run `python -m paper_2608_13263_b200.build` "
                               "(needs nvcc); this package has no CPU fallback")
-        lib = ctypes.CDLL(LIB_PATH)
+        if path in _libs:
+            _lib = _libs[path]
+            return _lib
+        lib = ctypes.CDLL(path)
         lib.vtoken_create.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(ctypes.c_void_p)]
         lib.vtoken_destroy.argtypes = [ctypes.c_void_p]
         lib.vtoken_destroy.restype = None
@@ -162,8 +176,24 @@ def load():
         lib.vtoken_slot_cache_mark.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32] + \
                                               [ctypes.c_void_p] * 4
         lib.vtoken_slot_cache_update.argtypes = [ctypes.c_void_p] * 13
+        lib.vtoken_checked_build.argtypes = []
+        _libs[path] = lib
         _lib = lib
     return _lib
+
+
+def use_library(flavour: str) -> str:
+    """Selects the build every later call of this module goes to: "production" (libvtoken.so) or
+    "checked" (libvtoken_checked.so: the same sources compiled with -DVTOKEN_CHECKED, every index
+    into scratch, tables and pools range-checked, an out-of-range access skipped and reported as
+    VTOKEN_FLAG_CHECK_FAILED).  Returns the previous flavour.  Contexts belong to the library that
+    created them: destroy them before switching."""
+    global _lib, _flavour
+    if flavour not in ("production", "checked"):
+        raise ValueError(flavour)
+    prev, _flavour = _flavour, flavour
+    _lib = None
+    return prev
 
 
 def _ptr(x):
@@ -198,10 +228,19 @@ def _check(rc, where, ctx=None):
 
 def vtoken_create(num_layers, num_blocks, block_size, num_kv_heads, head_dim, k_pool, v_pool, max_requests,
                   max_tokens, max_table_blocks, max_free_blocks, elem_bytes=2, layer_stride_bytes=0, max_ctas=0,
-                  copy_variant=0) -> int:
+                  copy_variant=0, coresident=0, wait_limit_ms=0, plain_launches=0, tuning=None,
+                  debug_stall_item=0) -> int:
+    """``tuning``: dict with any of warps, stages, rows, depth, ahead, fixed_shares, chunk, ctas (the fields of
+    vtoken_copy_tuning; giving it sets ``enabled``)."""
+    t = CopyTuning()
+    if tuning:
+        t.enabled = 1
+        t.depth, t.ahead = 2, 2                   # the defaults of the two fields whose zero means something
+        for k, v in tuning.items():
+            setattr(t, k, int(v))
     cfg = Config(num_layers, num_blocks, block_size, num_kv_heads, head_dim, elem_bytes, _ptr(k_pool), _ptr(v_pool),
                  layer_stride_bytes, max_requests, max_tokens, max_table_blocks, max_free_blocks, max_ctas,
-                 copy_variant)
+                 copy_variant, coresident, wait_limit_ms, plain_launches, t, debug_stall_item)
     ctx = ctypes.c_void_p()
     _check(load().vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)), "vtoken_create")
     return ctx.value
@@ -281,6 +320,10 @@ def vtoken_copy_grid(ctx) -> dict:
     v = [ctypes.c_int32() for _ in range(4)]
     _check(load().vtoken_copy_grid(ctx, *[ctypes.byref(x) for x in v]), "vtoken_copy_grid")
     return dict(ctas=v[0].value, threads=v[1].value, smem_bytes=v[2].value, variant=v[3].value)
+
+
+def vtoken_checked_build() -> int:
+    return int(load().vtoken_checked_build())
 
 
 def vtoken_scratch_bytes(ctx) -> int:

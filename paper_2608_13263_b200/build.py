@@ -1,6 +1,9 @@
 """Builds the CUDA library in-tree with nvcc for sm_100a:
 
   libvtoken.so          the repack library (C ABI of include/vtoken.h)
+  libvtoken_checked.so  the same sources with -DVTOKEN_CHECKED: every index into scratch, tables and pools
+                        range-checked (an out-of-range access is skipped and flagged, never a fault), and the
+                        stall hook of the time-out test; used by the tests in place of a memory sanitizer
 
 ``python -m paper_2608_13263_b200.build`` rebuilds when a source is newer than its library.
 """
@@ -17,6 +20,7 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 
 LIB = os.path.join(PKG, "libvtoken.so")
+CHECKED_LIB = os.path.join(PKG, "libvtoken_checked.so")
 
 LIB_SOURCES = ["api.cu", "plan.cu", "copy.cu", "gather.cu", "gather_static.cu", "runtime.cu", "plan_partial.cu",
                "waves.cu", "slot_cache.cu", "check.cu"]
@@ -54,6 +58,8 @@ def _build(lib: str, sources, verbose: bool, extra=()) -> None:
 def build(force: bool = False, verbose: bool = False) -> None:
     if force or _stale(LIB, LIB_SOURCES):
         _build(LIB, LIB_SOURCES, verbose)
+    if force or _stale(CHECKED_LIB, LIB_SOURCES):
+        _build(CHECKED_LIB, LIB_SOURCES, verbose, extra=["-DVTOKEN_CHECKED"])
 
 
 if __name__ == "__main__":

@@ -24,8 +24,8 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
-                    ctx->dst_blocks, ctx->counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
-                    ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->part_shared, ctx->req_shared, ctx->req_detach,
+                    ctx->dst_blocks, ctx->counts, ctx->rt_counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
+                    ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->g_tile_n, ctx->g_req_part, ctx->g_req_before, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
                     ctx->stage.num_requests, ctx->stage.bt_blocks,
                     ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
@@ -83,12 +83,6 @@ int ensure_stage(vtoken_ctx *ctx)
 
 }  // namespace
 
-bool vtk_dependent_launch_enabled()
-{
-    const char *e = getenv("VTOKEN_PDL");      // read at every launch: a test can switch it between calls
-    return e == nullptr || atoi(e) != 0;
-}
-
 extern "C" {
 
 int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
@@ -97,7 +91,8 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     *out_ctx = nullptr;
     if (cfg->num_layers < 1 || cfg->num_blocks < 1 || cfg->block_size < 1 || cfg->num_kv_heads < 1 ||
         cfg->head_dim < 1 || cfg->elem_bytes < 1 || !cfg->k_pool || !cfg->v_pool || cfg->max_requests < 1 ||
-        cfg->max_tokens < 1 || cfg->max_table_blocks < 1 || cfg->max_free_blocks < 0 || cfg->max_ctas < 0)
+        cfg->max_tokens < 1 || cfg->max_table_blocks < 1 || cfg->max_free_blocks < 0 || cfg->max_ctas < 0 ||
+        cfg->debug_stall_item < 0)
         return VTOKEN_EINVAL;
     const int64_t row_bytes = (int64_t)cfg->num_kv_heads * cfg->head_dim * cfg->elem_bytes;
     const int64_t slots = (int64_t)cfg->num_blocks * cfg->block_size;
@@ -136,11 +131,16 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->dst_src, cap * cfg->block_size);
     A(&ctx->dst_blocks, cap);
     A(&ctx->counts, 1);
+    A(&ctx->rt_counts, 1);
+    if (rc == VTOKEN_OK && cudaMemset(ctx->rt_counts, 0, sizeof(vtoken_counts)) != cudaSuccess) rc = VTOKEN_ECUDA;
     A(&ctx->g_src, cfg->max_tokens);
     A(&ctx->g_total, 1);
     A(&ctx->g_ids, cfg->max_tokens);
     A(&ctx->g_req, cfg->max_tokens);
     A(&ctx->g_offsets, (int64_t)cfg->max_requests + 1);
+    A(&ctx->g_tile_n, (cfg->max_tokens + 1023) / 1024 + 1);
+    A(&ctx->g_req_part, (int64_t)cfg->max_requests + 1);
+    A(&ctx->g_req_before, (int64_t)cfg->max_requests + 1);
     A(&ctx->tile_mov, (cfg->max_tokens + 1023) / 1024 + 1);
     A(&ctx->tile_shared, (cfg->max_tokens + 1023) / 1024 + 1);
     A(&ctx->part_mov, (int64_t)cfg->max_requests + 1);
@@ -209,8 +209,12 @@ int vtoken_read_counts(vtoken_ctx *ctx, vtoken_counts *host_out, void *cuda_stre
 {
     if (!ctx || !host_out) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint32_t rt_flags = 0;
     VTK_CUDA(ctx, cudaMemcpyAsync(host_out, ctx->counts, sizeof(vtoken_counts), cudaMemcpyDeviceToHost, st));
+    VTK_CUDA(ctx, cudaMemcpyAsync(&rt_flags, &ctx->rt_counts->error_flags, sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    VTK_CUDA(ctx, cudaMemsetAsync(&ctx->rt_counts->error_flags, 0, sizeof(uint32_t), st));   // reported once
     VTK_CUDA(ctx, cudaStreamSynchronize(st));
+    host_out->error_flags |= rt_flags;
     return VTOKEN_OK;
 }
 
@@ -219,6 +223,7 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
 {
     if (!ctx || !h) return VTOKEN_EINVAL;
     if (opts && opts->max_source_blocks < 0) return VTOKEN_EINVAL;
+    if (opts && opts->detach_den != 0) return VTOKEN_EINVAL;    // the host front end has no released list
     if (!h->bt_offsets || !h->bt_blocks || !h->tt_offsets || !h->tt_slots || !h->keep || !h->free_blocks ||
         !h->new_bt_offsets || !h->new_bt_blocks || !h->new_tt_slots || !h->freed_blocks || !h->req_status ||
         !h->counts)
@@ -277,7 +282,6 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
     out.req_status = s.req_status;
     out.counts = s.counts;
     out.released_blocks = nullptr;
-    if (opts && opts->detach_den != 0) return VTOKEN_EINVAL;    // the host front end has no released list
     if (opts) {
         vtoken_partial_opts dopts = *opts;
         dopts.protect = opts->protect ? s.protect : nullptr;
@@ -350,5 +354,14 @@ int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int
 }
 
 int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx) { return ctx ? ctx->scratch_bytes : 0; }
+
+int vtoken_checked_build(void)
+{
+#ifdef VTOKEN_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 }  // extern "C"

@@ -29,7 +29,11 @@ struct vtoken_ctx {
     int32_t *req_status;       // [max_requests]
     int32_t *dst_src;          // [cap_dst_blocks * S] inverse plan: source slot of each destination slot, -1 = none
     int32_t *dst_blocks;       // [cap_dst_blocks] physical id of each destination block, -1 = skip
-    vtoken_counts *counts;     // one struct
+    vtoken_counts *counts;     // one struct: counts of the last plan, flags of the plan and its copy
+    vtoken_counts *rt_counts;  // one struct, only error_flags is used: flags raised by every call outside plan / repack
+                               // (logical gather, slot mapping, digest, token-table runtime, slot cache).  Those calls
+                               // belong to the compute stream and may overlap a plan in flight on a side stream, whose
+                               // scan kernel stores `counts` as a whole
     int32_t *tile_n;           // [ceil(max_tokens / 1024) + 1] live tokens per tile of the token table, then scanned
     int32_t *req_part;         // [max_requests + 1] live tokens between a request's tile start and its first entry
     int32_t *req_before;       // [max_requests + 1] live (partial planner: moving) tokens of the table before the request's first entry
@@ -54,6 +58,9 @@ struct vtoken_ctx {
     int32_t *g_req;            // [max_tokens] request of each output row (digest)
     int32_t *g_offsets;        // [max_requests + 1] first output row of each request (digest)
     unsigned int *g_ticket;    // [2] work tickets of the gather's row copy (zero between launches)
+    int32_t *g_tile_n, *g_req_part, *g_req_before;   // like tile_n / req_part / req_before, owned by the gather family
+                                                     // (logical gather, slot mapping, digest): these calls run on the
+                                                     // compute stream while a plan may be in flight on a side stream
 
     // device staging of vtoken_repack_host (DEVICE), allocated on first use
     struct {
@@ -87,7 +94,8 @@ struct vtoken_ctx {
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
 int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st);
 int vtk_configure_copy(vtoken_ctx *ctx);
-bool vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t *g_total, int32_t layer_begin,
+// > 0: launched; 0: the context has no bulk configuration for these rows; < 0: VTOKEN_* error
+int vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t *g_total, int32_t layer_begin,
                             int32_t layer_end, void *out_k, void *out_v, int64_t out_capacity, cudaStream_t st);
 int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
                       const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select,
@@ -116,11 +124,14 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
 __device__ __forceinline__ void vtk_wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void vtk_release_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-bool vtk_dependent_launch_enabled();   // VTOKEN_PDL=0 turns the launch attribute off (the device side is then a no-op)
+// launch shape of the copy kernel when vtoken_config.coresident is set
+constexpr int VTK_CORESIDENT_WARPS = 8;
+constexpr int VTK_CORESIDENT_STAGES = 3;
 
+// cfg.plain_launches turns the launch attribute off (the device side is then a no-op)
 template <typename... P, typename... A>
-inline cudaError_t vtk_launch_dependent(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
-                                        A... args)
+inline cudaError_t vtk_launch_dependent(const vtoken_ctx *ctx, void (*kernel)(P...), dim3 grid, dim3 block, size_t smem,
+                                        cudaStream_t st, A... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -131,7 +142,7 @@ inline cudaError_t vtk_launch_dependent(void (*kernel)(P...), dim3 grid, dim3 bl
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = vtk_dependent_launch_enabled() ? 1 : 0;
+    cfg.numAttrs = ctx->cfg.plain_launches ? 0 : 1;
     return cudaLaunchKernelEx(&cfg, kernel, P(args)...);
 }
 

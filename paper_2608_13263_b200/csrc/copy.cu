@@ -16,8 +16,6 @@
 //                   contiguous destination range.  Every wait is bounded.
 #include "common.cuh"
 
-#include <cstdio>
-#include <cstdlib>
 
 namespace {
 
@@ -394,14 +392,23 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
 int vtk_configure_copy(vtoken_ctx *ctx)
 {
     const int S = ctx->cfg.block_size;
+    const vtoken_copy_tuning &tune = ctx->cfg.tuning;
+    const bool tuned = tune.enabled != 0;
     int variant = ctx->cfg.copy_variant;
-    if (const char *e = getenv("VTOKEN_COPY_VARIANT")) { if (variant == 0) variant = atoi(e); }
     // bulk copies need 16-byte multiples (checked at create) and a row that fits a stage.  Small rows
     // belong on the bulk path too: the register path spends a warp per row whatever its size (measured
     // on B200 with 256 / 128 / 64 / 16-byte rows: 2.0 / 1.0 / 0.5 / 0.14 TB/s against 6.1 / 4.6 / 2.6 /
     // 0.3 TB/s through the rings, where an item is up to 32 rows)
     if (variant == 0) variant = ctx->row_bytes <= 32768 ? 2 : 1;
     if (variant != 1 && variant != 2) return VTOKEN_EINVAL;
+    if (ctx->cfg.wait_limit_ms < 0 || ctx->cfg.wait_limit_ms > 60000) return VTOKEN_EINVAL;
+    ctx->wait_limit_ns = ctx->cfg.wait_limit_ms ? (int64_t)ctx->cfg.wait_limit_ms * 1000000ll : 2000000000ll;
+    ctx->stall_item = -1;
+#ifdef VTOKEN_CHECKED
+    if (ctx->cfg.debug_stall_item > 0) ctx->stall_item = ctx->cfg.debug_stall_item - 1;
+#else
+    if (ctx->cfg.debug_stall_item != 0) return VTOKEN_EINVAL;      // the hook exists in the checked build only
+#endif
 
     int ctas_per_sm;
     if (variant == 1) {
@@ -409,18 +416,22 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctx->copy_smem = 0;
         ctas_per_sm = 8;
     } else {
-        // tuning knobs "warps,stages,rows,depth,ahead": warps per CTA, ring size, rows per item, loads
-        // issued ahead, plan entries fetched ahead.  Defaults: 8 warps x 6 stages x 4 KB items = 192 KB of staging per SM, two
-        // items loading ahead, three stores in flight per warp.  Measured on B200: shapes from 4 to
-        // 32 KB per item land within about 3 % of each other; below 4 KB per warp-step with only
-        // 8 warps per SM the pipeline becomes issue-bound.
+        // Launch shape: warps per CTA, ring stages per warp, rows per item, items loading ahead of the one
+        // being stored, plan entries fetched ahead.  Default: 8 warps x 6 stages x 4 KiB items = 192 KiB of
+        // staging per SM, two items loading ahead, three stores in flight per warp.  Measured on B200:
+        // shapes from 4 to 32 KiB per item land within about 3 % of each other; below 4 KiB per warp-step
+        // with only 8 warps per SM the pipeline becomes issue-bound.  The co-resident shape leaves most of
+        // the SM's shared memory to a kernel running beside the repack (see vtoken.h).
         int warps = 8, stages = 6, rows = 0, depth = 2, ahead = 2;
-        if (const char *e = getenv("VTOKEN_BULK_TUNE")) sscanf(e, "%d,%d,%d,%d,%d", &warps, &stages, &rows, &depth, &ahead);
+        if (ctx->cfg.coresident) { warps = VTK_CORESIDENT_WARPS; stages = VTK_CORESIDENT_STAGES; }
+        if (tuned) {
+            if (tune.warps > 0) warps = tune.warps;
+            if (tune.stages > 0) stages = tune.stages;
+            rows = tune.rows;
+            depth = tune.depth;
+            ahead = tune.ahead;
+        }
         ctx->bulk_ahead = ahead == 1 ? 1 : 2;
-        ctx->wait_limit_ns = 2000000000ll;
-        if (const char *e = getenv("VTOKEN_WAIT_LIMIT_MS")) { long v = atol(e); if (v >= 1 && v <= 60000) ctx->wait_limit_ns = v * 1000000ll; }
-        ctx->stall_item = -1;
-        if (const char *e = getenv("VTOKEN_TEST_STALL_ITEM")) ctx->stall_item = atoll(e);
         if (rows <= 0) rows = (int)(4096 / ctx->row_bytes);
         // an item is `rows` consecutive destination slots inside one block: a power of two
         // (<= 32, one row per lane) that divides the block size
@@ -447,12 +458,12 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctx->bulk_rows = rows;
         ctx->copy_threads = warps * 32;
         ctx->copy_smem = (int)smem;
-        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_MAX_SMEM));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_MAX_SMEM));
+        VTK_CUDA(ctx, cudaFuncSetAttribute(copy_bulk_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BULK_MAX_SMEM));
         // tickets are 32-bit: every item of a launch must have an index below 2^31
         ctx->copy_dynamic = (int64_t)ctx->cap_dst_blocks * (S / rows) * 2 * ctx->cfg.num_layers < (int64_t)INT32_MAX;
-        if (const char *e = getenv("VTOKEN_COPY_DYNAMIC")) ctx->copy_dynamic = ctx->copy_dynamic && atoi(e) != 0;
+        if (tuned && tune.fixed_shares) ctx->copy_dynamic = false;
         // one ticket per >= 16 KiB of destination bytes and never fewer than 4 items: measured on B200, one
         // ticket per 8 KiB already runs into the throughput of atomics on one address (4.5 instead of 6.7 TB/s)
         {
@@ -460,13 +471,14 @@ int vtk_configure_copy(vtoken_ctx *ctx)
             int64_t c = (16384 + item_bytes - 1) / item_bytes;
             ctx->copy_chunk = (int)(c < 4 ? 4 : (c > 64 ? 64 : c));
         }
-        if (const char *e = getenv("VTOKEN_COPY_CHUNK")) { int v = atoi(e); if (v >= 1 && v <= 1024) ctx->copy_chunk = v; }
+        if (tuned && tune.chunk >= 1 && tune.chunk <= 1024) ctx->copy_chunk = tune.chunk;
         ctas_per_sm = (int)((227 * 1024) / (smem + 2048));
         if (ctas_per_sm < 1) ctas_per_sm = 1;
         if (ctas_per_sm > 8) ctas_per_sm = 8;
+        if (ctx->cfg.coresident) ctas_per_sm = 1;
     }
     int ctas = ctx->num_sms * ctas_per_sm;
-    if (const char *e = getenv("VTOKEN_COPY_CTAS")) { int v = atoi(e); if (v > 0) ctas = v; }
+    if (tuned && tune.ctas > 0) ctas = tune.ctas;
     if (ctx->cfg.max_ctas > 0 && ctas > ctx->cfg.max_ctas) ctas = ctx->cfg.max_ctas;
     ctx->copy_ctas = ctas;
     ctx->copy_variant = variant;
@@ -491,32 +503,33 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     a.ticket = ctx->copy_ticket;
     const dim3 grid(ctx->copy_ctas), block(ctx->copy_threads);
     if (ctx->copy_variant == 1)
-        VTK_CUDA(ctx, vtk_launch_dependent(copy_rows_kernel, grid, block, 0, st, a));
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, copy_rows_kernel, grid, block, 0, st, a));
     else if (ctx->copy_dynamic)
-        VTK_CUDA(ctx, vtk_launch_dependent(copy_bulk_kernel<true, false>, grid, block, (size_t)ctx->copy_smem, st, a,
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, copy_bulk_kernel<true, false>, grid, block, (size_t)ctx->copy_smem, st, a,
                                            ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, ctx->copy_chunk));
     else
-        VTK_CUDA(ctx, vtk_launch_dependent(copy_bulk_kernel<false, false>, grid, block, (size_t)ctx->copy_smem, st, a,
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, copy_bulk_kernel<false, false>, grid, block, (size_t)ctx->copy_smem, st, a,
                                            ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead, 1));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
 
-// The row copy of vtoken_gather_logical through the bulk path (false: the context has no bulk
-// configuration for these rows; the caller uses its register kernel).
-bool vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t *g_total, int32_t layer_begin,
+// The row copy of vtoken_gather_logical through the bulk path.  Returns 1 when the kernel was launched,
+// 0 when the context has no bulk configuration for these rows (the caller uses its register kernel),
+// VTOKEN_ECUDA when the launch failed (the CUDA error is kept in the context).
+int vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t *g_total, int32_t layer_begin,
                             int32_t layer_end, void *out_k, void *out_v, int64_t out_capacity, cudaStream_t st)
 {
-    if (ctx->copy_variant != 2 || !ctx->copy_dynamic || ctx->g_ticket == nullptr) return false;
+    if (ctx->copy_variant != 2 || !ctx->copy_dynamic || ctx->g_ticket == nullptr) return 0;
     // tickets are 32-bit: every item must have an index below 2^31
     const int64_t items = (ctx->cfg.max_tokens + ctx->bulk_rows - 1) / ctx->bulk_rows * 2 * (layer_end - layer_begin);
-    if (items >= (int64_t)INT32_MAX) return false;
+    if (items >= (int64_t)INT32_MAX) return 0;
     CopyArgs a;
     a.k_pool = (uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (uint8_t *)ctx->cfg.v_pool;
     a.dst_src = nullptr;
     a.dst_blocks = nullptr;
-    a.counts = ctx->counts;
+    a.counts = ctx->rt_counts;            // gather mode reads no count from it: only the time-out flag goes there
     a.layer_stride = ctx->layer_stride;
     a.row_bytes = ctx->row_bytes;
     a.S = ctx->bulk_rows;                 // parts = 1: unused in gather mode
@@ -531,9 +544,8 @@ bool vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t
     a.out_v = (uint8_t *)out_v;
     a.out_capacity = out_capacity;
     a.layer_begin = layer_begin;
-    if (vtk_launch_dependent(copy_bulk_kernel<true, true>, dim3(ctx->copy_ctas), dim3(ctx->copy_threads),
-                             (size_t)ctx->copy_smem, st, a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead,
-                             ctx->copy_chunk) != cudaSuccess)
-        ctx->last_cuda_error = (int)cudaGetLastError();      // reported by the caller's cudaGetLastError check too
-    return true;
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, copy_bulk_kernel<true, true>, dim3(ctx->copy_ctas), dim3(ctx->copy_threads),
+                                       (size_t)ctx->copy_smem, st, a, ctx->bulk_stages, ctx->bulk_depth, ctx->bulk_ahead,
+                                       ctx->copy_chunk));
+    return 1;
 }

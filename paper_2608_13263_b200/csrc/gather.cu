@@ -318,22 +318,22 @@ __global__ void __launch_bounds__(VTK_TILE_NT) gather_assign_flat_kernel(GatherA
 // count -> scan -> assign: flat tiles when the context has their scratch, else the per-request kernels
 int launch_index(vtoken_ctx *ctx, GatherArgs &a, cudaStream_t st)
 {
-    if (ctx->tile_n != nullptr) {
-        a.tile_n = ctx->tile_n;
-        a.req_part = ctx->req_part;
-        a.req_before = ctx->req_before;
+    if (ctx->g_tile_n != nullptr) {
+        a.tile_n = ctx->g_tile_n;
+        a.req_part = ctx->g_req_part;
+        a.req_before = ctx->g_req_before;
         a.num_tiles = (int32_t)((ctx->cfg.max_tokens + VTK_TILE - 1) / VTK_TILE);
         a.vec_in = ((uintptr_t)a.tt_slots % 16 == 0 && (a.keep == nullptr || (uintptr_t)a.keep % 4 == 0)) ? 1 : 0;
         a.table_cap = ctx->cfg.max_tokens;
-        VTK_CUDA(ctx, vtk_launch_dependent(gather_tiles_kernel, dim3(a.num_tiles + ctx->cfg.max_requests + 1),
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_tiles_kernel, dim3(a.num_tiles + ctx->cfg.max_requests + 1),
                                            dim3(VTK_TILE_NT), 0, st, a));
-        VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_flat_kernel, dim3(1), dim3(1024), 0, st, a));
-        VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_flat_kernel, dim3(a.num_tiles), dim3(VTK_TILE_NT), 0, st, a));
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_scan_flat_kernel, dim3(1), dim3(1024), 0, st, a));
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_assign_flat_kernel, dim3(a.num_tiles), dim3(VTK_TILE_NT), 0, st, a));
         return VTOKEN_OK;
     }
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_count_kernel, dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_assign_kernel, dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_count_kernel, dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_scan_kernel, dim3(1), dim3(1024), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_assign_kernel, dim3(ctx->cfg.max_requests * a.parts), dim3(G_NT), 0, st, a));
     return VTOKEN_OK;
 }
 
@@ -552,7 +552,7 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     a.g_req = ctx->g_req;
     a.digest = (unsigned long long *)out_digest;
     a.g_total = ctx->g_total;
-    a.counts = ctx->counts;
+    a.counts = ctx->rt_counts;
     a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (const uint8_t *)ctx->cfg.v_pool;
     a.out_k = a.out_v = nullptr;
@@ -567,7 +567,7 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     a.parts = G_PARTS;
     VTK_CUDA(ctx, cudaMemsetAsync(out_digest, 0, sizeof(uint64_t) * (size_t)ctx->cfg.max_requests, st));
     { const int rc = launch_index(ctx, a, st); if (rc != VTOKEN_OK) return rc; }
-    VTK_CUDA(ctx, vtk_launch_dependent(gather_digest_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_digest_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -591,7 +591,7 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     a.g_req = nullptr;
     a.digest = nullptr;
     a.g_total = ctx->g_total;
-    a.counts = ctx->counts;
+    a.counts = ctx->rt_counts;
     a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (const uint8_t *)ctx->cfg.v_pool;
     a.out_k = (uint8_t *)out_k;
@@ -609,9 +609,11 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
     // the rows go through the bulk-copy rings when the context has them (vtoken_create does; the
     // context-free entry point does not), else through the register kernel
     const bool aligned = (((uintptr_t)out_k | (uintptr_t)out_v) & 15) == 0;
-    if (!(aligned && vtk_launch_gather_bulk(ctx, ctx->g_src, ctx->g_total, layer_begin, layer_end, out_k, out_v,
-                                            out_capacity_tokens, st)))
-        VTK_CUDA(ctx, vtk_launch_dependent(gather_copy_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
+    const int bulk = aligned ? vtk_launch_gather_bulk(ctx, ctx->g_src, ctx->g_total, layer_begin, layer_end, out_k, out_v,
+                                                      out_capacity_tokens, st) : 0;
+    if (bulk < 0) return bulk;
+    if (bulk == 0)
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_copy_kernel, dim3(ctx->num_sms * 8), dim3(GC_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -640,7 +642,7 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     a.g_req = nullptr;
     a.digest = nullptr;
     a.g_total = ctx->g_total;
-    a.counts = ctx->counts;
+    a.counts = ctx->rt_counts;
     a.k_pool = a.v_pool = nullptr;
     a.out_k = a.out_v = nullptr;
     a.layer_stride = 0;

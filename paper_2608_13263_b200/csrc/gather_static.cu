@@ -108,6 +108,7 @@ extern "C" int vtoken_gather_logical_noalloc(const void *k_pool, const void *v_p
     ctx.slots_per_layer = slots;
     ctx.num_sms = slot->num_sms;
     ctx.counts = reinterpret_cast<vtoken_counts *>(slot->scratch + OFF_COUNTS);
+    ctx.rt_counts = ctx.counts;
     ctx.g_total = reinterpret_cast<int32_t *>(slot->scratch + OFF_TOTAL);
     ctx.part_n = reinterpret_cast<int32_t *>(slot->scratch + OFF_REQ_N);
     ctx.g_src = reinterpret_cast<int32_t *>(slot->scratch + OFF_SRC);
@@ -119,7 +120,7 @@ extern "C" int vtoken_gather_logical_noalloc(const void *k_pool, const void *v_p
                            out_v, out_capacity_tokens, out_offsets, st);
     if (rc != VTOKEN_OK) return rc;
     if (error_flags) {
-        if (cudaMemcpyAsync(error_flags, &ctx.counts->error_flags, sizeof(uint32_t), cudaMemcpyDeviceToDevice, st) !=
+        if (cudaMemcpyAsync(error_flags, &ctx.rt_counts->error_flags, sizeof(uint32_t), cudaMemcpyDeviceToDevice, st) !=
             cudaSuccess)
             return VTOKEN_ECUDA;
     }

@@ -396,9 +396,9 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.vec_out = ((uintptr_t)out->new_tt_slots % 16 == 0) ? 1 : 0;
 
     const int R = ctx->cfg.max_requests;
-    VTK_CUDA(ctx, vtk_launch_dependent(plan_tiles_kernel, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(plan_scan_kernel, dim3(1), dim3(SCAN_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(plan_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_tiles_kernel, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_scan_kernel, dim3(1), dim3(SCAN_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

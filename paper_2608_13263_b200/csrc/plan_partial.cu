@@ -712,11 +712,11 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
     // n_b and blk_src share one allocation: one node clears both
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, (sizeof(int32_t) + 1) * (size_t)ctx->cfg.num_blocks, st));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_tiles_kernel<0>, tiles_grid, dim3(TILE_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_blocks_kernel, dim3(R), dim3(PP_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_tiles_kernel<1>, tiles_grid, dim3(TILE_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_scan_kernel, dim3(1), dim3(PP_SCAN_NT), 0, st, a));
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_tiles_kernel<0>, tiles_grid, dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_blocks_kernel, dim3(R), dim3(PP_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_tiles_kernel<1>, tiles_grid, dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_scan_kernel, dim3(1), dim3(PP_SCAN_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
     ctx->has_plan = true;
     return VTOKEN_OK;
@@ -741,15 +741,15 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     const int R = ctx->cfg.max_requests;
     VTK_CUDA(ctx, cudaMemsetAsync(n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
     a.vec_in = ((uintptr_t)tt_slots % 16 == 0 && (uintptr_t)keep % 4 == 0) ? 1 : 0;
-    VTK_CUDA(ctx, vtk_launch_dependent(pp_tiles_kernel<0>, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_tiles_kernel<0>, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
     if (hist) {
         VTK_CUDA(ctx, cudaMemsetAsync(hist, 0, sizeof(uint64_t) * (size_t)(ctx->cfg.block_size + 1), st));
-        VTK_CUDA(ctx, vtk_launch_dependent(pp_hist_kernel, dim3(ctx->num_sms * 4), dim3(256), 0, st, num_requests, R,
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_hist_kernel, dim3(ctx->num_sms * 4), dim3(256), 0, st, num_requests, R,
                                            bt_offsets, bt_blocks, (const int32_t *)n_b, ctx->cfg.block_size,
                                            ctx->cfg.num_blocks, (unsigned long long *)hist, ctx->counts));
     }
     if (summary)
-        VTK_CUDA(ctx, vtk_launch_dependent(pp_summary_kernel, dim3(1), dim3(1024), 0, st, num_requests, R, bt_offsets,
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_summary_kernel, dim3(1), dim3(1024), 0, st, num_requests, R, bt_offsets,
                                            tt_offsets, ctx->cfg.max_tokens, (const int32_t *)ctx->tile_n,
                                            (long long *)summary));
     VTK_CUDA(ctx, cudaGetLastError());

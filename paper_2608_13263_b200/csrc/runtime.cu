@@ -99,10 +99,11 @@ __global__ void __launch_bounds__(RT_NT) sync_kernel(const int32_t *num_requests
     for (int i = threadIdx.x; i < (int)can; i += RT_NT) {
         const int p = phys + i;                              // position in the block list
         const int blk = bt_blocks[b0 + p / S];
-        if (blk < 0 || blk >= num_blocks) flags |= VTOKEN_FLAG_BAD_BLOCK;
-        tt_slots[base + len + i] = blk * S + p % S;          // slot = block_id * S + offset
-        keep[base + len + i] = 1;
-        if (COUNTED && blk >= 0 && blk < num_blocks) {       // one more live token in that block
+        const bool ok = blk >= 0 && blk < num_blocks;
+        if (!ok) flags |= VTOKEN_FLAG_BAD_BLOCK;             // registered without a physical copy: slot -1, not kept
+        tt_slots[base + len + i] = ok ? blk * S + p % S : -1;   // slot = block_id * S + offset
+        keep[base + len + i] = ok ? 1 : 0;
+        if (COUNTED && ok) {                                 // one more live token in that block
             atomicAdd(&lv.n_b[blk], 1);
             ++counted;
         }
@@ -194,9 +195,9 @@ int vtoken_evict_tokens(vtoken_ctx *ctx, const int32_t *num_victims, int32_t max
     if (max_victims == 0) return VTOKEN_OK;
     int grid = (max_victims + RT_NT - 1) / RT_NT;
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
-    VTK_CUDA(ctx, vtk_launch_dependent(evict_kernel<false>, dim3(grid), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, evict_kernel<false>, dim3(grid), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
                                        num_victims, max_victims, victim_req, victim_tok, num_requests,
-                                       ctx->cfg.max_requests, tt_offsets, tt_len, keep, ctx->counts, Liveness{}));
+                                       ctx->cfg.max_requests, tt_offsets, tt_len, keep, ctx->rt_counts, Liveness{}));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -214,9 +215,9 @@ int vtoken_evict_tokens_counted(vtoken_ctx *ctx, const int32_t *num_victims, int
     int grid = (max_victims + RT_NT - 1) / RT_NT;
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
     const Liveness lv{n_b, (unsigned long long *)live_total, tt_slots, ctx->slots_per_layer, ctx->cfg.block_size};
-    VTK_CUDA(ctx, vtk_launch_dependent(evict_kernel<true>, dim3(grid), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, evict_kernel<true>, dim3(grid), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
                                        num_victims, max_victims, victim_req, victim_tok, num_requests,
-                                       ctx->cfg.max_requests, tt_offsets, tt_len, keep, ctx->counts, lv));
+                                       ctx->cfg.max_requests, tt_offsets, tt_len, keep, ctx->rt_counts, lv));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -229,11 +230,11 @@ int vtoken_sync_new_tokens(vtoken_ctx *ctx, const int32_t *num_requests, const i
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !tt_len || !phys_len || !bt_offsets ||
         !bt_blocks || !new_len)
         return VTOKEN_EINVAL;
-    VTK_CUDA(ctx, vtk_launch_dependent(sync_kernel<false>,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, sync_kernel<false>,
                                        dim3(ctx->cfg.max_requests), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
                                        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots,
                                        keep, tt_len, phys_len, bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks,
-                                       ctx->counts, Liveness{}));
+                                       ctx->rt_counts, Liveness{}));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -247,11 +248,11 @@ int vtoken_sync_new_tokens_counted(vtoken_ctx *ctx, const int32_t *num_requests,
         !bt_blocks || !new_len || !n_b)
         return VTOKEN_EINVAL;
     const Liveness lv{n_b, (unsigned long long *)live_total, nullptr, ctx->slots_per_layer, ctx->cfg.block_size};
-    VTK_CUDA(ctx, vtk_launch_dependent(sync_kernel<true>,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, sync_kernel<true>,
                                        dim3(ctx->cfg.max_requests), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
                                        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots,
                                        keep, tt_len, phys_len, bt_offsets, bt_blocks, new_len, ctx->cfg.num_blocks,
-                                       ctx->counts, lv));
+                                       ctx->rt_counts, lv));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }
@@ -263,7 +264,7 @@ int vtoken_apply_moves(vtoken_ctx *ctx, const int32_t *num_requests, const int32
 {
     if (!ctx || !num_requests || !tt_offsets || !tt_slots || !keep || !new_tt_slots) return VTOKEN_EINVAL;
     if (phys_len && !req_status) return VTOKEN_EINVAL;
-    VTK_CUDA(ctx, vtk_launch_dependent(apply_moves_kernel,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, apply_moves_kernel,
                                        dim3(ctx->cfg.max_requests), dim3(RT_NT), 0, (cudaStream_t)cuda_stream,
                                        num_requests, ctx->cfg.max_requests, ctx->cfg.block_size, tt_offsets, tt_slots,
                                        keep, phys_len, new_tt_slots, req_status, new_bt_offsets, append_pos));

@@ -106,7 +106,7 @@ int vtoken_slot_cache_mark(vtoken_ctx *ctx, uint8_t *dirty, const int32_t *num_v
     const int64_t span = max_victims > ctx->cfg.max_requests ? max_victims : ctx->cfg.max_requests;
     int grid = (int)((span + 255) / 256);
     if (grid > ctx->num_sms * 8) grid = ctx->num_sms * 8;
-    VTK_CUDA(ctx, vtk_launch_dependent(slot_cache_mark_kernel, dim3(grid), dim3(256), 0, (cudaStream_t)cuda_stream,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, slot_cache_mark_kernel, dim3(grid), dim3(256), 0, (cudaStream_t)cuda_stream,
                                        dirty,
                                        max_victims > 0 ? num_victims : nullptr, max_victims,
                                        max_victims > 0 ? victim_req : nullptr, req_status, num_requests,
@@ -125,10 +125,10 @@ int vtoken_slot_cache_update(vtoken_ctx *ctx, const int32_t *num_requests, const
         return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     if (stats) VTK_CUDA(ctx, cudaMemsetAsync(stats, 0, 2 * sizeof(int32_t), st));
-    VTK_CUDA(ctx, vtk_launch_dependent(slot_cache_update_kernel,
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, slot_cache_update_kernel,
                                        dim3(ctx->cfg.max_requests), dim3(SC_NT), 0, st, num_requests,
                                        ctx->cfg.max_requests, tt_offsets, tt_slots, keep, tt_len, dirty, cache_slots,
-                                       cache_ids, cache_len, cache_seen, stats, ctx->slots_per_layer, ctx->counts));
+                                       cache_ids, cache_len, cache_seen, stats, ctx->slots_per_layer, ctx->rt_counts));
     VTK_CUDA(ctx, cudaGetLastError());
     return VTOKEN_OK;
 }

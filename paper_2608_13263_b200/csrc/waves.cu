@@ -169,7 +169,7 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         int blocks = (int)((span + COMMIT_NT - 1) / COMMIT_NT);
         if (blocks < 1) blocks = 1;
         if (blocks > ctx->num_sms * 8) blocks = ctx->num_sms * 8;
-        VTK_CUDA(ctx, vtk_launch_dependent(wave_commit_kernel, dim3(blocks), dim3(COMMIT_NT), 0, st, a));
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, wave_commit_kernel, dim3(blocks), dim3(COMMIT_NT), 0, st, a));
         VTK_CUDA(ctx, cudaGetLastError());
 
         cur.bt_offsets = po.new_bt_offsets;

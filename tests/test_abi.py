@@ -43,10 +43,10 @@ def test_strerror_and_argument_errors_without_gpu():
     # NULL arguments are rejected before any CUDA call
     assert lib.vtoken_create(None, None) == binding.EINVAL
     assert lib.vtoken_repack(None, None) == binding.EINVAL
-    cfg = binding.Config(1, 4, 16, 1, 4, 2, 256, 512, 0, 1, 16, 4, 4, 0, 0)   # row_bytes = 8: not a multiple of 16
+    cfg = binding.Config(1, 4, 16, 1, 4, 2, 256, 512, 0, 1, 16, 4, 4)   # row_bytes = 8: not a multiple of 16
     ctx = ctypes.c_void_p()
     assert lib.vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)) == binding.EINVAL
-    cfg = binding.Config(1, 4, 16, 1, 8, 2, 257, 512, 0, 1, 16, 4, 4, 0, 0)   # misaligned pool
+    cfg = binding.Config(1, 4, 16, 1, 8, 2, 257, 512, 0, 1, 16, 4, 4)   # misaligned pool
     assert lib.vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)) == binding.EINVAL
 
 
@@ -56,7 +56,8 @@ def test_header_is_plain_c_and_ctypes_layouts_match(tmp_path):
     import subprocess
     structs = {"vtoken_config": binding.Config, "vtoken_plan_in": binding.PlanIn, "vtoken_counts": binding.Counts,
                "vtoken_plan_out": binding.PlanOut, "vtoken_partial_opts": binding.PartialOpts,
-               "vtoken_host_tables": binding.HostTables, "vtoken_waves_out": binding.WavesOut}
+               "vtoken_host_tables": binding.HostTables, "vtoken_waves_out": binding.WavesOut,
+               "vtoken_copy_tuning": binding.CopyTuning}
     lines = ['#include <stddef.h>', '#include <stdio.h>', '#include "vtoken.h"', 'int main(void) {']
     for cname, cls in structs.items():
         lines.append(f'printf("{cname} %zu", sizeof({cname}));')

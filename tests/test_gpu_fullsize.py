@@ -24,16 +24,16 @@ CASES = [
 ]
 
 
-def _fit(name, kw, free_bytes):
-    """The workload at full size, or with the request count halved until the pools fit."""
-    import inspect
-    gen = wl.CONFIGS[name]
-    requests = inspect.signature(gen).parameters["requests"].default
-    while True:
-        w = gen(seed=0, requests=requests, **kw)
-        if 2 * w.pool_bytes + (3 << 30) < free_bytes or requests == 1:
-            return w, requests
-        requests //= 2
+def _full_size(name, kw, free_bytes):
+    """The workload at the size the benchmark is quoted on.  When its pools do not fit the memory
+    that is free on this (shared) GPU the test is skipped with that reason: passing on a smaller
+    problem would say nothing about the full-size claim."""
+    w = wl.CONFIGS[name](seed=0, **kw)
+    need = 2 * w.pool_bytes + (3 << 30)
+    if need >= free_bytes:
+        pytest.skip(f"{name}: pools of {2 * w.pool_bytes / 2 ** 30:.1f} GiB (+3 GiB of tables and scratch) do not fit "
+                    f"the {free_bytes / 2 ** 30:.1f} GiB free on this GPU")
+    return w
 
 
 @pytest.mark.parametrize("name,kw", CASES, ids=[f"{n}{'-S32' if k else ''}" for n, k in CASES])
@@ -42,7 +42,7 @@ def test_full_size_graph_side_stream(name, kw):
     from harness.device import DeviceProblem, origin_map
     torch.cuda.empty_cache()
     free_bytes, _ = torch.cuda.mem_get_info()
-    w, requests = _fit(name, kw, free_bytes)
+    w = _full_size(name, kw, free_bytes)
     prob = DeviceProblem(w, fill_seed=1)
     side = torch.cuda.Stream()
     side.wait_stream(torch.cuda.current_stream())
@@ -77,7 +77,7 @@ def test_full_size_graph_side_stream(name, kw):
                                w.free_blocks, out["new_bt_offsets"], out["new_bt_blocks"], out["new_tt_slots"],
                                out["freed_blocks"], out["num_free_consumed"], out["req_status"], w.select,
                                w.thr_num, w.thr_den) == 0
-    if name != "tiny" and requests == len(np.diff(w.tt_offsets)):
+    if name != "tiny":
         assert p.num_moves > 10000
 
     # (1) every word of both pools

@@ -37,11 +37,12 @@ def assert_tables_equal(out, p, w):
     assert np.array_equal(out["freed_blocks"], p.freed_blocks)
 
 
-def run_and_compare(w, copy_variant=0, num_free=None, whole_pool=True, capacity_slack=0):
+def run_and_compare(w, copy_variant=0, num_free=None, whole_pool=True, capacity_slack=0, **ctx_options):
     """plan + repack on the GPU, oracle on the host, compare everything."""
     from harness.device import DeviceProblem
     torch = _torch()
-    prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=copy_variant, capacity_slack=capacity_slack)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=copy_variant, capacity_slack=capacity_slack,
+                         **ctx_options)
     nf_dev = None
     if num_free is not None:
         nf_dev = torch.tensor([num_free], dtype=torch.int32, device=prob.device)
@@ -108,31 +109,31 @@ def test_block_sizes_and_row_bytes(S, heads, head_dim, variant):
 
 @pytest.mark.parametrize("tune", ["1,2,1,0,1", "1,12,1,10,2", "8,6,2,2,2", "4,3,8,1,1", "2,3,16,1,2", "8,12,1,4,1",
                                   "3,5,4,3,2", "8,2,32,0,2"])
-def test_bulk_copy_ring_shapes(tune, monkeypatch):
-    """Every ring shape the tuning knob can select (warps, stages, rows per item, loads ahead,
+def test_bulk_copy_ring_shapes(tune):
+    """Every ring shape the tuning fields can select (warps, stages, rows per item, loads ahead,
     plan entries ahead) must give the same bytes: whole pools against the oracle."""
-    monkeypatch.setenv("VTOKEN_BULK_TUNE", tune)
+    tuning = dict(zip(("warps", "stages", "rows", "depth", "ahead"), (int(x) for x in tune.split(","))))
     for w in (wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2),
               wl.longctx_scissor(seed=5, requests=2, lo=1500, hi=2500, layers=2, block_size=32),
               wl.mistral7b_random(seed=6, requests=4, lo=30, hi=300, layers=1, heads=4, head_dim=128, block_size=48)):
-        run_and_compare(w, copy_variant=2)
+        run_and_compare(w, copy_variant=2, tuning=tuning)
+    run_and_compare(wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2), copy_variant=2, coresident=1)
 
 
 @pytest.mark.parametrize("dynamic,chunk", [("0", "4"), ("1", "1"), ("1", "3"), ("1", "64"), ("1", "1000")])
-def test_copy_work_distribution_modes(dynamic, chunk, monkeypatch):
+def test_copy_work_distribution_modes(dynamic, chunk):
     """Fixed shares per warp and ticket distribution with several chunk sizes (one item per ticket,
     an odd count, more items per ticket than a small launch has): the same bytes, whole pools
     against the oracle, also when the context is reused for a second plan (the ticket counter must
     be back at zero)."""
-    monkeypatch.setenv("VTOKEN_COPY_DYNAMIC", dynamic)
-    monkeypatch.setenv("VTOKEN_COPY_CHUNK", chunk)
+    tuning = dict(fixed_shares=int(dynamic == "0"), chunk=int(chunk))
     for w in (wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2),
               wl.longctx_scissor(seed=5, requests=2, lo=1500, hi=2500, layers=2, block_size=32),
               wl.tiny(seed=1)):
-        run_and_compare(w, copy_variant=2)
+        run_and_compare(w, copy_variant=2, tuning=tuning)
     from harness.device import DeviceProblem
     w = wl.llama8b_h2o(seed=2, requests=5, lo=200, hi=900, layers=2)
-    prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=2)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=2, tuning=tuning)
     p = vto.plan_workload(w)
     k, v = host_pools(w)
     vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
@@ -147,18 +148,19 @@ def test_copy_work_distribution_modes(dynamic, chunk, monkeypatch):
 
 
 @pytest.mark.parametrize("pdl", ["0", "1"])
-def test_launch_modes_give_the_same_result(pdl, monkeypatch):
+def test_launch_modes_give_the_same_result(pdl):
     """Plain stream-ordered launches and programmatic dependent launches (a kernel may become resident
     while its predecessor finishes and waits for it on the device): the same tables and bytes, for both
     copy paths, with launches issued back to back on one stream without host synchronisation between
     plan, copy and the next plan."""
-    monkeypatch.setenv("VTOKEN_PDL", pdl)
+    plain = int(pdl == "0")
     from harness.device import DeviceProblem
     torch = _torch()
     for variant in (1, 2):
-        run_and_compare(wl.mistral7b_random(seed=9, requests=6, lo=80, hi=600, layers=2), copy_variant=variant)
+        run_and_compare(wl.mistral7b_random(seed=9, requests=6, lo=80, hi=600, layers=2), copy_variant=variant,
+                        plain_launches=plain)
         w = wl.llama8b_h2o(seed=4, requests=6, lo=200, hi=900, layers=2)
-        prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=variant)
+        prob = DeviceProblem(w, fill_seed=FILL_SEED, copy_variant=variant, plain_launches=plain)
         p = vto.plan_workload(w)
         k, v = host_pools(w)
         vto.apply_moves_pools(k, v, p.move_src, p.move_dst)

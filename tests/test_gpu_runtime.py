@@ -320,7 +320,9 @@ def test_serving_loop_matches_oracle_step_by_step(seed, S, partial_options, wave
                     assert np.array_equal(rows_k[i], dev.payload(r, tok, l, 0, dev.row_elems))
                     assert np.array_equal(rows_v[i], dev.payload(r, tok, l, 1, dev.row_elems))
     assert repacked_something
-    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] == 0
+    # random victim lists name tokens outside the registered range now and then (skipped, flagged); the flags
+    # of the calls outside plan / repack stay up until they are read
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] & ~vt.FLAG_BAD_VICTIM == 0
     dev.close()
 
 
@@ -365,7 +367,107 @@ def test_runtime_flags_and_edges():
     assert np.array_equal(small.cpu().numpy(), o_slots[:4])
     assert np.array_equal(dev.map_offsets.cpu().numpy(), o_off)
     assert vt.vtoken_read_counts(dev.ctx)["error_flags"] & vt.FLAG_GATHER_OVERFLOW
+    # flags of these calls are reported once
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] == 0
     dev.close()
+
+
+def test_append_into_a_block_list_with_a_bad_id():
+    """A block id outside [0, num_blocks), fabricated on the host: the tokens that would land in it are
+    registered without a physical copy (slot -1, not kept), the flag is raised, everything else is as
+    the oracle computes it for the valid part, and nothing faults."""
+    import torch
+    S = 4
+    blocks = [np.array([2, 99, 7], np.int32), np.array([5, -3], np.int32)]        # 99 and -3 do not exist
+    st = ServingState.empty(S, capacities=[12, 8], block_lists=blocks, num_blocks=12)
+    dev = DeviceServing(st)
+    dev.upload_blocks(st)
+    dev.new_len.copy_(torch.tensor([11, 6], dtype=torch.int32))
+    vt.vtoken_sync_new_tokens(dev.ctx, num_requests=dev.num_requests, tt_offsets=dev.tt_offsets,
+                              tt_slots=dev.tt_slots, keep=dev.keep, tt_len=dev.tt_len, phys_len=dev.phys_len,
+                              bt_offsets=dev.bt_offsets, bt_blocks=dev.bt_blocks, new_len=dev.new_len)
+    torch.cuda.synchronize()
+    slots, keep = dev.tt_slots.cpu().numpy(), dev.keep.cpu().numpy()
+    assert slots[:11].tolist() == [8, 9, 10, 11, -1, -1, -1, -1, 28, 29, 30] and slots[11] == -1
+    assert keep[:12].tolist() == [1, 1, 1, 1, 0, 0, 0, 0, 1, 1, 1, 0]
+    assert slots[12:18].tolist() == [20, 21, 22, 23, -1, -1] and keep[12:18].tolist() == [1, 1, 1, 1, 0, 0]
+    assert dev.tt_len.cpu().numpy().tolist() == [11, 6] and dev.phys_len.cpu().numpy().tolist() == [11, 6]
+    assert vt.vtoken_read_counts(dev.ctx)["error_flags"] == vt.FLAG_BAD_BLOCK
+    # the unmapped tokens are invisible to the slot mapping, like every token without a physical copy
+    g_slots, g_ids, g_off = dev.slot_mapping()
+    o_slots, o_ids, o_off = vto.build_slot_mapping(st.tt_offsets, slots, keep)
+    assert np.array_equal(g_slots, o_slots) and np.array_equal(g_ids, o_ids) and np.array_equal(g_off, o_off)
+    assert (g_slots >= 0).all()
+    dev.close()
+
+
+def test_slot_mapping_overlaps_plan_and_repack_on_another_stream():
+    """The slot mapping is built every decode step on the compute stream while a plan and its copy run
+    on a side stream (Sec. 3.3.4).  The two use separate scratch: replayed against each other many
+    times without any ordering between the streams, both must still equal the oracle."""
+    import torch
+    from harness import workloads as wl
+    from harness.device import DeviceProblem
+    w = wl.steady_state(seed=3, requests=96, lo=200, hi=3000, layers=2, heads=2, head_dim=64)
+    prob = DeviceProblem(w, fill_seed=1)
+    dev = prob.device
+    T, R = w.num_tokens, w.num_requests
+    i32 = dict(dtype=torch.int32, device=dev)
+    m_slots, m_ids, m_off = torch.full((T,), -5, **i32), torch.full((T,), -5, **i32), torch.full((R + 1,), -5, **i32)
+    digest = torch.zeros(prob.max_requests, dtype=torch.int64, device=dev)
+    main, side = torch.cuda.Stream(), torch.cuda.Stream()
+
+    def mapping(st):
+        vt.vtoken_build_slot_mapping(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                     tt_slots=prob.tt_slots, keep=prob.keep, select=None, out_slots=m_slots,
+                                     out_token_ids=m_ids, out_capacity=T, out_offsets=m_off, stream=st)
+        vt.vtoken_digest_logical(prob.ctx, num_requests=prob.num_requests, tt_offsets=prob.tt_offsets,
+                                 tt_slots=prob.tt_slots, keep=prob.keep, select=None, layer_begin=0,
+                                 layer_end=w.num_layers, out_digest=digest, stream=st)
+
+    def relocation(st):
+        prob.plan(stream=st)
+        prob.repack(stream=st)
+
+    for fn, st in ((mapping, main), (relocation, side)):     # warm-up outside the captures
+        with torch.cuda.stream(st):
+            fn(st)
+    torch.cuda.synchronize()
+    g_map, g_rel = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_map, stream=main):
+        mapping(torch.cuda.current_stream())
+    with torch.cuda.graph(g_rel, stream=side):
+        relocation(torch.cuda.current_stream())
+    torch.cuda.synchronize()
+    m_slots.fill_(-5)
+    prob.new_tt_slots.fill_(-9)
+    torch.cuda.synchronize()
+    for _ in range(40):                                       # no event between the two streams
+        with torch.cuda.stream(main):
+            g_map.replay()
+        with torch.cuda.stream(side):
+            g_rel.replay()
+    torch.cuda.synchronize()
+
+    o_slots, o_ids, o_off = vto.build_slot_mapping(w.tt_offsets, w.tt_slots, w.keep)
+    n = len(o_slots)
+    assert np.array_equal(m_off.cpu().numpy(), o_off)
+    assert np.array_equal(m_slots.cpu().numpy()[:n], o_slots) and np.array_equal(m_ids.cpu().numpy()[:n], o_ids)
+    out = prob.outputs()
+    p = vto.plan_workload(w)
+    assert out["error_flags"] == 0 and out["num_moves"] == p.num_moves
+    assert np.array_equal(out["new_tt_slots"], p.new_tt_slots) and np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
+    assert np.array_equal(out["freed_blocks"], p.freed_blocks) and np.array_equal(out["req_status"], p.req_status)
+    k = np.stack([wl.fill_slab(1, 0, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
+    v = np.stack([wl.fill_slab(1, 1, l, w.num_layers, w.slots_per_layer, w.row_elems) for l in range(w.num_layers)])
+    want, _ = vto.digest_logical(k, v, w.tt_slots[w.tt_offsets[0]:w.tt_offsets[1]],
+                                 w.keep[w.tt_offsets[0]:w.tt_offsets[1]])
+    assert int(digest[0].item()) & (2 ** 64 - 1) == int(want) & (2 ** 64 - 1)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst, threads=2)
+    assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
+    assert prob.read_counts()["error_flags"] == 0
+    prob.close()
 
 
 def test_slot_mapping_full_size_tables_match_oracle():

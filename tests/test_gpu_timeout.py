@@ -4,8 +4,8 @@ flight land and returns -- the kernel ends, the context and the GPU stay usable.
 
 The stall is produced without faulting anything: a test hook arms the barrier of ONE work item
 with 16 bytes that no copy will ever deliver (every real copy still runs and completes).  The
-hook and the limit are read from the environment when a context is created."""
-import os
+hook exists only in the checked build of the library (vtoken_config.debug_stall_item; the
+production library refuses the field), the limit is vtoken_config.wait_limit_ms."""
 
 import numpy as np
 import pytest
@@ -21,13 +21,22 @@ def test_wait_runs_out_sets_flag_and_context_survives():
     import torch
     from harness.device import DeviceProblem
     w = wl.llama8b_h2o(seed=0, requests=4, lo=200, hi=600, layers=2)
-    os.environ["VTOKEN_WAIT_LIMIT_MS"] = "20"
-    os.environ["VTOKEN_TEST_STALL_ITEM"] = "5"
+    # the production library has no such hook
+    with pytest.raises(vt.VtokenError) as e:
+        DeviceProblem(w, fill_seed=1, copy_variant=2, wait_limit_ms=20, debug_stall_item=6)
+    assert e.value.code == vt.EINVAL
+    prev = vt.use_library("checked")
     try:
-        prob = DeviceProblem(w, fill_seed=1, copy_variant=2)
+        assert vt.vtoken_checked_build() == 1
+        _stalled_launch_and_recovery(w)
     finally:
-        del os.environ["VTOKEN_WAIT_LIMIT_MS"]
-        del os.environ["VTOKEN_TEST_STALL_ITEM"]
+        vt.use_library(prev)
+
+
+def _stalled_launch_and_recovery(w):
+    import torch
+    from harness.device import DeviceProblem
+    prob = DeviceProblem(w, fill_seed=1, copy_variant=2, wait_limit_ms=20, debug_stall_item=6)   # item 5
     prob.plan()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()

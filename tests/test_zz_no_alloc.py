@@ -4,15 +4,17 @@ cannot take cudaMalloc's device-wide synchronisation, an embedder that forbids a
 calls).  Its scratch is a fixed array in the library image, shared by all calls and carrying
 the previous call's contents, so the check is: two calls in a row, the second on different
 tables with fewer live tokens, each bit-identical to what the context-based
-vtoken_gather_logical returns for the same inputs.
+vtoken_gather_logical returns for the same inputs, and each compared directly with the CPU
+oracle's logical view of the same pools as well.
 
 Collected last on purpose (file name), so a failure here cannot hide any other test.
 """
 import numpy as np
 import pytest
 
-from paper_2608_13263_b200 import binding as vt
 from harness import workloads as wl
+from oracle import vto
+from paper_2608_13263_b200 import binding as vt
 
 pytestmark = pytest.mark.gpu
 
@@ -58,6 +60,31 @@ def test_noalloc_gather_equals_context_gather_twice_in_a_row():
         assert torch.equal(got, exp)
     assert torch.equal(off1[:R + 1], eoff1[:R + 1]) and torch.equal(off2[:R + 1], eoff2[:R + 1])
     assert int(f1) == 0 and int(f2) == 0
+
+    # ... and against the oracle itself: per request, per layer, K and V, rows in token-id order
+    def slab(kv, layer):
+        return wl.fill_slab(1, kv, layer, w.num_layers, w.slots_per_layer, w.row_elems)
+
+    def check_against_oracle(got_k, got_v, got_off, keep, l0, l1, selected):
+        off = got_off.cpu().numpy()
+        for li, layer in enumerate(range(l0, l1)):
+            ks, vs = slab(0, layer), slab(1, layer)
+            gk = got_k[li].cpu().numpy().view(np.uint16)
+            gv = got_v[li].cpu().numpy().view(np.uint16)
+            for r in range(R):
+                t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
+                if not selected(r):
+                    assert off[r + 1] == off[r]
+                    continue
+                kp = None if keep is None else keep[t0:t1]
+                want_k = vto.gather_logical(ks, w.tt_slots[t0:t1], kp)
+                want_v = vto.gather_logical(vs, w.tt_slots[t0:t1], kp)
+                assert off[r + 1] - off[r] == len(want_k)
+                assert np.array_equal(gk[off[r]:off[r + 1]], want_k), (layer, r)
+                assert np.array_equal(gv[off[r]:off[r + 1]], want_v), (layer, r)
+
+    check_against_oracle(k1, v1, off1, None, 0, 3, lambda r: True)
+    check_against_oracle(k2, v2, off2, w.keep, 1, 2, lambda r: r % 2 == 0)
 
     # overflow is reported through error_flags, like the context version reports it in its counts
     k3, v3, off3, f3 = noalloc(prob.tt_slots, None, 0, 1, resident - 7)

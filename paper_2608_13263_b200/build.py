@@ -22,7 +22,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(PKG, "libvtoken.so")
 CHECKED_LIB = os.path.join(PKG, "libvtoken_checked.so")
 
-LIB_SOURCES = ["api.cu", "plan.cu", "copy.cu", "gather.cu", "gather_static.cu", "runtime.cu", "plan_partial.cu",
+LIB_SOURCES = ["api.cu", "plan.cu", "plan_small.cu", "copy.cu", "gather.cu", "gather_static.cu", "runtime.cu", "plan_partial.cu",
                "waves.cu", "slot_cache.cu", "check.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -24,7 +24,7 @@ int dev_alloc(vtoken_ctx *ctx, T **p, int64_t count)
 void free_all(vtoken_ctx *ctx)
 {
     void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
-                    ctx->dst_blocks, ctx->counts, ctx->rt_counts, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
+                    ctx->dst_blocks, ctx->counts, ctx->rt_counts, ctx->plan_header, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->g_tile_n, ctx->g_req_part, ctx->g_req_before, ctx->part_shared, ctx->req_shared, ctx->req_detach,
                     ctx->req_rel_base,
                     ctx->stage.num_requests, ctx->stage.bt_blocks,
@@ -123,6 +123,7 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     auto A = [&](auto **p, int64_t n) { if (rc == VTOKEN_OK) rc = dev_alloc(ctx, p, n); };
     A(&ctx->req_n, cfg->max_requests);
     A(&ctx->req_dst_base, cfg->max_requests);
+    A(&ctx->plan_header, 4);
     A(&ctx->tile_n, (cfg->max_tokens + 1023) / 1024 + 1);
     A(&ctx->req_part, (int64_t)cfg->max_requests + 1);
     A(&ctx->req_before, (int64_t)cfg->max_requests + 1);

@@ -21,7 +21,8 @@ struct vtoken_ctx {
     bool has_plan;
 
     // planner scratch (DEVICE)
-    int32_t *req_n;            // [max_requests] live tokens
+    int32_t *req_n;            // [max_requests] live tokens (partial planner)
+    int32_t *plan_header;      // [4] small-table planner: R, T, num_free, first entry as its count kernel read them
     int32_t *part_n;           // [max_requests * VTK_PLAN_PARTS] live tokens per request part: only the context-free
                                // gather entry point (per-request index kernels) sets it, from its static scratch
     int32_t *req_dst_base;     // [max_requests] first destination block (index into the free list)
@@ -92,6 +93,7 @@ struct vtoken_ctx {
 
 // host launchers, one per translation unit
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
+int vtk_launch_plan_small(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
 int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st);
 int vtk_configure_copy(vtoken_ctx *ctx);
 // > 0: launched; 0: the context has no bulk configuration for these rows; < 0: VTOKEN_* error

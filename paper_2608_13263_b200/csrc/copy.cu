@@ -154,8 +154,10 @@ __device__ __forceinline__ void bulk_wait_read_n(int n)
         default: bulk_wait_read<10>(); break;
     }
 }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// every bulk store of this thread has read its shared-memory source (the global writes complete with the kernel)
+__device__ __forceinline__ void bulk_wait_all_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
+constexpr int TAIL_ITEMS_PER_WARP = 2;      // items per warp that are handed out singly at the end of a launch
 constexpr int BULK_MAX_WARPS = 16;
 constexpr int BULK_MAX_STAGES = 12;
 constexpr int BULK_MAX_SMEM = 216 * 1024;   // dynamic shared memory cap: leaves room for the static barrier arrays
@@ -252,20 +254,42 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
     // one address for a ticket at the same instant are served one after the other (about 3 us until the
     // last one has its answer), and nothing can start before.  The counter hands out the chunks behind
     // those (its value + number of warps); those requests are made a chunk ahead, off the critical path.
-    unsigned ticket = (unsigned)gw, chunk_base = 0, chunk_pos = (unsigned)chunk;
+    // The last items of a launch are handed out one per ticket: with a whole chunk per ticket to the end the
+    // warps would finish up to a chunk (about 3 us of a warp's time) apart, which a launch of tens of
+    // microseconds feels.  Tickets below n_big stand for `chunk` items, the ones behind them for one item.
+    const unsigned tail_items = min(total_items, (unsigned)gstride * (unsigned)TAIL_ITEMS_PER_WARP);
+    const unsigned n_big = (total_items - tail_items) / (unsigned)chunk;
+    const unsigned big_items = n_big * (unsigned)chunk;
+    unsigned ticket = (unsigned)gw, chunk_base = 0, chunk_len = 0, chunk_pos = 0;
+    unsigned finished_rank = 0xffffffffu;       // lane 0: how many warps had run out of tickets before this one
+    bool exhausted = false;
     auto take_ticket = [&]() { if (lane == 0) ticket = atomicAdd(&a.ticket[0], 1u) + (unsigned)gstride; };
     auto fetch = [&](Entry &e) {           // reads the next item of this warp, moves on
         e.dst0 = -1;
         e.src = -1;
         e.idx = 0;
         if (DYNAMIC) {
-            if (chunk_pos == (unsigned)chunk) {             // next chunk: its ticket was requested a chunk ago
+            if (chunk_pos == chunk_len && !exhausted) {     // next chunk: its ticket was requested a chunk ago
                 const unsigned t = __shfl_sync(0xffffffffu, ticket, 0);
-                chunk_base = t < 0x7fffffffu / (unsigned)chunk ? t * (unsigned)chunk : 0x7fffffffu;
+                if (t < n_big) {
+                    chunk_base = t * (unsigned)chunk;
+                    chunk_len = (unsigned)chunk;
+                } else {
+                    const unsigned single = t - n_big;
+                    chunk_base = single < total_items - big_items ? big_items + single : 0x7fffffffu;
+                    chunk_len = 1;
+                }
                 chunk_pos = 0;
-                if (chunk_base < total_items) take_ticket();
+                if (chunk_base < total_items) {
+                    take_ticket();
+                } else {
+                    // out of tickets: say so now, while this warp's last items are still in flight, so that the
+                    // counters are back at zero by the time the last warp leaves (see the end of the kernel)
+                    exhausted = true;
+                    if (lane == 0) finished_rank = atomicAdd(&a.ticket[1], 1u);
+                }
             }
-            const unsigned i = chunk_base + chunk_pos;
+            const unsigned i = exhausted ? 0x7fffffffu : chunk_base + chunk_pos;
             ++chunk_pos;
             e.slab = num_slabs;
             if (i < total_items) {
@@ -374,12 +398,13 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         }
         if (lane == 0) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_TIMEOUT);
     }
-    bulk_wait_all();
+    bulk_wait_all_read();
     if (DYNAMIC && lane == 0) {
-        // the last warp of the grid to get here puts the counters back for the next launch; every
-        // other warp has stopped taking tickets by then
-        __threadfence();
-        if (atomicAdd(&a.ticket[1], 1u) == (unsigned)gstride - 1u) {
+        // the last warp of the grid to run out of tickets puts the counters back for the next launch: every
+        // other warp has stopped taking tickets by then.  (A warp that timed out may not have run out: it
+        // reports in here, so that the count is complete either way.)
+        if (finished_rank == 0xffffffffu) finished_rank = atomicAdd(&a.ticket[1], 1u);
+        if (finished_rank == (unsigned)gstride - 1u) {
             a.ticket[0] = 0u;
             a.ticket[1] = 0u;
         }

@@ -51,6 +51,24 @@ __global__ void fill_kernel(uint8_t *pool, int kv, int L, int layer_begin, int l
     }
 }
 
+// Address-encoding fill (a debugging aid): every 8 bytes of a row say where the row was filled --
+// low word = slot, high word = pool (bit 31), layer (bits 16..30), index of the 8-byte group in the row
+// (bits 0..15) -- so that a row found in the wrong place names the place it came from.
+__global__ void fill_address_kernel(uint8_t *pool, int kv, int layer_begin, int layer_end, int64_t slots_per_layer,
+                                    int row_elems, int64_t layer_stride)
+{
+    const int groups = row_elems / 4;                     // 8-byte groups per row
+    const int64_t per_layer = slots_per_layer * groups;
+    const int64_t total = per_layer * (layer_end - layer_begin);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int layer = layer_begin + (int)(i / per_layer);
+        const int64_t r = i % per_layer;
+        const uint32_t slot = (uint32_t)(r / groups), g = (uint32_t)(r % groups);
+        const uint32_t hi = ((uint32_t)kv << 31) | ((uint32_t)layer << 16) | g;
+        *reinterpret_cast<uint2 *>(pool + (int64_t)(layer - layer_begin) * layer_stride + r * 8) = make_uint2(slot, hi);
+    }
+}
+
 // Every slot s of every layer must hold the fill of slot origin[s] (origin[s] == s: untouched).
 __global__ void verify_kernel(const uint8_t *pool, int kv, int L, int64_t slots_per_layer, int row_elems,
                               int64_t layer_stride, uint64_t seed, const int32_t *origin,
@@ -137,6 +155,20 @@ int vth_fill(void *dst, int kv, int num_layers, int layer_begin, int layer_end, 
     if (layer_stride_bytes == 0) layer_stride_bytes = slots_per_layer * row_elems * 2;
     fill_kernel<<<sm_count() * 16, 256, 0, (cudaStream_t)stream>>>((uint8_t *)dst, kv, num_layers, layer_begin, layer_end,
                                                             slots_per_layer, row_elems, layer_stride_bytes, seed);
+    return cudaGetLastError() == cudaSuccess ? 0 : -3;
+}
+
+// Address-encoding fill of layers [layer_begin, layer_end) of pool kv; row_elems a multiple of 4, at most
+// 65536 groups per row and 32768 layers.
+int vth_fill_address(void *dst, int kv, int num_layers, int layer_begin, int layer_end, int64_t slots_per_layer,
+                     int row_elems, int64_t layer_stride_bytes, void *stream)
+{
+    if (!dst || row_elems % 4 != 0 || row_elems / 4 > 65536 || num_layers > 32768 || layer_begin < 0 ||
+        layer_end > num_layers || layer_begin >= layer_end)
+        return -1;
+    if (layer_stride_bytes == 0) layer_stride_bytes = slots_per_layer * row_elems * 2;
+    fill_address_kernel<<<sm_count() * 16, 256, 0, (cudaStream_t)stream>>>((uint8_t *)dst, kv, layer_begin, layer_end,
+                                                                        slots_per_layer, row_elems, layer_stride_bytes);
     return cudaGetLastError() == cudaSuccess ? 0 : -3;
 }
 

@@ -19,9 +19,11 @@ from .workloads import Workload
 class DeviceProblem:
     def __init__(self, w: Workload, device="cuda:0", fill_seed: int = 1, copy_variant: int = 0, max_ctas: int = 0,
                  capacity_slack: int = 0, allocate_pools: bool = True, wave_capacity: bool = False,
-                 ctx_capacity: dict = None, **ctx_options):
+                 ctx_capacity: dict = None, fill_mode: str = "random", **ctx_options):
         """``ctx_options``: further keyword arguments of ``vtoken_create`` (coresident, wait_limit_ms,
-        plain_launches, tuning, debug_stall_item)."""
+        plain_launches, tuning, debug_stall_item).  ``fill_mode``: "random" (the seeded pool fill) or
+        "address" (every row says where it was filled: a debugging aid)."""
+        self.fill_mode = fill_mode
         self.w = w
         self.device = torch.device(device)
         self.fill_seed = fill_seed
@@ -90,8 +92,12 @@ class DeviceProblem:
     def fill_pools(self, stream=None):
         w = self.w
         for kv, pool in ((0, self.k_pool), (1, self.v_pool)):
-            vh.vth_fill(pool, kv, w.num_layers, 0, w.num_layers, w.slots_per_layer, w.row_elems, self.fill_seed,
-                        stream=stream)
+            if self.fill_mode == "address":
+                vh.vth_fill_address(pool, kv, w.num_layers, 0, w.num_layers, w.slots_per_layer, w.row_elems,
+                                    stream=stream)
+            else:
+                vh.vth_fill(pool, kv, w.num_layers, 0, w.num_layers, w.slots_per_layer, w.row_elems, self.fill_seed,
+                            stream=stream)
 
     def fresh_slab(self, kv: int, layer: int) -> torch.Tensor:
         """Pre-repack content of one (K|V, layer) slab, regenerated on the device."""

@@ -9,7 +9,7 @@ from paper_2608_13263_b200.binding import _ptr, _stream
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libvtoken_harness.so")
-SYMBOLS = ["vth_fill", "vth_verify", "vth_decode_read"]
+SYMBOLS = ["vth_fill", "vth_fill_address", "vth_verify", "vth_decode_read"]
 
 _lib = None
 
@@ -28,6 +28,8 @@ def load():
         lib = ctypes.CDLL(LIB_PATH)
         lib.vth_fill.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
                                  ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p]
+        lib.vth_fill_address.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                         ctypes.c_int64, ctypes.c_int, ctypes.c_int64, ctypes.c_void_p]
         lib.vth_verify.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int64, ctypes.c_int,
                                    ctypes.c_int64, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         lib.vth_decode_read.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
@@ -43,6 +45,14 @@ def vth_fill(dst, kv, num_layers, layer_begin, layer_end, slots_per_layer, row_e
                          layer_stride_bytes, seed, _stream(stream))
     if rc != 0:
         raise RuntimeError(f"vth_fill failed: {rc}")
+
+
+def vth_fill_address(dst, kv, num_layers, layer_begin, layer_end, slots_per_layer, row_elems,
+                     layer_stride_bytes=0, stream=None) -> None:
+    rc = load().vth_fill_address(_ptr(dst), kv, num_layers, layer_begin, layer_end, slots_per_layer, row_elems,
+                                 layer_stride_bytes, _stream(stream))
+    if rc != 0:
+        raise RuntimeError(f"vth_fill_address failed: {rc}")
 
 
 def vth_verify(pool, kv, num_layers, slots_per_layer, row_elems, seed, origin, mismatches,

@@ -94,6 +94,29 @@ def fill_slab(seed: int, kv: int, layer: int, num_layers: int, slots_per_layer: 
                      np.arange(slots_per_layer, dtype=np.uint64))
 
 
+def fill_slab_address(kv: int, layer: int, slots_per_layer: int, row_elems: int) -> np.ndarray:
+    """Address-encoding fill of one (K|V, layer) slab, uint16 [slots_per_layer, row_elems]: every 8 bytes
+    of a row say where the row was filled -- low 32-bit word = slot, high word = pool (bit 31), layer
+    (bits 16..30), index of the 8-byte group in the row (bits 0..15).  Identical to the harness kernel;
+    a row found in the wrong place names the place it came from (``decode_row_address``)."""
+    groups = row_elems // 4
+    out = np.empty((slots_per_layer, groups, 2), dtype=np.uint32)
+    out[:, :, 0] = np.arange(slots_per_layer, dtype=np.uint32)[:, None]
+    out[:, :, 1] = (np.uint32(kv) << np.uint32(31)) | (np.uint32(layer) << np.uint32(16)) | np.arange(groups, dtype=np.uint32)[None, :]
+    return out.reshape(slots_per_layer, groups * 2).view(np.uint16).reshape(slots_per_layer, row_elems)
+
+
+def decode_row_address(row: np.ndarray):
+    """(kv, layer, slot) an address-filled row says it came from, or None when its 8-byte groups disagree
+    (bytes of several rows, or not an address fill at all)."""
+    w = np.ascontiguousarray(row).view(np.uint32).reshape(-1, 2)
+    slot, hi = w[:, 0], w[:, 1]
+    kv, layer, group = hi >> np.uint32(31), (hi >> np.uint32(16)) & np.uint32(0x7FFF), hi & np.uint32(0xFFFF)
+    ok = (slot == slot[0]).all() and (kv == kv[0]).all() and (layer == layer[0]).all() and \
+        (group == np.arange(len(group), dtype=np.uint32)).all()
+    return (int(kv[0]), int(layer[0]), int(slot[0])) if ok else None
+
+
 # --------------------------------------------------------------------------------------
 @dataclasses.dataclass
 class Workload:

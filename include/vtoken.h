@@ -538,6 +538,12 @@ int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int
                      int32_t *variant);                   /* launch shape of the copy kernel */
 int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx);      /* device scratch held by the context */
 int vtoken_checked_build(void);                           /* 1: this library was compiled with VTOKEN_CHECKED */
+/* Self-test of the checked build: one thread reads element `index` of a context scratch array of
+ * max_requests int32 through the same checked accessor every kernel of that build uses, and stores what
+ * it read to *out_value (DEVICE).  Inside the array: the element.  Outside: nothing is read there,
+ * VTOKEN_FLAG_CHECK_FAILED is raised (vtoken_read_counts), nothing faults.  The production library
+ * returns VTOKEN_EINVAL. */
+int vtoken_debug_probe(vtoken_ctx *ctx, int64_t index, int32_t *out_value, void *cuda_stream);
 
 #ifdef __cplusplus
 }

@@ -25,7 +25,8 @@ SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "v
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
            "vtoken_slot_cache_update", "vtoken_repack_host_partial", "vtoken_check_tables",
-           "vtoken_evict_tokens_counted", "vtoken_sync_new_tokens_counted", "vtoken_checked_build"]
+           "vtoken_evict_tokens_counted", "vtoken_sync_new_tokens_counted", "vtoken_checked_build",
+           "vtoken_debug_probe"]
 
 
 class VtokenError(RuntimeError):
@@ -177,6 +178,7 @@ def load():
                                               [ctypes.c_void_p] * 4
         lib.vtoken_slot_cache_update.argtypes = [ctypes.c_void_p] * 13
         lib.vtoken_checked_build.argtypes = []
+        lib.vtoken_debug_probe.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p]
         _libs[path] = lib
         _lib = lib
     return _lib
@@ -324,6 +326,10 @@ def vtoken_copy_grid(ctx) -> dict:
 
 def vtoken_checked_build() -> int:
     return int(load().vtoken_checked_build())
+
+
+def vtoken_debug_probe(ctx, index: int, out_value, stream=None) -> None:
+    _check(load().vtoken_debug_probe(ctx, index, _ptr(out_value), _stream(stream)), "vtoken_debug_probe", ctx)
 
 
 def vtoken_scratch_bytes(ctx) -> int:

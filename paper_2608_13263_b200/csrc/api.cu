@@ -356,6 +356,26 @@ int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int
 
 int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx) { return ctx ? ctx->scratch_bytes : 0; }
 
+namespace {
+__global__ void probe_kernel(vtk_arr<int32_t> arr, int64_t index, int32_t *out)
+{
+    *out = arr[index];          // checked build: outside [0, n) this reads a dummy element and raises the flag
+}
+}  // namespace
+
+int vtoken_debug_probe(vtoken_ctx *ctx, int64_t index, int32_t *out_value, void *cuda_stream)
+{
+#ifdef VTOKEN_CHECKED
+    if (!ctx || !out_value) return VTOKEN_EINVAL;
+    probe_kernel<<<1, 1, 0, (cudaStream_t)cuda_stream>>>(VTK_ARR(ctx, ctx->req_n, ctx->cfg.max_requests), index, out_value);
+    VTK_CUDA(ctx, cudaGetLastError());
+    return VTOKEN_OK;
+#else
+    (void)ctx; (void)index; (void)out_value; (void)cuda_stream;
+    return VTOKEN_EINVAL;       // the production library has no checked arrays to probe
+#endif
+}
+
 int vtoken_checked_build(void)
 {
 #ifdef VTOKEN_CHECKED

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "vtoken.h"
 
 #define VTK_PLAN_PARTS 8   // token ranges per request in the planner
@@ -90,6 +92,56 @@ struct vtoken_ctx {
     unsigned int *copy_ticket; // [2] DEVICE: next item, finished warps (zero between launches)
     int bulk_warps, bulk_stages, bulk_rows, bulk_depth, bulk_ahead;   // bulk path: warps per CTA, ring size, rows per item, loads ahead
 };
+
+// ---------------------------------------------------------------------------------------
+// Device arrays as the kernels see them.  In the production build vtk_arr<T> is a bare pointer.
+// In the checked build (-DVTOKEN_CHECKED, libvtoken_checked.so) it also carries the number of
+// elements the array holds and the address of a flag word of the context: an index outside
+// [0, n) raises VTOKEN_FLAG_CHECK_FAILED there and the access goes to a dummy element instead
+// -- it is skipped, nothing faults, the kernel goes on.  The tests run against both builds and
+// require the flag to stay clear: the place of a memory sanitizer, which also catches what a
+// comparison of results cannot (a read beyond an array, a stray write into scratch).
+// ---------------------------------------------------------------------------------------
+#ifdef VTOKEN_CHECKED
+static __device__ __align__(16) unsigned long long vtk_dummy[4];
+#endif
+
+template <typename T>
+struct vtk_arr {
+    T *p;
+#ifdef VTOKEN_CHECKED
+    int64_t n;
+    uint32_t *flag;
+    __host__ __device__ vtk_arr() : p(nullptr), n(0), flag(nullptr) {}
+    __host__ __device__ vtk_arr(T *p_, int64_t n_, uint32_t *flag_) : p(p_), n(n_), flag(flag_) {}
+    __device__ __forceinline__ T &bad() const
+    {
+        if (flag) atomicOr(flag, (uint32_t)VTOKEN_FLAG_CHECK_FAILED);
+        return *reinterpret_cast<T *>(vtk_dummy);
+    }
+    __device__ __forceinline__ T &operator[](int64_t i) const { return (p == nullptr || i < 0 || i >= n) ? bad() : p[i]; }
+    // `count` elements from element i on as a bare pointer (vector accesses)
+    __device__ __forceinline__ T *at(int64_t i, int64_t count = 1) const
+    {
+        return (p == nullptr || i < 0 || i + count > n) ? &bad() : p + i;
+    }
+#else
+    __host__ __device__ vtk_arr() : p(nullptr) {}
+    __host__ __device__ vtk_arr(T *p_, int64_t, uint32_t *) : p(p_) {}
+    __device__ __forceinline__ T &operator[](int64_t i) const { return p[i]; }
+    __device__ __forceinline__ T *at(int64_t i, int64_t = 1) const { return p + i; }
+#endif
+    __device__ __forceinline__ T &operator*() const { return (*this)[0]; }
+    __device__ __forceinline__ T *operator->() const { return at(0); }
+    __host__ __device__ __forceinline__ bool null() const { return p == nullptr; }
+};
+
+// the flag word the checked build reports to: the context's word for the calls outside plan / repack,
+// which no kernel overwrites and vtoken_read_counts reports (and clears)
+#define VTK_CHECK_FLAG(ctx) (&(ctx)->rt_counts->error_flags)
+// binds `n` elements at `ptr` (capacity known to the context) for a kernel
+#define VTK_ARR(ctx, ptr, n) \
+    vtk_arr<typename std::remove_pointer<typename std::decay<decltype(ptr)>::type>::type>((ptr), (int64_t)(n), VTK_CHECK_FLAG(ctx))
 
 // host launchers, one per translation unit
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
@@ -189,7 +241,8 @@ __device__ __forceinline__ int vtk_block_rank(bool flag, int *warp_sums, int &to
 // Range [off[r], off[r+1]) of request r in a CSR table, clipped to the create-time capacity of that
 // table: entries at or beyond `cap` (and ranges that run backwards) do not exist for the planners,
 // whose output buffers are sized by the capacities.  Returns true when something was clipped.
-__device__ __forceinline__ bool vtk_range(const int32_t *off, int r, int64_t cap, int64_t &lo, int64_t &hi)
+template <typename Off>
+__device__ __forceinline__ bool vtk_range(const Off &off, int r, int64_t cap, int64_t &lo, int64_t &hi)
 {
     const int64_t a = off[r], b = off[r + 1];
     lo = a < 0 ? 0 : (a > cap ? cap : a);
@@ -236,7 +289,8 @@ constexpr int VTK_TILE_TOK = 4;
 constexpr int VTK_TILE = VTK_TILE_NT * VTK_TILE_TOK;
 
 // first table entry of request r (r == R: one past the last entry), clipped to the table capacity
-__device__ __forceinline__ int64_t vtk_clipped_offset(const int32_t *off, int r, int64_t cap)
+template <typename Off>
+__device__ __forceinline__ int64_t vtk_clipped_offset(const Off &off, int r, int64_t cap)
 {
     const int64_t o = off[r];
     return o < 0 ? 0 : (o > cap ? cap : o);
@@ -246,7 +300,14 @@ __device__ __forceinline__ int64_t vtk_clipped_offset(const int32_t *off, int r,
 // Entries in front of `first` (the first request's first entry) belong to no request and count as dead.
 // vec: tt_slots is 16-byte and keep 4-byte aligned (t is a multiple of four).  keep == nullptr: every entry
 // with a slot counts as kept.
-__device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, const uint8_t *keep, int vec, int64_t t,
+// element i of a bare pointer or of a vtk_arr, `count` elements as a bare pointer
+template <typename T> __device__ __forceinline__ T *vtk_at(T *p, int64_t i, int64_t = 1) { return p + i; }
+template <typename T> __device__ __forceinline__ T *vtk_at(const vtk_arr<T> &a, int64_t i, int64_t count = 1) { return a.at(i, count); }
+template <typename T> __device__ __forceinline__ bool vtk_null(T *p) { return p == nullptr; }
+template <typename T> __device__ __forceinline__ bool vtk_null(const vtk_arr<T> &a) { return a.null(); }
+
+template <typename Slots, typename Keep>
+__device__ __forceinline__ unsigned vtk_load_entries(const Slots &tt_slots, const Keep &keep, int vec, int64_t t,
                                                      int64_t first, int64_t T, int64_t slots_per_layer,
                                                      int32_t (&slot)[VTK_TILE_TOK], bool &bad)
 {
@@ -254,14 +315,15 @@ __device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, co
 #pragma unroll
     for (int k = 0; k < VTK_TILE_TOK; ++k) slot[k] = -1;
     if (vec && t + VTK_TILE_TOK <= T) {
-        const int4 s4 = *reinterpret_cast<const int4 *>(tt_slots + t);
-        const uchar4 k4 = keep ? *reinterpret_cast<const uchar4 *>(keep + t) : make_uchar4(1, 1, 1, 1);
+        const int4 s4 = *reinterpret_cast<const int4 *>(vtk_at(tt_slots, t, VTK_TILE_TOK));
+        const uchar4 k4 = !vtk_null(keep) ? *reinterpret_cast<const uchar4 *>(vtk_at(keep, t, VTK_TILE_TOK))
+                                          : make_uchar4(1, 1, 1, 1);
         slot[0] = s4.x; slot[1] = s4.y; slot[2] = s4.z; slot[3] = s4.w;
         kp[0] = k4.x; kp[1] = k4.y; kp[2] = k4.z; kp[3] = k4.w;
     } else {
 #pragma unroll
         for (int k = 0; k < VTK_TILE_TOK; ++k)
-            if (t + k < T) { slot[k] = tt_slots[t + k]; kp[k] = keep ? keep[t + k] : 1; }
+            if (t + k < T) { slot[k] = tt_slots[t + k]; kp[k] = !vtk_null(keep) ? keep[t + k] : 1; }
     }
     unsigned bits = 0;
 #pragma unroll
@@ -277,7 +339,8 @@ __device__ __forceinline__ unsigned vtk_load_entries(const int32_t *tt_slots, co
 // owner of an entry: the last request whose first entry is at or before it; -1: the entry lies in
 // front of the first request -- each found by one warp (warps 0 and 1, all lanes) with a 32-way
 // search over the offsets; tile_req[2] is shared memory, valid after the caller's next barrier.
-__device__ __forceinline__ void vtk_tile_owners(const int32_t *off, int R, int64_t cap, int64_t base, int64_t T,
+template <typename Off>
+__device__ __forceinline__ void vtk_tile_owners(const Off &off, int R, int64_t cap, int64_t base, int64_t T,
                                                 int *tile_req)
 {
     const int warp = threadIdx.x >> 5, lane = vtk_lane();
@@ -298,7 +361,8 @@ __device__ __forceinline__ void vtk_tile_owners(const int32_t *off, int R, int64
 }
 
 // The request that owns entry t of the tile whose owners are in tile_req (-1: none).
-__device__ __forceinline__ int vtk_entry_owner(const int32_t *off, int64_t cap, const int *tile_req, int64_t t)
+template <typename Off>
+__device__ __forceinline__ int vtk_entry_owner(const Off &off, int64_t cap, const int *tile_req, int64_t t)
 {
     int lo = tile_req[0], hi = (tile_req[1] > tile_req[0] ? tile_req[1] : tile_req[0]) + 1;
     while (hi - lo > 1) {                   // offset(lo) <= t (or lo == -1); offset(hi) > t
@@ -309,10 +373,11 @@ __device__ __forceinline__ int vtk_entry_owner(const int32_t *off, int64_t cap, 
 }
 
 // A token is live when it owns a slot inside the pool and the policy kept it.
-__device__ __forceinline__ bool vtk_live(int32_t slot, const uint8_t *keep, int64_t t, int64_t slots_per_layer,
+template <typename Keep>
+__device__ __forceinline__ bool vtk_live(int32_t slot, const Keep &keep, int64_t t, int64_t slots_per_layer,
                                          bool &bad_slot)
 {
     if (slot < 0) return false;
     if ((int64_t)slot >= slots_per_layer) { bad_slot = true; return false; }
-    return keep == nullptr || keep[t] != 0;
+    return vtk_null(keep) || keep[t] != 0;
 }

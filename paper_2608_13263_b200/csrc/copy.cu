@@ -21,9 +21,10 @@ namespace {
 
 struct CopyArgs {
     uint8_t *k_pool, *v_pool;
-    const int32_t *dst_src, *dst_blocks;
-    vtoken_counts *counts;
+    vtk_arr<const int32_t> dst_src, dst_blocks;
+    vtk_arr<vtoken_counts> counts;
     int64_t layer_stride, row_bytes;
+    int64_t slots_per_layer;   // rows of a slab (the checked build refuses a row outside)
     int32_t S, L, rows;        // rows per item (bulk path)
     int64_t wait_limit_ns;     // bound of every wait on a shared-memory barrier (bulk path)
     int64_t stall_item;        // -1, or the global index of one item whose barrier is armed with bytes that
@@ -31,7 +32,7 @@ struct CopyArgs {
     unsigned int *ticket;      // dynamic item distribution: [0] next item index, [1] warps that have finished
     // gather mode (logical view): rows g_src[0 .. *g_total) of layers [layer_begin, layer_begin + L) go to the
     // dense buffers out_k / out_v, [L][out_capacity][row_bytes]
-    const int32_t *g_src, *g_total;
+    vtk_arr<const int32_t> g_src, g_total;
     uint8_t *out_k, *out_v;
     int64_t out_capacity;
     int32_t layer_begin;
@@ -74,6 +75,12 @@ __global__ void __launch_bounds__(REG_NT) copy_rows_kernel(CopyArgs a)
         const int j = (int)(ds / a.S);
         const int32_t blk = a.dst_blocks[j];
         if (blk < 0) continue;
+#ifdef VTOKEN_CHECKED
+        if ((int64_t)src >= a.slots_per_layer || ((int64_t)blk + 1) * a.S > a.slots_per_layer) {
+            atomicOr(&a.counts->error_flags, (uint32_t)VTOKEN_FLAG_CHECK_FAILED);     // a row outside its slab: skipped
+            continue;
+        }
+#endif
         uint8_t *base = slab_base(a, slab);
         const uint4 *sp = reinterpret_cast<const uint4 *>(base + (int64_t)src * a.row_bytes);
         uint4 *dp = reinterpret_cast<uint4 *>(base + ((int64_t)blk * a.S + (ds - (int64_t)j * a.S)) * a.row_bytes);
@@ -340,7 +347,15 @@ __global__ void __launch_bounds__(BULK_MAX_WARPS * 32) copy_bulk_kernel(CopyArgs
         } else {
             fetch(e1);                               // in flight for one step
         }
-        const bool valid = e.src >= 0 && e.dst0 >= 0;
+        bool valid = e.src >= 0 && e.dst0 >= 0;
+#ifdef VTOKEN_CHECKED
+        // a source row outside its slab, or a destination range outside the slab / the output buffer: skipped
+        if (valid && ((int64_t)e.src >= a.slots_per_layer ||
+                      (int64_t)e.dst0 + lane >= (GATHER ? a.out_capacity : a.slots_per_layer))) {
+            atomicOr(&a.counts->error_flags, (uint32_t)VTOKEN_FLAG_CHECK_FAILED);
+            valid = false;
+        }
+#endif
         uint8_t *base, *dst_base;
         if (GATHER) {
             const int li = e.slab < a.L ? e.slab : e.slab - a.L;
@@ -515,11 +530,12 @@ int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st)
     CopyArgs a;
     a.k_pool = (uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (uint8_t *)ctx->cfg.v_pool;
-    a.dst_src = ctx->dst_src;
-    a.dst_blocks = ctx->dst_blocks;
-    a.counts = ctx->counts;
+    a.dst_src = VTK_ARR(ctx, (const int32_t *)ctx->dst_src, (int64_t)ctx->cap_dst_blocks * ctx->cfg.block_size);
+    a.dst_blocks = VTK_ARR(ctx, (const int32_t *)ctx->dst_blocks, ctx->cap_dst_blocks);
+    a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.layer_stride = ctx->layer_stride;
     a.row_bytes = ctx->row_bytes;
+    a.slots_per_layer = ctx->slots_per_layer;
     a.S = ctx->cfg.block_size;
     a.L = ctx->cfg.num_layers;
     a.rows = ctx->bulk_rows;
@@ -552,19 +568,20 @@ int vtk_launch_gather_bulk(vtoken_ctx *ctx, const int32_t *g_src, const int32_t 
     CopyArgs a;
     a.k_pool = (uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (uint8_t *)ctx->cfg.v_pool;
-    a.dst_src = nullptr;
-    a.dst_blocks = nullptr;
-    a.counts = ctx->rt_counts;            // gather mode reads no count from it: only the time-out flag goes there
+    a.dst_src = vtk_arr<const int32_t>();
+    a.dst_blocks = vtk_arr<const int32_t>();
+    a.counts = VTK_ARR(ctx, ctx->rt_counts, 1);   // gather mode reads no count from it: only the time-out flag goes there
     a.layer_stride = ctx->layer_stride;
     a.row_bytes = ctx->row_bytes;
+    a.slots_per_layer = ctx->slots_per_layer;
     a.S = ctx->bulk_rows;                 // parts = 1: unused in gather mode
     a.L = layer_end - layer_begin;
     a.rows = ctx->bulk_rows;
     a.wait_limit_ns = ctx->wait_limit_ns;
     a.stall_item = -1;
     a.ticket = ctx->g_ticket;
-    a.g_src = g_src;
-    a.g_total = g_total;
+    a.g_src = VTK_ARR(ctx, g_src, ctx->cfg.max_tokens);
+    a.g_total = VTK_ARR(ctx, g_total, 1);
     a.out_k = (uint8_t *)out_k;
     a.out_v = (uint8_t *)out_v;
     a.out_capacity = out_capacity;

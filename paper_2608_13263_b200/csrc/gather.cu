@@ -14,12 +14,12 @@ constexpr int G_NT = 512;
 constexpr int G_PARTS = VTK_PLAN_PARTS;
 
 struct GatherArgs {
-    const int32_t *num_requests, *tt_offsets, *tt_slots;
-    const uint8_t *keep, *select;
-    int32_t *req_n, *part_n, *out_offsets, *g_src, *g_total;
-    int32_t *g_ids, *g_req;      // logical id / request of each output row, or NULL
-    unsigned long long *digest;  // per-request digest (digest kernel only)
-    vtoken_counts *counts;
+    vtk_arr<const int32_t> num_requests, tt_offsets, tt_slots;
+    vtk_arr<const uint8_t> keep, select;
+    vtk_arr<int32_t> req_n, part_n, out_offsets, g_src, g_total;
+    vtk_arr<int32_t> g_ids, g_req;      // logical id / request of each output row, or NULL
+    vtk_arr<unsigned long long> digest;  // per-request digest (digest kernel only)
+    vtk_arr<vtoken_counts> counts;
     const uint8_t *k_pool, *v_pool;
     uint8_t *out_k, *out_v;
     int64_t layer_stride, row_bytes, slots_per_layer, out_capacity, max_tokens;
@@ -27,7 +27,7 @@ struct GatherArgs {
     int32_t parts;               // token ranges (CTAs) per request, <= G_PARTS (the stride of part_n)
     // flat tiling (contexts made by vtoken_create; see plan.cu): live tokens per tile, then before every tile;
     // live tokens between the start of a request boundary's tile and the boundary; live tokens before a request
-    int32_t *tile_n, *req_part, *req_before;
+    vtk_arr<int32_t> tile_n, req_part, req_before;
     int32_t num_tiles, vec_in;
     int64_t table_cap;           // capacity of the token table: offsets are clipped to it
 };
@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(G_NT) gather_count_kernel(GatherArgs a)
     if (r >= g_requests(a)) return;
     int n = 0;
     bool bad = false;
-    if (a.select == nullptr || a.select[r] != 0) {
+    if (a.select.null() || a.select[r] != 0) {
         int64_t p0, p1;
         g_part_range(a.tt_offsets[r], a.tt_offsets[r + 1], c, a.parts, p0, p1);
         for (int64_t t = p0 + threadIdx.x; t < p1; t += G_NT)
@@ -129,7 +129,7 @@ __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
     __shared__ int warp_sums[G_NT / 32 + 1];
     const int r = blockIdx.x / a.parts, c = blockIdx.x % a.parts;
     if (r >= g_requests(a)) return;
-    if (a.select != nullptr && a.select[r] == 0) return;
+    if (!a.select.null() && a.select[r] == 0) return;
     const int64_t t0 = a.tt_offsets[r];
     int64_t p0, p1;
     g_part_range(t0, a.tt_offsets[r + 1], c, a.parts, p0, p1);
@@ -149,8 +149,8 @@ __global__ void __launch_bounds__(G_NT) gather_assign_kernel(GatherArgs a)
         carry += total;
         if (live && i < cap) {
             a.g_src[i] = slot;
-            if (a.g_ids != nullptr) a.g_ids[i] = (int32_t)(t - t0);
-            if (a.g_req != nullptr) a.g_req[i] = r;
+            if (!a.g_ids.null()) a.g_ids[i] = (int32_t)(t - t0);
+            if (!a.g_req.null()) a.g_req[i] = r;
         }
     }
 }
@@ -238,7 +238,7 @@ __global__ void __launch_bounds__(1024) gather_scan_flat_kernel(GatherArgs a)
         if (r < R) {
             const int before = live_before(r);
             a.req_before[r] = before;
-            if (a.select == nullptr || a.select[r] != 0) v = live_before(r + 1) - before;
+            if (a.select.null() || a.select[r] != 0) v = live_before(r + 1) - before;
             if (v < 0) v = 0;                                // offsets that run backwards
         }
         const int incl = vtk_block_incl_scan<int>(v, warp_tot, 0, shfl_int) + carry;
@@ -288,7 +288,7 @@ __global__ void __launch_bounds__(VTK_TILE_NT) gather_assign_flat_kernel(GatherA
     int first_row = 0;
     bool sel = false;
     auto load_request = [&]() {
-        sel = a.select == nullptr || a.select[r] != 0;
+        sel = a.select.null() || a.select[r] != 0;
         first_row = a.out_offsets[r] - a.req_before[r];      // output row of a token = this + its running count
         t0 = g_offset(a, r);
     };
@@ -309,8 +309,8 @@ __global__ void __launch_bounds__(VTK_TILE_NT) gather_assign_flat_kernel(GatherA
         const int64_t i = (int64_t)first_row + before + __popc(bits & ((1u << k) - 1u));
         if (i < 0 || i >= cap) continue;
         a.g_src[i] = slot[k];
-        if (a.g_ids != nullptr) a.g_ids[i] = (int32_t)(t + k - t0);
-        if (a.g_req != nullptr) a.g_req[i] = r;
+        if (!a.g_ids.null()) a.g_ids[i] = (int32_t)(t + k - t0);
+        if (!a.g_req.null()) a.g_req[i] = r;
     }
     if (bad) atomicOr(&a.counts->error_flags, VTOKEN_FLAG_BAD_SLOT);
 }
@@ -319,11 +319,14 @@ __global__ void __launch_bounds__(VTK_TILE_NT) gather_assign_flat_kernel(GatherA
 int launch_index(vtoken_ctx *ctx, GatherArgs &a, cudaStream_t st)
 {
     if (ctx->g_tile_n != nullptr) {
-        a.tile_n = ctx->g_tile_n;
-        a.req_part = ctx->g_req_part;
-        a.req_before = ctx->g_req_before;
+        a.tile_n = VTK_ARR(ctx, ctx->g_tile_n, (ctx->cfg.max_tokens + VTK_TILE - 1) / VTK_TILE + 1);
+        a.req_part = VTK_ARR(ctx, ctx->g_req_part, (int64_t)ctx->cfg.max_requests + 1);
+        a.req_before = VTK_ARR(ctx, ctx->g_req_before, (int64_t)ctx->cfg.max_requests + 1);
         a.num_tiles = (int32_t)((ctx->cfg.max_tokens + VTK_TILE - 1) / VTK_TILE);
-        a.vec_in = ((uintptr_t)a.tt_slots % 16 == 0 && (a.keep == nullptr || (uintptr_t)a.keep % 4 == 0)) ? 1 : 0;
+        a.vec_in = ((uintptr_t)a.tt_slots.p % 16 == 0 && (a.keep.null() || (uintptr_t)a.keep.p % 4 == 0)) ? 1 : 0;
+#ifdef VTOKEN_CHECKED
+        a.vec_in = 0;              // one checked access per entry instead of one per four
+#endif
         a.table_cap = ctx->cfg.max_tokens;
         VTK_CUDA(ctx, vtk_launch_dependent(ctx, gather_tiles_kernel, dim3(a.num_tiles + ctx->cfg.max_requests + 1),
                                            dim3(VTK_TILE_NT), 0, st, a));
@@ -528,6 +531,26 @@ __global__ void __launch_bounds__(GC_NT, 3) gather_digest_kernel(GatherArgs a)
     flush();
 }
 
+// the table inputs and the scratch every call of the gather family uses
+void bind_inputs(vtoken_ctx *ctx, GatherArgs &a, const int32_t *num_requests, const int32_t *tt_offsets,
+                 const int32_t *tt_slots, const uint8_t *keep, const uint8_t *select)
+{
+    const vtoken_config &c = ctx->cfg;
+    a.num_requests = VTK_ARR(ctx, num_requests, 1);
+    a.tt_offsets = VTK_ARR(ctx, tt_offsets, (int64_t)c.max_requests + 1);
+    a.tt_slots = VTK_ARR(ctx, tt_slots, c.max_tokens);
+    a.keep = VTK_ARR(ctx, keep, c.max_tokens);
+    a.select = VTK_ARR(ctx, select, c.max_requests);
+    a.req_n = VTK_ARR(ctx, ctx->req_n, c.max_requests);
+    a.part_n = VTK_ARR(ctx, ctx->part_n, (int64_t)c.max_requests * G_PARTS);
+    a.g_total = VTK_ARR(ctx, ctx->g_total, 1);
+    a.counts = VTK_ARR(ctx, ctx->rt_counts, 1);
+    a.g_ids = vtk_arr<int32_t>();
+    a.g_req = vtk_arr<int32_t>();
+    a.digest = vtk_arr<unsigned long long>();
+    a.tile_n = a.req_part = a.req_before = vtk_arr<int32_t>();
+}
+
 }  // namespace
 
 extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_requests, const int32_t *tt_offsets,
@@ -539,20 +562,12 @@ extern "C" int vtoken_digest_logical(vtoken_ctx *ctx, const int32_t *num_request
     if (layer_begin < 0 || layer_end > ctx->cfg.num_layers || layer_begin >= layer_end) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     GatherArgs a;
-    a.num_requests = num_requests;
-    a.tt_offsets = tt_offsets;
-    a.tt_slots = tt_slots;
-    a.keep = keep;
-    a.select = select;
-    a.req_n = ctx->req_n;
-    a.part_n = ctx->part_n;
-    a.out_offsets = out_offsets ? out_offsets : ctx->g_offsets;
-    a.g_src = ctx->g_src;
-    a.g_ids = ctx->g_ids;
-    a.g_req = ctx->g_req;
-    a.digest = (unsigned long long *)out_digest;
-    a.g_total = ctx->g_total;
-    a.counts = ctx->rt_counts;
+    bind_inputs(ctx, a, num_requests, tt_offsets, tt_slots, keep, select);
+    a.out_offsets = VTK_ARR(ctx, out_offsets ? out_offsets : ctx->g_offsets, (int64_t)ctx->cfg.max_requests + 1);
+    a.g_src = VTK_ARR(ctx, ctx->g_src, ctx->cfg.max_tokens);
+    a.g_ids = VTK_ARR(ctx, ctx->g_ids, ctx->cfg.max_tokens);
+    a.g_req = VTK_ARR(ctx, ctx->g_req, ctx->cfg.max_tokens);
+    a.digest = VTK_ARR(ctx, (unsigned long long *)out_digest, ctx->cfg.max_requests);
     a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (const uint8_t *)ctx->cfg.v_pool;
     a.out_k = a.out_v = nullptr;
@@ -578,20 +593,9 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
                       int64_t out_capacity_tokens, int32_t *out_offsets, cudaStream_t st)
 {
     GatherArgs a;
-    a.num_requests = num_requests;
-    a.tt_offsets = tt_offsets;
-    a.tt_slots = tt_slots;
-    a.keep = keep;
-    a.select = select;
-    a.req_n = ctx->req_n;
-    a.part_n = ctx->part_n;
-    a.out_offsets = out_offsets;
-    a.g_src = ctx->g_src;
-    a.g_ids = nullptr;
-    a.g_req = nullptr;
-    a.digest = nullptr;
-    a.g_total = ctx->g_total;
-    a.counts = ctx->rt_counts;
+    bind_inputs(ctx, a, num_requests, tt_offsets, tt_slots, keep, select);
+    a.out_offsets = VTK_ARR(ctx, out_offsets, (int64_t)ctx->cfg.max_requests + 1);
+    a.g_src = VTK_ARR(ctx, ctx->g_src, ctx->cfg.max_tokens);
     a.k_pool = (const uint8_t *)ctx->cfg.k_pool;
     a.v_pool = (const uint8_t *)ctx->cfg.v_pool;
     a.out_k = (uint8_t *)out_k;
@@ -629,20 +633,10 @@ extern "C" int vtoken_build_slot_mapping(vtoken_ctx *ctx, const int32_t *num_req
     if (out_capacity < 0) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     GatherArgs a;
-    a.num_requests = num_requests;
-    a.tt_offsets = tt_offsets;
-    a.tt_slots = tt_slots;
-    a.keep = keep;
-    a.select = select;
-    a.req_n = ctx->req_n;
-    a.part_n = ctx->part_n;
-    a.out_offsets = out_offsets;
-    a.g_src = out_slots;
-    a.g_ids = out_token_ids;
-    a.g_req = nullptr;
-    a.digest = nullptr;
-    a.g_total = ctx->g_total;
-    a.counts = ctx->rt_counts;
+    bind_inputs(ctx, a, num_requests, tt_offsets, tt_slots, keep, select);
+    a.out_offsets = VTK_ARR(ctx, out_offsets, (int64_t)ctx->cfg.max_requests + 1);
+    a.g_src = VTK_ARR(ctx, out_slots, out_capacity);
+    a.g_ids = VTK_ARR(ctx, out_token_ids, out_capacity);
     a.k_pool = a.v_pool = nullptr;
     a.out_k = a.out_v = nullptr;
     a.layer_stride = 0;

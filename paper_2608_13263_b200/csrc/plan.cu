@@ -25,21 +25,21 @@ constexpr int SCAN_NT = 1024;                    // threads of the single scan C
 
 struct PlanArgs {
     // inputs
-    const int32_t *num_requests, *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
-    const uint8_t *keep, *select;
+    vtk_arr<const int32_t> num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots;
+    vtk_arr<const uint8_t> keep, select;
     uint32_t thr_num, thr_den;
-    const int32_t *free_blocks, *num_free;
+    vtk_arr<const int32_t> free_blocks, num_free;
     // outputs
-    int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *out_status;
-    vtoken_counts *out_counts;
+    vtk_arr<int32_t> new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, out_status;
+    vtk_arr<vtoken_counts> out_counts;
     // context
-    int32_t *req_n, *req_dst_base, *req_freed_base, *req_status, *dst_src, *dst_blocks;
-    int32_t *tile_n;        // [num_tiles + 1] live tokens per tile (sign bit: a slot outside the pool); after the
-                            // scan: live tokens before the tile
-    int32_t *req_part;      // [max_requests + 1] live tokens between the start of the tile that holds the
-                            // request's first entry and that entry
-    int32_t *req_before;    // [max_requests + 1] live tokens before the request's first entry
-    vtoken_counts *counts;
+    vtk_arr<int32_t> req_n, req_dst_base, req_freed_base, req_status, dst_src, dst_blocks;
+    vtk_arr<int32_t> tile_n;  // [num_tiles + 1] live tokens per tile (sign bit: a slot outside the pool); after the
+                              // scan: live tokens before the tile
+    vtk_arr<int32_t> req_part;    // [max_requests + 1] live tokens between the start of the tile that holds the
+                                  // request's first entry and that entry
+    vtk_arr<int32_t> req_before;  // [max_requests + 1] live tokens before the request's first entry
+    vtk_arr<vtoken_counts> counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks, num_tiles;
     int32_t vec_in, vec_out;   // tt_slots 16-byte / keep 4-byte aligned; new_tt_slots 16-byte aligned
     int64_t slots_per_layer, max_tokens, max_table_blocks;
@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
             nb = (int)(hi - lo);
         }
         const int need = (int)(((int64_t)n + a.S - 1) / a.S);       // ceil(T_live / S)
-        bool sel = valid && (a.select == nullptr || a.select[r] != 0);
+        bool sel = valid && (a.select.null() || a.select[r] != 0);
         if (sel && a.thr_den != 0)
             sel = (unsigned long long)n * a.thr_den <
                   (unsigned long long)a.thr_num * (unsigned long long)nb * (unsigned long long)a.S;
@@ -339,7 +339,7 @@ __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
         a.dst_src[(int64_t)(dst_base + j) * S + off] = slot[k];
     }
     if (owned && a.vec_out) {
-        *reinterpret_cast<int4 *>(a.new_tt_slots + t) = make_int4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<int4 *>(a.new_tt_slots.at(t, TILE_TOK)) = make_int4(out[0], out[1], out[2], out[3]);
     } else {
         // the ragged end of the table, or entries in front of the first request (left untouched)
         const int64_t first = clipped_offset(a, 0);
@@ -363,33 +363,35 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
         return vtk_launch_plan_small(ctx, in, out, st);
 #endif
     PlanArgs a;
-    a.num_requests = in->num_requests;
-    a.bt_offsets = in->bt_offsets;
-    a.bt_blocks = in->bt_blocks;
-    a.tt_offsets = in->tt_offsets;
-    a.tt_slots = in->tt_slots;
-    a.keep = in->keep;
-    a.select = in->select;
+    const vtoken_config &c = ctx->cfg;
+    const int64_t tiles_cap = (c.max_tokens + TILE - 1) / TILE;
+    a.num_requests = VTK_ARR(ctx, in->num_requests, 1);
+    a.bt_offsets = VTK_ARR(ctx, in->bt_offsets, (int64_t)c.max_requests + 1);
+    a.bt_blocks = VTK_ARR(ctx, in->bt_blocks, c.max_table_blocks);
+    a.tt_offsets = VTK_ARR(ctx, in->tt_offsets, (int64_t)c.max_requests + 1);
+    a.tt_slots = VTK_ARR(ctx, in->tt_slots, c.max_tokens);
+    a.keep = VTK_ARR(ctx, in->keep, c.max_tokens);
+    a.select = VTK_ARR(ctx, in->select, c.max_requests);
     a.thr_num = in->thr_num;
     a.thr_den = in->thr_den;
-    a.free_blocks = in->free_blocks;
-    a.num_free = in->num_free;
-    a.new_bt_offsets = out->new_bt_offsets;
-    a.new_bt_blocks = out->new_bt_blocks;
-    a.new_tt_slots = out->new_tt_slots;
-    a.freed_blocks = out->freed_blocks;
-    a.out_status = out->req_status;
-    a.out_counts = out->counts;
-    a.req_n = ctx->req_n;
-    a.req_dst_base = ctx->req_dst_base;
-    a.req_freed_base = ctx->req_freed_base;
-    a.req_status = ctx->req_status;
-    a.dst_src = ctx->dst_src;
-    a.dst_blocks = ctx->dst_blocks;
-    a.tile_n = ctx->tile_n;
-    a.req_part = ctx->req_part;
-    a.req_before = ctx->req_before;
-    a.counts = ctx->counts;
+    a.free_blocks = VTK_ARR(ctx, in->free_blocks, c.max_free_blocks);
+    a.num_free = VTK_ARR(ctx, in->num_free, 1);
+    a.new_bt_offsets = VTK_ARR(ctx, out->new_bt_offsets, (int64_t)c.max_requests + 1);
+    a.new_bt_blocks = VTK_ARR(ctx, out->new_bt_blocks, c.max_table_blocks);
+    a.new_tt_slots = VTK_ARR(ctx, out->new_tt_slots, c.max_tokens);
+    a.freed_blocks = VTK_ARR(ctx, out->freed_blocks, c.max_table_blocks);
+    a.out_status = VTK_ARR(ctx, out->req_status, c.max_requests);
+    a.out_counts = VTK_ARR(ctx, out->counts, 1);
+    a.req_n = VTK_ARR(ctx, ctx->req_n, c.max_requests);
+    a.req_dst_base = VTK_ARR(ctx, ctx->req_dst_base, c.max_requests);
+    a.req_freed_base = VTK_ARR(ctx, ctx->req_freed_base, c.max_requests);
+    a.req_status = VTK_ARR(ctx, ctx->req_status, c.max_requests);
+    a.dst_src = VTK_ARR(ctx, ctx->dst_src, (int64_t)ctx->cap_dst_blocks * c.block_size);
+    a.dst_blocks = VTK_ARR(ctx, ctx->dst_blocks, ctx->cap_dst_blocks);
+    a.tile_n = VTK_ARR(ctx, ctx->tile_n, tiles_cap + 1);
+    a.req_part = VTK_ARR(ctx, ctx->req_part, (int64_t)c.max_requests + 1);
+    a.req_before = VTK_ARR(ctx, ctx->req_before, (int64_t)c.max_requests + 1);
+    a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
     a.max_requests = ctx->cfg.max_requests;
@@ -403,6 +405,9 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     // arrays allow it; tiles start at multiples of 1024 entries, so the base addresses decide
     a.vec_in = ((uintptr_t)in->tt_slots % 16 == 0 && (uintptr_t)in->keep % 4 == 0) ? 1 : 0;
     a.vec_out = ((uintptr_t)out->new_tt_slots % 16 == 0) ? 1 : 0;
+#ifdef VTOKEN_CHECKED
+    a.vec_in = a.vec_out = 0;      // one checked access per entry instead of one per four
+#endif
 
     const int R = ctx->cfg.max_requests;
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_tiles_kernel, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));

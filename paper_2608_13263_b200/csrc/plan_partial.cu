@@ -39,23 +39,23 @@ constexpr int PP_SCAN_NT = 1024;
 constexpr int TILE_NT = VTK_TILE_NT, TILE_TOK = VTK_TILE_TOK, TILE = VTK_TILE;
 
 struct PArgs {
-    const int32_t *num_requests, *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
-    const uint8_t *keep, *select, *protect;
+    vtk_arr<const int32_t> num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots;
+    vtk_arr<const uint8_t> keep, select, protect;
     uint32_t thr_num, thr_den, util_num, util_den, theta_num, theta_den, detach_num, detach_den;
     int32_t max_sources;
-    const int32_t *free_blocks, *num_free;
-    int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *released_blocks, *out_status;
-    vtoken_counts *out_counts;
-    int32_t *req_n, *req_ns, *req_nsrc, *req_dst_base, *req_freed_base, *req_status;
-    int32_t *req_shared, *req_detach, *req_rel_base;
+    vtk_arr<const int32_t> free_blocks, num_free;
+    vtk_arr<int32_t> new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, released_blocks, out_status;
+    vtk_arr<vtoken_counts> out_counts;
+    vtk_arr<int32_t> req_n, req_ns, req_nsrc, req_dst_base, req_freed_base, req_status;
+    vtk_arr<int32_t> req_shared, req_detach, req_rel_base;
     // flat tiling: counts per tile ([num_tiles + 1]; live and moving become running counts in the scan
     // kernel; the sign bit of a live count says "a slot outside the pool in this tile") and counts
     // between the start of the tile that holds a request's first entry and that entry ([max_requests + 1])
-    int32_t *tile_live, *tile_mov, *tile_shared, *part_live, *part_mov, *part_shared;
-    int32_t *req_before;     // [max_requests + 1] moving tokens of the table before the request's first entry
-    int32_t *dst_src, *dst_blocks, *n_b;
-    uint8_t *blk_src;
-    vtoken_counts *counts;
+    vtk_arr<int32_t> tile_live, tile_mov, tile_shared, part_live, part_mov, part_shared;
+    vtk_arr<int32_t> req_before;     // [max_requests + 1] moving tokens of the table before the request's first entry
+    vtk_arr<int32_t> dst_src, dst_blocks, n_b;
+    vtk_arr<uint8_t> blk_src;
+    vtk_arr<vtoken_counts> counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
     int32_t num_tiles, vec_in, vec_out;
     int64_t slots_per_layer, max_tokens, max_table_blocks;
@@ -126,7 +126,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
     const int R = pp_requests(a);
     const int64_t T = pp_offset(a, R);
     const int lane = vtk_lane(), warp = threadIdx.x >> 5;
-    const bool may_detach = a.protect != nullptr && a.detach_den != 0;
+    const bool may_detach = !a.protect.null() && a.detach_den != 0;
     // A CTA counts over the entries [base, limit): a whole tile, or (the CTAs behind the tiles, one per
     // request boundary) the entries between the start of the boundary's tile and the boundary.
     const bool is_tile = (int)blockIdx.x < a.num_tiles;
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
                 flags |= VTOKEN_FLAG_BAD_BLOCK;
                 blk = -1;
             } else {
-                eligible = !(a.protect != nullptr && a.protect[blk] != 0);
+                eligible = !(!a.protect.null() && a.protect[blk] != 0);
                 shared += !eligible;
                 if (eligible && a.util_den != 0)
                     eligible = (unsigned long long)a.n_b[blk] * a.util_den <
@@ -222,7 +222,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
         if (eligible && (a.max_sources <= 0 || rank < a.max_sources)) a.blk_src[blk] = 1;
     }
     int ns = (a.max_sources > 0 && carry > a.max_sources) ? a.max_sources : carry;
-    if (a.protect != nullptr && a.detach_den != 0) {
+    if (!a.protect.null() && a.detach_den != 0) {
         // copy-on-write detach: the request leaves its protected blocks when its own live tokens
         // fill less than detach_num / detach_den of them; then every one of them is a source
         __syncthreads();
@@ -358,7 +358,7 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
     for (int base = 0; base < R; base += PP_SCAN_NT) {
         const int r = base + tid;
         const bool valid = r < R;
-        const bool may_detach = a.protect != nullptr && a.detach_den != 0;
+        const bool may_detach = !a.protect.null() && a.detach_den != 0;
         int n = 0, nsrc = 0, nb = 0, ns = 0, nrel = 0;
         if (valid) {
             n = a.req_n[r];
@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(PP_SCAN_NT) pp_scan_kernel(PArgs a)
             nb = (int)(hi - lo);
         }
         const int need = (int)(((int64_t)nsrc + a.S - 1) / a.S);   // ceil(T_live / S) over the source blocks
-        bool sel = valid && triggered && (a.select == nullptr || a.select[r] != 0);
+        bool sel = valid && triggered && (a.select.null() || a.select[r] != 0);
         if (sel && a.thr_den != 0)
             sel = (unsigned long long)n * a.thr_den <
                   (unsigned long long)a.thr_num * (unsigned long long)nb * (unsigned long long)a.S;
@@ -425,7 +425,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
     const int R = pp_requests(a);
     const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
     const int S = a.S;
-    const bool may_detach = a.protect != nullptr && a.detach_den != 0;
+    const bool may_detach = !a.protect.null() && a.detach_den != 0;
     uint32_t flags = 0;
 
     if ((int)blockIdx.x >= a.num_tiles) {
@@ -548,7 +548,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
         a.dst_src[(int64_t)(dst_base + j) * S + off] = slot[k];
     }
     if (owned && a.vec_out) {
-        *reinterpret_cast<int4 *>(a.new_tt_slots + t) = make_int4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<int4 *>(a.new_tt_slots.at(t, TILE_TOK)) = make_int4(out[0], out[1], out[2], out[3]);
     } else {
         const int64_t first = pp_offset(a, 0);
 #pragma unroll
@@ -625,27 +625,29 @@ __global__ void __launch_bounds__(1024) pp_summary_kernel(const int32_t *num_req
 
 void fill_args(PArgs &a, vtoken_ctx *ctx)
 {
-    a.req_n = ctx->req_n;
-    a.tile_live = ctx->tile_n;
-    a.tile_mov = ctx->tile_mov;
-    a.tile_shared = ctx->tile_shared;
-    a.part_live = ctx->req_part;
-    a.part_mov = ctx->part_mov;
-    a.req_before = ctx->req_before;
-    a.req_ns = ctx->req_ns;
-    a.req_nsrc = ctx->req_nsrc;
-    a.req_dst_base = ctx->req_dst_base;
-    a.req_freed_base = ctx->req_freed_base;
-    a.req_status = ctx->req_status;
-    a.dst_src = ctx->dst_src;
-    a.dst_blocks = ctx->dst_blocks;
-    a.n_b = ctx->n_b;
-    a.blk_src = ctx->blk_src;
-    a.part_shared = ctx->part_shared;
-    a.req_shared = ctx->req_shared;
-    a.req_detach = ctx->req_detach;
-    a.req_rel_base = ctx->req_rel_base;
-    a.counts = ctx->counts;
+    const vtoken_config &c = ctx->cfg;
+    const int64_t tiles_cap = (c.max_tokens + TILE - 1) / TILE + 1, r1 = (int64_t)c.max_requests + 1;
+    a.req_n = VTK_ARR(ctx, ctx->req_n, c.max_requests);
+    a.tile_live = VTK_ARR(ctx, ctx->tile_n, tiles_cap);
+    a.tile_mov = VTK_ARR(ctx, ctx->tile_mov, tiles_cap);
+    a.tile_shared = VTK_ARR(ctx, ctx->tile_shared, tiles_cap);
+    a.part_live = VTK_ARR(ctx, ctx->req_part, r1);
+    a.part_mov = VTK_ARR(ctx, ctx->part_mov, r1);
+    a.req_before = VTK_ARR(ctx, ctx->req_before, r1);
+    a.req_ns = VTK_ARR(ctx, ctx->req_ns, c.max_requests);
+    a.req_nsrc = VTK_ARR(ctx, ctx->req_nsrc, c.max_requests);
+    a.req_dst_base = VTK_ARR(ctx, ctx->req_dst_base, c.max_requests);
+    a.req_freed_base = VTK_ARR(ctx, ctx->req_freed_base, c.max_requests);
+    a.req_status = VTK_ARR(ctx, ctx->req_status, c.max_requests);
+    a.dst_src = VTK_ARR(ctx, ctx->dst_src, (int64_t)ctx->cap_dst_blocks * c.block_size);
+    a.dst_blocks = VTK_ARR(ctx, ctx->dst_blocks, ctx->cap_dst_blocks);
+    a.n_b = VTK_ARR(ctx, ctx->n_b, c.num_blocks);
+    a.blk_src = VTK_ARR(ctx, ctx->blk_src, c.num_blocks);
+    a.part_shared = VTK_ARR(ctx, ctx->part_shared, r1);
+    a.req_shared = VTK_ARR(ctx, ctx->req_shared, c.max_requests);
+    a.req_detach = VTK_ARR(ctx, ctx->req_detach, c.max_requests);
+    a.req_rel_base = VTK_ARR(ctx, ctx->req_rel_base, c.max_requests);
+    a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
     a.max_requests = ctx->cfg.max_requests;
@@ -677,14 +679,15 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     cudaStream_t st = (cudaStream_t)cuda_stream;
     PArgs a;
     fill_args(a, ctx);
-    a.num_requests = in->num_requests;
-    a.bt_offsets = in->bt_offsets;
-    a.bt_blocks = in->bt_blocks;
-    a.tt_offsets = in->tt_offsets;
-    a.tt_slots = in->tt_slots;
-    a.keep = in->keep;
-    a.select = in->select;
-    a.protect = opts->protect;
+    const vtoken_config &c = ctx->cfg;
+    a.num_requests = VTK_ARR(ctx, in->num_requests, 1);
+    a.bt_offsets = VTK_ARR(ctx, in->bt_offsets, (int64_t)c.max_requests + 1);
+    a.bt_blocks = VTK_ARR(ctx, in->bt_blocks, c.max_table_blocks);
+    a.tt_offsets = VTK_ARR(ctx, in->tt_offsets, (int64_t)c.max_requests + 1);
+    a.tt_slots = VTK_ARR(ctx, in->tt_slots, c.max_tokens);
+    a.keep = VTK_ARR(ctx, in->keep, c.max_tokens);
+    a.select = VTK_ARR(ctx, in->select, c.max_requests);
+    a.protect = VTK_ARR(ctx, opts->protect, c.num_blocks);
     a.thr_num = in->thr_num;
     a.thr_den = in->thr_den;
     a.util_num = opts->util_num;
@@ -694,18 +697,21 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     a.detach_num = opts->detach_num;
     a.detach_den = opts->detach_den;
     a.max_sources = opts->max_source_blocks;
-    a.free_blocks = in->free_blocks;
-    a.num_free = in->num_free;
-    a.new_bt_offsets = out->new_bt_offsets;
-    a.new_bt_blocks = out->new_bt_blocks;
-    a.new_tt_slots = out->new_tt_slots;
-    a.freed_blocks = out->freed_blocks;
-    a.released_blocks = out->released_blocks;
-    a.out_status = out->req_status;
-    a.out_counts = out->counts;
+    a.free_blocks = VTK_ARR(ctx, in->free_blocks, c.max_free_blocks);
+    a.num_free = VTK_ARR(ctx, in->num_free, 1);
+    a.new_bt_offsets = VTK_ARR(ctx, out->new_bt_offsets, (int64_t)c.max_requests + 1);
+    a.new_bt_blocks = VTK_ARR(ctx, out->new_bt_blocks, c.max_table_blocks);
+    a.new_tt_slots = VTK_ARR(ctx, out->new_tt_slots, c.max_tokens);
+    a.freed_blocks = VTK_ARR(ctx, out->freed_blocks, c.max_table_blocks);
+    a.released_blocks = VTK_ARR(ctx, out->released_blocks, c.max_table_blocks);
+    a.out_status = VTK_ARR(ctx, out->req_status, c.max_requests);
+    a.out_counts = VTK_ARR(ctx, out->counts, 1);
 
     a.vec_in = ((uintptr_t)in->tt_slots % 16 == 0 && (uintptr_t)in->keep % 4 == 0) ? 1 : 0;
     a.vec_out = ((uintptr_t)out->new_tt_slots % 16 == 0) ? 1 : 0;
+#ifdef VTOKEN_CHECKED
+    a.vec_in = a.vec_out = 0;      // one checked access per entry instead of one per four
+#endif
 
     const int R = ctx->cfg.max_requests;
     const dim3 tiles_grid(a.num_tiles + R + 1);
@@ -731,16 +737,20 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
     PArgs a;
     memset(&a, 0, sizeof(a));
     fill_args(a, ctx);
-    a.num_requests = num_requests;
-    a.bt_offsets = bt_offsets;
-    a.bt_blocks = bt_blocks;
-    a.tt_offsets = tt_offsets;
-    a.tt_slots = tt_slots;
-    a.keep = keep;
-    a.n_b = n_b;
+    const vtoken_config &c = ctx->cfg;
+    a.num_requests = VTK_ARR(ctx, num_requests, 1);
+    a.bt_offsets = VTK_ARR(ctx, bt_offsets, (int64_t)c.max_requests + 1);
+    a.bt_blocks = VTK_ARR(ctx, bt_blocks, c.max_table_blocks);
+    a.tt_offsets = VTK_ARR(ctx, tt_offsets, (int64_t)c.max_requests + 1);
+    a.tt_slots = VTK_ARR(ctx, tt_slots, c.max_tokens);
+    a.keep = VTK_ARR(ctx, keep, c.max_tokens);
+    a.n_b = VTK_ARR(ctx, n_b, c.num_blocks);
     const int R = ctx->cfg.max_requests;
     VTK_CUDA(ctx, cudaMemsetAsync(n_b, 0, sizeof(int32_t) * (size_t)ctx->cfg.num_blocks, st));
     a.vec_in = ((uintptr_t)tt_slots % 16 == 0 && (uintptr_t)keep % 4 == 0) ? 1 : 0;
+#ifdef VTOKEN_CHECKED
+    a.vec_in = 0;
+#endif
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_tiles_kernel<0>, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
     if (hist) {
         VTK_CUDA(ctx, cudaMemsetAsync(hist, 0, sizeof(uint64_t) * (size_t)(ctx->cfg.block_size + 1), st));

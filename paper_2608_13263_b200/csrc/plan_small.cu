@@ -30,21 +30,22 @@ constexpr int MIN_CTAS = 4;                      // resident CTAs per SM the ass
 
 struct PlanArgs {
     // inputs
-    const int32_t *num_requests, *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots;
-    const uint8_t *keep, *select;
+    vtk_arr<const int32_t> num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots;
+    vtk_arr<const uint8_t> keep, select;
     uint32_t thr_num, thr_den;
-    const int32_t *free_blocks, *num_free;
+    vtk_arr<const int32_t> free_blocks, num_free;
     // outputs
-    int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *out_status;
-    vtoken_counts *out_counts;
+    vtk_arr<int32_t> new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, out_status;
+    vtk_arr<vtoken_counts> out_counts;
     // context
-    int32_t *dst_src, *dst_blocks;
-    int32_t *req_n;         // [max_requests] live tokens per request as the plan saw them (read by the commit of a wave)
-    int32_t *tile_n;        // [num_tiles] live tokens per tile (sign bit: a slot outside the pool)
-    int32_t *req_part;      // [max_requests + 1] live tokens between the start of the tile that holds the
-                            // request's first entry and that entry
-    int32_t *header;        // [4] R, T, num_free as the count kernel read them: one load instead of a chain of three
-    vtoken_counts *counts;
+    vtk_arr<int32_t> dst_src, dst_blocks;
+    vtk_arr<int32_t> req_n;     // [max_requests] live tokens per request as the plan saw them (read by the commit of a wave)
+    vtk_arr<int32_t> tile_n;    // [num_tiles] live tokens per tile (sign bit: a slot outside the pool)
+    vtk_arr<int32_t> req_part;  // [max_requests + 1] live tokens between the start of the tile that holds the
+                                // request's first entry and that entry
+    vtk_arr<int32_t> header;    // [4] R, T, num_free, first entry as the count kernel read them: one load instead
+                                // of a chain of three
+    vtk_arr<vtoken_counts> counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks, num_tiles;
     int32_t vec_in, vec_out;   // tt_slots 16-byte / keep 4-byte aligned; new_tt_slots 16-byte aligned
     int64_t slots_per_layer, max_tokens, max_table_blocks;
@@ -177,7 +178,7 @@ __device__ __forceinline__ void load_round(const PlanArgs &a, int R, int r0, Rou
     }
 #pragma unroll
     for (int k = 0; k < RQ_PER_THREAD; ++k)
-        in.sel[k] = (a.select != nullptr && r_mine + k < R) ? a.select[r_mine + k] : (unsigned char)1;
+        in.sel[k] = (!a.select.null() && r_mine + k < R) ? a.select[r_mine + k] : (unsigned char)1;
 }
 
 __device__ __forceinline__ int64_t clip_to(int64_t o, int64_t cap) { return o < 0 ? 0 : (o > cap ? cap : o); }
@@ -309,13 +310,12 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
     __shared__ TileRequest tile_rq[TILE];
     __shared__ unsigned start_bits[TILE / 32];   // one bit per entry of the tile at which a request starts
     __shared__ int warp_sums[TILE_NT / 32];
-    __shared__ int scan_carry;
     __shared__ Request own;                  // request CTAs: their request
     vtk_release_successor();
     vtk_wait_for_predecessor();
     const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
     const int S = a.S;
-    const int4 hdr = *reinterpret_cast<const int4 *>(a.header);
+    const int4 hdr = *reinterpret_cast<const int4 *>(a.header.at(0, 4));
     const int R = hdr.x;
     const int64_t T = hdr.y, first_entry = hdr.w;
     int nf = hdr.z;
@@ -336,8 +336,8 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
     uint8_t kp[TILE_TOK] = {0, 0, 0, 0};
     if (is_tile) {
         if (a.vec_in && t + TILE_TOK <= T) {
-            const int4 s4 = *reinterpret_cast<const int4 *>(a.tt_slots + t);
-            const uchar4 k4 = *reinterpret_cast<const uchar4 *>(a.keep + t);
+            const int4 s4 = *reinterpret_cast<const int4 *>(a.tt_slots.at(t, TILE_TOK));
+            const uchar4 k4 = *reinterpret_cast<const uchar4 *>(a.keep.at(t, TILE_TOK));
             slot[0] = s4.x; slot[1] = s4.y; slot[2] = s4.z; slot[3] = s4.w;
             kp[0] = k4.x; kp[1] = k4.y; kp[2] = k4.z; kp[3] = k4.w;
         } else {
@@ -365,7 +365,6 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
         st.cut = Sums{0, 0, 0, 0, 0};
         st.cut_r = NO_CUT;
         st.flags = 0;
-        scan_carry = 0;
     }
 
     // running live count at every tile start, from the tile counts in shared memory (above): every thread
@@ -515,7 +514,7 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
         // the destination blocks (up to four loads in flight), then the stores
         int blk[TILE_TOK];
 #pragma unroll
-        for (int k = 0; k < TILE_TOK; ++k) blk[k] = dst[k] >= 0 ? __ldg(a.free_blocks + dst[k]) : 0;
+        for (int k = 0; k < TILE_TOK; ++k) blk[k] = dst[k] >= 0 ? __ldg(a.free_blocks.at(dst[k])) : 0;
 #pragma unroll
         for (int k = 0; k < TILE_TOK; ++k) {
             if (dst[k] < 0) continue;
@@ -523,7 +522,7 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
             a.dst_src[dst[k] * S + off_in_block[k]] = slot[k];
         }
         if (owned && a.vec_out) {
-            *reinterpret_cast<int4 *>(a.new_tt_slots + t) = make_int4(out[0], out[1], out[2], out[3]);
+            *reinterpret_cast<int4 *>(a.new_tt_slots.at(t, TILE_TOK)) = make_int4(out[0], out[1], out[2], out[3]);
         } else {
             // the ragged end of the table, or entries in front of the first request (left untouched)
 #pragma unroll
@@ -540,30 +539,31 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
 int vtk_launch_plan_small(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st)
 {
     PlanArgs a;
-    a.num_requests = in->num_requests;
-    a.bt_offsets = in->bt_offsets;
-    a.bt_blocks = in->bt_blocks;
-    a.tt_offsets = in->tt_offsets;
-    a.tt_slots = in->tt_slots;
-    a.keep = in->keep;
-    a.select = in->select;
+    const vtoken_config &c = ctx->cfg;
+    a.num_requests = VTK_ARR(ctx, in->num_requests, 1);
+    a.bt_offsets = VTK_ARR(ctx, in->bt_offsets, (int64_t)c.max_requests + 1);
+    a.bt_blocks = VTK_ARR(ctx, in->bt_blocks, c.max_table_blocks);
+    a.tt_offsets = VTK_ARR(ctx, in->tt_offsets, (int64_t)c.max_requests + 1);
+    a.tt_slots = VTK_ARR(ctx, in->tt_slots, c.max_tokens);
+    a.keep = VTK_ARR(ctx, in->keep, c.max_tokens);
+    a.select = VTK_ARR(ctx, in->select, c.max_requests);
     a.thr_num = in->thr_num;
     a.thr_den = in->thr_den;
-    a.free_blocks = in->free_blocks;
-    a.num_free = in->num_free;
-    a.new_bt_offsets = out->new_bt_offsets;
-    a.new_bt_blocks = out->new_bt_blocks;
-    a.new_tt_slots = out->new_tt_slots;
-    a.freed_blocks = out->freed_blocks;
-    a.out_status = out->req_status;
-    a.out_counts = out->counts;
-    a.dst_src = ctx->dst_src;
-    a.dst_blocks = ctx->dst_blocks;
-    a.req_n = ctx->req_n;
-    a.tile_n = ctx->tile_n;
-    a.req_part = ctx->req_part;
-    a.header = ctx->plan_header;
-    a.counts = ctx->counts;
+    a.free_blocks = VTK_ARR(ctx, in->free_blocks, c.max_free_blocks);
+    a.num_free = VTK_ARR(ctx, in->num_free, 1);
+    a.new_bt_offsets = VTK_ARR(ctx, out->new_bt_offsets, (int64_t)c.max_requests + 1);
+    a.new_bt_blocks = VTK_ARR(ctx, out->new_bt_blocks, c.max_table_blocks);
+    a.new_tt_slots = VTK_ARR(ctx, out->new_tt_slots, c.max_tokens);
+    a.freed_blocks = VTK_ARR(ctx, out->freed_blocks, c.max_table_blocks);
+    a.out_status = VTK_ARR(ctx, out->req_status, c.max_requests);
+    a.out_counts = VTK_ARR(ctx, out->counts, 1);
+    a.dst_src = VTK_ARR(ctx, ctx->dst_src, (int64_t)ctx->cap_dst_blocks * c.block_size);
+    a.dst_blocks = VTK_ARR(ctx, ctx->dst_blocks, ctx->cap_dst_blocks);
+    a.req_n = VTK_ARR(ctx, ctx->req_n, c.max_requests);
+    a.tile_n = VTK_ARR(ctx, ctx->tile_n, (c.max_tokens + TILE - 1) / TILE + 1);
+    a.req_part = VTK_ARR(ctx, ctx->req_part, (int64_t)c.max_requests + 1);
+    a.header = VTK_ARR(ctx, ctx->plan_header, 4);
+    a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
     a.max_requests = ctx->cfg.max_requests;

@@ -152,3 +152,123 @@ def test_digest_is_invariant_under_repack_and_catches_defects():
         k3 = k2.copy()
         k3[1, new[live[0]], 3] ^= 1                                      # one bit of one K row
         assert vto.digest_logical(k3, v2, new) != after
+
+
+# ---- discriminating power: the digest definition is frozen; these pins say what it must tell apart ----
+def _one_request(seed=9, tokens=40, layers=3, head_dim=32):
+    """One request on an identity layout, everything kept: tt_slots, pools [L, slots, row] of 64-byte rows."""
+    w = wl.tiny(seed=seed, requests=1, lo=tokens, hi=tokens, p_keep=1.0, layers=layers, heads=1, head_dim=head_dim)
+    k, v = pools(w)
+    tt = w.tt_slots[w.tt_offsets[0]:w.tt_offsets[1]].copy()
+    return w, k, v, tt
+
+
+def test_digest_tells_every_word_swap_inside_a_group_apart():
+    """The four 8-byte words of a 32-byte group enter one product: each is bound to its place by its own
+    key, so exchanging any two of them (within a group, across the two groups of a row, across rows)
+    must change the digest."""
+    w, k, v, tt = _one_request()
+    base = vto.digest_logical(k, v, tt)[0]
+    seen = {base}
+    row = k[1, tt[5]].view("<u8")                      # 64-byte row: words 0..3 = group 0, 4..7 = group 1
+    assert len(row) == 8 and len(set(row.tolist())) == 8
+    for a in range(8):
+        for b in range(a + 1, 8):
+            k2 = k.copy()
+            r2 = k2[1, tt[5]].view("<u8")
+            r2[a], r2[b] = row[b], row[a]
+            d = vto.digest_logical(k2, v, tt)[0]
+            assert d not in seen, (a, b)
+            seen.add(d)
+    # the same word pair exchanged between two different rows of the slab
+    k2 = k.copy()
+    x, y = k2[0, tt[3]].view("<u8"), k2[0, tt[4]].view("<u8")
+    x[2], y[2] = k[0, tt[4]].view("<u8")[2], k[0, tt[3]].view("<u8")[2]
+    assert vto.digest_logical(k2, v, tt)[0] not in seen
+
+
+def test_digest_tells_rows_slabs_and_layers_apart():
+    w, k, v, tt = _one_request()
+    base = vto.digest_logical(k, v, tt)[0]
+    # a row exchanged between two requests: request A takes one slot of request B and the other way round
+    w2 = wl.mistral7b_random(seed=8, requests=2, lo=30, hi=60, layers=2, heads=1, head_dim=16, rho_lo=1.0, rho_hi=1.0)
+    k2, v2 = pools(w2)
+    ta = w2.tt_slots[w2.tt_offsets[0]:w2.tt_offsets[1]].copy()
+    tb = w2.tt_slots[w2.tt_offsets[1]:w2.tt_offsets[2]].copy()
+    da, db = vto.digest_logical(k2, v2, ta)[0], vto.digest_logical(k2, v2, tb)[0]
+    ta2, tb2 = ta.copy(), tb.copy()
+    ta2[7], tb2[11] = tb[11], ta[7]
+    assert vto.digest_logical(k2, v2, ta2)[0] != da and vto.digest_logical(k2, v2, tb2)[0] != db
+    # K and V exchanged as a whole, and for one layer only
+    assert vto.digest_logical(v, k, tt)[0] != base
+    k3, v3 = k.copy(), v.copy()
+    k3[1], v3[1] = v[1], k[1]
+    assert vto.digest_logical(k3, v3, tt)[0] != base
+    # layers permuted (both pools alike), every permutation of three layers
+    import itertools
+    seen = {base}
+    for perm in itertools.permutations(range(3)):
+        if perm == (0, 1, 2):
+            continue
+        d = vto.digest_logical(np.ascontiguousarray(k[list(perm)]), np.ascontiguousarray(v[list(perm)]), tt)[0]
+        assert d not in seen, perm
+        seen.add(d)
+    # a sub-range of layers is a different digest from the whole
+    assert vto.digest_logical(k, v, tt, 0, 2)[0] != base
+
+
+def test_digest_of_ten_thousand_single_bit_flips_never_collides():
+    """10 000 different single-bit flips of one request's K/V bytes: every one of them changes the digest
+    (zero collisions with the intact digest).  Two DIFFERENT flips may give the same digest in exactly one
+    way, which the definition implies and this test pins down: words j and j + 2 of a 32-byte group are
+    added before the multiply, so flipping the same bit position in both moves the sum by the same power
+    of two when the two bits agree (after the per-word keys); every collision among the flips must be of
+    that kind.  (The digest is a relocation check -- rows, tokens, slabs, words in the wrong place -- not
+    an error-correcting code.)  Evaluated incrementally: the digest is a sum over (token, slab, group)
+    terms, so a flip changes exactly one term, recomputed here with numpy and checked against the oracle
+    on a sample."""
+    w, k, v, tt = _one_request(tokens=64, layers=4, head_dim=64)        # 128-byte rows, 8 slabs
+    L, n = k.shape[0], len(tt)
+    base = vto.digest_logical(k, v, tt)[0]
+    rng = np.random.default_rng(5)
+    M = (1 << 64) - 1
+    row_bits = k.shape[2] * 16
+
+    def term(kk, vv, tok, slab):
+        """Digest contribution of (token tok, slab): numpy evaluation of the one row with its own key."""
+        src = (kk if slab < L else vv)[slab % L, tt[tok]]
+        words = np.ascontiguousarray(src).view("<u8").astype(np.uint64)[None, None, :]
+        with np.errstate(over="ignore"):
+            key = mix(np.array([((tok * A + tok) * B + slab) * C & M], dtype=np.uint64))[None, None, :]
+            j = np.arange(words.shape[-1], dtype=np.uint64)[None, None, :]
+            x = words ^ (key + j * np.uint64(D))
+            a_, b_ = x[..., 0::4] + x[..., 2::4], x[..., 1::4] + x[..., 3::4]
+            return int(fold128(a_, b_).sum(dtype=np.uint64))
+
+    # the decomposition is exact: the sum of all terms is the oracle's digest (rank == id here: every token kept)
+    assert sum(term(k, v, t, s) for t in range(n) for s in range(2 * L)) & M == base
+    seen = {}
+    checked_in_full = 0
+    collisions = 0
+    flips = rng.choice(n * 2 * L * row_bits, size=10000, replace=False)         # 10 000 different bits
+    for trial, f in enumerate(flips.tolist()):
+        tok, slab, bit = f // (2 * L * row_bits), f // row_bits % (2 * L), f % row_bits
+        pool = k if slab < L else v
+        old = term(k, v, tok, slab)
+        pool[slab % L, tt[tok], bit // 16] ^= np.uint16(1 << (bit % 16))
+        new = term(k, v, tok, slab)
+        d = (base - old + new) & M
+        if trial % 500 == 0:                                            # the shortcut against the oracle itself
+            assert vto.digest_logical(k, v, tt)[0] == d
+            checked_in_full += 1
+        pool[slab % L, tt[tok], bit // 16] ^= np.uint16(1 << (bit % 16))
+        assert d != base, (tok, slab, bit)                              # every flip is detected
+        if d in seen:
+            tok2, slab2, bit2 = seen[d]
+            # same token, slab and group, same bit position, words two apart
+            assert (tok2, slab2) == (tok, slab) and bit2 // 256 == bit // 256 and bit2 % 64 == bit % 64 and \
+                abs(bit2 // 64 - bit // 64) == 2, ((tok, slab, bit), (tok2, slab2, bit2))
+            collisions += 1
+        seen[d] = (tok, slab, bit)
+    assert checked_in_full == 20 and len(seen) + collisions == 10000
+    assert collisions < 150                                             # about 50 expected from the pair count

@@ -152,6 +152,8 @@ class DeviceProblem:
                                req_append_pos=torch.full((self.max_requests,), -9, **i32),
                                free_out=torch.full((self.max_free,), -9, **i32),
                                num_free_out=torch.full((1,), -9, **i32),
+                               released=torch.full((self.max_table_blocks,), -9, **i32),
+                               num_released=torch.full((1,), -9, **i32),
                                counts=torch.zeros((num_waves, 8), **i32),
                                workspace=torch.empty(max(16, nbytes), dtype=torch.uint8, device=dev), nbytes=nbytes)
         wv = self._waves
@@ -164,7 +166,8 @@ class DeviceProblem:
                                free_out=wv["free_out"], num_free_out=wv["num_free_out"], wave_counts=wv["counts"],
                                free_capacity=self.max_free, workspace=wv["workspace"], workspace_bytes=wv["nbytes"],
                                select=self.select, thr_num=self.w.thr_num, thr_den=self.w.thr_den, partial=partial,
-                               req_append_pos=wv["req_append_pos"], stream=stream)
+                               req_append_pos=wv["req_append_pos"], released_blocks=wv["released"],
+                               num_released=wv["num_released"], stream=stream)
 
     def waves_outputs(self, num_waves: int) -> dict:
         """Host copies of the outputs of ``repack_waves``."""
@@ -184,6 +187,7 @@ class DeviceProblem:
         out["req_append_pos"] = wv["req_append_pos"].cpu().numpy()[:R]
         nfo = int(wv["num_free_out"].item())
         out["free_out"] = wv["free_out"].cpu().numpy()[:nfo]
+        out["released_blocks"] = wv["released"].cpu().numpy()[:int(wv["num_released"].item())]
         return out
 
     def read_counts(self, stream=None) -> dict:

@@ -299,8 +299,9 @@ typedef struct {
  * reference counts decide when such a block is free) instead of freed_blocks; counts.num_released
  * says how many.  max_source_blocks bounds the unprotected sources only.  The gain gate is unchanged
  * (destinations < sources, in the request's own table), so whether the POOL gains depends on the
- * other holders: enabling detach is the caller's policy decision.  Not available in
- * vtoken_repack_waves and vtoken_repack_host_partial (VTOKEN_EINVAL). */
+ * other holders: enabling detach is the caller's policy decision.  vtoken_repack_waves and
+ * vtoken_repack_host_partial take the threshold too; each has a released list of its own in its
+ * output struct. */
 int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
                         const vtoken_plan_out *out, void *cuda_stream);
 
@@ -340,6 +341,10 @@ typedef struct {                   /* all DEVICE pointers, written by vtoken_rep
                                       VTOKEN_FLAG_CAPACITY is raised */
     void *workspace;               /* DEVICE scratch, 16-byte aligned, owned by the caller */
     int64_t workspace_bytes;       /* >= vtoken_waves_workspace_bytes (VTOKEN_ECAPACITY otherwise) */
+    int32_t *released_blocks;      /* capacity max_table_blocks: references to shared blocks dropped by the waves'
+                                      copy-on-write detaches, wave after wave (wave_counts[k].num_released each);
+                                      needed when opts has a detach threshold, may be NULL otherwise */
+    int32_t *num_released;         /* device scalar or NULL: entries of released_blocks after the last wave */
 } vtoken_waves_out;
 
 /* Bytes of workspace vtoken_repack_waves needs for this context and free_capacity. */
@@ -469,12 +474,15 @@ typedef struct {                   /* all HOST pointers */
     int32_t *freed_blocks;         /* [bt_offsets[R]] */
     int32_t *req_status;           /* [R] */
     vtoken_counts *counts;
+    int32_t *released_blocks;      /* [bt_offsets[R]] or NULL: references dropped by a copy-on-write detach
+                                      (vtoken_repack_host_partial with a detach threshold; counts->num_released) */
 } vtoken_host_tables;
 int vtoken_repack_host(vtoken_ctx *ctx, const vtoken_host_tables *tables, void *cuda_stream);
 
 /* The same front end with the partial planner (vtoken_plan_partial): opts as there, except that
  * opts->protect, when given, is a HOST array of num_blocks bytes (copied to the device with the
- * tables).  opts must not be NULL. */
+ * tables).  opts must not be NULL.  With a detach threshold tables->released_blocks must be given
+ * (VTOKEN_EINVAL otherwise). */
 int vtoken_repack_host_partial(vtoken_ctx *ctx, const vtoken_host_tables *tables, const vtoken_partial_opts *opts,
                                void *cuda_stream);
 

@@ -459,6 +459,7 @@ class WavePlan:
     move_dst: np.ndarray
     wave_move_offsets: np.ndarray
     wave_counts: list             # one dict per wave
+    released_blocks: np.ndarray = None    # references dropped by copy-on-write detaches, wave after wave
 
 
 def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_waves, select=None,
@@ -485,9 +486,10 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
     o, protect = None, None
     if partial is not None:
         protect = _u8(partial.get("protect"))
-        util, theta = partial.get("util", (0, 0)), partial.get("theta", (0, 0))
+        util, theta, detach = partial.get("util", (0, 0)), partial.get("theta", (0, 0)), partial.get("detach", (0, 0))
         o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1],
-                         partial.get("max_source_blocks", 0), theta[0], theta[1], 0, 0)
+                         partial.get("max_source_blocks", 0), theta[0], theta[1], detach[0], detach[1])
+    released = np.full(max(nbt, 1), -7, np.int32)
     rc = lib().vto_plan_waves(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
                               _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
                               _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),
@@ -496,7 +498,7 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
                               ctypes.c_int32(num_waves), _p(new_bt_offsets, np.int32), _p(new_bt_blocks, np.int32),
                               _p(new_tt_slots, np.int32), _p(status, np.int32), _p(wave, np.int32),
                               _p(apos, np.int32), _p(free_out, np.int32), ctypes.byref(nfo), _p(msrc, np.int32), _p(mdst, np.int32),
-                              ctypes.c_int64(cap), offs.ctypes.data_as(ctypes.c_void_p), counts)
+                              ctypes.c_int64(cap), offs.ctypes.data_as(ctypes.c_void_p), counts, _p(released, np.int32))
     if rc != 0:
         raise ValueError(f"vto_plan_waves failed: {rc}")
     total = int(offs[num_waves])
@@ -504,4 +506,4 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
     return WavePlan(new_bt_offsets, new_bt_blocks[:int(new_bt_offsets[R])].copy(), new_tt_slots[:T].copy(),
                     status[:R].copy(), wave[:R].copy(), apos[:R].copy(), free_out[:nfo.value].copy(),
                     msrc[:total].copy(),
-                    mdst[:total].copy(), offs, wc)
+                    mdst[:total].copy(), offs, wc, released[:sum(c["num_released"] for c in wc)].copy())

@@ -774,12 +774,12 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
                    int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
                    int32_t *req_status, int32_t *req_wave, int32_t *req_append_pos, int32_t *free_out,
                    int32_t *num_free_out, int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
-                   int64_t *wave_move_offsets, vto_counts *wave_counts)
+                   int64_t *wave_move_offsets, vto_counts *wave_counts, int32_t *released_blocks)
 {
     if (R < 0 || S < 1 || num_free < 0 || num_waves < 1 || !bt_offsets || !tt_offsets || !num_free_out ||
         !wave_move_offsets || !wave_counts)
         return VTO_EINVAL;
-    if (opts && opts->detach_den != 0) return VTO_EINVAL;   /* detach is an option of single plans */
+    if (opts && opts->detach_den != 0 && !released_blocks) return VTO_EINVAL;   /* a detach needs its list */
     const int64_t T = tt_offsets[R], nbt = bt_offsets[R];
     const size_t nT = (size_t)(T > 0 ? T : 1), nB = (size_t)(nbt > 0 ? nbt : 1), nR = (size_t)R + 1;
     const size_t nP = (size_t)num_free + nB;
@@ -791,9 +791,11 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
     int32_t *pool = malloc(nP * sizeof(int32_t)), *pool_next = malloc(nP * sizeof(int32_t));
     int32_t *freed = malloc(nB * sizeof(int32_t)), *status = malloc(nR * sizeof(int32_t));
     int32_t *msrc = malloc(nT * sizeof(int32_t)), *mdst = malloc(nT * sizeof(int32_t));
+    int32_t *rel = malloc(nB * sizeof(int32_t));
+    int64_t total_released = 0;
     int rc = VTO_OK;
     if (!cur_bto || !nxt_bto || !cur_btb || !nxt_btb || !cur_tts || !nxt_tts || !pool || !pool_next || !freed ||
-        !status || !msrc || !mdst) {
+        !status || !msrc || !mdst || !rel) {
         rc = VTO_EINVAL;
         goto done;
     }
@@ -815,12 +817,15 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
         /* one planning round against the pool as it stands (Sec. 3.3.2 admission, 3.3.3 planning) */
         if (opts)
             rc = vto_plan_partial(R, S, NB, cur_bto, cur_btb, tt_offsets, cur_tts, keep, select, thr_num, thr_den,
-                                  pool, pool_n, opts, nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c, NULL);
+                                  pool, pool_n, opts, nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c, rel);
         else
             rc = vto_plan(R, S, cur_bto, cur_btb, tt_offsets, cur_tts, keep, select, thr_num, thr_den, pool, pool_n,
                           nxt_bto, nxt_btb, nxt_tts, freed, status, msrc, mdst, &c);
         if (rc != VTO_OK) goto done;
         wave_counts[k] = c;
+        /* references to shared blocks dropped by this wave's detaches, in wave order (a request that has left
+         * its shared blocks no longer lists them, so no reference is dropped twice) */
+        for (int32_t i = 0; opts && released_blocks && i < c.num_released; ++i) released_blocks[total_released++] = rel[i];
         /* its copies, in wave order */
         if (total_moves + c.num_moves > move_capacity) {
             rc = VTO_EINVAL;
@@ -873,7 +878,7 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
     *num_free_out = pool_n;
 done:
     free(cur_bto); free(nxt_bto); free(cur_btb); free(nxt_btb); free(cur_tts); free(nxt_tts);
-    free(pool); free(pool_next); free(freed); free(status); free(msrc); free(mdst);
+    free(pool); free(pool_next); free(freed); free(status); free(msrc); free(mdst); free(rel);
     return rc;
 }
 

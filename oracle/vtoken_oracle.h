@@ -292,6 +292,8 @@ int vto_digest_logical(const uint8_t *k_pool, const uint8_t *v_pool, int64_t lay
  * wave_counts[num_waves] = counts of every wave; move_src / move_dst = the move lists of all
  * waves back to back, wave k in [wave_move_offsets[k], wave_move_offsets[k+1]) -- they must be
  * applied in this order, because a later wave overwrites blocks an earlier wave has read.
+ * released_blocks (capacity: total old blocks; may be NULL without a detach threshold) = the references to
+ * shared blocks the waves' copy-on-write detaches dropped, wave after wave (wave_counts[k].num_released each).
  * Returns VTO_EINVAL when move_capacity is too small. */
 int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
                    const int32_t *bt_offsets, const int32_t *bt_blocks,
@@ -302,7 +304,7 @@ int vto_plan_waves(int32_t R, int32_t S, int32_t NB,
                    int32_t *new_bt_offsets, int32_t *new_bt_blocks, int32_t *new_tt_slots,
                    int32_t *req_status, int32_t *req_wave, int32_t *req_append_pos, int32_t *free_out,
                    int32_t *num_free_out, int32_t *move_src, int32_t *move_dst, int64_t move_capacity,
-                   int64_t *wave_move_offsets, vto_counts *wave_counts);
+                   int64_t *wave_move_offsets, vto_counts *wave_counts, int32_t *released_blocks);
 
 int vto_openmp_threads(void);   /* max OpenMP threads of this build, 1 when built without */
 

@@ -89,7 +89,8 @@ class WavesOut(ctypes.Structure):
                 ("new_tt_slots", ctypes.c_void_p), ("req_status", ctypes.c_void_p), ("req_wave", ctypes.c_void_p),
                 ("req_append_pos", ctypes.c_void_p), ("free_out", ctypes.c_void_p), ("num_free_out", ctypes.c_void_p), ("wave_counts", ctypes.c_void_p),
                 ("free_capacity", ctypes.c_int32), ("workspace", ctypes.c_void_p),
-                ("workspace_bytes", ctypes.c_int64)]
+                ("workspace_bytes", ctypes.c_int64), ("released_blocks", ctypes.c_void_p),
+                ("num_released", ctypes.c_void_p)]
 
 
 class HostTables(ctypes.Structure):
@@ -101,7 +102,7 @@ class HostTables(ctypes.Structure):
                 ("free_blocks", ctypes.c_void_p), ("num_free", ctypes.c_int32),
                 ("new_bt_offsets", ctypes.c_void_p), ("new_bt_blocks", ctypes.c_void_p),
                 ("new_tt_slots", ctypes.c_void_p), ("freed_blocks", ctypes.c_void_p),
-                ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p)]
+                ("req_status", ctypes.c_void_p), ("counts", ctypes.c_void_p), ("released_blocks", ctypes.c_void_p)]
 
 
 _lib = None
@@ -296,14 +297,15 @@ def vtoken_repack_host(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, 
 def vtoken_repack_host_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
                                num_free, new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status,
                                select=None, thr_num=0, thr_den=0, protect=None, util=(0, 0), max_source_blocks=0,
-                               theta=(0, 0), stream=None) -> dict:
-    """vtoken_repack_host with the partial planner; ``protect`` is a HOST array of num_blocks bytes."""
+                               theta=(0, 0), detach=(0, 0), released_blocks=None, stream=None) -> dict:
+    """vtoken_repack_host with the partial planner; ``protect`` is a HOST array of num_blocks bytes,
+    ``released_blocks`` a HOST array of bt_offsets[R] entries (needed with a detach threshold)."""
     c = Counts()
     h = HostTables(num_requests, _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                    _ptr(select), thr_num, thr_den, _ptr(free_blocks), num_free, _ptr(new_bt_offsets),
                    _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks), _ptr(req_status),
-                   ctypes.addressof(c))
-    po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1])
+                   ctypes.addressof(c), _ptr(released_blocks))
+    po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1], detach[0], detach[1])
     _check(load().vtoken_repack_host_partial(ctx, ctypes.byref(h), ctypes.byref(po), _stream(stream)),
            "vtoken_repack_host_partial", ctx)
     return c.as_dict()
@@ -452,14 +454,15 @@ def vtoken_waves_workspace_bytes(ctx, free_capacity: int) -> int:
 def vtoken_repack_waves(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
                         num_waves, new_bt_offsets, new_bt_blocks, new_tt_slots, req_status, req_wave, free_out,
                         num_free_out, wave_counts, free_capacity, workspace, workspace_bytes, select=None, thr_num=0,
-                        thr_den=0, partial=None, req_append_pos=None, stream=None) -> None:
+                        thr_den=0, partial=None, req_append_pos=None, released_blocks=None, num_released=None,
+                        stream=None) -> None:
     """``partial``: None for the whole-request planner, else a dict with the option keywords of
-    vtoken_plan_partial (protect, util, max_source_blocks, theta)."""
+    vtoken_plan_partial (protect, util, max_source_blocks, theta, detach)."""
     pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                  _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
     wout = WavesOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(req_status), _ptr(req_wave),
                     _ptr(req_append_pos), _ptr(free_out), _ptr(num_free_out), _ptr(wave_counts), free_capacity, _ptr(workspace),
-                    workspace_bytes)
+                    workspace_bytes, _ptr(released_blocks), _ptr(num_released))
     po = None
     if partial is not None:
         util, theta = partial.get("util", (0, 0)), partial.get("theta", (0, 0))

@@ -31,7 +31,7 @@ void free_all(vtoken_ctx *ctx)
                     ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
                     ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
                     ctx->stage.new_tt_slots, ctx->stage.freed_blocks, ctx->stage.req_status, ctx->stage.counts,
-                    ctx->stage.protect};
+                    ctx->stage.protect, ctx->stage.released_blocks};
     for (void *p : ptrs)
         if (p) cudaFree(p);
     if (ctx->stage.h_scalars) cudaFreeHost(ctx->stage.h_scalars);
@@ -224,7 +224,8 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
 {
     if (!ctx || !h) return VTOKEN_EINVAL;
     if (opts && opts->max_source_blocks < 0) return VTOKEN_EINVAL;
-    if (opts && opts->detach_den != 0) return VTOKEN_EINVAL;    // the host front end has no released list
+    const bool detach = opts && opts->protect != nullptr && opts->detach_den != 0;
+    if (detach && !h->released_blocks) return VTOKEN_EINVAL;    // a detach threshold needs the list of dropped references
     if (!h->bt_offsets || !h->bt_blocks || !h->tt_offsets || !h->tt_slots || !h->keep || !h->free_blocks ||
         !h->new_bt_offsets || !h->new_bt_blocks || !h->new_tt_slots || !h->freed_blocks || !h->req_status ||
         !h->counts)
@@ -283,6 +284,13 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
     out.req_status = s.req_status;
     out.counts = s.counts;
     out.released_blocks = nullptr;
+    if (detach) {
+        if (!s.released_blocks) {                     // device copy of the released list, on first use
+            rc = dev_alloc(ctx, &s.released_blocks, ctx->cfg.max_table_blocks);
+            if (rc != VTOKEN_OK) return rc;
+        }
+        out.released_blocks = s.released_blocks;
+    }
     if (opts) {
         vtoken_partial_opts dopts = *opts;
         dopts.protect = opts->protect ? s.protect : nullptr;
@@ -305,6 +313,7 @@ static int repack_host(vtoken_ctx *ctx, const vtoken_host_tables *h, const vtoke
     if (T) D2H(h->new_tt_slots, s.new_tt_slots, T * sizeof(int32_t));
     if (NBT) D2H(h->freed_blocks, s.freed_blocks, NBT * sizeof(int32_t));
     if (R) D2H(h->req_status, s.req_status, R * sizeof(int32_t));
+    if (detach && NBT) D2H(h->released_blocks, s.released_blocks, NBT * sizeof(int32_t));
     VTK_CUDA(ctx, cudaEventRecord(s.copied, s.aux));
     st = caller;
     VTK_CUDA(ctx, cudaStreamWaitEvent(st, s.copied, 0));

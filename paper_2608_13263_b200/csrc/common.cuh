@@ -72,6 +72,7 @@ struct vtoken_ctx {
         int32_t *bt_offsets, *bt_blocks, *tt_offsets, *tt_slots, *free_blocks;
         uint8_t *keep, *select;
         uint8_t *protect;              // [num_blocks], vtoken_repack_host_partial only (allocated on first use)
+        int32_t *released_blocks;      // [max_table_blocks], vtoken_repack_host_partial with a detach threshold (first use)
         int32_t *new_bt_offsets, *new_bt_blocks, *new_tt_slots, *freed_blocks, *req_status;
         vtoken_counts *counts;
         int32_t *h_scalars;            // HOST, pinned mirror of the small inputs of the call in flight: {num_requests,

@@ -25,6 +25,12 @@ struct CommitArgs {
     const vtoken_counts *ctx_counts;  // the context's copy: carries the flags raised by the copy kernel
     int32_t *pool_next, *num_pool_next;
     int32_t free_capacity;
+    // references dropped by copy-on-write detaches: this wave's list goes behind those of the waves before it
+    const int32_t *released_k;        // or NULL
+    const vtoken_counts *all_counts;  // counts of the waves so far ([wave + 1])
+    int32_t *released_out, *num_released_out;
+    int64_t released_capacity;
+    int32_t last;                     // 1: the last wave (writes the total)
 };
 
 __global__ void __launch_bounds__(COMMIT_NT) wave_commit_kernel(CommitArgs a)
@@ -67,6 +73,15 @@ __global__ void __launch_bounds__(COMMIT_NT) wave_commit_kernel(CommitArgs a)
     }
     for (int i = gtid; i < (int)total; i += gsz)
         a.pool_next[i] = i < rest ? a.pool[consumed + i] : a.freed[i - rest];
+    if (a.released_k != nullptr) {
+        int64_t base = 0;
+        for (int k = 0; k < a.wave; ++k) base += a.all_counts[k].num_released;
+        const int n = a.wave_counts->num_released;
+        for (int i = gtid; i < n && base + i < a.released_capacity; i += gsz) a.released_out[base + i] = a.released_k[i];
+        if (gtid == 0 && a.last && a.num_released_out != nullptr) *a.num_released_out = (int32_t)(base + n);
+    } else if (gtid == 0 && a.last && a.num_released_out != nullptr) {
+        *a.num_released_out = 0;
+    }
     if (gtid == 0) {
         *a.num_pool_next = (int)total;
         a.wave_counts->error_flags |= a.ctx_counts->error_flags | (over ? VTOKEN_FLAG_CAPACITY : 0u);
@@ -74,7 +89,7 @@ __global__ void __launch_bounds__(COMMIT_NT) wave_commit_kernel(CommitArgs a)
 }
 
 struct Layout {                       // workspace carve-up, every part 16-byte aligned
-    int64_t freed, status, num_pool, pool, bt_offsets, bt_blocks, tt_slots, total;
+    int64_t freed, released, status, num_pool, pool, bt_offsets, bt_blocks, tt_slots, total;
 };
 
 Layout layout_of(const vtoken_ctx *ctx, int32_t free_capacity)
@@ -84,6 +99,7 @@ Layout layout_of(const vtoken_ctx *ctx, int32_t free_capacity)
     Layout l;
     int64_t o = 0;
     l.freed = o;      o += up(4 * c.max_table_blocks);
+    l.released = o;   o += up(4 * c.max_table_blocks);
     l.status = o;     o += up(4 * (int64_t)c.max_requests);
     l.num_pool = o;   o += 16;
     l.pool = o;       o += up(4 * (int64_t)(free_capacity > 1 ? free_capacity : 1));
@@ -115,7 +131,8 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         !out->free_out || !out->num_free_out || !out->wave_counts || !out->workspace)
         return VTOKEN_EINVAL;
     if (out->free_capacity < 0 || ((uintptr_t)out->workspace & 15)) return VTOKEN_EINVAL;
-    if (opts && opts->detach_den != 0) return VTOKEN_EINVAL;     // detach is an option of single plans
+    const bool detach = opts && opts->protect != nullptr && opts->detach_den != 0;
+    if (detach && !out->released_blocks) return VTOKEN_EINVAL;   // a detach threshold needs the list of dropped references
     if (out->free_capacity > ctx->cfg.max_free_blocks) return VTOKEN_ECAPACITY;
     const Layout l = layout_of(ctx, out->free_capacity);
     if (out->workspace_bytes < l.total) return VTOKEN_ECAPACITY;
@@ -140,7 +157,7 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         po.freed_blocks = at(l.freed);
         po.req_status = at(l.status);
         po.counts = out->wave_counts + k;
-        po.released_blocks = nullptr;
+        po.released_blocks = detach ? at(l.released) : nullptr;
         int rc = opts ? vtoken_plan_partial(ctx, &cur, opts, &po, cuda_stream) : vtoken_plan(ctx, &cur, &po, cuda_stream);
         if (rc != VTOKEN_OK) return rc;
         rc = vtk_launch_copy(ctx, st);
@@ -165,6 +182,12 @@ int vtoken_repack_waves(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
         a.pool_next = pool[w];
         a.num_pool_next = num_pool[w];
         a.free_capacity = out->free_capacity;
+        a.released_k = detach ? po.released_blocks : nullptr;
+        a.all_counts = out->wave_counts;
+        a.released_out = out->released_blocks;
+        a.num_released_out = out->num_released;
+        a.released_capacity = ctx->cfg.max_table_blocks;
+        a.last = k == num_waves - 1;
         int64_t span = out->free_capacity > ctx->cfg.max_requests ? out->free_capacity : ctx->cfg.max_requests;
         int blocks = (int)((span + COMMIT_NT - 1) / COMMIT_NT);
         if (blocks < 1) blocks = 1;

@@ -272,7 +272,7 @@ def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach):
     prob.close()
 
 
-def test_detach_needs_a_released_list_and_is_refused_by_the_composite_entry_points():
+def test_detach_needs_a_released_list_everywhere():
     import torch
     from harness.device import DeviceProblem
     w, protect = wl.shared_prefix(seed=3, groups=1, degree=2, prefix_len=64, suffix_len=80, layers=1, heads=1,
@@ -285,7 +285,81 @@ def test_detach_needs_a_released_list_and_is_refused_by_the_composite_entry_poin
         prob.plan_partial(protect=prot, detach=(1, 1))
     assert e.value.code == vt.EINVAL
     prob.released_blocks = saved
+    # the wave entry point and the host front end want a list of their own
+    prob.repack_waves(2, partial=dict(protect=prot, util=(1, 1)))          # allocates the wave buffers
+    wv = prob._waves
+    args = dict(num_requests=prob.num_requests, bt_offsets=prob.bt_offsets, bt_blocks=prob.bt_blocks,
+                tt_offsets=prob.tt_offsets, tt_slots=prob.tt_slots, keep=prob.keep, free_blocks=prob.free_blocks,
+                num_free=prob.num_free, num_waves=2, new_bt_offsets=prob.new_bt_offsets,
+                new_bt_blocks=prob.new_bt_blocks, new_tt_slots=prob.new_tt_slots, req_status=prob.req_status,
+                req_wave=wv["req_wave"], free_out=wv["free_out"], num_free_out=wv["num_free_out"],
+                wave_counts=wv["counts"], free_capacity=prob.max_free, workspace=wv["workspace"],
+                workspace_bytes=wv["nbytes"])
     with pytest.raises(vt.VtokenError) as e:
-        prob.repack_waves(2, partial=dict(protect=prot, detach=(1, 1)))
+        vt.vtoken_repack_waves(prob.ctx, partial=dict(protect=prot, detach=(1, 1)), **args)
     assert e.value.code == vt.EINVAL
+    prob.close()
+
+
+@pytest.mark.parametrize("degree", [2, 4])
+@pytest.mark.parametrize("detach", [(1, 1), (1, 2)], ids=lambda d: f"detach{d[0]}_{d[1]}")
+def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, detach):
+    """Copy-on-write detach through vtoken_repack_waves (references dropped wave after wave, in one list)
+    and through vtoken_repack_host_partial (host tables in and out): tables, lists and every byte of both
+    pools against the oracle."""
+    import torch
+    from harness.device import DeviceProblem, origin_map
+    w, protect = wl.shared_prefix(seed=7, groups=2, degree=degree, prefix_len=256, suffix_len=600, layers=2, heads=1,
+                                  head_dim=64)
+    opts = dict(util=(1, 1), max_source_blocks=12, detach=detach)
+    # ---- waves with a short pool: the detaches are spread over several waves
+    need = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                            w.free_blocks, protect=protect, **opts).num_dst_blocks
+    nf = max(2, need // 3)
+    W = 4
+    v = vto.plan_waves(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                       w.free_blocks[:nf], W, partial=dict(protect=protect, **opts))
+    prob = DeviceProblem(w, fill_seed=FILL_SEED, wave_capacity=True)
+    prot = torch.from_numpy(protect).to(prob.device)
+    nf_dev = torch.tensor([nf], dtype=torch.int32, device=prob.device)
+    prob.repack_waves(W, num_free=nf_dev, partial=dict(protect=prot, **opts))
+    out = prob.waves_outputs(W)
+    assert all(c["error_flags"] == 0 for c in out["wave_counts"])
+    assert [c["num_moves"] for c in out["wave_counts"]] == [c["num_moves"] for c in v.wave_counts]
+    assert np.array_equal(out["new_tt_slots"], v.new_tt_slots) and np.array_equal(out["new_bt_blocks"], v.new_bt_blocks)
+    assert np.array_equal(out["new_bt_offsets"], v.new_bt_offsets) and np.array_equal(out["req_status"], v.req_status)
+    assert np.array_equal(out["free_out"], v.free_out) and np.array_equal(out["req_wave"], v.req_wave)
+    assert np.array_equal(out["released_blocks"], v.released_blocks)
+    if detach == (1, 1):
+        assert len(v.released_blocks) > 0 and sum(1 for c in v.wave_counts if c["num_released"]) >= 1
+    assert prob.verify_pools(origin_map(w.slots_per_layer, v.move_src, v.move_dst, v.wave_move_offsets)) == 0
+    assert (prob._waves["released"][len(v.released_blocks):].cpu().numpy() == -9).all()
+    prob.close()
+
+    # ---- the host front end
+    p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                         w.free_blocks, protect=protect, **opts)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    R, T, NBT = w.num_requests, w.num_tokens, len(w.bt_blocks)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    h_in = dict(bt_offsets=pin(w.bt_offsets), bt_blocks=pin(w.bt_blocks), tt_offsets=pin(w.tt_offsets),
+                tt_slots=pin(w.tt_slots), keep=pin(w.keep), free_blocks=pin(w.free_blocks))
+    h_out = dict(new_bt_offsets=torch.zeros(R + 1, dtype=torch.int32).pin_memory(),
+                 new_bt_blocks=torch.zeros(NBT, dtype=torch.int32).pin_memory(),
+                 new_tt_slots=torch.zeros(T, dtype=torch.int32).pin_memory(),
+                 freed_blocks=torch.zeros(NBT, dtype=torch.int32).pin_memory(),
+                 req_status=torch.zeros(R, dtype=torch.int32).pin_memory(),
+                 released_blocks=torch.full((NBT,), -9, dtype=torch.int32).pin_memory())
+    with pytest.raises(vt.VtokenError) as e:                 # no released list: refused before anything is enqueued
+        vt.vtoken_repack_host_partial(prob.ctx, num_requests=R, num_free=len(w.free_blocks), protect=protect, **opts,
+                                      **h_in, **{k: x for k, x in h_out.items() if k != "released_blocks"})
+    assert e.value.code == vt.EINVAL
+    c = vt.vtoken_repack_host_partial(prob.ctx, num_requests=R, num_free=len(w.free_blocks), protect=protect, **opts,
+                                      **h_in, **h_out)
+    assert c["error_flags"] == 0 and c["num_moves"] == p.num_moves and c["num_released"] == len(p.released_blocks)
+    assert np.array_equal(h_out["new_tt_slots"].numpy(), p.new_tt_slots)
+    assert np.array_equal(h_out["new_bt_blocks"].numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
+    assert np.array_equal(h_out["freed_blocks"].numpy()[:p.num_freed], p.freed_blocks)
+    assert np.array_equal(h_out["released_blocks"].numpy()[:c["num_released"]], p.released_blocks)
+    assert prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst)) == 0
     prob.close()

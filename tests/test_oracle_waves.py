@@ -237,3 +237,70 @@ def test_move_list_order_matters_when_blocks_are_reused():
     order = np.concatenate([np.arange(o[1], o[-1]), np.arange(0, o[1])])       # wave 0 last
     vto.apply_moves_slab(bad, v.move_src[order], v.move_dst[order])
     assert not np.array_equal(bad[v.new_tt_slots[live], 0], w.tt_slots[live])
+
+
+@pytest.mark.parametrize("degree", [1, 2, 4])
+@pytest.mark.parametrize("detach", [Fraction(1, 1), Fraction(1, 2), Fraction(1, 8)])
+def test_waves_with_copy_on_write_detach_against_a_replay(degree, detach):
+    """Repack in waves on the shared-prefix workload with a detach threshold: wave by wave the definition
+    twin plans on what the previous wave committed; tables, pool, statuses and the list of dropped
+    references (wave after wave, each reference once) must be the oracle's, one wave must equal the single
+    partial plan, and every request must still see exactly its own payloads -- shared blocks keep their
+    bytes for the sharers that stayed."""
+    w, protect = wl.shared_prefix(seed=3, groups=2, degree=degree, prefix_len=48, suffix_len=150, layers=1, heads=1,
+                                  head_dim=8, block_size=4)
+    S, R = w.block_size, w.num_requests
+    prot = set(np.flatnonzero(protect).tolist())
+    opts = dict(protect=protect, util=(1, 1), max_source_blocks=6, detach=(detach.numerator, detach.denominator))
+    twin_kw = dict(protect=prot, util=Fraction(1, 1), max_sources=6, detach=detach)
+    one = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                           w.free_blocks, **opts)
+    v1 = vto.plan_waves(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks, 1,
+                        partial=opts)
+    assert np.array_equal(v1.new_tt_slots, one.new_tt_slots) and np.array_equal(v1.new_bt_blocks, one.new_bt_blocks)
+    assert np.array_equal(v1.released_blocks, one.released_blocks) and v1.wave_counts[0]["num_released"] == len(one.released_blocks)
+
+    need = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                            w.free_blocks, **opts).num_dst_blocks
+    for nf in sorted({max(1, need // 5), max(2, need // 2), need}):
+        free = w.free_blocks[:nf].tolist()
+        v = vto.plan_waves(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, free, 5,
+                           partial=opts)
+        # the replay: dictionary of slot contents (a slot's content is named by the slot it was filled in)
+        bt = [w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]].tolist() for r in range(R)]
+        tt = [w.tt_slots[w.tt_offsets[r]:w.tt_offsets[r + 1]].tolist() for r in range(R)]
+        keeps = [w.keep[w.tt_offsets[r]:w.tt_offsets[r + 1]].tolist() for r in range(R)]
+        content = {s: s for s in range(w.slots_per_layer)}
+        pool, released, status = list(free), [], [0] * R
+        per_wave = []
+        for k in range(5):
+            d = repack_partial_definition(S, bt, tt, keeps, pool, **twin_kw)
+            for src, dst in d["moves"]:
+                content[dst] = content[src]
+            for r in range(R):
+                status[r] = 1 if d["status"][r] == 1 else (status[r] if status[r] == 1 else d["status"][r])
+            bt, tt = d["new_bt"], d["new_tt"]
+            pool = pool[d["consumed"]:] + d["freed"]
+            released += d["released"]
+            per_wave.append(len(d["released"]))
+        for r in range(R):
+            assert v.new_bt_blocks[v.new_bt_offsets[r]:v.new_bt_offsets[r + 1]].tolist() == bt[r]
+            assert v.new_tt_slots[w.tt_offsets[r]:w.tt_offsets[r + 1]].tolist() == tt[r]
+        assert v.free_out.tolist() == pool and v.req_status.tolist() == status
+        assert v.released_blocks.tolist() == released
+        assert [c["num_released"] for c in v.wave_counts] == per_wave
+        # the oracle's own move list, in its order, leaves every live token with the content of its old slot
+        mine = {s: s for s in range(w.slots_per_layer)}
+        for s, dd in zip(v.move_src.tolist(), v.move_dst.tolist()):
+            mine[dd] = mine[s]
+        for r in range(R):
+            old = w.tt_slots[w.tt_offsets[r]:w.tt_offsets[r + 1]].tolist()
+            for t, s in enumerate(tt[r]):
+                if s >= 0:
+                    assert keeps[r][t] and mine[s] == old[t] and content[s] == old[t]
+        # a reference is dropped at most once per request and block, and only to protected blocks
+        assert all(b in prot for b in released)
+        if detach == Fraction(1, 1) and nf == need:
+            assert released, "with this threshold and a full pool some request leaves its prefix"
+        # shared blocks are never reclaimed nor handed out
+        assert not (set(pool) & prot)

@@ -42,7 +42,7 @@ DEFAULT_CONFIG = "steady_state"
 OTHER_CONFIGS = [("llama8b_h2o", 0), ("mistral7b_random", 0), ("longctx_scissor", 0), ("steady_state", 32)]
 # launch shapes of the copy kernel tried beside the decode-read proxy: (grid cap, warps per CTA, ring stages)
 SWEEP_CTAS = (148, 111, 74, 37, 18)
-SWEEP_RINGS = ((8, 6), (8, 3), (4, 3))       # 192, 96, 48 KiB of shared memory per CTA with 4 KiB items
+SWEEP_RINGS = ((8, 6), (8, 4), (8, 3), (4, 3))       # 192, 128, 96, 48 KiB of shared memory per CTA with 4 KiB items
 
 
 def measured_peak():
@@ -324,7 +324,7 @@ def measure(args, ranks, dev, side, name, block_size, main):
     w, scale = fit_workload(args, name, seed, block_size, asked, dev)
     steps, warmup = args.steps, args.warmup
     prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas,
-                         wave_capacity=main and args.waves > 0, coresident=args.coresident)
+                         wave_capacity=main and args.waves > 0, urgent=args.urgent)
     partial_opts = dict(util=(1, 1), theta=(1, 4))     # fully live blocks stay; the paper's default trigger F > 0.25
     partial = main and args.plan_mode == "partial"
 
@@ -675,17 +675,19 @@ def run_proxy(args, prob, w, side, do_plan, bytes_per_step, dev, sweep):
     out.update(point(None, "as timed above"))
     if sweep:
         pts = []
-        for warps, stages in SWEEP_RINGS:
-            for ctas in SWEEP_CTAS:
+        rings = SWEEP_RINGS if not args.sweep_rings else [tuple(int(x) for x in r.split("x"))
+                                                          for r in args.sweep_rings.split(",")]
+        for warps, stages in rings:
+            for ctas in (SWEEP_CTAS if not args.sweep_rings else SWEEP_CTAS[:2]):
                 ctx = prob.make_ctx(max_ctas=ctas, copy_variant=2, tuning=dict(warps=warps, stages=stages))
                 try:
                     pts.append(point(ctx, f"{ctas} CTAs x {warps} warps x {stages} stages"))
                 finally:
                     torch.cuda.synchronize(dev)
                     vt.vtoken_destroy(ctx)
-        ctx = prob.make_ctx(coresident=1)
+        ctx = prob.make_ctx(urgent=1)
         try:
-            out["coresident_profile"] = point(ctx, "vtoken_config.coresident = 1")
+            out["urgent_profile"] = point(ctx, "vtoken_config.urgent = 1")
         finally:
             torch.cuda.synchronize(dev)
             vt.vtoken_destroy(ctx)
@@ -1071,12 +1073,14 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0, help="copy path: 0 auto, 1 registers, 2 bulk copy")
     ap.add_argument("--max-ctas", type=int, default=0)
-    ap.add_argument("--coresident", type=int, default=0, help="1: the copy kernel's launch shape for running beside decode")
+    ap.add_argument("--urgent", type=int, default=0, help="1: the copy kernel's launch shape that takes the larger share beside decode")
     ap.add_argument("--scale-requests", type=float, default=1.0)
     ap.add_argument("--oracle-layers", type=int, default=0,
                     help="layers in the CPU-baseline sample (0: 8, or 4 when a slab exceeds 1 GiB)")
     ap.add_argument("--no-proxy", action="store_true", help="skip the run beside the decode-read proxy")
     ap.add_argument("--no-sweep", action="store_true", help="skip the sweep of copy-kernel launch shapes beside the proxy")
+    ap.add_argument("--sweep-rings", default="", help="ring shapes of the sweep as warps x stages, e.g. 8x4,12x3 "
+                    "(default: 8x6, 8x4, 8x3, 4x3 = 192, 128, 96, 48 KiB per CTA); with this flag only the two largest grids are tried")
     ap.add_argument("--no-configs", action="store_true", help="skip the other roofline workloads (`configs`)")
     ap.add_argument("--proxy-ctas", type=int, default=0)
     ap.add_argument("--runtime", action="store_true", help="also time the token-table runtime kernels")

@@ -101,7 +101,7 @@ enum {
 
 /* Launch shape of the bulk-copy kernel (tuning and tests; the defaults are the measured best).
  * With enabled == 0 every field is ignored.  With enabled != 0: warps per CTA (0 => 8, at most 16),
- * ring stages per warp (0 => 6, 2 .. 12), rows per work item (0 => 4 KiB worth; rounded down to a
+ * ring stages per warp (0 => 4, 2 .. 12), rows per work item (0 => 4 KiB worth; rounded down to a
  * power of two that divides the block size, at most 32), work items loading ahead of the one being
  * stored (0 .. stages - 2), plan entries fetched ahead (1 or 2), fixed_shares != 0: every warp gets a
  * fixed share of the work items instead of taking them from a ticket counter, chunk = items per
@@ -124,13 +124,13 @@ typedef struct {
     int32_t max_ctas;              /* copy-kernel grid cap (co-residency with other work); 0 => auto */
     int32_t copy_variant;          /* 0 auto (bulk-copy path when row_bytes <= 32768, else register path);
                                       1 register path; 2 bulk-copy (TMA) path */
-    int32_t coresident;            /* 0: the copy kernel takes the whole GPU (one CTA per SM with 192 KiB of
-                                      shared-memory rings) -- the shape for a repack that runs alone, e.g. after the
-                                      step's forward has returned (Sec. 3.3.4).  1: the shape for a repack that
-                                      overlaps a decode kernel (the overlapped operation Sec. 5 measures as a
-                                      stress test): smaller rings, so that the other kernel's CTAs keep most of
-                                      every SM's shared memory and the two share HBM bandwidth instead of the
-                                      repack starving or being starved */
+    int32_t urgent;                /* 0: the default ring shape of the copy kernel (128 KiB of shared memory per SM): as
+                                      fast alone as any larger one, and the shape with which a repack beside a
+                                      bandwidth-bound decode kernel costs that kernel least (the overlapped operation
+                                      Sec. 5 measures as a stress test; 99 KiB of every SM's shared memory stay free).
+                                      1: smaller rings (96 KiB) with which the repack takes the larger share of HBM
+                                      beside such a kernel -- for a relocation that has to finish soon, e.g. under
+                                      the memory pressure of Sec. 3.3.2 */
     int32_t wait_limit_ms;         /* bound of every wait inside a kernel, 1 .. 60000; 0 => 2000 */
     int32_t plain_launches;        /* 0: every kernel of the library is launched with programmatic stream
                                       serialization, i.e. it may become resident while the previous kernel in the

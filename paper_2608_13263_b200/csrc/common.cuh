@@ -179,9 +179,14 @@ int vtk_launch_gather(vtoken_ctx *ctx, const int32_t *num_requests, const int32_
 __device__ __forceinline__ void vtk_wait_for_predecessor() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void vtk_release_successor() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-// launch shape of the copy kernel when vtoken_config.coresident is set
-constexpr int VTK_CORESIDENT_WARPS = 8;
-constexpr int VTK_CORESIDENT_STAGES = 3;
+// Ring shape of the bulk-copy kernel (warps per CTA x stages per warp, 4 KiB per stage).  Default 8 x 4 =
+// 128 KiB per SM: alone it copies as fast as 8 x 6 (6.69 TB/s on the steady-state workload), beside a
+// bandwidth-bound read kernel the two together move 7.07 TB/s instead of 6.27 (repack 2.26 + reader 4.81
+// instead of 1.98 + 4.29), and 99 KiB of every SM's shared memory stay free for the other kernel.
+// vtoken_config.urgent: 8 x 3 = 96 KiB, with which the repack takes the larger share beside the reader
+// (3.82 + 2.93 TB/s).
+constexpr int VTK_DEFAULT_WARPS = 8, VTK_DEFAULT_STAGES = 4;
+constexpr int VTK_URGENT_WARPS = 8, VTK_URGENT_STAGES = 3;
 
 // cfg.plain_launches turns the launch attribute off (the device side is then a no-op)
 template <typename... P, typename... A>

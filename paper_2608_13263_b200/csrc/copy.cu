@@ -457,13 +457,13 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctas_per_sm = 8;
     } else {
         // Launch shape: warps per CTA, ring stages per warp, rows per item, items loading ahead of the one
-        // being stored, plan entries fetched ahead.  Default: 8 warps x 6 stages x 4 KiB items = 192 KiB of
-        // staging per SM, two items loading ahead, three stores in flight per warp.  Measured on B200:
-        // shapes from 4 to 32 KiB per item land within about 3 % of each other; below 4 KiB per warp-step
-        // with only 8 warps per SM the pipeline becomes issue-bound.  The co-resident shape leaves most of
-        // the SM's shared memory to a kernel running beside the repack (see vtoken.h).
-        int warps = 8, stages = 6, rows = 0, depth = 2, ahead = 2;
-        if (ctx->cfg.coresident) { warps = VTK_CORESIDENT_WARPS; stages = VTK_CORESIDENT_STAGES; }
+        // being stored, plan entries fetched ahead.  Default: 8 warps x 4 stages x 4 KiB items = 128 KiB of
+        // staging per SM, two items loading ahead, one store in flight per warp.  Measured on B200: alone,
+        // shapes from 96 to 192 KiB per SM and from 4 to 32 KiB per item land within a few per cent of each
+        // other; below 4 KiB per warp-step with only 8 warps per SM the pipeline becomes issue-bound; beside a
+        // bandwidth-bound kernel the ring size decides how the two share HBM (see common.cuh).
+        int warps = VTK_DEFAULT_WARPS, stages = VTK_DEFAULT_STAGES, rows = 0, depth = 2, ahead = 2;
+        if (ctx->cfg.urgent) { warps = VTK_URGENT_WARPS; stages = VTK_URGENT_STAGES; }
         if (tuned) {
             if (tune.warps > 0) warps = tune.warps;
             if (tune.stages > 0) stages = tune.stages;
@@ -515,7 +515,6 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         ctas_per_sm = (int)((227 * 1024) / (smem + 2048));
         if (ctas_per_sm < 1) ctas_per_sm = 1;
         if (ctas_per_sm > 8) ctas_per_sm = 8;
-        if (ctx->cfg.coresident) ctas_per_sm = 1;
     }
     int ctas = ctx->num_sms * ctas_per_sm;
     if (tuned && tune.ctas > 0) ctas = tune.ctas;

@@ -324,7 +324,7 @@ def measure(args, ranks, dev, side, name, block_size, main):
     w, scale = fit_workload(args, name, seed, block_size, asked, dev)
     steps, warmup = args.steps, args.warmup
     prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas,
-                         wave_capacity=main and args.waves > 0, urgent=args.urgent)
+                         wave_capacity=main and args.waves > 0, **{})
     partial_opts = dict(util=(1, 1), theta=(1, 4))     # fully live blocks stay; the paper's default trigger F > 0.25
     partial = main and args.plan_mode == "partial"
 
@@ -685,12 +685,6 @@ def run_proxy(args, prob, w, side, do_plan, bytes_per_step, dev, sweep):
                 finally:
                     torch.cuda.synchronize(dev)
                     vt.vtoken_destroy(ctx)
-        ctx = prob.make_ctx(urgent=1)
-        try:
-            out["urgent_profile"] = point(ctx, "vtoken_config.urgent = 1")
-        finally:
-            torch.cuda.synchronize(dev)
-            vt.vtoken_destroy(ctx)
         out["sweep"] = pts
     return out
 
@@ -1073,7 +1067,6 @@ def main():
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--variant", type=int, default=0, help="copy path: 0 auto, 1 registers, 2 bulk copy")
     ap.add_argument("--max-ctas", type=int, default=0)
-    ap.add_argument("--urgent", type=int, default=0, help="1: the copy kernel's launch shape that takes the larger share beside decode")
     ap.add_argument("--scale-requests", type=float, default=1.0)
     ap.add_argument("--oracle-layers", type=int, default=0,
                     help="layers in the CPU-baseline sample (0: 8, or 4 when a slab exceeds 1 GiB)")

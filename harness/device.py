@@ -20,7 +20,7 @@ class DeviceProblem:
     def __init__(self, w: Workload, device="cuda:0", fill_seed: int = 1, copy_variant: int = 0, max_ctas: int = 0,
                  capacity_slack: int = 0, allocate_pools: bool = True, wave_capacity: bool = False,
                  ctx_capacity: dict = None, fill_mode: str = "random", **ctx_options):
-        """``ctx_options``: further keyword arguments of ``vtoken_create`` (urgent, wait_limit_ms,
+        """``ctx_options``: further keyword arguments of ``vtoken_create`` (wait_limit_ms,
         plain_launches, tuning, debug_stall_item).  ``fill_mode``: "random" (the seeded pool fill) or
         "address" (every row says where it was filled: a debugging aid)."""
         self.fill_mode = fill_mode

@@ -121,16 +121,13 @@ typedef struct {
     int64_t max_tokens;            /* upper bound of the token-table length (sum of request lengths) */
     int64_t max_table_blocks;      /* upper bound of the block-table length (sum over requests) */
     int32_t max_free_blocks;       /* upper bound of num_free */
-    int32_t max_ctas;              /* copy-kernel grid cap (co-residency with other work); 0 => auto */
+    int32_t max_ctas;              /* copy-kernel grid cap, 0 => one CTA per SM.  The default launch shape (128 KiB of
+                                      shared-memory rings per SM) is also the one with which a repack beside a
+                                      bandwidth-bound decode kernel costs that kernel least (the overlapped operation
+                                      Sec. 5 measures as a stress test); a smaller grid gives the other kernel a larger
+                                      share of HBM still, at the price of a slower repack */
     int32_t copy_variant;          /* 0 auto (bulk-copy path when row_bytes <= 32768, else register path);
                                       1 register path; 2 bulk-copy (TMA) path */
-    int32_t urgent;                /* 0: the default ring shape of the copy kernel (128 KiB of shared memory per SM): as
-                                      fast alone as any larger one, and the shape with which a repack beside a
-                                      bandwidth-bound decode kernel costs that kernel least (the overlapped operation
-                                      Sec. 5 measures as a stress test; 99 KiB of every SM's shared memory stay free).
-                                      1: smaller rings (96 KiB) with which the repack takes the larger share of HBM
-                                      beside such a kernel -- for a relocation that has to finish soon, e.g. under
-                                      the memory pressure of Sec. 3.3.2 */
     int32_t wait_limit_ms;         /* bound of every wait inside a kernel, 1 .. 60000; 0 => 2000 */
     int32_t plain_launches;        /* 0: every kernel of the library is launched with programmatic stream
                                       serialization, i.e. it may become resident while the previous kernel in the

@@ -52,7 +52,7 @@ class Config(ctypes.Structure):
                 ("layer_stride_bytes", ctypes.c_int64), ("max_requests", ctypes.c_int32),
                 ("max_tokens", ctypes.c_int64), ("max_table_blocks", ctypes.c_int64),
                 ("max_free_blocks", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
-                ("copy_variant", ctypes.c_int32), ("urgent", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
+                ("copy_variant", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
                 ("plain_launches", ctypes.c_int32), ("tuning", CopyTuning), ("debug_stall_item", ctypes.c_int64)]
 
 
@@ -231,7 +231,7 @@ def _check(rc, where, ctx=None):
 
 def vtoken_create(num_layers, num_blocks, block_size, num_kv_heads, head_dim, k_pool, v_pool, max_requests,
                   max_tokens, max_table_blocks, max_free_blocks, elem_bytes=2, layer_stride_bytes=0, max_ctas=0,
-                  copy_variant=0, urgent=0, wait_limit_ms=0, plain_launches=0, tuning=None,
+                  copy_variant=0, wait_limit_ms=0, plain_launches=0, tuning=None,
                   debug_stall_item=0) -> int:
     """``tuning``: dict with any of warps, stages, rows, depth, ahead, fixed_shares, chunk, ctas (the fields of
     vtoken_copy_tuning; giving it sets ``enabled``)."""
@@ -243,7 +243,7 @@ def vtoken_create(num_layers, num_blocks, block_size, num_kv_heads, head_dim, k_
             setattr(t, k, int(v))
     cfg = Config(num_layers, num_blocks, block_size, num_kv_heads, head_dim, elem_bytes, _ptr(k_pool), _ptr(v_pool),
                  layer_stride_bytes, max_requests, max_tokens, max_table_blocks, max_free_blocks, max_ctas,
-                 copy_variant, urgent, wait_limit_ms, plain_launches, t, debug_stall_item)
+                 copy_variant, wait_limit_ms, plain_launches, t, debug_stall_item)
     ctx = ctypes.c_void_p()
     _check(load().vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)), "vtoken_create")
     return ctx.value

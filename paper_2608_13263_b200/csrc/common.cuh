@@ -183,10 +183,8 @@ __device__ __forceinline__ void vtk_release_successor() { asm volatile("griddepc
 // 128 KiB per SM: alone it copies as fast as 8 x 6 (6.69 TB/s on the steady-state workload), beside a
 // bandwidth-bound read kernel the two together move 7.07 TB/s instead of 6.27 (repack 2.26 + reader 4.81
 // instead of 1.98 + 4.29), and 99 KiB of every SM's shared memory stay free for the other kernel.
-// vtoken_config.urgent: 8 x 3 = 96 KiB, with which the repack takes the larger share beside the reader
-// (3.82 + 2.93 TB/s).
+// (8 x 3 = 96 KiB came out bimodal from run to run, alone and beside the reader: not offered.)
 constexpr int VTK_DEFAULT_WARPS = 8, VTK_DEFAULT_STAGES = 4;
-constexpr int VTK_URGENT_WARPS = 8, VTK_URGENT_STAGES = 3;
 
 // cfg.plain_launches turns the launch attribute off (the device side is then a no-op)
 template <typename... P, typename... A>

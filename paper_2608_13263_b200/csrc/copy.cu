@@ -463,7 +463,6 @@ int vtk_configure_copy(vtoken_ctx *ctx)
         // other; below 4 KiB per warp-step with only 8 warps per SM the pipeline becomes issue-bound; beside a
         // bandwidth-bound kernel the ring size decides how the two share HBM (see common.cuh).
         int warps = VTK_DEFAULT_WARPS, stages = VTK_DEFAULT_STAGES, rows = 0, depth = 2, ahead = 2;
-        if (ctx->cfg.urgent) { warps = VTK_URGENT_WARPS; stages = VTK_URGENT_STAGES; }
         if (tuned) {
             if (tune.warps > 0) warps = tune.warps;
             if (tune.stages > 0) stages = tune.stages;

@@ -117,7 +117,7 @@ def test_bulk_copy_ring_shapes(tune):
               wl.longctx_scissor(seed=5, requests=2, lo=1500, hi=2500, layers=2, block_size=32),
               wl.mistral7b_random(seed=6, requests=4, lo=30, hi=300, layers=1, heads=4, head_dim=128, block_size=48)):
         run_and_compare(w, copy_variant=2, tuning=tuning)
-    run_and_compare(wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2), copy_variant=2, urgent=1)
+    run_and_compare(wl.mistral7b_random(seed=5, requests=7, lo=60, hi=700, layers=2), copy_variant=2, max_ctas=37)
 
 
 @pytest.mark.parametrize("dynamic,chunk", [("0", "4"), ("1", "1"), ("1", "3"), ("1", "64"), ("1", "1000")])

@@ -595,13 +595,15 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
     if (may_detach && !released_blocks) return VTO_EINVAL;
     int32_t *n_b = (int32_t *)malloc(sizeof(int32_t) * (size_t)NB);
     uint8_t *is_source = (uint8_t *)malloc((size_t)NB);     /* per physical block, for the request at hand */
-    if (!n_b || !is_source) { free(n_b); free(is_source); return VTO_EINVAL; }
+    int32_t *own_live = (int32_t *)calloc((size_t)NB, sizeof(int32_t));   /* n_rb: live tokens of the request at
+                                                                             hand stored in block b */
+    if (!n_b || !is_source || !own_live) { free(n_b); free(is_source); free(own_live); return VTO_EINVAL; }
 
     /* eligibility metadata: per-block liveness and the global waste ratio F (Sec. 3.3.1) */
     int64_t live_total = 0, N = 0;
     int rc = vto_block_liveness(R, S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, n_b, NULL,
                                 &live_total, &N);
-    if (rc != VTO_OK) { free(n_b); free(is_source); return rc; }
+    if (rc != VTO_OK) { free(n_b); free(is_source); free(own_live); return rc; }
     /* F > theta  <=>  (N*S - live) * den > num * N*S, in integers */
     int triggered = 1;
     if (opts->theta_den != 0) {
@@ -628,6 +630,10 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                 if (is_live(tt_slots, keep, t)) n_shared += opts->protect[tt_slots[t] / S] != 0;
             detach = ns_shared > 0 &&
                      (uint64_t)n_shared * opts->detach_den < (uint64_t)opts->detach_num * (uint64_t)ns_shared * (uint64_t)S;
+            /* block by block instead: the census of the request's own live tokens per block */
+            if (opts->detach_per_block)
+                for (int64_t t = t0; t < t1; ++t)
+                    if (is_live(tt_slots, keep, t)) ++own_live[tt_slots[t] / S];
         }
 
         /* source blocks: unprotected, low utilisation, at most B of them in table order (Sec. 3.3.3) */
@@ -640,7 +646,12 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                 eligible = (uint64_t)n_b[b] * opts->util_den < (uint64_t)opts->util_num * (uint64_t)S;
             if (eligible && opts->max_source_blocks > 0 && ns_unprotected >= opts->max_source_blocks) eligible = 0;
             ns_unprotected += eligible;
-            if (shared && detach) eligible = 1;             /* every shared block of a detaching request */
+            if (shared && may_detach) {
+                if (opts->detach_per_block)                /* the shared blocks this request fills poorly */
+                    eligible = (uint64_t)own_live[b] * opts->detach_den < (uint64_t)opts->detach_num * (uint64_t)S;
+                else
+                    eligible = detach;                     /* every shared block of a detaching request */
+            }
             is_source[b] = (uint8_t)eligible;
             ns += eligible;
         }
@@ -698,6 +709,9 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
             for (int32_t j = b0; j < b1; ++j) new_bt_blocks[new_bt_fill++] = bt_blocks[j];
         }
         for (int32_t j = b0; j < b1; ++j) is_source[bt_blocks[j]] = 0;
+        if (may_detach && opts->detach_per_block)
+            for (int64_t t = t0; t < t1; ++t)
+                if (is_live(tt_slots, keep, t)) own_live[tt_slots[t] / S] = 0;
     }
     new_bt_offsets[R] = new_bt_fill;
     counts->num_moves = num_moves;
@@ -707,7 +721,7 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
     counts->num_admitted = num_admitted;
     counts->num_deferred = num_deferred;
     counts->num_released = num_released;
-    free(n_b); free(is_source);
+    free(n_b); free(is_source); free(own_live);
     return VTO_OK;
 }
 

@@ -224,12 +224,15 @@ typedef struct {
     uint32_t detach_num, detach_den; /* copy-on-write detach: a request leaves ALL its protected blocks when its own
                                      live tokens in them fill less than detach_num / detach_den of those blocks;
                                      detach_den == 0: never (protected blocks always stay) */
+    uint32_t detach_per_block;    /* non-zero: the detach threshold is applied to every protected block of the
+                                     request by itself: it leaves block b when its own live tokens stored in b
+                                     number n_rb with n_rb * detach_den < detach_num * S, and stays in the others */
 } vto_partial_opts;
 
-/* Relocation planning that evacuates only low-utilisation source blocks (Sec. 3.3.3):
- * the paper's planner "selects eligible low-utilization source blocks, computes the live-token
- * footprint" T_live of those blocks, needs ceil(T_live / S) destinations and admits the plan only
- * when the sources release more blocks than that.  Everything else as vto_plan, except:
+/* Relocation planning that evacuates only low-utilisation source blocks (Sec. 3.3.3): the planner
+ * picks the eligible, poorly filled blocks of a request as sources, counts the live tokens T_live
+ * stored in them, needs ceil(T_live / S) destinations and admits the plan only when the sources
+ * release more blocks than that.  Everything else as vto_plan, except:
  *   - only live tokens stored in source blocks move (logical order, destinations filled completely);
  *     live tokens in the other blocks keep their slots; dead tokens become -1;
  *   - new block table of a repacked request = its non-source blocks in old order, then its
@@ -238,15 +241,19 @@ typedef struct {
  * With util_den == 0, protect == NULL, B == 0 and theta_den == 0 the result equals vto_plan's.
  * NB = number of physical blocks (size of protect and of the internal n_b).
  *
- * Copy-on-write detach (the paper's outlook for shared-prefix blocks, Sec. 5 "Compatibility with
- * Prefix Caching" and Sec. 6: copy-on-write "when the expected reclamation benefit justifies the
- * extra copy"): with detach_den != 0, a request whose own live tokens occupy less than
+ * Copy-on-write detach (the paper's outlook for shared-prefix blocks, Sec. 5 on prefix caching and
+ * Sec. 6: copy a request's tokens out of shared blocks once the blocks that brings back outweigh
+ * the copy): with detach_den != 0, a request whose own live tokens occupy less than
  * detach_num / detach_den of its protected blocks (n_shared * den < num * ns_shared * S) treats all
  * of them as sources too: its live tokens there are COPIED to its destinations with the rest (the
  * shared blocks keep their bytes for the other holders), the blocks leave its table, and they are
  * listed in released_blocks (references dropped; the caller's reference counts decide when such a
  * block is free) instead of freed_blocks.  B bounds the unprotected sources only.  The gain gate
- * is unchanged: destinations < sources, counted in the request's own table. */
+ * is unchanged: destinations < sources, counted in the request's own table.
+ * With detach_per_block the same threshold is applied block by block: the request leaves exactly
+ * those protected blocks of its table in which its own live tokens fill less than the fraction
+ * (n_rb * den < num * S; the other holders' tokens do not count), and keeps the others in place,
+ * at the head of its new table with its other kept blocks. */
 int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      const int32_t *bt_offsets, const int32_t *bt_blocks,
                      const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,

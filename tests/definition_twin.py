@@ -75,11 +75,13 @@ def to_csr(lists):
 
 
 def repack_partial_definition(S, block_tables, token_tables, keeps, free, select=None, thr=None, protect=(),
-                              util=None, max_sources=0, theta=None, detach=None):
+                              util=None, max_sources=0, theta=None, detach=None, detach_per_block=False):
     """Definition-level statement of the partial plan: only low-utilisation, unprotected blocks are
     evacuated.  protect: set of block ids; util / theta / detach: Fraction or None.  With ``detach`` a
     request whose own live tokens fill less than that fraction of its protected blocks leaves all of
-    them (copy-on-write): they become sources too and are listed under ``released``."""
+    them (copy-on-write): they become sources too and are listed under ``released``.  With
+    ``detach_per_block`` the fraction is taken block by block: the request leaves exactly the protected
+    blocks in which its own live tokens fill less than ``detach`` of the S slots."""
     R = len(token_tables)
     live = [[t for t, (s, k) in enumerate(zip(token_tables[r], keeps[r])) if s >= 0 and k] for r in range(R)]
     per_block = {}
@@ -102,8 +104,12 @@ def repack_partial_definition(S, block_tables, token_tables, keeps, free, select
                 picked.append(b)
         shared = [b for b in block_tables[r] if b in protect]
         mine_in_shared = sum(1 for t in live[r] if token_tables[r][t] // S in protect)
-        goes = detach is not None and shared and Fraction(mine_in_shared, len(shared) * S) < detach
-        leaving.append(set(shared) if goes else set())
+        if detach is not None and detach_per_block:
+            mine_in = lambda b: sum(1 for t in live[r] if token_tables[r][t] // S == b)
+            leaving.append({b for b in shared if Fraction(mine_in(b), S) < detach})
+        else:
+            goes = detach is not None and shared and Fraction(mine_in_shared, len(shared) * S) < detach
+            leaving.append(set(shared) if goes else set())
         # table order is kept: a source is an unprotected pick or a shared block of a leaving request
         sources.append([b for b in block_tables[r] if b in set(picked) or b in leaving[r]])
     moving = [[t for t in live[r] if token_tables[r][t] // S in set(sources[r])] for r in range(R)]

@@ -138,7 +138,7 @@ def test_source_bound_B_takes_the_first_eligible_blocks_in_table_order():
     assert vto.plan_partial(S, 10, [0, 5], bt, [0, 20], tt, keep, free, max_source_blocks=1).req_status.tolist() == [vto.NO_GAIN]
 
 
-def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB, detach=None):
+def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB, detach=None, per_block=False):
     bt_off, bt_flat = to_csr(bts)
     tt_off, tt_flat = to_csr(tts)
     _, keep_flat = to_csr(keeps)
@@ -148,8 +148,10 @@ def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB,
     p = vto.plan_partial(S, NB, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free,
                          select=None if select is None else np.array(select, np.uint8),
                          thr_num=fr(thr)[0], thr_den=fr(thr)[1], protect=prot if protect else None,
-                         util=fr(util), max_source_blocks=B, theta=fr(theta), detach=fr(detach))
-    d = repack_partial_definition(S, bts, tts, keeps, list(free), select, thr, set(protect), util, B, theta, detach)
+                         util=fr(util), max_source_blocks=B, theta=fr(theta), detach=fr(detach),
+                         detach_per_block=per_block)
+    d = repack_partial_definition(S, bts, tts, keeps, list(free), select, thr, set(protect), util, B, theta, detach,
+                                  per_block)
     assert p.released_blocks.tolist() == d["released"]
     nbo, nbf = to_csr(d["new_bt"])
     _, ntf = to_csr(d["new_tt"])
@@ -303,3 +305,145 @@ def test_detach_on_the_shared_prefix_workload(degree):
     q = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
                          protect=protect)
     assert q.released_blocks.tolist() == [] and len(q.new_bt_blocks) > len(p.new_bt_blocks)
+
+
+# ---- copy-on-write detach decided per shared block -------------------------------------------------
+def test_per_block_detach_bruteforce_against_the_definition_twin():
+    """Three requests over three protected blocks (0, 4 and 1; request 2 holds only one of them) with
+    private blocks behind them, S = 3 so that a block can be 0/3 .. 3/3 full of one request's tokens;
+    random keep masks x thresholds x utilisation x source bounds x pool sizes, block-by-block rule."""
+    rng = np.random.default_rng(17)
+    S = 3
+    bts = [[0, 4, 1, 6], [0, 4, 1, 7, 3], [4, 8]]
+    tts = [[0, 1, 2, 12, 13, 14, 3, 4, 5, 18, 19, -1], [0, 1, 2, 12, 13, 14, 3, 4, 5, 21, 22, 23, 9, -1, 11],
+           [12, 13, 14, 24, 25]]
+    NB = 16
+    seen = set()
+    for _ in range(50):
+        keeps = [rng.integers(0, 2, len(t)).tolist() for t in tts]
+        for detach in (Fraction(1, 3), Fraction(1, 2), Fraction(2, 3), Fraction(1, 1), Fraction(4, 3)):
+            for util in (None, Fraction(1, 1)):
+                for B in (0, 1):
+                    for c in (0, 1, 3, 6):
+                        free = np.array([9, 5, 10, 11, 12, 13][:c], np.int32)
+                        _compare(S, bts, tts, keeps, free, None, None, (0, 4, 1), util, B, None, NB, detach, True)
+            d = repack_partial_definition(S, bts, tts, keeps, [9, 5, 10, 11, 12, 13], protect={0, 4, 1}, detach=detach,
+                                          detach_per_block=True)
+            for r in range(3):
+                shared = [b for b in bts[r] if b in (0, 4, 1)]
+                seen.add((len(shared), sum(b in d["new_bt"][r] for b in shared)))
+    # the sample really holds requests that left some of their shared blocks and stayed in others
+    assert {(3, 1), (3, 2), (3, 0), (3, 3), (1, 0), (1, 1)} <= seen
+
+
+def test_per_block_detach_by_hand():
+    """S = 4.  Request 0 holds shared blocks 0, 1, 2 and private block 5; of its prefix tokens it keeps
+    3 in block 0, 1 in block 1 and 2 in block 2; request 1 keeps everything.  At threshold 1/2 it leaves
+    block 1 only (1/4 < 1/2; 2/4 is not below 1/2: strict); at 3/4 blocks 1 and 2; the request-level
+    rule at 1/2 would have kept all three (6 of 12 slots)."""
+    S = 4
+    bts = [[0, 1, 2, 5], [0, 1, 2, 6]]
+    tts = [list(range(12)) + [20, 21, 22], list(range(12)) + [24]]
+    keeps = [[1, 1, 1, 0,  0, 1, 0, 0,  1, 0, 0, 1,  1, 0, 1], [1] * 13]
+    bt_off, bt_flat = to_csr(bts)
+    tt_off, tt_flat = to_csr(tts)
+    _, keep_flat = to_csr(keeps)
+    protect = np.zeros(12, np.uint8)
+    protect[[0, 1, 2]] = 1
+    free = np.array([7, 8, 9], np.int32)
+    run = lambda d, pb: vto.plan_partial(S, 12, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free, protect=protect,
+                                         util=(1, 1), detach=d, detach_per_block=pb)
+    whole = run((1, 2), False)
+    assert whole.released_blocks.tolist() == [] and whole.req_status.tolist() == [vto.NO_GAIN, vto.NO_GAIN]
+    half = run((1, 2), True)
+    # sources: shared 1 (1 live) and private 5 (2 of 4 live) -> 3 tokens -> 1 destination < 2 sources
+    assert half.req_status.tolist() == [vto.REPACKED, vto.NO_GAIN]
+    assert half.released_blocks.tolist() == [1] and half.freed_blocks.tolist() == [5]
+    assert half.new_bt_blocks.tolist() == [0, 2, 7, 0, 1, 2, 6]
+    assert half.new_tt_slots[:15].tolist() == [0, 1, 2, -1, -1, 28, -1, -1, 8, -1, -1, 11, 29, -1, 30]
+    assert half.new_tt_slots[15:].tolist() == tts[1]                       # the other sharer is untouched
+    assert list(zip(half.move_src.tolist(), half.move_dst.tolist())) == [(5, 28), (20, 29), (22, 30)]
+    more = run((3, 4), True)
+    # blocks 1 and 2 and private 5: 1 + 2 + 2 = 5 tokens -> 2 destinations < 3 sources
+    assert more.released_blocks.tolist() == [1, 2] and more.freed_blocks.tolist() == [5]
+    assert more.new_bt_blocks.tolist() == [0, 7, 8, 0, 1, 2, 6]
+    assert more.new_tt_slots[:15].tolist() == [0, 1, 2, -1, -1, 28, -1, -1, 29, -1, -1, 30, 31, -1, 32]
+    assert len(more.released_blocks) == 2 and more.num_moves == 5
+
+
+def test_per_block_detach_meets_the_request_level_rule_where_the_two_must_agree():
+    """(a) A threshold above one empties every protected block under either rule.  (b) With one
+    protected block per request the block is the request's whole shared part.  (c) Threshold 0/1:
+    nothing is below it, both equal the conservative plan."""
+    w, protect = wl.shared_prefix(seed=3, groups=3, degree=2, prefix_len=48, suffix_len=80, layers=1, heads=1,
+                                  head_dim=8, block_size=4)
+    S = w.block_size
+    run = lambda **kw: vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
+                                        w.free_blocks, util=(1, 1), **kw)
+    same = lambda p, q: all(np.array_equal(getattr(p, f), getattr(q, f)) for f in
+                            ("new_bt_offsets", "new_bt_blocks", "new_tt_slots", "freed_blocks", "released_blocks",
+                             "req_status", "move_src", "move_dst"))
+    assert same(run(protect=protect, detach=(5, 4)), run(protect=protect, detach=(5, 4), detach_per_block=True))
+    assert len(run(protect=protect, detach=(5, 4)).released_blocks) > 0
+    one = np.zeros_like(protect)                 # protect only the first block of every request's table
+    one[w.bt_blocks[w.bt_offsets[:-1]]] = 1
+    # (the other prefix blocks are then unprotected blocks in several tables: plan request by request)
+    for r in range(w.num_requests):
+        sel = np.zeros(w.num_requests, np.uint8)
+        sel[r] = 1
+        for d in ((1, 4), (1, 2), (3, 4), (1, 1)):
+            assert same(run(protect=one, detach=d, select=sel), run(protect=one, detach=d, select=sel,
+                                                                    detach_per_block=True))
+    cons = run(protect=protect)
+    assert same(cons, run(protect=protect, detach=(0, 1), detach_per_block=True))
+    assert same(cons, run(protect=protect, detach=(0, 1)))
+
+
+@pytest.mark.parametrize("degree", [1, 2, 4])
+@pytest.mark.parametrize("detach", [(1, 4), (1, 2), (3, 4)])
+def test_per_block_detach_on_the_shared_prefix_workload(degree, detach):
+    """Block-by-block detach on the prefix-cache workload: a request leaves exactly the prefix blocks it
+    fills below the threshold (counted from its own mask), keeps the others at the head of its table,
+    the shared blocks are never freed, written to or changed, and every request sees its own tokens."""
+    w, protect = wl.shared_prefix(seed=10 + degree, groups=2, degree=degree, prefix_len=64, suffix_len=96, layers=1,
+                                  heads=1, head_dim=8, block_size=4)
+    S = w.block_size
+    p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
+                         protect=protect, detach=detach, detach_per_block=True)
+    shared = set(np.flatnonzero(protect).tolist())
+    live = (w.tt_slots >= 0) & (w.keep != 0)
+    assert not (set(p.freed_blocks.tolist()) & shared) and not (set((p.move_dst // S).tolist()) & shared)
+    assert set(p.released_blocks.tolist()) <= shared
+    slab = np.arange(w.slots_per_layer * 2, dtype=np.int64).reshape(-1, 2)
+    before = slab.copy()
+    vto.apply_moves_slab(slab, p.move_src, p.move_dst)
+    shared_rows = np.isin(np.arange(w.slots_per_layer) // S, sorted(shared))
+    assert np.array_equal(slab[shared_rows], before[shared_rows])
+    released = p.released_blocks.tolist()
+    cursor = 0
+    some_left = some_stayed = False
+    for r in range(w.num_requests):
+        t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
+        old = w.bt_blocks[w.bt_offsets[r]:w.bt_offsets[r + 1]].tolist()
+        new = p.new_bt_blocks[p.new_bt_offsets[r]:p.new_bt_offsets[r + 1]].tolist()
+        assert np.array_equal(vto.gather_logical(before, w.tt_slots[t0:t1], w.keep[t0:t1]),
+                              vto.gather_logical(slab, p.new_tt_slots[t0:t1]))
+        if p.req_status[r] != vto.REPACKED:
+            assert new == old
+            continue
+        mine = np.bincount(w.tt_slots[t0:t1][live[t0:t1]] // S, minlength=w.num_blocks)
+        leaves = [b for b in old if b in shared and mine[b] * detach[1] < detach[0] * S]
+        stays = [b for b in old if b in shared and b not in leaves]
+        assert released[cursor:cursor + len(leaves)] == leaves
+        cursor += len(leaves)
+        assert new[:len(stays)] == stays and not (set(new) & set(leaves))
+        # its tokens in the blocks it stays in keep their slots; those in the blocks it left were copied out
+        slots, now = w.tt_slots[t0:t1], p.new_tt_slots[t0:t1]
+        in_stay = live[t0:t1] & np.isin(slots // S, stays)
+        in_left = live[t0:t1] & np.isin(slots // S, leaves)
+        assert np.array_equal(now[in_stay], slots[in_stay]) and not np.isin(now[in_left] // S, sorted(shared)).any()
+        some_left |= bool(leaves)
+        some_stayed |= bool(stays)
+    assert cursor == len(released)
+    if detach == (1, 2):
+        assert some_left and some_stayed            # the threshold really splits the prefix

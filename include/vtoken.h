@@ -277,6 +277,9 @@ typedef struct {
     uint32_t detach_num, detach_den; /* copy-on-write detach: a request leaves ALL its protected blocks when its own
                                       live tokens in them fill less than detach_num / detach_den of those blocks
                                       (n_shared * den < num * ns_shared * S); detach_den == 0: never */
+    uint32_t detach_per_block;     /* non-zero: the threshold is applied to every protected block of the request by
+                                      itself -- it leaves block b when its own live tokens stored in b number n_rb
+                                      with n_rb * detach_den < detach_num * S, and stays in the others */
 } vtoken_partial_opts;
 
 /* vtoken_plan restricted to source blocks.  Differences from vtoken_plan: only live tokens stored
@@ -298,7 +301,14 @@ typedef struct {
  * (destinations < sources, in the request's own table), so whether the POOL gains depends on the
  * other holders: enabling detach is the caller's policy decision.  vtoken_repack_waves and
  * vtoken_repack_host_partial take the threshold too; each has a released list of its own in its
- * output struct. */
+ * output struct.
+ * With detach_per_block the threshold is applied block by block instead: the request leaves exactly
+ * those protected blocks of its table in which its own live tokens (not the other holders') fill
+ * less than the fraction of the S slots, and keeps the others in place, in old order with its other
+ * kept blocks.  The planner then takes a census of every request's live tokens per protected table
+ * entry (one more kernel and a memset of 16 B per block-table entry in front of the plan; a lookup
+ * per live token in a protected block).  A token stored in a protected block that its request's
+ * table does not list stays where it is. */
 int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
                         const vtoken_plan_out *out, void *cuda_stream);
 

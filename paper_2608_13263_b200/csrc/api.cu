@@ -26,7 +26,7 @@ void free_all(vtoken_ctx *ctx)
     void *ptrs[] = {ctx->tile_n, ctx->req_part, ctx->req_before, ctx->req_n, ctx->req_dst_base, ctx->req_freed_base, ctx->req_status, ctx->dst_src,
                     ctx->dst_blocks, ctx->counts, ctx->rt_counts, ctx->plan_header, ctx->g_src, ctx->g_total, ctx->g_ids, ctx->g_req, ctx->g_offsets, ctx->tile_mov, ctx->tile_shared, ctx->part_mov, ctx->req_ns, ctx->req_nsrc,
                     ctx->n_b, ctx->slot_bits, ctx->copy_ticket, ctx->g_ticket, ctx->g_tile_n, ctx->g_req_part, ctx->g_req_before, ctx->part_shared, ctx->req_shared, ctx->req_detach,
-                    ctx->req_rel_base,
+                    ctx->req_rel_base, ctx->cow,
                     ctx->stage.num_requests, ctx->stage.bt_blocks,
                     ctx->stage.tt_slots, ctx->stage.free_blocks, ctx->stage.keep,
                     ctx->stage.new_bt_offsets, ctx->stage.new_bt_blocks,
@@ -158,6 +158,7 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->req_shared, cfg->max_requests);
     A(&ctx->req_detach, cfg->max_requests);
     A(&ctx->req_rel_base, cfg->max_requests);
+    A(&ctx->cow, 2 * (int64_t)cfg->max_table_blocks);
     if (rc == VTOKEN_OK && cudaMemset(ctx->counts, 0, sizeof(vtoken_counts)) != cudaSuccess) rc = VTOKEN_ECUDA;
     if (rc == VTOKEN_OK) rc = vtk_configure_copy(ctx);
     if (rc != VTOKEN_OK) { free_all(ctx); delete ctx; return rc; }

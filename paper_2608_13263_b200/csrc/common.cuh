@@ -52,6 +52,8 @@ struct vtoken_ctx {
     int32_t *req_shared;       // [max_requests] protected entries of the request's block table
     int32_t *req_detach;       // [max_requests] 1 = the request leaves its protected blocks (copy-on-write detach)
     int32_t *req_rel_base;     // [max_requests] first entry in released_blocks
+    unsigned long long *cow;   // [2 * max_table_blocks] detach per shared block: every request's hash from a protected
+                               // block of its table to its own live tokens there ((block id + 1) << 32 | count)
     uint32_t *slot_bits;       // [ceil(num_blocks * S / 32)] one bit per slot (vtoken_check_tables)
 
     // gather_logical scratch (DEVICE)

@@ -28,6 +28,17 @@
 // tokens there are copied out with the rest, and the blocks are listed as released references
 // instead of reclaimed blocks.  "Source" is therefore a per-request notion for protected blocks
 // (req_detach[r]) and a per-block one (blk_src[b]) for the others.
+//
+// Detach decided per shared block (opts->detach_per_block): the request leaves exactly the protected
+// blocks that its own live tokens fill below the threshold.  That needs the census n_rb (live
+// tokens of request r stored in block b) for every protected entry of every block table, and every
+// token must find the count of its own (request, block) pair.  Each request owns the range
+// [2 * bt_offsets[r], 2 * bt_offsets[r + 1]) of one scratch array as a private open-addressing hash
+// from block id to count (twice as many places as it can have protected entries, so a probe
+// sequence always ends): cleared by a memset node, filled with the protected entries by one more
+// kernel in front of tiles<0>, counted into by tiles<0> (integer atomics), read by blocks, tiles<1>
+// and assign.  A token in a protected block that its request's table does not list finds nothing
+// and stays where it is.
 #include "common.cuh"
 
 #include <cstring>
@@ -42,6 +53,7 @@ struct PArgs {
     vtk_arr<const int32_t> num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots;
     vtk_arr<const uint8_t> keep, select, protect;
     uint32_t thr_num, thr_den, util_num, util_den, theta_num, theta_den, detach_num, detach_den;
+    uint32_t per_block;              // detach decided per protected block (the census in cow)
     int32_t max_sources;
     vtk_arr<const int32_t> free_blocks, num_free;
     vtk_arr<int32_t> new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, released_blocks, out_status;
@@ -55,6 +67,7 @@ struct PArgs {
     vtk_arr<int32_t> req_before;     // [max_requests + 1] moving tokens of the table before the request's first entry
     vtk_arr<int32_t> dst_src, dst_blocks, n_b;
     vtk_arr<uint8_t> blk_src;
+    vtk_arr<unsigned long long> cow; // [2 * max_table_blocks] per-request hashes: (block id + 1) << 32 | own live tokens
     vtk_arr<vtoken_counts> counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
     int32_t num_tiles, vec_in, vec_out;
@@ -84,12 +97,87 @@ __device__ __forceinline__ int pp_block_sum(int n, int *warp_n)
     return s;   // valid in thread 0
 }
 
-// ---- tiles: live / moving tokens per tile and in front of request boundaries, per-block liveness ----
-// does a live token of request r in block b move?  (b is a source of its request, or r leaves its
-// protected blocks and b is one of them)
-__device__ __forceinline__ bool pp_moves(const PArgs &a, bool detach, int32_t b)
+// ---- the per-request census of own live tokens in protected blocks -------------------------------
+// The hash of request r: `size` places from `base` on (size == 0: the request has no block table).
+struct CowTable {
+    int64_t base, size;
+};
+__device__ __forceinline__ CowTable pp_cow_table(const PArgs &a, int r)
 {
-    return a.blk_src[b] != 0 || (detach && a.protect[b] != 0);
+    int64_t b0, b1;
+    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
+    return CowTable{2 * b0, 2 * (b1 - b0)};
+}
+__device__ __forceinline__ int64_t pp_cow_first(const CowTable &h, int32_t b)
+{
+    return (int64_t)(((uint32_t)b * 2654435761u) % (uint64_t)h.size);
+}
+// Place of block b in the table (nullptr: not there).  INSERT: take the first free place on the way.
+template <bool INSERT>
+__device__ __forceinline__ unsigned long long *pp_cow_find(const PArgs &a, const CowTable &h, int32_t b)
+{
+    if (h.size <= 0) return nullptr;
+    const unsigned long long tag = (unsigned long long)(uint32_t)(b + 1) << 32;
+    int64_t i = pp_cow_first(h, b);
+    for (int64_t probes = 0; probes < h.size; ++probes) {           // bounded: at most once around the table
+        unsigned long long *p = &a.cow[h.base + i];
+        unsigned long long e = *p;
+        if (INSERT && e == 0) {
+            e = atomicCAS(p, 0ull, tag);
+            if (e == 0) return p;
+        }
+        if ((e >> 32) == (tag >> 32)) return p;
+        if (e == 0) return nullptr;
+        i = i + 1 == h.size ? 0 : i + 1;
+    }
+    return nullptr;
+}
+// does request r leave protected block b?  (its own live tokens there fill less than the threshold)
+__device__ __forceinline__ bool pp_cow_leaves(const PArgs &a, const CowTable &h, int32_t b)
+{
+    const unsigned long long *p = pp_cow_find<false>(a, h, b);
+    if (!p) return false;
+    return (*p & 0xffffffffull) * a.detach_den < (unsigned long long)a.detach_num * (unsigned long long)a.S;
+}
+
+// one CTA per request: its protected table entries enter its hash
+__global__ void __launch_bounds__(256) pp_cow_insert_kernel(PArgs a)
+{
+    vtk_release_successor();
+    vtk_wait_for_predecessor();
+    const int r = blockIdx.x;
+    if (r >= pp_requests(a)) return;
+    int64_t b0, b1;
+    vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
+    const CowTable h{2 * b0, 2 * (b1 - b0)};
+    for (int64_t j = b0 + threadIdx.x; j < b1; j += 256) {
+        const int32_t blk = a.bt_blocks[j];
+        if (blk < 0 || blk >= a.num_blocks) continue;              // flagged by the blocks kernel
+        if (a.protect[blk] != 0) pp_cow_find<true>(a, h, blk);
+    }
+}
+
+// ---- tiles: live / moving tokens per tile and in front of request boundaries, per-block liveness ----
+// What decides whether a live token of the request at hand moves out of a protected block.
+struct Owner {
+    bool detach;         // the request leaves protected blocks (all of them, or those the census names)
+    CowTable cow;        // per-block rule: its census
+};
+__device__ __forceinline__ Owner pp_owner(const PArgs &a, int r)
+{
+    Owner o{false, CowTable{0, 0}};
+    if (r < 0) return o;
+    o.detach = a.req_detach[r] != 0;
+    if (o.detach && a.per_block) o.cow = pp_cow_table(a, r);
+    return o;
+}
+// does a live token of that request in block b move?  (b is a source of its request, or the request
+// leaves protected blocks and b is one of those it leaves)
+__device__ __forceinline__ bool pp_moves(const PArgs &a, const Owner &o, int32_t b)
+{
+    if (a.blk_src[b] != 0) return true;
+    if (!o.detach || a.protect[b] == 0) return false;
+    return a.per_block ? pp_cow_leaves(a, o.cow, b) : true;
 }
 
 // Bits of the thread's live entries that move.  Without a detach threshold that is a property of the
@@ -100,21 +188,22 @@ __device__ __forceinline__ unsigned pp_moving_bits(const PArgs &a, unsigned bits
 {
     unsigned mov = 0;
     int64_t next = may_detach ? pp_offset(a, r + 1 <= R ? r + 1 : R) : 0;
-    bool detach = may_detach && r >= 0 && a.req_detach[r] != 0;
+    Owner o = may_detach ? pp_owner(a, r) : Owner{false, CowTable{0, 0}};
 #pragma unroll
     for (int k = 0; k < TILE_TOK; ++k) {
         if (may_detach && t + k >= next && r + 1 < R) {
             while (r + 1 < R && pp_offset(a, r + 1) <= t + k) ++r;
             next = pp_offset(a, r + 1);
-            detach = r >= 0 && a.req_detach[r] != 0;
+            o = pp_owner(a, r);
         }
         if ((bits >> k) & 1u)
-            if (pp_moves(a, detach, slot[k] / a.S)) mov |= 1u << k;
+            if (pp_moves(a, o, slot[k] / a.S)) mov |= 1u << k;
     }
     return mov;
 }
 
 // mode 0: live tokens per tile, n_b (and, with a detach threshold, the live tokens in protected
+// blocks, or -- per-block rule -- the census of every request's own live tokens in its protected
 // blocks); mode 1: live tokens that move.
 template <int MODE>
 __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
@@ -148,13 +237,36 @@ __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
     const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, pp_offset(a, 0), limit, a.slots_per_layer, slot, bad);
     int n = 0, n_sh = 0;
     if (MODE == 0) {
+        const bool census = may_detach && a.per_block != 0 && is_tile;   // uniform over the CTA
+        int r = -1;
+        int64_t next = 0;
+        CowTable h{0, 0};
+        if (census) {
+            vtk_tile_owners(a.tt_offsets, R, a.max_tokens, base, limit, tile_req);
+            __syncthreads();
+            if (t < limit) r = vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t);
+            next = pp_offset(a, r + 1 <= R ? r + 1 : R);
+            if (r >= 0) h = pp_cow_table(a, r);
+        }
 #pragma unroll
         for (int k = 0; k < TILE_TOK; ++k) {
+            if (census && t + k >= next && r + 1 < R) {
+                while (r + 1 < R && pp_offset(a, r + 1) <= t + k) ++r;
+                next = pp_offset(a, r + 1);
+                h = pp_cow_table(a, r);
+            }
             if (!((bits >> k) & 1u)) continue;
             const int blk = slot[k] / a.S;
             if (is_tile) atomicAdd(&a.n_b[blk], 1);          // the tile CTAs see every entry exactly once
             ++n;
-            if (may_detach) n_sh += a.protect[blk] != 0;
+            if (may_detach) {
+                const bool prot = a.protect[blk] != 0;
+                n_sh += prot;
+                if (census && prot && r >= 0) {
+                    unsigned long long *p = pp_cow_find<false>(a, h, blk);
+                    if (p) atomicAdd(p, 1ull);                  // the count lives in the low half
+                }
+            }
         }
     } else {
         int r = -1;
@@ -197,8 +309,10 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
     int64_t b0, b1;
     vtk_range(a.bt_offsets, r, a.max_table_blocks, b0, b1);
     int carry = 0;               // eligible entries before this chunk
-    int shared = 0;              // protected entries seen by this thread
+    int shared = 0;              // protected entries seen by this thread (per-block rule: those the request leaves)
     uint32_t flags = 0;
+    const bool per_block = !a.protect.null() && a.detach_den != 0 && a.per_block != 0;
+    const CowTable h{2 * b0, 2 * (b1 - b0)};
     for (int64_t jb = b0; jb < b1; jb += PP_NT) {
         const int64_t j = jb + threadIdx.x;
         bool eligible = false;
@@ -210,7 +324,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
                 blk = -1;
             } else {
                 eligible = !(!a.protect.null() && a.protect[blk] != 0);
-                shared += !eligible;
+                if (!eligible) shared += per_block ? (pp_cow_leaves(a, h, blk) ? 1 : 0) : 1;
                 if (eligible && a.util_den != 0)
                     eligible = (unsigned long long)a.n_b[blk] * a.util_den <
                                (unsigned long long)a.util_num * (unsigned long long)a.S;
@@ -222,7 +336,16 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
         if (eligible && (a.max_sources <= 0 || rank < a.max_sources)) a.blk_src[blk] = 1;
     }
     int ns = (a.max_sources > 0 && carry > a.max_sources) ? a.max_sources : carry;
-    if (!a.protect.null() && a.detach_den != 0) {
+    if (per_block) {
+        // block by block: the protected entries the request leaves are sources, the others stay
+        __syncthreads();
+        const int ns_leaving = pp_block_sum(shared, warp_sums);         // valid in thread 0
+        if (threadIdx.x == 0) {
+            a.req_detach[r] = ns_leaving > 0 ? 1 : 0;
+            a.req_shared[r] = ns_leaving;
+            ns += ns_leaving;
+        }
+    } else if (!a.protect.null() && a.detach_den != 0) {
         // copy-on-write detach: the request leaves its protected blocks when its own live tokens
         // fill less than detach_num / detach_den of them; then every one of them is a source
         __syncthreads();
@@ -451,10 +574,11 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
                 a.dst_blocks[dst_base + j] = blk;
             }
             for (int i = nsrc + tid; i < need * S; i += TILE_NT) a.dst_src[(int64_t)dst_base * S + i] = -1;
-            // kept blocks in old order, unprotected sources to the reclaimed list and protected sources (of a
-            // detaching request) to the released list, each in old order
+            // kept blocks in old order, unprotected sources to the reclaimed list and the protected blocks the
+            // request leaves to the released list, each in old order
             const int f0 = a.req_freed_base[r];
             const int l0 = detach ? a.req_rel_base[r] : 0;
+            const CowTable h{2 * b0, 2 * (b1 - b0)};
             int carry_src = 0, carry_rel = 0;
             for (int64_t jb = b0; jb < b1; jb += TILE_NT) {
                 const int64_t j = jb + tid;
@@ -464,7 +588,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
                     blk = a.bt_blocks[j];
                     if (blk >= 0 && blk < a.num_blocks) {
                         src = a.blk_src[blk] != 0;
-                        rel = detach && a.protect[blk] != 0;
+                        rel = detach && a.protect[blk] != 0 && (a.per_block == 0 || pp_cow_leaves(a, h, blk));
                     }
                 }
                 int total;
@@ -647,6 +771,8 @@ void fill_args(PArgs &a, vtoken_ctx *ctx)
     a.req_shared = VTK_ARR(ctx, ctx->req_shared, c.max_requests);
     a.req_detach = VTK_ARR(ctx, ctx->req_detach, c.max_requests);
     a.req_rel_base = VTK_ARR(ctx, ctx->req_rel_base, c.max_requests);
+    a.cow = VTK_ARR(ctx, ctx->cow, 2 * (int64_t)c.max_table_blocks);
+    a.per_block = 0;
     a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
@@ -696,6 +822,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     a.theta_den = opts->theta_den;
     a.detach_num = opts->detach_num;
     a.detach_den = opts->detach_den;
+    a.per_block = (opts->protect != nullptr && opts->detach_den != 0 && opts->detach_per_block != 0) ? 1u : 0u;
     a.max_sources = opts->max_source_blocks;
     a.free_blocks = VTK_ARR(ctx, in->free_blocks, c.max_free_blocks);
     a.num_free = VTK_ARR(ctx, in->num_free, 1);
@@ -718,6 +845,10 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
     // n_b and blk_src share one allocation: one node clears both
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, (sizeof(int32_t) + 1) * (size_t)ctx->cfg.num_blocks, st));
+    if (a.per_block) {
+        VTK_CUDA(ctx, cudaMemsetAsync(ctx->cow, 0, sizeof(unsigned long long) * 2 * (size_t)c.max_table_blocks, st));
+        VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_cow_insert_kernel, dim3(R), dim3(256), 0, st, a));
+    }
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_tiles_kernel<0>, tiles_grid, dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_blocks_kernel, dim3(R), dim3(PP_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_tiles_kernel<1>, tiles_grid, dim3(TILE_NT), 0, st, a));

@@ -234,20 +234,22 @@ def test_repack_host_partial_entry_point(opts):
 
 @pytest.mark.parametrize("detach", [(1, 1), (1, 2), (1, 4), (1, 100)], ids=lambda d: f"detach{d[0]}_{d[1]}")
 @pytest.mark.parametrize("degree", [1, 2, 4, 8])
-def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach):
-    """Requests leave their shared prefix when their own tokens fill too little of it: tables, the
-    reclaimed and the released lists, counts and whole pools against the oracle; the shared blocks
-    keep their bytes."""
+@pytest.mark.parametrize("per_block", [False, True], ids=["per_request", "per_block"])
+def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach, per_block):
+    """Requests leave their shared prefix when their own tokens fill too little of it -- all of it at
+    once, or block by block: tables, the reclaimed and the released lists, counts and whole pools
+    against the oracle; the shared blocks keep their bytes."""
     import torch
     from harness.device import DeviceProblem
     w, protect = wl.shared_prefix(seed=10 + degree, groups=2, degree=degree, prefix_len=256, suffix_len=320, layers=2,
                                   heads=2, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
-    prob.plan_partial(protect=torch.from_numpy(protect).to(prob.device), util=(1, 1), detach=detach)
+    prob.plan_partial(protect=torch.from_numpy(protect).to(prob.device), util=(1, 1), detach=detach,
+                      detach_per_block=per_block)
     prob.repack()
     out = prob.outputs()
     p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
-                         w.free_blocks, protect=protect, util=(1, 1), detach=detach)
+                         w.free_blocks, protect=protect, util=(1, 1), detach=detach, detach_per_block=per_block)
     assert out["error_flags"] == 0
     for n in ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"):
         assert out[n] == getattr(p, n), n
@@ -258,10 +260,14 @@ def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach):
     assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
     assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
     assert np.array_equal(out["freed_blocks"], p.freed_blocks)
-    if detach == (1, 1):
+    if detach == (1, 1) and not per_block:
         assert out["num_released"] == degree * 2 * w.notes["prefix_blocks"]       # every sharer left every prefix block
-    if detach == (1, 100):
+    if detach == (1, 100) and not per_block:
         assert out["num_released"] == 0                                           # nobody is that sparse
+    if per_block and detach == (1, 4):
+        # the block rule really splits prefixes here: some request keeps part of its shared blocks
+        kept_shared = np.isin(p.new_bt_blocks, np.flatnonzero(protect)).sum()
+        assert 0 < out["num_released"] and kept_shared > 0
     k, v = host_pools(w)
     k0 = k.copy()
     vto.apply_moves_pools(k, v, p.move_src, p.move_dst)
@@ -303,7 +309,8 @@ def test_detach_needs_a_released_list_everywhere():
 
 @pytest.mark.parametrize("degree", [2, 4])
 @pytest.mark.parametrize("detach", [(1, 1), (1, 2)], ids=lambda d: f"detach{d[0]}_{d[1]}")
-def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, detach):
+@pytest.mark.parametrize("per_block", [False, True], ids=["per_request", "per_block"])
+def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, detach, per_block):
     """Copy-on-write detach through vtoken_repack_waves (references dropped wave after wave, in one list)
     and through vtoken_repack_host_partial (host tables in and out): tables, lists and every byte of both
     pools against the oracle."""
@@ -311,7 +318,7 @@ def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, deta
     from harness.device import DeviceProblem, origin_map
     w, protect = wl.shared_prefix(seed=7, groups=2, degree=degree, prefix_len=256, suffix_len=600, layers=2, heads=1,
                                   head_dim=64)
-    opts = dict(util=(1, 1), max_source_blocks=12, detach=detach)
+    opts = dict(util=(1, 1), max_source_blocks=12, detach=detach, detach_per_block=per_block)
     # ---- waves with a short pool: the detaches are spread over several waves
     need = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
                             w.free_blocks, protect=protect, **opts).num_dst_blocks
@@ -361,5 +368,43 @@ def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, deta
     assert np.array_equal(h_out["new_bt_blocks"].numpy()[:len(p.new_bt_blocks)], p.new_bt_blocks)
     assert np.array_equal(h_out["freed_blocks"].numpy()[:p.num_freed], p.freed_blocks)
     assert np.array_equal(h_out["released_blocks"].numpy()[:c["num_released"]], p.released_blocks)
+    assert prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst)) == 0
+    prob.close()
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_fuzz_detach_on_random_shared_prefix_shapes(seed):
+    """Random prefix-cache shapes (block size, sharing degree, prefix and suffix lengths, kept
+    fraction), thresholds, source bounds and pool cuts, both forms of the detach rule, some requests
+    deselected: tables, lists, counts and every byte of both pools against the oracle."""
+    import torch
+    from harness.device import DeviceProblem, origin_map
+    rng = np.random.default_rng(7000 + seed)
+    S = int(rng.choice([1, 2, 4, 16, 32]))
+    w, protect = wl.shared_prefix(seed=seed, groups=int(rng.integers(1, 4)), degree=int(rng.integers(1, 6)),
+                                  prefix_len=S * max(1, 8 // S) * int(rng.integers(1, 40)),
+                                  suffix_len=int(rng.integers(1, 30 * max(S, 8) + 2)),
+                                  layers=1, heads=1, head_dim=64, block_size=S,
+                                  budget_frac=float(rng.choice([0.1, 0.2, 0.5, 0.9])))
+    if rng.random() < 0.5:
+        w.select = rng.integers(0, 2, size=w.num_requests).astype(np.uint8)
+    opts = dict(util=[(0, 0), (1, 1), (1, 2)][int(rng.integers(0, 3))],
+                max_source_blocks=int(rng.choice([0, 0, 2, 9])),
+                detach=[(1, 1), (1, 2), (1, 4), (3, 4), (5, 4), (1, 16)][int(rng.integers(0, 6))],
+                detach_per_block=bool(seed % 4 != 3))
+    num_free = None if rng.random() < 0.5 else int(rng.integers(0, len(w.free_blocks) + 1))
+    p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
+                         w.select, w.thr_num, w.thr_den, num_free=num_free, protect=protect, **opts)
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    nf_dev = None if num_free is None else torch.tensor([num_free], dtype=torch.int32, device=prob.device)
+    prob.plan_partial(num_free=nf_dev, protect=torch.from_numpy(protect).to(prob.device), **opts)
+    prob.repack()
+    out = prob.outputs()
+    assert out["error_flags"] == 0
+    for n in ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"):
+        assert out[n] == getattr(p, n), n
+    assert out["num_released"] == len(p.released_blocks)
+    for n in ("released_blocks", "req_status", "new_bt_offsets", "new_bt_blocks", "new_tt_slots", "freed_blocks"):
+        assert np.array_equal(out[n], getattr(p, n)), n
     assert prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst)) == 0
     prob.close()

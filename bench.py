@@ -968,9 +968,22 @@ def run_plan_only(args):
                                 elem_bytes=w.elem_bytes)
     side = torch.cuda.Stream(device=dev)
     partial_opts = dict(util=(1, 1), theta=(1, 4))
+    # a protect mask over the first quarter of every block table (the place a shared prefix would take), for the
+    # latency of the copy-on-write rules: all protected blocks of a request at once / block by block
+    import numpy as np
+    protect = np.zeros(w.num_blocks, np.uint8)
+    for r in range(w.num_requests):
+        b0, b1 = int(w.bt_offsets[r]), int(w.bt_offsets[r + 1])
+        protect[w.bt_blocks[b0:b0 + (b1 - b0) // 4]] = 1
+    protect = torch.from_numpy(protect).to(dev)
     res = {}
     for label, fn in (("whole", lambda st: prob.plan(stream=st)),
-                      ("partial", lambda st: prob.plan_partial(stream=st, **partial_opts))):
+                      ("partial", lambda st: prob.plan_partial(stream=st, **partial_opts)),
+                      ("partial_protect", lambda st: prob.plan_partial(stream=st, protect=protect, **partial_opts)),
+                      ("partial_detach_per_request", lambda st: prob.plan_partial(stream=st, protect=protect, detach=(1, 2),
+                                                                                   **partial_opts)),
+                      ("partial_detach_per_block", lambda st: prob.plan_partial(stream=st, protect=protect, detach=(1, 2),
+                                                                                 detach_per_block=True, **partial_opts))):
         with torch.cuda.stream(side):
             fn(side)
         side.synchronize()
@@ -988,7 +1001,8 @@ def run_plan_only(args):
         side.synchronize()
         out = prob.outputs()
         res[label] = {"us": e0.elapsed_time(e1) / args.steps * 1e3, "tokens_moved": out["num_moves"],
-                      "requests_repacked": out["num_admitted"], "error_flags": out["error_flags"]}
+                      "requests_repacked": out["num_admitted"], "references_released": out["num_released"],
+                      "error_flags": out["error_flags"]}
     T = w.num_tokens
     print(json.dumps({"mode": "plan-only", "config": {"workload": f"{w.name} (seed {args.seed})",
                                                       "requests": w.num_requests, "table_entries": T,

@@ -187,17 +187,19 @@ __device__ __forceinline__ unsigned pp_moving_bits(const PArgs &a, unsigned bits
                                                    bool may_detach, int R, int64_t t, int r)
 {
     unsigned mov = 0;
+    if (bits == 0) return 0;                // nothing live (also: entries outside the table, whose owner would
+                                            // have to be searched from the first request on)
     int64_t next = may_detach ? pp_offset(a, r + 1 <= R ? r + 1 : R) : 0;
     Owner o = may_detach ? pp_owner(a, r) : Owner{false, CowTable{0, 0}};
 #pragma unroll
     for (int k = 0; k < TILE_TOK; ++k) {
-        if (may_detach && t + k >= next && r + 1 < R) {
+        if (!((bits >> k) & 1u)) continue;
+        if (may_detach && t + k >= next && r + 1 < R) {      // owners are stepped at live entries only
             while (r + 1 < R && pp_offset(a, r + 1) <= t + k) ++r;
             next = pp_offset(a, r + 1);
             o = pp_owner(a, r);
         }
-        if ((bits >> k) & 1u)
-            if (pp_moves(a, o, slot[k] / a.S)) mov |= 1u << k;
+        if (pp_moves(a, o, slot[k] / a.S)) mov |= 1u << k;
     }
     return mov;
 }
@@ -244,18 +246,20 @@ __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
         if (census) {
             vtk_tile_owners(a.tt_offsets, R, a.max_tokens, base, limit, tile_req);
             __syncthreads();
-            if (t < limit) r = vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t);
-            next = pp_offset(a, r + 1 <= R ? r + 1 : R);
-            if (r >= 0) h = pp_cow_table(a, r);
+            if (t < limit && bits != 0) {
+                r = vtk_entry_owner(a.tt_offsets, a.max_tokens, tile_req, t);
+                next = pp_offset(a, r + 1 <= R ? r + 1 : R);
+                if (r >= 0) h = pp_cow_table(a, r);
+            }
         }
 #pragma unroll
         for (int k = 0; k < TILE_TOK; ++k) {
-            if (census && t + k >= next && r + 1 < R) {
+            if (!((bits >> k) & 1u)) continue;
+            if (census && t + k >= next && r + 1 < R) {      // owners are stepped at live entries only
                 while (r + 1 < R && pp_offset(a, r + 1) <= t + k) ++r;
                 next = pp_offset(a, r + 1);
                 h = pp_cow_table(a, r);
             }
-            if (!((bits >> k) & 1u)) continue;
             const int blk = slot[k] / a.S;
             if (is_tile) atomicAdd(&a.n_b[blk], 1);          // the tile CTAs see every entry exactly once
             ++n;

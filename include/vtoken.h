@@ -136,6 +136,10 @@ typedef struct {
                                       kernels loses about 1 us per boundary, results are identical, and a caller's
                                       own kernel that follows in the stream is ordered as usual.  1: plain
                                       stream-ordered launches */
+    int32_t plan_variant;          /* whole-request planner: 0 auto; 1 three kernels (count, scan, assign); 2 two
+                                      kernels, every CTA redoing the scan over the requests (tables whose grid of
+                                      tiles + requests is resident at once; larger capacities fall back to 1).
+                                      Same results either way; other values are VTOKEN_EINVAL */
     vtoken_copy_tuning tuning;     /* see above; all zero => defaults */
     int64_t debug_stall_item;      /* must be 0 for the production library (VTOKEN_EINVAL otherwise).  The checked
                                       build (libvtoken_checked.so) arms the barrier of work item
@@ -552,6 +556,8 @@ int vtoken_last_cuda_error(const vtoken_ctx *ctx);       /* cudaError_t of the l
 int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int32_t *smem_bytes,
                      int32_t *variant);                   /* launch shape of the copy kernel */
 int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx);      /* device scratch held by the context */
+int vtoken_plan_form(const vtoken_ctx *ctx);              /* planner form vtoken_plan uses for this context's
+                                                             capacities: 1 or 2 as vtoken_config.plan_variant */
 int vtoken_checked_build(void);                           /* 1: this library was compiled with VTOKEN_CHECKED */
 /* Self-test of the checked build: one thread reads element `index` of a context scratch array of
  * max_requests int32 through the same checked accessor every kernel of that build uses, and stores what

@@ -20,7 +20,7 @@ FLAG_BAD_VICTIM, FLAG_APPEND_STOPPED, FLAG_CHECK_FAILED = 64, 128, 256
 
 SYMBOLS = ["vtoken_create", "vtoken_destroy", "vtoken_plan", "vtoken_repack", "vtoken_gather_logical",
            "vtoken_read_counts", "vtoken_repack_host", "vtoken_strerror", "vtoken_last_cuda_error",
-           "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
+           "vtoken_copy_grid", "vtoken_scratch_bytes", "vtoken_plan_form", "vtoken_gather_logical_noalloc", "vtoken_evict_tokens",
            "vtoken_sync_new_tokens", "vtoken_build_slot_mapping", "vtoken_apply_moves",
            "vtoken_block_liveness", "vtoken_plan_partial", "vtoken_digest_logical",
            "vtoken_waves_workspace_bytes", "vtoken_repack_waves", "vtoken_slot_cache_mark",
@@ -53,7 +53,8 @@ class Config(ctypes.Structure):
                 ("max_tokens", ctypes.c_int64), ("max_table_blocks", ctypes.c_int64),
                 ("max_free_blocks", ctypes.c_int32), ("max_ctas", ctypes.c_int32),
                 ("copy_variant", ctypes.c_int32), ("wait_limit_ms", ctypes.c_int32),
-                ("plain_launches", ctypes.c_int32), ("tuning", CopyTuning), ("debug_stall_item", ctypes.c_int64)]
+                ("plain_launches", ctypes.c_int32), ("plan_variant", ctypes.c_int32), ("tuning", CopyTuning),
+                ("debug_stall_item", ctypes.c_int64)]
 
 
 class PlanIn(ctypes.Structure):
@@ -159,6 +160,8 @@ def load():
         lib.vtoken_copy_grid.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 4
         lib.vtoken_scratch_bytes.argtypes = [ctypes.c_void_p]
         lib.vtoken_scratch_bytes.restype = ctypes.c_int64
+        lib.vtoken_plan_form.argtypes = [ctypes.c_void_p]
+        lib.vtoken_plan_form.restype = ctypes.c_int
         lib.vtoken_gather_logical_noalloc.argtypes = (
             [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int64,
              ctypes.c_int64, ctypes.c_void_p, ctypes.c_int32] + [ctypes.c_void_p] * 4 +
@@ -232,7 +235,7 @@ def _check(rc, where, ctx=None):
 
 def vtoken_create(num_layers, num_blocks, block_size, num_kv_heads, head_dim, k_pool, v_pool, max_requests,
                   max_tokens, max_table_blocks, max_free_blocks, elem_bytes=2, layer_stride_bytes=0, max_ctas=0,
-                  copy_variant=0, wait_limit_ms=0, plain_launches=0, tuning=None,
+                  copy_variant=0, wait_limit_ms=0, plain_launches=0, tuning=None, plan_variant=0,
                   debug_stall_item=0) -> int:
     """``tuning``: dict with any of warps, stages, rows, depth, ahead, fixed_shares, chunk, ctas (the fields of
     vtoken_copy_tuning; giving it sets ``enabled``)."""
@@ -244,7 +247,7 @@ def vtoken_create(num_layers, num_blocks, block_size, num_kv_heads, head_dim, k_
             setattr(t, k, int(v))
     cfg = Config(num_layers, num_blocks, block_size, num_kv_heads, head_dim, elem_bytes, _ptr(k_pool), _ptr(v_pool),
                  layer_stride_bytes, max_requests, max_tokens, max_table_blocks, max_free_blocks, max_ctas,
-                 copy_variant, wait_limit_ms, plain_launches, t, debug_stall_item)
+                 copy_variant, wait_limit_ms, plain_launches, plan_variant, t, debug_stall_item)
     ctx = ctypes.c_void_p()
     _check(load().vtoken_create(ctypes.byref(cfg), ctypes.byref(ctx)), "vtoken_create")
     return ctx.value
@@ -339,6 +342,10 @@ def vtoken_debug_probe(ctx, index: int, out_value, stream=None) -> None:
 
 def vtoken_scratch_bytes(ctx) -> int:
     return load().vtoken_scratch_bytes(ctx)
+
+
+def vtoken_plan_form(ctx) -> int:
+    return load().vtoken_plan_form(ctx)
 
 
 NOALLOC_MAX_REQUESTS = 4096

@@ -97,6 +97,7 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     const int64_t row_bytes = (int64_t)cfg->num_kv_heads * cfg->head_dim * cfg->elem_bytes;
     const int64_t slots = (int64_t)cfg->num_blocks * cfg->block_size;
     if (row_bytes % 16 != 0) return VTOKEN_EINVAL;
+    if (cfg->plan_variant < 0 || cfg->plan_variant > 2) return VTOKEN_EINVAL;
     if (slots >= (int64_t)INT32_MAX) return VTOKEN_EINVAL;            // slots are int32
     if (cfg->max_tokens >= (int64_t)INT32_MAX || cfg->max_table_blocks >= (int64_t)INT32_MAX) return VTOKEN_EINVAL;
     const int64_t stride = cfg->layer_stride_bytes ? cfg->layer_stride_bytes : slots * row_bytes;
@@ -161,6 +162,7 @@ int vtoken_create(const vtoken_config *cfg, vtoken_ctx **out_ctx)
     A(&ctx->cow, 2 * (int64_t)cfg->max_table_blocks);
     if (rc == VTOKEN_OK && cudaMemset(ctx->counts, 0, sizeof(vtoken_counts)) != cudaSuccess) rc = VTOKEN_ECUDA;
     if (rc == VTOKEN_OK) rc = vtk_configure_copy(ctx);
+    if (rc == VTOKEN_OK) rc = vtk_configure_plan(ctx);
     if (rc != VTOKEN_OK) { free_all(ctx); delete ctx; return rc; }
     *out_ctx = ctx;
     return VTOKEN_OK;
@@ -365,6 +367,8 @@ int vtoken_copy_grid(const vtoken_ctx *ctx, int32_t *ctas, int32_t *threads, int
 }
 
 int64_t vtoken_scratch_bytes(const vtoken_ctx *ctx) { return ctx ? ctx->scratch_bytes : 0; }
+
+int vtoken_plan_form(const vtoken_ctx *ctx) { return ctx ? ctx->plan_form : VTOKEN_EINVAL; }
 
 namespace {
 __global__ void probe_kernel(vtk_arr<int32_t> arr, int64_t index, int32_t *out)

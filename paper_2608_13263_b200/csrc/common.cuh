@@ -52,6 +52,7 @@ struct vtoken_ctx {
     int32_t *req_shared;       // [max_requests] protected entries of the request's block table
     int32_t *req_detach;       // [max_requests] 1 = the request leaves its protected blocks (copy-on-write detach)
     int32_t *req_rel_base;     // [max_requests] first entry in released_blocks
+    int plan_form;             // whole-request planner of this context: 1 three kernels (plan.cu), 2 two kernels (plan_small.cu)
     unsigned long long *cow;   // [2 * max_table_blocks] detach per shared block: every request's hash from a protected
                                // block of its table to its own live tokens there ((block id + 1) << 32 | count)
     uint32_t *slot_bits;       // [ceil(num_blocks * S / 32)] one bit per slot (vtoken_check_tables)
@@ -149,6 +150,7 @@ struct vtk_arr {
 // host launchers, one per translation unit
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
 int vtk_launch_plan_small(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st);
+int vtk_configure_plan(vtoken_ctx *ctx);         // once per context: which form of the whole-request planner it uses
 int vtk_launch_copy(vtoken_ctx *ctx, cudaStream_t st);
 int vtk_configure_copy(vtoken_ctx *ctx);
 // > 0: launched; 0: the context has no bulk configuration for these rows; < 0: VTOKEN_* error

@@ -353,15 +353,8 @@ __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
 
 int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st)
 {
-    // A table whose whole grid is resident at once takes the two-kernel planner (plan_small.cu): one kernel
-    // boundary less, at the price of a scan that every CTA redoes -- which pays while the CTAs are few.
-    // Measured on B200 (whole plan, graph replay): 8.2 instead of 11.5 us on a 4-request table, even up to
-    // about 330 tiles + 256 requests, 49 instead of 27 us at 2 196 tiles + 512 requests.  The checked build
-    // always takes the three kernels below, so that both planners see the small tables of the tests.
-#ifndef VTOKEN_CHECKED
-    if ((ctx->cfg.max_tokens + TILE - 1) / TILE + ctx->cfg.max_requests + 1 <= (int64_t)ctx->num_sms * 4)
-        return vtk_launch_plan_small(ctx, in, out, st);
-#endif
+    // the two-kernel form (plan_small.cu; vtk_configure_plan chose at create time)
+    if (ctx->plan_form == 2) return vtk_launch_plan_small(ctx, in, out, st);
     PlanArgs a;
     const vtoken_config &c = ctx->cfg;
     const int64_t tiles_cap = (c.max_tokens + TILE - 1) / TILE;

@@ -15,7 +15,10 @@
 // (header; entries, tile counts and request inputs; free-list entries).  The redundant scan costs
 // every CTA about 2 us of issue slots, which a grid of one wave hides and a grid of five does not:
 // measured on B200, 8.2 us instead of 11.5 on a 4-request table, even at 160 and 330 tiles, 49 us
-// instead of 27 at 2 196 tiles -- hence the size limit (vtk_launch_plan decides).
+// instead of 27 at 2 196 tiles -- hence the size limit (vtk_configure_plan decides).  A grid of one wave
+// that redoes the scan once per CTA, keeps its results in shared memory and walks over the tiles in steps
+// of the grid size was measured too: 30.9 us on the same table (four to five dependent rounds of loads
+// per CTA in a row at half the occupancy of the three-kernel assign pass), so large tables keep three kernels.
 #include "common.cuh"
 
 namespace {
@@ -534,6 +537,25 @@ __global__ void __launch_bounds__(TILE_NT, MIN_CTAS) plan_small_assign_kernel(Pl
 }
 
 }  // namespace
+
+// Which form of the whole-request planner this context uses (ctx->plan_form: 1 three kernels, 2 two kernels).
+// Two kernels instead of three -- one kernel boundary less, at the price of a scan over the requests that
+// every CTA redoes -- pay while the whole grid (tiles + requests + 1 CTAs) is resident at once, so that the
+// scan is paid once per resident CTA; everything else takes the three kernels.  vtoken_config.plan_variant
+// forces a form where it fits.  The checked build defaults to the three kernels.
+int vtk_configure_plan(vtoken_ctx *ctx)
+{
+    const int64_t roles = (ctx->cfg.max_tokens + TILE - 1) / TILE + ctx->cfg.max_requests + 1;
+    const bool resident_ok = roles <= (int64_t)ctx->num_sms * MIN_CTAS;
+    int form = ctx->cfg.plan_variant;
+#ifdef VTOKEN_CHECKED
+    if (form == 0) form = 1;
+#endif
+    if (form == 0) form = resident_ok ? 2 : 1;
+    if (form == 2 && !resident_ok) form = 1;
+    ctx->plan_form = form;
+    return VTOKEN_OK;
+}
 
 // The caller (vtk_launch_plan) has checked that the grid is small enough for this planner.
 int vtk_launch_plan_small(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st)

@@ -4,8 +4,8 @@ slab is compared with the array's size; an index outside it raises VTOKEN_FLAG_C
 is skipped, nothing faults.  This file runs the parity tests of the other files once more against that
 build -- same oracle, same bit-exact bar -- and requires the flag to stay clear, which also covers what a
 comparison of results cannot see: a read beyond an array, a stray write into the context's scratch.
-(The checked build always plans with the three-kernel planner, the production build uses the
-two-kernel one on tables this small: between the two runs both are exercised.)"""
+(The checked build plans with the three-kernel planner unless told otherwise, the production build
+uses the two-kernel one on tables this small; the two-kernel planner is run under the checker as well.)"""
 import numpy as np
 import pytest
 
@@ -81,6 +81,7 @@ def test_small_configs_whole_pool(checked):
     for w in tp.small_configs():
         for variant in (1, 2):
             tp.run_and_compare(w, copy_variant=variant)      # tables, lists, counts, every byte; flags == 0
+        tp.run_and_compare(w, copy_variant=2, plan_variant=2, whole_pool=False)      # the two-kernel planner's indices
 
 
 def test_edges_and_shapes(checked):

@@ -1,0 +1,111 @@
+"""The whole-request planner exists in two forms that must give the same plan: three kernels
+(count, scan, assign) and two kernels in which every CTA redoes the scan over the requests.
+`vtoken_plan` picks one from the context's capacities (small tables: two kernels);
+`vtoken_config.plan_variant` forces one.  This file runs the parity, edge-case, wave and serving-loop
+tests of the other files once per form -- same oracle, same bit-exact bar -- and checks that the form
+asked for is the form that ran (in most of the contexts: a few tests ask for capacities of thousands
+of requests, which only the three kernels take)."""
+import numpy as np
+import pytest
+
+from harness import workloads as wl
+from oracle import vto
+from paper_2608_13263_b200 import binding as vt
+
+pytestmark = pytest.mark.gpu
+
+FORMS = {1: "three_kernels", 2: "two_kernels"}
+
+
+@pytest.fixture(params=sorted(FORMS), ids=lambda f: FORMS[f])
+def form(request, monkeypatch):
+    """Every context created inside the test plans with this form."""
+    create = vt.vtoken_create
+    seen = []
+
+    def create_with_form(*args, **kw):
+        kw.setdefault("plan_variant", request.param)
+        ctx = create(*args, **kw)
+        seen.append(vt.vtoken_plan_form(ctx))
+        return ctx
+
+    monkeypatch.setattr(vt, "vtoken_create", create_with_form)
+
+    class Seen:
+        @staticmethod
+        def check():
+            # (a context whose capacities are beyond a resident grid falls back to the three kernels)
+            assert seen and all(f in (request.param, 1) for f in seen)
+            assert sum(f == request.param for f in seen) * 2 > len(seen), "the form asked for hardly ever ran"
+            seen.clear()
+
+        @staticmethod
+        def forget():
+            seen.clear()
+
+    yield Seen
+    if seen:
+        Seen.check()
+
+
+def test_small_configs_and_shapes(form):
+    import test_gpu_parity as tp
+    for w in tp.small_configs():
+        tp.run_and_compare(w, copy_variant=2)
+    for S, heads, head_dim in ((1, 1, 8), (3, 2, 64), (48, 8, 128), (5, 3, 8)):
+        w = wl.mistral7b_random(seed=S, requests=5, lo=10, hi=40 * S + 20, layers=2, heads=heads, head_dim=head_dim,
+                                block_size=S)
+        tp.run_and_compare(w, copy_variant=1)
+
+
+def test_edge_cases(form):
+    import test_gpu_parity as tp
+    tp.test_edge_all_keep_all_evict_empty_and_boundaries()
+    tp.test_edge_free_list_cut_at_every_length()
+    tp.test_edge_select_threshold_and_holes()
+    tp.test_repeated_repack_and_idempotence()
+    tp.test_tables_that_are_not_16_byte_aligned("whole")
+    tp.test_token_table_that_does_not_start_at_entry_zero("whole")
+    form.check()
+    # capacities beyond a resident grid: the two-kernel form may not fit and then falls back to the three kernels
+    tp.test_long_and_one_token_requests_in_one_batch()
+    tp.test_out_of_range_ids_raise_flags_not_faults(4, 64)
+    tp.test_counts_above_capacity_are_clamped_and_flagged()
+    tp.test_tables_beyond_the_context_capacities_are_clipped("whole")
+    tp.test_capacities_larger_than_the_problem()
+    form.forget()
+
+
+def test_graph_replay_host_tables_and_waves(form):
+    import test_gpu_parity as tp
+    import test_gpu_waves as tw
+    tp.test_graph_capture_side_stream_replay_with_new_contents()
+    tp.test_repack_host_tables_entry_point()
+    ws = tw.small_configs()
+    tw.test_waves_with_the_headroom_of_one_request(ws[1], 3)      # the commit of a wave reads the planner's scratch
+    tw.test_waves_pool_sizes(ws[2], 0.5)
+
+
+def test_fuzz_and_serving_loop(form):
+    import test_gpu_fuzz as tf
+    import test_gpu_runtime as tr
+    for seed in range(12):
+        tf.test_fuzz_whole_and_partial_plans(seed)
+    for seed in range(4):
+        tf.test_fuzz_repack_in_waves(seed)
+    tr.test_serving_loop_matches_oracle_step_by_step(0, 4, (), ())
+
+
+def test_many_requests_per_tile_and_many_tiles_per_request(form):
+    """Hundreds of one- and two-token requests inside single tiles (every thread steps over request
+    boundaries), then a few requests of several tiles each, then both mixed with empty requests."""
+    import test_gpu_parity as tp
+    rng = np.random.default_rng(3)
+    S = 4
+    for lens in ([1, 2] * 250, [5000, 3000, 4100], [0, 1, 2500, 0, 0, 3, 1, 1, 2047, 1025, 0, 2, 7000, 1, 0]):
+        keeps = [rng.random(n) < 0.6 for n in lens]
+        w = tp._custom(S, lens, keeps, free_extra=4000)
+        tp.run_and_compare(w, copy_variant=1)
+        p = vto.plan_workload(w)
+        for nf in (0, 1, p.num_dst_blocks // 2, max(0, p.num_dst_blocks - 1)):
+            tp.run_and_compare(w, copy_variant=1, num_free=nf, whole_pool=False)

@@ -24,7 +24,7 @@ struct vtoken_ctx {
 
     // planner scratch (DEVICE)
     int32_t *req_n;            // [max_requests] live tokens (partial planner)
-    int32_t *plan_header;      // [4] small-table planner: R, T, num_free, first entry as its count kernel read them
+    int32_t *plan_header;      // [4] R, T, num_free, first entry as the first kernel of a plan read them (one load downstream)
     int32_t *part_n;           // [max_requests * VTK_PLAN_PARTS] live tokens per request part: only the context-free
                                // gather entry point (per-request index kernels) sets it, from its static scratch
     int32_t *req_dst_base;     // [max_requests] first destination block (index into the free list)

@@ -39,6 +39,8 @@ struct PlanArgs {
     vtk_arr<int32_t> req_part;    // [max_requests + 1] live tokens between the start of the tile that holds the
                                   // request's first entry and that entry
     vtk_arr<int32_t> req_before;  // [max_requests + 1] live tokens before the request's first entry
+    vtk_arr<int32_t> header;      // [4] R, T, num_free, first entry as the tiles kernel read them: one load for the
+                                  // kernels behind it instead of a chain of dependent ones
     vtk_arr<vtoken_counts> counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks, num_tiles;
     int32_t vec_in, vec_out;   // tt_slots 16-byte / keep 4-byte aligned; new_tt_slots 16-byte aligned
@@ -77,6 +79,12 @@ __global__ void __launch_bounds__(TILE_NT) plan_tiles_kernel(PlanArgs a)
     const int R = clamp_requests(a);
     const int64_t T = clipped_offset(a, R);
     const int lane = vtk_lane(), warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        a.header[0] = R;
+        a.header[1] = (int32_t)T;
+        a.header[2] = *a.num_free;
+        a.header[3] = (int32_t)clipped_offset(a, 0);
+    }
     // A CTA counts the live entries of [base, limit): a whole tile, or -- the CTAs behind the tiles, one
     // per request boundary -- the entries between the start of the boundary's tile and the boundary
     // (entries the tile's own CTA counts as well; flags are raised there).  Either way one pass.
@@ -128,6 +136,28 @@ __device__ __forceinline__ Acc shfl_up(const Acc &v, int d)
                __shfl_up_sync(0xffffffffu, v.admitted, d), __shfl_up_sync(0xffffffffu, v.deferred, d)};
 }
 
+constexpr int SCAN_STAGED = 8192;                // running counts of that many tiles are kept in shared memory
+
+// What the scan reads from global memory for one request, requested in one go.
+struct ScanInputs {
+    int tt0, tt1, bt0, bt1, part0, part1;
+    unsigned char sel;
+};
+__device__ __forceinline__ ScanInputs load_scan_inputs(const PlanArgs &a, int r, int R)
+{
+    ScanInputs in{0, 0, 0, 0, 0, 0, 1};
+    if (r < R) {
+        in.tt0 = a.tt_offsets[r];
+        in.tt1 = a.tt_offsets[r + 1];
+        in.bt0 = a.bt_offsets[r];
+        in.bt1 = a.bt_offsets[r + 1];
+        in.part0 = a.req_part[r];          // (scratch of the tiles kernel: only used when the offset is inside a tile)
+        in.part1 = a.req_part[r + 1];
+        if (!a.select.null()) in.sel = a.select[r];
+    }
+    return in;
+}
+
 __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 {
     __shared__ long long warp_ll[32];
@@ -135,68 +165,98 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
     __shared__ long long carry_need;
     __shared__ Acc carry;
     __shared__ int warp_i[32];
-    __shared__ int carry_live;
     __shared__ unsigned int all_flags;
+    __shared__ int staged[SCAN_STAGED + 1];
     const int tid = threadIdx.x;
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    const int R = clamp_requests(a);
+    // R, T and num_free in one load; the inputs of the first 1024 requests and the tile counts are requested
+    // right behind it, before anything is computed
+    const int4 hdr = *reinterpret_cast<const int4 *>(a.header.at(0, 4));
+    const int R = hdr.x;
+    const int64_t T = hdr.y;
+    int nf = hdr.z;
     uint32_t flags = 0;
     if (tid == 0) {
-        if (*a.num_requests > a.max_requests || *a.num_requests < 0) flags |= VTOKEN_FLAG_CAPACITY;
+        const int raw = *a.num_requests;
+        if (raw > a.max_requests || raw < 0) flags |= VTOKEN_FLAG_CAPACITY;
+        if (nf > a.max_free_blocks) flags |= VTOKEN_FLAG_CAPACITY;
         carry_need = 0;
-        carry_live = 0;
         all_flags = 0;
         carry = Acc{0, 0, 0, 0, 0, 0};
     }
-    int nf = *a.num_free;
-    if (nf > a.max_free_blocks && tid == 0) flags |= VTOKEN_FLAG_CAPACITY;
     nf = nf < 0 ? 0 : (nf > a.cap_dst_blocks ? a.cap_dst_blocks : nf);
-    __syncthreads();
+    ScanInputs in = load_scan_inputs(a, tid, R);
 
     auto shfl_ll = [](long long v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
     auto shfl_acc = [](const Acc &v, int d) { return shfl_up(v, d); };
     auto shfl_int = [](int v, int d) { return __shfl_up_sync(0xffffffffu, v, d); };
 
-    // live tokens before every tile (in place: tile_n[i] becomes the sum of the tiles before i; one
-    // entry past the last tile holds the total)
-    const int64_t T = clipped_offset(a, R);
+    // live tokens before every tile (in place: tile_n[i] becomes the sum of the tiles before i; one entry
+    // past the last tile holds the total): every thread sums a run of consecutive tiles, one scan over the
+    // runs, every thread writes the running counts of its run -- to global memory for the assign kernel
+    // and, while they fit, to shared memory for the request pass below
     const int tiles = (int)((T + TILE - 1) / TILE);
-    for (int base = 0; base <= tiles; base += SCAN_NT) {
-        const int i = base + tid;
-        const int raw = i < tiles ? a.tile_n[i] : 0;
-        if (raw < 0) flags |= VTOKEN_FLAG_BAD_SLOT;
-        const int v = raw & 0x7fffffff;
-        const int incl = vtk_block_incl_scan<int>(v, warp_i, 0, shfl_int) + carry_live;
-        if (i <= tiles) a.tile_n[i] = incl - v;
-        __syncthreads();
-        if (tid == SCAN_NT - 1) carry_live = incl;
-        __syncthreads();
+    const bool fits = tiles <= SCAN_STAGED;
+    {
+        const int per = (tiles + 1 + SCAN_NT - 1) / SCAN_NT;
+        const int j0 = min(tiles + 1, tid * per), j1 = min(tiles + 1, j0 + per);
+        int sum = 0, any = 0;
+        if (per <= 4) {
+            int v[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) v[k] = (j0 + k < j1 && j0 + k < tiles) ? a.tile_n[j0 + k] : 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { sum += v[k] & 0x7fffffff; any |= v[k]; }
+            __syncthreads();                                       // (carry_need, carry, all_flags are set)
+            int run = vtk_block_incl_scan<int>(sum, warp_i, 0, shfl_int) - sum;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                if (j0 + k < j1) {
+                    a.tile_n[j0 + k] = run;
+                    if (fits) staged[j0 + k] = run;
+                }
+                run += v[k] & 0x7fffffff;
+            }
+        } else {
+            for (int j = j0; j < j1; ++j) { const int v = j < tiles ? a.tile_n[j] : 0; sum += v & 0x7fffffff; any |= v; }
+            __syncthreads();
+            int run = vtk_block_incl_scan<int>(sum, warp_i, 0, shfl_int) - sum;
+            for (int j = j0; j < j1; ++j) {
+                const int v = j < tiles ? (a.tile_n[j] & 0x7fffffff) : 0;
+                a.tile_n[j] = run;
+                if (fits) staged[j] = run;
+                run += v;
+            }
+        }
+        if (any < 0) flags |= VTOKEN_FLAG_BAD_SLOT;
     }
+    __syncthreads();
+    const int32_t *before_tile = fits ? staged : a.tile_n.at(0, (int64_t)tiles + 1);
+    auto clip = [](int64_t o, int64_t cap) { return o < 0 ? (int64_t)0 : (o > cap ? cap : o); };
     // live tokens before table entry o = live tokens before its tile + those between the tile's start and o
-    auto live_before = [&](int r) {
-        const int64_t o = clipped_offset(a, r);
-        return a.tile_n[o / TILE] + (o % TILE != 0 ? a.req_part[r] : 0);
-    };
+    auto live_before = [&](int64_t o, int part) { return before_tile[o / TILE] + (o % TILE != 0 ? part : 0); };
 
     for (int base = 0; base < R; base += SCAN_NT) {
         const int r = base + tid;
         const bool valid = r < R;
+        if (base > 0) in = load_scan_inputs(a, r, R);
         int n = 0, nb = 0;
         if (valid) {
-            const int before = live_before(r);
-            n = live_before(r + 1) - before;
+            // table ranges clipped to the create-time capacities (a range that runs backwards is empty)
+            const int64_t t0 = clip(in.tt0, a.max_tokens), t1 = clip(in.tt1, a.max_tokens);
+            const int64_t lo = clip(in.bt0, a.max_table_blocks), b1 = clip(in.bt1, a.max_table_blocks);
+            const int64_t hi = b1 < lo ? lo : b1;
+            if (lo != in.bt0 || hi != in.bt1 || t0 != in.tt0 || (t1 < t0 ? t0 : t1) != in.tt1) flags |= VTOKEN_FLAG_CAPACITY;
+            const int before = live_before(t0, in.part0);
+            n = live_before(t1, in.part1) - before;
             if (n < 0) n = 0;                                // offsets that run backwards
             a.req_before[r] = before;
             a.req_n[r] = n;
-            int64_t lo, hi, t0, t1;
-            const bool clipped = vtk_range(a.bt_offsets, r, a.max_table_blocks, lo, hi) |
-                                 vtk_range(a.tt_offsets, r, a.max_tokens, t0, t1);
-            if (clipped) flags |= VTOKEN_FLAG_CAPACITY;     // tables beyond the create-time capacities
             nb = (int)(hi - lo);
         }
         const int need = (int)(((int64_t)n + a.S - 1) / a.S);       // ceil(T_live / S)
-        bool sel = valid && (a.select.null() || a.select[r] != 0);
+        bool sel = valid && in.sel != 0;
         if (sel && a.thr_den != 0)
             sel = (unsigned long long)n * a.thr_den <
                   (unsigned long long)a.thr_num * (unsigned long long)nb * (unsigned long long)a.S;
@@ -242,13 +302,14 @@ __global__ void __launch_bounds__(SCAN_NT) plan_scan_kernel(PlanArgs a)
 }
 
 // ---- assign ----------------------------------------------------------------------------
-__global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
+__global__ void __launch_bounds__(TILE_NT, 8) plan_assign_kernel(PlanArgs a)
 {
     __shared__ int warp_sums[TILE_NT / 32];
     __shared__ int tile_req[2];
     vtk_release_successor();
     vtk_wait_for_predecessor();
-    const int R = clamp_requests(a);
+    const int4 hdr = *reinterpret_cast<const int4 *>(a.header.at(0, 4));      // R, T, num_free, first entry
+    const int R = hdr.x;
     const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
     const int S = a.S;
     uint32_t flags = 0;
@@ -288,13 +349,13 @@ __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
     }
 
     // token table: rank of each live token in logical order -> destination slot
-    const int64_t T = clipped_offset(a, R);
+    const int64_t T = hdr.y, first = hdr.w;
     const int64_t base = (int64_t)blockIdx.x * TILE;
     if (base >= T) return;
     const int64_t t = base + tid * TILE_TOK;
     int32_t slot[TILE_TOK];
     bool bad = false;
-    const unsigned bits = load_entries(a, t, T, slot, bad);
+    const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, first, T, a.slots_per_layer, slot, bad);
     // live tokens of the whole table before this thread's first entry
     const int cnt = __popc(bits);
     const int incl = vtk_warp_incl_scan(cnt);
@@ -342,7 +403,6 @@ __global__ void __launch_bounds__(TILE_NT) plan_assign_kernel(PlanArgs a)
         *reinterpret_cast<int4 *>(a.new_tt_slots.at(t, TILE_TOK)) = make_int4(out[0], out[1], out[2], out[3]);
     } else {
         // the ragged end of the table, or entries in front of the first request (left untouched)
-        const int64_t first = clipped_offset(a, 0);
 #pragma unroll
         for (int k = 0; k < TILE_TOK; ++k)
             if (t + k < T && t + k >= first) a.new_tt_slots[t + k] = out[k];
@@ -384,6 +444,7 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
     a.tile_n = VTK_ARR(ctx, ctx->tile_n, tiles_cap + 1);
     a.req_part = VTK_ARR(ctx, ctx->req_part, (int64_t)c.max_requests + 1);
     a.req_before = VTK_ARR(ctx, ctx->req_before, (int64_t)c.max_requests + 1);
+    a.header = VTK_ARR(ctx, ctx->plan_header, 4);
     a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;

@@ -415,7 +415,7 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
 {
     // the two-kernel form (plan_small.cu; vtk_configure_plan chose at create time)
     if (ctx->plan_form == 2) return vtk_launch_plan_small(ctx, in, out, st);
-    PlanArgs a;
+    PlanArgs a{};
     const vtoken_config &c = ctx->cfg;
     const int64_t tiles_cap = (c.max_tokens + TILE - 1) / TILE;
     a.num_requests = VTK_ARR(ctx, in->num_requests, 1);

@@ -807,7 +807,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     if (opts->max_source_blocks < 0) return VTOKEN_EINVAL;
     if (opts->protect != nullptr && opts->detach_den != 0 && !out->released_blocks) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    PArgs a;
+    PArgs a{};
     fill_args(a, ctx);
     const vtoken_config &c = ctx->cfg;
     a.num_requests = VTK_ARR(ctx, in->num_requests, 1);
@@ -869,8 +869,7 @@ int vtoken_block_liveness(vtoken_ctx *ctx, const int32_t *num_requests, const in
 {
     if (!ctx || !num_requests || !bt_offsets || !bt_blocks || !tt_offsets || !tt_slots || !n_b) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    PArgs a;
-    memset(&a, 0, sizeof(a));
+    PArgs a{};                                   // the planning options stay zero: only the counting pass runs
     fill_args(a, ctx);
     const vtoken_config &c = ctx->cfg;
     a.num_requests = VTK_ARR(ctx, num_requests, 1);

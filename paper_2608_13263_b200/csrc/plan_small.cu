@@ -560,7 +560,7 @@ int vtk_configure_plan(vtoken_ctx *ctx)
 // The caller (vtk_launch_plan) has checked that the grid is small enough for this planner.
 int vtk_launch_plan_small(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan_out *out, cudaStream_t st)
 {
-    PlanArgs a;
+    PlanArgs a{};
     const vtoken_config &c = ctx->cfg;
     a.num_requests = VTK_ARR(ctx, in->num_requests, 1);
     a.bt_offsets = VTK_ARR(ctx, in->bt_offsets, (int64_t)c.max_requests + 1);

@@ -676,3 +676,46 @@ def test_decode_read_proxy_is_undisturbed_by_a_concurrent_repack():
     assert np.array_equal(prob.k_pool.cpu().numpy().view(np.uint16), k)
     assert np.array_equal(prob.v_pool.cpu().numpy().view(np.uint16), v)
     prob.close()
+
+
+@pytest.mark.parametrize("tp", [2, 8])
+def test_tensor_parallel_shards_repack_identically(tp):
+    """Under tensor parallelism every shard holds the same blocks with its share of the KV heads
+    (Sec. 6: shard-local block ids, nothing to exchange): the same tables planned on a shard's
+    context give the same plan, and its pools after the repack are the head slice of the unsharded
+    result -- which is the oracle's.  tp = 8 with 8 heads leaves rows of one head (256 bytes)."""
+    import dataclasses
+    from harness.device import DeviceProblem
+    torch = _torch()
+    w = wl.llama8b_h2o(seed=4, requests=5, lo=200, hi=700, layers=2, heads=8, head_dim=128)
+    full = DeviceProblem(w, fill_seed=FILL_SEED)
+    L, slots, H, D = w.num_layers, w.slots_per_layer, w.num_kv_heads, w.head_dim
+    before_k = full.k_pool.view(L, slots, H, D).clone()
+    before_v = full.v_pool.view(L, slots, H, D).clone()
+    full.plan()
+    full.repack()
+    out = full.outputs()
+    p = vto.plan_workload(w)
+    assert_tables_equal(out, p, w)
+    k, v = host_pools(w)
+    vto.apply_moves_pools(k, v, p.move_src, p.move_dst, threads=2)
+    assert np.array_equal(full.k_pool.cpu().numpy().view(np.uint16), k)
+    assert np.array_equal(full.v_pool.cpu().numpy().view(np.uint16), v)
+    after_k, after_v = full.k_pool.view(L, slots, H, D), full.v_pool.view(L, slots, H, D)
+    per = H // tp
+    ws = dataclasses.replace(w, num_kv_heads=per)
+    for s in range(tp):
+        heads = slice(s * per, (s + 1) * per)
+        shard = DeviceProblem(ws, fill_seed=FILL_SEED)
+        shard.k_pool.copy_(before_k[:, :, heads, :].reshape(L, slots, per * D))
+        shard.v_pool.copy_(before_v[:, :, heads, :].reshape(L, slots, per * D))
+        shard.plan()
+        shard.repack()
+        so = shard.outputs()
+        assert so["error_flags"] == 0
+        for name in ("new_bt_offsets", "new_bt_blocks", "new_tt_slots", "freed_blocks", "req_status", "num_moves"):
+            assert np.array_equal(so[name], out[name]), name
+        assert torch.equal(shard.k_pool.view(L, slots, per, D), after_k[:, :, heads, :])
+        assert torch.equal(shard.v_pool.view(L, slots, per, D), after_v[:, :, heads, :])
+        shard.close()
+    full.close()

@@ -367,7 +367,7 @@ class _PartialOpts(ctypes.Structure):
     _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
                 ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32),
                 ("detach_num", ctypes.c_uint32), ("detach_den", ctypes.c_uint32),
-                ("detach_per_block", ctypes.c_uint32)]
+                ("detach_rule", ctypes.c_uint32)]
 
 
 def block_liveness(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep=None):
@@ -388,7 +388,7 @@ def block_liveness(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep=None
 
 def plan_partial(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, select=None, thr_num=0,
                  thr_den=0, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
-                 detach=(0, 0), detach_per_block=False) -> Plan:
+                 detach=(0, 0), detach_rule=0) -> Plan:
     bt_offsets, bt_blocks = _i32(bt_offsets), _i32(bt_blocks)
     tt_offsets, tt_slots = _i32(tt_offsets), _i32(tt_slots)
     keep, select, free_blocks, protect = _u8(keep), _u8(select), _i32(free_blocks), _u8(protect)
@@ -408,7 +408,7 @@ def plan_partial(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_
     c = _Counts()
     released = np.full(max(nbt, 1), -7, np.int32)
     o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1], max_source_blocks,
-                     theta[0], theta[1], detach[0], detach[1], int(bool(detach_per_block)))
+                     theta[0], theta[1], detach[0], detach[1], int(detach_rule))
     rc = lib().vto_plan_partial(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
                                 _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),
                                 _p(tt_slots, np.int32), _p(keep, np.uint8), _p(select, np.uint8),
@@ -490,7 +490,7 @@ def plan_waves(S, NB, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_bl
         util, theta, detach = partial.get("util", (0, 0)), partial.get("theta", (0, 0)), partial.get("detach", (0, 0))
         o = _PartialOpts(None if protect is None else protect.ctypes.data, util[0], util[1],
                          partial.get("max_source_blocks", 0), theta[0], theta[1], detach[0], detach[1],
-                         int(bool(partial.get("detach_per_block", False))))
+                         int(partial.get("detach_rule", 0)))
     released = np.full(max(nbt, 1), -7, np.int32)
     rc = lib().vto_plan_waves(ctypes.c_int32(R), ctypes.c_int32(S), ctypes.c_int32(NB),
                               _p(bt_offsets, np.int32), _p(bt_blocks, np.int32), _p(tt_offsets, np.int32),

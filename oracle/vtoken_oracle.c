@@ -593,6 +593,7 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
     if (R < 0 || S < 1 || NB < 1 || num_free < 0 || !opts || !counts) return VTO_EINVAL;
     const int may_detach = opts->protect != NULL && opts->detach_den != 0;
     if (may_detach && !released_blocks) return VTO_EINVAL;
+    if (opts->detach_rule > 2) return VTO_EINVAL;
     int32_t *n_b = (int32_t *)malloc(sizeof(int32_t) * (size_t)NB);
     uint8_t *is_source = (uint8_t *)malloc((size_t)NB);     /* per physical block, for the request at hand */
     int32_t *own_live = (int32_t *)calloc((size_t)NB, sizeof(int32_t));   /* n_rb: live tokens of the request at
@@ -631,7 +632,7 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
             detach = ns_shared > 0 &&
                      (uint64_t)n_shared * opts->detach_den < (uint64_t)opts->detach_num * (uint64_t)ns_shared * (uint64_t)S;
             /* block by block instead: the census of the request's own live tokens per block */
-            if (opts->detach_per_block)
+            if (opts->detach_rule == 1)
                 for (int64_t t = t0; t < t1; ++t)
                     if (is_live(tt_slots, keep, t)) ++own_live[tt_slots[t] / S];
         }
@@ -647,8 +648,10 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
             if (eligible && opts->max_source_blocks > 0 && ns_unprotected >= opts->max_source_blocks) eligible = 0;
             ns_unprotected += eligible;
             if (shared && may_detach) {
-                if (opts->detach_per_block)                /* the shared blocks this request fills poorly */
+                if (opts->detach_rule == 1)                /* the shared blocks this request fills poorly */
                     eligible = (uint64_t)own_live[b] * opts->detach_den < (uint64_t)opts->detach_num * (uint64_t)S;
+                else if (opts->detach_rule == 2)           /* the shared blocks all their holders together fill poorly */
+                    eligible = (uint64_t)n_b[b] * opts->detach_den < (uint64_t)opts->detach_num * (uint64_t)S;
                 else
                     eligible = detach;                     /* every shared block of a detaching request */
             }
@@ -709,7 +712,7 @@ int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
             for (int32_t j = b0; j < b1; ++j) new_bt_blocks[new_bt_fill++] = bt_blocks[j];
         }
         for (int32_t j = b0; j < b1; ++j) is_source[bt_blocks[j]] = 0;
-        if (may_detach && opts->detach_per_block)
+        if (may_detach && opts->detach_rule == 1)
             for (int64_t t = t0; t < t1; ++t)
                 if (is_live(tt_slots, keep, t)) own_live[tt_slots[t] / S] = 0;
     }

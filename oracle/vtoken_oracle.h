@@ -224,9 +224,11 @@ typedef struct {
     uint32_t detach_num, detach_den; /* copy-on-write detach: a request leaves ALL its protected blocks when its own
                                      live tokens in them fill less than detach_num / detach_den of those blocks;
                                      detach_den == 0: never (protected blocks always stay) */
-    uint32_t detach_per_block;    /* non-zero: the detach threshold is applied to every protected block of the
-                                     request by itself: it leaves block b when its own live tokens stored in b
-                                     number n_rb with n_rb * detach_den < detach_num * S, and stays in the others */
+    uint32_t detach_rule;         /* what the detach threshold is applied to.  0: the request's protected blocks as a
+                                     whole (above).  1: every protected block by itself, counting the request's own
+                                     live tokens in it: it leaves b when n_rb * detach_den < detach_num * S and stays
+                                     in the others.  2: every protected block by itself, counting the live tokens of
+                                     ALL holders (n_b): every holder leaves b when n_b * detach_den < detach_num * S */
 } vto_partial_opts;
 
 /* Relocation planning that evacuates only low-utilisation source blocks (Sec. 3.3.3): the planner
@@ -250,10 +252,16 @@ typedef struct {
  * listed in released_blocks (references dropped; the caller's reference counts decide when such a
  * block is free) instead of freed_blocks.  B bounds the unprotected sources only.  The gain gate
  * is unchanged: destinations < sources, counted in the request's own table.
- * With detach_per_block the same threshold is applied block by block: the request leaves exactly
+ * With detach_rule 1 the same threshold is applied block by block: the request leaves exactly
  * those protected blocks of its table in which its own live tokens fill less than the fraction
  * (n_rb * den < num * S; the other holders' tokens do not count), and keeps the others in place,
- * at the head of its new table with its other kept blocks. */
+ * at the head of its new table with its other kept blocks.
+ * With detach_rule 2 the block is judged by everything stored in it: n_b, the live tokens of all
+ * its holders (one count per referencing token-table entry).  Every holder reaches the same verdict
+ * on the same number, so a block is left by all the planned holders or by none: the copies its
+ * holders make (n_b tokens in all) cost less than the block they give back exactly when n_b < S,
+ * which is the threshold 1/1 -- the paper's condition "when the benefit justifies the copy" as a
+ * test the planner can make without knowing who else holds the block. */
 int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      const int32_t *bt_offsets, const int32_t *bt_blocks,
                      const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,

@@ -75,13 +75,14 @@ def to_csr(lists):
 
 
 def repack_partial_definition(S, block_tables, token_tables, keeps, free, select=None, thr=None, protect=(),
-                              util=None, max_sources=0, theta=None, detach=None, detach_per_block=False):
+                              util=None, max_sources=0, theta=None, detach=None, detach_rule=0):
     """Definition-level statement of the partial plan: only low-utilisation, unprotected blocks are
     evacuated.  protect: set of block ids; util / theta / detach: Fraction or None.  With ``detach`` a
     request whose own live tokens fill less than that fraction of its protected blocks leaves all of
     them (copy-on-write): they become sources too and are listed under ``released``.  With
-    ``detach_per_block`` the fraction is taken block by block: the request leaves exactly the protected
-    blocks in which its own live tokens fill less than ``detach`` of the S slots."""
+    ``detach_rule`` 1 the fraction is taken block by block: the request leaves exactly the protected
+    blocks in which its own live tokens fill less than ``detach`` of the S slots; with 2 the block is
+    judged by the live tokens of all requests stored in it."""
     R = len(token_tables)
     live = [[t for t, (s, k) in enumerate(zip(token_tables[r], keeps[r])) if s >= 0 and k] for r in range(R)]
     per_block = {}
@@ -104,9 +105,11 @@ def repack_partial_definition(S, block_tables, token_tables, keeps, free, select
                 picked.append(b)
         shared = [b for b in block_tables[r] if b in protect]
         mine_in_shared = sum(1 for t in live[r] if token_tables[r][t] // S in protect)
-        if detach is not None and detach_per_block:
+        if detach is not None and detach_rule == 1:
             mine_in = lambda b: sum(1 for t in live[r] if token_tables[r][t] // S == b)
             leaving.append({b for b in shared if Fraction(mine_in(b), S) < detach})
+        elif detach is not None and detach_rule == 2:
+            leaving.append({b for b in shared if Fraction(per_block.get(b, 0), S) < detach})
         else:
             goes = detach is not None and shared and Fraction(mine_in_shared, len(shared) * S) < detach
             leaving.append(set(shared) if goes else set())

@@ -138,7 +138,7 @@ def test_source_bound_B_takes_the_first_eligible_blocks_in_table_order():
     assert vto.plan_partial(S, 10, [0, 5], bt, [0, 20], tt, keep, free, max_source_blocks=1).req_status.tolist() == [vto.NO_GAIN]
 
 
-def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB, detach=None, per_block=False):
+def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB, detach=None, rule=0):
     bt_off, bt_flat = to_csr(bts)
     tt_off, tt_flat = to_csr(tts)
     _, keep_flat = to_csr(keeps)
@@ -149,9 +149,9 @@ def _compare(S, bts, tts, keeps, free, select, thr, protect, util, B, theta, NB,
                          select=None if select is None else np.array(select, np.uint8),
                          thr_num=fr(thr)[0], thr_den=fr(thr)[1], protect=prot if protect else None,
                          util=fr(util), max_source_blocks=B, theta=fr(theta), detach=fr(detach),
-                         detach_per_block=per_block)
+                         detach_rule=rule)
     d = repack_partial_definition(S, bts, tts, keeps, list(free), select, thr, set(protect), util, B, theta, detach,
-                                  per_block)
+                                  rule)
     assert p.released_blocks.tolist() == d["released"]
     nbo, nbf = to_csr(d["new_bt"])
     _, ntf = to_csr(d["new_tt"])
@@ -326,9 +326,9 @@ def test_per_block_detach_bruteforce_against_the_definition_twin():
                 for B in (0, 1):
                     for c in (0, 1, 3, 6):
                         free = np.array([9, 5, 10, 11, 12, 13][:c], np.int32)
-                        _compare(S, bts, tts, keeps, free, None, None, (0, 4, 1), util, B, None, NB, detach, True)
+                        _compare(S, bts, tts, keeps, free, None, None, (0, 4, 1), util, B, None, NB, detach, 1)
             d = repack_partial_definition(S, bts, tts, keeps, [9, 5, 10, 11, 12, 13], protect={0, 4, 1}, detach=detach,
-                                          detach_per_block=True)
+                                          detach_rule=1)
             for r in range(3):
                 shared = [b for b in bts[r] if b in (0, 4, 1)]
                 seen.add((len(shared), sum(b in d["new_bt"][r] for b in shared)))
@@ -352,7 +352,7 @@ def test_per_block_detach_by_hand():
     protect[[0, 1, 2]] = 1
     free = np.array([7, 8, 9], np.int32)
     run = lambda d, pb: vto.plan_partial(S, 12, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free, protect=protect,
-                                         util=(1, 1), detach=d, detach_per_block=pb)
+                                         util=(1, 1), detach=d, detach_rule=int(pb))
     whole = run((1, 2), False)
     assert whole.released_blocks.tolist() == [] and whole.req_status.tolist() == [vto.NO_GAIN, vto.NO_GAIN]
     half = run((1, 2), True)
@@ -383,7 +383,7 @@ def test_per_block_detach_meets_the_request_level_rule_where_the_two_must_agree(
     same = lambda p, q: all(np.array_equal(getattr(p, f), getattr(q, f)) for f in
                             ("new_bt_offsets", "new_bt_blocks", "new_tt_slots", "freed_blocks", "released_blocks",
                              "req_status", "move_src", "move_dst"))
-    assert same(run(protect=protect, detach=(5, 4)), run(protect=protect, detach=(5, 4), detach_per_block=True))
+    assert same(run(protect=protect, detach=(5, 4)), run(protect=protect, detach=(5, 4), detach_rule=1))
     assert len(run(protect=protect, detach=(5, 4)).released_blocks) > 0
     one = np.zeros_like(protect)                 # protect only the first block of every request's table
     one[w.bt_blocks[w.bt_offsets[:-1]]] = 1
@@ -393,9 +393,9 @@ def test_per_block_detach_meets_the_request_level_rule_where_the_two_must_agree(
         sel[r] = 1
         for d in ((1, 4), (1, 2), (3, 4), (1, 1)):
             assert same(run(protect=one, detach=d, select=sel), run(protect=one, detach=d, select=sel,
-                                                                    detach_per_block=True))
+                                                                    detach_rule=1))
     cons = run(protect=protect)
-    assert same(cons, run(protect=protect, detach=(0, 1), detach_per_block=True))
+    assert same(cons, run(protect=protect, detach=(0, 1), detach_rule=1))
     assert same(cons, run(protect=protect, detach=(0, 1)))
 
 
@@ -409,7 +409,7 @@ def test_per_block_detach_on_the_shared_prefix_workload(degree, detach):
                                   heads=1, head_dim=8, block_size=4)
     S = w.block_size
     p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
-                         protect=protect, detach=detach, detach_per_block=True)
+                         protect=protect, detach=detach, detach_rule=1)
     shared = set(np.flatnonzero(protect).tolist())
     live = (w.tt_slots >= 0) & (w.keep != 0)
     assert not (set(p.freed_blocks.tolist()) & shared) and not (set((p.move_dst // S).tolist()) & shared)
@@ -447,3 +447,107 @@ def test_per_block_detach_on_the_shared_prefix_workload(degree, detach):
     assert cursor == len(released)
     if detach == (1, 2):
         assert some_left and some_stayed            # the threshold really splits the prefix
+
+
+# ---- copy-on-write detach decided per shared block from the live tokens of all its holders ----------
+def test_all_holders_detach_bruteforce_against_the_definition_twin():
+    """The tables of the per-block brute force (three requests over three protected blocks, S = 3), rule 2:
+    a protected block is left by every planned holder when everything stored in it -- one count per
+    referencing token-table entry -- fills less than the threshold of a block."""
+    rng = np.random.default_rng(23)
+    S = 3
+    bts = [[0, 4, 1, 6], [0, 4, 1, 7, 3], [4, 8]]
+    tts = [[0, 1, 2, 12, 13, 14, 3, 4, 5, 18, 19, -1], [0, 1, 2, 12, 13, 14, 3, 4, 5, 21, 22, 23, 9, -1, 11],
+           [12, 13, 14, 24, 25]]
+    NB = 16
+    verdicts = set()
+    for _ in range(50):
+        keeps = [(rng.random(len(t)) < rng.choice([0.15, 0.4, 0.8])).astype(int).tolist() for t in tts]
+        for detach in (Fraction(1, 3), Fraction(2, 3), Fraction(1, 1), Fraction(4, 3), Fraction(7, 3)):
+            for util in (None, Fraction(1, 1)):
+                for B in (0, 1):
+                    for c in (0, 1, 3, 6):
+                        free = np.array([9, 5, 10, 11, 12, 13][:c], np.int32)
+                        _compare(S, bts, tts, keeps, free, None, None, (0, 4, 1), util, B, None, NB, detach, 2)
+            d = repack_partial_definition(S, bts, tts, keeps, [9, 5, 10, 11, 12, 13], protect={0, 4, 1}, detach=detach,
+                                          detach_rule=2)
+            # every admitted holder of a block reaches the same verdict on it
+            for b in (0, 4, 1):
+                held = [r for r in range(3) if b in bts[r] and d["status"][r] == 1]
+                gone = [r for r in held if b not in d["new_bt"][r]]
+                assert len(gone) in (0, len(held))
+                if held:
+                    verdicts.add(bool(gone))
+    assert verdicts == {True, False}
+
+
+def test_all_holders_detach_by_hand():
+    """S = 4, blocks 0 and 1 shared by two requests.  Block 0: request 0 keeps one token, request 1 keeps
+    two -> n_b = 3 < 4: both leave it at threshold 1/1.  Block 1: one + three -> n_b = 4: not below a block,
+    both stay -- although request 0 alone fills a quarter of it (rule 1 would let it go).  At 3/4 nobody
+    leaves block 0 either (3/4 is not below 3/4)."""
+    S = 4
+    bts = [[0, 1, 5], [0, 1, 6]]
+    tts = [list(range(8)) + [20, 21, 22, 23], list(range(8)) + [24, 25, 26, 27]]
+    keeps = [[1, 0, 0, 0,  0, 1, 0, 0,  1, 0, 0, 0], [0, 1, 1, 0,  1, 0, 1, 1,  0, 0, 1, 0]]
+    bt_off, bt_flat = to_csr(bts)
+    tt_off, tt_flat = to_csr(tts)
+    _, keep_flat = to_csr(keeps)
+    protect = np.zeros(12, np.uint8)
+    protect[[0, 1]] = 1
+    free = np.array([7, 8, 9, 10], np.int32)
+    run = lambda d, rule: vto.plan_partial(S, 12, bt_off, bt_flat, tt_off, tt_flat, keep_flat, free, protect=protect,
+                                           util=(1, 1), detach=d, detach_rule=rule)
+    p = run((1, 1), 2)
+    assert p.req_status.tolist() == [vto.REPACKED, vto.REPACKED]
+    assert p.released_blocks.tolist() == [0, 0] and p.freed_blocks.tolist() == [5, 6]
+    # request 0: tokens 0 (block 0) and 20 (block 5) move to block 7; it stays in block 1
+    assert p.new_bt_blocks.tolist() == [1, 7, 1, 8]
+    assert p.new_tt_slots[:12].tolist() == [28, -1, -1, -1, -1, 5, -1, -1, 29, -1, -1, -1]
+    assert p.new_tt_slots[12:].tolist() == [-1, 32, 33, -1, 4, -1, 6, 7, -1, -1, 34, -1]
+    assert list(zip(p.move_src.tolist(), p.move_dst.tolist())) == [(0, 28), (20, 29), (1, 32), (2, 33), (26, 34)]
+    own = run((1, 1), 1)                       # by its own tokens request 0 would leave block 1 as well
+    assert own.released_blocks.tolist()[:2] == [0, 1]
+    strict = run((3, 4), 2)
+    assert strict.released_blocks.tolist() == []
+
+
+@pytest.mark.parametrize("degree", [1, 2, 4, 8])
+def test_all_holders_detach_on_the_shared_prefix_workload(degree):
+    """Threshold 1/1 on the prefix-cache workload (H2O keeps about a fifth per request): what is left is
+    decided by bincount over all holders' live tokens; a block every holder left appears once per holder in
+    the released list and in no new table, shared bytes stay, every request sees its tokens.  With degree 1
+    the rule equals the per-block rule on own tokens."""
+    w, protect = wl.shared_prefix(seed=20 + degree, groups=2, degree=degree, prefix_len=64, suffix_len=96, layers=1,
+                                  heads=1, head_dim=8, block_size=4)
+    S = w.block_size
+    extra = 400                                     # room for every private copy
+    NB = w.num_blocks + extra
+    free = np.concatenate([w.free_blocks, np.arange(w.num_blocks, NB, dtype=np.int32)])
+    prot = np.concatenate([protect, np.zeros(extra, np.uint8)])
+    run = lambda rule: vto.plan_partial(S, NB, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, free,
+                                        protect=prot, detach=(1, 1), detach_rule=rule)
+    p = run(2)
+    live = (w.tt_slots >= 0) & (w.keep != 0)
+    n_b = np.bincount(w.tt_slots[live] // S, minlength=NB)
+    shared = np.flatnonzero(prot)
+    leaves = {int(b) for b in shared if n_b[b] < S}
+    assert p.num_admitted == w.num_requests
+    assert sorted(p.released_blocks.tolist()) == sorted(b for b in leaves for _ in range(degree))
+    assert not (set(p.new_bt_blocks.tolist()) & leaves)
+    for b in set(shared.tolist()) - leaves:
+        assert (p.new_bt_blocks == b).sum() == degree
+    slab = np.arange(NB * S * 2, dtype=np.int64).reshape(-1, 2)
+    before = slab.copy()
+    vto.apply_moves_slab(slab, p.move_src, p.move_dst)
+    rows = np.isin(np.arange(NB * S) // S, shared)
+    assert np.array_equal(slab[rows], before[rows])
+    for r in range(w.num_requests):
+        t0, t1 = w.tt_offsets[r], w.tt_offsets[r + 1]
+        assert np.array_equal(vto.gather_logical(before, w.tt_slots[t0:t1], w.keep[t0:t1]),
+                              vto.gather_logical(slab, p.new_tt_slots[t0:t1]))
+    if degree == 1:
+        q = run(1)
+        assert np.array_equal(p.new_tt_slots, q.new_tt_slots) and np.array_equal(p.released_blocks, q.released_blocks)
+    if degree == 8:
+        assert len(leaves) < len(shared)            # eight holders fill most prefix blocks beyond one block's worth

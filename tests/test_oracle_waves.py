@@ -241,21 +241,22 @@ def test_move_list_order_matters_when_blocks_are_reused():
 
 @pytest.mark.parametrize("degree", [1, 2, 4])
 @pytest.mark.parametrize("detach", [Fraction(1, 1), Fraction(1, 2), Fraction(1, 8)])
-@pytest.mark.parametrize("per_block", [False, True])
-def test_waves_with_copy_on_write_detach_against_a_replay(degree, detach, per_block):
+@pytest.mark.parametrize("rule", [0, 1, 2])
+def test_waves_with_copy_on_write_detach_against_a_replay(degree, detach, rule):
     """Repack in waves on the shared-prefix workload with a detach threshold: wave by wave the definition
     twin plans on what the previous wave committed; tables, pool, statuses and the list of dropped
     references (wave after wave, each reference once) must be the oracle's, one wave must equal the single
     partial plan, and every request must still see exactly its own payloads -- shared blocks keep their
-    bytes for the sharers that stayed.  Both forms of the rule: all protected blocks of a request at
-    once, and block by block (later waves then see a request that still holds part of its prefix)."""
+    bytes for the sharers that stayed.  All three forms of the rule: all protected blocks of a request at
+    once, block by block on its own tokens, block by block on all holders' tokens (later waves then see
+    requests that still hold part of their prefix)."""
     w, protect = wl.shared_prefix(seed=3, groups=2, degree=degree, prefix_len=48, suffix_len=150, layers=1, heads=1,
                                   head_dim=8, block_size=4)
     S, R = w.block_size, w.num_requests
     prot = set(np.flatnonzero(protect).tolist())
     opts = dict(protect=protect, util=(1, 1), max_source_blocks=6, detach=(detach.numerator, detach.denominator),
-                detach_per_block=per_block)
-    twin_kw = dict(protect=prot, util=Fraction(1, 1), max_sources=6, detach=detach, detach_per_block=per_block)
+                detach_rule=rule)
+    twin_kw = dict(protect=prot, util=Fraction(1, 1), max_sources=6, detach=detach, detach_rule=rule)
     one = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
                            w.free_blocks, **opts)
     v1 = vto.plan_waves(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks, 1,

@@ -983,7 +983,9 @@ def run_plan_only(args):
                       ("partial_detach_per_request", lambda st: prob.plan_partial(stream=st, protect=protect, detach=(1, 2),
                                                                                    **partial_opts)),
                       ("partial_detach_per_block", lambda st: prob.plan_partial(stream=st, protect=protect, detach=(1, 2),
-                                                                                 detach_per_block=True, **partial_opts))):
+                                                                                 detach_rule=1, **partial_opts)),
+                      ("partial_detach_all_holders", lambda st: prob.plan_partial(stream=st, protect=protect, detach=(1, 2),
+                                                                                   detach_rule=2, **partial_opts))):
         with torch.cuda.stream(side):
             fn(side)
         side.synchronize()

@@ -126,7 +126,7 @@ class DeviceProblem:
                        stream=stream)
 
     def plan_partial(self, stream=None, num_free=None, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
-                     detach=(0, 0), detach_per_block=False, ctx=None):
+                     detach=(0, 0), detach_rule=0, ctx=None):
         vt.vtoken_plan_partial(ctx or self.ctx, num_requests=self.num_requests, bt_offsets=self.bt_offsets,
                                bt_blocks=self.bt_blocks, tt_offsets=self.tt_offsets, tt_slots=self.tt_slots,
                                keep=self.keep, free_blocks=self.free_blocks,
@@ -136,7 +136,7 @@ class DeviceProblem:
                                req_status=self.req_status, counts=self.counts, select=self.select,
                                thr_num=self.w.thr_num, thr_den=self.w.thr_den, protect=protect, util=util,
                                max_source_blocks=max_source_blocks, theta=theta, detach=detach,
-                               detach_per_block=detach_per_block, released_blocks=self.released_blocks,
+                               detach_rule=detach_rule, released_blocks=self.released_blocks,
                                stream=stream)
 
     def repack(self, stream=None, ctx=None):

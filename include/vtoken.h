@@ -281,9 +281,12 @@ typedef struct {
     uint32_t detach_num, detach_den; /* copy-on-write detach: a request leaves ALL its protected blocks when its own
                                       live tokens in them fill less than detach_num / detach_den of those blocks
                                       (n_shared * den < num * ns_shared * S); detach_den == 0: never */
-    uint32_t detach_per_block;     /* non-zero: the threshold is applied to every protected block of the request by
-                                      itself -- it leaves block b when its own live tokens stored in b number n_rb
-                                      with n_rb * detach_den < detach_num * S, and stays in the others */
+    uint32_t detach_rule;          /* what the threshold is applied to.  0: the request's protected blocks as a whole
+                                      (above).  1: every protected block by itself, on the request's own live tokens
+                                      in it: it leaves b when n_rb * detach_den < detach_num * S and stays in the
+                                      others.  2: every protected block by itself, on the live tokens of ALL its
+                                      holders: every holder leaves b when n_b * detach_den < detach_num * S.
+                                      Other values: VTOKEN_EINVAL */
 } vtoken_partial_opts;
 
 /* vtoken_plan restricted to source blocks.  Differences from vtoken_plan: only live tokens stored
@@ -306,13 +309,19 @@ typedef struct {
  * other holders: enabling detach is the caller's policy decision.  vtoken_repack_waves and
  * vtoken_repack_host_partial take the threshold too; each has a released list of its own in its
  * output struct.
- * With detach_per_block the threshold is applied block by block instead: the request leaves exactly
+ * With detach_rule 1 the threshold is applied block by block instead: the request leaves exactly
  * those protected blocks of its table in which its own live tokens (not the other holders') fill
  * less than the fraction of the S slots, and keeps the others in place, in old order with its other
  * kept blocks.  The planner then takes a census of every request's live tokens per protected table
  * entry (one more kernel and a memset of 16 B per block-table entry in front of the plan; a lookup
  * per live token in a protected block).  A token stored in a protected block that its request's
- * table does not list stays where it is. */
+ * table does not list stays where it is.
+ * With detach_rule 2 a protected block is judged by everything stored in it, n_b = the live tokens
+ * of all its holders (one count per referencing token-table entry): every holder reaches the same
+ * verdict, so the block is left by all the holders this plan repacks or by none.  The copies made
+ * on leaving it (n_b tokens in all) take less room than the block they give back exactly when
+ * n_b < S -- threshold 1/1 -- which makes this the rule under which the POOL gains whenever all
+ * holders are repacked; it costs nothing beyond the plain partial plan (no census, no owners). */
 int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_partial_opts *opts,
                         const vtoken_plan_out *out, void *cuda_stream);
 

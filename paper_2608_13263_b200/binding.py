@@ -83,7 +83,7 @@ class PartialOpts(ctypes.Structure):
     _fields_ = [("protect", ctypes.c_void_p), ("util_num", ctypes.c_uint32), ("util_den", ctypes.c_uint32),
                 ("max_source_blocks", ctypes.c_int32), ("theta_num", ctypes.c_uint32), ("theta_den", ctypes.c_uint32),
                 ("detach_num", ctypes.c_uint32), ("detach_den", ctypes.c_uint32),
-                ("detach_per_block", ctypes.c_uint32)]
+                ("detach_rule", ctypes.c_uint32)]
 
 
 class WavesOut(ctypes.Structure):
@@ -301,7 +301,7 @@ def vtoken_repack_host(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, 
 def vtoken_repack_host_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks,
                                num_free, new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status,
                                select=None, thr_num=0, thr_den=0, protect=None, util=(0, 0), max_source_blocks=0,
-                               theta=(0, 0), detach=(0, 0), released_blocks=None, detach_per_block=False,
+                               theta=(0, 0), detach=(0, 0), released_blocks=None, detach_rule=0,
                                stream=None) -> dict:
     """vtoken_repack_host with the partial planner; ``protect`` is a HOST array of num_blocks bytes,
     ``released_blocks`` a HOST array of bt_offsets[R] entries (needed with a detach threshold)."""
@@ -311,7 +311,7 @@ def vtoken_repack_host_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_o
                    _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks), _ptr(req_status),
                    ctypes.addressof(c), _ptr(released_blocks))
     po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1], detach[0], detach[1],
-                     int(bool(detach_per_block)))
+                     int(detach_rule))
     _check(load().vtoken_repack_host_partial(ctx, ctypes.byref(h), ctypes.byref(po), _stream(stream)),
            "vtoken_repack_host_partial", ctx)
     return c.as_dict()
@@ -439,13 +439,13 @@ def vtoken_block_liveness(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offset
 def vtoken_plan_partial(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots, keep, free_blocks, num_free,
                         new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, req_status, counts, select=None,
                         thr_num=0, thr_den=0, protect=None, util=(0, 0), max_source_blocks=0, theta=(0, 0),
-                        detach=(0, 0), released_blocks=None, detach_per_block=False, stream=None) -> None:
+                        detach=(0, 0), released_blocks=None, detach_rule=0, stream=None) -> None:
     pin = PlanIn(_ptr(num_requests), _ptr(bt_offsets), _ptr(bt_blocks), _ptr(tt_offsets), _ptr(tt_slots), _ptr(keep),
                  _ptr(select), thr_num, thr_den, _ptr(free_blocks), _ptr(num_free))
     pout = PlanOut(_ptr(new_bt_offsets), _ptr(new_bt_blocks), _ptr(new_tt_slots), _ptr(freed_blocks),
                    _ptr(req_status), _ptr(counts), _ptr(released_blocks))
     po = PartialOpts(_ptr(protect), util[0], util[1], max_source_blocks, theta[0], theta[1], detach[0], detach[1],
-                     int(bool(detach_per_block)))
+                     int(detach_rule))
     _check(load().vtoken_plan_partial(ctx, ctypes.byref(pin), ctypes.byref(po), ctypes.byref(pout), _stream(stream)),
            "vtoken_plan_partial", ctx)
 
@@ -480,6 +480,6 @@ def vtoken_repack_waves(ctx, *, num_requests, bt_offsets, bt_blocks, tt_offsets,
         detach = partial.get("detach", (0, 0))
         po = ctypes.byref(PartialOpts(_ptr(partial.get("protect")), util[0], util[1],
                                       partial.get("max_source_blocks", 0), theta[0], theta[1], detach[0], detach[1],
-                                      int(bool(partial.get("detach_per_block", False)))))
+                                      int(partial.get("detach_rule", 0))))
     _check(load().vtoken_repack_waves(ctx, ctypes.byref(pin), po, num_waves, ctypes.byref(wout), _stream(stream)),
            "vtoken_repack_waves", ctx)

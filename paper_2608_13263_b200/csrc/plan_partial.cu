@@ -29,8 +29,13 @@
 // instead of reclaimed blocks.  "Source" is therefore a per-request notion for protected blocks
 // (req_detach[r]) and a per-block one (blk_src[b]) for the others.
 //
-// Detach decided per shared block (opts->detach_per_block): the request leaves exactly the protected
-// blocks that its own live tokens fill below the threshold.  That needs the census n_rb (live
+// Detach decided per shared block on all holders' tokens (opts->detach_rule 2): a protected block whose
+// n_b is below the threshold is left by every planned holder.  The blocks kernel marks it blk_src = 2
+// (every holder writes the same value), after which its tokens move like those of any other source and
+// the block-table writers list it under released instead of reclaimed; no owner of an entry is needed.
+//
+// Detach decided per shared block on the request's own tokens (opts->detach_rule 1): the request leaves
+// exactly the protected blocks that its own live tokens fill below the threshold.  That needs the census n_rb (live
 // tokens of request r stored in block b) for every protected entry of every block table, and every
 // token must find the count of its own (request, block) pair.  Each request owns the range
 // [2 * bt_offsets[r], 2 * bt_offsets[r + 1]) of one scratch array as a private open-addressing hash
@@ -53,7 +58,8 @@ struct PArgs {
     vtk_arr<const int32_t> num_requests, bt_offsets, bt_blocks, tt_offsets, tt_slots;
     vtk_arr<const uint8_t> keep, select, protect;
     uint32_t thr_num, thr_den, util_num, util_den, theta_num, theta_den, detach_num, detach_den;
-    uint32_t per_block;              // detach decided per protected block (the census in cow)
+    uint32_t rule;                   // detach rule: 0 per request, 1 per protected block on the request's own tokens (the
+                                     // census in cow), 2 per protected block on all holders' tokens (n_b; blk_src == 2)
     int32_t max_sources;
     vtk_arr<const int32_t> free_blocks, num_free;
     vtk_arr<int32_t> new_bt_offsets, new_bt_blocks, new_tt_slots, freed_blocks, released_blocks, out_status;
@@ -66,7 +72,7 @@ struct PArgs {
     vtk_arr<int32_t> tile_live, tile_mov, tile_shared, part_live, part_mov, part_shared;
     vtk_arr<int32_t> req_before;     // [max_requests + 1] moving tokens of the table before the request's first entry
     vtk_arr<int32_t> dst_src, dst_blocks, n_b;
-    vtk_arr<uint8_t> blk_src;
+    vtk_arr<uint8_t> blk_src;        // 1: source of its request; 2: protected block that every planned holder leaves
     vtk_arr<unsigned long long> cow; // [2 * max_table_blocks] per-request hashes: (block id + 1) << 32 | own live tokens
     vtk_arr<vtoken_counts> counts;
     int32_t S, num_blocks, max_requests, cap_dst_blocks, max_free_blocks;
@@ -168,7 +174,7 @@ __device__ __forceinline__ Owner pp_owner(const PArgs &a, int r)
     Owner o{false, CowTable{0, 0}};
     if (r < 0) return o;
     o.detach = a.req_detach[r] != 0;
-    if (o.detach && a.per_block) o.cow = pp_cow_table(a, r);
+    if (o.detach && a.rule == 1) o.cow = pp_cow_table(a, r);
     return o;
 }
 // does a live token of that request in block b move?  (b is a source of its request, or the request
@@ -177,7 +183,7 @@ __device__ __forceinline__ bool pp_moves(const PArgs &a, const Owner &o, int32_t
 {
     if (a.blk_src[b] != 0) return true;
     if (!o.detach || a.protect[b] == 0) return false;
-    return a.per_block ? pp_cow_leaves(a, o.cow, b) : true;
+    return a.rule == 1 ? pp_cow_leaves(a, o.cow, b) : true;
 }
 
 // Bits of the thread's live entries that move.  Without a detach threshold that is a property of the
@@ -217,7 +223,8 @@ __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
     const int R = pp_requests(a);
     const int64_t T = pp_offset(a, R);
     const int lane = vtk_lane(), warp = threadIdx.x >> 5;
-    const bool may_detach = !a.protect.null() && a.detach_den != 0;
+    // (rule 2 needs no owners: the blocks its holders leave are marked in blk_src like any other source)
+    const bool may_detach = !a.protect.null() && a.detach_den != 0 && a.rule != 2;
     // A CTA counts over the entries [base, limit): a whole tile, or (the CTAs behind the tiles, one per
     // request boundary) the entries between the start of the boundary's tile and the boundary.
     const bool is_tile = (int)blockIdx.x < a.num_tiles;
@@ -239,7 +246,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_tiles_kernel(PArgs a)
     const unsigned bits = vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, pp_offset(a, 0), limit, a.slots_per_layer, slot, bad);
     int n = 0, n_sh = 0;
     if (MODE == 0) {
-        const bool census = may_detach && a.per_block != 0 && is_tile;   // uniform over the CTA
+        const bool census = may_detach && a.rule == 1 && is_tile;        // uniform over the CTA
         int r = -1;
         int64_t next = 0;
         CowTable h{0, 0};
@@ -315,7 +322,7 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
     int carry = 0;               // eligible entries before this chunk
     int shared = 0;              // protected entries seen by this thread (per-block rule: those the request leaves)
     uint32_t flags = 0;
-    const bool per_block = !a.protect.null() && a.detach_den != 0 && a.per_block != 0;
+    const bool per_block = !a.protect.null() && a.detach_den != 0 && a.rule != 0;
     const CowTable h{2 * b0, 2 * (b1 - b0)};
     for (int64_t jb = b0; jb < b1; jb += PP_NT) {
         const int64_t j = jb + threadIdx.x;
@@ -328,7 +335,17 @@ __global__ void __launch_bounds__(PP_NT) pp_blocks_kernel(PArgs a)
                 blk = -1;
             } else {
                 eligible = !(!a.protect.null() && a.protect[blk] != 0);
-                if (!eligible) shared += per_block ? (pp_cow_leaves(a, h, blk) ? 1 : 0) : 1;
+                if (!eligible) {
+                    bool leaves = true;                    // rule 0: decided below for all protected entries at once
+                    if (a.rule == 1 && per_block) leaves = pp_cow_leaves(a, h, blk);
+                    if (a.rule == 2 && per_block) {
+                        // everything stored in the block, whoever holds it: every holder finds the same answer
+                        leaves = (unsigned long long)a.n_b[blk] * a.detach_den <
+                                 (unsigned long long)a.detach_num * (unsigned long long)a.S;
+                        if (leaves) a.blk_src[blk] = 2;
+                    }
+                    shared += leaves ? 1 : 0;
+                }
                 if (eligible && a.util_den != 0)
                     eligible = (unsigned long long)a.n_b[blk] * a.util_den <
                                (unsigned long long)a.util_num * (unsigned long long)a.S;
@@ -552,7 +569,8 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
     const int R = pp_requests(a);
     const int tid = threadIdx.x, lane = vtk_lane(), warp = tid >> 5;
     const int S = a.S;
-    const bool may_detach = !a.protect.null() && a.detach_den != 0;
+    const bool any_detach = !a.protect.null() && a.detach_den != 0;
+    const bool may_detach = any_detach && a.rule != 2;      // owners of entries are needed (see pp_tiles_kernel)
     uint32_t flags = 0;
 
     if ((int)blockIdx.x >= a.num_tiles) {
@@ -564,7 +582,7 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
         const int nb = (int)(b1 - b0);
         const int64_t cap_bt = a.max_table_blocks;               // every table write below stays inside its buffer
         const bool adm = a.req_status[r] == VTOKEN_REPACKED;
-        const bool detach = adm && may_detach && a.req_detach[r] != 0;
+        const bool detach = adm && any_detach && a.req_detach[r] != 0;
         const int nsrc = a.req_nsrc[r], ns = a.req_ns[r];
         const int need = (int)(((int64_t)nsrc + S - 1) / S);
         const int dst_base = a.req_dst_base[r];
@@ -591,8 +609,9 @@ __global__ void __launch_bounds__(TILE_NT) pp_assign_kernel(PArgs a)
                 if (j < b1) {
                     blk = a.bt_blocks[j];
                     if (blk >= 0 && blk < a.num_blocks) {
-                        src = a.blk_src[blk] != 0;
-                        rel = detach && a.protect[blk] != 0 && (a.per_block == 0 || pp_cow_leaves(a, h, blk));
+                        src = a.blk_src[blk] == 1;
+                        if (a.rule == 2) rel = detach && a.blk_src[blk] == 2;
+                        else rel = detach && a.protect[blk] != 0 && (a.rule == 0 || pp_cow_leaves(a, h, blk));
                     }
                 }
                 int total;
@@ -776,7 +795,7 @@ void fill_args(PArgs &a, vtoken_ctx *ctx)
     a.req_detach = VTK_ARR(ctx, ctx->req_detach, c.max_requests);
     a.req_rel_base = VTK_ARR(ctx, ctx->req_rel_base, c.max_requests);
     a.cow = VTK_ARR(ctx, ctx->cow, 2 * (int64_t)c.max_table_blocks);
-    a.per_block = 0;
+    a.rule = 0;
     a.counts = VTK_ARR(ctx, ctx->counts, 1);
     a.S = ctx->cfg.block_size;
     a.num_blocks = ctx->cfg.num_blocks;
@@ -804,7 +823,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     if (!out->new_bt_offsets || !out->new_bt_blocks || !out->new_tt_slots || !out->freed_blocks ||
         !out->req_status || !out->counts)
         return VTOKEN_EINVAL;
-    if (opts->max_source_blocks < 0) return VTOKEN_EINVAL;
+    if (opts->max_source_blocks < 0 || opts->detach_rule > 2) return VTOKEN_EINVAL;
     if (opts->protect != nullptr && opts->detach_den != 0 && !out->released_blocks) return VTOKEN_EINVAL;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     PArgs a{};
@@ -826,7 +845,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     a.theta_den = opts->theta_den;
     a.detach_num = opts->detach_num;
     a.detach_den = opts->detach_den;
-    a.per_block = (opts->protect != nullptr && opts->detach_den != 0 && opts->detach_per_block != 0) ? 1u : 0u;
+    a.rule = (opts->protect != nullptr && opts->detach_den != 0) ? opts->detach_rule : 0u;
     a.max_sources = opts->max_source_blocks;
     a.free_blocks = VTK_ARR(ctx, in->free_blocks, c.max_free_blocks);
     a.num_free = VTK_ARR(ctx, in->num_free, 1);
@@ -849,7 +868,7 @@ int vtoken_plan_partial(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->counts, 0, sizeof(vtoken_counts), st));
     // n_b and blk_src share one allocation: one node clears both
     VTK_CUDA(ctx, cudaMemsetAsync(ctx->n_b, 0, (sizeof(int32_t) + 1) * (size_t)ctx->cfg.num_blocks, st));
-    if (a.per_block) {
+    if (a.rule == 1) {
         VTK_CUDA(ctx, cudaMemsetAsync(ctx->cow, 0, sizeof(unsigned long long) * 2 * (size_t)c.max_table_blocks, st));
         VTK_CUDA(ctx, vtk_launch_dependent(ctx, pp_cow_insert_kernel, dim3(R), dim3(256), 0, st, a));
     }

@@ -111,9 +111,10 @@ def test_partial_planner_detach_and_waves(checked):
             tpp.test_partial_plans_small_whole_pool(w, opts)
     tpp.test_block_liveness_matches_oracle(small[2])
     # copy-on-write detach on the shared-prefix workload: released list, shared bytes untouched
-    tpp.test_copy_on_write_detach_on_the_shared_prefix_workload(4, (1, 2), False)
-    tpp.test_copy_on_write_detach_on_the_shared_prefix_workload(4, (1, 4), True)     # census hashes and their probes
-    tpp.test_detach_through_the_wave_entry_point_and_the_host_front_end(2, (1, 2), True)
+    tpp.test_copy_on_write_detach_on_the_shared_prefix_workload(4, (1, 2), 0)
+    tpp.test_copy_on_write_detach_on_the_shared_prefix_workload(4, (1, 4), 1)        # census hashes and their probes
+    tpp.test_copy_on_write_detach_on_the_shared_prefix_workload(2, (1, 1), 2)
+    tpp.test_detach_through_the_wave_entry_point_and_the_host_front_end(2, (1, 2), 1)
     tpp.test_shared_prefix_workload(2)
     # repack in waves, whole and partial: pool hand-over between the waves, commit kernel
     ws = tw.small_configs()

@@ -60,7 +60,7 @@ def test_fuzz_whole_and_partial_plans(seed):
             if rng.random() < 0.6:
                 opts["detach"] = [(1, 1), (1, 2), (3, 4)][int(rng.integers(0, 3))]
                 # (a generator of its own: the problems of the other seeds stay what they were)
-                opts["detach_per_block"] = bool(np.random.default_rng(5000 + seed).random() < 0.5)
+                opts["detach_rule"] = int(np.random.default_rng(5000 + seed).integers(0, 3))
     variant = int(rng.choice([0, 1, 2])) if w.row_bytes >= 16 else 1
     prob = DeviceProblem(w, fill_seed=seed, copy_variant=variant)
     from paper_2608_13263_b200 import binding as vt

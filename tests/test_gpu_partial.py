@@ -234,22 +234,22 @@ def test_repack_host_partial_entry_point(opts):
 
 @pytest.mark.parametrize("detach", [(1, 1), (1, 2), (1, 4), (1, 100)], ids=lambda d: f"detach{d[0]}_{d[1]}")
 @pytest.mark.parametrize("degree", [1, 2, 4, 8])
-@pytest.mark.parametrize("per_block", [False, True], ids=["per_request", "per_block"])
-def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach, per_block):
+@pytest.mark.parametrize("rule", [0, 1, 2], ids=["per_request", "per_block_own", "per_block_all"])
+def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach, rule):
     """Requests leave their shared prefix when their own tokens fill too little of it -- all of it at
-    once, or block by block: tables, the reclaimed and the released lists, counts and whole pools
-    against the oracle; the shared blocks keep their bytes."""
+    once, block by block, or block by block judged by all holders' tokens: tables, the reclaimed and the
+    released lists, counts and whole pools against the oracle; the shared blocks keep their bytes."""
     import torch
     from harness.device import DeviceProblem
     w, protect = wl.shared_prefix(seed=10 + degree, groups=2, degree=degree, prefix_len=256, suffix_len=320, layers=2,
                                   heads=2, head_dim=64)
     prob = DeviceProblem(w, fill_seed=FILL_SEED)
     prob.plan_partial(protect=torch.from_numpy(protect).to(prob.device), util=(1, 1), detach=detach,
-                      detach_per_block=per_block)
+                      detach_rule=rule)
     prob.repack()
     out = prob.outputs()
     p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
-                         w.free_blocks, protect=protect, util=(1, 1), detach=detach, detach_per_block=per_block)
+                         w.free_blocks, protect=protect, util=(1, 1), detach=detach, detach_rule=rule)
     assert out["error_flags"] == 0
     for n in ("num_moves", "num_dst_blocks", "num_freed", "num_free_consumed", "num_admitted", "num_deferred"):
         assert out[n] == getattr(p, n), n
@@ -260,11 +260,16 @@ def test_copy_on_write_detach_on_the_shared_prefix_workload(degree, detach, per_
     assert np.array_equal(out["new_bt_blocks"], p.new_bt_blocks)
     assert np.array_equal(out["new_tt_slots"], p.new_tt_slots)
     assert np.array_equal(out["freed_blocks"], p.freed_blocks)
-    if detach == (1, 1) and not per_block:
+    if detach == (1, 1) and rule == 0:
         assert out["num_released"] == degree * 2 * w.notes["prefix_blocks"]       # every sharer left every prefix block
-    if detach == (1, 100) and not per_block:
+    if detach == (1, 100) and rule == 0:
         assert out["num_released"] == 0                                           # nobody is that sparse
-    if per_block and detach == (1, 4):
+    if rule == 2 and p.num_admitted == w.num_requests:
+        # judged by all holders' tokens: a shared block stays in every sharer's table or in none
+        shared = np.flatnonzero(protect)
+        held = np.bincount(p.new_bt_blocks[np.isin(p.new_bt_blocks, shared)], minlength=w.num_blocks)[shared]
+        assert set(held.tolist()) <= {0, degree}
+    if rule == 1 and detach == (1, 4):
         # the block rule really splits prefixes here: some request keeps part of its shared blocks
         kept_shared = np.isin(p.new_bt_blocks, np.flatnonzero(protect)).sum()
         assert 0 < out["num_released"] and kept_shared > 0
@@ -309,8 +314,8 @@ def test_detach_needs_a_released_list_everywhere():
 
 @pytest.mark.parametrize("degree", [2, 4])
 @pytest.mark.parametrize("detach", [(1, 1), (1, 2)], ids=lambda d: f"detach{d[0]}_{d[1]}")
-@pytest.mark.parametrize("per_block", [False, True], ids=["per_request", "per_block"])
-def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, detach, per_block):
+@pytest.mark.parametrize("rule", [0, 1, 2], ids=["per_request", "per_block_own", "per_block_all"])
+def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, detach, rule):
     """Copy-on-write detach through vtoken_repack_waves (references dropped wave after wave, in one list)
     and through vtoken_repack_host_partial (host tables in and out): tables, lists and every byte of both
     pools against the oracle."""
@@ -318,7 +323,7 @@ def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, deta
     from harness.device import DeviceProblem, origin_map
     w, protect = wl.shared_prefix(seed=7, groups=2, degree=degree, prefix_len=256, suffix_len=600, layers=2, heads=1,
                                   head_dim=64)
-    opts = dict(util=(1, 1), max_source_blocks=12, detach=detach, detach_per_block=per_block)
+    opts = dict(util=(1, 1), max_source_blocks=12, detach=detach, detach_rule=rule)
     # ---- waves with a short pool: the detaches are spread over several waves
     need = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep,
                             w.free_blocks, protect=protect, **opts).num_dst_blocks
@@ -375,7 +380,7 @@ def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, deta
 @pytest.mark.parametrize("seed", range(16))
 def test_fuzz_detach_on_random_shared_prefix_shapes(seed):
     """Random prefix-cache shapes (block size, sharing degree, prefix and suffix lengths, kept
-    fraction), thresholds, source bounds and pool cuts, both forms of the detach rule, some requests
+    fraction), thresholds, source bounds and pool cuts, the three detach rules, some requests
     deselected: tables, lists, counts and every byte of both pools against the oracle."""
     import torch
     from harness.device import DeviceProblem, origin_map
@@ -391,7 +396,7 @@ def test_fuzz_detach_on_random_shared_prefix_shapes(seed):
     opts = dict(util=[(0, 0), (1, 1), (1, 2)][int(rng.integers(0, 3))],
                 max_source_blocks=int(rng.choice([0, 0, 2, 9])),
                 detach=[(1, 1), (1, 2), (1, 4), (3, 4), (5, 4), (1, 16)][int(rng.integers(0, 6))],
-                detach_per_block=bool(seed % 4 != 3))
+                detach_rule=(1, 2, 1, 0, 2, 2)[seed % 6])
     num_free = None if rng.random() < 0.5 else int(rng.integers(0, len(w.free_blocks) + 1))
     p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
                          w.select, w.thr_num, w.thr_den, num_free=num_free, protect=protect, **opts)

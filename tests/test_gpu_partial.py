@@ -413,3 +413,65 @@ def test_fuzz_detach_on_random_shared_prefix_shapes(seed):
         assert np.array_equal(out[n], getattr(p, n)), n
     assert prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst)) == 0
     prob.close()
+
+
+@pytest.mark.parametrize("degree", [1, 2, 4])
+def test_caller_side_of_copy_on_write_with_reference_counts(degree):
+    """The whole protocol around a copy-on-write plan, as a caller with reference counts runs it: plan with
+    the all-holders rule at 1/1, repack, adopt the new tables, drop one reference per entry of the released
+    list, hand the blocks whose count reached zero back to the free list together with the reclaimed ones.
+    Then the library's own precondition checker must accept the new state (no block free and held, unique
+    mapping outside the blocks still shared), the relocation digest of every request must be what it was,
+    and the pool must have gained exactly the blocks the tables lost."""
+    import torch
+    from harness.device import DeviceProblem
+    from test_gpu_fuzz import _digest
+    w, protect = wl.shared_prefix(seed=40 + degree, groups=3, degree=degree, prefix_len=256, suffix_len=300, layers=2,
+                                  heads=2, head_dim=64)
+    S, R = w.block_size, w.num_requests
+    # room for every private copy: the generator sizes the pool for the conservative plan
+    extra = 600
+    w.num_blocks += extra
+    w.free_blocks = np.concatenate([w.free_blocks, np.arange(w.num_blocks - extra, w.num_blocks, dtype=np.int32)])
+    protect = np.concatenate([protect, np.zeros(extra, np.uint8)])
+    refcount = np.bincount(w.bt_blocks, minlength=w.num_blocks)              # holders per block, as the caller tracks them
+    assert set(refcount[protect != 0].tolist()) == {degree}
+    prob = DeviceProblem(w, fill_seed=FILL_SEED)
+    prot = torch.from_numpy(protect).to(prob.device)
+    before = _digest(prob, vt, prob.tt_slots, prob.keep)
+    prob.plan_partial(protect=prot, util=(1, 1), detach=(1, 1), detach_rule=2)
+    prob.repack()
+    out = prob.outputs()
+    p = vto.plan_partial(S, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots, w.keep, w.free_blocks,
+                         protect=protect, util=(1, 1), detach=(1, 1), detach_rule=2)
+    assert out["error_flags"] == 0 and out["num_admitted"] == R == p.num_admitted
+    assert np.array_equal(out["released_blocks"], p.released_blocks) and out["num_released"] > 0
+    # ---- the caller's bookkeeping
+    refcount -= np.bincount(out["released_blocks"], minlength=w.num_blocks)
+    assert (refcount >= 0).all()
+    unshared = np.flatnonzero((protect != 0) & (refcount == 0))              # every holder left: free again
+    still_shared = (protect != 0) & (refcount > 0)
+    if degree > 1:
+        assert set(refcount[still_shared].tolist()) <= {degree}              # left by all holders or by none
+    new_free = np.concatenate([w.free_blocks[out["num_free_consumed"]:], out["freed_blocks"], unshared]).astype(np.int32)
+    new_bt, new_off = out["new_bt_blocks"], out["new_bt_offsets"]
+    blocks_before, blocks_after = len(set(w.bt_blocks.tolist())), len(set(new_bt.tolist()))
+    assert len(new_free) - len(w.free_blocks) == blocks_before - blocks_after > 0
+    # ---- the new state through the library's checker and the relocation digest
+    i32 = dict(dtype=torch.int32, device=prob.device)
+    d_bt = torch.zeros(prob.max_table_blocks, **i32)
+    d_bt[:len(new_bt)] = torch.from_numpy(new_bt)
+    free_cap = torch.zeros(max(len(new_free), 1), **i32)
+    free_cap[:len(new_free)] = torch.from_numpy(new_free)
+    ctx2 = vt.vtoken_create(w.num_layers, w.num_blocks, S, w.num_kv_heads, w.head_dim, prob.k_pool, prob.v_pool,
+                            prob.max_requests, prob.max_tokens, prob.max_table_blocks, max(len(new_free), 1))
+    bits = torch.full((1,), -1, **i32)
+    vt.vtoken_check_tables(ctx2, num_requests=prob.num_requests, bt_offsets=torch.from_numpy(new_off).to(prob.device),
+                           bt_blocks=d_bt, tt_offsets=prob.tt_offsets, tt_slots=prob.new_tt_slots, free_blocks=free_cap,
+                           num_free=torch.tensor([len(new_free)], **i32), out_bits=bits,
+                           protect=torch.from_numpy(still_shared.astype(np.uint8)).to(prob.device))
+    torch.cuda.synchronize()
+    assert int(bits.item()) == 0
+    vt.vtoken_destroy(ctx2)
+    assert np.array_equal(before, _digest(prob, vt, prob.new_tt_slots, None))
+    prob.close()

@@ -1016,6 +1016,88 @@ def run_plan_only(args):
 
 
 
+def run_prefix_cache(args):
+    """The paper's prefix-cache compatibility experiment (Sec. 5, Table 1) in synthetic form, at its
+    shape: Llama-3.1-8B-shaped pools, `--groups` prompts each shared by 1 / 2 / 4 / 8 requests, an 8K-token
+    shared prefix and an 8K-token private suffix per request, an H2O-style mask that keeps a fifth.
+    Per sharing degree: the conservative plan (shared blocks stay, private suffixes are repacked) and the
+    copy-on-write plan that judges a shared block by all its holders' live tokens (threshold 1/1), each as
+    one captured graph of plan + copy on the side stream, checked against the oracle (tables in full,
+    every word of both pools through the oracle's move list), then timed.  One JSON line."""
+    import torch
+    from harness import workloads as wl
+    from harness.device import DeviceProblem, origin_map
+    sys.path.insert(0, ROOT)
+    from oracle import vto
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(dev)
+    side = torch.cuda.Stream(device=dev)
+    rows = []
+    for degree in (1, 2, 4, 8):
+        R = args.groups * degree
+        w, protect = wl.shared_prefix(seed=args.seed, groups=args.groups, degree=degree, prefix_len=8192,
+                                      suffix_len=8192, extra_free=R * 8192 // 16 // 4)
+        free_b, total_b = torch.cuda.mem_get_info(dev)
+        need = 2 * w.num_layers * w.slots_per_layer * w.row_bytes
+        if need > free_b - (6 << 30):
+            rows.append({"degree": degree, "skipped": f"pools of {need / 2 ** 30:.1f} GiB do not fit the free memory"})
+            continue
+        prob = DeviceProblem(w, device=dev)
+        prot = torch.from_numpy(protect).to(dev)
+        blocks_before = len(set(w.bt_blocks.tolist()))
+        entry = {"degree": degree, "requests": R, "logical_tokens": int(w.num_tokens),
+                 "blocks_allocated": blocks_before, "shared_blocks": int(protect.sum()),
+                 "pool_GiB": need / 2 ** 30, "plans": {}}
+        for label, opts in (("conservative", dict(util=(1, 1))),
+                            ("copy_on_write_all_holders", dict(util=(1, 1), detach=(1, 1), detach_rule=2))):
+            with torch.cuda.stream(side):
+                prob.plan_partial(protect=prot, stream=side, **opts)
+                prob.repack(stream=side)
+            side.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                prob.plan_partial(protect=prot, stream=torch.cuda.current_stream(), **opts)
+                prob.repack(stream=torch.cuda.current_stream())
+            prob.fill_pools()
+            torch.cuda.synchronize(dev)
+            with torch.cuda.stream(side):
+                g.replay()
+            side.synchronize()
+            out = prob.outputs()
+            parity = "skipped"
+            if not args.no_verify:
+                p = vto.plan_partial(w.block_size, w.num_blocks, w.bt_offsets, w.bt_blocks, w.tt_offsets, w.tt_slots,
+                                     w.keep, w.free_blocks, protect=protect, **opts)
+                ok = (out["error_flags"] == 0 and all(np.array_equal(out[k], getattr(p, k)) for k in
+                      ("new_bt_offsets", "new_bt_blocks", "new_tt_slots", "freed_blocks", "released_blocks", "req_status")))
+                bad = prob.verify_pools(origin_map(w.slots_per_layer, p.move_src, p.move_dst))
+                parity = "ok" if ok and bad == 0 else f"FAILED (tables_ok={ok}, mismatching_words={bad})"
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.cuda.stream(side):
+                for _ in range(args.warmup):
+                    g.replay()
+                e0.record(side)
+                for _ in range(args.steps):
+                    g.replay()
+                e1.record(side)
+            side.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            moved = out["num_moves"]
+            after = len(set(out["new_bt_blocks"].tolist()))
+            entry["plans"][label] = {
+                "blocks_retained": after, "retained_block_reduction": 1 - after / blocks_before,
+                "tokens_moved": moved, "references_released": out["num_released"],
+                "requests_repacked": out["num_admitted"], "ms_plan_and_copy": ms,
+                "GBs": 2 * moved * w.token_bytes / (ms * 1e-3) / 1e9 if ms > 0 else 0.0, "parity": parity}
+        rows.append(entry)
+        prob.close()
+        del prob
+        torch.cuda.empty_cache()
+    print(json.dumps({"mode": "prefix-cache", "shape": "L=32, H=8, D=128, S=16; 8192 shared + 8192 private tokens per request, H2O-style mask keeping 20 %",
+                      "groups": args.groups, "steps": args.steps, "warmup": args.warmup, "degrees": rows,
+                      "gpu": torch.cuda.get_device_name(dev)}))
+
+
 # ----------------------------------------------------------------------------------------------
 # N > 1 without a launcher: this process starts one rank per GPU itself
 # ----------------------------------------------------------------------------------------------
@@ -1084,6 +1166,9 @@ def main():
     ap.add_argument("--variant", type=int, default=0, help="copy path: 0 auto, 1 registers, 2 bulk copy")
     ap.add_argument("--max-ctas", type=int, default=0)
     ap.add_argument("--scale-requests", type=float, default=1.0)
+    ap.add_argument("--prefix-cache", action="store_true",
+                    help="the prefix-cache experiment in synthetic form: sharing degrees 1-8, conservative and copy-on-write plans")
+    ap.add_argument("--groups", type=int, default=4, help="--prefix-cache: number of shared prompts")
     ap.add_argument("--oracle-layers", type=int, default=0,
                     help="layers in the CPU-baseline sample (0: 8, or 4 when a slab exceeds 1 GiB)")
     ap.add_argument("--no-proxy", action="store_true", help="skip the run beside the decode-read proxy")
@@ -1114,6 +1199,8 @@ def main():
         run_reference(args)
     elif args.plan_only:
         run_plan_only(args)
+    elif args.prefix_cache:
+        run_prefix_cache(args)
     else:
         run_cuda(args)
 

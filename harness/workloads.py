@@ -358,13 +358,15 @@ def streaming_window(seed: int = 0, requests: int = 64, lo: int = 1024, hi: int 
 
 def shared_prefix(seed: int = 0, groups: int = 4, degree: int = 4, prefix_len: int = 8192, suffix_len: int = 8192,
                   layers: int = 32, heads: int = 8, head_dim: int = 128, block_size: int = 16,
-                  budget_frac: float = 0.2):
+                  budget_frac: float = 0.2, extra_free: int = 0):
     """Prefix-cache workload shaped like the paper's compatibility experiment (Sec. 5, Table 1):
     ``groups`` prompts, each shared by ``degree`` requests that reference the SAME physical
     blocks for the first ``prefix_len`` tokens and own a private suffix of ``suffix_len`` tokens;
     H2O-style mask per request over prefix + suffix.  ``prefix_len`` must be a multiple of the
     block size so that shared and private blocks do not mix.  Returns (workload, protect) where
-    protect[b] = 1 marks the shared blocks, which a plan must leave in place."""
+    protect[b] = 1 marks the shared blocks, which a plan must leave in place.  The free list holds
+    the destinations of the private suffixes plus 256 blocks; ``extra_free`` adds room for plans that
+    copy tokens out of shared blocks as well."""
     S = block_size
     assert prefix_len % S == 0
     rng = np.random.Generator(np.random.PCG64(seed))
@@ -378,7 +380,7 @@ def shared_prefix(seed: int = 0, groups: int = 4, degree: int = 4, prefix_len: i
     suf_blocks = -(-suffix_len // S)
     private_live = [int(k[prefix_len:].sum()) for k in keeps]
     dst_total = sum(-(-x // S) for x in private_live)
-    NB = groups * pre_blocks + R * suf_blocks + dst_total + 256
+    NB = groups * pre_blocks + R * suf_blocks + dst_total + 256 + extra_free
     perm = rng.permutation(NB).astype(np.int32)
     shared = [perm[g * pre_blocks:(g + 1) * pre_blocks] for g in range(groups)]
     cursor = groups * pre_blocks

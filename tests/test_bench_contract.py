@@ -63,3 +63,24 @@ def test_cuda_arm_prints_the_agreed_line_on_the_tiny_configuration():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
     assert {"sm_mhz", "sm_max_mhz", "reasons"} <= set(d["clocks"])
     assert "decode_step_policy_adapter" in d["runtime"]
+
+
+@pytest.mark.gpu
+def test_prefix_cache_mode_is_checked_against_the_oracle_for_every_degree():
+    """`bench.py --prefix-cache` with one prompt group: four sharing degrees, two plans each, every run
+    compared with the oracle inside the benchmark; the copy-on-write plan never retains more blocks than
+    the conservative one."""
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--prefix-cache", "--groups", "1",
+                          "--steps", "3", "--warmup", "3"], cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["mode"] == "prefix-cache" and [e["degree"] for e in d["degrees"]] == [1, 2, 4, 8]
+    for e in d["degrees"]:
+        if "skipped" in e:
+            continue
+        cons, cow = e["plans"]["conservative"], e["plans"]["copy_on_write_all_holders"]
+        assert cons["parity"] == "ok" and cow["parity"] == "ok"
+        assert cons["references_released"] == 0 and cow["blocks_retained"] <= cons["blocks_retained"]
+        assert cons["requests_repacked"] == e["requests"]

@@ -50,8 +50,9 @@ def form(request, monkeypatch):
 
 def test_small_configs_and_shapes(form):
     import test_gpu_parity as tp
-    for w in tp.small_configs():
-        tp.run_and_compare(w, copy_variant=2)
+    for i, w in enumerate(tp.small_configs()):
+        # (the planner form does not reach the copy kernel: tables and lists in full, both pools for one workload)
+        tp.run_and_compare(w, copy_variant=2, whole_pool=(i == 1))
     for S, heads, head_dim in ((1, 1, 8), (3, 2, 64), (48, 8, 128), (5, 3, 8)):
         w = wl.mistral7b_random(seed=S, requests=5, lo=10, hi=40 * S + 20, layers=2, heads=heads, head_dim=head_dim,
                                 block_size=S)

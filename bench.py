@@ -324,7 +324,7 @@ def measure(args, ranks, dev, side, name, block_size, main):
     w, scale = fit_workload(args, name, seed, block_size, asked, dev)
     steps, warmup = args.steps, args.warmup
     prob = DeviceProblem(w, device=dev, fill_seed=1, copy_variant=args.variant, max_ctas=args.max_ctas,
-                         wave_capacity=main and args.waves > 0, **{})
+                         wave_capacity=main and args.waves > 0)
     partial_opts = dict(util=(1, 1), theta=(1, 4))     # fully live blocks stay; the paper's default trigger F > 0.25
     partial = main and args.plan_mode == "partial"
 

@@ -189,9 +189,9 @@ int vto_apply_moves(int32_t R, int32_t S, const int32_t *tt_offsets, int32_t *tt
 
 /* ---- cached slot-translation arrays (Sec. 3.2, last paragraph; Sec. 4) -------------------------
  * The worker keeps, per request, the slots of its active tokens in token-id order -- the array a
- * decode step translates through -- and refreshes it only after structural changes: "when a
- * sequence grows append-only, the cache is updated by appending the new entries; a full rebuild is
- * triggered only on structural changes (eviction, relocation ...)".
+ * decode step translates through -- and refreshes it only after structural changes: growth of a
+ * sequence at its end is taken in by appending the new entries, and only an eviction or a
+ * relocation of the request makes the array be rebuilt.
  * Layout: the cache of request r lives in cache_slots / cache_ids [tt_offsets[r] ..) (same capacity
  * as its token table); cache_len[r] entries are valid and cover the first cache_seen[r] registered
  * tokens.
@@ -260,8 +260,9 @@ typedef struct {
  * its holders (one count per referencing token-table entry).  Every holder reaches the same verdict
  * on the same number, so a block is left by all the planned holders or by none: the copies its
  * holders make (n_b tokens in all) cost less than the block they give back exactly when n_b < S,
- * which is the threshold 1/1 -- the paper's condition "when the benefit justifies the copy" as a
- * test the planner can make without knowing who else holds the block. */
+ * which is the threshold 1/1 -- the paper's condition for copy-on-write (the reclaimed capacity
+ * must outweigh the extra copy) as a test the planner can make without knowing who else holds
+ * the block. */
 int vto_plan_partial(int32_t R, int32_t S, int32_t NB,
                      const int32_t *bt_offsets, const int32_t *bt_blocks,
                      const int32_t *tt_offsets, const int32_t *tt_slots, const uint8_t *keep,

@@ -1,6 +1,8 @@
 """GPU parity of the eligibility metadata (per-block liveness, histogram, F) and of partial
 plans (low-utilisation sources, protected blocks, source bound, global trigger) against the
 oracle: tables, lists, counts and whole pools, bit-exact."""
+import os
+
 import numpy as np
 import pytest
 
@@ -377,7 +379,7 @@ def test_detach_through_the_wave_entry_point_and_the_host_front_end(degree, deta
     prob.close()
 
 
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", range(16 * max(1, int(os.environ.get("VTOKEN_FUZZ_SCALE", "1")))))
 def test_fuzz_detach_on_random_shared_prefix_shapes(seed):
     """Random prefix-cache shapes (block size, sharing degree, prefix and suffix lengths, kept
     fraction), thresholds, source bounds and pool cuts, the three detach rules, some requests

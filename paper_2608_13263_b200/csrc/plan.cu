@@ -64,59 +64,87 @@ __device__ __forceinline__ void raise_flags(const PlanArgs &a, uint32_t flags)
     atomicOr(&a.out_counts->error_flags, flags);
 }
 
-__device__ __forceinline__ unsigned load_entries(const PlanArgs &a, int64_t t, int64_t T, int32_t (&slot)[TILE_TOK],
-                                                 bool &bad)
-{
-    return vtk_load_entries(a.tt_slots, a.keep, a.vec_in, t, clipped_offset(a, 0), T, a.slots_per_layer, slot, bad);
-}
-
 // ---- tiles -----------------------------------------------------------------------------
+constexpr int TILES_PER_CTA = 4;                 // tiles a counting CTA takes: the loads of all of them are in flight
+                                                 // together, and the grid of a 2 M-entry table is one wave
+
+__host__ __device__ __forceinline__ int tile_ctas(int num_tiles) { return (num_tiles + TILES_PER_CTA - 1) / TILES_PER_CTA; }
+
 __global__ void __launch_bounds__(TILE_NT) plan_tiles_kernel(PlanArgs a)
 {
-    __shared__ int warp_n[TILE_NT / 32];
+    __shared__ int warp_n[TILES_PER_CTA][TILE_NT / 32];
+    __shared__ unsigned int bad_tiles;
     vtk_release_successor();
     vtk_wait_for_predecessor();
     const int R = clamp_requests(a);
     const int64_t T = clipped_offset(a, R);
+    const int64_t first = clipped_offset(a, 0);
     const int lane = vtk_lane(), warp = threadIdx.x >> 5;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         a.header[0] = R;
         a.header[1] = (int32_t)T;
         a.header[2] = *a.num_free;
-        a.header[3] = (int32_t)clipped_offset(a, 0);
+        a.header[3] = (int32_t)first;
     }
-    // A CTA counts the live entries of [base, limit): a whole tile, or -- the CTAs behind the tiles, one
-    // per request boundary -- the entries between the start of the boundary's tile and the boundary
-    // (entries the tile's own CTA counts as well; flags are raised there).  Either way one pass.
-    const bool is_tile = (int)blockIdx.x < a.num_tiles;
-    const int r = (int)blockIdx.x - a.num_tiles;
-    int64_t base, limit;
-    if (is_tile) {
-        base = (int64_t)blockIdx.x * TILE;
-        limit = T;
-        if (base >= T) return;
-    } else {
-        if (r > R) return;
-        limit = clipped_offset(a, r);
-        base = limit / TILE * TILE;
-        if (base == limit) return;                       // nothing in front of it: the scan does not read req_part[r]
+    if (threadIdx.x == 0) bad_tiles = 0u;
+    const int n_tile_ctas = tile_ctas(a.num_tiles);
+    if ((int)blockIdx.x < n_tile_ctas) {
+        // TILES_PER_CTA consecutive tiles, every entry of the table exactly once
+        const int tile0 = (int)blockIdx.x * TILES_PER_CTA;
+        if ((int64_t)tile0 * TILE >= T) return;
+        int n[TILES_PER_CTA];
+        unsigned bad_bits = 0;
+#pragma unroll
+        for (int k = 0; k < TILES_PER_CTA; ++k) {
+            const int64_t base = (int64_t)(tile0 + k) * TILE;
+            int32_t slot[TILE_TOK];
+            bool bad = false;
+            n[k] = base < T ? __popc(vtk_load_entries(a.tt_slots, a.keep, a.vec_in, base + threadIdx.x * TILE_TOK, first, T,
+                                                      a.slots_per_layer, slot, bad))
+                            : 0;
+            if (bad) bad_bits |= 1u << k;
+        }
+#pragma unroll
+        for (int k = 0; k < TILES_PER_CTA; ++k) {
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) n[k] += __shfl_down_sync(0xffffffffu, n[k], d);
+            if (lane == 0) warp_n[k][warp] = n[k];
+        }
+        __syncthreads();                                  // (bad_tiles is zero by now)
+        if (bad_bits) atomicOr(&bad_tiles, bad_bits);
+        __syncthreads();
+        if (threadIdx.x < TILES_PER_CTA && (int64_t)(tile0 + threadIdx.x) * TILE < T) {
+            const int k = threadIdx.x;
+            int s = 0;
+#pragma unroll
+            for (int w = 0; w < TILE_NT / 32; ++w) s += warp_n[k][w];
+            // a slot outside the pool somewhere in the tile travels in the sign bit (the count is at most
+            // 1024): the scan kernel turns it into VTOKEN_FLAG_BAD_SLOT, and nothing has to be zeroed
+            // before this kernel
+            a.tile_n[tile0 + k] = s | (((bad_tiles >> k) & 1u) ? (int)0x80000000 : 0);
+        }
+        return;
     }
+    // the CTAs behind those, one per request boundary: the live entries between the start of the boundary's
+    // tile and the boundary (entries the tile's own CTA counts as well; flags are raised there)
+    const int r = (int)blockIdx.x - n_tile_ctas;
+    if (r > R) return;
+    const int64_t limit = clipped_offset(a, r);
+    const int64_t base = limit / TILE * TILE;
+    if (base == limit) return;                           // nothing in front of it: the scan does not read req_part[r]
     bool bad = false;
     int32_t slot[TILE_TOK];
-    int n = __popc(load_entries(a, base + threadIdx.x * TILE_TOK, limit, slot, bad));
+    int n = __popc(vtk_load_entries(a.tt_slots, a.keep, a.vec_in, base + threadIdx.x * TILE_TOK, first, limit,
+                                    a.slots_per_layer, slot, bad));
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) n += __shfl_down_sync(0xffffffffu, n, d);
-    if (lane == 0) warp_n[warp] = n;
-    const int any_bad = __syncthreads_or(bad);
+    if (lane == 0) warp_n[0][warp] = n;
+    __syncthreads();
     if (threadIdx.x == 0) {
         int s = 0;
 #pragma unroll
-        for (int w = 0; w < TILE_NT / 32; ++w) s += warp_n[w];
-        // a slot outside the pool somewhere in the tile travels in the sign bit (the count is at most
-        // 1024): the scan kernel turns it into VTOKEN_FLAG_BAD_SLOT, and nothing has to be zeroed
-        // before this kernel
-        if (is_tile) a.tile_n[blockIdx.x] = s | (any_bad ? (int)0x80000000 : 0);
-        else a.req_part[r] = s;
+        for (int w = 0; w < TILE_NT / 32; ++w) s += warp_n[0][w];
+        a.req_part[r] = s;
     }
 }
 
@@ -464,7 +492,7 @@ int vtk_launch_plan(vtoken_ctx *ctx, const vtoken_plan_in *in, const vtoken_plan
 #endif
 
     const int R = ctx->cfg.max_requests;
-    VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_tiles_kernel, dim3(a.num_tiles + R + 1), dim3(TILE_NT), 0, st, a));
+    VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_tiles_kernel, dim3(tile_ctas(a.num_tiles) + R + 1), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_scan_kernel, dim3(1), dim3(SCAN_NT), 0, st, a));
     VTK_CUDA(ctx, vtk_launch_dependent(ctx, plan_assign_kernel, dim3(a.num_tiles + R), dim3(TILE_NT), 0, st, a));
     VTK_CUDA(ctx, cudaGetLastError());
